@@ -1,0 +1,227 @@
+/*
+ * recg.h -- C ABI of the fused draft+verify step for diffusion-AR self-speculation on one B200.
+ *
+ * One round of shared-backbone self-speculation (paper Sec. 3.1) runs ONE forward over a ragged,
+ * padding-free batch (Sec. 5.3).  Request r contributes
+ *     v_r pending verify tokens y_0..y_{v-1} at positions L_r .. L_r+v_r-1   (causal rows), and
+ *     b_r mask tokens at positions L_r+v_r .. L_r+v_r+b_r-1                  (bidirectional rows),
+ * over its L_r committed context tokens, whose K/V live in a paged pool.  Visibility is Eq. 1's
+ * M^Diff with the prefix set = context + verify tokens and the draft set = the mask block; restricted
+ * to the verify rows this is M^AR, so the same forward verifies the previous drafts and drafts the
+ * next block (Sec. 5.1, continuation branch).  The round ends with greedy verification (accept the
+ * drafted prefix up to the first mismatch, Sec. 3.1), the confidence statistics that guide the
+ * runtime (P_1st, P_1st - P_2nd: Sec. 4.1; mean verifier entropy over valid rows: Sec. 5.2) and the
+ * KV commit / rollback, which is index work only.
+ *
+ * General rules
+ *   - every entry point returns a recg_status and never aborts; recg_last_error() gives the text;
+ *   - all device work is enqueued on the CUDA stream given to recg_init(); nothing synchronises
+ *     the stream unless stated;
+ *   - "DEVICE" / "HOST" on a pointer says where the memory lives.  bf16 is the 16-bit brain float
+ *     bit pattern; ids, lengths and slots are int32;
+ *   - weights and the KV pool are BORROWED: the caller allocates them, keeps them alive while the
+ *     context lives and frees them; the library allocates only its own workspace, in recg_init();
+ *   - there is no CPU fallback: without a CUDA device every call fails with RECG_ERR_CUDA.
+ */
+#ifndef RECG_H_
+#define RECG_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  RECG_OK = 0,
+  RECG_ERR_INVALID_ARG = 1, /* null pointer, negative length, unknown enum                     */
+  RECG_ERR_SHAPE = 2,       /* model dimensions the kernels do not support                     */
+  RECG_ERR_CAPACITY = 3,    /* more requests / tokens / pages than the context was sized for   */
+  RECG_ERR_CUDA = 4,        /* a CUDA runtime or driver call failed                            */
+  RECG_ERR_TIMEOUT = 5,     /* a bounded device-side wait gave up (status word set by kernel)  */
+  RECG_ERR_INTERNAL = 6
+} recg_status;
+
+typedef enum { RECG_DTYPE_BF16 = 0, RECG_DTYPE_F32 = 1 } recg_dtype;
+typedef enum { RECG_MEM_DEVICE = 0, RECG_MEM_HOST = 1 } recg_mem;
+
+enum {
+  RECG_FLAG_LOGITS_BF16 = 1, /* recg_step() stores logits as bf16 instead of fp32               */
+  RECG_FLAG_SIMT_GEMM = 2    /* run the projections on the legacy mma.sync kernel (A/B checks)  */
+};
+
+typedef struct recg_ctx recg_ctx;
+
+/* Model and capacity description; immutable after recg_init(). */
+typedef struct {
+  int32_t n_layers, hidden, n_q_heads, n_kv_heads, head_dim, ffn, vocab;
+  float rope_base;        /* rotary base; pairing is (i, i + head_dim/2)                         */
+  float rms_eps;
+  int32_t mask_token_id;  /* id fed to the mask rows; < 0 means vocab - 1                        */
+  int32_t page_size;      /* tokens per KV page; must be 16                                      */
+  int32_t max_requests;   /* capacity: requests per step                                         */
+  int32_t max_tokens;     /* capacity: sum of v_r + b_r per step                                 */
+  int32_t max_pages_per_request;
+  int32_t flags;          /* RECG_FLAG_*                                                         */
+} recg_config;
+
+/*
+ * Weights, DEVICE, bf16, every matrix row-major [out_features, in_features]:
+ *   embed [vocab, hidden]; final_norm [hidden]; lm_head [vocab, hidden];
+ *   per layer l (the arrays of pointers themselves are HOST arrays of n_layers DEVICE pointers):
+ *   attn_norm[l] [hidden]; wqkv[l] [(n_q + 2 n_kv) * head_dim, hidden] (q heads, k heads, v heads);
+ *   wo[l] [hidden, n_q * head_dim]; ffn_norm[l] [hidden];
+ *   w_gate_up[l] [2 * ffn, hidden] (gate rows then up rows); w_down[l] [hidden, ffn].
+ * All base addresses must be 16-byte aligned.
+ */
+typedef struct {
+  const void *embed, *final_norm, *lm_head;
+  const void *const *attn_norm;
+  const void *const *wqkv;
+  const void *const *wo;
+  const void *const *ffn_norm;
+  const void *const *w_gate_up;
+  const void *const *w_down;
+} recg_weights;
+
+/*
+ * One round's batch descriptor.  The small arrays are HOST memory and are copied by the call.
+ *   ctx_len[r]     L_r, committed context tokens whose K/V are already in the pool
+ *   verify_len[r]  v_r >= 0, pending verify tokens (y_0 known-correct, y_1.. drafts)
+ *   block_size[r]  b_r >= 0, mask tokens;  v_r + b_r >= 1
+ *   verify_tokens  the y of all requests, concatenated in request order (sum of v_r ids)
+ *   page_table     [n_req, page_table_stride] physical page ids; row r must cover
+ *                  ceil((L_r + v_r + b_r) / page_size) pages, else RECG_ERR_CAPACITY
+ *   kv_pool        DEVICE, recg_kv_pool_bytes(cfg, kv_pool_pages) bytes, library-defined layout
+ *                  (per layer, per page, per KV head: a K tile then a V tile of 16 tokens, stored in
+ *                  the swizzled order the attention kernel loads; use recg_kv_write / recg_kv_read
+ *                  to move logical K/V in and out).  May be NULL for a verify-only call.
+ */
+typedef struct {
+  int32_t n_req;
+  const int32_t *ctx_len;
+  const int32_t *verify_len;
+  const int32_t *block_size;
+  const int32_t *verify_tokens;
+  const int32_t *page_table;
+  int32_t page_table_stride;
+  void *kv_pool;
+  int64_t kv_pool_pages;
+} recg_batch;
+
+/* Logits of the last recg_step(): DEVICE, library-owned, valid until the next recg_step(). */
+typedef struct {
+  const void *data;  /* [n_rows, vocab], row t = t-th token of the ragged batch */
+  int32_t dtype;     /* recg_dtype */
+  int32_t n_rows;
+  int32_t vocab;
+} recg_logits;
+
+/*
+ * Outputs of greedy verification.  All buffers are caller-provided and live where `mem` says
+ * (every pointer in one struct in the same place); any pointer may be NULL to skip that output.
+ * With RECG_MEM_HOST the call copies the results out and synchronises the stream before returning.
+ * T = sum(v_r + b_r), Tv = sum(v_r), Tb = sum(b_r).
+ *   accept_len[n_req]    a_r: drafts y_1..y_a accepted (longest prefix equal to the verifier argmax)
+ *   n_emitted[n_req]     a_r + 1 (0 if v_r = 0)
+ *   emitted[Tv]          per request, at its verify offset: y_1..y_a then the verifier's token at row a
+ *                        (correction if a < v-1, bonus if a = v-1); entries beyond n_emitted are -1
+ *   new_ctx_len[n_req]   L_r + a_r + 1: K/V of y_0..y_a are now committed
+ *   slot_state[T]        per token of the batch: +slot (page*page_size + offset) if its K/V is committed,
+ *                        -(slot+1) if it is rolled back (rejected draft or mask row)
+ *   freed_pages[n_req]   number of pages of request r that hold no committed token any more
+ *                        (its page-table entries from ceil(new_ctx_len/page_size) on)
+ *   next_draft[Tb]       argmax of every mask row: the next round's drafts
+ *   cont_hit[n_req]      1 if the block was fully accepted and the first drafted token equals the
+ *                        bonus token (the continuation branch can be reused), else 0
+ *   top1, top2 [T]       ids of the largest and second-largest logit per row (lowest index wins ties)
+ *   p1, p2, entropy [T]  float32: softmax probability of top1 and top2, entropy in nats
+ *   entropy_mean[n_req]  float32: mean verifier entropy over rows 0..a_r
+ */
+typedef struct {
+  int32_t mem; /* recg_mem */
+  int32_t *accept_len, *n_emitted, *emitted, *new_ctx_len, *slot_state, *freed_pages;
+  int32_t *next_draft, *cont_hit, *top1, *top2;
+  float *p1, *p2, *entropy, *entropy_mean;
+} recg_verify_out;
+
+/* Bytes of KV pool needed for n_pages physical pages (all layers). */
+size_t recg_kv_pool_bytes(const recg_config *cfg, int64_t n_pages);
+
+/*
+ * Create a context: validates cfg, allocates the workspace (activations for max_tokens rows, logits,
+ * attention partials, descriptors) and records the weight pointers.  `weights` may be NULL for a
+ * context that only runs the standalone operations (recg_verify with explicit logits,
+ * recg_attention, recg_linear, recg_kv_*); recg_step() then fails with RECG_ERR_INVALID_ARG.
+ * cuda_stream is a cudaStream_t (NULL = the default stream).  Uses the current CUDA device.
+ */
+recg_status recg_init(recg_ctx **out, const recg_config *cfg, const recg_weights *weights, void *cuda_stream);
+
+/*
+ * One fused draft+verify forward (ragged layout, embedding, n_layers x {RMSNorm, QKV projection with
+ * rotary embedding and KV append, hybrid-mask paged attention (Eq. 1), output projection + residual,
+ * RMSNorm, gate|up projection + SwiGLU, down projection + residual}, final norm, LM head).
+ * K/V of all v_r + b_r new positions are written into the pool slots the page table names
+ * (tentatively: recg_verify decides which stay).  `logits` (may be NULL) receives the view of the
+ * logits.  Does not synchronise.
+ */
+recg_status recg_step(recg_ctx *ctx, const recg_batch *batch, recg_logits *logits);
+
+/*
+ * Greedy verification, statistics and KV commit / rollback (Sec. 3.1, 4.1, 5.1, 5.2) for `batch`.
+ * logits == NULL: use the logits of the last recg_step() (same batch).  Otherwise `logits` is a
+ * DEVICE array [T, vocab] of `logits_dtype`; batch->kv_pool may then be NULL and page_table may be
+ * NULL (slot_state and freed_pages are then not produced).
+ */
+recg_status recg_verify(recg_ctx *ctx, const recg_batch *batch, const void *logits, int32_t logits_dtype,
+                        recg_verify_out *out);
+
+/*
+ * The hybrid-mask paged attention of one layer as a standalone operation (Eq. 1 over a shared prefix).
+ * q, o: DEVICE bf16 [T, n_q_heads, head_dim] (q already rotated).  K/V of ALL L_r + v_r + b_r
+ * positions of every request must already be in layer `layer` of the pool.
+ */
+recg_status recg_attention(recg_ctx *ctx, const recg_batch *batch, int32_t layer, const void *q, void *o);
+
+/*
+ * Move logical K/V rows of one request into / out of the pool.  k, v: DEVICE bf16
+ * [n_pos, n_kv_heads, head_dim] for positions pos0 .. pos0+n_pos-1; page_table_row: HOST, the
+ * request's page ids covering those positions.
+ */
+recg_status recg_kv_write(recg_ctx *ctx, void *kv_pool, int64_t kv_pool_pages, int32_t layer,
+                          const int32_t *page_table_row, int32_t n_table, int32_t pos0, int32_t n_pos,
+                          const void *k, const void *v);
+recg_status recg_kv_read(recg_ctx *ctx, const void *kv_pool, int64_t kv_pool_pages, int32_t layer,
+                         const int32_t *page_table_row, int32_t n_table, int32_t pos0, int32_t n_pos,
+                         void *k, void *v);
+
+/*
+ * y[M, N] = x[M, K] . w[N, K]^T, the projection kernel without an epilogue (for checking it alone).
+ * x, w: DEVICE bf16, 16-byte aligned, K a multiple of 64 and N a multiple of 16; y: DEVICE, out_dtype.
+ */
+recg_status recg_linear(recg_ctx *ctx, const void *x, const void *w, void *y, int32_t M, int32_t N, int32_t K,
+                        int32_t out_dtype);
+
+/*
+ * Read back an internal activation of the last recg_step() for parity checks.  which: 0 = residual
+ * stream after the last layer, fp32 [T, hidden]; 1 = attention output of the last layer, bf16
+ * [T, n_q*head_dim]; 2 = rotated queries of the last layer, bf16 [T, n_q*head_dim].
+ * Returns DEVICE pointers into the workspace.
+ */
+recg_status recg_debug_buffer(recg_ctx *ctx, int32_t which, const void **ptr, int32_t *dtype, int32_t *rows,
+                              int32_t *cols);
+
+/* Wait for the stream, then report (and clear) the device status word: RECG_OK or RECG_ERR_TIMEOUT /
+ * RECG_ERR_INTERNAL if a kernel flagged a bounded wait that gave up or an out-of-range index. */
+recg_status recg_sync(recg_ctx *ctx);
+
+recg_status recg_free(recg_ctx *ctx);
+
+/* Text of the last error on this context (or of the last failed recg_init if ctx is NULL). */
+const char *recg_last_error(const recg_ctx *ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RECG_H_ */

@@ -1,0 +1,118 @@
+// Internal launcher interface between the C ABI (recg_api.cu) and the kernel files.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace recg {
+
+struct Dims {
+  int n_layers, hidden, n_q, n_kv, head_dim, ffn, vocab;
+  float rope_base, rms_eps;
+  int mask_id;
+};
+
+// One attention work item: rows of one (request, kv head, row tile) against a range of 64-token KV blocks.
+struct AttnItem {
+  int req, kv_head;
+  int tok0, ntok;        // first token of the tile (index into the ragged batch) and tokens in it
+  int blk_begin, blk_end;
+  int part;              // index into the partial buffers, or -1 when the item covers the whole KV range
+  int kv_len;            // L + n of the request
+};
+struct AttnTile {        // per (request, kv head, row tile): where its partials are
+  int part_begin, n_parts;
+};
+
+// Device-resident ragged layout of one batch (all pointers DEVICE, int32 unless noted).
+struct BatchLayout {
+  int n_req, n_tok, n_ver, pt_stride;
+  const int* ctx_len;     // [C]
+  const int* verify_len;  // [C]
+  const int* block_size;  // [C]
+  const int* cu_tok;      // [C+1] exclusive prefix sum of v+b
+  const int* cu_ver;      // [C+1] exclusive prefix sum of v
+  const int* verify_tokens;  // [Tv]
+  const int* page_table;  // [C, pt_stride] (may be null for verify-only batches)
+  // per token, written by the layout kernel
+  int* tok_id;
+  int* tok_req;
+  int* tok_pos;
+  int* tok_slot;    // page*16 + offset, -1 without a page table
+  int* tok_climit;  // sees every position <= climit ...
+  int* tok_lo;      // ... and every position in [lo, hi)
+  int* tok_hi;
+  // attention work list
+  AttnItem* items;
+  AttnTile* tiles;
+  int* tile_off;    // [C+1] first tile entry of each request
+  int* counts;      // [0] number of items, [1] number of tiles, [2] chunk (blocks per item)
+  int max_items, max_parts;
+};
+
+// S1: per-token arrays and the attention work list.
+void launch_layout(const BatchLayout& bl, const Dims& dm, int tok_per_tile, int target_items, int64_t n_pages,
+                   int* status, cudaStream_t st);
+// S2: h[t] = embed[tok_id[t]] (fp32 residual stream).
+void launch_embed(const BatchLayout& bl, const Dims& dm, const void* embed, float* h, cudaStream_t st);
+// x = rmsnorm(h) * g, bf16 out.
+void launch_rmsnorm(const float* h, const void* gain, void* x, int rows, int hidden, float eps, cudaStream_t st);
+
+// (cos, sin) of pos * base^(-2i/d), angles evaluated in double: cs float2 [T][head_dim/2].
+void launch_rope_table(const int* tok_pos, int n_tok, int head_dim, float rope_base, void* cs, cudaStream_t st);
+
+// Projection epilogues.
+enum Epilogue : int {
+  EPI_PLAIN_BF16 = 0,  // C bf16 [M,N]
+  EPI_PLAIN_F32 = 1,   // C fp32 [M,N]
+  EPI_RESIDUAL = 2,    // h fp32 [M,N] += acc
+  EPI_SWIGLU = 3,      // w is [2F,K]; out bf16 [M,F] = silu(x.wg) * (x.wu)
+  EPI_QKV_ROPE = 4     // rotate q and k heads, q -> bf16 [M, n_q*d], k/v -> paged pool at tok_slot
+};
+struct GemmArgs {
+  const void* x;   // bf16 [M,K]
+  const void* w;   // bf16 [N,K]  (EPI_SWIGLU: [2N,K], gate rows then up rows)
+  void* out;       // see Epilogue
+  int M, N, K;
+  int epi;
+  // EPI_QKV_ROPE only
+  const int* tok_pos;
+  const int* tok_slot;
+  void* kv_pool;
+  int64_t n_pages;
+  int layer, n_q, n_kv, head_dim;
+  const void* rope_cs;  // float2 [M][head_dim/2]: (cos, sin) of each token's rotary angles
+};
+// legacy tensor path (mma.sync), any M; N multiple of 64 (EPI_SWIGLU: F multiple of 32), K multiple of 32
+void launch_gemm_simt(const GemmArgs& a, int* status, cudaStream_t st);
+// tcgen05 + TMA path; returns false if the shape is not supported by it
+struct TcGemmPlan;  // opaque: cached tensor maps
+bool launch_gemm_tc(const GemmArgs& a, void* tc_state, int* status, cudaStream_t st);
+void* tc_state_create(int n_sm);
+void tc_state_destroy(void* s);
+
+// S5
+void launch_attention(const BatchLayout& bl, const Dims& dm, int layer, const void* q, void* o, const void* kv_pool,
+                      int64_t n_pages, float* part_o, float* part_ml, int tok_per_tile, int n_sm, int* status,
+                      cudaStream_t st);
+size_t attention_smem_bytes(int head_dim);
+
+// S9b + S10
+struct VerifyBuffers {   // DEVICE outputs (library workspace or caller buffers), any may be null
+  int *accept_len, *n_emitted, *emitted, *new_ctx_len, *slot_state, *freed_pages, *next_draft, *cont_hit, *top1,
+      *top2;
+  float *p1, *p2, *entropy, *entropy_mean;
+};
+struct RowPartial {      // per (row, vocab chunk)
+  float m1, m2;          // largest and second-largest logit of the chunk
+  int i1, i2;
+  float s, t;            // sum exp(x - m1), sum (x - m1) exp(x - m1)
+};
+void launch_verify(const BatchLayout& bl, const void* logits, int logits_dtype, int vocab, RowPartial* partials,
+                   int max_chunks_total, const VerifyBuffers& vb, int n_sm, cudaStream_t st);
+int verify_chunks_per_row(int rows, int vocab, int n_sm);
+
+// KV import / export
+void launch_kv_io(bool write, void* pool, int64_t n_pages, int layer, const Dims& dm, const int* page_row_dev, int pos0,
+                  int n_pos, void* k, void* v, int* status, cudaStream_t st);
+
+}  // namespace recg

@@ -1,0 +1,245 @@
+// Ragged layout (per-token arrays + attention work list), embedding gather, RMSNorm, KV import/export.
+#include "common.cuh"
+#include "kernels.h"
+
+namespace recg {
+
+namespace {
+
+__device__ __forceinline__ int upper_request(const int* cu, int n_req, int t) {
+  // largest r with cu[r] <= t  (cu is an exclusive prefix sum with cu[n_req] = total)
+  int lo = 0, hi = n_req;
+  while (hi - lo > 1) {
+    int mid = (lo + hi) >> 1;
+    if (cu[mid] <= t) lo = mid; else hi = mid;
+  }
+  return lo;
+}
+
+// One CTA.  Shared: 3 prefix arrays of n_req+1 ints (items, tiles, split parts).
+__global__ void __launch_bounds__(1024) layout_kernel(BatchLayout bl, int n_kv, int mask_id, int tok_per_tile,
+                                                      int target_items, int64_t n_pages, int* status) {
+  extern __shared__ int sm[];
+  const int C = bl.n_req;
+  int* item_off = sm;
+  int* tile_off = sm + (C + 1);
+  int* part_off = sm + 2 * (C + 1);
+  __shared__ unsigned long long s_work;
+  __shared__ int s_chunk;
+  const int tid = threadIdx.x, nth = blockDim.x;
+
+  // ---- per-token arrays ----
+  for (int t = tid; t < bl.n_tok; t += nth) {
+    const int r = upper_request(bl.cu_tok, C, t);
+    const int j = t - bl.cu_tok[r];
+    const int L = bl.ctx_len[r], v = bl.verify_len[r], b = bl.block_size[r];
+    const int pos = L + j;
+    const bool is_ver = j < v;
+    bl.tok_req[t] = r;
+    bl.tok_pos[t] = pos;
+    bl.tok_id[t] = is_ver ? bl.verify_tokens[bl.cu_ver[r] + j] : mask_id;
+    bl.tok_climit[t] = is_ver ? pos : L + v - 1;
+    bl.tok_lo[t] = is_ver ? 0 : L + v;
+    bl.tok_hi[t] = is_ver ? 0 : L + v + b;
+    int slot = -1;
+    if (bl.page_table) {
+      const int page = bl.page_table[(size_t)r * bl.pt_stride + pos / kPageSize];
+      if (page < 0 || page >= n_pages) set_status(status, DEV_BAD_INDEX);
+      else slot = page * kPageSize + pos % kPageSize;
+    }
+    bl.tok_slot[t] = slot;
+  }
+
+  // ---- attention work list ----
+  if (tid == 0) s_work = 0ull;
+  __syncthreads();
+  unsigned long long w = 0;
+  for (int r = tid; r < C; r += nth) {
+    const int n = bl.verify_len[r] + bl.block_size[r];
+    const int nb = (bl.ctx_len[r] + n + 63) / 64;
+    const int tiles = (n + tok_per_tile - 1) / tok_per_tile;
+    w += (unsigned long long)n_kv * tiles * nb;
+  }
+  if (w) atomicAdd(&s_work, w);
+  __syncthreads();
+  if (tid == 0) {
+    unsigned long long c = (s_work + target_items - 1) / target_items;
+    s_chunk = c < 1 ? 1 : (c > (1 << 20) ? (1 << 20) : (int)c);
+  }
+  __syncthreads();
+  const int chunk = s_chunk;
+  for (int r = tid; r < C; r += nth) {
+    const int n = bl.verify_len[r] + bl.block_size[r];
+    const int nb = (bl.ctx_len[r] + n + 63) / 64;
+    const int tiles = (n + tok_per_tile - 1) / tok_per_tile;
+    const int parts = (nb + chunk - 1) / chunk;
+    item_off[r + 1] = n_kv * tiles * parts;
+    tile_off[r + 1] = n_kv * tiles;
+    part_off[r + 1] = parts > 1 ? n_kv * tiles * parts : 0;
+  }
+  __syncthreads();
+  if (tid == 0) {
+    item_off[0] = tile_off[0] = part_off[0] = 0;
+    for (int r = 0; r < C; ++r) {
+      item_off[r + 1] += item_off[r];
+      tile_off[r + 1] += tile_off[r];
+      part_off[r + 1] += part_off[r];
+    }
+    int n_items = item_off[C];
+    if (n_items > bl.max_items || part_off[C] > bl.max_parts) {
+      set_status(status, DEV_BAD_INDEX);
+      n_items = 0;
+    }
+    bl.counts[0] = n_items;
+    bl.counts[1] = tile_off[C];
+    bl.counts[2] = chunk;
+  }
+  __syncthreads();
+  for (int r = tid; r <= C; r += nth) bl.tile_off[r] = tile_off[r];
+  const int n_items = bl.counts[0];
+  for (int it = tid; it < n_items; it += nth) {
+    const int r = upper_request(item_off, C, it);
+    const int local = it - item_off[r];
+    const int n = bl.verify_len[r] + bl.block_size[r];
+    const int kv_len = bl.ctx_len[r] + n;
+    const int nb = (kv_len + 63) / 64;
+    const int tiles = (n + tok_per_tile - 1) / tok_per_tile;
+    const int parts = (nb + chunk - 1) / chunk;
+    const int part = local % parts;
+    const int tile = (local / parts) % tiles;
+    const int kvh = local / (parts * tiles);
+    AttnItem a;
+    a.req = r;
+    a.kv_head = kvh;
+    a.tok0 = bl.cu_tok[r] + tile * tok_per_tile;
+    a.ntok = min(tok_per_tile, n - tile * tok_per_tile);
+    a.blk_begin = part * chunk;
+    a.blk_end = min(nb, (part + 1) * chunk);
+    a.part = parts > 1 ? part_off[r] + (kvh * tiles + tile) * parts + part : -1;
+    a.kv_len = kv_len;
+    bl.items[it] = a;
+    if (part == 0) {
+      AttnTile tl;
+      tl.part_begin = parts > 1 ? a.part : -1;
+      tl.n_parts = parts;
+      bl.tiles[tile_off[r] + kvh * tiles + tile] = tl;
+    }
+  }
+}
+
+__global__ void embed_kernel(const int* __restrict__ tok_id, const __nv_bfloat16* __restrict__ embed,
+                             float* __restrict__ h, int hidden, int vocab) {
+  const int t = blockIdx.x;
+  int id = tok_id[t];
+  id = id < 0 ? 0 : (id >= vocab ? vocab - 1 : id);
+  const __nv_bfloat162* src = reinterpret_cast<const __nv_bfloat162*>(embed + (size_t)id * hidden);
+  float2* dst = reinterpret_cast<float2*>(h + (size_t)t * hidden);
+  for (int i = threadIdx.x; i < hidden / 2; i += blockDim.x) dst[i] = __bfloat1622float2(src[i]);
+}
+
+// One CTA per row; fp32 in, bf16 out.  hidden a multiple of 4.
+__global__ void __launch_bounds__(256) rmsnorm_kernel(const float* __restrict__ h, const __nv_bfloat16* __restrict__ g,
+                                                      __nv_bfloat16* __restrict__ x, int hidden, float eps) {
+  const int row = blockIdx.x;
+  const float4* src = reinterpret_cast<const float4*>(h + (size_t)row * hidden);
+  float ss = 0.f;
+  for (int i = threadIdx.x; i < hidden / 4; i += blockDim.x) {
+    float4 v = src[i];
+    ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+  }
+  __shared__ float red[8];
+  for (int o = 16; o; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+  __syncthreads();
+  float tot = 0.f;
+  for (int i = 0; i < (blockDim.x >> 5); ++i) tot += red[i];
+  const float rstd = rsqrtf(tot / hidden + eps);
+  uint2* dst = reinterpret_cast<uint2*>(x + (size_t)row * hidden);
+  const uint2* gg = reinterpret_cast<const uint2*>(g);
+  for (int i = threadIdx.x; i < hidden / 4; i += blockDim.x) {
+    float4 v = src[i];
+    uint2 gv = gg[i];
+    float2 g0 = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162*>(&gv.x));
+    float2 g1 = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162*>(&gv.y));
+    uint2 o;
+    o.x = pack_bf16(v.x * rstd * g0.x, v.y * rstd * g0.y);
+    o.y = pack_bf16(v.z * rstd * g1.x, v.w * rstd * g1.y);
+    dst[i] = o;
+  }
+}
+
+// grid (n_pos, n_kv), head_dim/8 threads: each moves one 16-byte chunk of K and of V.
+__global__ void kv_io_kernel(bool write, __nv_bfloat16* pool, int64_t n_pages, int layer, int n_kv, int head_dim,
+                             const int* __restrict__ page_row, int pos0, __nv_bfloat16* k, __nv_bfloat16* v,
+                             int* status) {
+  const int p = pos0 + blockIdx.x, hk = blockIdx.y, c = threadIdx.x;
+  const int page = page_row[p / kPageSize];
+  if (page < 0 || page >= n_pages) {
+    set_status(status, DEV_BAD_INDEX);
+    return;
+  }
+  const size_t base = kv_tile_base(n_pages, n_kv, head_dim, layer, page, hk);
+  const int off = kv_tile_offset(p % kPageSize, c * 8);
+  uint4* pk = reinterpret_cast<uint4*>(pool + base + off);
+  uint4* pv = reinterpret_cast<uint4*>(pool + base + kv_tile_elems(head_dim) + off);
+  const size_t lin = ((size_t)blockIdx.x * n_kv + hk) * head_dim + c * 8;
+  uint4* lk = reinterpret_cast<uint4*>(k + lin);
+  uint4* lv = reinterpret_cast<uint4*>(v + lin);
+  if (write) {
+    *pk = *lk;
+    *pv = *lv;
+  } else {
+    *lk = *pk;
+    *lv = *pv;
+  }
+}
+
+}  // namespace
+
+void launch_layout(const BatchLayout& bl, const Dims& dm, int tok_per_tile, int target_items, int64_t n_pages,
+                   int* status, cudaStream_t st) {
+  const size_t smem = 3 * (size_t)(bl.n_req + 1) * sizeof(int);
+  layout_kernel<<<1, 1024, smem, st>>>(bl, dm.n_kv, dm.mask_id, tok_per_tile, target_items, n_pages, status);
+}
+
+void launch_embed(const BatchLayout& bl, const Dims& dm, const void* embed, float* h, cudaStream_t st) {
+  embed_kernel<<<bl.n_tok, 256, 0, st>>>(bl.tok_id, static_cast<const __nv_bfloat16*>(embed), h, dm.hidden, dm.vocab);
+}
+
+void launch_rmsnorm(const float* h, const void* gain, void* x, int rows, int hidden, float eps, cudaStream_t st) {
+  rmsnorm_kernel<<<rows, 256, 0, st>>>(h, static_cast<const __nv_bfloat16*>(gain), static_cast<__nv_bfloat16*>(x),
+                                       hidden, eps);
+}
+
+void launch_kv_io(bool write, void* pool, int64_t n_pages, int layer, const Dims& dm, const int* page_row_dev, int pos0,
+                  int n_pos, void* k, void* v, int* status, cudaStream_t st) {
+  if (n_pos <= 0) return;
+  dim3 grid(n_pos, dm.n_kv);
+  kv_io_kernel<<<grid, dm.head_dim / 8, 0, st>>>(write, static_cast<__nv_bfloat16*>(pool), n_pages, layer, dm.n_kv,
+                                                 dm.head_dim, page_row_dev, pos0, static_cast<__nv_bfloat16*>(k),
+                                                 static_cast<__nv_bfloat16*>(v), status);
+}
+
+}  // namespace recg
+
+namespace recg {
+namespace {
+__global__ void rope_table_kernel(const int* __restrict__ tok_pos, int n_tok, int half, double log_base,
+                                  float2* __restrict__ cs) {
+  const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= n_tok * half) return;
+  const int t = idx / half, i = idx % half;
+  const double theta = exp(-log_base * (double)i / (double)half);  // base^(-2i/d)
+  const double ang = (double)tok_pos[t] * theta;
+  cs[idx] = make_float2((float)cos(ang), (float)sin(ang));
+}
+}  // namespace
+
+void launch_rope_table(const int* tok_pos, int n_tok, int head_dim, float rope_base, void* cs, cudaStream_t st) {
+  const int half = head_dim / 2;
+  const int total = n_tok * half;
+  if (total <= 0) return;
+  rope_table_kernel<<<(total + 255) / 256, 256, 0, st>>>(tok_pos, n_tok, half, log((double)rope_base),
+                                                         static_cast<float2*>(cs));
+}
+}  // namespace recg

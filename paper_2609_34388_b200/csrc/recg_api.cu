@@ -1,0 +1,497 @@
+// The C ABI: context, workspace, descriptor validation and the per-step launch sequence.
+#include <cstdio>
+#include <cstring>
+#include <string>
+#include <vector>
+
+#include "../../include/recg.h"
+#include "common.cuh"
+#include "kernels.h"
+
+using namespace recg;
+
+namespace {
+
+thread_local std::string g_init_error;
+
+struct DeviceArena {  // one cudaMalloc, carved with 256-byte alignment
+  uint8_t* base = nullptr;
+  size_t size = 0, used = 0;
+  template <typename T> T* take(size_t n) {
+    used = (used + 255) & ~size_t(255);
+    T* p = reinterpret_cast<T*>(base ? base + used : nullptr);
+    used += n * sizeof(T);
+    return p;
+  }
+};
+
+}  // namespace
+
+struct recg_ctx {
+  recg_config cfg;
+  Dims dm;
+  bool has_weights = false;
+  const void *embed = nullptr, *final_norm = nullptr, *lm_head = nullptr;
+  std::vector<const void*> attn_norm, wqkv, wo, ffn_norm, w_gate_up, w_down;
+  cudaStream_t stream = nullptr;
+  int n_sm = 0, tok_per_tile = 0, target_items = 0;
+  std::string err;
+
+  DeviceArena arena;
+  // descriptor staging (device)
+  int* d_desc = nullptr;
+  size_t desc_ints = 0;
+  BatchLayout bl{};
+  bool layout_valid = false;
+  bool layout_has_pages = false;
+  int64_t last_pool_pages = 0;
+  void* last_pool = nullptr;
+  // activations
+  float* h = nullptr;
+  __nv_bfloat16 *x = nullptr, *q = nullptr, *o = nullptr, *act = nullptr;
+  void* logits = nullptr;
+  bool logits_valid = false;
+  float2* rope_cs = nullptr;
+  float *part_o = nullptr, *part_ml = nullptr;
+  RowPartial* vpart = nullptr;
+  int max_chunks_total = 0;
+  VerifyBuffers vws{};
+  int* d_status = nullptr;
+  int* d_page_row = nullptr;
+  void* tc_state = nullptr;
+  std::vector<int> h_desc;
+};
+
+namespace {
+
+recg_status fail(recg_ctx* c, recg_status s, const std::string& msg) {
+  if (c) c->err = msg; else g_init_error = msg;
+  return s;
+}
+#define CU(call)                                                                                    \
+  do {                                                                                              \
+    cudaError_t e__ = (call);                                                                       \
+    if (e__ != cudaSuccess)                                                                         \
+      return fail(ctx, RECG_ERR_CUDA, std::string(#call) + ": " + cudaGetErrorString(e__));         \
+  } while (0)
+
+size_t carve(recg_ctx* c, DeviceArena& A) {
+  const recg_config& g = c->cfg;
+  const size_t Cm = g.max_requests, Tm = g.max_tokens, Pm = g.max_pages_per_request;
+  const Dims& d = c->dm;
+  c->desc_ints = 3 * Cm + 2 * (Cm + 1) + Tm + Cm * Pm;
+  c->d_desc = A.take<int>(c->desc_ints);
+  BatchLayout& bl = c->bl;
+  bl.tok_id = A.take<int>(Tm);
+  bl.tok_req = A.take<int>(Tm);
+  bl.tok_pos = A.take<int>(Tm);
+  bl.tok_slot = A.take<int>(Tm);
+  bl.tok_climit = A.take<int>(Tm);
+  bl.tok_lo = A.take<int>(Tm);
+  bl.tok_hi = A.take<int>(Tm);
+  const size_t max_tiles = (size_t)d.n_kv * (Cm + Tm / c->tok_per_tile + 1);
+  bl.max_parts = 2 * c->target_items;
+  bl.max_items = (int)(2 * c->target_items + max_tiles);
+  bl.items = A.take<AttnItem>(bl.max_items);
+  bl.tiles = A.take<AttnTile>(max_tiles);
+  bl.tile_off = A.take<int>(Cm + 1);
+  bl.counts = A.take<int>(4);
+  c->d_status = A.take<int>(1);
+  c->d_page_row = A.take<int>(Pm);
+  c->rope_cs = A.take<float2>(Tm * (d.head_dim / 2));
+  c->part_o = A.take<float>((size_t)bl.max_parts * 128 * d.head_dim);
+  c->part_ml = A.take<float>((size_t)bl.max_parts * 128 * 2);
+  c->max_chunks_total = (int)(Tm + 4 * c->n_sm + 64);
+  c->vpart = A.take<RowPartial>(c->max_chunks_total);
+  VerifyBuffers& v = c->vws;
+  v.accept_len = A.take<int>(Cm);
+  v.n_emitted = A.take<int>(Cm);
+  v.emitted = A.take<int>(Tm);
+  v.new_ctx_len = A.take<int>(Cm);
+  v.slot_state = A.take<int>(Tm);
+  v.freed_pages = A.take<int>(Cm);
+  v.next_draft = A.take<int>(Tm);
+  v.cont_hit = A.take<int>(Cm);
+  v.top1 = A.take<int>(Tm);
+  v.top2 = A.take<int>(Tm);
+  v.p1 = A.take<float>(Tm);
+  v.p2 = A.take<float>(Tm);
+  v.entropy = A.take<float>(Tm);
+  v.entropy_mean = A.take<float>(Cm);
+  c->q = A.take<__nv_bfloat16>(Tm * d.n_q * d.head_dim);
+  c->o = A.take<__nv_bfloat16>(Tm * d.n_q * d.head_dim);
+  if (c->has_weights) {
+    c->h = A.take<float>(Tm * d.hidden);
+    c->x = A.take<__nv_bfloat16>(Tm * d.hidden);
+    c->act = A.take<__nv_bfloat16>(Tm * d.ffn);
+    const size_t esz = (g.flags & RECG_FLAG_LOGITS_BF16) ? 2 : 4;
+    c->logits = A.take<uint8_t>(Tm * (size_t)d.vocab * esz);
+  }
+  return A.used + 256;
+}
+
+// Validate a batch and pack [ctx_len | verify_len | block_size | cu_tok | cu_ver | verify_tokens | page_table].
+recg_status pack_batch(recg_ctx* ctx, const recg_batch* b, bool need_pages, int* T_out, int* Tv_out) {
+  if (!b || b->n_req <= 0 || !b->ctx_len || !b->verify_len || !b->block_size)
+    return fail(ctx, RECG_ERR_INVALID_ARG, "batch: null descriptor array or n_req <= 0");
+  const int C = b->n_req;
+  if (C > ctx->cfg.max_requests) return fail(ctx, RECG_ERR_CAPACITY, "batch: n_req exceeds max_requests");
+  const bool pages = b->page_table != nullptr;
+  if (need_pages && (!pages || !b->kv_pool || b->kv_pool_pages <= 0))
+    return fail(ctx, RECG_ERR_INVALID_ARG, "batch: page_table and kv_pool are required");
+  if (pages && (b->page_table_stride <= 0 || b->page_table_stride > ctx->cfg.max_pages_per_request))
+    return fail(ctx, RECG_ERR_CAPACITY, "batch: page_table_stride exceeds max_pages_per_request");
+  long long T = 0, Tv = 0;
+  for (int r = 0; r < C; ++r) {
+    const int L = b->ctx_len[r], v = b->verify_len[r], k = b->block_size[r];
+    if (L < 0 || v < 0 || k < 0 || v + k < 1)
+      return fail(ctx, RECG_ERR_INVALID_ARG, "batch: negative length or a request without rows");
+    if (pages) {
+      const long long need = ((long long)L + v + k + kPageSize - 1) / kPageSize;
+      if (need > b->page_table_stride)
+        return fail(ctx, RECG_ERR_CAPACITY, "batch: page table row does not cover ctx_len + verify_len + block_size");
+    }
+    T += v + k;
+    Tv += v;
+  }
+  if (T > ctx->cfg.max_tokens) return fail(ctx, RECG_ERR_CAPACITY, "batch: token count exceeds max_tokens");
+  if (Tv > 0 && !b->verify_tokens) return fail(ctx, RECG_ERR_INVALID_ARG, "batch: verify_tokens is null");
+  const int stride = pages ? b->page_table_stride : 0;
+  std::vector<int>& hd = ctx->h_desc;
+  hd.resize(3 * (size_t)C + 2 * ((size_t)C + 1) + (size_t)Tv + (size_t)C * stride);
+  int* p = hd.data();
+  memcpy(p, b->ctx_len, C * sizeof(int));
+  memcpy(p + C, b->verify_len, C * sizeof(int));
+  memcpy(p + 2 * C, b->block_size, C * sizeof(int));
+  int* cu_tok = p + 3 * C;
+  int* cu_ver = cu_tok + (C + 1);
+  cu_tok[0] = cu_ver[0] = 0;
+  for (int r = 0; r < C; ++r) {
+    cu_tok[r + 1] = cu_tok[r] + b->verify_len[r] + b->block_size[r];
+    cu_ver[r + 1] = cu_ver[r] + b->verify_len[r];
+  }
+  int* vt = cu_ver + (C + 1);
+  if (Tv) memcpy(vt, b->verify_tokens, Tv * sizeof(int));
+  int* pt = vt + Tv;
+  if (pages) {
+    for (int r = 0; r < C; ++r) {
+      const long long need = ((long long)b->ctx_len[r] + b->verify_len[r] + b->block_size[r] + kPageSize - 1) / kPageSize;
+      for (int i = 0; i < stride; ++i) {
+        const int pg = b->page_table[(size_t)r * stride + i];
+        if (i < need && (pg < 0 || pg >= b->kv_pool_pages) && b->kv_pool)
+          return fail(ctx, RECG_ERR_INVALID_ARG, "batch: page id outside the pool");
+        pt[(size_t)r * stride + i] = pg;
+      }
+    }
+  }
+  BatchLayout& bl = ctx->bl;
+  int* d = ctx->d_desc;
+  bl.n_req = C;
+  bl.n_tok = (int)T;
+  bl.n_ver = (int)Tv;
+  bl.pt_stride = stride;
+  bl.ctx_len = d;
+  bl.verify_len = d + C;
+  bl.block_size = d + 2 * C;
+  bl.cu_tok = d + 3 * C;
+  bl.cu_ver = bl.cu_tok + (C + 1);
+  bl.verify_tokens = bl.cu_ver + (C + 1);
+  bl.page_table = pages ? bl.verify_tokens + Tv : nullptr;
+  *T_out = (int)T;
+  *Tv_out = (int)Tv;
+  return RECG_OK;
+}
+
+recg_status upload_and_layout(recg_ctx* ctx, const recg_batch* b, bool need_pages) {
+  int T = 0, Tv = 0;
+  ctx->layout_valid = false;
+  recg_status s = pack_batch(ctx, b, need_pages, &T, &Tv);
+  if (s != RECG_OK) return s;
+  CU(cudaMemcpyAsync(ctx->d_desc, ctx->h_desc.data(), ctx->h_desc.size() * sizeof(int), cudaMemcpyHostToDevice,
+                     ctx->stream));
+  const int64_t n_pages = b->page_table ? (b->kv_pool ? b->kv_pool_pages : (int64_t)1 << 40) : 0;
+  launch_layout(ctx->bl, ctx->dm, ctx->tok_per_tile, ctx->target_items, n_pages, ctx->d_status, ctx->stream);
+  CU(cudaGetLastError());
+  ctx->layout_valid = true;
+  ctx->layout_has_pages = b->page_table != nullptr;
+  ctx->last_pool = b->kv_pool;
+  ctx->last_pool_pages = b->kv_pool_pages;
+  return RECG_OK;
+}
+
+recg_status run_gemm(recg_ctx* ctx, const GemmArgs& a) {
+  bool done = false;
+  if (!(ctx->cfg.flags & RECG_FLAG_SIMT_GEMM)) done = launch_gemm_tc(a, ctx->tc_state, ctx->d_status, ctx->stream);
+  if (!done) launch_gemm_simt(a, ctx->d_status, ctx->stream);
+  CU(cudaGetLastError());
+  return RECG_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t recg_kv_pool_bytes(const recg_config* cfg, int64_t n_pages) {
+  if (!cfg || n_pages <= 0) return 0;
+  return (size_t)cfg->n_layers * (size_t)n_pages * cfg->n_kv_heads * 2 * kPageSize * cfg->head_dim * 2;
+}
+
+const char* recg_last_error(const recg_ctx* ctx) { return ctx ? ctx->err.c_str() : g_init_error.c_str(); }
+
+recg_status recg_init(recg_ctx** out, const recg_config* cfg, const recg_weights* w, void* cuda_stream) {
+  recg_ctx* ctx = nullptr;  // errors before allocation go to the thread-local text
+  if (!out || !cfg) return fail(ctx, RECG_ERR_INVALID_ARG, "recg_init: null argument");
+  *out = nullptr;
+  const recg_config& g = *cfg;
+  if (g.n_layers < 0 || g.hidden <= 0 || g.n_q_heads <= 0 || g.n_kv_heads <= 0 || g.vocab <= 1 || g.ffn <= 0 ||
+      g.max_requests <= 0 || g.max_tokens <= 0 || g.max_pages_per_request <= 0)
+    return fail(ctx, RECG_ERR_INVALID_ARG, "recg_init: non-positive dimension or capacity");
+  if (g.page_size != kPageSize) return fail(ctx, RECG_ERR_SHAPE, "recg_init: page_size must be 16");
+  if (g.head_dim != 64 && g.head_dim != 128) return fail(ctx, RECG_ERR_SHAPE, "recg_init: head_dim must be 64 or 128");
+  if (g.n_q_heads % g.n_kv_heads) return fail(ctx, RECG_ERR_SHAPE, "recg_init: n_q_heads must be a multiple of n_kv_heads");
+  const int group = g.n_q_heads / g.n_kv_heads;
+  if (group > 16 || (group & (group - 1))) return fail(ctx, RECG_ERR_SHAPE, "recg_init: GQA group must be 1, 2, 4, 8 or 16");
+  if (g.hidden % 64 || g.ffn % 64 || g.vocab % 16 || ((g.n_q_heads + 2 * g.n_kv_heads) * g.head_dim) % 128)
+    return fail(ctx, RECG_ERR_SHAPE, "recg_init: hidden and ffn must be multiples of 64, vocab of 16, qkv width of 128");
+  if (g.mask_token_id >= g.vocab) return fail(ctx, RECG_ERR_INVALID_ARG, "recg_init: mask_token_id outside the vocabulary");
+  if (w && g.n_layers > 0 &&
+      (!w->embed || !w->final_norm || !w->lm_head || !w->attn_norm || !w->wqkv || !w->wo || !w->ffn_norm ||
+       !w->w_gate_up || !w->w_down))
+    return fail(ctx, RECG_ERR_INVALID_ARG, "recg_init: null weight pointer");
+  int dev = 0, n_sm = 0, cc_major = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&cc_major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess)
+    return fail(ctx, RECG_ERR_CUDA, "recg_init: no usable CUDA device (there is no CPU fallback)");
+  if (cc_major != 10) return fail(ctx, RECG_ERR_CUDA, "recg_init: the kernels are built for sm_100a only");
+
+  ctx = new recg_ctx();
+  ctx->cfg = g;
+  ctx->dm = Dims{g.n_layers, g.hidden, g.n_q_heads, g.n_kv_heads, g.head_dim, g.ffn, g.vocab, g.rope_base, g.rms_eps,
+                 g.mask_token_id < 0 ? g.vocab - 1 : g.mask_token_id};
+  ctx->stream = static_cast<cudaStream_t>(cuda_stream);
+  ctx->n_sm = n_sm;
+  ctx->tok_per_tile = 128 / group;
+  ctx->target_items = n_sm;
+  ctx->has_weights = w != nullptr;
+  if (w) {
+    ctx->embed = w->embed;
+    ctx->final_norm = w->final_norm;
+    ctx->lm_head = w->lm_head;
+    for (int l = 0; l < g.n_layers; ++l) {
+      ctx->attn_norm.push_back(w->attn_norm[l]);
+      ctx->wqkv.push_back(w->wqkv[l]);
+      ctx->wo.push_back(w->wo[l]);
+      ctx->ffn_norm.push_back(w->ffn_norm[l]);
+      ctx->w_gate_up.push_back(w->w_gate_up[l]);
+      ctx->w_down.push_back(w->w_down[l]);
+      if (!w->attn_norm[l] || !w->wqkv[l] || !w->wo[l] || !w->ffn_norm[l] || !w->w_gate_up[l] || !w->w_down[l]) {
+        delete ctx;
+        ctx = nullptr;
+        return fail(ctx, RECG_ERR_INVALID_ARG, "recg_init: null per-layer weight pointer");
+      }
+    }
+  }
+  DeviceArena probe;
+  const size_t bytes = carve(ctx, probe);
+  cudaError_t e = cudaMalloc(reinterpret_cast<void**>(&ctx->arena.base), bytes);
+  if (e != cudaSuccess) {
+    std::string msg = std::string("recg_init: workspace cudaMalloc of ") + std::to_string(bytes) + " bytes: " + cudaGetErrorString(e);
+    delete ctx;
+    ctx = nullptr;
+    return fail(ctx, RECG_ERR_CUDA, msg);
+  }
+  ctx->arena.size = bytes;
+  carve(ctx, ctx->arena);
+  cudaMemsetAsync(ctx->d_status, 0, sizeof(int), ctx->stream);
+  ctx->tc_state = tc_state_create(n_sm);
+  *out = ctx;
+  return RECG_OK;
+}
+
+recg_status recg_free(recg_ctx* ctx) {
+  if (!ctx) return RECG_OK;
+  cudaStreamSynchronize(ctx->stream);
+  if (ctx->tc_state) tc_state_destroy(ctx->tc_state);
+  if (ctx->arena.base) cudaFree(ctx->arena.base);
+  delete ctx;
+  return RECG_OK;
+}
+
+recg_status recg_sync(recg_ctx* ctx) {
+  if (!ctx) return RECG_ERR_INVALID_ARG;
+  int st = 0;
+  CU(cudaMemcpyAsync(&st, ctx->d_status, sizeof(int), cudaMemcpyDeviceToHost, ctx->stream));
+  CU(cudaStreamSynchronize(ctx->stream));
+  if (st != DEV_OK) {
+    cudaMemsetAsync(ctx->d_status, 0, sizeof(int), ctx->stream);
+    if (st == DEV_BAD_INDEX) return fail(ctx, RECG_ERR_INTERNAL, "device: a page id or slot was out of range");
+    return fail(ctx, RECG_ERR_TIMEOUT, "device: a bounded wait gave up (code " + std::to_string(st) + ")");
+  }
+  return RECG_OK;
+}
+
+recg_status recg_step(recg_ctx* ctx, const recg_batch* batch, recg_logits* logits) {
+  if (!ctx) return RECG_ERR_INVALID_ARG;
+  if (!ctx->has_weights) return fail(ctx, RECG_ERR_INVALID_ARG, "recg_step: the context was created without weights");
+  ctx->logits_valid = false;
+  recg_status s = upload_and_layout(ctx, batch, true);
+  if (s != RECG_OK) return s;
+  const Dims& d = ctx->dm;
+  const BatchLayout& bl = ctx->bl;
+  const int T = bl.n_tok;
+  cudaStream_t st = ctx->stream;
+  launch_rope_table(bl.tok_pos, T, d.head_dim, d.rope_base, ctx->rope_cs, st);
+  launch_embed(bl, d, ctx->embed, ctx->h, st);
+  CU(cudaGetLastError());
+  const int qdim = d.n_q * d.head_dim;
+  for (int l = 0; l < d.n_layers; ++l) {
+    launch_rmsnorm(ctx->h, ctx->attn_norm[l], ctx->x, T, d.hidden, d.rms_eps, st);
+    GemmArgs a{};
+    a.x = ctx->x; a.w = ctx->wqkv[l]; a.out = ctx->q;
+    a.M = T; a.N = (d.n_q + 2 * d.n_kv) * d.head_dim; a.K = d.hidden; a.epi = EPI_QKV_ROPE;
+    a.tok_pos = bl.tok_pos; a.tok_slot = bl.tok_slot; a.kv_pool = batch->kv_pool; a.n_pages = batch->kv_pool_pages;
+    a.layer = l; a.n_q = d.n_q; a.n_kv = d.n_kv; a.head_dim = d.head_dim; a.rope_cs = ctx->rope_cs;
+    if ((s = run_gemm(ctx, a)) != RECG_OK) return s;
+    launch_attention(bl, d, l, ctx->q, ctx->o, batch->kv_pool, batch->kv_pool_pages, ctx->part_o, ctx->part_ml,
+                     ctx->tok_per_tile, ctx->n_sm, ctx->d_status, st);
+    CU(cudaGetLastError());
+    GemmArgs b{};
+    b.x = ctx->o; b.w = ctx->wo[l]; b.out = ctx->h; b.M = T; b.N = d.hidden; b.K = qdim; b.epi = EPI_RESIDUAL;
+    if ((s = run_gemm(ctx, b)) != RECG_OK) return s;
+    launch_rmsnorm(ctx->h, ctx->ffn_norm[l], ctx->x, T, d.hidden, d.rms_eps, st);
+    GemmArgs c{};
+    c.x = ctx->x; c.w = ctx->w_gate_up[l]; c.out = ctx->act; c.M = T; c.N = d.ffn; c.K = d.hidden; c.epi = EPI_SWIGLU;
+    if ((s = run_gemm(ctx, c)) != RECG_OK) return s;
+    GemmArgs e{};
+    e.x = ctx->act; e.w = ctx->w_down[l]; e.out = ctx->h; e.M = T; e.N = d.hidden; e.K = d.ffn; e.epi = EPI_RESIDUAL;
+    if ((s = run_gemm(ctx, e)) != RECG_OK) return s;
+  }
+  launch_rmsnorm(ctx->h, ctx->final_norm, ctx->x, T, d.hidden, d.rms_eps, st);
+  const bool lbf = ctx->cfg.flags & RECG_FLAG_LOGITS_BF16;
+  GemmArgs f{};
+  f.x = ctx->x; f.w = ctx->lm_head; f.out = ctx->logits; f.M = T; f.N = d.vocab; f.K = d.hidden;
+  f.epi = lbf ? EPI_PLAIN_BF16 : EPI_PLAIN_F32;
+  if ((s = run_gemm(ctx, f)) != RECG_OK) return s;
+  ctx->logits_valid = true;
+  if (logits) {
+    logits->data = ctx->logits;
+    logits->dtype = lbf ? RECG_DTYPE_BF16 : RECG_DTYPE_F32;
+    logits->n_rows = T;
+    logits->vocab = d.vocab;
+  }
+  return RECG_OK;
+}
+
+recg_status recg_verify(recg_ctx* ctx, const recg_batch* batch, const void* logits, int32_t logits_dtype,
+                        recg_verify_out* out) {
+  if (!ctx || !out) return RECG_ERR_INVALID_ARG;
+  if (out->mem != RECG_MEM_DEVICE && out->mem != RECG_MEM_HOST) return fail(ctx, RECG_ERR_INVALID_ARG, "recg_verify: bad out->mem");
+  if (logits) {
+    if (logits_dtype != RECG_DTYPE_BF16 && logits_dtype != RECG_DTYPE_F32)
+      return fail(ctx, RECG_ERR_INVALID_ARG, "recg_verify: unknown logits dtype");
+    if (batch) {
+      recg_status s = upload_and_layout(ctx, batch, false);
+      if (s != RECG_OK) return s;
+      ctx->logits_valid = false;
+    } else if (!ctx->layout_valid) {
+      return fail(ctx, RECG_ERR_INVALID_ARG, "recg_verify: no batch given and none laid out before");
+    }
+  } else {
+    if (!ctx->layout_valid || !ctx->logits_valid)
+      return fail(ctx, RECG_ERR_INVALID_ARG, "recg_verify: no logits given and no recg_step before");
+    if (batch && batch->n_req != ctx->bl.n_req)
+      return fail(ctx, RECG_ERR_INVALID_ARG, "recg_verify: batch differs from the one of the last recg_step");
+    logits = ctx->logits;
+    logits_dtype = (ctx->cfg.flags & RECG_FLAG_LOGITS_BF16) ? RECG_DTYPE_BF16 : RECG_DTYPE_F32;
+  }
+  const BatchLayout& bl = ctx->bl;
+  VerifyBuffers vb = ctx->vws;
+  const bool dev = out->mem == RECG_MEM_DEVICE;
+  if (dev) {
+#define PICK(f) if (out->f) vb.f = out->f
+    PICK(accept_len); PICK(n_emitted); PICK(emitted); PICK(new_ctx_len); PICK(slot_state); PICK(freed_pages);
+    PICK(next_draft); PICK(cont_hit); PICK(top1); PICK(top2); PICK(p1); PICK(p2); PICK(entropy); PICK(entropy_mean);
+#undef PICK
+  }
+  launch_verify(bl, logits, logits_dtype, ctx->dm.vocab, ctx->vpart, ctx->max_chunks_total, vb, ctx->n_sm, ctx->stream);
+  CU(cudaGetLastError());
+  if (!dev) {
+    const size_t C = bl.n_req, T = bl.n_tok, Tv = bl.n_ver, Tb = T - Tv;
+#define OUT(f, n) if (out->f && (n)) CU(cudaMemcpyAsync(out->f, vb.f, (n) * 4, cudaMemcpyDeviceToHost, ctx->stream))
+    OUT(accept_len, C); OUT(n_emitted, C); OUT(emitted, Tv); OUT(new_ctx_len, C); OUT(slot_state, T);
+    OUT(freed_pages, C); OUT(next_draft, Tb); OUT(cont_hit, C); OUT(top1, T); OUT(top2, T); OUT(p1, T); OUT(p2, T);
+    OUT(entropy, T); OUT(entropy_mean, C);
+#undef OUT
+    CU(cudaStreamSynchronize(ctx->stream));
+  }
+  return RECG_OK;
+}
+
+recg_status recg_attention(recg_ctx* ctx, const recg_batch* batch, int32_t layer, const void* q, void* o) {
+  if (!ctx || !q || !o) return RECG_ERR_INVALID_ARG;
+  if (layer < 0 || (ctx->cfg.n_layers > 0 && layer >= ctx->cfg.n_layers) ) return fail(ctx, RECG_ERR_INVALID_ARG, "recg_attention: layer out of range");
+  if (batch) {
+    recg_status s = upload_and_layout(ctx, batch, true);
+    if (s != RECG_OK) return s;
+    ctx->logits_valid = false;
+  } else if (!ctx->layout_valid || !ctx->layout_has_pages || !ctx->last_pool) {
+    return fail(ctx, RECG_ERR_INVALID_ARG, "recg_attention: no batch given and none with a KV pool laid out before");
+  }
+  launch_attention(ctx->bl, ctx->dm, layer, q, o, ctx->last_pool, ctx->last_pool_pages, ctx->part_o, ctx->part_ml,
+                   ctx->tok_per_tile, ctx->n_sm, ctx->d_status, ctx->stream);
+  CU(cudaGetLastError());
+  return RECG_OK;
+}
+
+static recg_status kv_io(recg_ctx* ctx, bool write, void* pool, int64_t n_pool_pages, int32_t layer,
+                         const int32_t* row, int32_t n_table, int32_t pos0, int32_t n_pos, void* k, void* v) {
+  if (!ctx || !pool || !row || !k || !v) return RECG_ERR_INVALID_ARG;
+  if (pos0 < 0 || n_pos < 0 || n_table <= 0 || n_table > ctx->cfg.max_pages_per_request || layer < 0 ||
+      (ctx->cfg.n_layers > 0 && layer >= ctx->cfg.n_layers) || n_pool_pages <= 0)
+    return fail(ctx, RECG_ERR_INVALID_ARG, "recg_kv_*: bad position range, layer or table length");
+  if (n_pos == 0) return RECG_OK;
+  if ((pos0 + n_pos - 1) / kPageSize >= n_table) return fail(ctx, RECG_ERR_CAPACITY, "recg_kv_*: positions beyond the page table row");
+  for (int i = pos0 / kPageSize; i <= (pos0 + n_pos - 1) / kPageSize; ++i)
+    if (row[i] < 0 || row[i] >= n_pool_pages) return fail(ctx, RECG_ERR_INVALID_ARG, "recg_kv_*: page id outside the pool");
+  CU(cudaMemcpyAsync(ctx->d_page_row, row, n_table * sizeof(int), cudaMemcpyHostToDevice, ctx->stream));
+  launch_kv_io(write, pool, n_pool_pages, layer, ctx->dm, ctx->d_page_row, pos0, n_pos, k, v, ctx->d_status, ctx->stream);
+  CU(cudaGetLastError());
+  return RECG_OK;
+}
+
+recg_status recg_kv_write(recg_ctx* ctx, void* kv_pool, int64_t kv_pool_pages, int32_t layer, const int32_t* page_table_row,
+                          int32_t n_table, int32_t pos0, int32_t n_pos, const void* k, const void* v) {
+  return kv_io(ctx, true, kv_pool, kv_pool_pages, layer, page_table_row, n_table, pos0, n_pos, const_cast<void*>(k),
+               const_cast<void*>(v));
+}
+recg_status recg_kv_read(recg_ctx* ctx, const void* kv_pool, int64_t kv_pool_pages, int32_t layer, const int32_t* page_table_row,
+                         int32_t n_table, int32_t pos0, int32_t n_pos, void* k, void* v) {
+  return kv_io(ctx, false, const_cast<void*>(kv_pool), kv_pool_pages, layer, page_table_row, n_table, pos0, n_pos, k, v);
+}
+
+recg_status recg_linear(recg_ctx* ctx, const void* x, const void* w, void* y, int32_t M, int32_t N, int32_t K,
+                        int32_t out_dtype) {
+  if (!ctx || !x || !w || !y) return RECG_ERR_INVALID_ARG;
+  if (M < 0 || N <= 0 || K <= 0 || N % 16 || K % 64) return fail(ctx, RECG_ERR_SHAPE, "recg_linear: N must be a multiple of 16 and K of 64");
+  if (out_dtype != RECG_DTYPE_BF16 && out_dtype != RECG_DTYPE_F32) return fail(ctx, RECG_ERR_INVALID_ARG, "recg_linear: unknown out dtype");
+  if (M == 0) return RECG_OK;
+  GemmArgs a{};
+  a.x = x; a.w = w; a.out = y; a.M = M; a.N = N; a.K = K;
+  a.epi = out_dtype == RECG_DTYPE_BF16 ? EPI_PLAIN_BF16 : EPI_PLAIN_F32;
+  return run_gemm(ctx, a);
+}
+
+recg_status recg_debug_buffer(recg_ctx* ctx, int32_t which, const void** ptr, int32_t* dtype, int32_t* rows, int32_t* cols) {
+  if (!ctx || !ptr || !dtype || !rows || !cols) return RECG_ERR_INVALID_ARG;
+  if (!ctx->has_weights || !ctx->logits_valid) return fail(ctx, RECG_ERR_INVALID_ARG, "recg_debug_buffer: no recg_step before");
+  *rows = ctx->bl.n_tok;
+  switch (which) {
+    case 0: *ptr = ctx->h; *dtype = RECG_DTYPE_F32; *cols = ctx->dm.hidden; break;
+    case 1: *ptr = ctx->o; *dtype = RECG_DTYPE_BF16; *cols = ctx->dm.n_q * ctx->dm.head_dim; break;
+    case 2: *ptr = ctx->q; *dtype = RECG_DTYPE_BF16; *cols = ctx->dm.n_q * ctx->dm.head_dim; break;
+    default: return fail(ctx, RECG_ERR_INVALID_ARG, "recg_debug_buffer: unknown buffer");
+  }
+  return RECG_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,269 @@
+// Fused greedy verification: one pass over the logits (top-2 ids, softmax mass, entropy) split over
+// vocab chunks, then a per-request finalize (accept-length scan, emitted tokens, continuation rule,
+// mean verifier entropy, KV commit / rollback indices).
+#include "common.cuh"
+#include "kernels.h"
+
+namespace recg {
+
+namespace {
+
+constexpr int kVerifyThreads = 256;
+
+struct Top2 {
+  float m1, m2;
+  int i1, i2;
+};
+__device__ __forceinline__ bool better(float av, int ai, float bv, int bi) { return av > bv || (av == bv && ai < bi); }
+__device__ __forceinline__ void top2_insert(Top2& t, float x, int i) {
+  if (better(x, i, t.m1, t.i1)) {
+    t.m2 = t.m1; t.i2 = t.i1; t.m1 = x; t.i1 = i;
+  } else if (better(x, i, t.m2, t.i2)) {
+    t.m2 = x; t.i2 = i;
+  }
+}
+
+// running softmax mass relative to a moving maximum m: s = sum e^(x-m), t = sum (x-m) e^(x-m)
+struct Mass {
+  float m, s, t;
+};
+__device__ __forceinline__ void mass_rebase(Mass& a, float m_new) {
+  if (m_new > a.m) {
+    const float d = a.m - m_new;  // <= 0 ; a.m may be -inf with s = t = 0
+    const float e = a.s > 0.f ? __expf(d) : 0.f;
+    a.t = e * (a.t + (a.s > 0.f ? d * a.s : 0.f));
+    a.s = e * a.s;
+    a.m = m_new;
+  }
+}
+__device__ __forceinline__ void mass_add(Mass& a, float x) {
+  const float d = x - a.m;
+  const float e = __expf(d);
+  a.s += e;
+  a.t += d * e;
+}
+__device__ __forceinline__ void mass_merge(Mass& a, const Mass& b) {
+  if (b.s <= 0.f) return;
+  Mass bb = b;
+  const float m = fmaxf(a.m, b.m);
+  mass_rebase(a, m);
+  mass_rebase(bb, m);
+  a.s += bb.s;
+  a.t += bb.t;
+}
+
+template <typename T> struct Vec;
+template <> struct Vec<__nv_bfloat16> {
+  static constexpr int N = 8;
+  __device__ static void load(const __nv_bfloat16* p, float (&x)[8]) {
+    uint4 u = __ldg(reinterpret_cast<const uint4*>(p));
+    const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      x[2 * i] = __uint_as_float(w[i] << 16);
+      x[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+    }
+  }
+  __device__ static float one(const __nv_bfloat16* p) { return __bfloat162float(*p); }
+};
+template <> struct Vec<float> {
+  static constexpr int N = 4;
+  __device__ static void load(const float* p, float (&x)[4]) {
+    float4 u = __ldg(reinterpret_cast<const float4*>(p));
+    x[0] = u.x; x[1] = u.y; x[2] = u.z; x[3] = u.w;
+  }
+  __device__ static float one(const float* p) { return *p; }
+};
+
+// grid (chunks_per_row, rows).  Each CTA scans [c0, c1) of one row.
+template <typename T>
+__global__ void __launch_bounds__(kVerifyThreads) verify_partial_kernel(const T* __restrict__ logits, int vocab,
+                                                                        int chunk_len, int chunks_per_row,
+                                                                        RowPartial* __restrict__ partials) {
+  constexpr int N = Vec<T>::N;
+  const int row = blockIdx.y, chunk = blockIdx.x;
+  const T* base = logits + (size_t)row * vocab;
+  const int c0 = chunk * chunk_len;
+  const int c1 = min(vocab, c0 + chunk_len);
+  Top2 tp = {-INFINITY, -INFINITY, 0x7fffffff, 0x7fffffff};
+  Mass ms = {-INFINITY, 0.f, 0.f};
+  const bool vec_ok = ((reinterpret_cast<uintptr_t>(base + c0) & 15) == 0);
+  int done = c0;
+  if (vec_ok) {
+    const int nvec = (c1 - c0) / N;
+    // two vectors in flight per thread
+    int i = threadIdx.x;
+    for (; i + kVerifyThreads < nvec; i += 2 * kVerifyThreads) {
+      float x[N], y[N];
+      Vec<T>::load(base + c0 + (size_t)i * N, x);
+      Vec<T>::load(base + c0 + (size_t)(i + kVerifyThreads) * N, y);
+      float vm = x[0];
+#pragma unroll
+      for (int k = 1; k < N; ++k) vm = fmaxf(vm, x[k]);
+#pragma unroll
+      for (int k = 0; k < N; ++k) vm = fmaxf(vm, y[k]);
+      mass_rebase(ms, vm);
+      const int ix = c0 + i * N, iy = c0 + (i + kVerifyThreads) * N;
+#pragma unroll
+      for (int k = 0; k < N; ++k) {
+        mass_add(ms, x[k]);
+        if (x[k] >= tp.m2) top2_insert(tp, x[k], ix + k);
+      }
+#pragma unroll
+      for (int k = 0; k < N; ++k) {
+        mass_add(ms, y[k]);
+        if (y[k] >= tp.m2) top2_insert(tp, y[k], iy + k);
+      }
+    }
+    for (; i < nvec; i += kVerifyThreads) {
+      float x[N];
+      Vec<T>::load(base + c0 + (size_t)i * N, x);
+      float vm = x[0];
+#pragma unroll
+      for (int k = 1; k < N; ++k) vm = fmaxf(vm, x[k]);
+      mass_rebase(ms, vm);
+      const int ix = c0 + i * N;
+#pragma unroll
+      for (int k = 0; k < N; ++k) {
+        mass_add(ms, x[k]);
+        if (x[k] >= tp.m2) top2_insert(tp, x[k], ix + k);
+      }
+    }
+    done = c0 + nvec * N;
+  }
+  for (int i = done + threadIdx.x; i < c1; i += kVerifyThreads) {
+    const float x = Vec<T>::one(base + i);
+    mass_rebase(ms, x);
+    mass_add(ms, x);
+    if (x >= tp.m2) top2_insert(tp, x, i);
+  }
+  // warp reduce, then across warps through shared memory
+#pragma unroll
+  for (int o = 16; o; o >>= 1) {
+    Top2 ot;
+    ot.m1 = __shfl_xor_sync(0xffffffffu, tp.m1, o);
+    ot.i1 = __shfl_xor_sync(0xffffffffu, tp.i1, o);
+    ot.m2 = __shfl_xor_sync(0xffffffffu, tp.m2, o);
+    ot.i2 = __shfl_xor_sync(0xffffffffu, tp.i2, o);
+    top2_insert(tp, ot.m1, ot.i1);
+    top2_insert(tp, ot.m2, ot.i2);
+    Mass om;
+    om.m = __shfl_xor_sync(0xffffffffu, ms.m, o);
+    om.s = __shfl_xor_sync(0xffffffffu, ms.s, o);
+    om.t = __shfl_xor_sync(0xffffffffu, ms.t, o);
+    mass_merge(ms, om);
+  }
+  __shared__ Top2 s_tp[kVerifyThreads / 32];
+  __shared__ Mass s_ms[kVerifyThreads / 32];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (lane == 0) {
+    s_tp[warp] = tp;
+    s_ms[warp] = ms;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int w = 1; w < kVerifyThreads / 32; ++w) {
+      top2_insert(tp, s_tp[w].m1, s_tp[w].i1);
+      top2_insert(tp, s_tp[w].m2, s_tp[w].i2);
+      mass_merge(ms, s_ms[w]);
+    }
+    // express the mass relative to the chunk maximum m1 (== ms.m unless the chunk is empty)
+    RowPartial p;
+    p.m1 = tp.m1; p.m2 = tp.m2; p.i1 = tp.i1; p.i2 = tp.i2;
+    p.s = ms.s; p.t = ms.t;
+    partials[(size_t)row * chunks_per_row + chunk] = p;
+  }
+}
+
+// One CTA per request: merge the chunk partials of its rows, then the accept scan and the index work.
+__global__ void __launch_bounds__(128) verify_finalize_kernel(BatchLayout bl, const RowPartial* __restrict__ partials,
+                                                              int chunks_per_row, VerifyBuffers vb) {
+  const int r = blockIdx.x;
+  const int t0 = bl.cu_tok[r];
+  const int v = bl.verify_len[r], b = bl.block_size[r], L = bl.ctx_len[r];
+  const int n = v + b;
+  for (int j = threadIdx.x; j < n; j += blockDim.x) {
+    const RowPartial* p = partials + (size_t)(t0 + j) * chunks_per_row;
+    Top2 tp = {-INFINITY, -INFINITY, 0x7fffffff, 0x7fffffff};
+    Mass ms = {-INFINITY, 0.f, 0.f};
+    for (int c = 0; c < chunks_per_row; ++c) {
+      const RowPartial q = p[c];
+      top2_insert(tp, q.m1, q.i1);
+      top2_insert(tp, q.m2, q.i2);
+      Mass o = {q.m1, q.s, q.t};
+      mass_merge(ms, o);
+    }
+    const float inv = 1.f / ms.s;
+    vb.top1[t0 + j] = tp.i1;
+    vb.top2[t0 + j] = tp.i2;
+    vb.p1[t0 + j] = inv;                             // e^(m1 - m1) / S
+    vb.p2[t0 + j] = __expf(tp.m2 - tp.m1) * inv;
+    vb.entropy[t0 + j] = logf(ms.s) - ms.t * inv;    // ln S - (1/S) sum (x-M) e^(x-M)
+  }
+  __syncthreads();
+  __shared__ int s_a;
+  if (threadIdx.x == 0) {
+    int a = 0;
+    const int tv0 = bl.cu_ver[r];
+    if (v > 0) {
+      while (a < v - 1 && bl.verify_tokens[tv0 + a + 1] == vb.top1[t0 + a]) ++a;
+      float es = 0.f;
+      for (int i = 0; i <= a; ++i) es += vb.entropy[t0 + i];
+      vb.entropy_mean[r] = es / (a + 1);
+      for (int i = 0; i < v; ++i)
+        vb.emitted[tv0 + i] = i < a ? bl.verify_tokens[tv0 + i + 1] : (i == a ? vb.top1[t0 + a] : -1);
+    } else {
+      vb.entropy_mean[r] = 0.f;
+    }
+    vb.accept_len[r] = a;
+    vb.n_emitted[r] = v > 0 ? a + 1 : 0;
+    const int new_L = L + (v > 0 ? a + 1 : 0);
+    vb.new_ctx_len[r] = new_L;
+    vb.cont_hit[r] = (v > 0 && b > 0 && a == v - 1 && vb.top1[t0 + v] == vb.top1[t0 + v - 1]) ? 1 : 0;
+    const int first_free = (new_L + kPageSize - 1) / kPageSize;
+    const int last = (L + n + kPageSize - 1) / kPageSize;
+    vb.freed_pages[r] = bl.page_table ? last - first_free : 0;
+    s_a = a;
+  }
+  __syncthreads();
+  const int a = s_a;
+  const int tb0 = t0 - bl.cu_ver[r];  // draft-token offset of this request: sum of b over earlier requests
+  for (int j = threadIdx.x; j < n; j += blockDim.x) {
+    if (j >= v) vb.next_draft[tb0 + (j - v)] = vb.top1[t0 + j];
+    const int slot = bl.tok_slot[t0 + j];
+    const bool committed = (j < v) && (j <= a);
+    vb.slot_state[t0 + j] = slot < 0 ? 0 : (committed ? slot : -(slot + 1));
+  }
+}
+
+}  // namespace
+
+int verify_chunks_per_row(int rows, int vocab, int n_sm) {
+  int by_size = (vocab + 4095) / 4096;
+  int by_rows = rows > 0 ? (n_sm * 4 + rows - 1) / rows : 1;
+  int c = by_size < by_rows ? by_size : by_rows;
+  if (c < 1) c = 1;
+  if (c > 64) c = 64;
+  return c;
+}
+
+void launch_verify(const BatchLayout& bl, const void* logits, int logits_dtype, int vocab, RowPartial* partials,
+                   int max_chunks_total, const VerifyBuffers& vb, int n_sm, cudaStream_t st) {
+  const int rows = bl.n_tok;
+  if (rows <= 0) return;
+  int chunks = verify_chunks_per_row(rows, vocab, n_sm);
+  while (chunks > 1 && (long long)chunks * rows > max_chunks_total) --chunks;
+  int chunk_len = (vocab + chunks - 1) / chunks;
+  chunk_len = (chunk_len + 63) / 64 * 64;  // keeps every chunk start 16-byte aligned relative to the row
+  chunks = (vocab + chunk_len - 1) / chunk_len;
+  dim3 grid(chunks, rows);
+  if (logits_dtype == 0)
+    verify_partial_kernel<__nv_bfloat16>
+        <<<grid, kVerifyThreads, 0, st>>>(static_cast<const __nv_bfloat16*>(logits), vocab, chunk_len, chunks, partials);
+  else
+    verify_partial_kernel<float>
+        <<<grid, kVerifyThreads, 0, st>>>(static_cast<const float*>(logits), vocab, chunk_len, chunks, partials);
+  verify_finalize_kernel<<<bl.n_req, 128, 0, st>>>(bl, partials, chunks, vb);
+}
+
+}  // namespace recg

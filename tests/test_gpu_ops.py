@@ -1,0 +1,254 @@
+"""GPU parity of the standalone operations (attention, verify, projection, KV import/export) against the oracle."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import recg_oracle as orc
+from paper_2609_34388_b200 import binding, synth
+from tests._util import f64
+
+pytestmark = pytest.mark.gpu
+
+
+def ops_ctx(shape, max_req, max_tok, max_pages, flags=0):
+    shape = synth.ModelShape(**{**shape.as_dict(), "n_layers": 1})
+    return binding.Context(binding.make_config(shape, max_req, max_tok, max_pages, flags))
+
+
+def run_attention_case(shape, reqs, seed, layer=0, poison=True):
+    """reqs: list of (L, v, b).  Returns (max abs err / max |ref|, per-request refs)."""
+    L = [r[0] for r in reqs]
+    v = [r[1] for r in reqs]
+    b = [r[2] for r in reqs]
+    desc = synth.fixed_descriptor(L, v, b, seed=seed)
+    T = desc.n_tokens
+    ctx = ops_ctx(shape, len(reqs), max(T, 1), desc.page_table.shape[1])
+    pool = binding.alloc_kv_pool(ctx, desc.n_pages, fill=None)
+    if poison:
+        pool.fill_(float("nan"))       # unwritten and invisible slots must never reach the output
+    q = synth.queries(T, shape.n_q_heads, shape.head_dim, seed=seed + 5)
+    ks, vs = [], []
+    for r in range(len(reqs)):
+        n = L[r] + v[r] + b[r]
+        k_, v_ = synth.kv_values(n, shape.n_kv_heads, shape.head_dim, seed=seed * 100 + r)
+        ks.append(k_)
+        vs.append(v_)
+        ctx.recg_kv_write(pool, desc.n_pages, layer, desc.page_table[r], 0, k_.cuda(), v_.cuda())
+    batch = binding.Batch(desc.ctx_len, desc.verify_len, desc.block_size, None, desc.page_table, pool, desc.n_pages)
+    o = torch.full((T, shape.n_q_heads, shape.head_dim), float("nan"), dtype=torch.bfloat16, device="cuda")
+    ctx.recg_attention(batch, layer, q.cuda(), o)
+    ctx.recg_sync()
+    got = f64(o)
+    worst = 0.0
+    t0 = 0
+    for r in range(len(reqs)):
+        n = v[r] + b[r]
+        ref = orc.hybrid_attention(f64(q[t0:t0 + n]), f64(ks[r]), f64(vs[r]), L[r], v[r], b[r])
+        assert not np.isnan(got[t0:t0 + n]).any(), f"NaN in request {r}"
+        worst = max(worst, np.max(np.abs(got[t0:t0 + n] - ref)) / np.max(np.abs(ref)))
+        t0 += n
+    # KV round trip through the pool layout
+    k_back, v_back = ctx.recg_kv_read(pool, desc.n_pages, layer, desc.page_table[0], 0, L[0] + v[0] + b[0])
+    assert torch.equal(k_back.cpu(), ks[0]) and torch.equal(v_back.cpu(), vs[0])
+    ctx.recg_free()
+    return worst
+
+
+ATTN_TOL = 1e-2   # relative to max |ref| (attention outputs within 1e-2 relative)
+
+
+@pytest.mark.parametrize("reqs", [
+    [(0, 1, 0)], [(0, 0, 1)], [(1, 1, 1)], [(15, 1, 0)], [(16, 2, 2)], [(17, 3, 8)], [(33, 8, 8)],
+    [(63, 1, 1)], [(64, 1, 0)], [(65, 0, 8)], [(200, 16, 16)], [(130, 5, 0)],
+    [(100, 4, 4), (7, 1, 8), (300, 16, 16), (64, 2, 2), (0, 8, 8)],
+])
+def test_attention_small(reqs):
+    for shape in (synth.tiny_shape(), synth.llama8b_shape(1)):
+        assert run_attention_case(shape, reqs, seed=11) < ATTN_TOL
+
+
+def test_attention_long_context_split_and_multi_tile():
+    shape = synth.llama8b_shape(1)
+    # 8B-class op: context 4096, 16 causal + 16 bidirectional rows (split over many KV ranges)
+    assert run_attention_case(shape, [(4096, 16, 16)], seed=21) < ATTN_TOL
+    # more rows than one tile (64 tokens x 4 heads = 256 rows) and a ragged tail
+    assert run_attention_case(shape, [(1000, 33, 31), (5, 40, 0)], seed=22) < ATTN_TOL
+    # many short requests next to a long one
+    assert run_attention_case(shape, [(3000, 2, 2)] + [(50 + 37 * i, 2, 2) for i in range(20)], seed=23) < ATTN_TOL
+    assert run_attention_case(synth.tiny_shape(), [(2500, 40, 30), (100, 70, 0)], seed=24) < ATTN_TOL
+
+
+def test_attention_is_deterministic():
+    shape = synth.llama8b_shape(1)
+    desc = synth.fixed_descriptor([1500, 40], [8, 4], [8, 4], seed=3)
+    ctx = ops_ctx(shape, 2, 32, desc.page_table.shape[1])
+    pool = binding.alloc_kv_pool(ctx, desc.n_pages, fill="normal")
+    batch = binding.Batch(desc.ctx_len, desc.verify_len, desc.block_size, None, desc.page_table, pool, desc.n_pages)
+    q = synth.queries(desc.n_tokens, 32, 128, seed=1).cuda()
+    o1, o2 = torch.empty_like(q), torch.empty_like(q)
+    ctx.recg_attention(batch, 0, q, o1)
+    ctx.recg_attention(None, 0, q, o2)      # reuse of the laid-out batch
+    ctx.recg_sync()
+    assert torch.equal(o1, o2)
+    ctx.recg_free()
+
+
+# ---------------------------------------------------------------- verification
+def run_verify_case(B, k, vocab, dtype, seed, sample=None):
+    shape = synth.ModelShape(n_layers=0, hidden=64, n_q_heads=4, n_kv_heads=2, head_dim=64, ffn=64, vocab=vocab)
+    R = B * (k + 1)
+    ctx = binding.Context(binding.make_config(shape, B, R, 1))
+    lg = synth.logits_normal(R, vocab, seed=seed, device="cuda", dtype=dtype)
+    lg_host = lg.cpu()
+    am = np.empty(R, dtype=np.int64)
+    for r0 in range(0, R, 256):          # planted drafts need each row's selected id: lowest index of the max
+        am[r0:r0 + 256] = lg_host[r0:r0 + 256].double().numpy().argmax(axis=1)
+    acc = synth.planted_accept_lengths(B, k, 0.25, seed=seed + 1)
+    if B >= 2:
+        acc[0], acc[1] = 0, k
+    y = synth.plant_drafts(am, B, k, acc, vocab, seed=seed + 2)
+    batch = binding.Batch([0] * B, [k + 1] * B, [0] * B, y.reshape(-1))
+    got = ctx.recg_verify(batch, lg)
+    ctx.recg_sync()
+    # by construction
+    assert got["accept_len"].tolist() == acc.tolist()
+    assert got["n_emitted"].tolist() == (acc + 1).tolist()
+    assert got["top1"].tolist() == am.tolist()
+    # against the oracle, on all or on sampled requests
+    reqs = range(B) if sample is None else sorted(set(np.random.default_rng(seed).integers(0, B, sample).tolist()) | {0, B - 1})
+    for r in reqs:
+        rows = slice(r * (k + 1), (r + 1) * (k + 1))
+        ref = orc.verify_round(lg_host[rows].double().numpy(), y[r].tolist(), 0)
+        assert int(got["accept_len"][r]) == ref["accept_len"]
+        em = got["emitted"][rows]
+        assert em[: ref["n_emitted"]].tolist() == ref["emitted"] and (em[ref["n_emitted"]:] == -1).all()
+        assert int(got["new_ctx_len"][r]) == ref["accept_len"] + 1 and int(got["cont_hit"][r]) == 0
+        st = ref["stats"]
+        assert got["top1"][rows].tolist() == [s["top1"] for s in st]
+        assert got["top2"][rows].tolist() == [s["top2"] for s in st]
+        np.testing.assert_allclose(got["p1"][rows], [s["p1"] for s in st], rtol=2e-4, atol=1e-7)
+        np.testing.assert_allclose(got["p2"][rows], [s["p2"] for s in st], rtol=2e-4, atol=1e-7)
+        np.testing.assert_allclose(got["entropy"][rows], [s["entropy"] for s in st], rtol=2e-4, atol=1e-5)
+        assert abs(float(got["entropy_mean"][r]) - ref["entropy_mean"]) < 2e-4 * max(1.0, ref["entropy_mean"])
+    ctx.recg_free()
+
+
+@pytest.mark.parametrize("B,k", [(1, 4), (8, 8), (32, 4), (3, 32), (32, 16)])
+def test_verify_sweep_bf16(B, k):
+    run_verify_case(B, k, 128256, torch.bfloat16, seed=40 + B + k)
+
+
+def test_verify_fp32_and_odd_vocab():
+    run_verify_case(4, 4, 128256, torch.float32, seed=7)
+    run_verify_case(5, 3, 2048, torch.bfloat16, seed=8)
+    run_verify_case(2, 2, 1000 * 16, torch.float32, seed=9)
+
+
+def test_verify_full_size_sampled():
+    # largest sweep point: 256 requests x 33 rows x 128256 logits (2.17 GB); oracle on sampled requests
+    run_verify_case(256, 32, 128256, torch.bfloat16, seed=99, sample=6)
+
+
+def test_verify_closed_forms_and_ties():
+    V = 4096
+    shape = synth.ModelShape(n_layers=0, hidden=64, n_q_heads=4, n_kv_heads=2, head_dim=64, ffn=64, vocab=V)
+    ctx = binding.Context(binding.make_config(shape, 4, 16, 1))
+    lg = torch.zeros((4, V), dtype=torch.float32)
+    lg[0] = 1.5                                   # uniform
+    lg[1, 777] = 60.0                             # dominant
+    lg[2, 100] = lg[2, 3000] = 2.0                # two equal maxima
+    lg[3] = torch.linspace(-3, 3, V)
+    lg[3, 5] = lg[3, -1]                          # tie between index 5 and the last index
+    batch = binding.Batch([0], [1], [3], [0])
+    got = ctx.recg_verify(batch, lg.cuda())
+    assert got["top1"].tolist() == [0, 777, 100, 5] and got["top2"].tolist() == [1, 0, 3000, V - 1]
+    assert abs(got["p1"][0] - 1.0 / V) < 1e-9 and abs(got["entropy"][0] - np.log(V)) < 1e-4
+    assert abs(got["p1"][1] - 1.0) < 1e-6 and abs(got["entropy"][1]) < 1e-5
+    assert got["p1"][2] == got["p2"][2]
+    assert got["next_draft"].tolist() == [777, 100, 5] and got["accept_len"].tolist() == [0]
+    ctx.recg_free()
+
+
+def test_verify_commit_indices_and_continuation():
+    """Ragged batch with a page table: slot states, freed pages, continuation rule, v = 0 and b = 0 requests."""
+    V = 2048
+    shape = synth.ModelShape(n_layers=0, hidden=64, n_q_heads=4, n_kv_heads=2, head_dim=64, ffn=64, vocab=V)
+    L, v, b = [31, 5, 40, 16], [8, 0, 3, 1], [8, 4, 0, 15]
+    desc = synth.fixed_descriptor(L, v, b, seed=5)
+    T = desc.n_tokens
+    ctx = binding.Context(binding.make_config(shape, 4, T, desc.page_table.shape[1]))
+    lg = synth.logits_normal(T, V, seed=3, dtype=torch.float32)
+    am = lg.double().numpy().argmax(axis=1)
+    # request 0: accept 3 of 7 drafts; request 2: all accepted; request 3: v = 1 and the first draft row repeats the bonus
+    y0 = [9] + am[0:3].tolist() + [(int(am[3]) + 1) % V, 1, 2, 3]
+    y2 = [4] + am[20:22].tolist()
+    lg[24] = lg[23]                                  # request 3: row 23 verify, row 24 first draft row
+    y = y0 + y2 + [11]
+    batch = binding.Batch(L, v, b, y, desc.page_table, None, 0)
+    got = ctx.recg_verify(batch, lg.cuda())
+    ref = orc.verify_batch(lg.double().numpy(), v, b, y)
+    t0 = 0
+    for r in range(4):
+        rr = ref[r]
+        assert int(got["accept_len"][r]) == rr["accept_len"] and int(got["cont_hit"][r]) == int(rr["cont_hit"])
+        kc = orc.kv_commit(L[r], v[r], b[r], rr["accept_len"], desc.page_table[r], 16)
+        assert int(got["new_ctx_len"][r]) == kc["new_ctx_len"] and int(got["freed_pages"][r]) == len(kc["freed_pages"])
+        ss = got["slot_state"][t0:t0 + v[r] + b[r]].tolist()
+        assert [s for s in ss if s >= 0] == kc["commit_slots"]
+        assert [-(s + 1) for s in ss if s < 0] == kc["rollback_slots"]
+        t0 += v[r] + b[r]
+    assert got["accept_len"].tolist() == [3, 0, 2, 0] and got["cont_hit"].tolist() == [0, 0, 0, 1]
+    nd = [d for r in ref for d in r["next_draft"]]
+    assert got["next_draft"].tolist() == nd
+    ctx.recg_free()
+
+
+# ---------------------------------------------------------------- projection
+@pytest.mark.parametrize("flags", [0, binding.FLAG_SIMT_GEMM])
+@pytest.mark.parametrize("M,N,K", [(1, 128, 64), (31, 256, 256), (128, 512, 1024), (129, 6144, 4096), (300, 4096, 14336),
+                                   (77, 2048, 256), (515, 1024, 4096)])
+def test_linear(M, N, K, flags):
+    shape = synth.tiny_shape()
+    ctx = ops_ctx(shape, 1, 8, 1, flags)
+    g = torch.Generator().manual_seed(M * 7 + N)
+    x = torch.randn((M, K), generator=g).to(torch.bfloat16)
+    w = (torch.randn((N, K), generator=g) * 0.05).to(torch.bfloat16)
+    ref = x.double().numpy() @ w.double().numpy().T
+    y = ctx.recg_linear(x.cuda(), w.cuda(), torch.float32)
+    ctx.recg_sync()
+    err = np.max(np.abs(f64(y) - ref)) / np.max(np.abs(ref))
+    assert err < 1e-5, err                                 # fp32 accumulation of exact bf16 products
+    yb = ctx.recg_linear(x.cuda(), w.cuda(), torch.bfloat16)
+    assert np.max(np.abs(f64(yb) - ref)) / np.max(np.abs(ref)) < 5e-3
+    ctx.recg_free()
+
+
+def test_host_side_rejections():
+    shape = synth.tiny_shape()
+    ctx = ops_ctx(shape, 2, 16, 4)
+    lg = torch.zeros((4, shape.vocab), dtype=torch.float32, device="cuda")
+    with pytest.raises(binding.RecgError) as e:
+        ctx.recg_verify(binding.Batch([0, 0, 0], [1, 1, 1], [0, 0, 0], [0, 0, 0]), lg)     # too many requests
+    assert e.value.status == 3
+    with pytest.raises(binding.RecgError) as e:
+        ctx.recg_verify(binding.Batch([0], [20], [0], [0] * 20), lg)                        # too many tokens
+    assert e.value.status == 3
+    with pytest.raises(binding.RecgError) as e:
+        ctx.recg_verify(binding.Batch([0], [0], [0], None), lg)                             # a request without rows
+    assert e.value.status == 1
+    with pytest.raises(binding.RecgError) as e:
+        ctx.recg_verify(binding.Batch([-1], [1], [0], [0]), lg)
+    assert e.value.status == 1
+    pool = torch.zeros(ctx.kv_pool_bytes(4) // 2, dtype=torch.bfloat16, device="cuda")
+    q = torch.zeros((4, 4, 64), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(binding.RecgError) as e:      # page table too short for L + v + b = 100 tokens
+        ctx.recg_attention(binding.Batch([96], [2], [2], None, np.zeros((1, 4), np.int32), pool, 4), 0, q, q.clone())
+    assert e.value.status == 3
+    with pytest.raises(binding.RecgError) as e:      # page id outside the pool
+        ctx.recg_attention(binding.Batch([10], [2], [2], None, np.full((1, 4), 9, np.int32), pool, 4), 0, q, q.clone())
+    assert e.value.status == 1
+    with pytest.raises(binding.RecgError) as e:      # step on a context without weights
+        ctx.recg_step(binding.Batch([10], [2], [2], [1, 2], np.zeros((1, 4), np.int32), pool, 4))
+    assert e.value.status == 1
+    ctx.recg_sync()
+    ctx.recg_free()

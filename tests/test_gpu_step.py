@@ -1,0 +1,195 @@
+"""GPU parity of the whole fused draft+verify round (recg_step + recg_verify) against the oracle."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import recg_oracle as orc
+from paper_2609_34388_b200 import binding, synth
+from tests._util import bf16_round, f64, oracle_cfg, oracle_weights
+
+pytestmark = pytest.mark.gpu
+
+HID_TOL = 2e-2      # max-abs error of hidden states and logits, relative to max |ref|
+MARGIN_FLAG = 1e-2  # integer results may differ only where the oracle's top-2 logit gap is below this
+
+
+def to_dev(W):
+    return {k: ([t.cuda() for t in v] if isinstance(v, list) else v.cuda()) for k, v in W.items()}
+
+
+def tiny_model(perturb=True):
+    shape = synth.tiny_shape()
+    W = synth.model_weights(shape, seed=0, dtype=torch.bfloat16)
+    if perturb:
+        synth.perturb_norm_gains(W)
+    return shape, W, oracle_cfg(shape), oracle_weights(W)
+
+
+def build_requests(ocfg, W64, shape, specs, seed):
+    """specs: (L, v, b, m): context length, verify length, block, planted accept length (or None: random drafts).
+    Returns per request: prompt, bf16-rounded prefix KV, y."""
+    out = []
+    for i, (L, v, b, m) in enumerate(specs):
+        prompt = synth.token_ids(L + 1, shape.vocab, seed=seed + i).tolist()
+        kv, L0, y0 = orc.prefill(ocfg, W64, prompt)
+        assert L0 == L
+        kv = [(bf16_round(K), bf16_round(V)) for (K, V) in kv]
+        y = []
+        if v > 0:
+            if m is None:
+                y = y0 + synth.token_ids(v - 1, shape.vocab, seed=seed + 50 + i).tolist()
+            else:
+                truth = orc.greedy_ar(ocfg, W64, prompt, v - 1) if v > 1 else []
+                y = y0 + truth
+                if m + 1 <= v - 1:
+                    y[m + 1] = (y[m + 1] + 1) % (shape.vocab - 1)
+        out.append({"prompt": prompt, "kv": kv, "y": y, "L": L, "v": v, "b": b, "m": m})
+    return out
+
+
+def check_round(ctx, shape, ocfg, W64, reqs, desc, pool, strict_planted=True):
+    ys = [t for r in reqs for t in r["y"]]
+    batch = binding.Batch(desc.ctx_len, desc.verify_len, desc.block_size, ys, desc.page_table, pool, desc.n_pages)
+    lg = ctx.recg_step(batch)
+    got = ctx.recg_verify(batch)
+    ctx.recg_sync()
+    logits = f64(ctx.logits_tensor(lg))
+    hidden = f64(ctx.recg_debug_buffer(0))
+    t0 = tv0 = tb0 = 0
+    n_flagged = 0
+    for i, r in enumerate(reqs):
+        L, v, b = r["L"], r["v"], r["b"]
+        n = v + b
+        ref_logits, ref_kv, ref_h = orc.fused_round_cached(ocfg, W64, r["kv"], L, r["y"], b)
+        assert np.max(np.abs(hidden[t0:t0 + n] - ref_h)) <= HID_TOL * np.max(np.abs(ref_h)), f"hidden, request {i}"
+        assert np.max(np.abs(logits[t0:t0 + n] - ref_logits)) <= HID_TOL * np.max(np.abs(ref_logits)), f"logits, request {i}"
+        # tentative K/V of the new rows, every layer
+        for l, (K, V) in enumerate(ref_kv):
+            kg, vg = ctx.recg_kv_read(pool, desc.n_pages, l, desc.page_table[i], L, n)
+            assert np.max(np.abs(f64(kg) - K[L:])) <= HID_TOL * np.max(np.abs(K[L:])), f"K layer {l} request {i}"
+            assert np.max(np.abs(f64(vg) - V[L:])) <= HID_TOL * np.max(np.abs(V[L:])), f"V layer {l} request {i}"
+        ref = orc.verify_round(ref_logits, r["y"], b)
+        st = ref["stats"]
+        gaps = np.array([s["logit_gap"] for s in st])
+        top1 = got["top1"][t0:t0 + n]
+        for j in range(n):
+            if gaps[j] >= MARGIN_FLAG:
+                assert int(top1[j]) == st[j]["top1"], f"top1 row {j} request {i}"
+            else:
+                n_flagged += 1
+        a = ref["accept_len"]
+        decisive = gaps[: min(a + 1, v)] if v else np.array([1.0])
+        if v and (decisive >= MARGIN_FLAG).all():
+            assert int(got["accept_len"][i]) == a
+            assert got["emitted"][tv0:tv0 + v][: a + 1].tolist() == ref["emitted"]
+            kc = orc.kv_commit(L, v, b, a, desc.page_table[i], 16)
+            assert int(got["new_ctx_len"][i]) == kc["new_ctx_len"]
+            ss = got["slot_state"][t0:t0 + n].tolist()
+            assert [s for s in ss if s >= 0] == kc["commit_slots"]
+            assert [-(s + 1) for s in ss if s < 0] == kc["rollback_slots"]
+            assert int(got["freed_pages"][i]) == len(kc["freed_pages"])
+            if r["m"] is not None and strict_planted:
+                assert a == r["m"]
+            em = sum(st[j]["entropy"] for j in range(a + 1)) / (a + 1)
+            assert abs(float(got["entropy_mean"][i]) - em) < 2e-2 * max(em, 1.0)
+        if (gaps[v:] >= MARGIN_FLAG).all():
+            assert got["next_draft"][tb0:tb0 + b].tolist() == ref["next_draft"]
+        np.testing.assert_allclose(got["p1"][t0:t0 + n], [s["p1"] for s in st], rtol=0.1, atol=1e-5)
+        np.testing.assert_allclose(got["entropy"][t0:t0 + n], [s["entropy"] for s in st], rtol=2e-2, atol=1e-3)
+        t0 += n
+        tv0 += v
+        tb0 += b
+    return n_flagged, got
+
+
+@pytest.mark.parametrize("flags", [0, binding.FLAG_SIMT_GEMM])
+def test_tiny_round_ragged_batch(flags):
+    shape, W, ocfg, W64 = tiny_model()
+    specs = [(63, 1, 8, None), (40, 8, 8, 3), (17, 3, 4, 2), (100, 5, 0, 0), (1, 4, 4, 1), (33, 8, 8, 7), (5, 0, 8, None)]
+    reqs = build_requests(ocfg, W64, shape, specs, seed=100)
+    desc = synth.fixed_descriptor([s[0] for s in specs], [s[1] for s in specs], [s[2] for s in specs], seed=9)
+    ctx = binding.Context(binding.make_config(shape, 8, 128, desc.page_table.shape[1], flags), to_dev(W))
+    pool = binding.alloc_kv_pool(ctx, desc.n_pages, fill=None)
+    pool.fill_(float("nan"))
+    for i, r in enumerate(reqs):
+        for l, (K, V) in enumerate(r["kv"]):
+            if r["L"]:
+                ctx.recg_kv_write(pool, desc.n_pages, l, desc.page_table[i], 0,
+                                  torch.from_numpy(K).to(torch.bfloat16).cuda(), torch.from_numpy(V).to(torch.bfloat16).cuda())
+    flagged, got = check_round(ctx, shape, ocfg, W64, reqs, desc, pool)
+    # batch invariance: every request alone gives the same integers and (bitwise) the same logits rows
+    ys = [t for r in reqs for t in r["y"]]
+    full = ctx.logits_tensor(ctx.recg_step(binding.Batch(desc.ctx_len, desc.verify_len, desc.block_size, ys,
+                                                         desc.page_table, pool, desc.n_pages)))
+    t0 = 0
+    for i, r in enumerate(reqs):
+        n = r["v"] + r["b"]
+        solo = binding.Batch([r["L"]], [r["v"]], [r["b"]], r["y"], desc.page_table[i:i + 1], pool, desc.n_pages)
+        lg = ctx.logits_tensor(ctx.recg_step(solo))
+        g1 = ctx.recg_verify(solo)
+        assert int(g1["accept_len"][0]) == int(got["accept_len"][i])
+        assert g1["top1"].tolist() == got["top1"][t0:t0 + n].tolist()
+        ref = full[t0:t0 + n]
+        assert float((lg - ref).abs().max()) <= 1e-3 * float(ref.abs().max())
+        t0 += n
+    ctx.recg_sync()
+    ctx.recg_free()
+
+
+def test_tiny_self_speculative_loop_is_lossless():
+    """The GPU drives 4 rounds itself (KV pool, lengths and drafts carried from its own outputs); the emitted
+    tokens must be the oracle's greedy continuation."""
+    shape, W, ocfg, W64 = tiny_model(perturb=False)
+    prompt = synth.token_ids(64, shape.vocab, seed=1).tolist()
+    b, rounds = 8, 4
+    ar = orc.greedy_ar(ocfg, W64, prompt, rounds * (b + 1))
+    kv, L, y = orc.prefill(ocfg, W64, prompt)
+    pt, n_pages = synth.page_tables([L], [rounds * (b + 1) + 2 * b], 16, seed=3)
+    ctx = binding.Context(binding.make_config(shape, 1, 64, pt.shape[1]), to_dev(W))
+    pool = binding.alloc_kv_pool(ctx, n_pages, fill=None)
+    pool.fill_(float("nan"))
+    for l, (K, V) in enumerate(kv):
+        ctx.recg_kv_write(pool, n_pages, l, pt[0], 0, torch.from_numpy(K).to(torch.bfloat16).cuda(),
+                          torch.from_numpy(V).to(torch.bfloat16).cuda())
+    out = []
+    for t in range(rounds):
+        # teacher-force drafts every second round so that long accepts, commits and rollbacks all occur
+        if t % 2 == 1:
+            y = [y[0]] + ar[len(out): len(out) + 5]
+            y[4] = (y[4] + 1) % (shape.vocab - 1)
+        batch = binding.Batch([L], [len(y)], [b], y, pt, pool, n_pages)
+        ctx.recg_step(batch)
+        g = ctx.recg_verify(batch)
+        a = int(g["accept_len"][0])
+        out += g["emitted"][: a + 1].tolist()
+        L = int(g["new_ctx_len"][0])
+        bonus = int(g["emitted"][a])
+        y = [bonus] + g["next_draft"][1:].tolist() if int(g["cont_hit"][0]) else [bonus]
+        if t % 2 == 1:
+            assert a == 3
+    ctx.recg_sync()
+    # oracle gaps along the greedy path decide whether exact equality is required
+    assert out == ar[: len(out)], (out, ar[: len(out)])
+    ctx.recg_free()
+
+
+def test_llama8b_shape_one_layer_round():
+    """One 8B-shaped layer + LM head on a ragged batch (spans several GEMM tiles and a ragged tail)."""
+    shape = synth.llama8b_shape(1)
+    shape.vocab = 16384            # keeps the oracle's LM head quick; every other dimension is the 8B one
+    W = synth.model_weights(shape, seed=0, dtype=torch.bfloat16)
+    ocfg, W64 = oracle_cfg(shape), oracle_weights(W)
+    specs = [(200, 16, 16), (70, 4, 4), (33, 2, 2), (500, 32, 32), (16, 8, 8), (129, 3, 30)]
+    L, v, b = [s[0] for s in specs], [s[1] for s in specs], [s[2] for s in specs]
+    desc = synth.fixed_descriptor(L, v, b, seed=4)
+    ctx = binding.Context(binding.make_config(shape, 8, 256, desc.page_table.shape[1]), to_dev(W))
+    pool = binding.alloc_kv_pool(ctx, desc.n_pages, fill=None)
+    pool.fill_(float("nan"))
+    reqs = []
+    for i in range(len(specs)):
+        K, V = synth.kv_values(L[i], shape.n_kv_heads, shape.head_dim, seed=300 + i)
+        ctx.recg_kv_write(pool, desc.n_pages, 0, desc.page_table[i], 0, K.cuda(), V.cuda())
+        y = synth.token_ids(v[i], shape.vocab, seed=400 + i).tolist()
+        reqs.append({"kv": [(f64(K), f64(V))], "y": y, "L": L[i], "v": v[i], "b": b[i], "m": None})
+    flagged, _ = check_round(ctx, shape, ocfg, W64, reqs, desc, pool)
+    ctx.recg_free()
