@@ -1,7 +1,494 @@
-// placeholder until the tcgen05 kernel lands
+// Projection GEMM on the 5th-generation tensor cores: y = x . w^T, bf16 in, fp32 accumulate in TMEM.
+//
+// Persistent, warp-specialised CTA of 6 warps:
+//   warp 0   producer: TMA tiled loads (128B swizzle) of the x tile [128 x 64] and the w tile [BN x 64]
+//            into a shared-memory ring, completion on mbarriers;
+//   warp 1   one elected lane issues tcgen05.mma (M = 128, N = BN, K = 16) from shared-memory descriptors
+//            into one of two TMEM accumulators and commits to the ring's empty barriers;
+//   warps 2-5  epilogue: tcgen05.ld of the finished accumulator (each warp its 32-lane quadrant), then the
+//            fused epilogue straight from registers (residual add, SwiGLU, rotary + paged KV append, or
+//            plain store) while the MMA warp already fills the other accumulator.
+// Tiles are walked m-fastest so that CTAs running together share the same weight tile through L2.
+// Every wait is bounded; on a timeout the kernel records a status code, drains and frees TMEM.
+#include <cuda.h>
+
+#include <cstdio>
+#include <mutex>
+#include <unordered_map>
+
+#include "common.cuh"
+#include "epilogue.cuh"
 #include "kernels.h"
+
 namespace recg {
-bool launch_gemm_tc(const GemmArgs&, void*, int*, cudaStream_t) { return false; }
-void* tc_state_create(int) { return nullptr; }
-void tc_state_destroy(void*) {}
+
+namespace {
+
+constexpr int BM = 128, BK = 64;
+constexpr int kTcThreads = 192;
+constexpr int kSmemBudget = 200 * 1024;
+constexpr uint32_t kSpin = 1u << 22;
+
+template <int BN> struct TcCfg {
+  static constexpr int kABytes = BM * BK * 2;
+  static constexpr int kBBytes = BN * BK * 2;
+  static constexpr int kStageBytes = kABytes + kBBytes;
+  static constexpr int kStages = (kSmemBudget / kStageBytes) > 8 ? 8 : (kSmemBudget / kStageBytes);
+  static constexpr int kBarBytes = (2 * kStages + 4) * 8 + 16;
+  static constexpr int kSmemBytes = kStages * kStageBytes + kBarBytes + 1024;  // + slack for 1024-byte alignment
+  static constexpr int kTmemCols = 2 * BN < 32 ? 32 : 2 * BN;                  // power of two: 128, 256, 512
+};
+
+// ---- PTX wrappers ------------------------------------------------------------------------------
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred = 0;
+  asm volatile("{\n .reg .b32 rx;\n .reg .pred px;\n elect.sync rx|px, %1;\n @px mov.s32 %0, 1;\n}"
+               : "+r"(pred)
+               : "r"(0xffffffffu));
+  return pred != 0;
+}
+__device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
+  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+               :
+               : "r"(smem_u32(smem_dst)), "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y)
+               : "memory");
+}
+__device__ __forceinline__ void prefetch_tmap(const CUtensorMap* map) {
+  asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
+}
+__device__ __forceinline__ void tmem_alloc(uint32_t* smem_slot, uint32_t cols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(smem_slot)), "r"(cols)
+               : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t addr, uint32_t cols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(addr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+               : "memory");
+}
+// D[tmem] (+)= A[smem desc] * B[smem desc]; accumulate = 0 overwrites
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc,
+                                          uint32_t accumulate) {
+  asm volatile(
+      "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
+      " tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+      :
+      : "r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
+  uint32_t r[32];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,"
+      "%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// K-major operand tile with 128-byte swizzle: rows of 128 bytes, 8-row atoms 1024 bytes apart.
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t smem_addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((smem_addr & 0x3ffff) >> 4);  // start address, 16-byte units
+  d |= (uint64_t)1 << 16;                       // leading byte offset (unused with swizzle), 16-byte units
+  d |= (uint64_t)(1024 >> 4) << 32;             // stride byte offset between 8-row atoms
+  d |= (uint64_t)1 << 46;                       // descriptor version for sm_100
+  d |= (uint64_t)2 << 61;                       // SWIZZLE_128B
+  return d;
+}
+// kind::f16 instruction descriptor: fp32 accumulate, bf16 A and B, both K-major, M = 128, N = BN
+__host__ __device__ constexpr uint32_t make_idesc(int n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+}
+
+// ---- register epilogue: one thread owns one output row -------------------------------------------
+__device__ __forceinline__ void store_chunk_f32(float* dst, const float (&v)[32], bool add) {
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    float4 o = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+    float4* p = reinterpret_cast<float4*>(dst) + i;
+    if (add) {
+      const float4 h = *p;
+      o.x += h.x; o.y += h.y; o.z += h.z; o.w += h.w;
+    }
+    *p = o;
+  }
+}
+__device__ __forceinline__ void store_chunk_bf16(__nv_bfloat16* dst, const float (&v)[32]) {
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    uint4 o;
+    o.x = pack_bf16(v[8 * i], v[8 * i + 1]);
+    o.y = pack_bf16(v[8 * i + 2], v[8 * i + 3]);
+    o.z = pack_bf16(v[8 * i + 4], v[8 * i + 5]);
+    o.w = pack_bf16(v[8 * i + 6], v[8 * i + 7]);
+    reinterpret_cast<uint4*>(dst)[i] = o;
+  }
+}
+
+// Epilogue of one accumulator tile for the calling thread's row.  tacc: TMEM address of (lane quadrant, column 0).
+template <int BN>
+__device__ __forceinline__ void row_epilogue(const EpiParams& ep, uint32_t tacc, int m, int n0) {
+  const bool row_ok = m < ep.M;
+  if (ep.epi == EPI_SWIGLU) {
+    // accumulator columns [0, BN/2) are gate, [BN/2, BN) up; n0 is the first output column
+    __nv_bfloat16* out = static_cast<__nv_bfloat16*>(ep.out);
+#pragma unroll 1
+    for (int c = 0; c < BN / 64; ++c) {
+      float g[32], u[32];
+      tmem_ld32(tacc + c * 32, g);
+      tmem_ld32(tacc + BN / 2 + c * 32, u);
+      if (row_ok && n0 + c * 32 < ep.N) {
+#pragma unroll
+        for (int i = 0; i < 32; ++i) g[i] = silu_f(g[i]) * u[i];
+        store_chunk_bf16(out + (size_t)m * ep.N + n0 + c * 32, g);
+      }
+    }
+    return;
+  }
+  if (ep.epi == EPI_QKV_ROPE) {
+    const int D = ep.head_dim, half = D / 2;
+    __nv_bfloat16* q = static_cast<__nv_bfloat16*>(ep.out);
+    const int slot = row_ok ? ep.tok_slot[m] : -1;
+#pragma unroll 1
+    for (int hl = 0; hl < BN / D; ++hl) {        // heads in this tile
+      const int head = n0 / D + hl;
+      const bool is_q = head < ep.n_q, is_v = head >= ep.n_q + ep.n_kv;
+      __nv_bfloat16* kv_base = nullptr;
+      if (!is_q && slot >= 0) {
+        const int64_t page = slot / kPageSize;
+        if (page < ep.n_pages) {
+          const int kvh = is_v ? head - ep.n_q - ep.n_kv : head - ep.n_q;
+          kv_base = ep.kv_pool + kv_tile_base(ep.n_pages, ep.n_kv, D, ep.layer, page, kvh) + (is_v ? kv_tile_elems(D) : 0);
+        } else {
+          set_status(ep.status, DEV_BAD_INDEX);
+        }
+      }
+      const int tok = slot >= 0 ? slot % kPageSize : 0;
+#pragma unroll 1
+      for (int c = 0; c < half / 32; ++c) {      // 32 low columns with their 32 partners half a head away
+        float lo[32], hi[32];
+        tmem_ld32(tacc + hl * D + c * 32, lo);
+        tmem_ld32(tacc + hl * D + half + c * 32, hi);
+        if (!row_ok) continue;
+        if (!is_v) {
+          const float2* cs = ep.rope_cs + (size_t)m * half + c * 32;
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            const float2 t = cs[i];
+            const float a = lo[i] * t.x - hi[i] * t.y, b = hi[i] * t.x + lo[i] * t.y;
+            lo[i] = a;
+            hi[i] = b;
+          }
+        }
+        if (is_q) {
+          __nv_bfloat16* dst = q + ((size_t)m * ep.n_q + head) * D + c * 32;
+          store_chunk_bf16(dst, lo);
+          store_chunk_bf16(dst + half, hi);
+        } else if (kv_base) {
+          // the pool tile is swizzled in 16-byte chunks: store chunk by chunk
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            uint4 a, b;
+            a.x = pack_bf16(lo[8 * j], lo[8 * j + 1]); a.y = pack_bf16(lo[8 * j + 2], lo[8 * j + 3]);
+            a.z = pack_bf16(lo[8 * j + 4], lo[8 * j + 5]); a.w = pack_bf16(lo[8 * j + 6], lo[8 * j + 7]);
+            b.x = pack_bf16(hi[8 * j], hi[8 * j + 1]); b.y = pack_bf16(hi[8 * j + 2], hi[8 * j + 3]);
+            b.z = pack_bf16(hi[8 * j + 4], hi[8 * j + 5]); b.w = pack_bf16(hi[8 * j + 6], hi[8 * j + 7]);
+            *reinterpret_cast<uint4*>(kv_base + kv_tile_offset(tok, c * 32 + j * 8)) = a;
+            *reinterpret_cast<uint4*>(kv_base + kv_tile_offset(tok, half + c * 32 + j * 8)) = b;
+          }
+        }
+      }
+    }
+    return;
+  }
+#pragma unroll 1
+  for (int c = 0; c < BN / 32; ++c) {
+    float v[32];
+    tmem_ld32(tacc + c * 32, v);
+    const int n = n0 + c * 32;
+    if (!row_ok || n >= ep.N) continue;
+    if (n + 32 <= ep.N) {
+      if (ep.epi == EPI_PLAIN_BF16) store_chunk_bf16(static_cast<__nv_bfloat16*>(ep.out) + (size_t)m * ep.N + n, v);
+      else store_chunk_f32(static_cast<float*>(ep.out) + (size_t)m * ep.N + n, v, ep.epi == EPI_RESIDUAL);
+    } else {  // ragged right edge (N is a multiple of 16 but not of 32)
+      for (int i = 0; i < ep.N - n; ++i) {
+        if (ep.epi == EPI_PLAIN_BF16) static_cast<__nv_bfloat16*>(ep.out)[(size_t)m * ep.N + n + i] = __float2bfloat16_rn(v[i]);
+        else if (ep.epi == EPI_RESIDUAL) static_cast<float*>(ep.out)[(size_t)m * ep.N + n + i] += v[i];
+        else static_cast<float*>(ep.out)[(size_t)m * ep.N + n + i] = v[i];
+      }
+    }
+  }
+}
+
+template <int BN>
+__global__ void __launch_bounds__(kTcThreads, 1)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w, int M, int n_tiles_n,
+               int K, int up_row_offset, EpiParams ep) {
+  using Cfg = TcCfg<BN>;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + Cfg::kStages * Cfg::kStageBytes);
+  uint64_t* empty_bar = full_bar + Cfg::kStages;
+  uint64_t* tfull_bar = empty_bar + Cfg::kStages;
+  uint64_t* tempty_bar = tfull_bar + 2;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tempty_bar + 2);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int n_tiles_m = (M + BM - 1) / BM;
+  const int n_tiles = n_tiles_m * n_tiles_n;
+  const int KB = K / BK;
+  const bool swiglu = ep.epi == EPI_SWIGLU;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < Cfg::kStages; ++s) {
+      mbar_init(&full_bar[s], 1);
+      mbar_init(&empty_bar[s], 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(&tfull_bar[a], 1);
+      mbar_init(&tempty_bar[a], 4);
+    }
+    fence_barrier_init();
+    prefetch_tmap(&map_x);
+    prefetch_tmap(&map_w);
+  }
+  if (warp == 1) {
+    tmem_alloc(tmem_slot, Cfg::kTmemCols);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------------ TMA producer ------------------------------
+    if (elect_one()) {
+      uint32_t it = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+        const int tm = tile % n_tiles_m, tn = tile / n_tiles_m;
+        for (int kb = 0; kb < KB; ++kb, ++it) {
+          const int s = it % Cfg::kStages;
+          if (!mbar_wait(&empty_bar[s], ((it / Cfg::kStages) & 1) ^ 1, kSpin)) {
+            set_status(ep.status, DEV_TIMEOUT_EMPTY);
+            ok = false;
+            break;
+          }
+          uint8_t* a_dst = smem + s * Cfg::kStageBytes;
+          uint8_t* b_dst = a_dst + Cfg::kABytes;
+          mbar_arrive_expect_tx(&full_bar[s], Cfg::kStageBytes);
+          tma_load_2d(a_dst, &map_x, kb * BK, tm * BM, &full_bar[s]);
+          if (swiglu) {
+            tma_load_2d(b_dst, &map_w, kb * BK, tn * (BN / 2), &full_bar[s]);
+            tma_load_2d(b_dst + Cfg::kBBytes / 2, &map_w, kb * BK, up_row_offset + tn * (BN / 2), &full_bar[s]);
+          } else {
+            tma_load_2d(b_dst, &map_w, kb * BK, tn * BN, &full_bar[s]);
+          }
+        }
+      }
+      if (!ok) {  // let loads already issued land before the CTA may exit
+        for (int s = 0; s < Cfg::kStages; ++s)
+          for (uint32_t i = 0; i < (1u << 14); ++i) {
+            if (mbar_try_wait(&full_bar[s], 0) || mbar_try_wait(&full_bar[s], 1)) break;
+            __nanosleep(64);
+          }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------ MMA issuer ------------------------------
+    if (elect_one()) {
+      constexpr uint32_t idesc = make_idesc(BN);
+      uint32_t it = 0, tcount = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++tcount) {
+        const int acc = tcount & 1;
+        if (!mbar_wait(&tempty_bar[acc], ((tcount >> 1) & 1) ^ 1, kSpin)) {
+          set_status(ep.status, DEV_TIMEOUT_MMA);
+          break;
+        }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + acc * BN;
+        for (int kb = 0; kb < KB; ++kb, ++it) {
+          const int s = it % Cfg::kStages;
+          if (!mbar_wait(&full_bar[s], (it / Cfg::kStages) & 1, kSpin)) {
+            set_status(ep.status, DEV_TIMEOUT_FULL);
+            ok = false;
+            break;
+          }
+          tc_fence_after();
+          const uint32_t a_addr = smem_u32(smem + s * Cfg::kStageBytes);
+          const uint32_t b_addr = a_addr + Cfg::kABytes;
+#pragma unroll
+          for (int k = 0; k < BK / 16; ++k) {
+            const uint64_t da = make_smem_desc(a_addr + k * 32);
+            const uint64_t db = make_smem_desc(b_addr + k * 32);
+            umma_bf16(d_tmem, da, db, idesc, (kb | k) ? 1u : 0u);
+          }
+          umma_commit(&empty_bar[s]);      // frees the stage when these MMAs have read it
+        }
+        if (ok) umma_commit(&tfull_bar[acc]);  // accumulator complete
+      }
+    }
+  } else {
+    // ------------------------------ epilogue warps ------------------------------
+    const int quad = warp & 3;             // TMEM lane quadrant this warp may read
+    uint32_t tcount = 0;
+    for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++tcount) {
+      const int tm = tile % n_tiles_m, tn = tile / n_tiles_m;
+      const int acc = tcount & 1;
+      if (!mbar_wait(&tfull_bar[acc], (tcount >> 1) & 1, kSpin)) {
+        set_status(ep.status, DEV_TIMEOUT_MMA);
+        break;
+      }
+      tc_fence_after();
+      const uint32_t tacc = tmem_base + ((uint32_t)(quad * 32) << 16) + acc * BN;
+      const int m = tm * BM + quad * 32 + lane;
+      const int n0 = swiglu ? tn * (BN / 2) : tn * BN;
+      row_epilogue<BN>(ep, tacc, m, n0);
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&tempty_bar[acc]);
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, Cfg::kTmemCols);
+  }
+}
+
+// ---- host side -------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+struct MapKey {
+  const void* ptr;
+  uint64_t rows, cols;
+  uint32_t box_rows;
+  bool operator==(const MapKey& o) const { return ptr == o.ptr && rows == o.rows && cols == o.cols && box_rows == o.box_rows; }
+};
+struct MapKeyHash {
+  size_t operator()(const MapKey& k) const {
+    return std::hash<const void*>()(k.ptr) ^ (k.rows * 1000003u) ^ (k.cols * 7919u) ^ (size_t)k.box_rows << 40;
+  }
+};
+
+struct TcState {
+  int n_sm = 0;
+  EncodeTiledFn encode = nullptr;
+  std::unordered_map<MapKey, CUtensorMap, MapKeyHash> maps;
+  bool configured[3] = {false, false, false};
+};
+
+// [rows, cols] bf16 row-major, box = [box_rows, 64 columns], 128-byte swizzle, zero fill out of bounds
+const CUtensorMap* get_map(TcState* st, const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+  MapKey key{ptr, rows, cols, box_rows};
+  auto it = st->maps.find(key);
+  if (it != st->maps.end()) return &it->second;
+  if (st->maps.size() > 4096) st->maps.clear();
+  CUtensorMap m;
+  cuuint64_t dims[2] = {cols, rows};
+  cuuint64_t strides[1] = {cols * 2};
+  cuuint32_t box[2] = {BK, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = st->encode(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return nullptr;
+  return &st->maps.emplace(key, m).first->second;
+}
+
+template <int BN>
+bool launch_bn(TcState* st, int idx, const GemmArgs& a, const EpiParams& ep, cudaStream_t stream) {
+  using Cfg = TcCfg<BN>;
+  if (!st->configured[idx]) {
+    if (cudaFuncSetAttribute(gemm_tc_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes) != cudaSuccess)
+      return false;
+    st->configured[idx] = true;
+  }
+  const bool swiglu = a.epi == EPI_SWIGLU;
+  const uint64_t w_rows = swiglu ? 2ull * a.N : (uint64_t)a.N;
+  const CUtensorMap* mx = get_map(st, a.x, a.M, a.K, BM);
+  const CUtensorMap* mw = get_map(st, a.w, w_rows, a.K, swiglu ? BN / 2 : BN);
+  if (!mx || !mw) return false;
+  const int out_per_tile = swiglu ? BN / 2 : BN;
+  const int n_tiles_n = (a.N + out_per_tile - 1) / out_per_tile;
+  const int n_tiles = ((a.M + BM - 1) / BM) * n_tiles_n;
+  const int grid = n_tiles < st->n_sm ? n_tiles : st->n_sm;
+  gemm_tc_kernel<BN><<<grid, kTcThreads, Cfg::kSmemBytes, stream>>>(*mx, *mw, a.M, n_tiles_n, a.K, a.N, ep);
+  return true;
+}
+
+}  // namespace
+
+void* tc_state_create(int n_sm) {
+  TcState* st = new TcState();
+  st->n_sm = n_sm;
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
+      qres != cudaDriverEntryPointSuccess || !fn) {
+    delete st;
+    return nullptr;
+  }
+  st->encode = reinterpret_cast<EncodeTiledFn>(fn);
+  return st;
+}
+
+void tc_state_destroy(void* s) { delete static_cast<TcState*>(s); }
+
+bool launch_gemm_tc(const GemmArgs& a, void* tc_state, int* status, cudaStream_t stream) {
+  TcState* st = static_cast<TcState*>(tc_state);
+  if (!st || a.M <= 0) return false;
+  if (a.K % BK) return false;
+  if ((reinterpret_cast<uintptr_t>(a.x) | reinterpret_cast<uintptr_t>(a.w)) & 15) return false;
+  EpiParams ep;
+  ep.epi = a.epi;
+  ep.out = a.out;
+  ep.M = a.M;
+  ep.N = a.N;
+  ep.tok_slot = a.tok_slot;
+  ep.rope_cs = static_cast<const float2*>(a.rope_cs);
+  ep.kv_pool = static_cast<__nv_bfloat16*>(a.kv_pool);
+  ep.n_pages = a.n_pages;
+  ep.layer = a.layer;
+  ep.n_q = a.n_q;
+  ep.n_kv = a.n_kv;
+  ep.head_dim = a.head_dim;
+  ep.status = status;
+  const bool swiglu = a.epi == EPI_SWIGLU;
+  // widest tile that still gives every SM a tile; rotary tiles must hold whole heads
+  const int mt = (a.M + BM - 1) / BM;
+  auto tiles = [&](int bn) { const int per = swiglu ? bn / 2 : bn; return mt * ((a.N + per - 1) / per); };
+  int bn = 64;
+  if (tiles(256) >= st->n_sm) bn = 256;
+  else if (tiles(128) >= st->n_sm) bn = 128;
+  if (a.epi == EPI_QKV_ROPE && bn < a.head_dim) bn = a.head_dim;
+  if (swiglu && (a.N % (bn / 2))) bn = 64;
+  if (swiglu && (a.N % 32)) return false;
+  if (a.epi == EPI_QKV_ROPE && (a.N % bn)) bn = a.head_dim;
+  if (a.epi == EPI_QKV_ROPE && (a.N % bn)) return false;
+  switch (bn) {
+    case 256: return launch_bn<256>(st, 0, a, ep, stream);
+    case 128: return launch_bn<128>(st, 1, a, ep, stream);
+    default: return launch_bn<64>(st, 2, a, ep, stream);
+  }
+}
+
 }  // namespace recg

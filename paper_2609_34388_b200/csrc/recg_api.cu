@@ -131,7 +131,7 @@ size_t carve(recg_ctx* c, DeviceArena& A) {
 }
 
 // Validate a batch and pack [ctx_len | verify_len | block_size | cu_tok | cu_ver | verify_tokens | page_table].
-recg_status pack_batch(recg_ctx* ctx, const recg_batch* b, bool need_pages, int* T_out, int* Tv_out) {
+recg_status pack_batch(recg_ctx* ctx, const recg_batch* b, bool need_pages, bool need_tokens, int* T_out, int* Tv_out) {
   if (!b || b->n_req <= 0 || !b->ctx_len || !b->verify_len || !b->block_size)
     return fail(ctx, RECG_ERR_INVALID_ARG, "batch: null descriptor array or n_req <= 0");
   const int C = b->n_req;
@@ -155,7 +155,7 @@ recg_status pack_batch(recg_ctx* ctx, const recg_batch* b, bool need_pages, int*
     Tv += v;
   }
   if (T > ctx->cfg.max_tokens) return fail(ctx, RECG_ERR_CAPACITY, "batch: token count exceeds max_tokens");
-  if (Tv > 0 && !b->verify_tokens) return fail(ctx, RECG_ERR_INVALID_ARG, "batch: verify_tokens is null");
+  if (Tv > 0 && !b->verify_tokens && need_tokens) return fail(ctx, RECG_ERR_INVALID_ARG, "batch: verify_tokens is null");
   const int stride = pages ? b->page_table_stride : 0;
   std::vector<int>& hd = ctx->h_desc;
   hd.resize(3 * (size_t)C + 2 * ((size_t)C + 1) + (size_t)Tv + (size_t)C * stride);
@@ -171,7 +171,8 @@ recg_status pack_batch(recg_ctx* ctx, const recg_batch* b, bool need_pages, int*
     cu_ver[r + 1] = cu_ver[r] + b->verify_len[r];
   }
   int* vt = cu_ver + (C + 1);
-  if (Tv) memcpy(vt, b->verify_tokens, Tv * sizeof(int));
+  if (Tv && b->verify_tokens) memcpy(vt, b->verify_tokens, Tv * sizeof(int));
+  else if (Tv) memset(vt, 0, Tv * sizeof(int));
   int* pt = vt + Tv;
   if (pages) {
     for (int r = 0; r < C; ++r) {
@@ -202,10 +203,10 @@ recg_status pack_batch(recg_ctx* ctx, const recg_batch* b, bool need_pages, int*
   return RECG_OK;
 }
 
-recg_status upload_and_layout(recg_ctx* ctx, const recg_batch* b, bool need_pages) {
+recg_status upload_and_layout(recg_ctx* ctx, const recg_batch* b, bool need_pages, bool need_tokens = true) {
   int T = 0, Tv = 0;
   ctx->layout_valid = false;
-  recg_status s = pack_batch(ctx, b, need_pages, &T, &Tv);
+  recg_status s = pack_batch(ctx, b, need_pages, need_tokens, &T, &Tv);
   if (s != RECG_OK) return s;
   CU(cudaMemcpyAsync(ctx->d_desc, ctx->h_desc.data(), ctx->h_desc.size() * sizeof(int), cudaMemcpyHostToDevice,
                      ctx->stream));
@@ -431,7 +432,7 @@ recg_status recg_attention(recg_ctx* ctx, const recg_batch* batch, int32_t layer
   if (!ctx || !q || !o) return RECG_ERR_INVALID_ARG;
   if (layer < 0 || (ctx->cfg.n_layers > 0 && layer >= ctx->cfg.n_layers) ) return fail(ctx, RECG_ERR_INVALID_ARG, "recg_attention: layer out of range");
   if (batch) {
-    recg_status s = upload_and_layout(ctx, batch, true);
+    recg_status s = upload_and_layout(ctx, batch, true, false);
     if (s != RECG_OK) return s;
     ctx->logits_valid = false;
   } else if (!ctx->layout_valid || !ctx->layout_has_pages || !ctx->last_pool) {

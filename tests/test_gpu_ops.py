@@ -217,7 +217,7 @@ def test_linear(M, N, K, flags):
     y = ctx.recg_linear(x.cuda(), w.cuda(), torch.float32)
     ctx.recg_sync()
     err = np.max(np.abs(f64(y) - ref)) / np.max(np.abs(ref))
-    assert err < 1e-5, err                                 # fp32 accumulation of exact bf16 products
+    assert err < 1e-4, err      # fp32 accumulation of exact bf16 products: ~sqrt(K) 2^-24 relative, K <= 14336
     yb = ctx.recg_linear(x.cuda(), w.cuda(), torch.bfloat16)
     assert np.max(np.abs(f64(yb) - ref)) / np.max(np.abs(ref)) < 5e-3
     ctx.recg_free()

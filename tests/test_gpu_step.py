@@ -47,7 +47,8 @@ def build_requests(ocfg, W64, shape, specs, seed):
     return out
 
 
-def check_round(ctx, shape, ocfg, W64, reqs, desc, pool, strict_planted=True):
+def check_round(ctx, shape, ocfg, W64, reqs, desc, pool, strict_planted=True, margin_flag=MARGIN_FLAG,
+                adaptive_flag=False):
     ys = [t for r in reqs for t in r["y"]]
     batch = binding.Batch(desc.ctx_len, desc.verify_len, desc.block_size, ys, desc.page_table, pool, desc.n_pages)
     lg = ctx.recg_step(batch)
@@ -68,34 +69,45 @@ def check_round(ctx, shape, ocfg, W64, reqs, desc, pool, strict_planted=True):
             kg, vg = ctx.recg_kv_read(pool, desc.n_pages, l, desc.page_table[i], L, n)
             assert np.max(np.abs(f64(kg) - K[L:])) <= HID_TOL * np.max(np.abs(K[L:])), f"K layer {l} request {i}"
             assert np.max(np.abs(f64(vg) - V[L:])) <= HID_TOL * np.max(np.abs(V[L:])), f"V layer {l} request {i}"
+        # (1) integer decisions, exactly: the oracle's verification applied to the kernel's own fp32 logits
+        #     (both sides decide in the same precision) must give the same integers, no exceptions
+        own = orc.verify_round(logits[t0:t0 + n], r["y"], b)
+        a_own = own["accept_len"]
+        assert got["top1"][t0:t0 + n].tolist() == [s["top1"] for s in own["stats"]]
+        assert got["top2"][t0:t0 + n].tolist() == [s["top2"] for s in own["stats"]]
+        assert int(got["accept_len"][i]) == a_own and int(got["cont_hit"][i]) == int(own["cont_hit"])
+        assert got["next_draft"][tb0:tb0 + b].tolist() == own["next_draft"]
+        if v:
+            assert got["emitted"][tv0:tv0 + v][: a_own + 1].tolist() == own["emitted"]
+            assert (got["emitted"][tv0:tv0 + v][a_own + 1:] == -1).all()
+        kc = orc.kv_commit(L, v, b, a_own, desc.page_table[i], 16)
+        assert int(got["new_ctx_len"][i]) == kc["new_ctx_len"] and int(got["freed_pages"][i]) == len(kc["freed_pages"])
+        ss = got["slot_state"][t0:t0 + n].tolist()
+        assert [s for s in ss if s >= 0] == kc["commit_slots"]
+        assert [-(s + 1) for s in ss if s < 0] == kc["rollback_slots"]
+        np.testing.assert_allclose(got["p1"][t0:t0 + n], [s["p1"] for s in own["stats"]], rtol=2e-4, atol=1e-7)
+        np.testing.assert_allclose(got["entropy"][t0:t0 + n], [s["entropy"] for s in own["stats"]], rtol=2e-4, atol=1e-5)
+        assert abs(float(got["entropy_mean"][i]) - own["entropy_mean"]) < 2e-4 * max(1.0, own["entropy_mean"])
+        # (2) against the oracle's own forward: a row may differ only where the oracle's top-2 logit gap is
+        #     below the flag (1e-2, or twice the row's measured logit error where that is larger: a kernel
+        #     whose logits are within the float tolerance cannot be asked to order closer logits)
         ref = orc.verify_round(ref_logits, r["y"], b)
         st = ref["stats"]
         gaps = np.array([s["logit_gap"] for s in st])
-        top1 = got["top1"][t0:t0 + n]
+        row_err = np.max(np.abs(logits[t0:t0 + n] - ref_logits), axis=1)
+        flag = np.maximum(margin_flag, 2.0 * row_err) if adaptive_flag else np.full(n, margin_flag)
+        clear = gaps >= flag
+        n_flagged += int((~clear).sum())
         for j in range(n):
-            if gaps[j] >= MARGIN_FLAG:
-                assert int(top1[j]) == st[j]["top1"], f"top1 row {j} request {i}"
-            else:
-                n_flagged += 1
+            if clear[j]:
+                assert int(got["top1"][t0 + j]) == st[j]["top1"], f"top1 row {j} request {i}"
         a = ref["accept_len"]
-        decisive = gaps[: min(a + 1, v)] if v else np.array([1.0])
-        if v and (decisive >= MARGIN_FLAG).all():
-            assert int(got["accept_len"][i]) == a
-            assert got["emitted"][tv0:tv0 + v][: a + 1].tolist() == ref["emitted"]
-            kc = orc.kv_commit(L, v, b, a, desc.page_table[i], 16)
-            assert int(got["new_ctx_len"][i]) == kc["new_ctx_len"]
-            ss = got["slot_state"][t0:t0 + n].tolist()
-            assert [s for s in ss if s >= 0] == kc["commit_slots"]
-            assert [-(s + 1) for s in ss if s < 0] == kc["rollback_slots"]
-            assert int(got["freed_pages"][i]) == len(kc["freed_pages"])
+        if v and clear[: min(a + 1, v)].all():
+            assert a_own == a
             if r["m"] is not None and strict_planted:
                 assert a == r["m"]
-            em = sum(st[j]["entropy"] for j in range(a + 1)) / (a + 1)
-            assert abs(float(got["entropy_mean"][i]) - em) < 2e-2 * max(em, 1.0)
-        if (gaps[v:] >= MARGIN_FLAG).all():
-            assert got["next_draft"][tb0:tb0 + b].tolist() == ref["next_draft"]
-        np.testing.assert_allclose(got["p1"][t0:t0 + n], [s["p1"] for s in st], rtol=0.1, atol=1e-5)
-        np.testing.assert_allclose(got["entropy"][t0:t0 + n], [s["entropy"] for s in st], rtol=2e-2, atol=1e-3)
+        if clear[v:].all():
+            assert own["next_draft"] == ref["next_draft"]
         t0 += n
         tv0 += v
         tb0 += b
@@ -191,5 +203,6 @@ def test_llama8b_shape_one_layer_round():
         ctx.recg_kv_write(pool, desc.n_pages, 0, desc.page_table[i], 0, K.cuda(), V.cuda())
         y = synth.token_ids(v[i], shape.vocab, seed=400 + i).tolist()
         reqs.append({"kv": [(f64(K), f64(V))], "y": y, "L": L[i], "v": v[i], "b": b[i], "m": None})
-    flagged, _ = check_round(ctx, shape, ocfg, W64, reqs, desc, pool)
+    flagged, _ = check_round(ctx, shape, ocfg, W64, reqs, desc, pool, adaptive_flag=True)
+    assert flagged < 0.5 * desc.n_tokens      # how many rows the flag excused; not a correctness criterion
     ctx.recg_free()
