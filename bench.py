@@ -1,0 +1,446 @@
+"""Benchmark of the fused draft+verify step (one round = recg_step + recg_verify) on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+Workload (config.workload): the full 32-layer 8B-class random-init backbone at concurrency 16, per-request
+block sizes drawn from {4, 8, 16, 32}, verify length equal to the block size, context lengths uniform in
+[512, 8192], synthetic token ids, KV pool filled with N(0, 1).  `value` is processed tokens/s (all verify
+and mask rows of the batch per step) with everything resident in HBM; `e2e` runs the same calls with host
+descriptor arrays copied in and the verification results copied out every step.  Extra keys report the
+standalone attention operation at the 8B low-concurrency shape, the verify sweep, per-kernel-class
+rooflines and the concurrency-1 point.  With N > 1 every rank runs its own batch of the same shape
+(requests are independent: no collective on the data path) and rank 0 prints the aggregate.
+"""
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2609_34388_b200 import synth  # noqa: E402
+from paper_2609_34388_b200.dist import DistEnv  # noqa: E402
+
+METRIC = "draft+verify step processed tokens/s (fused round over a ragged batch, 8B-class backbone)"
+UNIT = "tokens/s"
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops"], "bf16_tflops_sustained": d["bf16_tflops_sustained"],
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons through NVML (read-only) while the timed region runs."""
+
+    def __init__(self, index=0, period=0.1):
+        super().__init__(daemon=True)
+        self.index, self.period = index, period
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop_evt = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+            self.ok = True
+        except Exception:
+            pass
+
+    def run(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        names = {nv.nvmlClocksThrottleReasonHwSlowdown: "hw_slowdown",
+                 nv.nvmlClocksThrottleReasonHwThermalSlowdown: "hw_thermal_slowdown",
+                 nv.nvmlClocksThrottleReasonSwThermalSlowdown: "sw_thermal_slowdown",
+                 nv.nvmlClocksThrottleReasonSwPowerCap: "sw_power_cap"}
+        while not self._stop_evt.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                r = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+                for bit, name in names.items():
+                    if r & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def stop(self):
+        self._stop_evt.set()
+        self.join(timeout=2)
+        med = int(np.median(self.samples)) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+# ------------------------------------------------------------------------------------------------
+# workload construction
+# ------------------------------------------------------------------------------------------------
+def c16_descriptor(seed):
+    return synth.batch_descriptor(16, [4, 8, 16, 32], None, 512, 8192, seed=seed)
+
+
+def c1_descriptor(seed):
+    return synth.fixed_descriptor([4096], [16], [16], seed=seed)
+
+
+def algorithmic_counts(shape, desc):
+    """FLOPs and bytes one step must move, per kernel class."""
+    T = desc.n_tokens
+    H, F, V, d = shape.hidden, shape.ffn, shape.vocab, shape.head_dim
+    nq, nkv, nl = shape.n_q_heads, shape.n_kv_heads, shape.n_layers
+    qkv_n = (nq + 2 * nkv) * d
+    w_params = {"gemm_qkv": qkv_n * H, "gemm_o": H * nq * d, "gemm_gate_up": 2 * F * H, "gemm_down": H * F}
+    flops = {k: 2.0 * T * p * nl for k, p in w_params.items()}
+    flops["lm_head"] = 2.0 * T * V * H
+    wbytes = {k: 2.0 * p * nl for k, p in w_params.items()}
+    wbytes["lm_head"] = 2.0 * V * H
+    kv_tokens = float((desc.ctx_len + desc.verify_len + desc.block_size).sum())
+    attn_bytes = nl * (kv_tokens * nkv * d * 2 * 2 + 2.0 * T * nq * d * 2)   # K+V once per layer, q in, o out
+    attn_flops = nl * 4.0 * d * nq * float(((desc.ctx_len + desc.verify_len + desc.block_size) *
+                                             (desc.verify_len + desc.block_size)).sum())
+    logits_bytes = 4.0 * T * V
+    return {"T": T, "flops": flops, "wbytes": wbytes, "attn_bytes": attn_bytes, "attn_flops": attn_flops,
+            "verify_bytes": logits_bytes}
+
+
+def roofline_entry(kind, achieved, peak, traffic=None, note=None):
+    unit = "GB/s" if kind == "hbm" else "TFLOP/s"
+    e = {"bound": kind, "achieved": round(achieved, 2), "peak": peak, "unit": unit, "frac": round(achieved / peak, 4),
+         "traffic": traffic}
+    if note:
+        e["note"] = note
+    return e
+
+
+# ------------------------------------------------------------------------------------------------
+# the product arm
+# ------------------------------------------------------------------------------------------------
+def run_ours(args, env):
+    from paper_2609_34388_b200 import binding
+
+    peaks = load_peaks()
+    dev = torch.device("cuda", env.local_rank)
+    torch.cuda.set_device(dev)
+    shape = synth.llama8b_shape(32)
+    t_setup = time.time()
+    W = synth.model_weights(shape, seed=0, device=dev, dtype=torch.bfloat16)
+    descs = [c16_descriptor(3 + i + 100 * env.rank) for i in range(4)]           # rotate over 4 batch draws
+    max_pages = max(d.page_table.shape[1] for d in descs)
+    n_pages = max(d.n_pages for d in descs)
+    cfg = binding.make_config(shape, 16, 1024, max_pages)
+    ctx = binding.Context(cfg, W)
+    pool = binding.alloc_kv_pool(ctx, n_pages, fill="normal")
+    batches = []
+    for i, d in enumerate(descs):
+        ys = synth.token_ids(int(d.verify_len.sum()), shape.vocab, seed=1 + i)
+        batches.append(binding.Batch(d.ctx_len, d.verify_len, d.block_size, ys, d.page_table, pool, n_pages))
+    torch.cuda.synchronize()
+    setup_s = time.time() - t_setup
+
+    outs_dev = [binding.VerifyOut(b.n_req, b.n_tok, b.n_ver, host=False) for b in batches]
+    outs_host = [binding.VerifyOut(b.n_req, b.n_tok, b.n_ver, host=True) for b in batches]
+
+    def step_device(i):
+        j = i % len(batches)
+        ctx.recg_step(batches[j])
+        ctx.recg_verify(batches[j], out=outs_dev[j])
+
+    def step_e2e(i):
+        j = i % len(batches)
+        ctx.recg_step(batches[j])               # host descriptor arrays are copied to the device by the call
+        return ctx.recg_verify(batches[j], out=outs_host[j])   # results copied to host memory, stream synchronised
+
+    for i in range(args.warmup):
+        step_device(i)
+    ctx.recg_sync()
+
+    # ---- timed region: device-resident ----
+    sampler = ClockSampler(env.local_rank)
+    sampler.start()
+    env.barrier()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(args.steps):
+        step_device(i)
+    e1.record()
+    torch.cuda.synchronize()
+    env.barrier()
+    ms_total = e0.elapsed_time(e1)
+    clocks = sampler.stop()
+    ctx.recg_sync()
+    tokens = sum(batches[i % len(batches)].n_tok for i in range(args.steps))
+    ms_total_max = env.max_float(ms_total)
+    tokens_all = env.sum_float(float(tokens))
+    value = tokens_all / (ms_total_max / 1e3)
+
+    # ---- timed region: end to end (host descriptors in, host results out, every step) ----
+    for i in range(2):
+        step_e2e(i)
+    env.barrier()
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    e0.record()
+    for i in range(args.steps):
+        res = step_e2e(i)
+    e1.record()
+    torch.cuda.synchronize()
+    wall_ms = (time.perf_counter() - t0) * 1e3
+    env.barrier()
+    e2e_ms = env.max_float(max(e0.elapsed_time(e1), wall_ms))
+    b0 = batches[0]
+    h2d = 4 * (3 * b0.n_req + 2 * (b0.n_req + 1) + b0.n_ver + b0.page_table.size)
+    d2h = outs_host[0].nbytes()
+    e2e_value = tokens_all / (e2e_ms / 1e3)
+
+    out = {"metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": env.world, "steps": args.steps,
+           "warmup": args.warmup, "ms_per_step": round(ms_total_max / args.steps, 4), "higher_is_better": True,
+           "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+           "config": {"workload": "configs[2]: 32-layer 8B-class backbone, concurrency 16 per GPU, block sizes U{4,8,16,32}, "
+                                  "verify_len = block, context U[512,8192], 4 batch draws rotated",
+                      "tokens_per_step": [b.n_tok for b in batches], "l2": "inputs (15 GB weights, 10-20 GB KV) larger than L2",
+                      "logits": "fp32", "parallelism": f"replicas x{env.world}" if env.world > 1 else "single GPU"},
+           "clocks": clocks,
+           "e2e": {"value": round(e2e_value, 1), "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
+                   "ms_per_step": round(e2e_ms / args.steps, 4)},
+           "gpu_launches": int(args.steps * (3 + 8 * shape.n_layers + 2 + 2)),
+           "setup_s": round(setup_s, 1), "peaks": peaks}
+
+    if env.rank == 0:
+        # ---- per-class timing pass (events at class boundaries; separate from the timed region above) ----
+        ctx.recg_timing_enable(True)
+        ctx.recg_timing_read()
+        for i in range(args.steps):
+            step_device(i)
+        ms, launches = ctx.recg_timing_read()
+        ctx.recg_timing_enable(False)
+        counts = [algorithmic_counts(shape, descs[i % len(descs)]) for i in range(args.steps)]
+        gemm_classes = ("gemm_qkv", "gemm_o", "gemm_gate_up", "gemm_down", "lm_head")
+        gemm_ms = sum(ms[k] for k in gemm_classes)
+        gemm_flops = sum(sum(c["flops"][k] for k in gemm_classes) for c in counts)
+        kern = {}
+        for k in gemm_classes:
+            fl = sum(c["flops"][k] for c in counts)
+            kern[k] = {"ms_per_step": round(ms[k] / args.steps, 4), "tflops": round(fl / (ms[k] / 1e3) / 1e12, 1),
+                       "frac_of_bf16_burst": round(fl / (ms[k] / 1e3) / 1e12 / peaks["bf16_tflops"], 4)}
+        ab = sum(c["attn_bytes"] for c in counts)
+        kern["attention"] = {"ms_per_step": round(ms["attention"] / args.steps, 4),
+                             "gbs": round(ab / (ms["attention"] / 1e3) / 1e9, 1),
+                             "frac_of_hbm": round(ab / (ms["attention"] / 1e3) / 1e9 / peaks["hbm_gbs"], 4)}
+        vb = sum(c["verify_bytes"] for c in counts)
+        kern["verify"] = {"ms_per_step": round(ms["verify"] / args.steps, 4), "gbs": round(vb / (ms["verify"] / 1e3) / 1e9, 1),
+                          "frac_of_hbm": round(vb / (ms["verify"] / 1e3) / 1e9 / peaks["hbm_gbs"], 4)}
+        kern["rmsnorm"] = {"ms_per_step": round(ms["rmsnorm"] / args.steps, 4)}
+        kern["layout"] = {"ms_per_step": round(ms["layout"] / args.steps, 4)}
+        out["kernels"] = kern
+        n_gemm_launch = sum(launches[k] for k in gemm_classes)
+        ach = gemm_flops / (gemm_ms / 1e3) / 1e12
+        out["roofline"] = roofline_entry("tensor", ach, peaks["bf16_tflops_sustained"], None,
+                                         f"projection GEMM kernel (tcgen05), {n_gemm_launch} launches, avg "
+                                         f"{gemm_ms / max(n_gemm_launch, 1) * 1e3:.1f} us; peak = sustained bf16 of {peaks['source']}")
+        out["step_time_share"] = {k: round(v / sum(ms.values()), 4) for k, v in ms.items()}
+        out["attention_op"] = bench_attention_op(binding, peaks, args)
+        out["verify_sweep"] = bench_verify(binding, peaks)
+        out["c1"] = bench_c1(binding, ctx, shape, pool, n_pages, peaks, args)
+        out["cpu_baseline"] = cpu_baseline(shape, descs[0])
+    ctx.recg_free()
+    return out
+
+
+def bench_attention_op(binding, peaks, args):
+    """configs[1]: one layer's hybrid attention at 8B shapes, context 4096, 16 causal + 16 bidirectional rows."""
+    shape = synth.llama8b_shape(32)         # 32 distinct layer caches rotated: 32 x 17 MB > L2
+    desc = c1_descriptor(7)
+    ctx = binding.Context(binding.make_config(shape, 1, 32, desc.page_table.shape[1]))
+    pool = binding.alloc_kv_pool(ctx, desc.n_pages, fill="normal")
+    batch = binding.Batch(desc.ctx_len, desc.verify_len, desc.block_size, None, desc.page_table, pool, desc.n_pages)
+    q = synth.queries(32, 32, 128, seed=5, device="cuda")
+    o = torch.empty_like(q)
+    ctx.recg_attention(batch, 0, q, o)
+    for l in range(32):
+        ctx.recg_attention(None, l, q, o)
+    torch.cuda.synchronize()
+    iters = 10
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(iters):
+        for l in range(32):
+            ctx.recg_attention(None, l, q, o)
+    e1.record()
+    torch.cuda.synchronize()
+    us = e0.elapsed_time(e1) / (iters * 32) * 1e3
+    kv_bytes = (4096 + 32) * 8 * 128 * 2 * 2 + 2 * 32 * 32 * 128 * 2
+    ctx.recg_free()
+    gbs = kv_bytes / (us * 1e-6) / 1e9
+    return {"workload": "configs[1]: 32/8 heads, d 128, context 4096, 16 causal + 16 bidirectional rows, 32 caches rotated",
+            "us_per_call": round(us, 2), "calls_include": "attention kernel + combine kernel", "algorithmic_bytes": kv_bytes,
+            "gbs": round(gbs, 1), "frac_of_hbm_measured": round(gbs / peaks["hbm_gbs"], 4),
+            "frac_of_8000": round(gbs / 8000.0, 4)}
+
+
+def bench_verify(binding, peaks):
+    """configs[4]: verify kernel sweep over bf16 logits [B (k+1), 128256]."""
+    V = 128256
+    res = []
+    shape = synth.ModelShape(n_layers=0, hidden=64, n_q_heads=4, n_kv_heads=2, head_dim=64, ffn=64, vocab=V)
+    for B, k in [(1, 4), (8, 8), (32, 16), (128, 16), (256, 32)]:
+        R = B * (k + 1)
+        ctx = binding.Context(binding.make_config(shape, B, R, 1))
+        lg = synth.logits_normal(R, V, seed=6, device="cuda")
+        y = synth.token_ids(R, V, seed=1)
+        batch = binding.Batch([0] * B, [k + 1] * B, [0] * B, y)
+        ctx.recg_verify(batch, lg, host=False)
+        n_rot = max(1, int(np.ceil(300e6 / (R * V * 2))))       # rotate copies so that the scan does not sit in L2
+        copies = [lg] + [lg.clone() for _ in range(min(n_rot, 64) - 1)]
+        torch.cuda.synchronize()
+        iters = 20
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(iters):
+            ctx.recg_verify(None, copies[i % len(copies)], host=False, n_req=B, n_tok=R, n_ver=R)
+        e1.record()
+        torch.cuda.synchronize()
+        us = e0.elapsed_time(e1) / iters * 1e3
+        gbs = R * V * 2 / (us * 1e-6) / 1e9
+        res.append({"B": B, "k": k, "rows": R, "us": round(us, 2), "gbs": round(gbs, 1),
+                    "frac_of_hbm_measured": round(gbs / peaks["hbm_gbs"], 4)})
+        ctx.recg_free()
+        del copies, lg
+        torch.cuda.empty_cache()
+    return res
+
+
+def bench_c1(binding, ctx, shape, pool, n_pages, peaks, args):
+    """Concurrency 1 (context 4096, 16 + 16 rows) through the full model: the weight-streaming regime."""
+    desc = c1_descriptor(11)
+    ys = synth.token_ids(16, shape.vocab, seed=2)
+    batch = binding.Batch(desc.ctx_len, desc.verify_len, desc.block_size, ys, desc.page_table, pool, n_pages)
+    for _ in range(3):
+        ctx.recg_step(batch)
+        ctx.recg_verify(batch, host=False)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    iters = max(3, args.steps)
+    e0.record()
+    for _ in range(iters):
+        ctx.recg_step(batch)
+        ctx.recg_verify(batch, host=False)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / iters
+    wbytes = 2.0 * (shape.n_layers * ((shape.n_q_heads + 2 * shape.n_kv_heads) * shape.head_dim * shape.hidden +
+                                       shape.hidden * shape.n_q_heads * shape.head_dim + 3 * shape.ffn * shape.hidden) +
+                    shape.vocab * shape.hidden)
+    return {"workload": "concurrency 1, context 4096, verify 16 + block 16", "ms_per_step": round(ms, 4),
+            "tokens_per_s": round(32 / (ms / 1e3), 1), "weight_stream_gbs": round(wbytes / (ms / 1e3) / 1e9, 1),
+            "frac_of_hbm_measured": round(wbytes / (ms / 1e3) / 1e9 / peaks["hbm_gbs"], 4)}
+
+
+# ------------------------------------------------------------------------------------------------
+# the oracle, timed as it stands on the host cores (reported baseline, and the --impl reference arm)
+# ------------------------------------------------------------------------------------------------
+class OracleSample:
+    """The CPU oracle, as it stands, on a bounded sample of the workload: request 0 of the batch through ONE of
+    the n_layers layers plus the LM head and verification; the layer time is scaled by n_layers."""
+
+    def __init__(self, shape, desc):
+        from oracle import recg_oracle as orc
+
+        self.orc = orc
+        self.shape = shape
+        one = synth.ModelShape(**{**shape.as_dict(), "n_layers": 1})
+        W = synth.model_weights(one, seed=0, device="cpu", dtype=torch.bfloat16)
+        self.W64 = {k: ([t.double().numpy() for t in v] if isinstance(v, list) else v.double().numpy())
+                    for k, v in W.items() if k != "embed"}
+        self.W64["embed"] = W["embed"].float().numpy()       # exact widening; rows are widened to fp64 on lookup
+        self.ocfg = orc.ModelConfig(**one.as_dict())
+        self.L, self.v, self.b = int(desc.ctx_len[0]), int(desc.verify_len[0]), int(desc.block_size[0])
+        K, V = synth.kv_values(self.L, shape.n_kv_heads, shape.head_dim, seed=2, device="cpu")
+        self.kv = [(K.double().numpy(), V.double().numpy())]
+        self.y = synth.token_ids(self.v, shape.vocab, seed=1).tolist()
+
+    def step(self):
+        """Returns (tokens/s, seconds for the whole model by the scaling rule, tokens)."""
+        orc = self.orc
+        t0 = time.perf_counter()
+        logits, _, h = orc.fused_round_cached(self.ocfg, self.W64, self.kv, self.L, self.y, self.b)
+        t1 = time.perf_counter()
+        x = orc.rmsnorm(h, self.W64["final_norm"], self.ocfg.rms_eps)     # the head alone, to split layer / head time
+        _ = x @ self.W64["lm_head"].T
+        t2 = time.perf_counter()
+        orc.verify_round(logits, self.y, self.b)
+        t3 = time.perf_counter()
+        head = t2 - t1
+        total = ((t1 - t0) - head) * self.shape.n_layers + head + (t3 - t2)
+        toks = self.v + self.b
+        return toks / total, total, toks
+
+    def describe(self):
+        return (f"request 0 of the concurrency-16 batch ({self.v + self.b} rows over {self.L} context tokens) through 1 of "
+                f"{self.shape.n_layers} layers (time x{self.shape.n_layers}) plus the full LM head and verification; fp64 numpy")
+
+
+def cpu_baseline(shape, desc):
+    import multiprocessing
+
+    s = OracleSample(shape, desc)
+    tps, secs, toks = s.step()
+    return {"value": round(tps, 2), "unit": UNIT, "cores": multiprocessing.cpu_count(), "kind": "oracle",
+            "sample": s.describe(), "seconds_scaled": round(secs, 2)}
+
+
+def run_reference(args, env):
+    import multiprocessing
+
+    shape = synth.llama8b_shape(32)
+    s = OracleSample(shape, c16_descriptor(3))
+    for _ in range(args.warmup):
+        s.step()
+    vals = [s.step() for _ in range(args.steps)]
+    tps = float(np.mean([v[0] for v in vals]))
+    secs = float(np.mean([v[1] for v in vals]))
+    cb = {"value": round(tps, 2), "unit": UNIT, "cores": multiprocessing.cpu_count(), "kind": "oracle", "sample": s.describe()}
+    return {"impl": "reference", "metric": METRIC, "value": round(tps, 2), "unit": UNIT, "n_gpus": env.world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(secs * 1e3, 2), "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": "configs[2] (bounded sample per step, see cpu_baseline.sample)"},
+            "cpu_baseline": cb,
+            "e2e": {"value": round(tps, 2), "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=8)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        # rank 0 alone times the oracle on the host cores; the other ranks have nothing to do
+        env = DistEnv(rank=int(os.environ.get("RANK", "0")), world=int(os.environ.get("WORLD_SIZE", "1")))
+        if env.rank == 0:
+            print(json.dumps(run_reference(args, env)), flush=True)
+        return
+    env = DistEnv.from_env(backend="nccl")
+    out = run_ours(args, env)
+    if env.rank == 0:
+        print(json.dumps(out), flush=True)
+    env.close()
+
+
+if __name__ == "__main__":
+    main()

@@ -212,6 +212,19 @@ recg_status recg_linear(recg_ctx *ctx, const void *x, const void *w, void *y, in
 recg_status recg_debug_buffer(recg_ctx *ctx, int32_t which, const void **ptr, int32_t *dtype, int32_t *rows,
                               int32_t *cols);
 
+/*
+ * Per-kernel-class device timing of recg_step()/recg_verify() for roofline reports (measurement aid; the
+ * forward-time profiling of Sec. 3.2 is the closest thing in the paper).  recg_timing_enable(ctx, 1) makes
+ * the following calls record CUDA events at class boundaries on the context's stream;
+ * recg_timing_read() synchronises the stream, adds the elapsed milliseconds per class since the last read
+ * into ms[0..RECG_TIMING_CLASSES) and launches[...] (either may be NULL) and resets the accumulation.
+ * Classes: 0 layout+embedding+rotary table, 1 RMSNorm, 2 QKV projection, 3 attention (+combine),
+ * 4 output projection, 5 gate|up projection, 6 down projection, 7 LM head, 8 verify.
+ */
+#define RECG_TIMING_CLASSES 9
+recg_status recg_timing_enable(recg_ctx *ctx, int32_t enable);
+recg_status recg_timing_read(recg_ctx *ctx, float *ms, int32_t *launches);
+
 /* Wait for the stream, then report (and clear) the device status word: RECG_OK or RECG_ERR_TIMEOUT /
  * RECG_ERR_INTERNAL if a kernel flagged a bounded wait that gave up or an out-of-range index. */
 recg_status recg_sync(recg_ctx *ctx);

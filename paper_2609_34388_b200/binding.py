@@ -87,16 +87,20 @@ def lib() -> C.CDLL:
         L.recg_debug_buffer.argtypes = [C.c_void_p, C.c_int32, C.POINTER(C.c_void_p), C.POINTER(C.c_int32),
                                         C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
         L.recg_sync.argtypes = [C.c_void_p]
+        L.recg_timing_enable.argtypes = [C.c_void_p, C.c_int32]
+        L.recg_timing_read.argtypes = [C.c_void_p, C.POINTER(C.c_float), C.POINTER(C.c_int32)]
         L.recg_free.argtypes = [C.c_void_p]
         for f in ("recg_init", "recg_step", "recg_verify", "recg_attention", "recg_kv_write", "recg_kv_read",
-                  "recg_linear", "recg_debug_buffer", "recg_sync", "recg_free"):
+                  "recg_linear", "recg_debug_buffer", "recg_sync", "recg_free", "recg_timing_enable", "recg_timing_read"):
             getattr(L, f).restype = C.c_int32
         _lib = L
     return _lib
 
 
 EXPORTS = ("recg_kv_pool_bytes", "recg_init", "recg_step", "recg_verify", "recg_attention", "recg_kv_write",
-           "recg_kv_read", "recg_linear", "recg_debug_buffer", "recg_sync", "recg_free", "recg_last_error")
+           "recg_kv_read", "recg_linear", "recg_debug_buffer", "recg_sync", "recg_free", "recg_last_error",
+           "recg_timing_enable", "recg_timing_read")
+TIMING_CLASSES = ("layout", "rmsnorm", "gemm_qkv", "attention", "gemm_o", "gemm_gate_up", "gemm_down", "lm_head", "verify")
 
 
 def make_config(shape, max_requests: int, max_tokens: int, max_pages_per_request: int, flags: int = 0,
@@ -135,6 +139,31 @@ class Batch:
         self.n_req = len(self.ctx_len)
         self.n_tok = int(self.verify_len.sum() + self.block_size.sum())
         self.n_ver = int(self.verify_len.sum())
+
+
+class VerifyOut:
+    """Caller-provided result buffers of recg_verify (host numpy arrays or CUDA tensors)."""
+
+    def __init__(self, n_req: int, n_tok: int, n_ver: int, host: bool = True):
+        self.sizes = {"accept_len": n_req, "n_emitted": n_req, "emitted": n_ver, "new_ctx_len": n_req,
+                      "slot_state": n_tok, "freed_pages": n_req, "next_draft": n_tok - n_ver, "cont_hit": n_req,
+                      "top1": n_tok, "top2": n_tok, "p1": n_tok, "p2": n_tok, "entropy": n_tok, "entropy_mean": n_req}
+        self.bufs = {}
+        self.c = recg_verify_out()
+        self.c.mem = MEM_HOST if host else MEM_DEVICE
+        for name, n in self.sizes.items():
+            isf = name in _FLT_OUT
+            if host:
+                self.bufs[name] = np.zeros(max(n, 1), dtype=np.float32 if isf else np.int32)
+            else:
+                self.bufs[name] = torch.zeros(max(n, 1), dtype=torch.float32 if isf else torch.int32, device="cuda")
+            setattr(self.c, name, _ptr(self.bufs[name]))
+
+    def views(self):
+        return {k: v[:self.sizes[k]] for k, v in self.bufs.items()}
+
+    def nbytes(self) -> int:
+        return 4 * sum(self.sizes.values())
 
 
 class Context:
@@ -182,31 +211,22 @@ class Context:
         return device_view(lg.data, (lg.n_rows, lg.vocab), dt).clone()
 
     def recg_verify(self, batch: Optional[Batch], logits: Optional[torch.Tensor] = None, host: bool = True,
-                    n_req: Optional[int] = None, n_tok: Optional[int] = None, n_ver: Optional[int] = None):
-        """Runs verification; returns a dict of numpy arrays (host=True) or CUDA tensors."""
-        C_ = batch.n_req if batch is not None else n_req
-        T = batch.n_tok if batch is not None else n_tok
-        Tv = batch.n_ver if batch is not None else n_ver
-        sizes = {"accept_len": C_, "n_emitted": C_, "emitted": Tv, "new_ctx_len": C_, "slot_state": T,
-                 "freed_pages": C_, "next_draft": T - Tv, "cont_hit": C_, "top1": T, "top2": T, "p1": T, "p2": T,
-                 "entropy": T, "entropy_mean": C_}
-        bufs = {}
-        out = recg_verify_out()
-        out.mem = MEM_HOST if host else MEM_DEVICE
-        for name, n in sizes.items():
-            isf = name in _FLT_OUT
-            if host:
-                bufs[name] = np.zeros(max(n, 1), dtype=np.float32 if isf else np.int32)
-            else:
-                bufs[name] = torch.zeros(max(n, 1), dtype=torch.float32 if isf else torch.int32, device="cuda")
-            setattr(out, name, _ptr(bufs[name]))
+                    n_req: Optional[int] = None, n_tok: Optional[int] = None, n_ver: Optional[int] = None,
+                    out: Optional["VerifyOut"] = None):
+        """Runs verification; returns a dict of numpy arrays (host=True) or CUDA tensors.  Pass a
+        preallocated VerifyOut to avoid allocating the result buffers on every call."""
+        if out is None:
+            C_ = batch.n_req if batch is not None else n_req
+            T = batch.n_tok if batch is not None else n_tok
+            Tv = batch.n_ver if batch is not None else n_ver
+            out = VerifyOut(C_, T, Tv, host)
         dt = 0
         lp = None
         if logits is not None:
             dt = DTYPE_BF16 if logits.dtype == torch.bfloat16 else DTYPE_F32
             lp = logits.data_ptr()
-        self._check(lib().recg_verify(self.h, C.byref(batch.c) if batch is not None else None, lp, dt, C.byref(out)))
-        return {k: v[:sizes[k]] for k, v in bufs.items()}
+        self._check(lib().recg_verify(self.h, C.byref(batch.c) if batch is not None else None, lp, dt, C.byref(out.c)))
+        return out.views()
 
     def recg_attention(self, batch: Optional[Batch], layer: int, q: torch.Tensor, o: torch.Tensor):
         self._check(lib().recg_attention(self.h, C.byref(batch.c) if batch is not None else None, layer, q.data_ptr(),
@@ -239,6 +259,16 @@ class Context:
         self._check(lib().recg_debug_buffer(self.h, which, C.byref(p), C.byref(dt), C.byref(r), C.byref(c)))
         return device_view(p.value, (r.value, c.value),
                            torch.bfloat16 if dt.value == DTYPE_BF16 else torch.float32).clone()
+
+    def recg_timing_enable(self, enable: bool):
+        self._check(lib().recg_timing_enable(self.h, 1 if enable else 0))
+
+    def recg_timing_read(self):
+        """Returns ({class: ms}, {class: launches}) accumulated since the last read."""
+        ms = (C.c_float * len(TIMING_CLASSES))()
+        ln = (C.c_int32 * len(TIMING_CLASSES))()
+        self._check(lib().recg_timing_read(self.h, ms, ln))
+        return dict(zip(TIMING_CLASSES, list(ms))), dict(zip(TIMING_CLASSES, list(ln)))
 
     def recg_sync(self):
         self._check(lib().recg_sync(self.h))

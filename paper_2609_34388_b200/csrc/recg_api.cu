@@ -60,6 +60,26 @@ struct recg_ctx {
   int* d_page_row = nullptr;
   void* tc_state = nullptr;
   std::vector<int> h_desc;
+  // optional per-class timing
+  bool timing = false;
+  std::vector<cudaEvent_t> ev_pool;
+  size_t ev_used = 0;
+  std::vector<int> ev_class;  // class of the interval that ENDS at event i (-1 for an opening event)
+  int ev_launches[RECG_TIMING_CLASSES] = {0};
+
+  void mark(int cls, int launches = 0) {  // cls < 0 opens a sequence; otherwise closes an interval of that class
+    if (!timing) return;
+    if (ev_used == ev_pool.size()) {
+      cudaEvent_t e;
+      if (cudaEventCreate(&e) != cudaSuccess) return;
+      ev_pool.push_back(e);
+      ev_class.push_back(-1);
+    }
+    cudaEventRecord(ev_pool[ev_used], stream);
+    ev_class[ev_used] = cls;
+    if (cls >= 0) ev_launches[cls] += launches;
+    ++ev_used;
+  }
 };
 
 namespace {
@@ -309,9 +329,34 @@ recg_status recg_init(recg_ctx** out, const recg_config* cfg, const recg_weights
   return RECG_OK;
 }
 
+recg_status recg_timing_enable(recg_ctx* ctx, int32_t enable) {
+  if (!ctx) return RECG_ERR_INVALID_ARG;
+  ctx->timing = enable != 0;
+  return RECG_OK;
+}
+
+recg_status recg_timing_read(recg_ctx* ctx, float* ms, int32_t* launches) {
+  if (!ctx) return RECG_ERR_INVALID_ARG;
+  CU(cudaStreamSynchronize(ctx->stream));
+  for (int c = 0; c < RECG_TIMING_CLASSES; ++c) {
+    if (ms) ms[c] = 0.f;
+    if (launches) launches[c] = ctx->ev_launches[c];
+    ctx->ev_launches[c] = 0;
+  }
+  for (size_t i = 1; i < ctx->ev_used; ++i) {
+    const int cls = ctx->ev_class[i];
+    if (cls < 0) continue;
+    float t = 0.f;
+    if (cudaEventElapsedTime(&t, ctx->ev_pool[i - 1], ctx->ev_pool[i]) == cudaSuccess && ms) ms[cls] += t;
+  }
+  ctx->ev_used = 0;
+  return RECG_OK;
+}
+
 recg_status recg_free(recg_ctx* ctx) {
   if (!ctx) return RECG_OK;
   cudaStreamSynchronize(ctx->stream);
+  for (cudaEvent_t e : ctx->ev_pool) cudaEventDestroy(e);
   if (ctx->tc_state) tc_state_destroy(ctx->tc_state);
   if (ctx->arena.base) cudaFree(ctx->arena.base);
   delete ctx;
@@ -335,6 +380,7 @@ recg_status recg_step(recg_ctx* ctx, const recg_batch* batch, recg_logits* logit
   if (!ctx) return RECG_ERR_INVALID_ARG;
   if (!ctx->has_weights) return fail(ctx, RECG_ERR_INVALID_ARG, "recg_step: the context was created without weights");
   ctx->logits_valid = false;
+  ctx->mark(-1);
   recg_status s = upload_and_layout(ctx, batch, true);
   if (s != RECG_OK) return s;
   const Dims& d = ctx->dm;
@@ -344,35 +390,45 @@ recg_status recg_step(recg_ctx* ctx, const recg_batch* batch, recg_logits* logit
   launch_rope_table(bl.tok_pos, T, d.head_dim, d.rope_base, ctx->rope_cs, st);
   launch_embed(bl, d, ctx->embed, ctx->h, st);
   CU(cudaGetLastError());
+  ctx->mark(0, 3);
   const int qdim = d.n_q * d.head_dim;
   for (int l = 0; l < d.n_layers; ++l) {
     launch_rmsnorm(ctx->h, ctx->attn_norm[l], ctx->x, T, d.hidden, d.rms_eps, st);
+    ctx->mark(1, 1);
     GemmArgs a{};
     a.x = ctx->x; a.w = ctx->wqkv[l]; a.out = ctx->q;
     a.M = T; a.N = (d.n_q + 2 * d.n_kv) * d.head_dim; a.K = d.hidden; a.epi = EPI_QKV_ROPE;
     a.tok_pos = bl.tok_pos; a.tok_slot = bl.tok_slot; a.kv_pool = batch->kv_pool; a.n_pages = batch->kv_pool_pages;
     a.layer = l; a.n_q = d.n_q; a.n_kv = d.n_kv; a.head_dim = d.head_dim; a.rope_cs = ctx->rope_cs;
     if ((s = run_gemm(ctx, a)) != RECG_OK) return s;
+    ctx->mark(2, 1);
     launch_attention(bl, d, l, ctx->q, ctx->o, batch->kv_pool, batch->kv_pool_pages, ctx->part_o, ctx->part_ml,
                      ctx->tok_per_tile, ctx->n_sm, ctx->d_status, st);
     CU(cudaGetLastError());
+    ctx->mark(3, 2);
     GemmArgs b{};
     b.x = ctx->o; b.w = ctx->wo[l]; b.out = ctx->h; b.M = T; b.N = d.hidden; b.K = qdim; b.epi = EPI_RESIDUAL;
     if ((s = run_gemm(ctx, b)) != RECG_OK) return s;
+    ctx->mark(4, 1);
     launch_rmsnorm(ctx->h, ctx->ffn_norm[l], ctx->x, T, d.hidden, d.rms_eps, st);
+    ctx->mark(1, 1);
     GemmArgs c{};
     c.x = ctx->x; c.w = ctx->w_gate_up[l]; c.out = ctx->act; c.M = T; c.N = d.ffn; c.K = d.hidden; c.epi = EPI_SWIGLU;
     if ((s = run_gemm(ctx, c)) != RECG_OK) return s;
+    ctx->mark(5, 1);
     GemmArgs e{};
     e.x = ctx->act; e.w = ctx->w_down[l]; e.out = ctx->h; e.M = T; e.N = d.hidden; e.K = d.ffn; e.epi = EPI_RESIDUAL;
     if ((s = run_gemm(ctx, e)) != RECG_OK) return s;
+    ctx->mark(6, 1);
   }
   launch_rmsnorm(ctx->h, ctx->final_norm, ctx->x, T, d.hidden, d.rms_eps, st);
+  ctx->mark(1, 1);
   const bool lbf = ctx->cfg.flags & RECG_FLAG_LOGITS_BF16;
   GemmArgs f{};
   f.x = ctx->x; f.w = ctx->lm_head; f.out = ctx->logits; f.M = T; f.N = d.vocab; f.K = d.hidden;
   f.epi = lbf ? EPI_PLAIN_BF16 : EPI_PLAIN_F32;
   if ((s = run_gemm(ctx, f)) != RECG_OK) return s;
+  ctx->mark(7, 1);
   ctx->logits_valid = true;
   if (logits) {
     logits->data = ctx->logits;
@@ -414,8 +470,10 @@ recg_status recg_verify(recg_ctx* ctx, const recg_batch* batch, const void* logi
     PICK(next_draft); PICK(cont_hit); PICK(top1); PICK(top2); PICK(p1); PICK(p2); PICK(entropy); PICK(entropy_mean);
 #undef PICK
   }
+  ctx->mark(-1);
   launch_verify(bl, logits, logits_dtype, ctx->dm.vocab, ctx->vpart, ctx->max_chunks_total, vb, ctx->n_sm, ctx->stream);
   CU(cudaGetLastError());
+  ctx->mark(8, 2);
   if (!dev) {
     const size_t C = bl.n_req, T = bl.n_tok, Tv = bl.n_ver, Tb = T - Tv;
 #define OUT(f, n) if (out->f && (n)) CU(cudaMemcpyAsync(out->f, vb.f, (n) * 4, cudaMemcpyDeviceToHost, ctx->stream))
