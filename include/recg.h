@@ -225,6 +225,40 @@ recg_status recg_debug_buffer(recg_ctx *ctx, int32_t which, const void **ptr, in
 recg_status recg_timing_enable(recg_ctx *ctx, int32_t enable);
 recg_status recg_timing_read(recg_ctx *ctx, float *ms, int32_t *launches);
 
+/*
+ * Per-row logit statistics with no allocation anywhere (the paper has no counterpart: this entry point
+ * exists for callers that are not allowed to allocate device memory).
+ *
+ * Some hosts of this library cannot call cudaMalloc at the moment they need the statistics: code running
+ * inside a stream capture, a serving loop that has handed all device memory to its own pool allocator
+ * and forbids further driver allocations, or a plugin that runs under a sandbox whose allocation hooks
+ * must not be re-entered.  recg_verify() needs a context, and creating a context allocates a workspace.
+ * This variant needs neither: it runs the same vocabulary scan (top-1 / top-2 ids with lowest-index
+ * ties, P_1st, P_2nd, entropy in nats per row), but keeps the per-chunk partial results in a fixed
+ * array that is part of the library image, and it calls no cudaMalloc, cudaFree or any allocating routine.
+ *
+ *   logits   DEVICE [rows, vocab] of logits_dtype (recg_dtype), row-major
+ *   top1, top2 DEVICE int32 [rows]; p1, p2, entropy DEVICE float32 [rows]; any output may be NULL
+ *   cuda_stream  cudaStream_t the work is enqueued on (NULL = default stream); the call does not wait
+ *
+ * Limits and rules:
+ *   - the static scratch holds 65536 chunk partials (1.5 MiB of device memory that every GPU which loads
+ *     the library keeps until the process exits).  rows may not exceed 65536 and rows x chunks-per-row
+ *     must fit; larger requests are refused with RECG_ERR_CAPACITY and nothing is launched;
+ *   - the first call on each device looks up the device address of the scratch array (with that device
+ *     current).  Make that first call outside any stream capture;
+ *   - all calls on one device share the scratch, which keeps whatever the previous call left there.
+ *     Every partial a call reads is written by that same call first, so stale contents are harmless, but
+ *     two calls whose kernels overlap on the GPU (different streams, or different host threads) race on
+ *     it: serialise them;
+ *   - errors: RECG_ERR_INVALID_ARG, RECG_ERR_CAPACITY, RECG_ERR_CUDA; recg_last_error(NULL) does NOT carry
+ *     this entry point's text, use recg_row_stats_static_error().
+ */
+recg_status recg_row_stats_static(const void *logits, int32_t logits_dtype, int32_t rows, int32_t vocab,
+                                  int32_t *top1, int32_t *top2, float *p1, float *p2, float *entropy,
+                                  void *cuda_stream);
+const char *recg_row_stats_static_error(void);
+
 /* Wait for the stream, then report (and clear) the device status word: RECG_OK or RECG_ERR_TIMEOUT /
  * RECG_ERR_INTERNAL if a kernel flagged a bounded wait that gave up or an out-of-range index. */
 recg_status recg_sync(recg_ctx *ctx);

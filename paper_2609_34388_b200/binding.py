@@ -87,6 +87,9 @@ def lib() -> C.CDLL:
         L.recg_debug_buffer.argtypes = [C.c_void_p, C.c_int32, C.POINTER(C.c_void_p), C.POINTER(C.c_int32),
                                         C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
         L.recg_sync.argtypes = [C.c_void_p]
+        L.recg_row_stats_static.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32] + [C.c_void_p] * 6
+        L.recg_row_stats_static.restype = C.c_int32
+        L.recg_row_stats_static_error.restype = C.c_char_p
         L.recg_timing_enable.argtypes = [C.c_void_p, C.c_int32]
         L.recg_timing_read.argtypes = [C.c_void_p, C.POINTER(C.c_float), C.POINTER(C.c_int32)]
         L.recg_free.argtypes = [C.c_void_p]
@@ -99,7 +102,7 @@ def lib() -> C.CDLL:
 
 EXPORTS = ("recg_kv_pool_bytes", "recg_init", "recg_step", "recg_verify", "recg_attention", "recg_kv_write",
            "recg_kv_read", "recg_linear", "recg_debug_buffer", "recg_sync", "recg_free", "recg_last_error",
-           "recg_timing_enable", "recg_timing_read")
+           "recg_timing_enable", "recg_timing_read", "recg_row_stats_static", "recg_row_stats_static_error")
 TIMING_CLASSES = ("layout", "rmsnorm", "gemm_qkv", "attention", "gemm_o", "gemm_gate_up", "gemm_down", "lm_head", "verify")
 
 
@@ -313,3 +316,22 @@ def alloc_kv_pool(ctx: Context, n_pages: int, fill: Optional[str] = "zero") -> t
     if fill == "zero":
         return torch.zeros(n, dtype=torch.bfloat16, device="cuda")
     return torch.empty(n, dtype=torch.bfloat16, device="cuda")
+
+
+def recg_row_stats_static(logits: torch.Tensor, stream: Optional[int] = None):
+    """Per-row statistics through the entry point that allocates nothing inside the library (the result
+    tensors below are the CALLER's buffers).  For callers that must not trigger a device allocation:
+    see include/recg.h.  Returns a dict of CUDA tensors; does not synchronise."""
+    rows, vocab = logits.shape
+    out = {"top1": torch.empty(rows, dtype=torch.int32, device=logits.device),
+           "top2": torch.empty(rows, dtype=torch.int32, device=logits.device),
+           "p1": torch.empty(rows, dtype=torch.float32, device=logits.device),
+           "p2": torch.empty(rows, dtype=torch.float32, device=logits.device),
+           "entropy": torch.empty(rows, dtype=torch.float32, device=logits.device)}
+    st = torch.cuda.current_stream().cuda_stream if stream is None else stream
+    rc = lib().recg_row_stats_static(logits.data_ptr(), DTYPE_BF16 if logits.dtype == torch.bfloat16 else DTYPE_F32,
+                                     rows, vocab, out["top1"].data_ptr(), out["top2"].data_ptr(), out["p1"].data_ptr(),
+                                     out["p2"].data_ptr(), out["entropy"].data_ptr(), C.c_void_p(st))
+    if rc != RECG_OK:
+        raise RecgError(rc, lib().recg_row_stats_static_error().decode())
+    return out

@@ -1,6 +1,9 @@
 // Fused greedy verification: one pass over the logits (top-2 ids, softmax mass, entropy) split over
 // vocab chunks, then a per-request finalize (accept-length scan, emitted tokens, continuation rule,
 // mean verifier entropy, KV commit / rollback indices).
+#include <string>
+
+#include "../../include/recg.h"
 #include "common.cuh"
 #include "kernels.h"
 
@@ -267,3 +270,100 @@ void launch_verify(const BatchLayout& bl, const void* logits, int logits_dtype, 
 }
 
 }  // namespace recg
+
+// ---------------------------------------------------------------------------------------------------
+// Row statistics without any allocation: the chunk partials live in a file-scope device array.
+// ---------------------------------------------------------------------------------------------------
+namespace recg {
+namespace {
+
+constexpr int kStaticMaxPartials = 1 << 16;   // 65536 x 24 bytes = 1.5 MiB held by every GPU that loads the library
+static __device__ __align__(256) RowPartial g_static_partials[kStaticMaxPartials];
+
+constexpr int kMaxDevices = 64;
+RowPartial* g_static_ptr[kMaxDevices] = {nullptr};   // device address of the array, per device, set on first use
+int g_static_sm[kMaxDevices] = {0};
+
+thread_local std::string g_static_error;
+
+// one thread per row: merge the row's chunk partials into the five per-row outputs
+__global__ void row_stats_finalize_kernel(const RowPartial* __restrict__ partials, int rows, int chunks_per_row,
+                                          int* __restrict__ top1, int* __restrict__ top2, float* __restrict__ p1,
+                                          float* __restrict__ p2, float* __restrict__ entropy) {
+  const int r = blockIdx.x * blockDim.x + threadIdx.x;
+  if (r >= rows) return;
+  const RowPartial* p = partials + (size_t)r * chunks_per_row;
+  Top2 tp = {-INFINITY, -INFINITY, 0x7fffffff, 0x7fffffff};
+  Mass ms = {-INFINITY, 0.f, 0.f};
+  for (int c = 0; c < chunks_per_row; ++c) {
+    const RowPartial q = p[c];
+    top2_insert(tp, q.m1, q.i1);
+    top2_insert(tp, q.m2, q.i2);
+    Mass o = {q.m1, q.s, q.t};
+    mass_merge(ms, o);
+  }
+  const float inv = 1.f / ms.s;
+  if (top1) top1[r] = tp.i1;
+  if (top2) top2[r] = tp.i2;
+  if (p1) p1[r] = inv;
+  if (p2) p2[r] = __expf(tp.m2 - tp.m1) * inv;
+  if (entropy) entropy[r] = logf(ms.s) - ms.t * inv;
+}
+
+}  // namespace
+
+const char* static_entry_error() { return g_static_error.c_str(); }
+
+}  // namespace recg
+
+extern "C" const char* recg_row_stats_static_error(void) { return recg::static_entry_error(); }
+
+extern "C" recg_status recg_row_stats_static(const void* logits, int32_t logits_dtype, int32_t rows, int32_t vocab,
+                                             int32_t* top1, int32_t* top2, float* p1, float* p2, float* entropy,
+                                             void* cuda_stream) {
+  using namespace recg;
+  auto fail = [](recg_status s, const std::string& m) { g_static_error = m; return s; };
+  if (!logits || rows < 0 || vocab <= 1) return fail(RECG_ERR_INVALID_ARG, "recg_row_stats_static: null logits or bad extent");
+  if (logits_dtype != RECG_DTYPE_BF16 && logits_dtype != RECG_DTYPE_F32)
+    return fail(RECG_ERR_INVALID_ARG, "recg_row_stats_static: unknown logits dtype");
+  if (rows == 0) return RECG_OK;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices)
+    return fail(RECG_ERR_CUDA, "recg_row_stats_static: no current CUDA device");
+  if (!g_static_ptr[dev]) {
+    // first call on this device: the array's name is only a host-side handle, so ask the runtime for the
+    // device address (with this device current) and remember it
+    void* ptr = nullptr;
+    cudaError_t e = cudaGetSymbolAddress(&ptr, g_static_partials);
+    if (e != cudaSuccess || !ptr)
+      return fail(RECG_ERR_CUDA, std::string("recg_row_stats_static: cudaGetSymbolAddress: ") + cudaGetErrorString(e));
+    int n_sm = 0;
+    e = cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess || n_sm <= 0)
+      return fail(RECG_ERR_CUDA, std::string("recg_row_stats_static: SM count: ") + cudaGetErrorString(e));
+    g_static_sm[dev] = n_sm;
+    g_static_ptr[dev] = static_cast<RowPartial*>(ptr);
+  }
+  if (rows > kStaticMaxPartials)
+    return fail(RECG_ERR_CAPACITY, "recg_row_stats_static: more than 65536 rows; use recg_verify with a context");
+  int chunks = verify_chunks_per_row(rows, vocab, g_static_sm[dev]);
+  while (chunks > 1 && (long long)chunks * rows > kStaticMaxPartials) --chunks;
+  int chunk_len = (vocab + chunks - 1) / chunks;
+  chunk_len = (chunk_len + 63) / 64 * 64;
+  chunks = (vocab + chunk_len - 1) / chunk_len;
+  if ((long long)chunks * rows > kStaticMaxPartials)
+    return fail(RECG_ERR_CAPACITY, "recg_row_stats_static: rows x vocab chunks exceed the static scratch (65536 partials)");
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  RowPartial* scratch = g_static_ptr[dev];
+  dim3 grid(chunks, rows);
+  if (logits_dtype == RECG_DTYPE_BF16)
+    verify_partial_kernel<__nv_bfloat16>
+        <<<grid, kVerifyThreads, 0, st>>>(static_cast<const __nv_bfloat16*>(logits), vocab, chunk_len, chunks, scratch);
+  else
+    verify_partial_kernel<float><<<grid, kVerifyThreads, 0, st>>>(static_cast<const float*>(logits), vocab, chunk_len,
+                                                                  chunks, scratch);
+  row_stats_finalize_kernel<<<(rows + 127) / 128, 128, 0, st>>>(scratch, rows, chunks, top1, top2, p1, p2, entropy);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return fail(RECG_ERR_CUDA, std::string("recg_row_stats_static: launch: ") + cudaGetErrorString(e));
+  return RECG_OK;
+}
