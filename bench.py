@@ -260,33 +260,58 @@ def run_ours(args, env):
     return out
 
 
-def bench_attention_op(binding, peaks, args):
-    """configs[1]: one layer's hybrid attention at 8B shapes, context 4096, 16 causal + 16 bidirectional rows."""
-    shape = synth.llama8b_shape(32)         # 32 distinct layer caches rotated: 32 x 17 MB > L2
-    desc = c1_descriptor(7)
-    ctx = binding.Context(binding.make_config(shape, 1, 32, desc.page_table.shape[1]))
-    pool = binding.alloc_kv_pool(ctx, desc.n_pages, fill="normal")
-    batch = binding.Batch(desc.ctx_len, desc.verify_len, desc.block_size, None, desc.page_table, pool, desc.n_pages)
-    q = synth.queries(32, 32, 128, seed=5, device="cuda")
-    o = torch.empty_like(q)
-    ctx.recg_attention(batch, 0, q, o)
-    for l in range(32):
-        ctx.recg_attention(None, l, q, o)
-    torch.cuda.synchronize()
-    iters = 10
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for _ in range(iters):
-        for l in range(32):
+def _time_graph(ctx_stream, fn, iters):
+    """Capture fn() (library launches on ctx_stream) into a CUDA graph and time `iters` replays with events, so that
+    short kernels are not hidden behind host launch latency.  Returns microseconds per replay."""
+    with torch.cuda.stream(ctx_stream):
+        fn()
+        ctx_stream.synchronize()
+        g = torch.cuda.CUDAGraph()
+        g.capture_begin()
+        fn()
+        g.capture_end()
+        for _ in range(2):
+            g.replay()
+        ctx_stream.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(ctx_stream)
+        for _ in range(iters):
+            g.replay()
+        e1.record(ctx_stream)
+        ctx_stream.synchronize()
+    return e0.elapsed_time(e1) / iters * 1e3
+
+
+def bench_attention_op(binding, peaks, args, desc=None, n_layers=32, label=None):
+    """configs[1]: one layer's hybrid attention at 8B shapes, context 4096, 16 causal + 16 bidirectional rows.
+    n_layers distinct layer caches are rotated so that the KV stream does not sit in L2; the calls of one rotation
+    are replayed from a CUDA graph (kernel time, not launch latency)."""
+    shape = synth.llama8b_shape(n_layers)
+    desc = c1_descriptor(7) if desc is None else desc
+    T = desc.n_tokens
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        ctx = binding.Context(binding.make_config(shape, desc.n_req, T, desc.page_table.shape[1]), stream=stream.cuda_stream)
+        pool = binding.alloc_kv_pool(ctx, desc.n_pages, fill="normal")
+        batch = binding.Batch(desc.ctx_len, desc.verify_len, desc.block_size, None, desc.page_table, pool, desc.n_pages)
+        q = synth.queries(T, 32, 128, seed=5, device="cuda")
+        o = torch.empty_like(q)
+        ctx.recg_attention(batch, 0, q, o)
+        stream.synchronize()
+
+    def rotation():
+        for l in range(n_layers):
             ctx.recg_attention(None, l, q, o)
-    e1.record()
-    torch.cuda.synchronize()
-    us = e0.elapsed_time(e1) / (iters * 32) * 1e3
-    kv_bytes = (4096 + 32) * 8 * 128 * 2 * 2 + 2 * 32 * 32 * 128 * 2
+
+    us = _time_graph(stream, rotation, 10) / n_layers
+    kv_tok = float((desc.ctx_len + desc.verify_len + desc.block_size).sum())
+    kv_bytes = kv_tok * 8 * 128 * 2 * 2 + 2 * T * 32 * 128 * 2
+    ctx.recg_sync()
     ctx.recg_free()
     gbs = kv_bytes / (us * 1e-6) / 1e9
-    return {"workload": "configs[1]: 32/8 heads, d 128, context 4096, 16 causal + 16 bidirectional rows, 32 caches rotated",
-            "us_per_call": round(us, 2), "calls_include": "attention kernel + combine kernel", "algorithmic_bytes": kv_bytes,
+    return {"workload": label or "configs[1]: 32/8 heads, d 128, context 4096, 16 causal + 16 bidirectional rows, "
+                                 f"{n_layers} caches rotated, CUDA-graph replay",
+            "us_per_call": round(us, 2), "calls_include": "attention kernel + combine kernel", "algorithmic_bytes": int(kv_bytes),
             "gbs": round(gbs, 1), "frac_of_hbm_measured": round(gbs / peaks["hbm_gbs"], 4),
             "frac_of_8000": round(gbs / 8000.0, 4)}
 
@@ -302,7 +327,8 @@ def bench_verify(binding, peaks):
         lg = synth.logits_normal(R, V, seed=6, device="cuda")
         y = synth.token_ids(R, V, seed=1)
         batch = binding.Batch([0] * B, [k + 1] * B, [0] * B, y)
-        ctx.recg_verify(batch, lg, host=False)
+        vout = binding.VerifyOut(B, R, R, host=False)
+        ctx.recg_verify(batch, lg, out=vout)
         n_rot = max(1, int(np.ceil(300e6 / (R * V * 2))))       # rotate copies so that the scan does not sit in L2
         copies = [lg] + [lg.clone() for _ in range(min(n_rot, 64) - 1)]
         torch.cuda.synchronize()
@@ -310,7 +336,7 @@ def bench_verify(binding, peaks):
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
         for i in range(iters):
-            ctx.recg_verify(None, copies[i % len(copies)], host=False, n_req=B, n_tok=R, n_ver=R)
+            ctx.recg_verify(None, copies[i % len(copies)], out=vout)
         e1.record()
         torch.cuda.synchronize()
         us = e0.elapsed_time(e1) / iters * 1e3
@@ -427,6 +453,8 @@ def main():
     ap.add_argument("--steps", type=int, default=8)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--only", default="", help="comma list of op-level sections to run alone (attention_op, verify_sweep): "
+                                               "small cases for profiling; prints their JSON and exits")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
@@ -434,6 +462,22 @@ def main():
         env = DistEnv(rank=int(os.environ.get("RANK", "0")), world=int(os.environ.get("WORLD_SIZE", "1")))
         if env.rank == 0:
             print(json.dumps(run_reference(args, env)), flush=True)
+        return
+    if args.only:
+        from paper_2609_34388_b200 import binding
+
+        peaks = load_peaks()
+        res = {}
+        for sec in args.only.split(","):
+            if sec == "attention_op":
+                res[sec] = bench_attention_op(binding, peaks, args)
+            elif sec == "attention_c16":
+                res[sec] = bench_attention_op(binding, peaks, args, desc=c16_descriptor(3), n_layers=4,
+                                              label="attention of configs[2]: 16 requests, blocks U{4,8,16,32}, context "
+                                                    "U[512,8192], 4 layer caches rotated, CUDA-graph replay")
+            elif sec == "verify_sweep":
+                res[sec] = bench_verify(binding, peaks)
+        print(json.dumps(res), flush=True)
         return
     env = DistEnv.from_env(backend="nccl")
     out = run_ours(args, env)

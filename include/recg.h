@@ -48,7 +48,8 @@ typedef enum { RECG_MEM_DEVICE = 0, RECG_MEM_HOST = 1 } recg_mem;
 
 enum {
   RECG_FLAG_LOGITS_BF16 = 1, /* recg_step() stores logits as bf16 instead of fp32               */
-  RECG_FLAG_SIMT_GEMM = 2    /* run the projections on the legacy mma.sync kernel (A/B checks)  */
+  RECG_FLAG_SIMT_GEMM = 2,   /* run the projections on the legacy mma.sync kernel (A/B checks)  */
+  RECG_FLAG_SIMT_ATTENTION = 4 /* run attention on the legacy mma.sync kernel (A/B checks)      */
 };
 
 typedef struct recg_ctx recg_ctx;

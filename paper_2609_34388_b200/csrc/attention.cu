@@ -33,7 +33,7 @@ struct AttnSmem {
 
 struct AttnParams {
   const AttnItem* items;
-  const int* counts;
+  const int* cta_off;
   const int* page_table;
   int pt_stride;
   const int* tok_climit;
@@ -70,62 +70,58 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attention_kernel(AttnParams P
   }
   __syncthreads();
 
-  const int n_items = P.counts[0];
+  const int item_begin = P.cta_off[blockIdx.x], item_end = P.cta_off[blockIdx.x + 1];
   uint32_t it = 0;  // running block counter, identical in producer and consumers
   bool aborted = false;
 
   if (warp == kConsumerWarps) {
     // ------------------------------ producer ------------------------------
-    if (lane == 0) {
-      for (int item = blockIdx.x; item < n_items && !aborted; item += gridDim.x) {
-        const AttnItem w = P.items[item];
-        const int n_req_pages = (w.kv_len + kPageSize - 1) / kPageSize;
-        const int* pt = P.page_table + (size_t)w.req * P.pt_stride;
-        for (int n = w.blk_begin; n < w.blk_end; ++n, ++it) {
-          const int s = it % kStages;
-          if (!mbar_wait(&empty_bar[s], ((it / kStages) & 1) ^ 1, kSpinLimit)) {
-            set_status(P.status, DEV_TIMEOUT_EMPTY);
-            aborted = true;
-            break;
-          }
-          int pages[kPagesPerBlock];
-          int n_valid = 0;
-#pragma unroll
-          for (int p = 0; p < kPagesPerBlock; ++p) {
-            const int lp = n * kPagesPerBlock + p;
-            int pg = -1;
-            if (lp < n_req_pages) {
-              pg = pt[lp];
-              if (pg < 0 || pg >= P.n_pages) {
-                set_status(P.status, DEV_BAD_INDEX);
-                pg = -1;
-              }
-            }
-            pages[p] = pg;
-            n_valid += pg >= 0;
-          }
-          if (n_valid == 0) {
-            mbar_arrive(&full_bar[s]);
-          } else {
-            mbar_arrive_expect_tx(&full_bar[s], n_valid * SM::kPageBytes);
-#pragma unroll
-            for (int p = 0; p < kPagesPerBlock; ++p) {
-              if (pages[p] >= 0) {
-                const __nv_bfloat16* src =
-                    P.pool + kv_tile_base(P.n_pages, P.n_kv, D, P.layer, pages[p], w.kv_head);
-                bulk_g2s(smem + s * SM::kStageBytes + p * SM::kPageBytes, src, SM::kPageBytes, &full_bar[s]);
-              }
-            }
-          }
+    for (int item = item_begin; item < item_end && !aborted; ++item) {
+      const AttnItem w = P.items[item];
+      const int n_req_pages = (w.kv_len + kPageSize - 1) / kPageSize;
+      const int* pt = P.page_table + (size_t)w.req * P.pt_stride;
+      // lanes 0..3 each own one page of the block; ids are fetched one block ahead of their use
+      auto fetch_page = [&](int n) -> int {
+        int pg = -1;
+        if (lane < kPagesPerBlock && n < w.blk_end) {
+          const int lp = n * kPagesPerBlock + lane;
+          if (lp < n_req_pages) pg = __ldg(pt + lp);   // validated when used
         }
+        return pg;
+      };
+      int pg_next = fetch_page(w.blk_begin);
+      for (int n = w.blk_begin; n < w.blk_end; ++n, ++it) {
+        const int s = it % kStages;
+        int my_pg = pg_next;
+        pg_next = fetch_page(n + 1);                   // in flight during this iteration
+        if (my_pg >= P.n_pages) {
+          set_status(P.status, DEV_BAD_INDEX);
+          my_pg = -1;
+        }
+        if (!mbar_wait(&empty_bar[s], ((it / kStages) & 1) ^ 1, kSpinLimit)) {
+          set_status(P.status, DEV_TIMEOUT_EMPTY);
+          aborted = true;
+          break;
+        }
+        const unsigned valid = __ballot_sync(0xffffffffu, my_pg >= 0);
+        if (lane == 0) {
+          if (valid == 0) mbar_arrive(&full_bar[s]);
+          else mbar_arrive_expect_tx(&full_bar[s], __popc(valid) * SM::kPageBytes);
+        }
+        __syncwarp();
+        if (my_pg >= 0) {
+          const __nv_bfloat16* src = P.pool + kv_tile_base(P.n_pages, P.n_kv, D, P.layer, my_pg, w.kv_head);
+          bulk_g2s(smem + s * SM::kStageBytes + lane * SM::kPageBytes, src, SM::kPageBytes, &full_bar[s]);
+        }
+        __syncwarp();
       }
-      if (aborted) {
-        // let copies already in flight land before the CTA may exit
-        for (int s = 0; s < kStages; ++s) {
-          for (uint32_t i = 0; i < (1u << 16); ++i) {
-            if (mbar_try_wait(&full_bar[s], 0) || mbar_try_wait(&full_bar[s], 1)) break;
-            __nanosleep(64);
-          }
+    }
+    if (aborted && lane == 0) {
+      // let copies already in flight land before the CTA may exit
+      for (int s = 0; s < kStages; ++s) {
+        for (uint32_t i = 0; i < (1u << 16); ++i) {
+          if (mbar_try_wait(&full_bar[s], 0) || mbar_try_wait(&full_bar[s], 1)) break;
+          __nanosleep(64);
         }
       }
     }
@@ -136,7 +132,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attention_kernel(AttnParams P
   const int g = lane >> 2, q4 = lane & 3;
   const uint32_t ring = smem_u32(smem);
 
-  for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
+  for (int item = item_begin; item < item_end; ++item) {
     const AttnItem w = P.items[item];
     const int R = w.ntok * P.group;
     const int RW = (R + 15) >> 4;
@@ -400,7 +396,7 @@ void launch_attention_t(const BatchLayout& bl, const Dims& dm, int layer, const 
   }
   AttnParams P;
   P.items = bl.items;
-  P.counts = bl.counts;
+  P.cta_off = bl.cta_off;
   P.page_table = bl.page_table;
   P.pt_stride = bl.pt_stride;
   P.tok_climit = bl.tok_climit;
@@ -432,7 +428,14 @@ size_t attention_smem_bytes(int head_dim) {
 
 void launch_attention(const BatchLayout& bl, const Dims& dm, int layer, const void* q, void* o, const void* kv_pool,
                       int64_t n_pages, float* part_o, float* part_ml, int tok_per_tile, int n_sm, int* status,
-                      cudaStream_t st) {
+                      cudaStream_t st, bool use_tc) {
+  if (use_tc && dm.head_dim == 128) {
+    launch_attention_tc_main(bl, dm, layer, q, o, kv_pool, n_pages, part_o, part_ml, n_sm, status, st);
+    dim3 grid(bl.n_tok, dm.n_q);
+    attention_combine_kernel<128><<<grid, 32, 0, st>>>(bl, dm.n_q, dm.n_q / dm.n_kv, tok_per_tile, part_o, part_ml,
+                                                       static_cast<__nv_bfloat16*>(o));
+    return;
+  }
   if (dm.head_dim == 64)
     launch_attention_t<64>(bl, dm, layer, q, o, kv_pool, n_pages, part_o, part_ml, tok_per_tile, n_sm, status, st);
   else

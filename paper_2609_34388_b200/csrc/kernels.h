@@ -45,12 +45,13 @@ struct BatchLayout {
   AttnItem* items;
   AttnTile* tiles;
   int* tile_off;    // [C+1] first tile entry of each request
-  int* counts;      // [0] number of items, [1] number of tiles, [2] chunk (blocks per item)
+  int* cta_off;     // [n_ctas+1] first item of each CTA of the persistent attention grid
+  int* counts;      // [0] number of items, [1] number of tiles, [2] blocks per CTA
   int max_items, max_parts;
 };
 
 // S1: per-token arrays and the attention work list.
-void launch_layout(const BatchLayout& bl, const Dims& dm, int tok_per_tile, int target_items, int64_t n_pages,
+void launch_layout(const BatchLayout& bl, const Dims& dm, int tok_per_tile, int n_ctas, int64_t n_pages,
                    int* status, cudaStream_t st);
 // S2: h[t] = embed[tok_id[t]] (fp32 residual stream).
 void launch_embed(const BatchLayout& bl, const Dims& dm, const void* embed, float* h, cudaStream_t st);
@@ -91,9 +92,13 @@ void* tc_state_create(int n_sm);
 void tc_state_destroy(void* s);
 
 // S5
+// use_tc: run the tcgen05 kernel (head_dim 128 only); otherwise the mma.sync kernel
 void launch_attention(const BatchLayout& bl, const Dims& dm, int layer, const void* q, void* o, const void* kv_pool,
                       int64_t n_pages, float* part_o, float* part_ml, int tok_per_tile, int n_sm, int* status,
-                      cudaStream_t st);
+                      cudaStream_t st, bool use_tc);
+void launch_attention_tc_main(const BatchLayout& bl, const Dims& dm, int layer, const void* q, void* o,
+                              const void* kv_pool, int64_t n_pages, float* part_o, float* part_ml, int n_sm, int* status,
+                              cudaStream_t st);
 size_t attention_smem_bytes(int head_dim);
 
 // S9b + S10

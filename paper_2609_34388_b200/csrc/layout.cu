@@ -16,16 +16,22 @@ __device__ __forceinline__ int upper_request(const int* cu, int n_req, int t) {
   return lo;
 }
 
-// One CTA.  Shared: 3 prefix arrays of n_req+1 ints (items, tiles, split parts).
+// One CTA.  Shared: 5 arrays of n_req+1 ints.
+//
+// Attention work list: the 64-token KV blocks of all (request, kv head, row tile) tiles form one line of W
+// blocks; it is cut into n_ctas equal contiguous ranges, one per CTA of the persistent attention grid, and
+// additionally at every tile boundary.  Each piece is an item; a tile cut by CTA boundaries gets one
+// partial slot per piece.  Every CTA therefore streams the same number of blocks (+-1).
 __global__ void __launch_bounds__(1024) layout_kernel(BatchLayout bl, int n_kv, int mask_id, int tok_per_tile,
-                                                      int target_items, int64_t n_pages, int* status) {
+                                                      int n_ctas, int64_t n_pages, int* status) {
   extern __shared__ int sm[];
   const int C = bl.n_req;
-  int* item_off = sm;
-  int* tile_off = sm + (C + 1);
-  int* part_off = sm + 2 * (C + 1);
-  __shared__ unsigned long long s_work;
-  __shared__ int s_chunk;
+  int* req_blk_off = sm;                 // first global block of request r
+  int* tile_off = sm + (C + 1);          // first tile entry of request r
+  int* item_off = sm + 2 * (C + 1);      // first item of request r
+  int* part_off = sm + 3 * (C + 1);      // first partial slot of request r
+  int* req_nb = sm + 4 * (C + 1);        // blocks per tile of request r
+  __shared__ int s_per, s_total_blocks;
   const int tid = threadIdx.x, nth = blockDim.x;
 
   // ---- per-token arrays ----
@@ -51,38 +57,45 @@ __global__ void __launch_bounds__(1024) layout_kernel(BatchLayout bl, int n_kv, 
   }
 
   // ---- attention work list ----
-  if (tid == 0) s_work = 0ull;
-  __syncthreads();
-  unsigned long long w = 0;
   for (int r = tid; r < C; r += nth) {
     const int n = bl.verify_len[r] + bl.block_size[r];
-    const int nb = (bl.ctx_len[r] + n + 63) / 64;
-    const int tiles = (n + tok_per_tile - 1) / tok_per_tile;
-    w += (unsigned long long)n_kv * tiles * nb;
-  }
-  if (w) atomicAdd(&s_work, w);
-  __syncthreads();
-  if (tid == 0) {
-    unsigned long long c = (s_work + target_items - 1) / target_items;
-    s_chunk = c < 1 ? 1 : (c > (1 << 20) ? (1 << 20) : (int)c);
-  }
-  __syncthreads();
-  const int chunk = s_chunk;
-  for (int r = tid; r < C; r += nth) {
-    const int n = bl.verify_len[r] + bl.block_size[r];
-    const int nb = (bl.ctx_len[r] + n + 63) / 64;
-    const int tiles = (n + tok_per_tile - 1) / tok_per_tile;
-    const int parts = (nb + chunk - 1) / chunk;
-    item_off[r + 1] = n_kv * tiles * parts;
-    tile_off[r + 1] = n_kv * tiles;
-    part_off[r + 1] = parts > 1 ? n_kv * tiles * parts : 0;
+    req_nb[r] = (bl.ctx_len[r] + n + 63) / 64;
+    tile_off[r + 1] = n_kv * ((n + tok_per_tile - 1) / tok_per_tile);
   }
   __syncthreads();
   if (tid == 0) {
-    item_off[0] = tile_off[0] = part_off[0] = 0;
+    req_blk_off[0] = 0;
+    tile_off[0] = 0;
+    long long w = 0;
+    for (int r = 0; r < C; ++r) {
+      w += (long long)tile_off[r + 1] * req_nb[r];
+      if (w > 0x3fffffff) w = 0x3fffffff;   // far beyond any pool; keeps the arithmetic in int
+      req_blk_off[r + 1] = (int)w;
+      tile_off[r + 1] += tile_off[r];
+    }
+    s_total_blocks = (int)w;
+    const int per = (int)((w + n_ctas - 1) / n_ctas);
+    s_per = per < 1 ? 1 : per;
+  }
+  __syncthreads();
+  const int per = s_per, W = s_total_blocks;
+  for (int r = tid; r < C; r += nth) {
+    const int nb = req_nb[r], nt = tile_off[r + 1] - tile_off[r];
+    int items = 0, parts_split = 0;
+    for (int k = 0; k < nt; ++k) {
+      const int g0 = req_blk_off[r] + k * nb, g1 = g0 + nb;
+      const int parts = (g1 - 1) / per - g0 / per + 1;
+      items += parts;
+      if (parts > 1) parts_split += parts;
+    }
+    item_off[r + 1] = items;
+    part_off[r + 1] = parts_split;
+  }
+  __syncthreads();
+  if (tid == 0) {
+    item_off[0] = part_off[0] = 0;
     for (int r = 0; r < C; ++r) {
       item_off[r + 1] += item_off[r];
-      tile_off[r + 1] += tile_off[r];
       part_off[r + 1] += part_off[r];
     }
     int n_items = item_off[C];
@@ -92,37 +105,43 @@ __global__ void __launch_bounds__(1024) layout_kernel(BatchLayout bl, int n_kv, 
     }
     bl.counts[0] = n_items;
     bl.counts[1] = tile_off[C];
-    bl.counts[2] = chunk;
+    bl.counts[2] = per;
   }
   __syncthreads();
-  for (int r = tid; r <= C; r += nth) bl.tile_off[r] = tile_off[r];
   const int n_items = bl.counts[0];
-  for (int it = tid; it < n_items; it += nth) {
-    const int r = upper_request(item_off, C, it);
-    const int local = it - item_off[r];
+  for (int r = tid; r <= C; r += nth) bl.tile_off[r] = tile_off[r];
+  for (int c = tid; c <= n_ctas; c += nth)
+    if ((long long)c * per >= W || n_items == 0) bl.cta_off[c] = n_items;   // CTAs without work
+  if (n_items == 0) return;
+  for (int r = tid; r < C; r += nth) {
     const int n = bl.verify_len[r] + bl.block_size[r];
     const int kv_len = bl.ctx_len[r] + n;
-    const int nb = (kv_len + 63) / 64;
-    const int tiles = (n + tok_per_tile - 1) / tok_per_tile;
-    const int parts = (nb + chunk - 1) / chunk;
-    const int part = local % parts;
-    const int tile = (local / parts) % tiles;
-    const int kvh = local / (parts * tiles);
-    AttnItem a;
-    a.req = r;
-    a.kv_head = kvh;
-    a.tok0 = bl.cu_tok[r] + tile * tok_per_tile;
-    a.ntok = min(tok_per_tile, n - tile * tok_per_tile);
-    a.blk_begin = part * chunk;
-    a.blk_end = min(nb, (part + 1) * chunk);
-    a.part = parts > 1 ? part_off[r] + (kvh * tiles + tile) * parts + part : -1;
-    a.kv_len = kv_len;
-    bl.items[it] = a;
-    if (part == 0) {
+    const int nb = req_nb[r], nt = tile_off[r + 1] - tile_off[r];
+    const int tiles = nt / n_kv;
+    int item = item_off[r], part = part_off[r];
+    for (int k = 0; k < nt; ++k) {
+      const int kvh = k / tiles, tile = k % tiles;
+      const int g0 = req_blk_off[r] + k * nb, g1 = g0 + nb;
+      const int c_first = g0 / per, c_last = (g1 - 1) / per;
+      const int parts = c_last - c_first + 1;
       AttnTile tl;
-      tl.part_begin = parts > 1 ? a.part : -1;
+      tl.part_begin = parts > 1 ? part : -1;
       tl.n_parts = parts;
-      bl.tiles[tile_off[r] + kvh * tiles + tile] = tl;
+      bl.tiles[tile_off[r] + k] = tl;
+      for (int c = c_first; c <= c_last; ++c, ++item) {
+        const int gs = max(g0, c * per), ge = min(g1, (c + 1) * per);
+        AttnItem a;
+        a.req = r;
+        a.kv_head = kvh;
+        a.tok0 = bl.cu_tok[r] + tile * tok_per_tile;
+        a.ntok = min(tok_per_tile, n - tile * tok_per_tile);
+        a.blk_begin = gs - g0;
+        a.blk_end = ge - g0;
+        a.part = parts > 1 ? part++ : -1;
+        a.kv_len = kv_len;
+        bl.items[item] = a;
+        if (gs == c * per) bl.cta_off[c] = item;   // first item of CTA c
+      }
     }
   }
 }
@@ -196,10 +215,10 @@ __global__ void kv_io_kernel(bool write, __nv_bfloat16* pool, int64_t n_pages, i
 
 }  // namespace
 
-void launch_layout(const BatchLayout& bl, const Dims& dm, int tok_per_tile, int target_items, int64_t n_pages,
+void launch_layout(const BatchLayout& bl, const Dims& dm, int tok_per_tile, int n_ctas, int64_t n_pages,
                    int* status, cudaStream_t st) {
-  const size_t smem = 3 * (size_t)(bl.n_req + 1) * sizeof(int);
-  layout_kernel<<<1, 1024, smem, st>>>(bl, dm.n_kv, dm.mask_id, tok_per_tile, target_items, n_pages, status);
+  const size_t smem = 5 * (size_t)(bl.n_req + 1) * sizeof(int);
+  layout_kernel<<<1, 1024, smem, st>>>(bl, dm.n_kv, dm.mask_id, tok_per_tile, n_ctas, n_pages, status);
 }
 
 void launch_embed(const BatchLayout& bl, const Dims& dm, const void* embed, float* h, cudaStream_t st) {

@@ -115,6 +115,7 @@ size_t carve(recg_ctx* c, DeviceArena& A) {
   bl.items = A.take<AttnItem>(bl.max_items);
   bl.tiles = A.take<AttnTile>(max_tiles);
   bl.tile_off = A.take<int>(Cm + 1);
+  bl.cta_off = A.take<int>(c->target_items + 1);
   bl.counts = A.take<int>(4);
   c->d_status = A.take<int>(1);
   c->d_page_row = A.take<int>(Pm);
@@ -403,7 +404,7 @@ recg_status recg_step(recg_ctx* ctx, const recg_batch* batch, recg_logits* logit
     if ((s = run_gemm(ctx, a)) != RECG_OK) return s;
     ctx->mark(2, 1);
     launch_attention(bl, d, l, ctx->q, ctx->o, batch->kv_pool, batch->kv_pool_pages, ctx->part_o, ctx->part_ml,
-                     ctx->tok_per_tile, ctx->n_sm, ctx->d_status, st);
+                     ctx->tok_per_tile, ctx->n_sm, ctx->d_status, st, !(ctx->cfg.flags & RECG_FLAG_SIMT_ATTENTION));
     CU(cudaGetLastError());
     ctx->mark(3, 2);
     GemmArgs b{};
@@ -497,7 +498,7 @@ recg_status recg_attention(recg_ctx* ctx, const recg_batch* batch, int32_t layer
     return fail(ctx, RECG_ERR_INVALID_ARG, "recg_attention: no batch given and none with a KV pool laid out before");
   }
   launch_attention(ctx->bl, ctx->dm, layer, q, o, ctx->last_pool, ctx->last_pool_pages, ctx->part_o, ctx->part_ml,
-                   ctx->tok_per_tile, ctx->n_sm, ctx->d_status, ctx->stream);
+                   ctx->tok_per_tile, ctx->n_sm, ctx->d_status, ctx->stream, !(ctx->cfg.flags & RECG_FLAG_SIMT_ATTENTION));
   CU(cudaGetLastError());
   return RECG_OK;
 }
