@@ -194,8 +194,8 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attention_kernel(AttnParams P
             const int token = nt * 8 + (lane & 7);
             const int pg = token >> 4, tok = token & 15;
             const int c = 4 * j + (lane >> 3);
-            const uint32_t addr =
-                stage + pg * SM::kPageBytes + (c >> 3) * 2048 + tok * 128 + (((c & 7) ^ (tok & 7)) << 4);
+            const uint32_t addr = stage + pg * SM::kPageBytes + ((tok >> 3) * (D / 64) + (c >> 3)) * 1024 +
+                                  (tok & 7) * 128 + (((c & 7) ^ (tok & 7)) << 4);
             uint32_t b0, b1, b2, b3;
             ldmatrix_x4(b0, b1, b2, b3, addr);
             mma_bf16_16816(sc[nt], qf[2 * j], b0, b1);
@@ -267,7 +267,8 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attention_kernel(AttnParams P
 #pragma unroll
           for (int jj = 0; jj < D / 16; ++jj) {
             const int c = 2 * jj + (mi >> 1);
-            const uint32_t addr = stage + kk * SM::kPageBytes + kPageSize * D * 2 + (c >> 3) * 2048 + tok * 128 +
+            const uint32_t addr = stage + kk * SM::kPageBytes + kPageSize * D * 2 +
+                                  ((tok >> 3) * (D / 64) + (c >> 3)) * 1024 + (tok & 7) * 128 +
                                   (((c & 7) ^ (tok & 7)) << 4);
             uint32_t b0, b1, b2, b3;
             ldmatrix_x4_trans(b0, b1, b2, b3, addr);

@@ -4,10 +4,9 @@
 // Per CTA (6 warps, one CTA per SM, persistent over the work list):
 //   warp 0    producer: streams 128-token KV blocks page by page, ONE 4 KB bulk copy per page and operand,
 //             into a ring of five 32 KB operand buffers (K and V of a block are separate entries, so K is
-//             released early); spare lanes prefetch the pages two blocks further on into L2.  A page tile
-//             ([2 dim halves][16 tokens][128 B], 128-byte swizzled) lands exactly as stored, and the MMA
-//             descriptors stride over pages: S is computed as two N = 64 halves (tokens 0-7 resp. 8-15
-//             of every page), which permutes the S / P columns consistently with the V operand's K order.
+//             released early).  A page tile (8-row, 128-byte-swizzled atoms ordered [token group][dim half])
+//             lands exactly as stored, and tiles copied back to back form one 128-token operand with a
+//             uniform 2 KB stride between token groups: K-major for S = Q K^T, MN-major for O += P V.
 //             The last, partly filled page of a request is copied by hand with the rows beyond its length
 //             zeroed, so stale pool contents can never reach an accumulator.
 //   warp 1    one elected lane issues tcgen05.mma: S = Q K^T (M 128 rows, N 128 tokens, K = d) into one
@@ -132,9 +131,9 @@ __device__ __forceinline__ uint64_t desc_mnmajor(uint32_t addr, uint32_t lbo_byt
 __device__ __forceinline__ void l2_prefetch(const void* gptr, uint32_t bytes) {
   asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(gptr), "r"(bytes) : "memory");
 }
-// S / P column c of a 128-token block holds token 16 * ((c & 63) >> 3) + 8 * (c >> 6) + (c & 7)
-__device__ __forceinline__ int col_token(int c) { return (((c & 63) >> 3) << 4) + ((c >> 6) << 3) + (c & 7); }
-constexpr uint32_t kIdescQK = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(64 >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+// S / P column c of a 128-token block holds token c
+__device__ __forceinline__ int col_token(int c) { return c; }
+constexpr uint32_t kIdescQK = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kBT >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
 constexpr uint32_t kIdescPV =
     (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(D >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
 
@@ -270,7 +269,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_tc_kernel(TcAttnParams 
 #pragma unroll
             for (int u = 0; u < 8; ++u) {
               const int c = u * 32 + lane;
-              v[u] = (((c >> 3) & 15) < valid_tok) ? __ldg(src + c) : make_uint4(0, 0, 0, 0);
+              v[u] = (((c >> 7) * 8 + ((c >> 3) & 7)) < valid_tok) ? __ldg(src + c) : make_uint4(0, 0, 0, 0);
             }
 #pragma unroll
             for (int u = 0; u < 8; ++u) *reinterpret_cast<uint4*>(stage + p * kTileBytes + (u * 32 + lane) * 16) = v[u];
@@ -316,13 +315,11 @@ __global__ void __launch_bounds__(kThreads, 1) attention_tc_kernel(TcAttnParams 
         tc_fence_after();
         const uint32_t k_addr = smem_base + kOffKV + s * kKVStageBytes;
 #pragma unroll
-        for (int g = 0; g < 2; ++g) {               // tokens 0-7 resp. 8-15 of every page -> S columns [64 g, 64 g + 64)
-#pragma unroll
-          for (int kk = 0; kk < D / 16; ++kk) {
-            const uint64_t da = desc_kmajor(q_addr + (kk >> 2) * (128 * 128) + (kk & 3) * 32);
-            const uint64_t db = desc_kmajor(k_addr + g * 1024 + (kk >> 2) * kSubBytes + (kk & 3) * 32, kTileBytes);
-            umma_bf16(tmem_base + sb * kBT + g * 64, da, db, kIdescQK, kk ? 1u : 0u);
-          }
+        for (int kk = 0; kk < D / 16; ++kk) {
+          const uint64_t da = desc_kmajor(q_addr + (kk >> 2) * (128 * 128) + (kk & 3) * 32);
+          // K block: 16 token groups (2 per page) 2 KB apart; the dim half selects the atom next door
+          const uint64_t db = desc_kmajor(k_addr + (kk >> 2) * 1024 + (kk & 3) * 32, 2048);
+          umma_bf16(tmem_base + sb * kBT, da, db, kIdescQK, kk ? 1u : 0u);
         }
         umma_commit(&kv_empty[s]);   // the K buffer is free once these MMAs have read it
         umma_commit(&s_full[sb]);
@@ -361,8 +358,8 @@ __global__ void __launch_bounds__(kThreads, 1) attention_tc_kernel(TcAttnParams 
 #pragma unroll
           for (int kk = 0; kk < kBT / 16; ++kk) {
             const uint64_t da = desc_kmajor(p_addr + pb * kPBytes + (kk >> 2) * (128 * 128) + (kk & 3) * 32);
-            // P columns [16 kk, 16 kk + 16): group g = kk >> 2 of pages 2 (kk & 3) and 2 (kk & 3) + 1
-            const uint64_t db = desc_mnmajor(v_addr + 2 * (kk & 3) * kTileBytes + (kk >> 2) * 1024, kSubBytes, kTileBytes);
+            // tokens [16 kk, 16 kk + 16) = page kk: two token groups 2 KB apart, the dim halves 1 KB apart
+            const uint64_t db = desc_mnmajor(v_addr + kk * kTileBytes, 1024, 2048);
             umma_bf16(tmem_base + 2 * kBT, da, db, kIdescPV, (n | kk) ? 1u : 0u);
           }
           umma_commit(&kv_empty[s]);
@@ -387,7 +384,6 @@ __global__ void __launch_bounds__(kThreads, 1) attention_tc_kernel(TcAttnParams 
       const int tok_end = min(w.blk_end * 64, w.kv_len);
       const int nblk = (tok_end - tok_begin + kBT - 1) / kBT;
       ITRACE(item_cnt, 0);
-      if (blockIdx.x == 29 && warp == 2 && lane == 0 && item_cnt < 16) { g_item[item_cnt][6] = nblk; g_item[item_cnt][7] = R; }
       // ---- stage Q in operand layout: [2 halves][128 rows][128 B], 16-byte chunks swizzled by row & 7 ----
       // only the R valid rows are staged: the other rows of the M = 128 operand yield S / O rows nobody reads.
       // Loads are issued in batches of 8 before any store so that their latencies overlap.
@@ -461,10 +457,15 @@ __global__ void __launch_bounds__(kThreads, 1) attention_tc_kernel(TcAttnParams 
                 if (!vis) sr[c][i] = 0xff800000u;   // -inf
               }
           }
+          {  // four independent chains instead of one 128-long dependent one
+            float mxa[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-          for (int c = 0; c < 4; ++c)
+            for (int c = 0; c < 4; ++c)
 #pragma unroll
-            for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(sr[c][i]));
+              for (int i = 0; i < 32; i += 2)
+                mxa[c] = fmaxf(mxa[c], fmaxf(__uint_as_float(sr[c][i]), __uint_as_float(sr[c][i + 1])));
+            mx = fmaxf(fmaxf(mxa[0], mxa[1]), fmaxf(mxa[2], mxa[3]));
+          }
         }
         // S has been read: the MMA warp may overwrite this buffer with the block after next
         tc_fence_before();
@@ -502,14 +503,14 @@ __global__ void __launch_bounds__(kThreads, 1) attention_tc_kernel(TcAttnParams 
             }
             tmem_st_wait();
           }
-          float ls = 0.f;
+          float lsa[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
           for (int c = 0; c < 4; ++c) {
 #pragma unroll
             for (int i = 0; i < 32; ++i) {
               const float p = exp2f(__uint_as_float(sr[c][i]) * P.scale_log2 - m_ref);   // exp2(-inf) = 0 for masked
               sr[c][i] = __float_as_uint(p);
-              ls += p;
+              lsa[i & 3] += p;
             }
             if (rvalid) {
 #pragma unroll
@@ -523,7 +524,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_tc_kernel(TcAttnParams 
               }
             }
           }
-          l_run += ls;
+          l_run += (lsa[0] + lsa[1]) + (lsa[2] + lsa[3]);
         }
         tc_fence_before();
         fence_proxy_async();

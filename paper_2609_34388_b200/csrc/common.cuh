@@ -95,17 +95,19 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 __device__ __forceinline__ float bf16_bits_to_float(uint16_t b) { return __uint_as_float(static_cast<uint32_t>(b) << 16); }
 
 // ---- KV pool addressing ------------------------------------------------------------------------
-// Pool = [layer][page][kv_head][K tile | V tile]; a tile holds 16 tokens x head_dim bf16 as
-// head_dim/64 sub-tiles of [16 tokens][64 elements = 128 bytes], the eight 16-byte chunks of a
-// row XOR-swizzled with (token & 7), so that both row-wise and transposed fragment loads from
-// shared memory are bank-conflict free after a plain linear copy of the tile.
+// Pool = [layer][page][kv_head][K tile | V tile]; a tile holds 16 tokens x head_dim bf16 as 8-row atoms
+// [token group g = tok / 8][dim half h = dim / 64][8 tokens][64 elements = 128 bytes], the eight 16-byte chunks
+// of a row XOR-swizzled with (token & 7).  An atom is exactly the tensor core's canonical 128-byte-swizzle atom
+// (K-major for K, MN-major for V), and because the token groups of consecutive pages are a constant
+// 2 * (head_dim / 64) atoms apart, tiles copied back to back into shared memory form a multi-page operand
+// with one uniform stride; row-wise and transposed ldmatrix loads from the same bytes are conflict free.
 constexpr int kPageSize = 16;
 
 __host__ __device__ __forceinline__ size_t kv_tile_elems(int head_dim) { return (size_t)kPageSize * head_dim; }
 // element offset of (token-in-page, dim) inside a tile
-__host__ __device__ __forceinline__ int kv_tile_offset(int tok, int dim) {
-  const int sub = dim >> 6, c = (dim >> 3) & 7, e = dim & 7;
-  return sub * (kPageSize * 64) + tok * 64 + ((c ^ (tok & 7)) << 3) + e;
+__host__ __device__ __forceinline__ int kv_tile_offset(int tok, int dim, int head_dim) {
+  const int atom = (tok >> 3) * (head_dim >> 6) + (dim >> 6), c = (dim >> 3) & 7, e = dim & 7, r = tok & 7;
+  return atom * 512 + r * 64 + ((c ^ r) << 3) + e;
 }
 // element offset of the K tile of (layer, page, kv_head); the V tile follows it
 __host__ __device__ __forceinline__ size_t kv_tile_base(int64_t n_pages, int n_kv, int head_dim, int layer,

@@ -81,8 +81,8 @@ __device__ __forceinline__ void tile_epilogue(const EpiParams& ep, const float* 
         }
         __nv_bfloat16* base = ep.kv_pool + kv_tile_base(ep.n_pages, ep.n_kv, D, ep.layer, page, kvh) +
                               (is_v ? kv_tile_elems(D) : 0);
-        *reinterpret_cast<uint32_t*>(base + kv_tile_offset(tok, i)) = plo;
-        *reinterpret_cast<uint32_t*>(base + kv_tile_offset(tok, i + half)) = phi;
+        *reinterpret_cast<uint32_t*>(base + kv_tile_offset(tok, i, D)) = plo;
+        *reinterpret_cast<uint32_t*>(base + kv_tile_offset(tok, i + half, D)) = phi;
       }
     }
     return;

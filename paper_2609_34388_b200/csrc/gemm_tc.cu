@@ -13,6 +13,8 @@
 #include <cuda.h>
 
 #include <cstdio>
+#include <cstdlib>
+#include <cmath>
 #include <mutex>
 #include <unordered_map>
 
@@ -137,9 +139,34 @@ __device__ __forceinline__ void store_chunk_bf16(__nv_bfloat16* dst, const float
   }
 }
 
-// Epilogue of one accumulator tile for the calling thread's row.  tacc: TMEM address of (lane quadrant, column 0).
-template <int BN>
-__device__ __forceinline__ void row_epilogue(const EpiParams& ep, uint32_t tacc, int m, int n0) {
+// Where the epilogue takes the thread's accumulator row from: TMEM, or the sum over the K splits' partial tiles.
+struct TmemLoader {
+  uint32_t tacc;   // TMEM address of (lane quadrant, column 0)
+  __device__ __forceinline__ void operator()(int col, float (&v)[32]) const { tmem_ld32(tacc + col, v); }
+};
+struct SplitLoader {
+  const float* row0;      // partial of split 0, this thread's row
+  size_t split_stride;    // floats between consecutive splits' partial tiles
+  int n_splits;
+  bool valid;             // rows beyond M were never parked
+  __device__ __forceinline__ void operator()(int col, float (&v)[32]) const {
+#pragma unroll
+    for (int i = 0; i < 32; ++i) v[i] = 0.f;
+    if (!valid) return;
+    for (int sp = 0; sp < n_splits; ++sp) {        // fixed order: the result does not depend on who arrived last
+      const float4* src = reinterpret_cast<const float4*>(row0 + sp * split_stride + col);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const float4 t = __ldcg(src + i);
+        v[4 * i] += t.x; v[4 * i + 1] += t.y; v[4 * i + 2] += t.z; v[4 * i + 3] += t.w;
+      }
+    }
+  }
+};
+
+// Epilogue of one accumulator tile for the calling thread's row.
+template <int BN, typename Loader>
+__device__ __forceinline__ void row_epilogue(const EpiParams& ep, const Loader& load, int m, int n0) {
   const bool row_ok = m < ep.M;
   if (ep.epi == EPI_SWIGLU) {
     // accumulator columns [0, BN/2) are gate, [BN/2, BN) up; n0 is the first output column
@@ -147,8 +174,8 @@ __device__ __forceinline__ void row_epilogue(const EpiParams& ep, uint32_t tacc,
 #pragma unroll 1
     for (int c = 0; c < BN / 64; ++c) {
       float g[32], u[32];
-      tmem_ld32(tacc + c * 32, g);
-      tmem_ld32(tacc + BN / 2 + c * 32, u);
+      load(c * 32, g);
+      load(BN / 2 + c * 32, u);
       if (row_ok && n0 + c * 32 < ep.N) {
 #pragma unroll
         for (int i = 0; i < 32; ++i) g[i] = silu_f(g[i]) * u[i];
@@ -179,8 +206,8 @@ __device__ __forceinline__ void row_epilogue(const EpiParams& ep, uint32_t tacc,
 #pragma unroll 1
       for (int c = 0; c < half / 32; ++c) {      // 32 low columns with their 32 partners half a head away
         float lo[32], hi[32];
-        tmem_ld32(tacc + hl * D + c * 32, lo);
-        tmem_ld32(tacc + hl * D + half + c * 32, hi);
+        load(hl * D + c * 32, lo);
+        load(hl * D + half + c * 32, hi);
         if (!row_ok) continue;
         if (!is_v) {
           const float2* cs = ep.rope_cs + (size_t)m * half + c * 32;
@@ -205,8 +232,8 @@ __device__ __forceinline__ void row_epilogue(const EpiParams& ep, uint32_t tacc,
             a.z = pack_bf16(lo[8 * j + 4], lo[8 * j + 5]); a.w = pack_bf16(lo[8 * j + 6], lo[8 * j + 7]);
             b.x = pack_bf16(hi[8 * j], hi[8 * j + 1]); b.y = pack_bf16(hi[8 * j + 2], hi[8 * j + 3]);
             b.z = pack_bf16(hi[8 * j + 4], hi[8 * j + 5]); b.w = pack_bf16(hi[8 * j + 6], hi[8 * j + 7]);
-            *reinterpret_cast<uint4*>(kv_base + kv_tile_offset(tok, c * 32 + j * 8)) = a;
-            *reinterpret_cast<uint4*>(kv_base + kv_tile_offset(tok, half + c * 32 + j * 8)) = b;
+            *reinterpret_cast<uint4*>(kv_base + kv_tile_offset(tok, c * 32 + j * 8, D)) = a;
+            *reinterpret_cast<uint4*>(kv_base + kv_tile_offset(tok, half + c * 32 + j * 8, D)) = b;
           }
         }
       }
@@ -216,7 +243,7 @@ __device__ __forceinline__ void row_epilogue(const EpiParams& ep, uint32_t tacc,
 #pragma unroll 1
   for (int c = 0; c < BN / 32; ++c) {
     float v[32];
-    tmem_ld32(tacc + c * 32, v);
+    load(c * 32, v);
     const int n = n0 + c * 32;
     if (!row_ok || n >= ep.N) continue;
     if (n + 32 <= ep.N) {
@@ -235,7 +262,7 @@ __device__ __forceinline__ void row_epilogue(const EpiParams& ep, uint32_t tacc,
 template <int BN>
 __global__ void __launch_bounds__(kTcThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w, int M, int n_tiles_n,
-               int K, int up_row_offset, EpiParams ep) {
+               int K, int up_row_offset, int n_splits, float* split_ws, int* split_counters, EpiParams ep) {
   using Cfg = TcCfg<BN>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -248,6 +275,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n_tiles_m = (M + BM - 1) / BM;
   const int n_tiles = n_tiles_m * n_tiles_n;
+  const int n_units = n_tiles * n_splits;   // a unit is (tile, K split); the splits of a tile are adjacent units
   const int KB = K / BK;
   const bool swiglu = ep.epi == EPI_SWIGLU;
 
@@ -278,9 +306,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     if (elect_one()) {
       uint32_t it = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+      for (int unit = blockIdx.x; unit < n_units && ok; unit += gridDim.x) {
+        const int tile = unit / n_splits, split = unit % n_splits;
         const int tm = tile % n_tiles_m, tn = tile / n_tiles_m;
-        for (int kb = 0; kb < KB; ++kb, ++it) {
+        const int kb0 = (split * KB) / n_splits, kb1 = ((split + 1) * KB) / n_splits;
+        for (int kb = kb0; kb < kb1; ++kb, ++it) {
           const int s = it % Cfg::kStages;
           if (!mbar_wait(&empty_bar[s], ((it / Cfg::kStages) & 1) ^ 1, kSpin)) {
             set_status(ep.status, DEV_TIMEOUT_EMPTY);
@@ -313,7 +343,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
       constexpr uint32_t idesc = make_idesc(BN);
       uint32_t it = 0, tcount = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++tcount) {
+      for (int unit = blockIdx.x; unit < n_units && ok; unit += gridDim.x, ++tcount) {
+        const int split = unit % n_splits;
+        const int kb0 = (split * KB) / n_splits, kb1 = ((split + 1) * KB) / n_splits;
         const int acc = tcount & 1;
         if (!mbar_wait(&tempty_bar[acc], ((tcount >> 1) & 1) ^ 1, kSpin)) {
           set_status(ep.status, DEV_TIMEOUT_MMA);
@@ -321,7 +353,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
         }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + acc * BN;
-        for (int kb = 0; kb < KB; ++kb, ++it) {
+        for (int kb = kb0; kb < kb1; ++kb, ++it) {
           const int s = it % Cfg::kStages;
           if (!mbar_wait(&full_bar[s], (it / Cfg::kStages) & 1, kSpin)) {
             set_status(ep.status, DEV_TIMEOUT_FULL);
@@ -335,7 +367,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
           for (int k = 0; k < BK / 16; ++k) {
             const uint64_t da = make_smem_desc(a_addr + k * 32);
             const uint64_t db = make_smem_desc(b_addr + k * 32);
-            umma_bf16(d_tmem, da, db, idesc, (kb | k) ? 1u : 0u);
+            umma_bf16(d_tmem, da, db, idesc, ((kb - kb0) | k) ? 1u : 0u);
           }
           umma_commit(&empty_bar[s]);      // frees the stage when these MMAs have read it
         }
@@ -346,7 +378,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     // ------------------------------ epilogue warps ------------------------------
     const int quad = warp & 3;             // TMEM lane quadrant this warp may read
     uint32_t tcount = 0;
-    for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++tcount) {
+    __shared__ int s_last;
+    for (int unit = blockIdx.x; unit < n_units; unit += gridDim.x, ++tcount) {
+      const int tile = unit / n_splits, split = unit % n_splits;
       const int tm = tile % n_tiles_m, tn = tile / n_tiles_m;
       const int acc = tcount & 1;
       if (!mbar_wait(&tfull_bar[acc], (tcount >> 1) & 1, kSpin)) {
@@ -355,12 +389,46 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
       }
       tc_fence_after();
       const uint32_t tacc = tmem_base + ((uint32_t)(quad * 32) << 16) + acc * BN;
-      const int m = tm * BM + quad * 32 + lane;
+      const int row_in_tile = quad * 32 + lane;
+      const int m = tm * BM + row_in_tile;
       const int n0 = swiglu ? tn * (BN / 2) : tn * BN;
-      row_epilogue<BN>(ep, tacc, m, n0);
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&tempty_bar[acc]);
+      if (n_splits == 1) {
+        row_epilogue<BN>(ep, TmemLoader{tacc}, m, n0);
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&tempty_bar[acc]);
+      } else {
+        // park this split's partial tile, release the accumulator, and let the LAST split to arrive reduce all
+        // partials in split order (deterministic) and run the fused epilogue
+        float* mine = split_ws + ((size_t)unit * BM + row_in_tile) * BN;
+#pragma unroll 1
+        for (int c = 0; c < BN / 32; ++c) {
+          float v[32];
+          tmem_ld32(tacc + c * 32, v);
+          if (m < ep.M) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+              __stcg(reinterpret_cast<float4*>(mine + c * 32) + i, make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]));
+          }
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&tempty_bar[acc]);
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (warp == 2 && lane == 0) {
+          __threadfence();   // cumulative: orders the partial rows all 128 threads wrote before the barrier
+          const int old = atomicAdd(&split_counters[tile], 1);
+          s_last = (old == n_splits - 1);
+          if (old == n_splits - 1) split_counters[tile] = 0;   // ready for the next launch
+          __threadfence();
+        }
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (s_last) {
+          SplitLoader ld{split_ws + ((size_t)tile * n_splits * BM + row_in_tile) * BN, (size_t)BM * BN, n_splits, m < ep.M};
+          row_epilogue<BN>(ep, ld, m, n0);
+        }
+        asm volatile("bar.sync 1, 128;" ::: "memory");       // s_last is reused by the next unit
+      }
     }
   }
 
@@ -389,8 +457,14 @@ struct MapKeyHash {
   }
 };
 
+constexpr size_t kSplitWsBytes = 96ull << 20;   // partial tiles of split-K launches
+constexpr int kSplitCounters = 1 << 16;
+
 struct TcState {
   int n_sm = 0;
+  int force_bn = 0, force_s = 1;
+  float* split_ws = nullptr;
+  int* split_counters = nullptr;
   EncodeTiledFn encode = nullptr;
   std::unordered_map<MapKey, CUtensorMap, MapKeyHash> maps;
   bool configured[3] = {false, false, false};
@@ -415,7 +489,7 @@ const CUtensorMap* get_map(TcState* st, const void* ptr, uint64_t rows, uint64_t
 }
 
 template <int BN>
-bool launch_bn(TcState* st, int idx, const GemmArgs& a, const EpiParams& ep, cudaStream_t stream) {
+bool launch_bn(TcState* st, int idx, const GemmArgs& a, const EpiParams& ep, int n_splits, cudaStream_t stream) {
   using Cfg = TcCfg<BN>;
   if (!st->configured[idx]) {
     if (cudaFuncSetAttribute(gemm_tc_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes) != cudaSuccess)
@@ -429,9 +503,10 @@ bool launch_bn(TcState* st, int idx, const GemmArgs& a, const EpiParams& ep, cud
   if (!mx || !mw) return false;
   const int out_per_tile = swiglu ? BN / 2 : BN;
   const int n_tiles_n = (a.N + out_per_tile - 1) / out_per_tile;
-  const int n_tiles = ((a.M + BM - 1) / BM) * n_tiles_n;
-  const int grid = n_tiles < st->n_sm ? n_tiles : st->n_sm;
-  gemm_tc_kernel<BN><<<grid, kTcThreads, Cfg::kSmemBytes, stream>>>(*mx, *mw, a.M, n_tiles_n, a.K, a.N, ep);
+  const int n_units = ((a.M + BM - 1) / BM) * n_tiles_n * n_splits;
+  const int grid = n_units < st->n_sm ? n_units : st->n_sm;
+  gemm_tc_kernel<BN><<<grid, kTcThreads, Cfg::kSmemBytes, stream>>>(*mx, *mw, a.M, n_tiles_n, a.K, a.N, n_splits,
+                                                                    st->split_ws, st->split_counters, ep);
   return true;
 }
 
@@ -448,10 +523,25 @@ void* tc_state_create(int n_sm) {
     return nullptr;
   }
   st->encode = reinterpret_cast<EncodeTiledFn>(fn);
+  if (const char* f = getenv("RECG_GEMM_FORCE")) sscanf(f, "%d,%d", &st->force_bn, &st->force_s);
+  if (cudaMalloc(reinterpret_cast<void**>(&st->split_ws), kSplitWsBytes) != cudaSuccess ||
+      cudaMalloc(reinterpret_cast<void**>(&st->split_counters), kSplitCounters * sizeof(int)) != cudaSuccess ||
+      cudaMemset(st->split_counters, 0, kSplitCounters * sizeof(int)) != cudaSuccess) {
+    if (st->split_ws) cudaFree(st->split_ws);
+    if (st->split_counters) cudaFree(st->split_counters);
+    delete st;
+    return nullptr;
+  }
   return st;
 }
 
-void tc_state_destroy(void* s) { delete static_cast<TcState*>(s); }
+void tc_state_destroy(void* s) {
+  TcState* st = static_cast<TcState*>(s);
+  if (!st) return;
+  if (st->split_ws) cudaFree(st->split_ws);
+  if (st->split_counters) cudaFree(st->split_counters);
+  delete st;
+}
 
 bool launch_gemm_tc(const GemmArgs& a, void* tc_state, int* status, cudaStream_t stream) {
   TcState* st = static_cast<TcState*>(tc_state);
@@ -473,21 +563,54 @@ bool launch_gemm_tc(const GemmArgs& a, void* tc_state, int* status, cudaStream_t
   ep.head_dim = a.head_dim;
   ep.status = status;
   const bool swiglu = a.epi == EPI_SWIGLU;
-  // widest tile that still gives every SM a tile; rotary tiles must hold whole heads
+  // Choose the tile width by a small cost model in microseconds, calibrated on B200: time = waves x k-blocks x
+  // (tensor time of one k-block at that width).  K is split only for thin problems (M <= 64) with a long K,
+  // where the partial tiles are small and the extra units fill the machine; the fixed hand-over of a split
+  // (fence, counter, reduction read) costs about as much as 16 k-blocks.  Rotary tiles must hold whole heads.
   const int mt = (a.M + BM - 1) / BM;
-  auto tiles = [&](int bn) { const int per = swiglu ? bn / 2 : bn; return mt * ((a.N + per - 1) / per); };
-  int bn = 64;
-  if (tiles(256) >= st->n_sm) bn = 256;
-  else if (tiles(128) >= st->n_sm) bn = 128;
-  if (a.epi == EPI_QKV_ROPE && bn < a.head_dim) bn = a.head_dim;
-  if (swiglu && (a.N % (bn / 2))) bn = 64;
+  const int KB = a.K / BK;
+  int best_bn = 0, best_s = 1;
+  double best_t = 1e30;
+  const int bns[3] = {256, 128, 64};
+  const double kb_tensor[3] = {0.44, 0.27, 0.22};
+  for (int bi = 0; bi < 3; ++bi) {
+    const int bn = bns[bi];
+    const int per = swiglu ? bn / 2 : bn;
+    if (a.epi == EPI_QKV_ROPE && (bn < a.head_dim || a.N % bn)) continue;
+    if (swiglu && (a.N % per)) continue;
+    const int tiles = mt * ((a.N + per - 1) / per);
+    const int max_split = (a.M <= 64 && KB >= 128) ? 4 : 1;
+    for (int sp = 1; sp <= max_split; ++sp) {
+      const long long units = (long long)tiles * sp;
+      if (sp > 1 && (units > kSplitCounters || (size_t)units * BM * bn * 4 > kSplitWsBytes)) break;
+      const long long waves = (units + st->n_sm - 1) / st->n_sm;
+      double t = (double)waves * ((KB + sp - 1) / sp) * kb_tensor[bi];
+      if (sp > 1) t += 4.0;
+      if (t < best_t) {
+        best_t = t;
+        best_bn = bn;
+        best_s = sp;
+      }
+    }
+  }
+  if (st->force_bn) {   // tuning aid: RECG_GEMM_FORCE="<bn>,<splits>"; ignored where it does not fit
+    const int bn = st->force_bn, sp = st->force_s;
+    const int per = swiglu ? bn / 2 : bn;
+    const long long units = (long long)mt * ((a.N + per - 1) / per) * sp;
+    const bool shape_ok = (bn == 256 || bn == 128 || bn == 64) && sp >= 1 && sp <= KB &&
+                          !(a.epi == EPI_QKV_ROPE && (bn < a.head_dim || a.N % bn)) && !(swiglu && (a.N % per));
+    const bool fits = sp == 1 || (units <= kSplitCounters && (size_t)units * BM * bn * 4 <= kSplitWsBytes);
+    if (shape_ok && fits) {
+      best_bn = bn;
+      best_s = sp;
+    }
+  }
+  if (!best_bn) return false;
   if (swiglu && (a.N % 32)) return false;
-  if (a.epi == EPI_QKV_ROPE && (a.N % bn)) bn = a.head_dim;
-  if (a.epi == EPI_QKV_ROPE && (a.N % bn)) return false;
-  switch (bn) {
-    case 256: return launch_bn<256>(st, 0, a, ep, stream);
-    case 128: return launch_bn<128>(st, 1, a, ep, stream);
-    default: return launch_bn<64>(st, 2, a, ep, stream);
+  switch (best_bn) {
+    case 256: return launch_bn<256>(st, 0, a, ep, best_s, stream);
+    case 128: return launch_bn<128>(st, 1, a, ep, best_s, stream);
+    default: return launch_bn<64>(st, 2, a, ep, best_s, stream);
   }
 }
 

@@ -198,7 +198,7 @@ __global__ void kv_io_kernel(bool write, __nv_bfloat16* pool, int64_t n_pages, i
     return;
   }
   const size_t base = kv_tile_base(n_pages, n_kv, head_dim, layer, page, hk);
-  const int off = kv_tile_offset(p % kPageSize, c * 8);
+  const int off = kv_tile_offset(p % kPageSize, c * 8, head_dim);
   uint4* pk = reinterpret_cast<uint4*>(pool + base + off);
   uint4* pv = reinterpret_cast<uint4*>(pool + base + kv_tile_elems(head_dim) + off);
   const size_t lin = ((size_t)blockIdx.x * n_kv + hk) * head_dim + c * 8;

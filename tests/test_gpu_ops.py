@@ -206,7 +206,8 @@ def test_verify_commit_indices_and_continuation():
 # ---------------------------------------------------------------- projection
 @pytest.mark.parametrize("flags", [0, binding.FLAG_SIMT_GEMM])
 @pytest.mark.parametrize("M,N,K", [(1, 128, 64), (31, 256, 256), (128, 512, 1024), (129, 6144, 4096), (300, 4096, 14336),
-                                   (77, 2048, 256), (515, 1024, 4096)])
+                                   (77, 2048, 256), (515, 1024, 4096), (32, 4096, 4096), (32, 4096, 14336),
+                                   (470, 4096, 14336), (16, 6144, 4096), (130, 128256, 4096)])
 def test_linear(M, N, K, flags):
     shape = synth.tiny_shape()
     ctx = ops_ctx(shape, 1, 8, 1, flags)
@@ -220,6 +221,8 @@ def test_linear(M, N, K, flags):
     assert err < 1e-4, err      # fp32 accumulation of exact bf16 products: ~sqrt(K) 2^-24 relative, K <= 14336
     yb = ctx.recg_linear(x.cuda(), w.cuda(), torch.bfloat16)
     assert np.max(np.abs(f64(yb) - ref)) / np.max(np.abs(ref)) < 5e-3
+    y2 = ctx.recg_linear(x.cuda(), w.cuda(), torch.float32)      # K-split partials are reduced in a fixed order
+    assert torch.equal(y, y2)
     ctx.recg_free()
 
 
