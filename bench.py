@@ -255,6 +255,7 @@ def run_ours(args, env):
         out["attention_op"] = bench_attention_op(binding, peaks, args)
         out["verify_sweep"] = bench_verify(binding, peaks)
         out["c1"] = bench_c1(binding, ctx, shape, pool, n_pages, peaks, args)
+        out["gemm_shapes"] = bench_gemm_shapes(binding, peaks)
         out["cpu_baseline"] = cpu_baseline(shape, descs[0])
     ctx.recg_free()
     return out
@@ -314,6 +315,41 @@ def bench_attention_op(binding, peaks, args, desc=None, n_layers=32, label=None)
             "us_per_call": round(us, 2), "calls_include": "attention kernel + combine kernel", "algorithmic_bytes": int(kv_bytes),
             "gbs": round(gbs, 1), "frac_of_hbm_measured": round(gbs / peaks["hbm_gbs"], 4),
             "frac_of_8000": round(gbs / 8000.0, 4)}
+
+
+def bench_gemm_shapes(binding, peaks):
+    """The five projection shapes of one 8B-class layer (+ LM head) as standalone y = x w^T calls (plain epilogue)."""
+    shape = synth.tiny_shape()
+    shape.n_layers = 1
+    ctx = binding.Context(binding.make_config(shape, 1, 8, 1))
+    out = []
+    for M in (32, 480, 1331):
+        for name, N, K in (("qkv", 6144, 4096), ("o", 4096, 4096), ("gate_up", 28672, 4096), ("down", 4096, 14336),
+                           ("lm_head", 128256, 4096)):
+            g = torch.Generator(device="cuda")
+            g.manual_seed(M + N)
+            x = torch.randn((M, K), generator=g, device="cuda").to(torch.bfloat16)
+            w = (torch.randn((N, K), generator=g, device="cuda") * 0.02).to(torch.bfloat16)
+            y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+            call = lambda: binding.lib().recg_linear(ctx.h, x.data_ptr(), w.data_ptr(), y.data_ptr(), M, N, K, 0)
+            for _ in range(3):
+                call()
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(10):
+                call()
+            e1.record()
+            torch.cuda.synchronize()
+            us = e0.elapsed_time(e1) / 10 * 1e3
+            tf = 2.0 * M * N * K / (us * 1e-6) / 1e12
+            gbs = N * K * 2 / (us * 1e-6) / 1e9
+            out.append({"M": M, "name": name, "N": N, "K": K, "us": round(us, 1), "tflops": round(tf, 1),
+                        "frac_of_bf16_burst": round(tf / peaks["bf16_tflops"], 4), "weight_gbs": round(gbs, 1),
+                        "frac_of_hbm_measured": round(gbs / peaks["hbm_gbs"], 4)})
+            del x, w, y
+    ctx.recg_free()
+    return out
 
 
 def bench_verify(binding, peaks):
@@ -453,7 +489,7 @@ def main():
     ap.add_argument("--steps", type=int, default=8)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--only", default="", help="comma list of op-level sections to run alone (attention_op, verify_sweep): "
+    ap.add_argument("--only", default="", help="comma list of op-level sections to run alone (attention_op, attention_c16, verify_sweep, gemm_shapes): "
                                                "small cases for profiling; prints their JSON and exits")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
@@ -477,6 +513,8 @@ def main():
                                                     "U[512,8192], 4 layer caches rotated, CUDA-graph replay")
             elif sec == "verify_sweep":
                 res[sec] = bench_verify(binding, peaks)
+            elif sec == "gemm_shapes":
+                res[sec] = bench_gemm_shapes(binding, peaks)
         print(json.dumps(res), flush=True)
         return
     env = DistEnv.from_env(backend="nccl")
