@@ -353,32 +353,34 @@ def bench_gemm_shapes(binding, peaks):
 
 
 def bench_verify(binding, peaks):
-    """configs[4]: verify kernel sweep over bf16 logits [B (k+1), 128256]."""
+    """configs[4]: verify kernel sweep over bf16 logits [B (k+1), 128256]; copies of the logits are rotated so
+    that the scan does not sit in L2, and one rotation is replayed from a CUDA graph (kernel time, not launch latency)."""
     V = 128256
     res = []
     shape = synth.ModelShape(n_layers=0, hidden=64, n_q_heads=4, n_kv_heads=2, head_dim=64, ffn=64, vocab=V)
     for B, k in [(1, 4), (8, 8), (32, 16), (128, 16), (256, 32)]:
         R = B * (k + 1)
-        ctx = binding.Context(binding.make_config(shape, B, R, 1))
-        lg = synth.logits_normal(R, V, seed=6, device="cuda")
-        y = synth.token_ids(R, V, seed=1)
-        batch = binding.Batch([0] * B, [k + 1] * B, [0] * B, y)
-        vout = binding.VerifyOut(B, R, R, host=False)
-        ctx.recg_verify(batch, lg, out=vout)
-        n_rot = max(1, int(np.ceil(300e6 / (R * V * 2))))       # rotate copies so that the scan does not sit in L2
-        copies = [lg] + [lg.clone() for _ in range(min(n_rot, 64) - 1)]
-        torch.cuda.synchronize()
-        iters = 20
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        for i in range(iters):
-            ctx.recg_verify(None, copies[i % len(copies)], out=vout)
-        e1.record()
-        torch.cuda.synchronize()
-        us = e0.elapsed_time(e1) / iters * 1e3
+        stream = torch.cuda.Stream()
+        with torch.cuda.stream(stream):
+            ctx = binding.Context(binding.make_config(shape, B, R, 1), stream=stream.cuda_stream)
+            lg = synth.logits_normal(R, V, seed=6, device="cuda")
+            y = synth.token_ids(R, V, seed=1)
+            batch = binding.Batch([0] * B, [k + 1] * B, [0] * B, y)
+            vout = binding.VerifyOut(B, R, R, host=False)
+            ctx.recg_verify(batch, lg, out=vout)
+            n_rot = max(2, min(64, int(np.ceil(300e6 / (R * V * 2)))))
+            copies = [lg] + [lg.clone() for _ in range(n_rot - 1)]
+            stream.synchronize()
+
+        def rotation():
+            for c in copies:
+                ctx.recg_verify(None, c, out=vout)
+
+        us = _time_graph(stream, rotation, 5) / len(copies)
         gbs = R * V * 2 / (us * 1e-6) / 1e9
         res.append({"B": B, "k": k, "rows": R, "us": round(us, 2), "gbs": round(gbs, 1),
                     "frac_of_hbm_measured": round(gbs / peaks["hbm_gbs"], 4)})
+        ctx.recg_sync()
         ctx.recg_free()
         del copies, lg
         torch.cuda.empty_cache()

@@ -110,7 +110,7 @@ struct VerifyBuffers {   // DEVICE outputs (library workspace or caller buffers)
 struct RowPartial {      // per (row, vocab chunk)
   float m1, m2;          // largest and second-largest logit of the chunk
   int i1, i2;
-  float s, t;            // sum exp(x - m1), sum (x - m1) exp(x - m1)
+  float s, t;            // sum exp(x - m1), sum x exp(x - m1)
 };
 void launch_verify(const BatchLayout& bl, const void* logits, int logits_dtype, int vocab, RowPartial* partials,
                    int max_chunks_total, const VerifyBuffers& vb, int n_sm, cudaStream_t st);

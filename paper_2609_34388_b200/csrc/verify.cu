@@ -26,24 +26,27 @@ __device__ __forceinline__ void top2_insert(Top2& t, float x, int i) {
   }
 }
 
-// running softmax mass relative to a moving maximum m: s = sum e^(x-m), t = sum (x-m) e^(x-m)
+// running softmax mass relative to a moving maximum m: s = sum e^(x-m), t = sum x e^(x-m)
+// (entropy = ln s - t/s + m).  Logits of -inf contribute nothing: they are clamped to a finite value whose
+// exponential underflows to zero, so that x * 0 stays 0.
 struct Mass {
   float m, s, t;
 };
+constexpr float kLog2e = 1.4426950408889634f;
 __device__ __forceinline__ void mass_rebase(Mass& a, float m_new) {
   if (m_new > a.m) {
-    const float d = a.m - m_new;  // <= 0 ; a.m may be -inf with s = t = 0
-    const float e = a.s > 0.f ? __expf(d) : 0.f;
-    a.t = e * (a.t + (a.s > 0.f ? d * a.s : 0.f));
-    a.s = e * a.s;
+    const float f = a.s > 0.f ? exp2f((a.m - m_new) * kLog2e) : 0.f;   // a.m may be -inf with s = t = 0
+    a.s *= f;
+    a.t *= f;
     a.m = m_new;
   }
 }
-__device__ __forceinline__ void mass_add(Mass& a, float x) {
-  const float d = x - a.m;
-  const float e = __expf(d);
+// neg_m2 = -m * log2(e), hoisted by the caller
+__device__ __forceinline__ void mass_add(Mass& a, float x, float neg_m2) {
+  const float xc = fmaxf(x, -3.0e38f);
+  const float e = exp2f(fmaf(xc, kLog2e, neg_m2));
   a.s += e;
-  a.t += d * e;
+  a.t = fmaf(xc, e, a.t);
 }
 __device__ __forceinline__ void mass_merge(Mass& a, const Mass& b) {
   if (b.s <= 0.f) return;
@@ -59,7 +62,10 @@ template <typename T> struct Vec;
 template <> struct Vec<__nv_bfloat16> {
   static constexpr int N = 8;
   __device__ static void load(const __nv_bfloat16* p, float (&x)[8]) {
-    uint4 u = __ldg(reinterpret_cast<const uint4*>(p));
+    uint4 u;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(u.x), "=r"(u.y), "=r"(u.z), "=r"(u.w)
+                 : "l"(p));
     const uint32_t w[4] = {u.x, u.y, u.z, u.w};
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
@@ -94,29 +100,41 @@ __global__ void __launch_bounds__(kVerifyThreads) verify_partial_kernel(const T*
   int done = c0;
   if (vec_ok) {
     const int nvec = (c1 - c0) / N;
-    // two vectors in flight per thread
+    // Four 16-byte loads in flight per thread.  In the loop the top-2 bookkeeping is branch-free and per VECTOR:
+    // each thread remembers its two vectors with the largest maximum (the two largest elements it has seen lie
+    // in those two vectors; strict comparisons keep the earlier vector on ties), and only after the loop are
+    // these two vectors re-read and searched element by element.  A per-element test would diverge in nearly
+    // every warp and cost more issue slots than the arithmetic.
+    float bv1 = -INFINITY, bv2 = -INFINITY;   // two largest vector maxima of this thread
+    int bi1 = -1, bi2 = -1;                   // their vector indices
+    auto track = [&](float vmax, int vec) {
+      const bool g1 = vmax > bv1, g2 = vmax > bv2;
+      bi2 = g1 ? bi1 : (g2 ? vec : bi2);
+      bv2 = g1 ? bv1 : (g2 ? vmax : bv2);
+      bi1 = g1 ? vec : bi1;
+      bv1 = g1 ? vmax : bv1;
+    };
     int i = threadIdx.x;
-    for (; i + kVerifyThreads < nvec; i += 2 * kVerifyThreads) {
-      float x[N], y[N];
-      Vec<T>::load(base + c0 + (size_t)i * N, x);
-      Vec<T>::load(base + c0 + (size_t)(i + kVerifyThreads) * N, y);
-      float vm = x[0];
+    for (; i + 3 * kVerifyThreads < nvec; i += 4 * kVerifyThreads) {
+      float x[4][N];
 #pragma unroll
-      for (int k = 1; k < N; ++k) vm = fmaxf(vm, x[k]);
+      for (int u = 0; u < 4; ++u) Vec<T>::load(base + c0 + (size_t)(i + u * kVerifyThreads) * N, x[u]);
+      float vm[4];
 #pragma unroll
-      for (int k = 0; k < N; ++k) vm = fmaxf(vm, y[k]);
-      mass_rebase(ms, vm);
-      const int ix = c0 + i * N, iy = c0 + (i + kVerifyThreads) * N;
+      for (int u = 0; u < 4; ++u) {
+        vm[u] = x[u][0];
+#pragma unroll
+        for (int k = 1; k < N; ++k) vm[u] = fmaxf(vm[u], x[u][k]);
+      }
+      mass_rebase(ms, fmaxf(fmaxf(vm[0], vm[1]), fmaxf(vm[2], vm[3])));
+      const float neg = ms.m > -INFINITY ? -ms.m * kLog2e : 0.f;   // all -inf so far: every term underflows to 0
 #pragma unroll
       for (int k = 0; k < N; ++k) {
-        mass_add(ms, x[k]);
-        if (x[k] >= tp.m2) top2_insert(tp, x[k], ix + k);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) mass_add(ms, x[u][k], neg);
       }
 #pragma unroll
-      for (int k = 0; k < N; ++k) {
-        mass_add(ms, y[k]);
-        if (y[k] >= tp.m2) top2_insert(tp, y[k], iy + k);
-      }
+      for (int u = 0; u < 4; ++u) track(vm[u], i + u * kVerifyThreads);
     }
     for (; i < nvec; i += kVerifyThreads) {
       float x[N];
@@ -125,19 +143,28 @@ __global__ void __launch_bounds__(kVerifyThreads) verify_partial_kernel(const T*
 #pragma unroll
       for (int k = 1; k < N; ++k) vm = fmaxf(vm, x[k]);
       mass_rebase(ms, vm);
-      const int ix = c0 + i * N;
+      const float neg = ms.m > -INFINITY ? -ms.m * kLog2e : 0.f;   // all -inf so far: every term underflows to 0
 #pragma unroll
-      for (int k = 0; k < N; ++k) {
-        mass_add(ms, x[k]);
-        if (x[k] >= tp.m2) top2_insert(tp, x[k], ix + k);
-      }
+      for (int k = 0; k < N; ++k) mass_add(ms, x[k], neg);
+      track(vm, i);
+    }
+    // element-level search of the two remembered vectors (in index order, so that ties resolve to the lowest index)
+    const int lo_vec = bi2 < 0 ? bi1 : min(bi1, bi2), hi_vec = bi2 < 0 ? -1 : max(bi1, bi2);
+    const int cand[2] = {lo_vec, hi_vec};
+#pragma unroll
+    for (int q = 0; q < 2; ++q) {
+      if (cand[q] < 0) continue;
+      float x[N];
+      Vec<T>::load(base + c0 + (size_t)cand[q] * N, x);
+#pragma unroll
+      for (int k = 0; k < N; ++k) top2_insert(tp, x[k], c0 + cand[q] * N + k);
     }
     done = c0 + nvec * N;
   }
   for (int i = done + threadIdx.x; i < c1; i += kVerifyThreads) {
     const float x = Vec<T>::one(base + i);
     mass_rebase(ms, x);
-    mass_add(ms, x);
+    mass_add(ms, x, ms.m > -INFINITY ? -ms.m * kLog2e : 0.f);
     if (x >= tp.m2) top2_insert(tp, x, i);
   }
   // warp reduce, then across warps through shared memory
@@ -201,7 +228,7 @@ __global__ void __launch_bounds__(128) verify_finalize_kernel(BatchLayout bl, co
     vb.top2[t0 + j] = tp.i2;
     vb.p1[t0 + j] = inv;                             // e^(m1 - m1) / S
     vb.p2[t0 + j] = __expf(tp.m2 - tp.m1) * inv;
-    vb.entropy[t0 + j] = logf(ms.s) - ms.t * inv;    // ln S - (1/S) sum (x-M) e^(x-M)
+    vb.entropy[t0 + j] = logf(ms.s) - ms.t * inv + ms.m;   // ln S - (1/S) sum x e^(x-M) + M
   }
   __syncthreads();
   __shared__ int s_a;
@@ -307,7 +334,7 @@ __global__ void row_stats_finalize_kernel(const RowPartial* __restrict__ partial
   if (top2) top2[r] = tp.i2;
   if (p1) p1[r] = inv;
   if (p2) p2[r] = __expf(tp.m2 - tp.m1) * inv;
-  if (entropy) entropy[r] = logf(ms.s) - ms.t * inv;
+  if (entropy) entropy[r] = logf(ms.s) - ms.t * inv + ms.m;
 }
 
 }  // namespace
