@@ -353,37 +353,45 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attention_kernel(AttnParams P
   }
 }
 
-// grid (T, n_q), D/4 threads: merges the KV-range partials of one (token, head) row.
+// Merges the KV-range partials of the tiles that were split.  A small persistent grid strides over the (tile, row)
+// table; tiles with a single part were written by the attention kernel itself and are skipped.  One warp per
+// query row, each lane D/32 consecutive dims.
 template <int D>
-__global__ void attention_combine_kernel(BatchLayout bl, int n_q, int group, int tok_per_tile,
-                                         const float* __restrict__ part_o, const float* __restrict__ part_ml,
-                                         __nv_bfloat16* __restrict__ o) {
-  const int t = blockIdx.x, h = blockIdx.y;
-  const int r = bl.tok_req[t];
-  const int j = t - bl.cu_tok[r];
-  const int n = bl.verify_len[r] + bl.block_size[r];
-  const int tiles = (n + tok_per_tile - 1) / tok_per_tile;
-  const int tile = j / tok_per_tile;
-  const int kvh = h / group;
-  const AttnTile tl = bl.tiles[bl.tile_off[r] + kvh * tiles + tile];
-  if (tl.n_parts <= 1) return;  // the attention kernel wrote this row itself
-  const int rho = (j % tok_per_tile) * group + (h % group);
-  float m = -1e30f;
-  for (int p = 0; p < tl.n_parts; ++p) m = fmaxf(m, part_ml[((size_t)(tl.part_begin + p) * 128 + rho) * 2]);
-  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-  float l = 0.f;
-  for (int p = 0; p < tl.n_parts; ++p) {
-    const size_t row = (size_t)(tl.part_begin + p) * 128 + rho;
-    const float wgt = exp2f(part_ml[row * 2] - m);
-    l += wgt * part_ml[row * 2 + 1];
-    const float4 v = reinterpret_cast<const float4*>(part_o + row * D)[threadIdx.x];
-    acc.x += wgt * v.x; acc.y += wgt * v.y; acc.z += wgt * v.z; acc.w += wgt * v.w;
+__global__ void __launch_bounds__(512) attention_combine_kernel(const AttnTile* __restrict__ tiles,
+                                                                const int* __restrict__ counts, int n_q, int group,
+                                                                const float* __restrict__ part_o,
+                                                                const float* __restrict__ part_ml,
+                                                                __nv_bfloat16* __restrict__ o) {
+  constexpr int E = D / 32;
+  const int n_tiles = counts[1];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  // work unit = 16 rows of a tile: units are strided over the grid, a CTA's 16 warps take one row each
+  for (int wu = blockIdx.x; wu < n_tiles * 8; wu += gridDim.x) {
+    const AttnTile tl = tiles[wu >> 3];
+    if (tl.n_parts <= 1) continue;
+    const int rho = (wu & 7) * 16 + warp;
+    if (rho < tl.ntok * group) {
+      float m = -1e30f;
+      for (int p = 0; p < tl.n_parts; ++p) m = fmaxf(m, part_ml[((size_t)(tl.part_begin + p) * 128 + rho) * 2]);
+      float acc[E];
+#pragma unroll
+      for (int e = 0; e < E; ++e) acc[e] = 0.f;
+      float l = 0.f;
+      for (int p = 0; p < tl.n_parts; ++p) {
+        const size_t row = (size_t)(tl.part_begin + p) * 128 + rho;
+        const float wgt = exp2f(part_ml[row * 2] - m);
+        l += wgt * part_ml[row * 2 + 1];
+        const float* src = part_o + row * D + lane * E;
+#pragma unroll
+        for (int e = 0; e < E; ++e) acc[e] += wgt * src[e];
+      }
+      const float inv = l > 0.f ? 1.f / l : 0.f;
+      const int j = rho / group, hg = rho % group;
+      __nv_bfloat16* dst = o + ((size_t)(tl.tok0 + j) * n_q + tl.kv_head * group + hg) * D + lane * E;
+#pragma unroll
+      for (int e = 0; e < E; e += 2) *reinterpret_cast<uint32_t*>(dst + e) = pack_bf16(acc[e] * inv, acc[e + 1] * inv);
+    }
   }
-  const float inv = l > 0.f ? 1.f / l : 0.f;
-  uint2 out;
-  out.x = pack_bf16(acc.x * inv, acc.y * inv);
-  out.y = pack_bf16(acc.z * inv, acc.w * inv);
-  reinterpret_cast<uint2*>(o + ((size_t)t * n_q + h) * D)[threadIdx.x] = out;
 }
 
 template <int D>
@@ -416,9 +424,8 @@ void launch_attention_t(const BatchLayout& bl, const Dims& dm, int layer, const 
   P.part_ml = part_ml;
   P.status = status;
   attention_kernel<D><<<n_sm, kAttnThreads, AttnSmem<D>::kTotal, st>>>(P);
-  dim3 grid(bl.n_tok, dm.n_q);
-  attention_combine_kernel<D><<<grid, D / 4, 0, st>>>(bl, dm.n_q, P.group, tok_per_tile, part_o, part_ml,
-                                                       static_cast<__nv_bfloat16*>(o));
+  attention_combine_kernel<D><<<2 * n_sm, 512, 0, st>>>(bl.tiles, bl.counts, dm.n_q, P.group, part_o, part_ml,
+                                                        static_cast<__nv_bfloat16*>(o));
 }
 
 }  // namespace
@@ -432,9 +439,8 @@ void launch_attention(const BatchLayout& bl, const Dims& dm, int layer, const vo
                       cudaStream_t st, bool use_tc) {
   if (use_tc && dm.head_dim == 128) {
     launch_attention_tc_main(bl, dm, layer, q, o, kv_pool, n_pages, part_o, part_ml, n_sm, status, st);
-    dim3 grid(bl.n_tok, dm.n_q);
-    attention_combine_kernel<128><<<grid, 32, 0, st>>>(bl, dm.n_q, dm.n_q / dm.n_kv, tok_per_tile, part_o, part_ml,
-                                                       static_cast<__nv_bfloat16*>(o));
+    attention_combine_kernel<128><<<2 * n_sm, 512, 0, st>>>(bl.tiles, bl.counts, dm.n_q, dm.n_q / dm.n_kv, part_o, part_ml,
+                                                            static_cast<__nv_bfloat16*>(o));
     return;
   }
   if (dm.head_dim == 64)

@@ -137,6 +137,11 @@ constexpr uint32_t kIdescQK = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(k
 constexpr uint32_t kIdescPV =
     (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(D >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
 
+// Two non-negative fp32 values to packed bf16, rounding to nearest (ties away from zero) with integer adds and
+// one byte permute: keeps the conversion off the transcendental unit, which already carries every exp2.
+__device__ __forceinline__ uint32_t pack_bf16_alu(uint32_t lo_bits, uint32_t hi_bits) {
+  return __byte_perm(lo_bits + 0x8000u, hi_bits + 0x8000u, 0x7632);
+}
 __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
   asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }

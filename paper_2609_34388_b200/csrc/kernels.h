@@ -19,8 +19,9 @@ struct AttnItem {
   int part;              // index into the partial buffers, or -1 when the item covers the whole KV range
   int kv_len;            // L + n of the request
 };
-struct AttnTile {        // per (request, kv head, row tile): where its partials are
+struct AttnTile {        // per (request, kv head, row tile): where its partials are, and which rows it covers
   int part_begin, n_parts;
+  int tok0, ntok, kv_head;
 };
 
 // Device-resident ragged layout of one batch (all pointers DEVICE, int32 unless noted).

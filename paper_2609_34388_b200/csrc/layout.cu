@@ -127,6 +127,9 @@ __global__ void __launch_bounds__(1024) layout_kernel(BatchLayout bl, int n_kv, 
       AttnTile tl;
       tl.part_begin = parts > 1 ? part : -1;
       tl.n_parts = parts;
+      tl.tok0 = bl.cu_tok[r] + tile * tok_per_tile;
+      tl.ntok = min(tok_per_tile, n - tile * tok_per_tile);
+      tl.kv_head = kvh;
       bl.tiles[tile_off[r] + k] = tl;
       for (int c = c_first; c <= c_last; ++c, ++item) {
         const int gs = max(g0, c * per), ge = min(g1, (c + 1) * per);
