@@ -128,35 +128,16 @@ __device__ __forceinline__ uint64_t desc_mnmajor(uint32_t addr, uint32_t lbo_byt
   return (uint64_t)((addr & 0x3ffff) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) | ((uint64_t)(sbo_bytes >> 4) << 32) |
          ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
 }
-__device__ __forceinline__ void l2_prefetch(const void* gptr, uint32_t bytes) {
-  asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(gptr), "r"(bytes) : "memory");
-}
 // S / P column c of a 128-token block holds token c
 __device__ __forceinline__ int col_token(int c) { return c; }
 constexpr uint32_t kIdescQK = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kBT >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
 constexpr uint32_t kIdescPV =
     (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(D >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
 
-// Two non-negative fp32 values to packed bf16, rounding to nearest (ties away from zero) with integer adds and
-// one byte permute: keeps the conversion off the transcendental unit, which already carries every exp2.
-__device__ __forceinline__ uint32_t pack_bf16_alu(uint32_t lo_bits, uint32_t hi_bits) {
-  return __byte_perm(lo_bits + 0x8000u, hi_bits + 0x8000u, 0x7632);
-}
 __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
   asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
 __device__ __forceinline__ void softmax_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
-
-#ifdef RECG_TRACE
-__device__ unsigned long long g_cta[256][4];
-__device__ unsigned long long g_item[16][8];
-#define ITRACE(it, slot) do { if (blockIdx.x == 29 && warp == 2 && lane == 0 && (it) < 16) { unsigned long long t_; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_)); g_item[it][slot] = t_; } } while (0)
-__device__ unsigned long long g_trace[3][64][8];
-#define TRACE(role, step, slot) do { if (blockIdx.x == 29 && (step) < 64) { unsigned long long t_; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_)); g_trace[role][step][slot] = t_; } } while (0)
-#else
-#define TRACE(role, step, slot) do { } while (0)
-#define ITRACE(it, slot) do { } while (0)
-#endif
 
 __global__ void __launch_bounds__(kThreads, 1) attention_tc_kernel(TcAttnParams P) {
   extern __shared__ uint8_t smem_raw[];
@@ -174,9 +155,6 @@ __global__ void __launch_bounds__(kThreads, 1) attention_tc_kernel(TcAttnParams 
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + kNumBars);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-#ifdef RECG_TRACE
-  if (threadIdx.x == 0) { unsigned long long t_; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_)); g_cta[blockIdx.x][0] = t_; }
-#endif
   if (threadIdx.x == 0) {
     for (int s = 0; s < kKVStages; ++s) {
       mbar_init(&kv_full[s], 1);
@@ -223,14 +201,11 @@ __global__ void __launch_bounds__(kThreads, 1) attention_tc_kernel(TcAttnParams 
       const int nblk = (tok_end - tok_begin + kBT - 1) / kBT;
       const int n_req_pages = (w.kv_len + kPageSize - 1) / kPageSize;
       const int* pt = P.page_table + (size_t)w.req * P.pt_stride;
-      // page ids are fetched in parallel one iteration ahead of their use: lanes 0..7 for the block that is
-      // copied next, lanes 8..15 for the block two further on, which they prefetch into L2
+      // page ids are fetched by lanes 0..7 in parallel, one iteration ahead of their use
       auto fetch_page = [&](int n) -> int {
         int pg = -1;
-        const int grp = lane >> 3;                   // 0: copy, 1: prefetch
-        const int nb = n + 2 * grp;
-        if (lane < 2 * kPagesPerBT && nb < nblk) {
-          const int lp = tok_begin / kPageSize + nb * kPagesPerBT + (lane & 7);
+        if (lane < kPagesPerBT && n < nblk) {
+          const int lp = tok_begin / kPageSize + n * kPagesPerBT + lane;
           if (lp < n_req_pages && lp * kPageSize < tok_end) pg = __ldg(pt + lp);   // validated when used
         }
         return pg;
@@ -243,8 +218,6 @@ __global__ void __launch_bounds__(kThreads, 1) attention_tc_kernel(TcAttnParams 
           set_status(P.status, DEV_BAD_INDEX);
           my_pg = -1;
         }
-        if (false && lane >= kPagesPerBT && lane < 2 * kPagesPerBT && my_pg >= 0)
-          l2_prefetch(P.pool + kv_tile_base(P.n_pages, P.n_kv, D, P.layer, my_pg, w.kv_head), 2 * kTileBytes);
         // lane p < 8 owns page p of the block: full pages go by bulk copy, the rest by hand
         const int first_tok = tok_begin + (n * kPagesPerBT + lane) * kPageSize;
         const int my_valid = (lane < kPagesPerBT && my_pg >= 0) ? min(kPageSize, w.kv_len - first_tok) : 0;
@@ -262,7 +235,6 @@ __global__ void __launch_bounds__(kThreads, 1) attention_tc_kernel(TcAttnParams 
             ok = false;
             break;
           }
-          if (lane == 0) TRACE(0, blk, part * 2);
           uint8_t* stage = smem + kOffKV + s * kKVStageBytes;
           if (hand_mask) {
             const int p = __ffs(hand_mask) - 1;            // at most one partly filled page per request
@@ -293,7 +265,6 @@ __global__ void __launch_bounds__(kThreads, 1) attention_tc_kernel(TcAttnParams 
             bulk_g2s(stage + lane * kTileBytes, src, kTileBytes, &kv_full[s]);
           }
           __syncwarp();
-          if (lane == 0) TRACE(0, blk, part * 2 + 1);
         }
       }
     }
@@ -314,9 +285,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_tc_kernel(TcAttnParams 
         const uint32_t qi = 2 * b;
         const int s = qi % kKVStages, sb = b & 1;
         if (!mbar_wait(&kv_full[s], (qi / kKVStages) & 1, kSpin)) { set_status(P.status, DEV_TIMEOUT_FULL); return false; }
-        TRACE(1, b, 0);
         if (!mbar_wait(&s_empty[sb], ((b >> 1) & 1) ^ 1, kSpin)) { set_status(P.status, DEV_TIMEOUT_MMA); return false; }
-        TRACE(1, b, 1);
         tc_fence_after();
         const uint32_t k_addr = smem_base + kOffKV + s * kKVStageBytes;
 #pragma unroll
@@ -349,7 +318,6 @@ __global__ void __launch_bounds__(kThreads, 1) attention_tc_kernel(TcAttnParams 
             ok = false;
             break;
           }
-          TRACE(1, blk, 2);
           const uint32_t qv = 2 * blk + 1;
           const int s = qv % kKVStages;
           if (!mbar_wait(&kv_full[s], (qv / kKVStages) & 1, kSpin)) {
@@ -358,7 +326,6 @@ __global__ void __launch_bounds__(kThreads, 1) attention_tc_kernel(TcAttnParams 
             break;
           }
           tc_fence_after();
-          TRACE(1, blk, 3);
           const uint32_t v_addr = smem_base + kOffKV + s * kKVStageBytes;
 #pragma unroll
           for (int kk = 0; kk < kBT / 16; ++kk) {
@@ -370,7 +337,6 @@ __global__ void __launch_bounds__(kThreads, 1) attention_tc_kernel(TcAttnParams 
           umma_commit(&kv_empty[s]);
           umma_commit(&p_empty[pb]);
           if (n == nblk - 1) umma_commit(o_full);
-          TRACE(1, blk, 4);
         }
       }
     }
@@ -388,7 +354,6 @@ __global__ void __launch_bounds__(kThreads, 1) attention_tc_kernel(TcAttnParams 
       const int tok_begin = w.blk_begin * 64;
       const int tok_end = min(w.blk_end * 64, w.kv_len);
       const int nblk = (tok_end - tok_begin + kBT - 1) / kBT;
-      ITRACE(item_cnt, 0);
       // ---- stage Q in operand layout: [2 halves][128 rows][128 B], 16-byte chunks swizzled by row & 7 ----
       // only the R valid rows are staged: the other rows of the M = 128 operand yield S / O rows nobody reads.
       // Loads are issued in batches of 8 before any store so that their latencies overlap.
@@ -416,7 +381,6 @@ __global__ void __launch_bounds__(kThreads, 1) attention_tc_kernel(TcAttnParams 
       fence_proxy_async();
       softmax_bar();
       if (sthread == 0) mbar_arrive(q_full);
-      ITRACE(item_cnt, 1);
 
       const bool rvalid = row < R;
       const bool warp_valid = quad * 32 < R;
@@ -434,7 +398,6 @@ __global__ void __launch_bounds__(kThreads, 1) attention_tc_kernel(TcAttnParams 
         const int sb = blk & 1;
         if (!mbar_wait(&s_full[sb], (blk >> 1) & 1, kSpin)) { set_status(P.status, DEV_TIMEOUT_MMA); ok = false; break; }
         tc_fence_after();
-        if (warp == 4 && lane == 0) TRACE(2, blk, 0);
         const int pos0 = tok_begin + n * kBT;
         uint32_t sr[4][32];   // the S row of this thread: 128 scores
         float mx = -INFINITY;
@@ -476,12 +439,10 @@ __global__ void __launch_bounds__(kThreads, 1) attention_tc_kernel(TcAttnParams 
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(&s_empty[sb]);
-        if (warp == 4 && lane == 0) TRACE(2, blk, 1);
         // the P V that last read this P buffer (two blocks ago) must be complete before it is overwritten
         const int pb = pv_cnt & 1;
         const uint32_t p_row = p_row0 + pb * kPBytes;
         if (!mbar_wait(&p_empty[pb], ((pv_cnt >> 1) & 1) ^ 1, kSpin)) { set_status(P.status, DEV_TIMEOUT_MMA); ok = false; break; }
-        if (warp == 4 && lane == 0) TRACE(2, blk, 2);
         if (warp_valid) {
           const float m_blk = mx * P.scale_log2;
           // move the reference maximum only when the row maximum outgrows it by more than 2^8 (or at the first
@@ -535,15 +496,12 @@ __global__ void __launch_bounds__(kThreads, 1) attention_tc_kernel(TcAttnParams 
         fence_proxy_async();
         __syncwarp();
         if (lane == 0) mbar_arrive(&p_full[pb]);
-        if (warp == 4 && lane == 0) TRACE(2, blk, 3);
       }
       if (!ok) break;
 
-      ITRACE(item_cnt, 2);
       // ---- read O once, write out: one row per thread ----
       if (!mbar_wait(o_full, item_cnt & 1, kSpin)) { set_status(P.status, DEV_TIMEOUT_MMA); ok = false; break; }
       tc_fence_after();
-      ITRACE(item_cnt, 3);
       if (warp_valid) {
         const int j = row / P.group, hg = row % P.group;
         const float inv = (w.part < 0) ? (l_run > 0.f ? 1.f / l_run : 0.f) : 1.f;
@@ -578,7 +536,6 @@ __global__ void __launch_bounds__(kThreads, 1) attention_tc_kernel(TcAttnParams 
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(o_empty);
-      ITRACE(item_cnt, 4);
       ++item_cnt;
       // all MMAs of this item have completed (the last o_full tracked them), so Q may be restaged
       softmax_bar();
@@ -587,9 +544,6 @@ __global__ void __launch_bounds__(kThreads, 1) attention_tc_kernel(TcAttnParams 
 
   tc_fence_before();
   __syncthreads();
-#ifdef RECG_TRACE
-  if (threadIdx.x == 0) { unsigned long long t_; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_)); g_cta[blockIdx.x][1] = t_; g_cta[blockIdx.x][2] = P.cta_off[blockIdx.x + 1] - P.cta_off[blockIdx.x]; }
-#endif
   if (warp == 1) {
     tc_fence_after();
     tmem_dealloc(tmem_base, kTmemCols);
@@ -597,12 +551,6 @@ __global__ void __launch_bounds__(kThreads, 1) attention_tc_kernel(TcAttnParams 
 }
 
 }  // namespace
-
-#ifdef RECG_TRACE
-extern "C" void recg_debug_trace(unsigned long long* out) { cudaMemcpyFromSymbol(out, g_trace, sizeof(unsigned long long) * 3 * 64 * 8); }
-extern "C" void recg_debug_item(unsigned long long* out) { cudaMemcpyFromSymbol(out, g_item, sizeof(unsigned long long) * 16 * 8); }
-extern "C" void recg_debug_cta(unsigned long long* out) { cudaMemcpyFromSymbol(out, g_cta, sizeof(unsigned long long) * 256 * 4); }
-#endif
 
 void launch_attention_tc_main(const BatchLayout& bl, const Dims& dm, int layer, const void* q, void* o,
                               const void* kv_pool, int64_t n_pages, float* part_o, float* part_ml, int n_sm, int* status,

@@ -36,8 +36,17 @@ template <int BN> struct TcCfg {
   static constexpr int kBBytes = BN * BK * 2;
   static constexpr int kStageBytes = kABytes + kBBytes;
   static constexpr int kStages = (kSmemBudget / kStageBytes) > 8 ? 8 : (kSmemBudget / kStageBytes);
-  static constexpr int kBarBytes = (2 * kStages + 4) * 8 + 16;
-  static constexpr int kSmemBytes = kStages * kStageBytes + kBarBytes + 1024;  // + slack for 1024-byte alignment
+  static constexpr int kMaxStages = 16;
+  // thin problems (M <= 32) load only 32 rows of x per stage: the stage shrinks and more stages fit.  The MMA
+  // still reads 128 rows; rows 32.. alias the bytes that follow (harmless: those accumulator rows are never
+  // stored), so the ring is followed by a pad that keeps the last stage's read inside the allocation.
+  static constexpr int kThinABytes = 32 * BK * 2;
+  static constexpr int kThinStageBytes = kThinABytes + kBBytes;
+  static constexpr int kThinStages =
+      (kSmemBudget / kThinStageBytes) > kMaxStages ? kMaxStages : (kSmemBudget / kThinStageBytes);
+  static constexpr int kRingBytes = kSmemBudget + kABytes;     // either ring plus the pad
+  static constexpr int kBarBytes = (2 * kMaxStages + 4) * 8 + 16;
+  static constexpr int kSmemBytes = kRingBytes + kBarBytes + 1024;  // + slack for 1024-byte alignment
   static constexpr int kTmemCols = 2 * BN < 32 ? 32 : 2 * BN;                  // power of two: 128, 256, 512
 };
 
@@ -145,24 +154,79 @@ struct TmemLoader {
   __device__ __forceinline__ void operator()(int col, float (&v)[32]) const { tmem_ld32(tacc + col, v); }
 };
 struct SplitLoader {
-  const float* row0;      // partial of split 0, this thread's row
-  size_t split_stride;    // floats between consecutive splits' partial tiles
-  int n_splits;
+  const float* ws;        // partial-tile workspace; slot s holds a [BM][bn] fp32 tile
+  int bn, row;            // tile width, this thread's row in the tile
+  int slot0;              // slot of part 0
+  int slot_next;          // slot of part 1; part p >= 1 is in slot_next + 2 (p - 1)
+  int n_parts;
   bool valid;             // rows beyond M were never parked
   __device__ __forceinline__ void operator()(int col, float (&v)[32]) const {
 #pragma unroll
     for (int i = 0; i < 32; ++i) v[i] = 0.f;
     if (!valid) return;
-    for (int sp = 0; sp < n_splits; ++sp) {        // fixed order: the result does not depend on who arrived last
-      const float4* src = reinterpret_cast<const float4*>(row0 + sp * split_stride + col);
+    // partial tiles are stored [column / 4][row][4]: a warp's 32 rows of one float4 column are 512 contiguous
+    // bytes.  Parts are added in part order (the result does not depend on who arrived last); the loads of two
+    // parts are issued together so that their latencies overlap.
+    const float4* base = reinterpret_cast<const float4*>(ws) + (size_t)(col / 4) * BM + row;
+    for (int p = 0; p < n_parts; p += 2) {
+      const int sa = p == 0 ? slot0 : slot_next + 2 * (p - 1);
+      const bool two = p + 1 < n_parts;
+      const int sb = slot_next + 2 * p;             // slot of part p + 1 (>= 1)
+      float4 a[8], b[8];
 #pragma unroll
       for (int i = 0; i < 8; ++i) {
-        const float4 t = __ldcg(src + i);
-        v[4 * i] += t.x; v[4 * i + 1] += t.y; v[4 * i + 2] += t.z; v[4 * i + 3] += t.w;
+        a[i] = __ldcg(base + ((size_t)sa * (bn / 4) + i) * BM);
+        b[i] = two ? __ldcg(base + ((size_t)sb * (bn / 4) + i) * BM) : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        v[4 * i] += a[i].x; v[4 * i + 1] += a[i].y; v[4 * i + 2] += a[i].z; v[4 * i + 3] += a[i].w;
+        v[4 * i] += b[i].x; v[4 * i + 1] += b[i].y; v[4 * i + 2] += b[i].z; v[4 * i + 3] += b[i].w;
       }
     }
   }
 };
+
+// Work decomposition ("stream-K"): the k-blocks of all output tiles form one line of n_tiles * KB units, tile
+// after tile; CTA c owns the contiguous range [c * per, (c + 1) * per).  With per a multiple of KB every CTA owns
+// whole tiles; otherwise a tile may be cut by CTA boundaries, and each owner computes its K range of it ("part").
+// Part p >= 1 of a tile is always the FIRST piece of its CTA, part 0 the last piece of its CTA (or the first, when
+// the CTA's range starts exactly at the tile): that decides the workspace slot, 2 * cta + (first piece ? 0 : 1).
+struct Piece {
+  int tile, kb0, kb1;     // k-block range [kb0, kb1) of the tile
+  int part, n_parts;      // which part of the tile this is
+  int slot;               // workspace slot if n_parts > 1
+  int slot0, slot_next;   // slots of part 0 and part 1 (for the reducing CTA)
+};
+// j-th piece of this CTA: first its whole tiles, then its range of the stream-K line (pos advances by reference)
+__device__ __forceinline__ Piece make_piece(int j, int dp_count, int dp_tiles, long long& pos, long long hi, int KB,
+                                            long long per, int cta, int grid) {
+  Piece p;
+  if (j < dp_count) {
+    p.tile = cta + j * grid;
+    p.kb0 = 0;
+    p.kb1 = KB;
+    p.part = 0;
+    p.n_parts = 1;
+    p.slot = p.slot0 = p.slot_next = 0;
+    return p;
+  }
+  p.tile = (int)(pos / KB);
+  p.kb0 = (int)(pos - (long long)p.tile * KB);
+  const long long room = hi - pos;
+  p.kb1 = (int)(room < KB - p.kb0 ? p.kb0 + room : KB);
+  const long long t0 = (long long)p.tile * KB, t1 = t0 + KB;
+  const int c_first = (int)(t0 / per), c_last = (int)((t1 - 1) / per);
+  p.n_parts = c_last - c_first + 1;
+  p.part = cta - c_first;
+  const bool first_piece = pos == (long long)cta * per;
+  p.slot = 2 * cta + (first_piece ? 0 : 1);
+  p.slot0 = 2 * c_first + (((long long)c_first * per >= t0) ? 0 : 1);
+  p.slot_next = 2 * (c_first + 1);
+  p.tile += dp_tiles;
+  pos += p.kb1 - p.kb0;
+  return p;
+}
 
 // Epilogue of one accumulator tile for the calling thread's row.
 template <int BN, typename Loader>
@@ -262,25 +326,34 @@ __device__ __forceinline__ void row_epilogue(const EpiParams& ep, const Loader& 
 template <int BN>
 __global__ void __launch_bounds__(kTcThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w, int M, int n_tiles_n,
-               int K, int up_row_offset, int n_splits, float* split_ws, int* split_counters, EpiParams ep) {
+               int K, int up_row_offset, int dp_tiles, long long per, int thin, float* split_ws, int* split_counters,
+               EpiParams ep) {
   using Cfg = TcCfg<BN>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + Cfg::kStages * Cfg::kStageBytes);
-  uint64_t* empty_bar = full_bar + Cfg::kStages;
-  uint64_t* tfull_bar = empty_bar + Cfg::kStages;
+  const int n_stages = thin ? Cfg::kThinStages : Cfg::kStages;
+  const int a_bytes = thin ? Cfg::kThinABytes : Cfg::kABytes;
+  const int stage_bytes = a_bytes + Cfg::kBBytes;
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + Cfg::kRingBytes);
+  uint64_t* empty_bar = full_bar + Cfg::kMaxStages;
+  uint64_t* tfull_bar = empty_bar + Cfg::kMaxStages;
   uint64_t* tempty_bar = tfull_bar + 2;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tempty_bar + 2);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n_tiles_m = (M + BM - 1) / BM;
   const int n_tiles = n_tiles_m * n_tiles_n;
-  const int n_units = n_tiles * n_splits;   // a unit is (tile, K split); the splits of a tile are adjacent units
   const int KB = K / BK;
   const bool swiglu = ep.epi == EPI_SWIGLU;
+  // schedule: tiles [0, dp_tiles) whole, strided over the grid (CTAs that run together share a weight tile
+  // through L2); then the k-blocks of tiles [dp_tiles, n_tiles) as one line cut into equal ranges per CTA
+  const long long range_lo = (long long)blockIdx.x * per;
+  const long long total = (long long)(n_tiles - dp_tiles) * KB;
+  const long long range_hi = range_lo + per < total ? range_lo + per : total;
+  const int dp_count = blockIdx.x < dp_tiles ? (dp_tiles - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < Cfg::kStages; ++s) {
+    for (int s = 0; s < n_stages; ++s) {
       mbar_init(&full_bar[s], 1);
       mbar_init(&empty_bar[s], 1);
     }
@@ -304,22 +377,26 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
   if (warp == 0) {
     // ------------------------------ TMA producer ------------------------------
     if (elect_one()) {
-      uint32_t it = 0;
+      int st_idx = 0;
+      uint32_t st_phase = 0;
       bool ok = true;
-      for (int unit = blockIdx.x; unit < n_units && ok; unit += gridDim.x) {
-        const int tile = unit / n_splits, split = unit % n_splits;
-        const int tm = tile % n_tiles_m, tn = tile / n_tiles_m;
-        const int kb0 = (split * KB) / n_splits, kb1 = ((split + 1) * KB) / n_splits;
-        for (int kb = kb0; kb < kb1; ++kb, ++it) {
-          const int s = it % Cfg::kStages;
-          if (!mbar_wait(&empty_bar[s], ((it / Cfg::kStages) & 1) ^ 1, kSpin)) {
+      long long pos = range_lo;
+      for (int j = 0; (j < dp_count || pos < range_hi) && ok; ++j) {
+        const Piece pc = make_piece(j, dp_count, dp_tiles, pos, range_hi, KB, per, blockIdx.x, gridDim.x);
+        const int tm = pc.tile % n_tiles_m, tn = pc.tile / n_tiles_m;
+        const int kb0 = pc.kb0, kb1 = pc.kb1;
+        for (int kb = kb0; kb < kb1; ++kb) {
+          const int s = st_idx;
+          const uint32_t ph = st_phase;
+          if (++st_idx == n_stages) { st_idx = 0; st_phase ^= 1; }
+          if (!mbar_wait(&empty_bar[s], ph ^ 1, kSpin)) {
             set_status(ep.status, DEV_TIMEOUT_EMPTY);
             ok = false;
             break;
           }
-          uint8_t* a_dst = smem + s * Cfg::kStageBytes;
-          uint8_t* b_dst = a_dst + Cfg::kABytes;
-          mbar_arrive_expect_tx(&full_bar[s], Cfg::kStageBytes);
+          uint8_t* a_dst = smem + s * stage_bytes;
+          uint8_t* b_dst = a_dst + a_bytes;
+          mbar_arrive_expect_tx(&full_bar[s], stage_bytes);
           tma_load_2d(a_dst, &map_x, kb * BK, tm * BM, &full_bar[s]);
           if (swiglu) {
             tma_load_2d(b_dst, &map_w, kb * BK, tn * (BN / 2), &full_bar[s]);
@@ -330,7 +407,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
         }
       }
       if (!ok) {  // let loads already issued land before the CTA may exit
-        for (int s = 0; s < Cfg::kStages; ++s)
+        for (int s = 0; s < n_stages; ++s)
           for (uint32_t i = 0; i < (1u << 14); ++i) {
             if (mbar_try_wait(&full_bar[s], 0) || mbar_try_wait(&full_bar[s], 1)) break;
             __nanosleep(64);
@@ -341,11 +418,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     // ------------------------------ MMA issuer ------------------------------
     if (elect_one()) {
       constexpr uint32_t idesc = make_idesc(BN);
-      uint32_t it = 0, tcount = 0;
+      int st_idx = 0;
+      uint32_t st_phase = 0, tcount = 0;
       bool ok = true;
-      for (int unit = blockIdx.x; unit < n_units && ok; unit += gridDim.x, ++tcount) {
-        const int split = unit % n_splits;
-        const int kb0 = (split * KB) / n_splits, kb1 = ((split + 1) * KB) / n_splits;
+      long long pos = range_lo;
+      for (int j = 0; (j < dp_count || pos < range_hi) && ok; ++j, ++tcount) {
+        const Piece pc = make_piece(j, dp_count, dp_tiles, pos, range_hi, KB, per, blockIdx.x, gridDim.x);
+        const int kb0 = pc.kb0, kb1 = pc.kb1;
         const int acc = tcount & 1;
         if (!mbar_wait(&tempty_bar[acc], ((tcount >> 1) & 1) ^ 1, kSpin)) {
           set_status(ep.status, DEV_TIMEOUT_MMA);
@@ -353,16 +432,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
         }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + acc * BN;
-        for (int kb = kb0; kb < kb1; ++kb, ++it) {
-          const int s = it % Cfg::kStages;
-          if (!mbar_wait(&full_bar[s], (it / Cfg::kStages) & 1, kSpin)) {
+        for (int kb = kb0; kb < kb1; ++kb) {
+          const int s = st_idx;
+          const uint32_t ph = st_phase;
+          if (++st_idx == n_stages) { st_idx = 0; st_phase ^= 1; }
+          if (!mbar_wait(&full_bar[s], ph, kSpin)) {
             set_status(ep.status, DEV_TIMEOUT_FULL);
             ok = false;
             break;
           }
           tc_fence_after();
-          const uint32_t a_addr = smem_u32(smem + s * Cfg::kStageBytes);
-          const uint32_t b_addr = a_addr + Cfg::kABytes;
+          const uint32_t a_addr = smem_u32(smem + s * stage_bytes);
+          const uint32_t b_addr = a_addr + a_bytes;
 #pragma unroll
           for (int k = 0; k < BK / 16; ++k) {
             const uint64_t da = make_smem_desc(a_addr + k * 32);
@@ -379,8 +460,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     const int quad = warp & 3;             // TMEM lane quadrant this warp may read
     uint32_t tcount = 0;
     __shared__ int s_last;
-    for (int unit = blockIdx.x; unit < n_units; unit += gridDim.x, ++tcount) {
-      const int tile = unit / n_splits, split = unit % n_splits;
+    long long pos = range_lo;
+    for (int j = 0; j < dp_count || pos < range_hi; ++j, ++tcount) {
+      const Piece pc = make_piece(j, dp_count, dp_tiles, pos, range_hi, KB, per, blockIdx.x, gridDim.x);
+      const int tile = pc.tile, n_splits = pc.n_parts;
       const int tm = tile % n_tiles_m, tn = tile / n_tiles_m;
       const int acc = tcount & 1;
       if (!mbar_wait(&tfull_bar[acc], (tcount >> 1) & 1, kSpin)) {
@@ -400,7 +483,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
       } else {
         // park this split's partial tile, release the accumulator, and let the LAST split to arrive reduce all
         // partials in split order (deterministic) and run the fused epilogue
-        float* mine = split_ws + ((size_t)unit * BM + row_in_tile) * BN;
+        float4* mine = reinterpret_cast<float4*>(split_ws) + (size_t)pc.slot * (BN / 4) * BM + row_in_tile;
 #pragma unroll 1
         for (int c = 0; c < BN / 32; ++c) {
           float v[32];
@@ -408,7 +491,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
           if (m < ep.M) {
 #pragma unroll
             for (int i = 0; i < 8; ++i)
-              __stcg(reinterpret_cast<float4*>(mine + c * 32) + i, make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]));
+              __stcg(mine + (size_t)(c * 8 + i) * BM, make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]));
           }
         }
         tc_fence_before();
@@ -424,7 +507,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
         }
         asm volatile("bar.sync 1, 128;" ::: "memory");
         if (s_last) {
-          SplitLoader ld{split_ws + ((size_t)tile * n_splits * BM + row_in_tile) * BN, (size_t)BM * BN, n_splits, m < ep.M};
+          SplitLoader ld{split_ws, BN, row_in_tile, pc.slot0, pc.slot_next, n_splits, m < ep.M};
           row_epilogue<BN>(ep, ld, m, n0);
         }
         asm volatile("bar.sync 1, 128;" ::: "memory");       // s_last is reused by the next unit
@@ -462,7 +545,7 @@ constexpr int kSplitCounters = 1 << 16;
 
 struct TcState {
   int n_sm = 0;
-  int force_bn = 0, force_s = 1;
+  int force_bn = 0, force_s = 0;
   float* split_ws = nullptr;
   int* split_counters = nullptr;
   EncodeTiledFn encode = nullptr;
@@ -489,7 +572,7 @@ const CUtensorMap* get_map(TcState* st, const void* ptr, uint64_t rows, uint64_t
 }
 
 template <int BN>
-bool launch_bn(TcState* st, int idx, const GemmArgs& a, const EpiParams& ep, int n_splits, cudaStream_t stream) {
+bool launch_bn(TcState* st, int idx, const GemmArgs& a, const EpiParams& ep, bool stream_k, cudaStream_t stream) {
   using Cfg = TcCfg<BN>;
   if (!st->configured[idx]) {
     if (cudaFuncSetAttribute(gemm_tc_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes) != cudaSuccess)
@@ -498,14 +581,29 @@ bool launch_bn(TcState* st, int idx, const GemmArgs& a, const EpiParams& ep, int
   }
   const bool swiglu = a.epi == EPI_SWIGLU;
   const uint64_t w_rows = swiglu ? 2ull * a.N : (uint64_t)a.N;
-  const CUtensorMap* mx = get_map(st, a.x, a.M, a.K, BM);
+  const int thin = a.M <= 32 ? 1 : 0;
+  const CUtensorMap* mx = get_map(st, a.x, a.M, a.K, thin ? 32 : BM);
   const CUtensorMap* mw = get_map(st, a.w, w_rows, a.K, swiglu ? BN / 2 : BN);
   if (!mx || !mw) return false;
   const int out_per_tile = swiglu ? BN / 2 : BN;
   const int n_tiles_n = (a.N + out_per_tile - 1) / out_per_tile;
-  const int n_units = ((a.M + BM - 1) / BM) * n_tiles_n * n_splits;
-  const int grid = n_units < st->n_sm ? n_units : st->n_sm;
-  gemm_tc_kernel<BN><<<grid, kTcThreads, Cfg::kSmemBytes, stream>>>(*mx, *mw, a.M, n_tiles_n, a.K, a.N, n_splits,
+  const int n_tiles = ((a.M + BM - 1) / BM) * n_tiles_n;
+  const long long KB = a.K / BK;
+  int grid = n_tiles < st->n_sm ? n_tiles : st->n_sm;
+  int dp_tiles = n_tiles;       // whole tiles, strided
+  long long per = 1;
+  if (stream_k) {
+    // all but the last one-to-two waves as whole tiles; the k-blocks of the remaining tiles evenly over all SMs
+    const int full = n_tiles / st->n_sm;
+    dp_tiles = full >= 2 ? (full - 1) * st->n_sm : 0;
+    const long long total = (long long)(n_tiles - dp_tiles) * KB;
+    grid = total < st->n_sm ? (int)total : st->n_sm;
+    per = (total + grid - 1) / grid;
+    if (per < 4 && total >= 4) per = 4;                 // keep pieces long enough to amortise their hand-over
+    const int g2 = (int)((total + per - 1) / per);
+    if (dp_tiles == 0) grid = g2;                       // (with whole tiles in front the grid stays at the SM count)
+  }
+  gemm_tc_kernel<BN><<<grid, kTcThreads, Cfg::kSmemBytes, stream>>>(*mx, *mw, a.M, n_tiles_n, a.K, a.N, dp_tiles, per, thin,
                                                                     st->split_ws, st->split_counters, ep);
   return true;
 }
@@ -563,13 +661,14 @@ bool launch_gemm_tc(const GemmArgs& a, void* tc_state, int* status, cudaStream_t
   ep.head_dim = a.head_dim;
   ep.status = status;
   const bool swiglu = a.epi == EPI_SWIGLU;
-  // Choose the tile width by a small cost model in microseconds, calibrated on B200: time = waves x k-blocks x
-  // (tensor time of one k-block at that width).  K is split only for thin problems (M <= 64) with a long K,
-  // where the partial tiles are small and the extra units fill the machine; the fixed hand-over of a split
-  // (fence, counter, reduction read) costs about as much as 16 k-blocks.  Rotary tiles must hold whole heads.
+  // Choose the tile width and the decomposition with a small cost model in microseconds, calibrated on B200:
+  // whole tiles cost waves x k-blocks x (tensor time of one k-block at that width); the stream-K decomposition
+  // spreads all k-blocks evenly over the SMs and pays a fixed hand-over for the cut tiles (park the partial,
+  // fence, counter, reduction read).  Rotary tiles must hold whole heads.
   const int mt = (a.M + BM - 1) / BM;
   const int KB = a.K / BK;
-  int best_bn = 0, best_s = 1;
+  int best_bn = 0;
+  bool best_sk = false;
   double best_t = 1e30;
   const int bns[3] = {256, 128, 64};
   const double kb_tensor[3] = {0.44, 0.27, 0.22};
@@ -579,38 +678,36 @@ bool launch_gemm_tc(const GemmArgs& a, void* tc_state, int* status, cudaStream_t
     if (a.epi == EPI_QKV_ROPE && (bn < a.head_dim || a.N % bn)) continue;
     if (swiglu && (a.N % per)) continue;
     const int tiles = mt * ((a.N + per - 1) / per);
-    const int max_split = (a.M <= 64 && KB >= 128) ? 4 : 1;
-    for (int sp = 1; sp <= max_split; ++sp) {
-      const long long units = (long long)tiles * sp;
-      if (sp > 1 && (units > kSplitCounters || (size_t)units * BM * bn * 4 > kSplitWsBytes)) break;
-      const long long waves = (units + st->n_sm - 1) / st->n_sm;
-      double t = (double)waves * ((KB + sp - 1) / sp) * kb_tensor[bi];
-      if (sp > 1) t += 4.0;
-      if (t < best_t) {
-        best_t = t;
-        best_bn = bn;
-        best_s = sp;
-      }
-    }
+    if (tiles > kSplitCounters) continue;
+    const long long waves = (tiles + st->n_sm - 1) / st->n_sm;
+    // a k-block costs its tensor time, or the time one SM needs to stream its share of the weight bytes (the
+    // mt CTAs that work on one weight tile at the same time share them through L2)
+    const double kbt = fmax(kb_tensor[bi], (bn * 128.0 / mt) / 35e3);
+    const double rows = a.M < BM ? a.M : BM;
+    const double t_plain = (double)waves * KB * kbt;
+    const double t_sk = ((double)tiles * KB / st->n_sm + 1.0) * kbt + 3.0 + rows * bn * 4.0 * 2.5 / 16e3;
+    if (t_plain < best_t) { best_t = t_plain; best_bn = bn; best_sk = false; }
+    // measured: with full 128-row tiles the hand-over of the cut tiles (15-27 us at the end of the kernel, when
+    // every reduction happens at once) eats the gain, so K ranges are only cut for thin problems
+    if (a.M <= 64 && (size_t)2 * st->n_sm * BM * bn * 4 <= kSplitWsBytes && t_sk < best_t) { best_t = t_sk; best_bn = bn; best_sk = true; }
   }
-  if (st->force_bn) {   // tuning aid: RECG_GEMM_FORCE="<bn>,<splits>"; ignored where it does not fit
-    const int bn = st->force_bn, sp = st->force_s;
+  if (st->force_bn) {   // tuning aid: RECG_GEMM_FORCE="<bn>,<0 whole tiles | 1 stream-K>"; ignored where it does not fit
+    const int bn = st->force_bn;
     const int per = swiglu ? bn / 2 : bn;
-    const long long units = (long long)mt * ((a.N + per - 1) / per) * sp;
-    const bool shape_ok = (bn == 256 || bn == 128 || bn == 64) && sp >= 1 && sp <= KB &&
-                          !(a.epi == EPI_QKV_ROPE && (bn < a.head_dim || a.N % bn)) && !(swiglu && (a.N % per));
-    const bool fits = sp == 1 || (units <= kSplitCounters && (size_t)units * BM * bn * 4 <= kSplitWsBytes);
-    if (shape_ok && fits) {
+    const bool shape_ok = (bn == 256 || bn == 128 || bn == 64) &&
+                          !(a.epi == EPI_QKV_ROPE && (bn < a.head_dim || a.N % bn)) && !(swiglu && (a.N % per)) &&
+                          mt * ((a.N + per - 1) / per) <= kSplitCounters;
+    if (shape_ok) {
       best_bn = bn;
-      best_s = sp;
+      best_sk = st->force_s != 0;
     }
   }
   if (!best_bn) return false;
   if (swiglu && (a.N % 32)) return false;
   switch (best_bn) {
-    case 256: return launch_bn<256>(st, 0, a, ep, best_s, stream);
-    case 128: return launch_bn<128>(st, 1, a, ep, best_s, stream);
-    default: return launch_bn<64>(st, 2, a, ep, best_s, stream);
+    case 256: return launch_bn<256>(st, 0, a, ep, best_sk, stream);
+    case 128: return launch_bn<128>(st, 1, a, ep, best_sk, stream);
+    default: return launch_bn<64>(st, 2, a, ep, best_sk, stream);
   }
 }
 

@@ -47,6 +47,7 @@ struct BatchLayout {
   AttnTile* tiles;
   int* tile_off;    // [C+1] first tile entry of each request
   int* cta_off;     // [n_ctas+1] first item of each CTA of the persistent attention grid
+  int* item_cta;    // [max_items] owning CTA of each item (scratch of the layout kernel)
   int* counts;      // [0] number of items, [1] number of tiles, [2] blocks per CTA
   int max_items, max_parts;
 };

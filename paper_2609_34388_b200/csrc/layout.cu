@@ -18,10 +18,13 @@ __device__ __forceinline__ int upper_request(const int* cu, int n_req, int t) {
 
 // One CTA.  Shared: 5 arrays of n_req+1 ints.
 //
-// Attention work list: the 64-token KV blocks of all (request, kv head, row tile) tiles form one line of W
-// blocks; it is cut into n_ctas equal contiguous ranges, one per CTA of the persistent attention grid, and
-// additionally at every tile boundary.  Each piece is an item; a tile cut by CTA boundaries gets one
-// partial slot per piece.  Every CTA therefore streams the same number of blocks (+-1).
+// Attention work list: the 64-token KV blocks of all (request, kv head, row tile) tiles form one line; every
+// tile is preceded by kItemCost virtual blocks that stand for the fixed cost of starting an item (staging Q,
+// refilling and draining the pipeline).  The line of W cost units is cut into n_ctas equal contiguous ranges,
+// one per CTA of the persistent attention grid, and additionally at every tile boundary.  Each piece that holds
+// real blocks is an item; a tile whose blocks are cut by CTA boundaries gets one partial slot per piece.
+constexpr int kItemCost = 3;
+
 __global__ void __launch_bounds__(1024) layout_kernel(BatchLayout bl, int n_kv, int mask_id, int tok_per_tile,
                                                       int n_ctas, int64_t n_pages, int* status) {
   extern __shared__ int sm[];
@@ -68,7 +71,7 @@ __global__ void __launch_bounds__(1024) layout_kernel(BatchLayout bl, int n_kv, 
     tile_off[0] = 0;
     long long w = 0;
     for (int r = 0; r < C; ++r) {
-      w += (long long)tile_off[r + 1] * req_nb[r];
+      w += (long long)tile_off[r + 1] * (req_nb[r] + kItemCost);
       if (w > 0x3fffffff) w = 0x3fffffff;   // far beyond any pool; keeps the arithmetic in int
       req_blk_off[r + 1] = (int)w;
       tile_off[r + 1] += tile_off[r];
@@ -83,7 +86,7 @@ __global__ void __launch_bounds__(1024) layout_kernel(BatchLayout bl, int n_kv, 
     const int nb = req_nb[r], nt = tile_off[r + 1] - tile_off[r];
     int items = 0, parts_split = 0;
     for (int k = 0; k < nt; ++k) {
-      const int g0 = req_blk_off[r] + k * nb, g1 = g0 + nb;
+      const int g0 = req_blk_off[r] + k * (nb + kItemCost) + kItemCost, g1 = g0 + nb;   // cost range of the real blocks
       const int parts = (g1 - 1) / per - g0 / per + 1;
       items += parts;
       if (parts > 1) parts_split += parts;
@@ -111,7 +114,7 @@ __global__ void __launch_bounds__(1024) layout_kernel(BatchLayout bl, int n_kv, 
   const int n_items = bl.counts[0];
   for (int r = tid; r <= C; r += nth) bl.tile_off[r] = tile_off[r];
   for (int c = tid; c <= n_ctas; c += nth)
-    if ((long long)c * per >= W || n_items == 0) bl.cta_off[c] = n_items;   // CTAs without work
+    bl.cta_off[c] = -1;                                                      // filled below
   if (n_items == 0) return;
   for (int r = tid; r < C; r += nth) {
     const int n = bl.verify_len[r] + bl.block_size[r];
@@ -121,7 +124,7 @@ __global__ void __launch_bounds__(1024) layout_kernel(BatchLayout bl, int n_kv, 
     int item = item_off[r], part = part_off[r];
     for (int k = 0; k < nt; ++k) {
       const int kvh = k / tiles, tile = k % tiles;
-      const int g0 = req_blk_off[r] + k * nb, g1 = g0 + nb;
+      const int g0 = req_blk_off[r] + k * (nb + kItemCost) + kItemCost, g1 = g0 + nb;
       const int c_first = g0 / per, c_last = (g1 - 1) / per;
       const int parts = c_last - c_first + 1;
       AttnTile tl;
@@ -136,17 +139,26 @@ __global__ void __launch_bounds__(1024) layout_kernel(BatchLayout bl, int n_kv, 
         AttnItem a;
         a.req = r;
         a.kv_head = kvh;
-        a.tok0 = bl.cu_tok[r] + tile * tok_per_tile;
-        a.ntok = min(tok_per_tile, n - tile * tok_per_tile);
+        a.tok0 = tl.tok0;
+        a.ntok = tl.ntok;
         a.blk_begin = gs - g0;
         a.blk_end = ge - g0;
         a.part = parts > 1 ? part++ : -1;
         a.kv_len = kv_len;
         bl.items[item] = a;
-        if (gs == c * per) bl.cta_off[c] = item;   // first item of CTA c
+        bl.item_cta[item] = c;
       }
     }
   }
+  // first item of every CTA: items are ordered by CTA, so a CTA's range starts where the owner changes
+  __syncthreads();
+  for (int it = tid; it < n_items; it += nth) {
+    const int c = bl.item_cta[it];
+    const int prev = it ? bl.item_cta[it - 1] : -1;
+    for (int cc = prev + 1; cc <= c; ++cc) bl.cta_off[cc] = it;   // CTAs between two owners have no items
+  }
+  const int last_owner = bl.item_cta[n_items - 1];
+  for (int c = last_owner + 1 + tid; c <= n_ctas; c += nth) bl.cta_off[c] = n_items;
 }
 
 __global__ void embed_kernel(const int* __restrict__ tok_id, const __nv_bfloat16* __restrict__ embed,

@@ -113,6 +113,7 @@ size_t carve(recg_ctx* c, DeviceArena& A) {
   bl.max_parts = 2 * c->target_items;
   bl.max_items = (int)(2 * c->target_items + max_tiles);
   bl.items = A.take<AttnItem>(bl.max_items);
+  bl.item_cta = A.take<int>(bl.max_items);
   bl.tiles = A.take<AttnTile>(max_tiles);
   bl.tile_off = A.take<int>(Cm + 1);
   bl.cta_off = A.take<int>(c->target_items + 1);
