@@ -78,6 +78,14 @@ def test_attention_long_context_split_and_multi_tile():
     assert run_attention_case(synth.tiny_shape(), [(2500, 40, 30), (100, 70, 0)], seed=24) < ATTN_TOL
 
 
+def test_attention_high_concurrency_mix():
+    """128 requests with the high-concurrency block mix {2,4,8,16} @ (.4,.3,.2,.1): about a thousand small tiles."""
+    shape = synth.llama8b_shape(1)
+    desc = synth.batch_descriptor(128, [2, 4, 8, 16], [0.4, 0.3, 0.2, 0.1], 40, 700, seed=31)
+    reqs = list(zip(desc.ctx_len.tolist(), desc.verify_len.tolist(), desc.block_size.tolist()))
+    assert run_attention_case(shape, reqs, seed=32) < ATTN_TOL
+
+
 def test_attention_is_deterministic():
     shape = synth.llama8b_shape(1)
     desc = synth.fixed_descriptor([1500, 40], [8, 4], [8, 4], seed=3)
