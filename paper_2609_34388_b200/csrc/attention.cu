@@ -60,6 +60,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attention_kernel(AttnParams P
   uint64_t* empty_bar = full_bar + kStages;
   float* merge = reinterpret_cast<float*>(smem + SM::kRingBytes);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  griddep_launch();
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
@@ -69,6 +70,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attention_kernel(AttnParams P
     fence_barrier_init();
   }
   __syncthreads();
+  griddep_wait();
 
   const int item_begin = P.cta_off[blockIdx.x], item_end = P.cta_off[blockIdx.x + 1];
   uint32_t it = 0;  // running block counter, identical in producer and consumers
@@ -363,6 +365,8 @@ __global__ void __launch_bounds__(512) attention_combine_kernel(const AttnTile* 
                                                                 const float* __restrict__ part_ml,
                                                                 __nv_bfloat16* __restrict__ o) {
   constexpr int E = D / 32;
+  griddep_launch();
+  griddep_wait();
   const int n_tiles = counts[1];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   // work unit = 16 rows of a tile: units are strided over the grid, a CTA's 16 warps take one row each
@@ -423,9 +427,9 @@ void launch_attention_t(const BatchLayout& bl, const Dims& dm, int layer, const 
   P.part_o = part_o;
   P.part_ml = part_ml;
   P.status = status;
-  attention_kernel<D><<<n_sm, kAttnThreads, AttnSmem<D>::kTotal, st>>>(P);
-  attention_combine_kernel<D><<<2 * n_sm, 512, 0, st>>>(bl.tiles, bl.counts, dm.n_q, P.group, part_o, part_ml,
-                                                        static_cast<__nv_bfloat16*>(o));
+  launch_pdl(attention_kernel<D>, dim3(n_sm), dim3(kAttnThreads), AttnSmem<D>::kTotal, st, P);
+  launch_pdl(attention_combine_kernel<D>, dim3(2 * n_sm), dim3(512), 0, st, (const AttnTile*)bl.tiles, (const int*)bl.counts,
+             dm.n_q, P.group, (const float*)part_o, (const float*)part_ml, static_cast<__nv_bfloat16*>(o));
 }
 
 }  // namespace
@@ -439,8 +443,9 @@ void launch_attention(const BatchLayout& bl, const Dims& dm, int layer, const vo
                       cudaStream_t st, bool use_tc) {
   if (use_tc && dm.head_dim == 128) {
     launch_attention_tc_main(bl, dm, layer, q, o, kv_pool, n_pages, part_o, part_ml, n_sm, status, st);
-    attention_combine_kernel<128><<<2 * n_sm, 512, 0, st>>>(bl.tiles, bl.counts, dm.n_q, dm.n_q / dm.n_kv, part_o, part_ml,
-                                                            static_cast<__nv_bfloat16*>(o));
+    launch_pdl(attention_combine_kernel<128>, dim3(2 * n_sm), dim3(512), 0, st, (const AttnTile*)bl.tiles,
+               (const int*)bl.counts, dm.n_q, dm.n_q / dm.n_kv, (const float*)part_o, (const float*)part_ml,
+               static_cast<__nv_bfloat16*>(o));
     return;
   }
   if (dm.head_dim == 64)

@@ -186,6 +186,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_tc_kernel(TcAttnParams 
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  griddep_wait();   // everything above touched only shared memory and TMEM
   const int item_begin = P.cta_off[blockIdx.x], item_end = P.cta_off[blockIdx.x + 1];
   const uint32_t smem_base = smem_u32(smem);
 
@@ -542,6 +543,10 @@ __global__ void __launch_bounds__(kThreads, 1) attention_tc_kernel(TcAttnParams 
     }
   }
 
+  // this CTA's work is done: let the next kernel's CTAs be scheduled (they run their prologue and then wait for
+  // this whole grid).  Signalling earlier would park their warps on the SMs while the softmax warps still need
+  // every issue slot.
+  griddep_launch();
   tc_fence_before();
   __syncthreads();
   if (warp == 1) {
@@ -580,7 +585,7 @@ void launch_attention_tc_main(const BatchLayout& bl, const Dims& dm, int layer, 
   P.part_o = part_o;
   P.part_ml = part_ml;
   P.status = status;
-  attention_tc_kernel<<<n_sm, kThreads, kSmemBytes, st>>>(P);
+  launch_pdl(attention_tc_kernel, dim3(n_sm), dim3(kThreads), kSmemBytes, st, P);
 }
 
 }  // namespace recg

@@ -23,6 +23,15 @@ __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));
 }
 
+// ---- programmatic dependent launch ------------------------------------------------------------------
+// Every kernel of a step is launched with programmatic stream serialisation: it signals at once that its
+// dependent may be scheduled (launch_dependents), runs its own prologue (barrier init, TMEM allocation, shared
+// memory clearing), and only then waits for the kernels before it to complete and flush (griddep_wait).  No
+// kernel reads or writes global memory before its wait, so the launch latency and prologue of kernel n+1 overlap
+// the tail of kernel n and nothing else changes.  Without the launch attribute both instructions do nothing.
+__device__ __forceinline__ void griddep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // ---- mbarrier ---------------------------------------------------------------------------------
 __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
@@ -113,6 +122,28 @@ __host__ __device__ __forceinline__ int kv_tile_offset(int tok, int dim, int hea
 __host__ __device__ __forceinline__ size_t kv_tile_base(int64_t n_pages, int n_kv, int head_dim, int layer,
                                                         int64_t page, int kv_head) {
   return ((((size_t)layer * n_pages + page) * n_kv + kv_head) * 2) * kv_tile_elems(head_dim);
+}
+
+// Host side: launch with the programmatic-serialisation attribute.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                              Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  // inside a stream capture the kernels become graph nodes, where plain edges measured faster than programmatic
+  // ones (21.4 vs 24.6 us for the attention + combine pair), so the attribute is only used on live streams
+  cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  if (cudaStreamIsCapturing(st, &cap) == cudaSuccess && cap == cudaStreamCaptureStatusNone) {
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+  }
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
 }  // namespace recg

@@ -38,6 +38,8 @@ __global__ void __launch_bounds__(THREADS) gemm_simt_kernel(const __nv_bfloat16*
   extern __shared__ __align__(16) uint8_t smem_raw[];
   __nv_bfloat16* sm = reinterpret_cast<__nv_bfloat16*>(smem_raw);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  griddep_launch();
+  griddep_wait();
   const int wm = warp >> 2, wn = warp & 3;
   const int m0 = blockIdx.y * BM;
   const bool swiglu = ep.epi == EPI_SWIGLU;
@@ -144,8 +146,8 @@ void launch_gemm_simt(const GemmArgs& a, int* status, cudaStream_t st) {
   const int out_per_tile = a.epi == EPI_SWIGLU ? BN / 2 : BN;
   dim3 grid((a.N + out_per_tile - 1) / out_per_tile, (a.M + BM - 1) / BM);
   if (a.M <= 0) return;
-  gemm_simt_kernel<<<grid, THREADS, SMEM_BYTES, st>>>(static_cast<const __nv_bfloat16*>(a.x),
-                                                      static_cast<const __nv_bfloat16*>(a.w), a.M, a.N, a.K, ep);
+  launch_pdl(gemm_simt_kernel, grid, dim3(THREADS), SMEM_BYTES, st, static_cast<const __nv_bfloat16*>(a.x),
+             static_cast<const __nv_bfloat16*>(a.w), a.M, a.N, a.K, ep);
 }
 
 }  // namespace recg

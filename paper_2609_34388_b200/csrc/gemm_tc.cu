@@ -373,6 +373,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  griddep_wait();   // everything above touched only shared memory and TMEM
 
   if (warp == 0) {
     // ------------------------------ TMA producer ------------------------------
@@ -515,6 +516,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     }
   }
 
+  griddep_launch();   // this CTA's work is done: the next kernel's CTAs may be scheduled onto freed SMs
   tc_fence_before();
   __syncthreads();
   if (warp == 1) {
@@ -603,8 +605,8 @@ bool launch_bn(TcState* st, int idx, const GemmArgs& a, const EpiParams& ep, boo
     const int g2 = (int)((total + per - 1) / per);
     if (dp_tiles == 0) grid = g2;                       // (with whole tiles in front the grid stays at the SM count)
   }
-  gemm_tc_kernel<BN><<<grid, kTcThreads, Cfg::kSmemBytes, stream>>>(*mx, *mw, a.M, n_tiles_n, a.K, a.N, dp_tiles, per, thin,
-                                                                    st->split_ws, st->split_counters, ep);
+  launch_pdl(gemm_tc_kernel<BN>, dim3(grid), dim3(kTcThreads), Cfg::kSmemBytes, stream, *mx, *mw, a.M, n_tiles_n, a.K, a.N,
+             dp_tiles, per, thin, st->split_ws, st->split_counters, ep);
   return true;
 }
 

@@ -36,6 +36,8 @@ __global__ void __launch_bounds__(1024) layout_kernel(BatchLayout bl, int n_kv, 
   int* req_nb = sm + 4 * (C + 1);        // blocks per tile of request r
   __shared__ int s_per, s_total_blocks;
   const int tid = threadIdx.x, nth = blockDim.x;
+  griddep_launch();
+  griddep_wait();   // the previous step's kernels may still be reading the arrays this kernel rewrites
 
   // ---- per-token arrays ----
   for (int t = tid; t < bl.n_tok; t += nth) {
@@ -163,6 +165,8 @@ __global__ void __launch_bounds__(1024) layout_kernel(BatchLayout bl, int n_kv, 
 
 __global__ void embed_kernel(const int* __restrict__ tok_id, const __nv_bfloat16* __restrict__ embed,
                              float* __restrict__ h, int hidden, int vocab) {
+  griddep_launch();
+  griddep_wait();
   const int t = blockIdx.x;
   int id = tok_id[t];
   id = id < 0 ? 0 : (id >= vocab ? vocab - 1 : id);
@@ -171,34 +175,60 @@ __global__ void embed_kernel(const int* __restrict__ tok_id, const __nv_bfloat16
   for (int i = threadIdx.x; i < hidden / 2; i += blockDim.x) dst[i] = __bfloat1622float2(src[i]);
 }
 
-// One CTA per row; fp32 in, bf16 out.  hidden a multiple of 4.
+// One CTA per row; fp32 in, bf16 out.  hidden a multiple of 4.  The row is read once and kept in registers
+// when it fits (hidden <= 256 threads x kRegVecs float4), otherwise it is read a second time.
+constexpr int kRegVecs = 8;
 __global__ void __launch_bounds__(256) rmsnorm_kernel(const float* __restrict__ h, const __nv_bfloat16* __restrict__ g,
                                                       __nv_bfloat16* __restrict__ x, int hidden, float eps) {
+  griddep_launch();
+  griddep_wait();
   const int row = blockIdx.x;
+  const int nvec = hidden / 4;
   const float4* src = reinterpret_cast<const float4*>(h + (size_t)row * hidden);
+  const bool in_regs = nvec <= 256 * kRegVecs;
+  float4 v[kRegVecs];
   float ss = 0.f;
-  for (int i = threadIdx.x; i < hidden / 4; i += blockDim.x) {
-    float4 v = src[i];
-    ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+  if (in_regs) {
+#pragma unroll
+    for (int u = 0; u < kRegVecs; ++u) {
+      const int i = threadIdx.x + u * 256;
+      v[u] = i < nvec ? src[i] : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+#pragma unroll
+    for (int u = 0; u < kRegVecs; ++u) ss += v[u].x * v[u].x + v[u].y * v[u].y + v[u].z * v[u].z + v[u].w * v[u].w;
+  } else {
+    for (int i = threadIdx.x; i < nvec; i += 256) {
+      const float4 t = src[i];
+      ss += t.x * t.x + t.y * t.y + t.z * t.z + t.w * t.w;
+    }
   }
   __shared__ float red[8];
   for (int o = 16; o; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
   if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
   __syncthreads();
   float tot = 0.f;
-  for (int i = 0; i < (blockDim.x >> 5); ++i) tot += red[i];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) tot += red[i];
   const float rstd = rsqrtf(tot / hidden + eps);
   uint2* dst = reinterpret_cast<uint2*>(x + (size_t)row * hidden);
   const uint2* gg = reinterpret_cast<const uint2*>(g);
-  for (int i = threadIdx.x; i < hidden / 4; i += blockDim.x) {
-    float4 v = src[i];
-    uint2 gv = gg[i];
-    float2 g0 = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162*>(&gv.x));
-    float2 g1 = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162*>(&gv.y));
+  auto emit = [&](int i, const float4& t) {
+    const uint2 gv = __ldg(gg + i);
+    const float2 g0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&gv.x));
+    const float2 g1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&gv.y));
     uint2 o;
-    o.x = pack_bf16(v.x * rstd * g0.x, v.y * rstd * g0.y);
-    o.y = pack_bf16(v.z * rstd * g1.x, v.w * rstd * g1.y);
+    o.x = pack_bf16(t.x * rstd * g0.x, t.y * rstd * g0.y);
+    o.y = pack_bf16(t.z * rstd * g1.x, t.w * rstd * g1.y);
     dst[i] = o;
+  };
+  if (in_regs) {
+#pragma unroll
+    for (int u = 0; u < kRegVecs; ++u) {
+      const int i = threadIdx.x + u * 256;
+      if (i < nvec) emit(i, v[u]);
+    }
+  } else {
+    for (int i = threadIdx.x; i < nvec; i += 256) emit(i, src[i]);
   }
 }
 
@@ -233,16 +263,17 @@ __global__ void kv_io_kernel(bool write, __nv_bfloat16* pool, int64_t n_pages, i
 void launch_layout(const BatchLayout& bl, const Dims& dm, int tok_per_tile, int n_ctas, int64_t n_pages,
                    int* status, cudaStream_t st) {
   const size_t smem = 5 * (size_t)(bl.n_req + 1) * sizeof(int);
-  layout_kernel<<<1, 1024, smem, st>>>(bl, dm.n_kv, dm.mask_id, tok_per_tile, n_ctas, n_pages, status);
+  launch_pdl(layout_kernel, dim3(1), dim3(1024), smem, st, bl, dm.n_kv, dm.mask_id, tok_per_tile, n_ctas, n_pages, status);
 }
 
 void launch_embed(const BatchLayout& bl, const Dims& dm, const void* embed, float* h, cudaStream_t st) {
-  embed_kernel<<<bl.n_tok, 256, 0, st>>>(bl.tok_id, static_cast<const __nv_bfloat16*>(embed), h, dm.hidden, dm.vocab);
+  launch_pdl(embed_kernel, dim3(bl.n_tok), dim3(256), 0, st, (const int*)bl.tok_id, static_cast<const __nv_bfloat16*>(embed), h,
+             dm.hidden, dm.vocab);
 }
 
 void launch_rmsnorm(const float* h, const void* gain, void* x, int rows, int hidden, float eps, cudaStream_t st) {
-  rmsnorm_kernel<<<rows, 256, 0, st>>>(h, static_cast<const __nv_bfloat16*>(gain), static_cast<__nv_bfloat16*>(x),
-                                       hidden, eps);
+  launch_pdl(rmsnorm_kernel, dim3(rows), dim3(256), 0, st, h, static_cast<const __nv_bfloat16*>(gain),
+             static_cast<__nv_bfloat16*>(x), hidden, eps);
 }
 
 void launch_kv_io(bool write, void* pool, int64_t n_pages, int layer, const Dims& dm, const int* page_row_dev, int pos0,
@@ -260,6 +291,8 @@ namespace recg {
 namespace {
 __global__ void rope_table_kernel(const int* __restrict__ tok_pos, int n_tok, int half, double log_base,
                                   float2* __restrict__ cs) {
+  griddep_launch();
+  griddep_wait();
   const int idx = blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= n_tok * half) return;
   const int t = idx / half, i = idx % half;
@@ -273,7 +306,7 @@ void launch_rope_table(const int* tok_pos, int n_tok, int head_dim, float rope_b
   const int half = head_dim / 2;
   const int total = n_tok * half;
   if (total <= 0) return;
-  rope_table_kernel<<<(total + 255) / 256, 256, 0, st>>>(tok_pos, n_tok, half, log((double)rope_base),
-                                                         static_cast<float2*>(cs));
+  launch_pdl(rope_table_kernel, dim3((total + 255) / 256), dim3(256), 0, st, tok_pos, n_tok, half,
+             log((double)rope_base), static_cast<float2*>(cs));
 }
 }  // namespace recg

@@ -90,6 +90,8 @@ __global__ void __launch_bounds__(kVerifyThreads) verify_partial_kernel(const T*
                                                                         int chunk_len, int chunks_per_row,
                                                                         RowPartial* __restrict__ partials) {
   constexpr int N = Vec<T>::N;
+  griddep_launch();
+  griddep_wait();
   const int row = blockIdx.y, chunk = blockIdx.x;
   const T* base = logits + (size_t)row * vocab;
   const int c0 = chunk * chunk_len;
@@ -208,6 +210,8 @@ __global__ void __launch_bounds__(kVerifyThreads) verify_partial_kernel(const T*
 // One CTA per request: merge the chunk partials of its rows, then the accept scan and the index work.
 __global__ void __launch_bounds__(128) verify_finalize_kernel(BatchLayout bl, const RowPartial* __restrict__ partials,
                                                               int chunks_per_row, VerifyBuffers vb) {
+  griddep_launch();
+  griddep_wait();
   const int r = blockIdx.x;
   const int t0 = bl.cu_tok[r];
   const int v = bl.verify_len[r], b = bl.block_size[r], L = bl.ctx_len[r];
@@ -288,12 +292,12 @@ void launch_verify(const BatchLayout& bl, const void* logits, int logits_dtype, 
   chunks = (vocab + chunk_len - 1) / chunk_len;
   dim3 grid(chunks, rows);
   if (logits_dtype == 0)
-    verify_partial_kernel<__nv_bfloat16>
-        <<<grid, kVerifyThreads, 0, st>>>(static_cast<const __nv_bfloat16*>(logits), vocab, chunk_len, chunks, partials);
+    launch_pdl(verify_partial_kernel<__nv_bfloat16>, grid, dim3(kVerifyThreads), 0, st,
+               static_cast<const __nv_bfloat16*>(logits), vocab, chunk_len, chunks, partials);
   else
-    verify_partial_kernel<float>
-        <<<grid, kVerifyThreads, 0, st>>>(static_cast<const float*>(logits), vocab, chunk_len, chunks, partials);
-  verify_finalize_kernel<<<bl.n_req, 128, 0, st>>>(bl, partials, chunks, vb);
+    launch_pdl(verify_partial_kernel<float>, grid, dim3(kVerifyThreads), 0, st, static_cast<const float*>(logits), vocab,
+               chunk_len, chunks, partials);
+  launch_pdl(verify_finalize_kernel, dim3(bl.n_req), dim3(128), 0, st, bl, (const RowPartial*)partials, chunks, vb);
 }
 
 }  // namespace recg
