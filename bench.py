@@ -457,25 +457,35 @@ def bench_c1(binding, ctx, shape, pool, n_pages, peaks, args):
     desc = c1_descriptor(11)
     ys = synth.token_ids(16, shape.vocab, seed=2)
     batch = binding.Batch(desc.ctx_len, desc.verify_len, desc.block_size, ys, desc.page_table, pool, n_pages)
+    vout = binding.VerifyOut(batch.n_req, batch.n_tok, batch.n_ver, host=False)
     for _ in range(3):
         ctx.recg_step(batch)
-        ctx.recg_verify(batch, host=False)
+        ctx.recg_verify(batch, out=vout)
     torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     iters = max(3, args.steps)
     e0.record()
     for _ in range(iters):
         ctx.recg_step(batch)
-        ctx.recg_verify(batch, host=False)
+        ctx.recg_verify(batch, out=vout)
     e1.record()
     torch.cuda.synchronize()
     ms = e0.elapsed_time(e1) / iters
+    ctx.recg_timing_enable(True)
+    ctx.recg_timing_read()
+    for _ in range(iters):
+        ctx.recg_step(batch)
+        ctx.recg_verify(batch, out=vout)
+    cms, _ = ctx.recg_timing_read()
+    ctx.recg_timing_enable(False)
+    classes = {k: round(v / iters, 4) for k, v in cms.items()}
     wbytes = 2.0 * (shape.n_layers * ((shape.n_q_heads + 2 * shape.n_kv_heads) * shape.head_dim * shape.hidden +
                                        shape.hidden * shape.n_q_heads * shape.head_dim + 3 * shape.ffn * shape.hidden) +
                     shape.vocab * shape.hidden)
     return {"workload": "concurrency 1, context 4096, verify 16 + block 16", "ms_per_step": round(ms, 4),
             "tokens_per_s": round(32 / (ms / 1e3), 1), "weight_stream_gbs": round(wbytes / (ms / 1e3) / 1e9, 1),
-            "frac_of_hbm_measured": round(wbytes / (ms / 1e3) / 1e9 / peaks["hbm_gbs"], 4)}
+            "frac_of_hbm_measured": round(wbytes / (ms / 1e3) / 1e9 / peaks["hbm_gbs"], 4),
+            "class_ms_per_step": classes}
 
 
 # ------------------------------------------------------------------------------------------------
