@@ -6,6 +6,7 @@
 // eight consumer warps hold 16 query rows each and, when the tile has fewer than 128 rows, share the
 // rows and split the KV blocks among themselves instead.  Only blocks that reach past the committed
 // context apply the visibility test; the prefix loop is mask-free.
+#include <cstdlib>
 #include "common.cuh"
 #include "kernels.h"
 
@@ -355,45 +356,77 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attention_kernel(AttnParams P
   }
 }
 
-// Merges the KV-range partials of the tiles that were split.  A small persistent grid strides over the (tile, row)
-// table; tiles with a single part were written by the attention kernel itself and are skipped.  One warp per
-// query row, each lane D/32 consecutive dims.
+// Merges the KV-range partials of the tiles that were split.  Tiles with a single part were written by the
+// attention kernel itself and are skipped.  Work unit = 16 rows of a tile, one warp per query row, each lane D/32
+// consecutive dims.  The kernel is latency bound (tile entry -> (max, sum) pairs -> partial rows), so every level
+// is fetched for all parts at once and the grid is sized to hold all rows in one or two waves.
 template <int D>
-__global__ void __launch_bounds__(512) attention_combine_kernel(const AttnTile* __restrict__ tiles,
+__global__ void __launch_bounds__(512, 3) attention_combine_kernel(const AttnTile* __restrict__ tiles,
                                                                 const int* __restrict__ counts, int n_q, int group,
                                                                 const float* __restrict__ part_o,
                                                                 const float* __restrict__ part_ml,
                                                                 __nv_bfloat16* __restrict__ o) {
   constexpr int E = D / 32;
+  constexpr int kMaxP = 4;     // parts fetched together; longer lists go round by round
   griddep_launch();
   griddep_wait();
   const int n_tiles = counts[1];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  // work unit = 16 rows of a tile: units are strided over the grid, a CTA's 16 warps take one row each
   for (int wu = blockIdx.x; wu < n_tiles * 8; wu += gridDim.x) {
     const AttnTile tl = tiles[wu >> 3];
     if (tl.n_parts <= 1) continue;
     const int rho = (wu & 7) * 16 + warp;
-    if (rho < tl.ntok * group) {
-      float m = -1e30f;
-      for (int p = 0; p < tl.n_parts; ++p) m = fmaxf(m, part_ml[((size_t)(tl.part_begin + p) * 128 + rho) * 2]);
-      float acc[E];
+    if (rho >= tl.ntok * group) continue;
+    float acc[E];
 #pragma unroll
-      for (int e = 0; e < E; ++e) acc[e] = 0.f;
-      float l = 0.f;
-      for (int p = 0; p < tl.n_parts; ++p) {
-        const size_t row = (size_t)(tl.part_begin + p) * 128 + rho;
-        const float wgt = exp2f(part_ml[row * 2] - m);
-        l += wgt * part_ml[row * 2 + 1];
-        const float* src = part_o + row * D + lane * E;
+    for (int e = 0; e < E; ++e) acc[e] = 0.f;
+    float m = -1e30f, l = 0.f;
+    for (int p0 = 0; p0 < tl.n_parts; p0 += kMaxP) {
+      const int np = min(kMaxP, tl.n_parts - p0);
+      float2 ml[kMaxP];
+      float v[kMaxP][E];
 #pragma unroll
-        for (int e = 0; e < E; ++e) acc[e] += wgt * src[e];
+      for (int p = 0; p < kMaxP; ++p) {
+        ml[p] = make_float2(-1e30f, 0.f);
+        if (p < np) {
+          const size_t row = (size_t)(tl.part_begin + p0 + p) * 128 + rho;
+          ml[p] = __ldcg(reinterpret_cast<const float2*>(part_ml) + row);
+          if constexpr (E == 4) {
+            const float4 t = __ldcg(reinterpret_cast<const float4*>(part_o + row * D) + lane);
+            v[p][0] = t.x; v[p][1] = t.y; v[p][2] = t.z; v[p][3] = t.w;
+          } else {
+            const float2 t = __ldcg(reinterpret_cast<const float2*>(part_o + row * D) + lane);
+            v[p][0] = t.x; v[p][1] = t.y;
+          }
+        }
       }
-      const float inv = l > 0.f ? 1.f / l : 0.f;
-      const int j = rho / group, hg = rho % group;
-      __nv_bfloat16* dst = o + ((size_t)(tl.tok0 + j) * n_q + tl.kv_head * group + hg) * D + lane * E;
+      float m_new = m;
 #pragma unroll
-      for (int e = 0; e < E; e += 2) *reinterpret_cast<uint32_t*>(dst + e) = pack_bf16(acc[e] * inv, acc[e + 1] * inv);
+      for (int p = 0; p < kMaxP; ++p) m_new = fmaxf(m_new, ml[p].x);
+      const float f = exp2f(m - m_new);
+      m = m_new;
+      l *= f;
+#pragma unroll
+      for (int e = 0; e < E; ++e) acc[e] *= f;
+#pragma unroll
+      for (int p = 0; p < kMaxP; ++p)
+        if (p < np) {
+          const float wgt = exp2f(ml[p].x - m);
+          l += wgt * ml[p].y;
+#pragma unroll
+          for (int e = 0; e < E; ++e) acc[e] += wgt * v[p][e];
+        }
+    }
+    const float inv = l > 0.f ? 1.f / l : 0.f;
+    const int j = rho / group, hg = rho % group;
+    __nv_bfloat16* dst = o + ((size_t)(tl.tok0 + j) * n_q + tl.kv_head * group + hg) * D + lane * E;
+    if constexpr (E == 4) {
+      uint2 pk;
+      pk.x = pack_bf16(acc[0] * inv, acc[1] * inv);
+      pk.y = pack_bf16(acc[2] * inv, acc[3] * inv);
+      *reinterpret_cast<uint2*>(dst) = pk;
+    } else {
+      *reinterpret_cast<uint32_t*>(dst) = pack_bf16(acc[0] * inv, acc[1] * inv);
     }
   }
 }
@@ -428,7 +461,7 @@ void launch_attention_t(const BatchLayout& bl, const Dims& dm, int layer, const 
   P.part_ml = part_ml;
   P.status = status;
   launch_pdl(attention_kernel<D>, dim3(n_sm), dim3(kAttnThreads), AttnSmem<D>::kTotal, st, P);
-  launch_pdl(attention_combine_kernel<D>, dim3(2 * n_sm), dim3(512), 0, st, (const AttnTile*)bl.tiles, (const int*)bl.counts,
+  launch_pdl(attention_combine_kernel<D>, dim3(4 * n_sm), dim3(512), 0, st, (const AttnTile*)bl.tiles, (const int*)bl.counts,
              dm.n_q, P.group, (const float*)part_o, (const float*)part_ml, static_cast<__nv_bfloat16*>(o));
 }
 
@@ -443,7 +476,7 @@ void launch_attention(const BatchLayout& bl, const Dims& dm, int layer, const vo
                       cudaStream_t st, bool use_tc) {
   if (use_tc && dm.head_dim == 128) {
     launch_attention_tc_main(bl, dm, layer, q, o, kv_pool, n_pages, part_o, part_ml, n_sm, status, st);
-    launch_pdl(attention_combine_kernel<128>, dim3(2 * n_sm), dim3(512), 0, st, (const AttnTile*)bl.tiles,
+    launch_pdl(attention_combine_kernel<128>, dim3(4 * n_sm), dim3(512), 0, st, (const AttnTile*)bl.tiles,
                (const int*)bl.counts, dm.n_q, dm.n_q / dm.n_kv, (const float*)part_o, (const float*)part_ml,
                static_cast<__nv_bfloat16*>(o));
     return;

@@ -1,22 +1,42 @@
 // Hybrid-mask paged-KV attention on the 5th-generation tensor cores (head_dim 128).
 //
 // Work items are the same as in attention.cu: (request, kv head, row tile of <= 128 query rows, KV range).
-// Per CTA (6 warps, one CTA per SM, persistent over the work list):
-//   warp 0    producer: streams 128-token KV blocks page by page, ONE 4 KB bulk copy per page and operand,
-//             into a ring of five 32 KB operand buffers (K and V of a block are separate entries, so K is
-//             released early).  A page tile (8-row, 128-byte-swizzled atoms ordered [token group][dim half])
-//             lands exactly as stored, and tiles copied back to back form one 128-token operand with a
-//             uniform 2 KB stride between token groups: K-major for S = Q K^T, MN-major for O += P V.
-//             The last, partly filled page of a request is copied by hand with the rows beyond its length
-//             zeroed, so stale pool contents can never reach an accumulator.
-//   warp 1    one elected lane issues tcgen05.mma: S = Q K^T (M 128 rows, N 128 tokens, K = d) into one
-//             of two TMEM buffers, and O += P V (N = d, K = 128 tokens) into a third, which accumulates
-//             over all blocks of the item.
-//   warps 2-5 softmax, ONE THREAD PER QUERY ROW (= TMEM lane): the S row is read from TMEM once, the
-//             probabilities are taken relative to a reference maximum that is only moved (and O rescaled
-//             in TMEM) when the row maximum outgrows it by more than 2^8, and bf16 P is written to shared
-//             memory in operand layout.  No cross-thread reductions are needed.  O is read once per item.
-// Only blocks that reach past a row's visibility limit evaluate the mask.  Every wait is bounded.
+// Per CTA (12 warps = 3 warpgroups, one CTA per SM, persistent over the work list):
+//   warps 0, 2  producers: warp 0 streams the K operand and warp 2 the V operand of each 128-token KV block,
+//             page by page, ONE 4 KB bulk copy per page, into a ring of 32 KB operand buffers (K and V of
+//             a block are separate entries, so K is released early).  A page tile (8-row, 128-byte-swizzled
+//             atoms ordered [token group][dim half]) lands exactly as stored, and tiles copied back to back
+//             form one 128-token operand with a uniform 2 KB stride between token groups: K-major for
+//             S = Q K^T, MN-major for O += P V.  The last, partly filled V page of a request is copied by
+//             hand with the rows beyond its length zeroed, so stale pool contents never reach an accumulator.
+//             Warp 0 also fetches the item's Q rows with two tiled TMA loads (box = 64 dims x the kv head's
+//             query heads x 128 / group tokens, 128-byte swizzle) into one of two Q buffers, so the Q of the
+//             next item is in place before the current item ends.
+//   warp 1    one elected lane issues tcgen05.mma: S = Q K^T (M 128 rows, N 128 tokens, K = d, both operands
+//             in shared memory) and O += P V (P read from TMEM, V from shared memory; N = d, K = 128 tokens).
+//             It runs ahead into the next item (its first S tiles) while the softmax groups still write
+//             the previous item's output.
+//   warps 4-7 and 8-11: two softmax groups.  The KV blocks of an item alternate between them (block n goes
+//             to group n & 1); each group has its own S buffer and O accumulator in TMEM and its own running
+//             (reference maximum, sum), i.e. the two groups are two independent partial attentions over
+//             the even and the odd blocks, merged once at the end of the item.  While one group is in its
+//             exp2 phase the other one reads S or waits for the tensor core.  Within a group ONE THREAD OWNS
+//             ONE QUERY ROW (= TMEM lane): the S row is read from TMEM once, probabilities are taken relative
+//             to a reference maximum that is only moved (and O rescaled in TMEM) when the row maximum
+//             outgrows it by more than 2^8, and bf16 P is written back over the first 64 columns of the same
+//             S buffer (two tokens per 32-bit column), from where the P V product reads it.  The tensor pipe
+//             executes in issue order, so the next S of a group is produced after its P has been consumed.
+//             No cross-thread reductions are needed.  At the end of an item group 0 finishes output dims
+//             [0,64) and group 1 dims [64,128) of every row from both accumulators; partial results (items
+//             that cover part of the KV range) go through a per-warp transposition in the item's Q buffer
+//             so that every global store is a full 128-byte line.
+//   Warpgroup 0 gives registers back (setmaxnreg) so that a softmax thread can hold a whole S row.
+// Only blocks that reach past a row's visibility limit evaluate the mask.  Every wait is bounded; a wait that
+// runs out raises a CTA-wide flag after which no wait blocks, so the kernel always ends.
+#include <cuda.h>
+#include <cstdio>
+#include <cstdlib>
+
 #include "common.cuh"
 #include "kernels.h"
 
@@ -28,22 +48,27 @@ constexpr int D = 128;
 constexpr int kBT = 128;                       // tokens per KV block
 constexpr int kPagesPerBT = kBT / kPageSize;   // 8
 constexpr int kSubBytes = kPageSize * 128;     // 2 KB: [16 tokens][64 dims]
-constexpr int kOperandHalf = kPagesPerBT * kSubBytes;  // 16 KB: one 64-wide half of a 128-token operand
 constexpr int kQBytes = 128 * D * 2;           // 32 KB
-constexpr int kPBytes = 128 * kBT * 2;         // 32 KB
 constexpr int kTileBytes = 2 * kSubBytes;        // 4 KB: the K (or V) tile of one page and head, as stored in the pool
 constexpr int kKVStageBytes = kPagesPerBT * kTileBytes;  // one operand (K or V) of a 128-token block: 32 KB
-constexpr int kKVStages = 4;                     // ring K0 V0 K1 V1 K2 ...: a K buffer is free after Q K^T, a V buffer after P V
-constexpr int kThreads = 224;                    // producer K, MMA, 4 softmax warps, producer V
+constexpr int kKStages = 3;                      // K ring: a buffer is free after its Q K^T
+constexpr int kVStages = 2;                      // V ring: a buffer is free after its P V.  The rings are separate so that a V
+                                                 // buffer never holds the unsanitised rows of a partly filled K page
+constexpr int kKVStages = kKStages + kVStages;
+constexpr int kThreads = 384;                    // warpgroup 0: producer K, MMA, producer V, idle; warpgroups 1, 2: softmax
+constexpr int kSoftThreads = 256;
 constexpr uint32_t kSpin = 1u << 22;
-constexpr int kTmemCols = 512;                 // S0 [0,128) S1 [128,256) O_blk [256,384)
+constexpr int kTmemCols = 512;                 // S of group 0 / 1 at [0,128) / [128,256), O of group 0 / 1 at [256,384) / [384,512);
+                                               // bf16 P of a group overwrites columns [0,64) of its S
+constexpr int kTmemO = 2 * kBT;
 
-constexpr int kOffQ = 0;
-constexpr int kOffP = kOffQ + kQBytes;
-constexpr int kOffKV = kOffP + 2 * kPBytes;    // P is double buffered: softmax of block n+1 overlaps P V of block n
-constexpr int kOffBar = kOffKV + kKVStages * kKVStageBytes;
-constexpr int kNumBars = 2 * kKVStages + 1 + 2 + 2 + 2 + 2 + 1 + 1;
-constexpr int kSmemBytes = kOffBar + kNumBars * 8 + 16 + 1024;
+constexpr int kOffQ = 0;                       // two Q buffers: item i uses buffer i & 1
+constexpr int kOffKV = kOffQ + 2 * kQBytes;
+constexpr int kOffML = kOffKV + kKVStages * kKVStageBytes;   // float2 [2 groups][128 rows]: (reference max, sum)
+constexpr int kOffBar = kOffML + 2 * 128 * 8;
+constexpr int kNumBars = 2 * kKVStages + 2 + 2 + 2 + 2 + 2 + 1;
+constexpr int kSmemBytes = kOffBar + kNumBars * 8 + 16 + 32;   // barriers, TMEM slot + flags + item range, first item
+static_assert(kSmemBytes <= 227 * 1024, "shared memory budget");
 
 struct TcAttnParams {
   const AttnItem* items;
@@ -53,7 +78,6 @@ struct TcAttnParams {
   const int* tok_climit;
   const int* tok_lo;
   const int* tok_hi;
-  const __nv_bfloat16* q;
   __nv_bfloat16* o;
   const __nv_bfloat16* pool;
   int64_t n_pages;
@@ -92,6 +116,15 @@ __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t da, uint64_t
       " tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
       :
       : "r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// A operand (M x 16 bf16, two K elements per 32-bit column) read from TMEM instead of shared memory
+__device__ __forceinline__ void umma_bf16_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t db, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
+      " tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}"
+      :
+      : "r"(tmem_d), "r"(tmem_a), "l"(db), "r"(idesc), "r"(accumulate)
       : "memory");
 }
 __device__ __forceinline__ void tmem_ld32_nowait(uint32_t taddr, uint32_t (&r)[32]) {
@@ -137,46 +170,86 @@ constexpr uint32_t kIdescPV =
 __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
   asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
-__device__ __forceinline__ void softmax_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+__device__ __forceinline__ void tma_load_3d(uint32_t smem_dst, const CUtensorMap* map, int x, int y, int z, uint64_t* bar) {
+  asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+               :
+               : "r"(smem_dst), "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y), "r"(z)
+               : "memory");
+}
+__device__ __forceinline__ void softmax_bar() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void reg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
+template <int N> __device__ __forceinline__ void reg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
 
-__global__ void __launch_bounds__(kThreads, 1) attention_tc_kernel(TcAttnParams P) {
-  extern __shared__ uint8_t smem_raw[];
-  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+
+__global__ void __launch_bounds__(kThreads, 1) attention_tc_kernel(const __grid_constant__ CUtensorMap qmap, TcAttnParams P) {
+  extern __shared__ __align__(1024) uint8_t smem[];
+  if (smem_u32(smem) & 1023u) {          // the swizzled operand layouts need a 1 KB aligned base
+    if (threadIdx.x == 0) set_status(P.status, DEV_BAD_INDEX);
+    return;
+  }
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kOffBar);
-  uint64_t* kv_full = bars;                 // [kKVStages]
+  uint64_t* kv_full = bars;                 // [kKVStages]: K ring first, then V ring
   uint64_t* kv_empty = bars + kKVStages;    // [kKVStages]
-  uint64_t* q_full = bars + 2 * kKVStages;
-  uint64_t* s_full = q_full + 1;            // [2]
-  uint64_t* s_empty = q_full + 3;           // [2]
-  uint64_t* p_full = q_full + 5;            // [2]
-  uint64_t* p_empty = q_full + 7;           // [2]
-  uint64_t* o_full = q_full + 9;
+  uint64_t* q_full = bars + 2 * kKVStages;  // [2]  per Q buffer
+  uint64_t* q_empty = q_full + 2;           // [2]
+  uint64_t* s_full = q_full + 4;            // [2]  per softmax group
+  uint64_t* p_full = q_full + 6;            // [2]
+  uint64_t* o_full = q_full + 8;            // [2]
   uint64_t* o_empty = q_full + 10;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + kNumBars);
+  float2* ml_smem = reinterpret_cast<float2*>(smem + kOffML);
+
+  // A wait that runs out records why and raises this flag; from then on no wait in this CTA blocks any more, so
+  // every warp still walks through its loops (and meets the others at the named barriers) and the kernel ends.
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  auto bwait = [&](uint64_t* bar, uint32_t parity, int code) {
+    if (*abort_flag) return;
+    if (!mbar_wait(bar, parity, kSpin)) {
+      set_status(P.status, code);
+      *abort_flag = 1;
+    }
+  };
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  if (threadIdx.x == 0) {
+  // Warp 0 waits for the kernels before this one and fetches the CTA's item range and first item while the other
+  // warps set up barriers, the zeroed ring and TMEM: two dependent round trips off everybody's critical path.
+  int* s_range = reinterpret_cast<int*>(tmem_slot + 2);
+  AttnItem* s_first = reinterpret_cast<AttnItem*>(tmem_slot + 4);
+  int item_begin = 0, item_end = 0;
+  AttnItem w_next = {};
+  if (warp == 0) {
+    griddep_wait();
+    item_begin = P.cta_off[blockIdx.x];
+    item_end = P.cta_off[blockIdx.x + 1];
+    if (item_begin < item_end) w_next = P.items[item_begin];
+    if (lane == 0) {
+      s_range[0] = item_begin;
+      s_range[1] = item_end;
+      *s_first = w_next;
+    }
+  }
+  if (threadIdx.x == 32) {
+    *abort_flag = 0;
     for (int s = 0; s < kKVStages; ++s) {
       mbar_init(&kv_full[s], 1);
       mbar_init(&kv_empty[s], 1);
     }
-    mbar_init(q_full, 1);
     for (int s = 0; s < 2; ++s) {
+      mbar_init(&q_full[s], 1);
+      mbar_init(&q_empty[s], 8);
       mbar_init(&s_full[s], 1);
-      mbar_init(&s_empty[s], 4);
-    }
-    for (int s = 0; s < 2; ++s) {
       mbar_init(&p_full[s], 4);
-      mbar_init(&p_empty[s], 1);
+      mbar_init(&o_full[s], 1);
     }
-    mbar_init(o_full, 1);
-    mbar_init(o_empty, 4);
+    mbar_init(o_empty, 8);
     fence_barrier_init();
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&qmap) : "memory");
   }
   // The operand ring starts out zeroed: later on a buffer only ever holds zeros, real K/V pages or hand-copied
   // pages, so V rows that no copy refreshes (pages beyond a request's end) are finite and 0 * V stays 0.
-  for (int c = threadIdx.x; c < kKVStages * kKVStageBytes / 16; c += kThreads)
-    reinterpret_cast<uint4*>(smem + kOffKV)[c] = make_uint4(0, 0, 0, 0);
+  if (warp != 0)
+    for (int c = threadIdx.x - 32; c < kKVStages * kKVStageBytes / 16; c += kThreads - 32)
+      reinterpret_cast<uint4*>(smem + kOffKV)[c] = make_uint4(0, 0, 0, 0);
   fence_proxy_async();
   if (warp == 1) {
     tmem_alloc(tmem_slot, kTmemCols);
@@ -186,56 +259,70 @@ __global__ void __launch_bounds__(kThreads, 1) attention_tc_kernel(TcAttnParams 
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  griddep_wait();   // everything above touched only shared memory and TMEM
-  const int item_begin = P.cta_off[blockIdx.x], item_end = P.cta_off[blockIdx.x + 1];
+  if (warp != 0) {
+    griddep_wait();   // these warps touched only shared memory and TMEM so far
+    item_begin = s_range[0];
+    item_end = s_range[1];
+    w_next = *s_first;
+  }
   const uint32_t smem_base = smem_u32(smem);
 
-  if (warp == 0 || warp == 6) {
-    // ------------------------------------ producers: warp 0 streams K, warp 6 streams V ------------------------------------
-    const int my_part = warp == 0 ? 0 : 1;
-    uint32_t blk = 0;  // running KV-block counter
-    bool ok = true;
-    for (int item = item_begin; item < item_end && ok; ++item) {
-      const AttnItem w = P.items[item];
-      const int tok_begin = w.blk_begin * 64;
-      const int tok_end = min(w.blk_end * 64, w.kv_len);
-      const int nblk = (tok_end - tok_begin + kBT - 1) / kBT;
-      const int n_req_pages = (w.kv_len + kPageSize - 1) / kPageSize;
-      const int* pt = P.page_table + (size_t)w.req * P.pt_stride;
-      // page ids are fetched by lanes 0..7 in parallel, one iteration ahead of their use
-      auto fetch_page = [&](int n) -> int {
-        int pg = -1;
-        if (lane < kPagesPerBT && n < nblk) {
-          const int lp = tok_begin / kPageSize + n * kPagesPerBT + lane;
-          if (lp < n_req_pages && lp * kPageSize < tok_end) pg = __ldg(pt + lp);   // validated when used
-        }
-        return pg;
-      };
-      int pg_next = fetch_page(0);
-      for (int n = 0; n < nblk && ok; ++n, ++blk) {
-        int my_pg = pg_next;
-        pg_next = fetch_page(n + 1);                 // in flight during this iteration
-        if (my_pg >= P.n_pages) {
-          set_status(P.status, DEV_BAD_INDEX);
-          my_pg = -1;
-        }
-        // lane p < 8 owns page p of the block: full pages go by bulk copy, the rest by hand
-        const int first_tok = tok_begin + (n * kPagesPerBT + lane) * kPageSize;
-        const int my_valid = (lane < kPagesPerBT && my_pg >= 0) ? min(kPageSize, w.kv_len - first_tok) : 0;
-        // K: every existing page goes by bulk copy (rows beyond the request's end are masked in S).
-        // V: full pages by bulk copy; the one partly filled page by hand with its stale rows zeroed (0 * stale
-        // could be NaN); pages beyond the end are not touched (the buffer holds finite data, see the start).
-        const bool my_bulk = my_part == 0 ? my_valid > 0 : my_valid == kPageSize;
-        const unsigned bulk_mask = __ballot_sync(0xffffffffu, my_bulk);
-        const unsigned hand_mask = my_part == 0 ? 0u : __ballot_sync(0xffffffffu, my_valid > 0 && my_valid < kPageSize);
-        for (int part = my_part; part <= my_part; ++part) {       // 0: the K operand, 1: the V operand
-          const uint32_t qi = 2 * blk + part;
-          const int s = qi % kKVStages;
-          if (!mbar_wait(&kv_empty[s], ((qi / kKVStages) & 1) ^ 1, kSpin)) {
-            set_status(P.status, DEV_TIMEOUT_EMPTY);
-            ok = false;
-            break;
+  if (warp < 4) {
+    reg_dec<64>();
+    if (warp == 0 || warp == 2) {
+      // ------------------------------------ producers: warp 0 streams Q and K, warp 2 streams V ------------------------------------
+      const int part = warp == 0 ? 0 : 1;
+      uint32_t blk = 0, item_cnt = 0;  // running KV-block and item counters
+      for (int item = item_begin; item < item_end; ++item, ++item_cnt) {
+        const AttnItem w = w_next;
+        if (item + 1 < item_end) w_next = P.items[item + 1];
+        const int tok_begin = w.blk_begin * 64;
+        const int tok_end = min(w.blk_end * 64, w.kv_len);
+        const int nblk = (tok_end - tok_begin + kBT - 1) / kBT;
+        const int n_req_pages = (w.kv_len + kPageSize - 1) / kPageSize;
+        const int* pt = P.page_table + (size_t)w.req * P.pt_stride;
+        // page ids are fetched by lanes 0..7 in parallel, one iteration ahead of their use
+        auto fetch_page = [&](int n) -> int {
+          int pg = -1;
+          if (lane < kPagesPerBT && n < nblk) {
+            const int lp = tok_begin / kPageSize + n * kPagesPerBT + lane;
+            if (lp < n_req_pages && lp * kPageSize < tok_end) pg = __ldg(pt + lp);   // validated when used
           }
+          return pg;
+        };
+        int pg_next = fetch_page(0);
+        if (part == 0) {
+          // Q rows of the item: (64 dims) x (the kv head's query heads) x (128 / group tokens from tok0); rows past the
+          // tile's own tokens belong to other tokens or are zero-filled, and nobody reads their S / O rows
+          const int buf = item_cnt & 1;
+          bwait(&q_empty[buf], ((item_cnt >> 1) & 1) ^ 1, DEV_TIMEOUT_EMPTY);
+          if (lane == 0) {
+            mbar_arrive_expect_tx(&q_full[buf], kQBytes);
+            const uint32_t dst = smem_base + kOffQ + buf * kQBytes;
+            tma_load_3d(dst, &qmap, 0, w.kv_head * P.group, w.tok0, &q_full[buf]);
+            tma_load_3d(dst + kQBytes / 2, &qmap, 64, w.kv_head * P.group, w.tok0, &q_full[buf]);
+          }
+          __syncwarp();
+        }
+        for (int n = 0; n < nblk; ++n, ++blk) {
+          int my_pg = pg_next;
+          pg_next = fetch_page(n + 1);                 // in flight during this iteration
+          if (my_pg >= P.n_pages) {
+            set_status(P.status, DEV_BAD_INDEX);
+            my_pg = -1;
+          }
+          // lane p < 8 owns page p of the block: full pages go by bulk copy, the rest by hand
+          const int first_tok = tok_begin + (n * kPagesPerBT + lane) * kPageSize;
+          const int my_valid = (lane < kPagesPerBT && my_pg >= 0) ? min(kPageSize, w.kv_len - first_tok) : 0;
+          // K: every existing page goes by bulk copy (rows beyond the request's end are masked in S).
+          // V: full pages by bulk copy; the one partly filled page by hand with its stale rows zeroed (0 * stale
+          // could be NaN); pages beyond the end are not touched (the buffer holds finite data, see the start).
+          const bool my_bulk = part == 0 ? my_valid > 0 : my_valid == kPageSize;
+          const unsigned bulk_mask = __ballot_sync(0xffffffffu, my_bulk);
+          const unsigned hand_mask = part == 0 ? 0u : __ballot_sync(0xffffffffu, my_valid > 0 && my_valid < kPageSize);
+          const int ring = part == 0 ? kKStages : kVStages;
+          const int s = (part == 0 ? 0 : kKStages) + blk % ring;
+          bwait(&kv_empty[s], ((blk / ring) & 1) ^ 1, DEV_TIMEOUT_EMPTY);
           uint8_t* stage = smem + kOffKV + s * kKVStageBytes;
           if (hand_mask) {
             const int p = __ffs(hand_mask) - 1;            // at most one partly filled page per request
@@ -243,16 +330,14 @@ __global__ void __launch_bounds__(kThreads, 1) attention_tc_kernel(TcAttnParams 
             const int valid_tok = __shfl_sync(0xffffffffu, my_valid, p);
             const uint4* src = reinterpret_cast<const uint4*>(
                                    P.pool + kv_tile_base(P.n_pages, P.n_kv, D, P.layer, pg, w.kv_head)) + part * 256;
-            uint4 v[8];
 #pragma unroll
             for (int u = 0; u < 8; ++u) {
               const int c = u * 32 + lane;
-              v[u] = (((c >> 7) * 8 + ((c >> 3) & 7)) < valid_tok) ? __ldg(src + c) : make_uint4(0, 0, 0, 0);
+              const uint4 v = (((c >> 7) * 8 + ((c >> 3) & 7)) < valid_tok) ? __ldg(src + c) : make_uint4(0, 0, 0, 0);
+              *reinterpret_cast<uint4*>(stage + p * kTileBytes + c * 16) = v;
             }
-#pragma unroll
-            for (int u = 0; u < 8; ++u) *reinterpret_cast<uint4*>(stage + p * kTileBytes + (u * 32 + lane) * 16) = v[u];
+            fence_proxy_async();
           }
-          if (hand_mask) fence_proxy_async();
           __syncwarp();
           if (lane == 0) {
             if (bulk_mask == 0) mbar_arrive(&kv_full[s]);
@@ -268,147 +353,117 @@ __global__ void __launch_bounds__(kThreads, 1) attention_tc_kernel(TcAttnParams 
           __syncwarp();
         }
       }
-    }
-    if (!ok && lane == 0) {
-      for (int s = 0; s < kKVStages; ++s)
-        for (uint32_t i = 0; i < (1u << 14); ++i) {
-          if (mbar_try_wait(&kv_full[s], 0) || mbar_try_wait(&kv_full[s], 1)) break;
-          __nanosleep(64);
-        }
-    }
-  } else if (warp == 1) {
-    // ------------------------------------ MMA issuer ------------------------------------
-    if (elect_one()) {
-      uint32_t blk = 0, item_cnt = 0, pv_cnt = 0;
-      bool ok = true;
-      const uint32_t q_addr = smem_base + kOffQ, p_addr = smem_base + kOffP;
-      auto issue_qk = [&](uint32_t b) -> bool {   // S[b & 1] = Q K^T for running block b
-        const uint32_t qi = 2 * b;
-        const int s = qi % kKVStages, sb = b & 1;
-        if (!mbar_wait(&kv_full[s], (qi / kKVStages) & 1, kSpin)) { set_status(P.status, DEV_TIMEOUT_FULL); return false; }
-        if (!mbar_wait(&s_empty[sb], ((b >> 1) & 1) ^ 1, kSpin)) { set_status(P.status, DEV_TIMEOUT_MMA); return false; }
-        tc_fence_after();
-        const uint32_t k_addr = smem_base + kOffKV + s * kKVStageBytes;
-#pragma unroll
-        for (int kk = 0; kk < D / 16; ++kk) {
-          const uint64_t da = desc_kmajor(q_addr + (kk >> 2) * (128 * 128) + (kk & 3) * 32);
-          // K block: 16 token groups (2 per page) 2 KB apart; the dim half selects the atom next door
-          const uint64_t db = desc_kmajor(k_addr + (kk >> 2) * 1024 + (kk & 3) * 32, 2048);
-          umma_bf16(tmem_base + sb * kBT, da, db, kIdescQK, kk ? 1u : 0u);
-        }
-        umma_commit(&kv_empty[s]);   // the K buffer is free once these MMAs have read it
-        umma_commit(&s_full[sb]);
-        return true;
-      };
-      for (int item = item_begin; item < item_end && ok; ++item, ++item_cnt) {
-        const AttnItem w = P.items[item];
-        const int tok_begin = w.blk_begin * 64;
-        const int tok_end = min(w.blk_end * 64, w.kv_len);
-        const int nblk = (tok_end - tok_begin + kBT - 1) / kBT;
-        if (!mbar_wait(q_full, item_cnt & 1, kSpin)) { set_status(P.status, DEV_TIMEOUT_FULL); break; }
-        // the previous item's O must have been read out before this item's first P V overwrites it
-        if (!mbar_wait(o_empty, (item_cnt & 1) ^ 1, kSpin)) { set_status(P.status, DEV_TIMEOUT_MMA); break; }
-        tc_fence_after();
-        if (!(ok = issue_qk(blk))) break;
-        for (int n = 0; n < nblk && ok; ++n, ++blk, ++pv_cnt) {
-          if (n + 1 < nblk && !(ok = issue_qk(blk + 1))) break;
-          // O (+)= P V for block n
-          const int pb = pv_cnt & 1;
-          if (!mbar_wait(&p_full[pb], (pv_cnt >> 1) & 1, kSpin)) {
-            set_status(P.status, DEV_TIMEOUT_MMA);
-            ok = false;
-            break;
+      if (*abort_flag && lane == 0) {     // gave up somewhere: let this warp's copies in flight land before exiting
+        for (int s = 0; s < kKVStages; ++s)
+          for (uint32_t i = 0; i < (1u << 14); ++i) {
+            if (mbar_try_wait(&kv_full[s], 0) || mbar_try_wait(&kv_full[s], 1)) break;
+            __nanosleep(64);
           }
-          const uint32_t qv = 2 * blk + 1;
-          const int s = qv % kKVStages;
-          if (!mbar_wait(&kv_full[s], (qv / kKVStages) & 1, kSpin)) {
-            set_status(P.status, DEV_TIMEOUT_FULL);
-            ok = false;
-            break;
-          }
+      }
+    } else if (warp == 1) {
+      // ------------------------------------ MMA issuer ------------------------------------
+      if (elect_one()) {
+        uint32_t blk = 0, item_cnt = 0;
+        uint32_t cp[2] = {0, 0};   // P V products issued for each softmax group so far
+        // S of group g = Q K^T for running block b.  The tensor pipe executes in issue order, so this runs after the
+        // group's previous P V, which read P out of the same TMEM columns.
+        auto issue_qk = [&](uint32_t b, int g, uint32_t q_addr) {
+          const int s = b % kKStages;
+          bwait(&kv_full[s], (b / kKStages) & 1, DEV_TIMEOUT_FULL);
           tc_fence_after();
-          const uint32_t v_addr = smem_base + kOffKV + s * kKVStageBytes;
+          const uint32_t k_addr = smem_base + kOffKV + s * kKVStageBytes;
 #pragma unroll
-          for (int kk = 0; kk < kBT / 16; ++kk) {
-            const uint64_t da = desc_kmajor(p_addr + pb * kPBytes + (kk >> 2) * (128 * 128) + (kk & 3) * 32);
-            // tokens [16 kk, 16 kk + 16) = page kk: two token groups 2 KB apart, the dim halves 1 KB apart
-            const uint64_t db = desc_mnmajor(v_addr + kk * kTileBytes, 1024, 2048);
-            umma_bf16(tmem_base + 2 * kBT, da, db, kIdescPV, (n | kk) ? 1u : 0u);
+          for (int kk = 0; kk < D / 16; ++kk) {
+            const uint64_t da = desc_kmajor(q_addr + (kk >> 2) * (128 * 128) + (kk & 3) * 32);
+            // K block: 16 token groups (2 per page) 2 KB apart; the dim half selects the atom next door
+            const uint64_t db = desc_kmajor(k_addr + (kk >> 2) * 1024 + (kk & 3) * 32, 2048);
+            umma_bf16(tmem_base + g * kBT, da, db, kIdescQK, kk ? 1u : 0u);
           }
-          umma_commit(&kv_empty[s]);
-          umma_commit(&p_empty[pb]);
-          if (n == nblk - 1) umma_commit(o_full);
+          umma_commit(&kv_empty[s]);   // the K buffer is free once these MMAs have read it
+          umma_commit(&s_full[g]);
+        };
+        for (int item = item_begin; item < item_end; ++item, ++item_cnt) {
+          const AttnItem w = w_next;
+          if (item + 1 < item_end) w_next = P.items[item + 1];
+          const int tok_begin = w.blk_begin * 64;
+          const int tok_end = min(w.blk_end * 64, w.kv_len);
+          const int nblk = (tok_end - tok_begin + kBT - 1) / kBT;
+          const int buf = item_cnt & 1;
+          const uint32_t q_addr = smem_base + kOffQ + buf * kQBytes;
+          bwait(&q_full[buf], (item_cnt >> 1) & 1, DEV_TIMEOUT_FULL);
+          tc_fence_after();
+          issue_qk(blk, 0, q_addr);
+          if (nblk > 1) issue_qk(blk + 1, 1, q_addr);
+          for (int n = 0; n < nblk; ++n, ++blk) {
+            const int g = n & 1;
+            // O of group g (+)= P V for block n: P (bf16, two tokens per 32-bit column) is read from TMEM
+            bwait(&p_full[g], cp[g] & 1, DEV_TIMEOUT_MMA);
+            ++cp[g];
+            // the previous item's accumulators must have been read out before this item's first products overwrite them
+            if (n < 2) bwait(o_empty, (item_cnt & 1) ^ 1, DEV_TIMEOUT_MMA);
+            const int s = kKStages + blk % kVStages;
+            bwait(&kv_full[s], (blk / kVStages) & 1, DEV_TIMEOUT_FULL);
+            tc_fence_after();
+            const uint32_t v_addr = smem_base + kOffKV + s * kKVStageBytes;
+#pragma unroll
+            for (int kk = 0; kk < kBT / 16; ++kk) {
+              // tokens [16 kk, 16 kk + 16) = page kk: two token groups 2 KB apart, the dim halves 1 KB apart
+              const uint64_t db = desc_mnmajor(v_addr + kk * kTileBytes, 1024, 2048);
+              umma_bf16_ts(tmem_base + kTmemO + g * D, tmem_base + g * kBT + kk * 8, db, kIdescPV, (n >= 2 || kk) ? 1u : 0u);
+            }
+            umma_commit(&kv_empty[s]);
+            if (n + 2 >= nblk) umma_commit(&o_full[g]);   // the last block of this group in the item
+            if (n + 2 < nblk) issue_qk(blk + 2, g, q_addr);
+          }
         }
       }
     }
-  } else if (warp < 6) {
+  } else {
+    reg_inc<216>();
     // ------------------------------------ softmax ------------------------------------
+    const int g = (warp - 4) >> 2;             // softmax group: takes blocks n = g, g + 2, ... of every item
     const int quad = warp & 3;
     const int row = quad * 32 + lane;          // query row of the tile = TMEM lane
-    const int sthread = (warp - 2) * 32 + lane;
     const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
-    uint32_t blk = 0, pv_cnt = 0, item_cnt = 0;
-    bool ok = true;
-    for (int item = item_begin; item < item_end && ok; ++item) {
-      const AttnItem w = P.items[item];
+    const uint32_t s_addr = lane_addr + g * kBT, o_addr = lane_addr + kTmemO + g * D;
+    uint32_t cs = 0, item_cnt = 0, o1_cnt = 0;   // blocks this group has taken; items; items with two or more blocks
+    // visibility triple of this thread's row, fetched one item ahead
+    auto row_vis = [&](const AttnItem& it, int& cl, int& lo, int& hi) {
+      cl = -1; lo = 0; hi = 0;
+      if (row < it.ntok * P.group) {
+        const int t = it.tok0 + row / P.group;
+        cl = P.tok_climit[t];
+        lo = P.tok_lo[t];
+        hi = P.tok_hi[t];
+      }
+    };
+    int nx_cl = -1, nx_lo = 0, nx_hi = 0;
+    if (item_begin < item_end) row_vis(w_next, nx_cl, nx_lo, nx_hi);
+    for (int item = item_begin; item < item_end; ++item) {
+      const AttnItem w = w_next;
+      if (item + 1 < item_end) w_next = P.items[item + 1];
       const int R = w.ntok * P.group;
       const int tok_begin = w.blk_begin * 64;
       const int tok_end = min(w.blk_end * 64, w.kv_len);
       const int nblk = (tok_end - tok_begin + kBT - 1) / kBT;
-      // ---- stage Q in operand layout: [2 halves][128 rows][128 B], 16-byte chunks swizzled by row & 7 ----
-      // only the R valid rows are staged: the other rows of the M = 128 operand yield S / O rows nobody reads.
-      // Loads are issued in batches of 8 before any store so that their latencies overlap.
-      for (int c0 = 0; c0 < R * 16; c0 += 128 * 8) {
-        uint4 v[8];
-#pragma unroll
-        for (int u = 0; u < 8; ++u) {
-          const int c = c0 + u * 128 + sthread;
-          v[u] = make_uint4(0, 0, 0, 0);
-          if (c < R * 16) {
-            const int r = c >> 4, ch = c & 15;
-            const int j = r / P.group, hg = r % P.group;
-            v[u] = __ldg(reinterpret_cast<const uint4*>(P.q + ((size_t)(w.tok0 + j) * P.n_q + w.kv_head * P.group + hg) * D) + ch);
-          }
-        }
-#pragma unroll
-        for (int u = 0; u < 8; ++u) {
-          const int c = c0 + u * 128 + sthread;
-          if (c < R * 16) {
-            const int r = c >> 4, ch = c & 15;
-            *reinterpret_cast<uint4*>(smem + kOffQ + (ch >> 3) * (128 * 128) + r * 128 + (((ch & 7) ^ (r & 7)) << 4)) = v[u];
-          }
-        }
-      }
-      fence_proxy_async();
-      softmax_bar();
-      if (sthread == 0) mbar_arrive(q_full);
-
       const bool rvalid = row < R;
       const bool warp_valid = quad * 32 < R;
-      int climit = -1, vlo = 0, vhi = 0;
-      if (rvalid) {
-        const int t = w.tok0 + row / P.group;
-        climit = P.tok_climit[t];
-        vlo = P.tok_lo[t];
-        vhi = P.tok_hi[t];
-      }
+      const int climit = nx_cl, vlo = nx_lo, vhi = nx_hi;
       float m_ref = -1e30f, l_run = 0.f;
-      const uint32_t p_row0 = smem_base + kOffP + row * 128;
+      bool first = true;
 
-      for (int n = 0; n < nblk && ok; ++n, ++blk, ++pv_cnt) {
-        const int sb = blk & 1;
-        if (!mbar_wait(&s_full[sb], (blk >> 1) & 1, kSpin)) { set_status(P.status, DEV_TIMEOUT_MMA); ok = false; break; }
+      for (int n = g; n < nblk; n += 2, ++cs) {
+        bwait(&s_full[g], cs & 1, DEV_TIMEOUT_MMA);
         tc_fence_after();
         const int pos0 = tok_begin + n * kBT;
         uint32_t sr[4][32];   // the S row of this thread: 128 scores
         float mx = -INFINITY;
-        bool need_mask = false;
         if (warp_valid) {
 #pragma unroll
-          for (int c = 0; c < 4; ++c) tmem_ld32_nowait(lane_addr + sb * kBT + c * 32, sr[c]);
+          for (int c = 0; c < 4; ++c) tmem_ld32_nowait(s_addr + c * 32, sr[c]);
           tmem_ld_wait();
           const int lim = min(climit, tok_end - 1);
-          need_mask = __any_sync(0xffffffffu, rvalid && (pos0 + kBT - 1 > lim));
+          const bool need_mask = __any_sync(0xffffffffu, rvalid && (pos0 + kBT - 1 > lim));
           if (need_mask) {
             // visible tokens of this row within the block: [0, a] and [b, c), as a 128-bit mask over tokens
             const int a = lim - pos0, b = vlo - pos0, cc = min(vhi, tok_end) - pos0;
@@ -435,111 +490,140 @@ __global__ void __launch_bounds__(kThreads, 1) attention_tc_kernel(TcAttnParams 
                 mxa[c] = fmaxf(mxa[c], fmaxf(__uint_as_float(sr[c][i]), __uint_as_float(sr[c][i + 1])));
             mx = fmaxf(fmaxf(mxa[0], mxa[1]), fmaxf(mxa[2], mxa[3]));
           }
-        }
-        // S has been read: the MMA warp may overwrite this buffer with the block after next
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&s_empty[sb]);
-        // the P V that last read this P buffer (two blocks ago) must be complete before it is overwritten
-        const int pb = pv_cnt & 1;
-        const uint32_t p_row = p_row0 + pb * kPBytes;
-        if (!mbar_wait(&p_empty[pb], ((pv_cnt >> 1) & 1) ^ 1, kSpin)) { set_status(P.status, DEV_TIMEOUT_MMA); ok = false; break; }
-        if (warp_valid) {
+          // This S was produced after the group's previous P V in tensor-pipe order, so that product is complete:
+          // O may be rescaled and the P columns rewritten.
           const float m_blk = mx * P.scale_log2;
           // move the reference maximum only when the row maximum outgrows it by more than 2^8 (or at the first
           // block): probabilities stay below 256 relative to the reference, well inside bf16 and fp32 range
           const bool grow = rvalid && (m_blk > m_ref + 8.f);
-          if (n == 0) {
+          if (n == g) {
             if (rvalid && m_blk > m_ref) m_ref = m_blk;
           } else if (__any_sync(0xffffffffu, grow)) {
-            // rare: O is rescaled in TMEM, which needs EVERY earlier P V complete (the previous one may still run)
-            if (!mbar_wait(&p_empty[pb ^ 1], (((pv_cnt - 1) >> 1) & 1), kSpin)) { set_status(P.status, DEV_TIMEOUT_MMA); ok = false; break; }
+            // rare: O is rescaled in TMEM
             const float m_new = grow ? m_blk : m_ref;
             const float f = exp2f(m_ref - m_new);
             m_ref = m_new;
             l_run *= f;
-            tc_fence_after();
 #pragma unroll 1
             for (int c = 0; c < D / 32; ++c) {
               uint32_t r[32];
-              tmem_ld32_nowait(lane_addr + 2 * kBT + c * 32, r);
+              tmem_ld32_nowait(o_addr + c * 32, r);
               tmem_ld_wait();
 #pragma unroll
               for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * f);
-              tmem_st32(lane_addr + 2 * kBT + c * 32, r);
+              tmem_st32(o_addr + c * 32, r);
             }
             tmem_st_wait();
           }
           float lsa[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-          for (int c = 0; c < 4; ++c) {
+          for (int h = 0; h < 2; ++h) {      // 64 tokens -> 32 packed columns [32 h, 32 h + 32) of this group's S buffer
+            uint32_t pk[32];
 #pragma unroll
-            for (int i = 0; i < 32; ++i) {
-              const float p = exp2f(__uint_as_float(sr[c][i]) * P.scale_log2 - m_ref);   // exp2(-inf) = 0 for masked
-              sr[c][i] = __float_as_uint(p);
-              lsa[i & 3] += p;
-            }
-            if (rvalid) {
+            for (int cc = 0; cc < 2; ++cc) {
+              const int c = 2 * h + cc;
 #pragma unroll
-              for (int j = 0; j < 4; ++j) {
-                const int ch = c * 4 + j;   // 16-byte chunk (8 tokens) of the row: half = ch >> 3
-                st_shared_v4(p_row + (ch >> 3) * (128 * 128) + (((ch & 7) ^ (row & 7)) << 4),
-                             pack_bf16(__uint_as_float(sr[c][8 * j]), __uint_as_float(sr[c][8 * j + 1])),
-                             pack_bf16(__uint_as_float(sr[c][8 * j + 2]), __uint_as_float(sr[c][8 * j + 3])),
-                             pack_bf16(__uint_as_float(sr[c][8 * j + 4]), __uint_as_float(sr[c][8 * j + 5])),
-                             pack_bf16(__uint_as_float(sr[c][8 * j + 6]), __uint_as_float(sr[c][8 * j + 7])));
+              for (int i = 0; i < 32; i += 2) {
+                const float p0 = exp2f(__uint_as_float(sr[c][i]) * P.scale_log2 - m_ref);   // exp2(-inf) = 0 for masked
+                const float p1 = exp2f(__uint_as_float(sr[c][i + 1]) * P.scale_log2 - m_ref);
+                lsa[(i >> 1) & 3] += p0 + p1;
+                pk[cc * 16 + (i >> 1)] = pack_bf16(p0, p1);
               }
             }
+            tmem_st32(s_addr + h * 32, pk);
           }
           l_run += (lsa[0] + lsa[1]) + (lsa[2] + lsa[3]);
+          tmem_st_wait();
         }
         tc_fence_before();
-        fence_proxy_async();
         __syncwarp();
-        if (lane == 0) mbar_arrive(&p_full[pb]);
+        if (lane == 0) mbar_arrive(&p_full[g]);
+        if (first) {      // the next item's descriptor has arrived by now: fetch its rows' visibility for later
+          first = false;
+          if (item + 1 < item_end) row_vis(w_next, nx_cl, nx_lo, nx_hi);
+        }
       }
-      if (!ok) break;
+      if (first && item + 1 < item_end) row_vis(w_next, nx_cl, nx_lo, nx_hi);   // this group had no block in the item
 
-      // ---- read O once, write out: one row per thread ----
-      if (!mbar_wait(o_full, item_cnt & 1, kSpin)) { set_status(P.status, DEV_TIMEOUT_MMA); ok = false; break; }
+      // ---- merge the two groups' partial attentions and write out: this group finishes dims [64 g, 64 g + 64) ----
+      const bool two = nblk >= 2;                 // group 1 took part in this item
+      const int buf = item_cnt & 1;
+      bwait(&o_full[0], item_cnt & 1, DEV_TIMEOUT_MMA);
+      if (two) {
+        bwait(&o_full[1], o1_cnt & 1, DEV_TIMEOUT_MMA);
+        ++o1_cnt;
+      }
       tc_fence_after();
+      ml_smem[g * 128 + row] = make_float2(m_ref, l_run);
+      softmax_bar();
       if (warp_valid) {
+        const float2 a0 = ml_smem[row];
+        const float2 a1 = two ? ml_smem[128 + row] : make_float2(-1e30f, 0.f);
+        const float m_all = fmaxf(a0.x, a1.x);
+        float f0 = exp2f(a0.x - m_all), f1 = two ? exp2f(a1.x - m_all) : 0.f;
+        const float l_all = a0.y * f0 + a1.y * f1;
+        const float inv = (w.part < 0) ? (l_all > 0.f ? 1.f / l_all : 0.f) : 1.f;
+        f0 *= inv;
+        f1 *= inv;
         const int j = row / P.group, hg = row % P.group;
-        const float inv = (w.part < 0) ? (l_run > 0.f ? 1.f / l_run : 0.f) : 1.f;
+        // all MMAs of the item are complete, so its Q buffer is free: 4 KB of it per warp serve as transposition space
+        float* stg = reinterpret_cast<float*>(smem + kOffQ + buf * kQBytes) + (warp - 4) * 1024;
+        const int nrow = min(32, R - quad * 32);
 #pragma unroll 1
-        for (int c = 0; c < D / 32; ++c) {
+        for (int cc = 0; cc < 2; ++cc) {
+          const int c = 2 * g + cc;               // 32-dim chunk of the output row
           uint32_t r[32];
-          tmem_ld32_nowait(lane_addr + 2 * kBT + c * 32, r);
+          tmem_ld32_nowait(lane_addr + kTmemO + c * 32, r);
           tmem_ld_wait();
-          if (!rvalid) continue;
-          if (w.part < 0) {
-            uint4* dst = reinterpret_cast<uint4*>(P.o + ((size_t)(w.tok0 + j) * P.n_q + w.kv_head * P.group + hg) * D + c * 32);
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-              uint4 v;
-              v.x = pack_bf16(__uint_as_float(r[8 * i]) * inv, __uint_as_float(r[8 * i + 1]) * inv);
-              v.y = pack_bf16(__uint_as_float(r[8 * i + 2]) * inv, __uint_as_float(r[8 * i + 3]) * inv);
-              v.z = pack_bf16(__uint_as_float(r[8 * i + 4]) * inv, __uint_as_float(r[8 * i + 5]) * inv);
-              v.w = pack_bf16(__uint_as_float(r[8 * i + 6]) * inv, __uint_as_float(r[8 * i + 7]) * inv);
-              dst[i] = v;
+          for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * f0);
+          if (two) {
+            uint32_t r1[32];
+            tmem_ld32_nowait(lane_addr + kTmemO + D + c * 32, r1);
+            tmem_ld_wait();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(fmaf(__uint_as_float(r1[i]), f1, __uint_as_float(r[i])));
+          }
+          if (w.part < 0) {
+            if (rvalid) {
+              uint4* dst = reinterpret_cast<uint4*>(P.o + ((size_t)(w.tok0 + j) * P.n_q + w.kv_head * P.group + hg) * D + c * 32);
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                uint4 v;
+                v.x = pack_bf16(__uint_as_float(r[8 * i]), __uint_as_float(r[8 * i + 1]));
+                v.y = pack_bf16(__uint_as_float(r[8 * i + 2]), __uint_as_float(r[8 * i + 3]));
+                v.z = pack_bf16(__uint_as_float(r[8 * i + 4]), __uint_as_float(r[8 * i + 5]));
+                v.w = pack_bf16(__uint_as_float(r[8 * i + 6]), __uint_as_float(r[8 * i + 7]));
+                dst[i] = v;
+              }
             }
           } else {
-            uint4* dst = reinterpret_cast<uint4*>(P.part_o + ((size_t)w.part * 128 + row) * D + c * 32);
+            // fp32 partial rows: element (lane, i) goes to word lane * 32 + (i ^ lane) (conflict free both ways), then
+            // every store instruction writes one full row segment of 128 bytes
 #pragma unroll
-            for (int i = 0; i < 8; ++i) dst[i] = make_uint4(r[4 * i], r[4 * i + 1], r[4 * i + 2], r[4 * i + 3]);
+            for (int i = 0; i < 32; ++i) stg[lane * 32 + (i ^ lane)] = __uint_as_float(r[i]);
+            __syncwarp();
+            float* dst = P.part_o + ((size_t)w.part * 128 + quad * 32) * D + c * 32 + lane;
+#pragma unroll 8
+            for (int rr = 0; rr < 32; ++rr)
+              if (rr < nrow) dst[(size_t)rr * D] = stg[rr * 32 + (lane ^ rr)];
+            __syncwarp();
           }
         }
-        if (rvalid && w.part >= 0) {
-          P.part_ml[((size_t)w.part * 128 + row) * 2 + 0] = m_ref;
-          P.part_ml[((size_t)w.part * 128 + row) * 2 + 1] = l_run;
+        if (g == 0 && rvalid && w.part >= 0) {
+          P.part_ml[((size_t)w.part * 128 + row) * 2 + 0] = m_all;
+          P.part_ml[((size_t)w.part * 128 + row) * 2 + 1] = l_all;
         }
       }
       tc_fence_before();
+      fence_proxy_async();    // the Q buffer goes back to the TMA unit
       __syncwarp();
-      if (lane == 0) mbar_arrive(o_empty);
+      if (lane == 0) {
+        mbar_arrive(o_empty);
+        mbar_arrive(&q_empty[buf]);
+      }
       ++item_cnt;
-      // all MMAs of this item have completed (the last o_full tracked them), so Q may be restaged
-      softmax_bar();
+      softmax_bar();          // the (max, sum) exchange area may be rewritten
     }
   }
 
@@ -553,6 +637,46 @@ __global__ void __launch_bounds__(kThreads, 1) attention_tc_kernel(TcAttnParams 
     tc_fence_after();
     tmem_dealloc(tmem_base, kTmemCols);
   }
+}
+
+// ---- host side: the tensor map over q -------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+struct QMapEntry {
+  const void* q;
+  int n_tok, n_q, group;
+  CUtensorMap map;
+};
+
+// q is bf16 [n_tok][n_q][128]; box = 64 dims x group heads x (128 / group) tokens, 128-byte swizzle, zero fill
+const CUtensorMap* q_tensor_map(const void* q, int n_tok, int n_q, int group) {
+  static EncodeTiledFn encode = nullptr;
+  static QMapEntry cache[16];
+  static int n_cached = 0, next_slot = 0;
+  for (int i = 0; i < n_cached; ++i)
+    if (cache[i].q == q && cache[i].n_tok == n_tok && cache[i].n_q == n_q && cache[i].group == group) return &cache[i].map;
+  if (!encode) {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess || !fn)
+      return nullptr;
+    encode = reinterpret_cast<EncodeTiledFn>(fn);
+  }
+  QMapEntry& e = cache[next_slot];
+  cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)n_q, (cuuint64_t)n_tok};
+  cuuint64_t strides[2] = {(cuuint64_t)D * 2, (cuuint64_t)n_q * D * 2};
+  cuuint32_t box[3] = {64, (cuuint32_t)group, (cuuint32_t)(128 / group)};
+  cuuint32_t estr[3] = {1, 1, 1};
+  if (encode(&e.map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(q), dims, strides, box, estr,
+             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+    return nullptr;
+  e.q = q; e.n_tok = n_tok; e.n_q = n_q; e.group = group;
+  next_slot = (next_slot + 1) % 16;
+  if (n_cached < 16) ++n_cached;
+  return &e.map;
 }
 
 }  // namespace
@@ -573,7 +697,6 @@ void launch_attention_tc_main(const BatchLayout& bl, const Dims& dm, int layer, 
   P.tok_climit = bl.tok_climit;
   P.tok_lo = bl.tok_lo;
   P.tok_hi = bl.tok_hi;
-  P.q = static_cast<const __nv_bfloat16*>(q);
   P.o = static_cast<__nv_bfloat16*>(o);
   P.pool = static_cast<const __nv_bfloat16*>(kv_pool);
   P.n_pages = n_pages;
@@ -585,7 +708,12 @@ void launch_attention_tc_main(const BatchLayout& bl, const Dims& dm, int layer, 
   P.part_o = part_o;
   P.part_ml = part_ml;
   P.status = status;
-  launch_pdl(attention_tc_kernel, dim3(n_sm), dim3(kThreads), kSmemBytes, st, P);
+  const CUtensorMap* qmap = q_tensor_map(q, bl.n_tok, dm.n_q, P.group);
+  if (!qmap) {
+    fprintf(stderr, "recg: cannot encode the tensor map over q\n");
+    return;
+  }
+  launch_pdl(attention_tc_kernel, dim3(n_sm), dim3(kThreads), kSmemBytes, st, *qmap, P);
 }
 
 }  // namespace recg
