@@ -157,7 +157,8 @@ struct SplitLoader {
   const float* ws;        // partial-tile workspace; slot s holds a [BM][bn] fp32 tile
   int bn, row;            // tile width, this thread's row in the tile
   int slot0;              // slot of part 0
-  int slot_next;          // slot of part 1; part p >= 1 is in slot_next + 2 (p - 1)
+  int slot_next;          // slot of part 1; part p >= 1 is in slot_next + slot_stride (p - 1)
+  int slot_stride;
   int n_parts;
   bool valid;             // rows beyond M were never parked
   __device__ __forceinline__ void operator()(int col, float (&v)[32]) const {
@@ -169,9 +170,9 @@ struct SplitLoader {
     // parts are issued together so that their latencies overlap.
     const float4* base = reinterpret_cast<const float4*>(ws) + (size_t)(col / 4) * BM + row;
     for (int p = 0; p < n_parts; p += 2) {
-      const int sa = p == 0 ? slot0 : slot_next + 2 * (p - 1);
+      const int sa = p == 0 ? slot0 : slot_next + slot_stride * (p - 1);
       const bool two = p + 1 < n_parts;
-      const int sb = slot_next + 2 * p;             // slot of part p + 1 (>= 1)
+      const int sb = slot_next + slot_stride * p;   // slot of part p + 1 (>= 1)
       float4 a[8], b[8];
 #pragma unroll
       for (int i = 0; i < 8; ++i) {
@@ -187,23 +188,29 @@ struct SplitLoader {
   }
 };
 
-// Work decomposition ("stream-K"): the k-blocks of all output tiles form one line of n_tiles * KB units, tile
-// after tile; CTA c owns the contiguous range [c * per, (c + 1) * per).  With per a multiple of KB every CTA owns
-// whole tiles; otherwise a tile may be cut by CTA boundaries, and each owner computes its K range of it ("part").
-// Part p >= 1 of a tile is always the FIRST piece of its CTA, part 0 the last piece of its CTA (or the first, when
-// the CTA's range starts exactly at the tile): that decides the workspace slot, 2 * cta + (first piece ? 0 : 1).
+// Work decomposition ("stream-K"), done per COLUMN of output tiles (the mt row tiles that share one weight tile):
+// the k-blocks of the columns form one line of n_cols * KB units, column after column; a TEAM of mt CTAs (CTA
+// team * mt + i works on row tile i) owns the contiguous range [team * per, (team + 1) * per) and walks it in
+// step, so that the members read the same weight k-blocks at the same time and share them through L2, exactly
+// like the CTAs of a wave of whole tiles.  A column may be cut by team boundaries; each owner computes its K range
+// of its row tile ("part").  Part p >= 1 of a tile is always the FIRST piece of its CTA, part 0 the last piece (or
+// the first, when the range starts exactly at the column): that decides the workspace slot,
+// 2 * cta + (first piece ? 0 : 1).
 struct Piece {
   int tile, kb0, kb1;     // k-block range [kb0, kb1) of the tile
   int part, n_parts;      // which part of the tile this is
   int slot;               // workspace slot if n_parts > 1
   int slot0, slot_next;   // slots of part 0 and part 1 (for the reducing CTA)
 };
-// j-th piece of this CTA: first its whole tiles, then its range of the stream-K line (pos advances by reference)
-__device__ __forceinline__ Piece make_piece(int j, int dp_count, int dp_tiles, long long& pos, long long hi, int KB,
-                                            long long per, int cta, int grid) {
+// Next piece of this CTA: first its range of the stream-K line (pos advances by reference), then its whole tiles
+// (jd counts them).  The cut tiles come first so that parking and reducing their partials overlaps the main loop
+// of the whole tiles that follow, instead of happening in every CTA at once at the end of the kernel.
+__device__ __forceinline__ Piece make_piece(int& jd, int dp_tiles, long long& pos, long long hi, int KB,
+                                            long long per, int cta, int grid, int mt) {
   Piece p;
-  if (j < dp_count) {
-    p.tile = cta + j * grid;
+  if (pos >= hi) {
+    p.tile = cta + jd * grid;
+    ++jd;
     p.kb0 = 0;
     p.kb1 = KB;
     p.part = 0;
@@ -211,19 +218,20 @@ __device__ __forceinline__ Piece make_piece(int j, int dp_count, int dp_tiles, l
     p.slot = p.slot0 = p.slot_next = 0;
     return p;
   }
-  p.tile = (int)(pos / KB);
-  p.kb0 = (int)(pos - (long long)p.tile * KB);
+  const int team = cta / mt, member = cta % mt;
+  const int col = (int)(pos / KB);
+  p.kb0 = (int)(pos - (long long)col * KB);
   const long long room = hi - pos;
   p.kb1 = (int)(room < KB - p.kb0 ? p.kb0 + room : KB);
-  const long long t0 = (long long)p.tile * KB, t1 = t0 + KB;
-  const int c_first = (int)(t0 / per), c_last = (int)((t1 - 1) / per);
+  const long long t0 = (long long)col * KB, t1 = t0 + KB;
+  const int c_first = (int)(t0 / per), c_last = (int)((t1 - 1) / per);    // first and last team on this column
   p.n_parts = c_last - c_first + 1;
-  p.part = cta - c_first;
-  const bool first_piece = pos == (long long)cta * per;
+  p.part = team - c_first;
+  const bool first_piece = pos == (long long)team * per;
   p.slot = 2 * cta + (first_piece ? 0 : 1);
-  p.slot0 = 2 * c_first + (((long long)c_first * per >= t0) ? 0 : 1);
-  p.slot_next = 2 * (c_first + 1);
-  p.tile += dp_tiles;
+  p.slot0 = 2 * (c_first * mt + member) + (((long long)c_first * per >= t0) ? 0 : 1);
+  p.slot_next = 2 * ((c_first + 1) * mt + member);
+  p.tile = dp_tiles + col * mt + member;
   pos += p.kb1 - p.kb0;
   return p;
 }
@@ -345,10 +353,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
   const int n_tiles = n_tiles_m * n_tiles_n;
   const int KB = K / BK;
   const bool swiglu = ep.epi == EPI_SWIGLU;
-  // schedule: tiles [0, dp_tiles) whole, strided over the grid (CTAs that run together share a weight tile
-  // through L2); then the k-blocks of tiles [dp_tiles, n_tiles) as one line cut into equal ranges per CTA
-  const long long range_lo = (long long)blockIdx.x * per;
-  const long long total = (long long)(n_tiles - dp_tiles) * KB;
+  // schedule: the k-blocks of tiles [dp_tiles, n_tiles) as one line cut into equal ranges per CTA; then tiles
+  // [0, dp_tiles) whole, strided over the grid (CTAs that run together share a weight tile through L2)
+  const long long total = (long long)((n_tiles - dp_tiles) / n_tiles_m) * KB;
+  const long long lo_raw = (long long)(blockIdx.x / n_tiles_m) * per;
+  const long long range_lo = lo_raw < total ? lo_raw : total;
   const long long range_hi = range_lo + per < total ? range_lo + per : total;
   const int dp_count = blockIdx.x < dp_tiles ? (dp_tiles - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
 
@@ -382,8 +391,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
       uint32_t st_phase = 0;
       bool ok = true;
       long long pos = range_lo;
-      for (int j = 0; (j < dp_count || pos < range_hi) && ok; ++j) {
-        const Piece pc = make_piece(j, dp_count, dp_tiles, pos, range_hi, KB, per, blockIdx.x, gridDim.x);
+      for (int jd = 0; (jd < dp_count || pos < range_hi) && ok;) {
+        const Piece pc = make_piece(jd, dp_tiles, pos, range_hi, KB, per, blockIdx.x, gridDim.x, n_tiles_m);
         const int tm = pc.tile % n_tiles_m, tn = pc.tile / n_tiles_m;
         const int kb0 = pc.kb0, kb1 = pc.kb1;
         for (int kb = kb0; kb < kb1; ++kb) {
@@ -423,8 +432,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
       uint32_t st_phase = 0, tcount = 0;
       bool ok = true;
       long long pos = range_lo;
-      for (int j = 0; (j < dp_count || pos < range_hi) && ok; ++j, ++tcount) {
-        const Piece pc = make_piece(j, dp_count, dp_tiles, pos, range_hi, KB, per, blockIdx.x, gridDim.x);
+      for (int jd = 0; (jd < dp_count || pos < range_hi) && ok; ++tcount) {
+        const Piece pc = make_piece(jd, dp_tiles, pos, range_hi, KB, per, blockIdx.x, gridDim.x, n_tiles_m);
         const int kb0 = pc.kb0, kb1 = pc.kb1;
         const int acc = tcount & 1;
         if (!mbar_wait(&tempty_bar[acc], ((tcount >> 1) & 1) ^ 1, kSpin)) {
@@ -462,8 +471,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     uint32_t tcount = 0;
     __shared__ int s_last;
     long long pos = range_lo;
-    for (int j = 0; j < dp_count || pos < range_hi; ++j, ++tcount) {
-      const Piece pc = make_piece(j, dp_count, dp_tiles, pos, range_hi, KB, per, blockIdx.x, gridDim.x);
+    for (int jd = 0; jd < dp_count || pos < range_hi; ++tcount) {
+      const Piece pc = make_piece(jd, dp_tiles, pos, range_hi, KB, per, blockIdx.x, gridDim.x, n_tiles_m);
       const int tile = pc.tile, n_splits = pc.n_parts;
       const int tm = tile % n_tiles_m, tn = tile / n_tiles_m;
       const int acc = tcount & 1;
@@ -508,7 +517,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
         }
         asm volatile("bar.sync 1, 128;" ::: "memory");
         if (s_last) {
-          SplitLoader ld{split_ws, BN, row_in_tile, pc.slot0, pc.slot_next, n_splits, m < ep.M};
+          SplitLoader ld{split_ws, BN, row_in_tile, pc.slot0, pc.slot_next, 2 * n_tiles_m, n_splits, m < ep.M};
           row_epilogue<BN>(ep, ld, m, n0);
         }
         asm volatile("bar.sync 1, 128;" ::: "memory");       // s_last is reused by the next unit
@@ -595,15 +604,18 @@ bool launch_bn(TcState* st, int idx, const GemmArgs& a, const EpiParams& ep, boo
   int dp_tiles = n_tiles;       // whole tiles, strided
   long long per = 1;
   if (stream_k) {
-    // all but the last one-to-two waves as whole tiles; the k-blocks of the remaining tiles evenly over all SMs
+    // all but the last one-to-two waves as whole tiles; the k-blocks of the remaining tile columns evenly over
+    // teams of mt CTAs (one per row tile)
+    const int mt = (a.M + BM - 1) / BM;
+    const int n_teams = st->n_sm / mt;                  // the caller made sure that mt <= n_sm
     const int full = n_tiles / st->n_sm;
-    dp_tiles = full >= 2 ? (full - 1) * st->n_sm : 0;
-    const long long total = (long long)(n_tiles - dp_tiles) * KB;
-    grid = total < st->n_sm ? (int)total : st->n_sm;
-    per = (total + grid - 1) / grid;
+    dp_tiles = full >= 2 ? ((full - 1) * st->n_sm / mt) * mt : 0;
+    const long long total = (long long)((n_tiles - dp_tiles) / mt) * KB;
+    const long long teams = total < n_teams ? total : n_teams;
+    per = (total + teams - 1) / teams;
     if (per < 4 && total >= 4) per = 4;                 // keep pieces long enough to amortise their hand-over
-    const int g2 = (int)((total + per - 1) / per);
-    if (dp_tiles == 0) grid = g2;                       // (with whole tiles in front the grid stays at the SM count)
+    const int used = (int)((total + per - 1) / per);    // teams that get a range
+    grid = dp_tiles ? st->n_sm : used * mt;             // (with whole tiles behind, the grid stays at the SM count)
   }
   launch_pdl(gemm_tc_kernel<BN>, dim3(grid), dim3(kTcThreads), Cfg::kSmemBytes, stream, *mx, *mw, a.M, n_tiles_n, a.K, a.N,
              dp_tiles, per, thin, st->split_ws, st->split_counters, ep);
@@ -687,11 +699,24 @@ bool launch_gemm_tc(const GemmArgs& a, void* tc_state, int* status, cudaStream_t
     const double kbt = fmax(kb_tensor[bi], (bn * 128.0 / mt) / 35e3);
     const double rows = a.M < BM ? a.M : BM;
     const double t_plain = (double)waves * KB * kbt;
-    const double t_sk = ((double)tiles * KB / st->n_sm + 1.0) * kbt + 3.0 + rows * bn * 4.0 * 2.5 / 16e3;
+    const int sk_ctas = mt <= st->n_sm ? (st->n_sm / mt) * mt : 1;     // teams of mt CTAs
+    const double t_sk = ((double)tiles * KB / sk_ctas + 1.0) * kbt + 3.0 + rows * bn * 4.0 * 2.5 / 16e3;
     if (t_plain < best_t) { best_t = t_plain; best_bn = bn; best_sk = false; }
-    // measured: with full 128-row tiles the hand-over of the cut tiles (15-27 us at the end of the kernel, when
-    // every reduction happens at once) eats the gain, so K ranges are only cut for thin problems
-    if (a.M <= 64 && (size_t)2 * st->n_sm * BM * bn * 4 <= kSplitWsBytes && t_sk < best_t) { best_t = t_sk; best_bn = bn; best_sk = true; }
+    const bool ws_fits = (size_t)2 * st->n_sm * BM * bn * 4 <= kSplitWsBytes && mt <= st->n_sm;
+    const long long full = tiles / st->n_sm, rem = tiles % st->n_sm;
+    if (ws_fits && full >= 2) {
+      // a ragged last wave: the last (n_sm + rem) tiles are cut evenly over the SMs and done FIRST, so that their
+      // hand-over (park the partial, counter, reduction by the last arriver) hides under the whole tiles after it.
+      // Measured: the cut tiles run a little slower than whole ones, so this only pays when the last wave would
+      // leave a good part of the machine idle (a nearly empty wave of whole tiles is cheap: its few CTAs run fast).
+      const double idle = rem ? (double)(st->n_sm - rem) / st->n_sm / (double)(full + 1) : 0.0;
+      const double t_h = (double)tiles * KB / st->n_sm * kbt + 2.0;
+      if (idle > 0.12 && t_h < best_t) { best_t = t_h; best_bn = bn; best_sk = true; }
+    } else if (ws_fits && t_sk < best_t) {
+      // no whole tiles to hide the hand-over under: it happens in every CTA at once at the end of the kernel and
+      // costs about 3 us + 0.6 us per KB of partial tile, which t_sk charges
+      best_t = t_sk; best_bn = bn; best_sk = true;
+    }
   }
   if (st->force_bn) {   // tuning aid: RECG_GEMM_FORCE="<bn>,<0 whole tiles | 1 stream-K>"; ignored where it does not fit
     const int bn = st->force_bn;
@@ -701,7 +726,7 @@ bool launch_gemm_tc(const GemmArgs& a, void* tc_state, int* status, cudaStream_t
                           mt * ((a.N + per - 1) / per) <= kSplitCounters;
     if (shape_ok) {
       best_bn = bn;
-      best_sk = st->force_s != 0;
+      best_sk = st->force_s != 0 && mt <= st->n_sm && (size_t)2 * st->n_sm * BM * bn * 4 <= kSplitWsBytes;
     }
   }
   if (!best_bn) return false;
