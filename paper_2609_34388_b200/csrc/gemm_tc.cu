@@ -45,7 +45,7 @@ template <int BN> struct TcCfg {
   static constexpr int kThinStages =
       (kSmemBudget / kThinStageBytes) > kMaxStages ? kMaxStages : (kSmemBudget / kThinStageBytes);
   static constexpr int kRingBytes = kSmemBudget + kABytes;     // either ring plus the pad
-  static constexpr int kBarBytes = (2 * kMaxStages + 4) * 8 + 16;
+  static constexpr int kBarBytes = (2 * kMaxStages + 5) * 8 + 16;
   static constexpr int kSmemBytes = kRingBytes + kBarBytes + 1024;  // + slack for 1024-byte alignment
   static constexpr int kTmemCols = 2 * BN < 32 ? 32 : 2 * BN;                  // power of two: 128, 256, 512
 };
@@ -183,6 +183,38 @@ struct SplitLoader {
       for (int i = 0; i < 8; ++i) {
         v[4 * i] += a[i].x; v[4 * i + 1] += a[i].y; v[4 * i + 2] += a[i].z; v[4 * i + 3] += a[i].w;
         v[4 * i] += b[i].x; v[4 * i + 1] += b[i].y; v[4 * i + 2] += b[i].z; v[4 * i + 3] += b[i].w;
+      }
+    }
+  }
+};
+
+// The reducing CTA's own part comes from its TMEM accumulator, the other parts from copies in shared memory (the
+// idle operand ring, one [BN/4][BM] float4 tile after the other in part order without the own part).  Parts are
+// added in part order starting from zero, exactly like SplitLoader, so both give the same bits.
+struct RingLoader {
+  uint32_t tacc;
+  const float4* ring;     // + row
+  int bn, own, n_parts;
+  // Every lane takes part, also those whose row lies beyond M (the TMEM load is a warp-wide instruction; their
+  // sums are never stored).
+  __device__ __forceinline__ void operator()(int col, float (&v)[32]) const {
+#pragma unroll
+    for (int i = 0; i < 32; ++i) v[i] = 0.f;
+    int k = 0;
+    for (int p = 0; p < n_parts; ++p) {
+      if (p == own) {
+        float t[32];
+        tmem_ld32(tacc + col, t);
+#pragma unroll
+        for (int i = 0; i < 32; ++i) v[i] += t[i];
+      } else {
+        const float4* src = ring + ((size_t)k * (bn / 4) + col / 4) * BM;
+        ++k;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const float4 a = src[(size_t)i * BM];
+          v[4 * i] += a.x; v[4 * i + 1] += a.y; v[4 * i + 2] += a.z; v[4 * i + 3] += a.w;
+        }
       }
     }
   }
@@ -346,7 +378,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
   uint64_t* empty_bar = full_bar + Cfg::kMaxStages;
   uint64_t* tfull_bar = empty_bar + Cfg::kMaxStages;
   uint64_t* tempty_bar = tfull_bar + 2;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tempty_bar + 2);
+  uint64_t* red_bar = tempty_bar + 2;      // completion of the partial tiles fetched into the idle ring (used once)
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(red_bar + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n_tiles_m = (M + BM - 1) / BM;
@@ -370,6 +403,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
       mbar_init(&tfull_bar[a], 1);
       mbar_init(&tempty_bar[a], 4);
     }
+    mbar_init(red_bar, 1);
     fence_barrier_init();
     prefetch_tmap(&map_x);
     prefetch_tmap(&map_w);
@@ -491,8 +525,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
         __syncwarp();
         if (lane == 0) mbar_arrive(&tempty_bar[acc]);
       } else {
-        // park this split's partial tile, release the accumulator, and let the LAST split to arrive reduce all
-        // partials in split order (deterministic) and run the fused epilogue
+        // park this split's partial tile and let the LAST split to arrive reduce all partials in split order
+        // (deterministic) and run the fused epilogue
         float4* mine = reinterpret_cast<float4*>(split_ws) + (size_t)pc.slot * (BN / 4) * BM + row_in_tile;
 #pragma unroll 1
         for (int c = 0; c < BN / 32; ++c) {
@@ -504,6 +538,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
               __stcg(mine + (size_t)(c * 8 + i) * BM, make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]));
           }
         }
+        // the accumulator may be handed back at once: the own part is read from TMEM again only when nothing follows
+        // in this CTA, and then nobody overwrites it
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(&tempty_bar[acc]);
@@ -517,8 +553,32 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
         }
         asm volatile("bar.sync 1, 128;" ::: "memory");
         if (s_last) {
-          SplitLoader ld{split_ws, BN, row_in_tile, pc.slot0, pc.slot_next, 2 * n_tiles_m, n_splits, m < ep.M};
-          row_epilogue<BN>(ep, ld, m, n0);
+          // When nothing follows in this CTA the operand ring is idle (every load was consumed before the accumulator
+          // completed): the other parts are fetched into it with bulk copies at full bandwidth and the own part is
+          // taken from TMEM.  Otherwise the parts are read from global memory while the next piece's main loop runs.
+          constexpr int kPartBytes = BM * BN * 4;
+          const bool final_piece = !(jd < dp_count || pos < range_hi);
+          if (final_piece && (n_splits - 1) * kPartBytes <= kSmemBudget) {
+            if (warp == 2 && lane == 0) {
+              asm volatile("fence.proxy.async;" ::: "memory");   // the parts were written with ordinary stores
+              mbar_arrive_expect_tx(red_bar, (uint32_t)((n_splits - 1) * kPartBytes));
+              int k = 0;
+              for (int p = 0; p < n_splits; ++p) {
+                if (p == pc.part) continue;
+                const int slot = p == 0 ? pc.slot0 : pc.slot_next + 2 * n_tiles_m * (p - 1);
+                const uint8_t* src = reinterpret_cast<const uint8_t*>(split_ws) + (size_t)slot * kPartBytes;
+                for (int off = 0; off < kPartBytes; off += 32768)
+                  bulk_g2s(smem + (size_t)k * kPartBytes + off, src + off, 32768, red_bar);
+                ++k;
+              }
+            }
+            if (!mbar_wait(red_bar, 0, kSpin)) set_status(ep.status, DEV_TIMEOUT_FULL);
+            RingLoader ld{tacc, reinterpret_cast<const float4*>(smem) + row_in_tile, BN, pc.part, n_splits};
+            row_epilogue<BN>(ep, ld, m, n0);
+          } else {
+            SplitLoader ld{split_ws, BN, row_in_tile, pc.slot0, pc.slot_next, 2 * n_tiles_m, n_splits, m < ep.M};
+            row_epilogue<BN>(ep, ld, m, n0);
+          }
         }
         asm volatile("bar.sync 1, 128;" ::: "memory");       // s_last is reused by the next unit
       }
