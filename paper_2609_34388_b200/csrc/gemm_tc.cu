@@ -31,9 +31,9 @@ constexpr int kTcThreads = 192;
 constexpr int kSmemBudget = 200 * 1024;
 constexpr uint32_t kSpin = 1u << 22;
 
-template <int BN> struct TcCfg {
+template <int BN, bool PAIR = false> struct TcCfg {
   static constexpr int kABytes = BM * BK * 2;
-  static constexpr int kBBytes = BN * BK * 2;
+  static constexpr int kBBytes = (PAIR ? BN / 2 : BN) * BK * 2;     // per CTA: a pair splits the weight tile
   static constexpr int kStageBytes = kABytes + kBBytes;
   static constexpr int kStages = (kSmemBudget / kStageBytes) > 8 ? 8 : (kSmemBudget / kStageBytes);
   static constexpr int kMaxStages = 16;
@@ -118,10 +118,89 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t smem_addr) {
   d |= (uint64_t)2 << 61;                       // SWIZZLE_128B
   return d;
 }
-// kind::f16 instruction descriptor: fp32 accumulate, bf16 A and B, both K-major, M = 128, N = BN
-__host__ __device__ constexpr uint32_t make_idesc(int n) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+// kind::f16 instruction descriptor: fp32 accumulate, bf16 A and B, both K-major, M = 128 (256 for a CTA pair), N = BN
+__host__ __device__ constexpr uint32_t make_idesc(int n, int m = BM) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
+
+// ---- CTA pairs (tcgen05 cta_group::2) ----------------------------------------------------------------
+// With PAIR a cluster of two CTAs computes tiles of 256 rows: each CTA loads its own 128 rows of x and its own
+// half of the weight tile per k-block (32 KB per stage instead of the 48 KB a single CTA needs for 128 x 256, so
+// six stages fit and a third fewer operand bytes cross L2 -> shared memory per flop); the tensor cores of the
+// pair read both halves of the weight tile, each CTA accumulates its 128 rows in its own TMEM.  Only the leader
+// CTA (cluster rank 0) issues MMAs.
+//   full barrier  (leader's):   the leader's producer arrives with the byte count of BOTH CTAs' loads; both CTAs'
+//                               TMA loads (cta_group::2 form, no multicast) complete on it
+//   empty barrier (per CTA):    tcgen05.commit multicast to both CTAs frees the stage in each
+//   accumulator full (per CTA): commit multicast; accumulator empty (leader's): all eight epilogue warps of the
+//                               pair arrive (the peer's remotely)
+// The scheduling unit is the cluster; the two CTAs of a cluster park and reduce their halves of a cut tile
+// independently (own slots, own counters).
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// the shared::cluster address of the same location in the CTA of rank `rank`
+__device__ __forceinline__ uint32_t mapa_rank(uint32_t addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t smem_dst, const CUtensorMap* map, int x, int y, uint32_t bar_cluster) {
+  asm volatile("cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+               :
+               : "r"(smem_dst), "l"(map), "r"(bar_cluster), "r"(x), "r"(y)
+               : "memory");
+}
+__device__ __forceinline__ void umma_bf16_pair(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc,
+                                               uint32_t accumulate) {
+  const uint32_t z = 0;
+  asm volatile(
+      "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
+      " tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5, %5, %5, %5, %5}, p;\n}"
+      :
+      : "r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate), "r"(z)
+      : "memory");
+}
+__device__ __forceinline__ void umma_commit_pair(uint64_t* bar) {   // arrives on this barrier in both CTAs
+  const uint16_t mask = 3;
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(
+                   smem_u32(bar)),
+               "h"(mask)
+               : "memory");
+}
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t* smem_slot, uint32_t cols) {
+  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(smem_slot)), "r"(cols)
+               : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish_pair() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t addr, uint32_t cols) {
+  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(addr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar_cluster) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar_cluster) : "memory");
+}
+// bounded wait that also orders against arrivals from the other CTA of the cluster
+__device__ __forceinline__ bool mbar_wait_cluster(uint64_t* bar, uint32_t parity, uint32_t max_iter) {
+  for (uint32_t i = 0; i < max_iter; ++i) {
+    uint32_t ok;
+    asm volatile(
+        "{\n .reg .pred p;\n mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    if (ok) return true;
+    if (i > 64) __nanosleep(32);
+  }
+  return false;
+}
+
 
 // ---- register epilogue: one thread owns one output row -------------------------------------------
 __device__ __forceinline__ void store_chunk_f32(float* dst, const float (&v)[32], bool add) {
@@ -363,12 +442,17 @@ __device__ __forceinline__ void row_epilogue(const EpiParams& ep, const Loader& 
   }
 }
 
-template <int BN>
+template <int BN, bool PAIR>
 __global__ void __launch_bounds__(kTcThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w, int M, int n_tiles_n,
                int K, int up_row_offset, int dp_tiles, long long per, int thin, float* split_ws, int* split_counters,
                EpiParams ep) {
-  using Cfg = TcCfg<BN>;
+  using Cfg = TcCfg<BN, PAIR>;
+  constexpr int kRows = PAIR ? 2 * BM : BM;              // rows of a scheduling unit's tile
+  constexpr int kSlotMul = PAIR ? 2 : 1;                 // the CTAs of a pair use separate slots and counters
+  const uint32_t rank = PAIR ? cluster_ctarank() : 0u;
+  const int unit = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;      // scheduling unit: CTA or cluster
+  const int n_units = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int n_stages = thin ? Cfg::kThinStages : Cfg::kStages;
@@ -382,17 +466,17 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(red_bar + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int n_tiles_m = (M + BM - 1) / BM;
+  const int n_tiles_m = (M + kRows - 1) / kRows;
   const int n_tiles = n_tiles_m * n_tiles_n;
   const int KB = K / BK;
   const bool swiglu = ep.epi == EPI_SWIGLU;
   // schedule: the k-blocks of tiles [dp_tiles, n_tiles) as one line cut into equal ranges per CTA; then tiles
   // [0, dp_tiles) whole, strided over the grid (CTAs that run together share a weight tile through L2)
   const long long total = (long long)((n_tiles - dp_tiles) / n_tiles_m) * KB;
-  const long long lo_raw = (long long)(blockIdx.x / n_tiles_m) * per;
+  const long long lo_raw = (long long)(unit / n_tiles_m) * per;
   const long long range_lo = lo_raw < total ? lo_raw : total;
   const long long range_hi = range_lo + per < total ? range_lo + per : total;
-  const int dp_count = blockIdx.x < dp_tiles ? (dp_tiles - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
+  const int dp_count = unit < dp_tiles ? (dp_tiles - 1 - unit) / n_units + 1 : 0;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < n_stages; ++s) {
@@ -401,7 +485,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(&tfull_bar[a], 1);
-      mbar_init(&tempty_bar[a], 4);
+      mbar_init(&tempty_bar[a], PAIR ? 8 : 4);
     }
     mbar_init(red_bar, 1);
     fence_barrier_init();
@@ -409,11 +493,17 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     prefetch_tmap(&map_w);
   }
   if (warp == 1) {
-    tmem_alloc(tmem_slot, Cfg::kTmemCols);
-    tmem_relinquish();
+    if constexpr (PAIR) {
+      tmem_alloc_pair(tmem_slot, Cfg::kTmemCols);
+      tmem_relinquish_pair();
+    } else {
+      tmem_alloc(tmem_slot, Cfg::kTmemCols);
+      tmem_relinquish();
+    }
   }
   tc_fence_before();
   __syncthreads();
+  if constexpr (PAIR) cluster_sync_all();   // both CTAs' barriers are initialised before anyone signals across
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
   griddep_wait();   // everything above touched only shared memory and TMEM
@@ -426,27 +516,37 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
       bool ok = true;
       long long pos = range_lo;
       for (int jd = 0; (jd < dp_count || pos < range_hi) && ok;) {
-        const Piece pc = make_piece(jd, dp_tiles, pos, range_hi, KB, per, blockIdx.x, gridDim.x, n_tiles_m);
+        const Piece pc = make_piece(jd, dp_tiles, pos, range_hi, KB, per, unit, n_units, n_tiles_m);
         const int tm = pc.tile % n_tiles_m, tn = pc.tile / n_tiles_m;
         const int kb0 = pc.kb0, kb1 = pc.kb1;
         for (int kb = kb0; kb < kb1; ++kb) {
           const int s = st_idx;
           const uint32_t ph = st_phase;
           if (++st_idx == n_stages) { st_idx = 0; st_phase ^= 1; }
-          if (!mbar_wait(&empty_bar[s], ph ^ 1, kSpin)) {
+          if (!(PAIR ? mbar_wait_cluster(&empty_bar[s], ph ^ 1, kSpin) : mbar_wait(&empty_bar[s], ph ^ 1, kSpin))) {
             set_status(ep.status, DEV_TIMEOUT_EMPTY);
             ok = false;
             break;
           }
           uint8_t* a_dst = smem + s * stage_bytes;
           uint8_t* b_dst = a_dst + a_bytes;
-          mbar_arrive_expect_tx(&full_bar[s], stage_bytes);
-          tma_load_2d(a_dst, &map_x, kb * BK, tm * BM, &full_bar[s]);
-          if (swiglu) {
-            tma_load_2d(b_dst, &map_w, kb * BK, tn * (BN / 2), &full_bar[s]);
-            tma_load_2d(b_dst + Cfg::kBBytes / 2, &map_w, kb * BK, up_row_offset + tn * (BN / 2), &full_bar[s]);
+          if constexpr (PAIR) {
+            // rank r loads rows [128 r, 128 r + 128) of the x tile and half r of the weight tile (SwiGLU: rank 0 the
+            // gate rows, rank 1 the up rows); all four loads of the pair complete on the leader's barrier
+            const uint32_t full0 = mapa_rank(smem_u32(&full_bar[s]), 0);
+            if (rank == 0) mbar_arrive_expect_tx(&full_bar[s], 2 * stage_bytes);
+            const int w_row = swiglu ? (rank == 0 ? tn * (BN / 2) : up_row_offset + tn * (BN / 2)) : tn * BN + (int)rank * (BN / 2);
+            tma_load_2d_pair(smem_u32(a_dst), &map_x, kb * BK, tm * kRows + (int)rank * BM, full0);
+            tma_load_2d_pair(smem_u32(b_dst), &map_w, kb * BK, w_row, full0);
           } else {
-            tma_load_2d(b_dst, &map_w, kb * BK, tn * BN, &full_bar[s]);
+            mbar_arrive_expect_tx(&full_bar[s], stage_bytes);
+            tma_load_2d(a_dst, &map_x, kb * BK, tm * BM, &full_bar[s]);
+            if (swiglu) {
+              tma_load_2d(b_dst, &map_w, kb * BK, tn * (BN / 2), &full_bar[s]);
+              tma_load_2d(b_dst + Cfg::kBBytes / 2, &map_w, kb * BK, up_row_offset + tn * (BN / 2), &full_bar[s]);
+            } else {
+              tma_load_2d(b_dst, &map_w, kb * BK, tn * BN, &full_bar[s]);
+            }
           }
         }
       }
@@ -460,17 +560,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     }
   } else if (warp == 1) {
     // ------------------------------ MMA issuer ------------------------------
-    if (elect_one()) {
-      constexpr uint32_t idesc = make_idesc(BN);
+    if (rank == 0 && elect_one()) {         // of a pair only the leader issues
+      constexpr uint32_t idesc = make_idesc(BN, kRows);
       int st_idx = 0;
       uint32_t st_phase = 0, tcount = 0;
       bool ok = true;
       long long pos = range_lo;
       for (int jd = 0; (jd < dp_count || pos < range_hi) && ok; ++tcount) {
-        const Piece pc = make_piece(jd, dp_tiles, pos, range_hi, KB, per, blockIdx.x, gridDim.x, n_tiles_m);
+        const Piece pc = make_piece(jd, dp_tiles, pos, range_hi, KB, per, unit, n_units, n_tiles_m);
         const int kb0 = pc.kb0, kb1 = pc.kb1;
         const int acc = tcount & 1;
-        if (!mbar_wait(&tempty_bar[acc], ((tcount >> 1) & 1) ^ 1, kSpin)) {
+        if (!(PAIR ? mbar_wait_cluster(&tempty_bar[acc], ((tcount >> 1) & 1) ^ 1, kSpin)
+                   : mbar_wait(&tempty_bar[acc], ((tcount >> 1) & 1) ^ 1, kSpin))) {
           set_status(ep.status, DEV_TIMEOUT_MMA);
           break;
         }
@@ -480,7 +581,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
           const int s = st_idx;
           const uint32_t ph = st_phase;
           if (++st_idx == n_stages) { st_idx = 0; st_phase ^= 1; }
-          if (!mbar_wait(&full_bar[s], ph, kSpin)) {
+          if (!(PAIR ? mbar_wait_cluster(&full_bar[s], ph, kSpin) : mbar_wait(&full_bar[s], ph, kSpin))) {
             set_status(ep.status, DEV_TIMEOUT_FULL);
             ok = false;
             break;
@@ -492,11 +593,17 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
           for (int k = 0; k < BK / 16; ++k) {
             const uint64_t da = make_smem_desc(a_addr + k * 32);
             const uint64_t db = make_smem_desc(b_addr + k * 32);
-            umma_bf16(d_tmem, da, db, idesc, ((kb - kb0) | k) ? 1u : 0u);
+            if constexpr (PAIR) umma_bf16_pair(d_tmem, da, db, idesc, ((kb - kb0) | k) ? 1u : 0u);
+            else umma_bf16(d_tmem, da, db, idesc, ((kb - kb0) | k) ? 1u : 0u);
           }
-          umma_commit(&empty_bar[s]);      // frees the stage when these MMAs have read it
+          // frees the stage (in both CTAs of a pair) when these MMAs have read it
+          if constexpr (PAIR) umma_commit_pair(&empty_bar[s]);
+          else umma_commit(&empty_bar[s]);
         }
-        if (ok) umma_commit(&tfull_bar[acc]);  // accumulator complete
+        if (ok) {                            // accumulator complete
+          if constexpr (PAIR) umma_commit_pair(&tfull_bar[acc]);
+          else umma_commit(&tfull_bar[acc]);
+        }
       }
     }
   } else {
@@ -506,28 +613,40 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     __shared__ int s_last;
     long long pos = range_lo;
     for (int jd = 0; jd < dp_count || pos < range_hi; ++tcount) {
-      const Piece pc = make_piece(jd, dp_tiles, pos, range_hi, KB, per, blockIdx.x, gridDim.x, n_tiles_m);
+      const Piece pc = make_piece(jd, dp_tiles, pos, range_hi, KB, per, unit, n_units, n_tiles_m);
       const int tile = pc.tile, n_splits = pc.n_parts;
       const int tm = tile % n_tiles_m, tn = tile / n_tiles_m;
       const int acc = tcount & 1;
-      if (!mbar_wait(&tfull_bar[acc], (tcount >> 1) & 1, kSpin)) {
+      if (!(PAIR ? mbar_wait_cluster(&tfull_bar[acc], (tcount >> 1) & 1, kSpin) : mbar_wait(&tfull_bar[acc], (tcount >> 1) & 1, kSpin))) {
         set_status(ep.status, DEV_TIMEOUT_MMA);
         break;
       }
       tc_fence_after();
       const uint32_t tacc = tmem_base + ((uint32_t)(quad * 32) << 16) + acc * BN;
       const int row_in_tile = quad * 32 + lane;
-      const int m = tm * BM + row_in_tile;
+      const int m = tm * kRows + (int)rank * BM + row_in_tile;
+      // hands the accumulator back to the MMA issuer (of a pair: the leader's barrier collects both CTAs' warps)
+      auto release_acc = [&]() {
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) {
+          if constexpr (PAIR) mbar_arrive_cluster(mapa_rank(smem_u32(&tempty_bar[acc]), 0));
+          else mbar_arrive(&tempty_bar[acc]);
+        }
+      };
       const int n0 = swiglu ? tn * (BN / 2) : tn * BN;
       if (n_splits == 1) {
         row_epilogue<BN>(ep, TmemLoader{tacc}, m, n0);
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&tempty_bar[acc]);
+        release_acc();
       } else {
         // park this split's partial tile and let the LAST split to arrive reduce all partials in split order
         // (deterministic) and run the fused epilogue
-        float4* mine = reinterpret_cast<float4*>(split_ws) + (size_t)pc.slot * (BN / 4) * BM + row_in_tile;
+        // (the two CTAs of a pair park and reduce their 128-row halves independently: slot and counter index are
+        // doubled and offset by the rank)
+        const int slot_mine = pc.slot * kSlotMul + (int)rank, slot0 = pc.slot0 * kSlotMul + (int)rank;
+        const int slot_next = pc.slot_next * kSlotMul + (int)rank, slot_stride = 2 * n_tiles_m * kSlotMul;
+        const int counter = tile * kSlotMul + (int)rank;
+        float4* mine = reinterpret_cast<float4*>(split_ws) + (size_t)slot_mine * (BN / 4) * BM + row_in_tile;
 #pragma unroll 1
         for (int c = 0; c < BN / 32; ++c) {
           float v[32];
@@ -540,15 +659,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
         }
         // the accumulator may be handed back at once: the own part is read from TMEM again only when nothing follows
         // in this CTA, and then nobody overwrites it
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&tempty_bar[acc]);
+        release_acc();
         asm volatile("bar.sync 1, 128;" ::: "memory");
         if (warp == 2 && lane == 0) {
           __threadfence();   // cumulative: orders the partial rows all 128 threads wrote before the barrier
-          const int old = atomicAdd(&split_counters[tile], 1);
+          const int old = atomicAdd(&split_counters[counter], 1);
           s_last = (old == n_splits - 1);
-          if (old == n_splits - 1) split_counters[tile] = 0;   // ready for the next launch
+          if (old == n_splits - 1) split_counters[counter] = 0;   // ready for the next launch
           __threadfence();
         }
         asm volatile("bar.sync 1, 128;" ::: "memory");
@@ -565,7 +682,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
               int k = 0;
               for (int p = 0; p < n_splits; ++p) {
                 if (p == pc.part) continue;
-                const int slot = p == 0 ? pc.slot0 : pc.slot_next + 2 * n_tiles_m * (p - 1);
+                const int slot = p == 0 ? slot0 : slot_next + slot_stride * (p - 1);
                 const uint8_t* src = reinterpret_cast<const uint8_t*>(split_ws) + (size_t)slot * kPartBytes;
                 for (int off = 0; off < kPartBytes; off += 32768)
                   bulk_g2s(smem + (size_t)k * kPartBytes + off, src + off, 32768, red_bar);
@@ -576,7 +693,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
             RingLoader ld{tacc, reinterpret_cast<const float4*>(smem) + row_in_tile, BN, pc.part, n_splits};
             row_epilogue<BN>(ep, ld, m, n0);
           } else {
-            SplitLoader ld{split_ws, BN, row_in_tile, pc.slot0, pc.slot_next, 2 * n_tiles_m, n_splits, m < ep.M};
+            SplitLoader ld{split_ws, BN, row_in_tile, slot0, slot_next, slot_stride, n_splits, m < ep.M};
             row_epilogue<BN>(ep, ld, m, n0);
           }
         }
@@ -588,11 +705,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
   griddep_launch();   // this CTA's work is done: the next kernel's CTAs may be scheduled onto freed SMs
   tc_fence_before();
   __syncthreads();
+  if constexpr (PAIR) cluster_sync_all();   // the peer may read this CTA's operands and signal its barriers until here
   if (warp == 1) {
     tc_fence_after();
-    tmem_dealloc(tmem_base, Cfg::kTmemCols);
+    if constexpr (PAIR) tmem_dealloc_pair(tmem_base, Cfg::kTmemCols);
+    else tmem_dealloc(tmem_base, Cfg::kTmemCols);
   }
 }
+
 
 // ---- host side -------------------------------------------------------------------------------------
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -621,7 +741,7 @@ struct TcState {
   int* split_counters = nullptr;
   EncodeTiledFn encode = nullptr;
   std::unordered_map<MapKey, CUtensorMap, MapKeyHash> maps;
-  bool configured[3] = {false, false, false};
+  bool configured[4] = {false, false, false, false};
 };
 
 // [rows, cols] bf16 row-major, box = [box_rows, 64 columns], 128-byte swizzle, zero fill out of bounds
@@ -642,44 +762,69 @@ const CUtensorMap* get_map(TcState* st, const void* ptr, uint64_t rows, uint64_t
   return &st->maps.emplace(key, m).first->second;
 }
 
-template <int BN>
+template <int BN, bool PAIR>
 bool launch_bn(TcState* st, int idx, const GemmArgs& a, const EpiParams& ep, bool stream_k, cudaStream_t stream) {
-  using Cfg = TcCfg<BN>;
+  using Cfg = TcCfg<BN, PAIR>;
   if (!st->configured[idx]) {
-    if (cudaFuncSetAttribute(gemm_tc_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes) != cudaSuccess)
+    if (cudaFuncSetAttribute(gemm_tc_kernel<BN, PAIR>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes) !=
+        cudaSuccess)
       return false;
     st->configured[idx] = true;
   }
+  constexpr int kRows = PAIR ? 2 * BM : BM;
   const bool swiglu = a.epi == EPI_SWIGLU;
   const uint64_t w_rows = swiglu ? 2ull * a.N : (uint64_t)a.N;
-  const int thin = a.M <= 32 ? 1 : 0;
+  const int thin = (!PAIR && a.M <= 32) ? 1 : 0;
   const CUtensorMap* mx = get_map(st, a.x, a.M, a.K, thin ? 32 : BM);
-  const CUtensorMap* mw = get_map(st, a.w, w_rows, a.K, swiglu ? BN / 2 : BN);
+  const CUtensorMap* mw = get_map(st, a.w, w_rows, a.K, (swiglu || PAIR) ? BN / 2 : BN);
   if (!mx || !mw) return false;
   const int out_per_tile = swiglu ? BN / 2 : BN;
   const int n_tiles_n = (a.N + out_per_tile - 1) / out_per_tile;
-  const int n_tiles = ((a.M + BM - 1) / BM) * n_tiles_n;
+  const int mt = (a.M + kRows - 1) / kRows;
+  const int n_tiles = mt * n_tiles_n;
   const long long KB = a.K / BK;
-  int grid = n_tiles < st->n_sm ? n_tiles : st->n_sm;
+  const int n_units = PAIR ? st->n_sm / 2 : st->n_sm;       // scheduling units: CTAs, or clusters of two
+  int units = n_tiles < n_units ? n_tiles : n_units;
   int dp_tiles = n_tiles;       // whole tiles, strided
   long long per = 1;
   if (stream_k) {
     // all but the last one-to-two waves as whole tiles; the k-blocks of the remaining tile columns evenly over
-    // teams of mt CTAs (one per row tile)
-    const int mt = (a.M + BM - 1) / BM;
-    const int n_teams = st->n_sm / mt;                  // the caller made sure that mt <= n_sm
-    const int full = n_tiles / st->n_sm;
-    dp_tiles = full >= 2 ? ((full - 1) * st->n_sm / mt) * mt : 0;
+    // teams of mt units (one per row tile)
+    const int n_teams = n_units / mt;                   // the caller made sure that mt <= n_units
+    const int full = n_tiles / n_units;
+    dp_tiles = full >= 2 ? ((full - 1) * n_units / mt) * mt : 0;
     const long long total = (long long)((n_tiles - dp_tiles) / mt) * KB;
     const long long teams = total < n_teams ? total : n_teams;
     per = (total + teams - 1) / teams;
     if (per < 4 && total >= 4) per = 4;                 // keep pieces long enough to amortise their hand-over
     const int used = (int)((total + per - 1) / per);    // teams that get a range
-    grid = dp_tiles ? st->n_sm : used * mt;             // (with whole tiles behind, the grid stays at the SM count)
+    units = dp_tiles ? n_units : used * mt;             // (with whole tiles behind, the grid stays at full size)
   }
-  launch_pdl(gemm_tc_kernel<BN>, dim3(grid), dim3(kTcThreads), Cfg::kSmemBytes, stream, *mx, *mw, a.M, n_tiles_n, a.K, a.N,
-             dp_tiles, per, thin, st->split_ws, st->split_counters, ep);
-  return true;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(PAIR ? 2 * units : units);
+  cfg.blockDim = dim3(kTcThreads);
+  cfg.dynamicSmemBytes = Cfg::kSmemBytes;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[2];
+  int n_attr = 0;
+  if (PAIR) {
+    attr[n_attr].id = cudaLaunchAttributeClusterDimension;
+    attr[n_attr].val.clusterDim.x = 2;
+    attr[n_attr].val.clusterDim.y = 1;
+    attr[n_attr].val.clusterDim.z = 1;
+    ++n_attr;
+  }
+  // programmatic dependent launch, except inside a stream capture (see launch_pdl)
+  cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+  if (cudaStreamIsCapturing(stream, &cap) == cudaSuccess && cap == cudaStreamCaptureStatusNone) {
+    attr[n_attr].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[n_attr].val.programmaticStreamSerializationAllowed = 1;
+    ++n_attr;
+  }
+  cfg.attrs = attr;
+  cfg.numAttrs = n_attr;
+  return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<BN, PAIR>, *mx, *mw, a.M, n_tiles_n, a.K, a.N, dp_tiles, per, thin,
+                            st->split_ws, st->split_counters, ep) == cudaSuccess;
 }
 
 }  // namespace
@@ -742,42 +887,54 @@ bool launch_gemm_tc(const GemmArgs& a, void* tc_state, int* status, cudaStream_t
   const int mt = (a.M + BM - 1) / BM;
   const int KB = a.K / BK;
   int best_bn = 0;
-  bool best_sk = false;
+  bool best_sk = false, best_pair = false;
   double best_t = 1e30;
-  const int bns[3] = {256, 128, 64};
-  const double kb_tensor[3] = {0.44, 0.27, 0.22};
-  for (int bi = 0; bi < 3; ++bi) {
+  // configurations: single CTAs with 128-row tiles of width 256 / 128 / 64, and CTA pairs with 256 x 256 tiles (a
+  // k-block of a pair takes about 0.87 of the single CTA's, for twice the rows: the pair halves the weight bytes
+  // each SM's tensor core pulls out of its own shared memory)
+  const int bns[4] = {256, 128, 64, 256};
+  const double kb_tensor[4] = {0.44, 0.27, 0.22, 0.385};
+  const bool pair_ok = a.M > BM && (swiglu ? a.N % 128 == 0 : a.N % 256 == 0) && !(a.epi == EPI_QKV_ROPE && 256 % a.head_dim);
+  for (int bi = 0; bi < 4; ++bi) {
     const int bn = bns[bi];
+    const bool pair = bi == 3;
+    if (pair && !pair_ok) continue;
+    const int rows_tile = pair ? 2 * BM : BM;
+    const int units = pair ? st->n_sm / 2 : st->n_sm;            // CTAs or clusters
+    const int mtc = (a.M + rows_tile - 1) / rows_tile;
     const int per = swiglu ? bn / 2 : bn;
     if (a.epi == EPI_QKV_ROPE && (bn < a.head_dim || a.N % bn)) continue;
     if (swiglu && (a.N % per)) continue;
-    const int tiles = mt * ((a.N + per - 1) / per);
-    if (tiles > kSplitCounters) continue;
-    const long long waves = (tiles + st->n_sm - 1) / st->n_sm;
+    const int tiles = mtc * ((a.N + per - 1) / per);
+    if (tiles * (pair ? 2 : 1) > kSplitCounters) continue;
+    const long long waves = (tiles + units - 1) / units;
     // a k-block costs its tensor time, or the time one SM needs to stream its share of the weight bytes (the
-    // mt CTAs that work on one weight tile at the same time share them through L2)
+    // CTAs that work on one weight tile at the same time share them through L2)
     const double kbt = fmax(kb_tensor[bi], (bn * 128.0 / mt) / 35e3);
     const double rows = a.M < BM ? a.M : BM;
     const double t_plain = (double)waves * KB * kbt;
-    const int sk_ctas = mt <= st->n_sm ? (st->n_sm / mt) * mt : 1;     // teams of mt CTAs
-    const double t_sk = ((double)tiles * KB / sk_ctas + 1.0) * kbt + 3.0 + rows * bn * 4.0 * 2.5 / 16e3;
-    if (t_plain < best_t) { best_t = t_plain; best_bn = bn; best_sk = false; }
-    const bool ws_fits = (size_t)2 * st->n_sm * BM * bn * 4 <= kSplitWsBytes && mt <= st->n_sm;
-    const long long full = tiles / st->n_sm, rem = tiles % st->n_sm;
+    const int sk_units = mtc <= units ? (units / mtc) * mtc : 1;     // teams of mtc units
+    const double t_sk = ((double)tiles * KB / sk_units + 1.0) * kbt + 3.0 + rows * bn * 4.0 * 2.5 / 16e3;
+    if (t_plain < best_t) { best_t = t_plain; best_bn = bn; best_sk = false; best_pair = pair; }
+    const bool ws_fits = (size_t)2 * st->n_sm * BM * bn * 4 <= kSplitWsBytes && mtc <= units;
+    const long long full = tiles / units, rem = tiles % units;
     if (ws_fits && full >= 2) {
-      // a ragged last wave: the last (n_sm + rem) tiles are cut evenly over the SMs and done FIRST, so that their
+      // a ragged last wave: the last (units + rem) tiles are cut evenly over the SMs and done FIRST, so that their
       // hand-over (park the partial, counter, reduction by the last arriver) hides under the whole tiles after it.
       // Measured: the cut tiles run a little slower than whole ones, so this only pays when the last wave would
-      // leave a good part of the machine idle (a nearly empty wave of whole tiles is cheap: its few CTAs run fast).
-      const double idle = rem ? (double)(st->n_sm - rem) / st->n_sm / (double)(full + 1) : 0.0;
-      const double t_h = (double)tiles * KB / st->n_sm * kbt + 2.0;
-      if (idle > 0.12 && t_h < best_t) { best_t = t_h; best_bn = bn; best_sk = true; }
+      // leave a good part of the machine idle.
+      const double idle = rem ? (double)(units - rem) / units / (double)(full + 1) : 0.0;
+      const double t_h = (double)tiles * KB / units * kbt + 2.0;
+      if (idle > 0.12 && t_h < best_t) { best_t = t_h; best_bn = bn; best_sk = true; best_pair = pair; }
     } else if (ws_fits && t_sk < best_t) {
       // no whole tiles to hide the hand-over under: it happens in every CTA at once at the end of the kernel and
       // costs about 3 us + 0.6 us per KB of partial tile, which t_sk charges
-      best_t = t_sk; best_bn = bn; best_sk = true;
+      best_t = t_sk; best_bn = bn; best_sk = true; best_pair = pair;
     }
   }
+  if (st->force_bn == 512) {    // tuning aid: the CTA-pair kernel, "512,<0 whole tiles | 1 stream-K>"
+    if (pair_ok && (a.M + 255) / 256 <= st->n_sm / 2) return launch_bn<256, true>(st, 3, a, ep, st->force_s != 0, stream);
+  } else
   if (st->force_bn) {   // tuning aid: RECG_GEMM_FORCE="<bn>,<0 whole tiles | 1 stream-K>"; ignored where it does not fit
     const int bn = st->force_bn;
     const int per = swiglu ? bn / 2 : bn;
@@ -786,15 +943,17 @@ bool launch_gemm_tc(const GemmArgs& a, void* tc_state, int* status, cudaStream_t
                           mt * ((a.N + per - 1) / per) <= kSplitCounters;
     if (shape_ok) {
       best_bn = bn;
+      best_pair = false;
       best_sk = st->force_s != 0 && mt <= st->n_sm && (size_t)2 * st->n_sm * BM * bn * 4 <= kSplitWsBytes;
     }
   }
   if (!best_bn) return false;
   if (swiglu && (a.N % 32)) return false;
+  if (best_pair) return launch_bn<256, true>(st, 3, a, ep, best_sk, stream);
   switch (best_bn) {
-    case 256: return launch_bn<256>(st, 0, a, ep, best_sk, stream);
-    case 128: return launch_bn<128>(st, 1, a, ep, best_sk, stream);
-    default: return launch_bn<64>(st, 2, a, ep, best_sk, stream);
+    case 256: return launch_bn<256, false>(st, 0, a, ep, best_sk, stream);
+    case 128: return launch_bn<128, false>(st, 1, a, ep, best_sk, stream);
+    default: return launch_bn<64, false>(st, 2, a, ep, best_sk, stream);
   }
 }
 
