@@ -506,12 +506,57 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
   if constexpr (PAIR) cluster_sync_all();   // both CTAs' barriers are initialised before anyone signals across
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  griddep_wait();   // everything above touched only shared memory and TMEM
+  // (each role waits for the kernels before this one where it first needs their results)
 
   if (warp == 0) {
     // ------------------------------ TMA producer ------------------------------
     if (elect_one()) {
-      int st_idx = 0;
+      // of a pair, rank r loads rows [128 r, 128 r + 128) of the x tile and half r of the weight tile (SwiGLU: rank 0
+      // the gate rows, rank 1 the up rows); all four loads of the pair complete on the leader's barrier
+      auto expect = [&](int s) {
+        if constexpr (PAIR) {
+          if (rank == 0) mbar_arrive_expect_tx(&full_bar[s], 2 * stage_bytes);
+        } else {
+          mbar_arrive_expect_tx(&full_bar[s], stage_bytes);
+        }
+      };
+      auto load_w = [&](int s, int kb, int tn) {
+        uint8_t* b_dst = smem + s * stage_bytes + a_bytes;
+        if constexpr (PAIR) {
+          const uint32_t full0 = mapa_rank(smem_u32(&full_bar[s]), 0);
+          const int w_row = swiglu ? (rank == 0 ? tn * (BN / 2) : up_row_offset + tn * (BN / 2)) : tn * BN + (int)rank * (BN / 2);
+          tma_load_2d_pair(smem_u32(b_dst), &map_w, kb * BK, w_row, full0);
+        } else if (swiglu) {
+          tma_load_2d(b_dst, &map_w, kb * BK, tn * (BN / 2), &full_bar[s]);
+          tma_load_2d(b_dst + Cfg::kBBytes / 2, &map_w, kb * BK, up_row_offset + tn * (BN / 2), &full_bar[s]);
+        } else {
+          tma_load_2d(b_dst, &map_w, kb * BK, tn * BN, &full_bar[s]);
+        }
+      };
+      auto load_x = [&](int s, int kb, int tm) {
+        uint8_t* a_dst = smem + s * stage_bytes;
+        if constexpr (PAIR) tma_load_2d_pair(smem_u32(a_dst), &map_x, kb * BK, tm * kRows + (int)rank * BM, mapa_rank(smem_u32(&full_bar[s]), 0));
+        else tma_load_2d(a_dst, &map_x, kb * BK, tm * BM, &full_bar[s]);
+      };
+      // The weights do not depend on the kernels before this one: the weight tiles of the first stages are requested
+      // BEFORE waiting for those kernels, so the ring fills while they drain (or while a short kernel such as the
+      // RMSNorm in front of this projection runs); the x tiles of those stages follow right after the wait.
+      int n_pre = 0, pre_kb0 = 0, pre_tm = 0;
+      if (dp_count > 0 || range_lo < range_hi) {
+        long long p0 = range_lo;
+        int j0 = 0;
+        const Piece pc = make_piece(j0, dp_tiles, p0, range_hi, KB, per, unit, n_units, n_tiles_m);
+        n_pre = pc.kb1 - pc.kb0 < n_stages ? pc.kb1 - pc.kb0 : n_stages;
+        pre_kb0 = pc.kb0;
+        pre_tm = pc.tile % n_tiles_m;
+        for (int i = 0; i < n_pre; ++i) {
+          expect(i);
+          load_w(i, pre_kb0 + i, pc.tile / n_tiles_m);
+        }
+      }
+      griddep_wait();
+      for (int i = 0; i < n_pre; ++i) load_x(i, pre_kb0 + i, pre_tm);
+      int st_idx = 0, issued = 0;
       uint32_t st_phase = 0;
       bool ok = true;
       long long pos = range_lo;
@@ -523,31 +568,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
           const int s = st_idx;
           const uint32_t ph = st_phase;
           if (++st_idx == n_stages) { st_idx = 0; st_phase ^= 1; }
+          if (issued < n_pre) {       // requested above
+            ++issued;
+            continue;
+          }
           if (!(PAIR ? mbar_wait_cluster(&empty_bar[s], ph ^ 1, kSpin) : mbar_wait(&empty_bar[s], ph ^ 1, kSpin))) {
             set_status(ep.status, DEV_TIMEOUT_EMPTY);
             ok = false;
             break;
           }
-          uint8_t* a_dst = smem + s * stage_bytes;
-          uint8_t* b_dst = a_dst + a_bytes;
-          if constexpr (PAIR) {
-            // rank r loads rows [128 r, 128 r + 128) of the x tile and half r of the weight tile (SwiGLU: rank 0 the
-            // gate rows, rank 1 the up rows); all four loads of the pair complete on the leader's barrier
-            const uint32_t full0 = mapa_rank(smem_u32(&full_bar[s]), 0);
-            if (rank == 0) mbar_arrive_expect_tx(&full_bar[s], 2 * stage_bytes);
-            const int w_row = swiglu ? (rank == 0 ? tn * (BN / 2) : up_row_offset + tn * (BN / 2)) : tn * BN + (int)rank * (BN / 2);
-            tma_load_2d_pair(smem_u32(a_dst), &map_x, kb * BK, tm * kRows + (int)rank * BM, full0);
-            tma_load_2d_pair(smem_u32(b_dst), &map_w, kb * BK, w_row, full0);
-          } else {
-            mbar_arrive_expect_tx(&full_bar[s], stage_bytes);
-            tma_load_2d(a_dst, &map_x, kb * BK, tm * BM, &full_bar[s]);
-            if (swiglu) {
-              tma_load_2d(b_dst, &map_w, kb * BK, tn * (BN / 2), &full_bar[s]);
-              tma_load_2d(b_dst + Cfg::kBBytes / 2, &map_w, kb * BK, up_row_offset + tn * (BN / 2), &full_bar[s]);
-            } else {
-              tma_load_2d(b_dst, &map_w, kb * BK, tn * BN, &full_bar[s]);
-            }
-          }
+          expect(s);
+          load_x(s, kb, tm);
+          load_w(s, kb, tn);
         }
       }
       if (!ok) {  // let loads already issued land before the CTA may exit
@@ -560,7 +592,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     }
   } else if (warp == 1) {
     // ------------------------------ MMA issuer ------------------------------
-    if (rank == 0 && elect_one()) {         // of a pair only the leader issues
+    if (rank == 0 && elect_one()) {         // of a pair only the leader issues (it touches shared memory and TMEM only)
       constexpr uint32_t idesc = make_idesc(BN, kRows);
       int st_idx = 0;
       uint32_t st_phase = 0, tcount = 0;
@@ -611,6 +643,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     const int quad = warp & 3;             // TMEM lane quadrant this warp may read
     uint32_t tcount = 0;
     __shared__ int s_last;
+    griddep_wait();                        // the epilogue reads and writes what earlier kernels produced
     long long pos = range_lo;
     for (int jd = 0; jd < dp_count || pos < range_hi; ++tcount) {
       const Piece pc = make_piece(jd, dp_tiles, pos, range_hi, KB, per, unit, n_units, n_tiles_m);
