@@ -717,8 +717,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                 if (p == pc.part) continue;
                 const int slot = p == 0 ? slot0 : slot_next + slot_stride * (p - 1);
                 const uint8_t* src = reinterpret_cast<const uint8_t*>(split_ws) + (size_t)slot * kPartBytes;
-                for (int off = 0; off < kPartBytes; off += 32768)
-                  bulk_g2s(smem + (size_t)k * kPartBytes + off, src + off, 32768, red_bar);
+                constexpr int kChunk = kPartBytes < 32768 ? kPartBytes : 32768;
+                for (int off = 0; off < kPartBytes; off += kChunk)
+                  bulk_g2s(smem + (size_t)k * kPartBytes + off, src + off, kChunk, red_bar);
                 ++k;
               }
             }
