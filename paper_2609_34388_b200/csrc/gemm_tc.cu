@@ -203,16 +203,20 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint64_t* bar, uint32_t parity
 
 
 // ---- register epilogue: one thread owns one output row -------------------------------------------
+// add = true accumulates into the fp32 residual stream with vector reductions at L2: every element receives
+// exactly one addend from exactly one thread per launch, so the result is the same single rounding as a
+// load-add-store, without the load's round trip in front of every chunk.
 __device__ __forceinline__ void store_chunk_f32(float* dst, const float (&v)[32], bool add) {
 #pragma unroll
   for (int i = 0; i < 8; ++i) {
-    float4 o = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
     float4* p = reinterpret_cast<float4*>(dst) + i;
     if (add) {
-      const float4 h = *p;
-      o.x += h.x; o.y += h.y; o.z += h.z; o.w += h.w;
+      asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(p), "f"(v[4 * i]), "f"(v[4 * i + 1]), "f"(v[4 * i + 2]),
+                   "f"(v[4 * i + 3])
+                   : "memory");
+    } else {
+      *p = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
     }
-    *p = o;
   }
 }
 __device__ __forceinline__ void store_chunk_bf16(__nv_bfloat16* dst, const float (&v)[32]) {
