@@ -28,7 +28,8 @@ namespace {
 
 constexpr int BM = 128, BK = 64;
 constexpr int kTcThreads = 192;
-constexpr int kSmemBudget = 200 * 1024;
+constexpr int kSmemBudget = 192 * 1024;     // operand ring (every configuration's stage size divides it)
+constexpr int kStageOutBytes = 4 * 4096;      // per epilogue warp: 32 rows x 32 fp32 for transposing output chunks
 constexpr uint32_t kSpin = 1u << 22;
 
 template <int BN, bool PAIR = false> struct TcCfg {
@@ -46,7 +47,7 @@ template <int BN, bool PAIR = false> struct TcCfg {
       (kSmemBudget / kThinStageBytes) > kMaxStages ? kMaxStages : (kSmemBudget / kThinStageBytes);
   static constexpr int kRingBytes = kSmemBudget + kABytes;     // either ring plus the pad
   static constexpr int kBarBytes = (2 * kMaxStages + 5) * 8 + 16;
-  static constexpr int kSmemBytes = kRingBytes + kBarBytes + 1024;  // + slack for 1024-byte alignment
+  static constexpr int kSmemBytes = kRingBytes + kStageOutBytes + kBarBytes + 1024;  // + slack for 1024-byte alignment
   static constexpr int kTmemCols = 2 * BN < 32 ? 32 : 2 * BN;                  // power of two: 128, 256, 512
 };
 
@@ -219,6 +220,52 @@ __device__ __forceinline__ void store_chunk_f32(float* dst, const float (&v)[32]
     }
   }
 }
+// Warp-wide stores of a 32-row x 32-column chunk (lane = row holds the row's 32 values): the chunk is transposed
+// through 4 KB of shared memory so that every store instruction writes whole 128-byte (fp32) or 64-byte (bf16)
+// row segments instead of 16 bytes in each of 32 different rows.  dst0 points at (row 0 of the warp, first column
+// of the chunk); rows >= valid_rows are not written.  Every lane must call.
+__device__ __forceinline__ void store_rows_f32(float* dst0, size_t row_stride, int valid_rows, const float (&v)[32], bool add,
+                                               float* stg, int lane) {
+  float4* s4 = reinterpret_cast<float4*>(stg);
+#pragma unroll
+  for (int q = 0; q < 8; ++q)
+    s4[lane * 8 + (q ^ (lane & 7))] = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+  __syncwarp();
+  const int rq = lane >> 3, q = lane & 7;
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    const int r = 4 * j + rq;
+    const float4 t = s4[r * 8 + (q ^ (r & 7))];
+    if (r < valid_rows) {
+      float4* p = reinterpret_cast<float4*>(dst0 + (size_t)r * row_stride) + q;
+      if (add) asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(p), "f"(t.x), "f"(t.y), "f"(t.z), "f"(t.w) : "memory");
+      else *p = t;
+    }
+  }
+  __syncwarp();
+}
+__device__ __forceinline__ void store_rows_bf16(__nv_bfloat16* dst0, size_t row_stride, int valid_rows, const float (&v)[32],
+                                                float* stg, int lane) {
+  uint4* s4 = reinterpret_cast<uint4*>(stg);
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    uint4 o;
+    o.x = pack_bf16(v[8 * q], v[8 * q + 1]);
+    o.y = pack_bf16(v[8 * q + 2], v[8 * q + 3]);
+    o.z = pack_bf16(v[8 * q + 4], v[8 * q + 5]);
+    o.w = pack_bf16(v[8 * q + 6], v[8 * q + 7]);
+    s4[lane * 4 + (q ^ (lane & 3))] = o;
+  }
+  __syncwarp();
+  const int rq = lane >> 2, q = lane & 3;
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const int r = 8 * j + rq;
+    const uint4 t = s4[r * 4 + (q ^ (r & 3))];
+    if (r < valid_rows) *(reinterpret_cast<uint4*>(dst0 + (size_t)r * row_stride) + q) = t;
+  }
+  __syncwarp();
+}
 __device__ __forceinline__ void store_chunk_bf16(__nv_bfloat16* dst, const float (&v)[32]) {
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
@@ -352,9 +399,13 @@ __device__ __forceinline__ Piece make_piece(int& jd, int dp_tiles, long long& po
 }
 
 // Epilogue of one accumulator tile for the calling thread's row.
+// stg: this warp's 4 KB transposition buffer.  All 32 lanes of the warp call together.
 template <int BN, typename Loader>
-__device__ __forceinline__ void row_epilogue(const EpiParams& ep, const Loader& load, int m, int n0) {
+__device__ __forceinline__ void row_epilogue(const EpiParams& ep, const Loader& load, int m, int n0, float* stg) {
   const bool row_ok = m < ep.M;
+  const int lane = threadIdx.x & 31;
+  const int m_base = m - lane;                                  // first row of this warp
+  const int valid_rows = ep.M - m_base < 0 ? 0 : (ep.M - m_base > 32 ? 32 : ep.M - m_base);
   if (ep.epi == EPI_SWIGLU) {
     // accumulator columns [0, BN/2) are gate, [BN/2, BN) up; n0 is the first output column
     __nv_bfloat16* out = static_cast<__nv_bfloat16*>(ep.out);
@@ -363,10 +414,10 @@ __device__ __forceinline__ void row_epilogue(const EpiParams& ep, const Loader& 
       float g[32], u[32];
       load(c * 32, g);
       load(BN / 2 + c * 32, u);
-      if (row_ok && n0 + c * 32 < ep.N) {
+      if (n0 + c * 32 < ep.N) {
 #pragma unroll
         for (int i = 0; i < 32; ++i) g[i] = silu_f(g[i]) * u[i];
-        store_chunk_bf16(out + (size_t)m * ep.N + n0 + c * 32, g);
+        store_rows_bf16(out + (size_t)m_base * ep.N + n0 + c * 32, ep.N, valid_rows, g, stg, lane);
       }
     }
     return;
@@ -432,11 +483,13 @@ __device__ __forceinline__ void row_epilogue(const EpiParams& ep, const Loader& 
     float v[32];
     load(c * 32, v);
     const int n = n0 + c * 32;
-    if (!row_ok || n >= ep.N) continue;
+    if (n >= ep.N) continue;
     if (n + 32 <= ep.N) {
-      if (ep.epi == EPI_PLAIN_BF16) store_chunk_bf16(static_cast<__nv_bfloat16*>(ep.out) + (size_t)m * ep.N + n, v);
-      else store_chunk_f32(static_cast<float*>(ep.out) + (size_t)m * ep.N + n, v, ep.epi == EPI_RESIDUAL);
-    } else {  // ragged right edge (N is a multiple of 16 but not of 32)
+      if (ep.epi == EPI_PLAIN_BF16)
+        store_rows_bf16(static_cast<__nv_bfloat16*>(ep.out) + (size_t)m_base * ep.N + n, ep.N, valid_rows, v, stg, lane);
+      else
+        store_rows_f32(static_cast<float*>(ep.out) + (size_t)m_base * ep.N + n, ep.N, valid_rows, v, ep.epi == EPI_RESIDUAL, stg, lane);
+    } else if (row_ok) {  // ragged right edge (N is a multiple of 16 but not of 32)
       for (int i = 0; i < ep.N - n; ++i) {
         if (ep.epi == EPI_PLAIN_BF16) static_cast<__nv_bfloat16*>(ep.out)[(size_t)m * ep.N + n + i] = __float2bfloat16_rn(v[i]);
         else if (ep.epi == EPI_RESIDUAL) static_cast<float*>(ep.out)[(size_t)m * ep.N + n + i] += v[i];
@@ -462,7 +515,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
   const int n_stages = thin ? Cfg::kThinStages : Cfg::kStages;
   const int a_bytes = thin ? Cfg::kThinABytes : Cfg::kABytes;
   const int stage_bytes = a_bytes + Cfg::kBBytes;
-  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + Cfg::kRingBytes);
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + Cfg::kRingBytes + kStageOutBytes);
   uint64_t* empty_bar = full_bar + Cfg::kMaxStages;
   uint64_t* tfull_bar = empty_bar + Cfg::kMaxStages;
   uint64_t* tempty_bar = tfull_bar + 2;
@@ -645,6 +698,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
   } else {
     // ------------------------------ epilogue warps ------------------------------
     const int quad = warp & 3;             // TMEM lane quadrant this warp may read
+    float* stg = reinterpret_cast<float*>(smem + Cfg::kRingBytes) + (warp - 2) * 1024;
     uint32_t tcount = 0;
     __shared__ int s_last;
     griddep_wait();                        // the epilogue reads and writes what earlier kernels produced
@@ -673,7 +727,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
       };
       const int n0 = swiglu ? tn * (BN / 2) : tn * BN;
       if (n_splits == 1) {
-        row_epilogue<BN>(ep, TmemLoader{tacc}, m, n0);
+        row_epilogue<BN>(ep, TmemLoader{tacc}, m, n0, stg);
         release_acc();
       } else {
         // park this split's partial tile and let the LAST split to arrive reduce all partials in split order
@@ -729,10 +783,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
             }
             if (!mbar_wait(red_bar, 0, kSpin)) set_status(ep.status, DEV_TIMEOUT_FULL);
             RingLoader ld{tacc, reinterpret_cast<const float4*>(smem) + row_in_tile, BN, pc.part, n_splits};
-            row_epilogue<BN>(ep, ld, m, n0);
+            row_epilogue<BN>(ep, ld, m, n0, stg);
           } else {
             SplitLoader ld{split_ws, BN, row_in_tile, slot0, slot_next, slot_stride, n_splits, m < ep.M};
-            row_epilogue<BN>(ep, ld, m, n0);
+            row_epilogue<BN>(ep, ld, m, n0, stg);
           }
         }
         asm volatile("bar.sync 1, 128;" ::: "memory");       // s_last is reused by the next unit
