@@ -446,8 +446,7 @@ __device__ __forceinline__ void row_epilogue(const EpiParams& ep, const Loader& 
         float lo[32], hi[32];
         load(hl * D + c * 32, lo);
         load(hl * D + half + c * 32, hi);
-        if (!row_ok) continue;
-        if (!is_v) {
+        if (row_ok && !is_v) {
           const float2* cs = ep.rope_cs + (size_t)m * half + c * 32;
 #pragma unroll
           for (int i = 0; i < 32; ++i) {
@@ -457,10 +456,10 @@ __device__ __forceinline__ void row_epilogue(const EpiParams& ep, const Loader& 
             hi[i] = b;
           }
         }
-        if (is_q) {
-          __nv_bfloat16* dst = q + ((size_t)m * ep.n_q + head) * D + c * 32;
-          store_chunk_bf16(dst, lo);
-          store_chunk_bf16(dst + half, hi);
+        if (is_q) {      // (the same for the whole warp)
+          __nv_bfloat16* dst0 = q + ((size_t)m_base * ep.n_q + head) * D + c * 32;
+          store_rows_bf16(dst0, (size_t)ep.n_q * D, valid_rows, lo, stg, lane);
+          store_rows_bf16(dst0 + half, (size_t)ep.n_q * D, valid_rows, hi, stg, lane);
         } else if (kv_base) {
           // the pool tile is swizzled in 16-byte chunks: store chunk by chunk
 #pragma unroll
