@@ -402,15 +402,19 @@ def bench_verify(binding, peaks):
 def bench_c128(binding, W, shape, peaks, args):
     """High-concurrency point: full model, 128 requests (see c128_descriptor), per-class times."""
     desc = c128_descriptor(5)
+    # the same context and pool also serve the concurrency sweep below (configs[2]'s recipe at other batch sizes)
+    sweep_descs = {C: synth.batch_descriptor(C, [4, 8, 16, 32], None, 512, 8192, seed=40 + C) for C in (1, 2, 4, 8, 16, 32, 64, 128)}
+    all_descs = [desc] + list(sweep_descs.values())
+    n_pages = max(d.n_pages for d in all_descs)
     free_b, _ = torch.cuda.mem_get_info()
-    cfg = binding.make_config(shape, 128, 2048, desc.page_table.shape[1])
-    need = binding.lib().recg_kv_pool_bytes(__import__("ctypes").byref(cfg), desc.n_pages)
-    if need + (8 << 30) > free_b:
+    cfg = binding.make_config(shape, 128, max(2048, max(d.n_tokens for d in all_descs)), max(d.page_table.shape[1] for d in all_descs))
+    need = binding.lib().recg_kv_pool_bytes(__import__("ctypes").byref(cfg), n_pages)
+    if need + (10 << 30) > free_b:
         return {"skipped": f"pool of {need / 1e9:.0f} GB does not fit in the {free_b / 1e9:.0f} GB that are free"}
     ctx = binding.Context(cfg, W)
-    pool = binding.alloc_kv_pool(ctx, desc.n_pages, fill="normal")
+    pool = binding.alloc_kv_pool(ctx, n_pages, fill="normal")
     ys = synth.token_ids(int(desc.verify_len.sum()), shape.vocab, seed=9)
-    batch = binding.Batch(desc.ctx_len, desc.verify_len, desc.block_size, ys, desc.page_table, pool, desc.n_pages)
+    batch = binding.Batch(desc.ctx_len, desc.verify_len, desc.block_size, ys, desc.page_table, pool, n_pages)
     vout = binding.VerifyOut(batch.n_req, batch.n_tok, batch.n_ver, host=False)
     for _ in range(3):
         ctx.recg_step(batch)
@@ -446,6 +450,34 @@ def bench_c128(binding, W, shape, peaks, args):
                     "frac_of_bf16_sustained": round(gemm_tf / peaks["bf16_tflops_sustained"], 4)},
            "attention": {"ms_per_step": round(attn_ms, 3), "gbs": round(attn_gbs, 1),
                          "frac_of_hbm_measured": round(attn_gbs / peaks["hbm_gbs"], 4)}}
+    # ---- tokens/s against concurrency: configs[2]'s recipe (blocks U{4,8,16,32}, verify_len = block, context
+    # U[512,8192]) at 1 .. 128 requests, one batch draw each, whole step (recg_step + recg_verify), device resident
+    sweep = []
+    for C, d in sweep_descs.items():
+        ysw = synth.token_ids(int(d.verify_len.sum()), shape.vocab, seed=50 + C)
+        bt = binding.Batch(d.ctx_len, d.verify_len, d.block_size, ysw, d.page_table, pool, n_pages)
+        vo = binding.VerifyOut(bt.n_req, bt.n_tok, bt.n_ver, host=False)
+        for _ in range(3):
+            ctx.recg_step(bt)
+            ctx.recg_verify(bt, out=vo)
+        torch.cuda.synchronize()
+        n_it = 5
+        e0.record()
+        for _ in range(n_it):
+            ctx.recg_step(bt)
+            ctx.recg_verify(bt, out=vo)
+        e1.record()
+        torch.cuda.synchronize()
+        msw = e0.elapsed_time(e1) / n_it
+        cw = algorithmic_counts(shape, d)
+        sweep.append({"concurrency": C, "tokens_per_step": bt.n_tok, "kv_tokens": int(np.sum(d.ctx_len + d.verify_len + d.block_size)),
+                      "ms_per_step": round(msw, 3), "tokens_per_s": round(bt.n_tok / (msw / 1e3), 1),
+                      "ideal_ms": round(max(sum(cw["wbytes"].values()) / peaks["hbm_gbs"] / 1e6,
+                                            sum(cw["flops"].values()) / peaks["bf16_tflops_sustained"] / 1e9) +
+                                        cw["attn_bytes"] / peaks["hbm_gbs"] / 1e6, 3)})
+    out["concurrency_sweep"] = {"workload": "configs[2] recipe at other batch sizes, one draw each, processed tokens/s of the whole step; "
+                                            "ideal_ms = max(weight stream, GEMM flops at sustained peak) + KV stream, of measured peaks",
+                                "points": sweep}
     ctx.recg_free()
     del pool
     torch.cuda.empty_cache()
