@@ -58,15 +58,15 @@ constexpr int kKVStages = kKStages + kVStages;
 constexpr int kThreads = 384;                    // warpgroup 0: producer K, MMA, producer V, idle; warpgroups 1, 2: softmax
 constexpr int kSoftThreads = 256;
 constexpr uint32_t kSpin = 1u << 22;
-constexpr int kTmemCols = 512;                 // S of group 0 / 1 at [0,128) / [128,256), O of group 0 / 1 at [256,384) / [384,512);
-                                               // bf16 P of a group overwrites columns [0,64) of its S
+constexpr int kTmemCols = 512;                 // two S buffers of 128 columns (stage & 1); group g owns columns [64 g, 64 g + 64) of each
+                                               // and overwrites the first 32 of them with its bf16 P; O of group g at 256 + 128 g
 constexpr int kTmemO = 2 * kBT;
 
 constexpr int kOffQ = 0;                       // two Q buffers: item i uses buffer i & 1
 constexpr int kOffKV = kOffQ + 2 * kQBytes;
 constexpr int kOffML = kOffKV + kKVStages * kKVStageBytes;   // float2 [2 groups][128 rows]: (reference max, sum)
 constexpr int kOffBar = kOffML + 2 * 128 * 8;
-constexpr int kNumBars = 2 * kKVStages + 2 + 2 + 2 + 2 + 2 + 1;
+constexpr int kNumBars = 2 * kKVStages + 2 + 2 + 2 + 4 + 1 + 1 + 1;
 constexpr int kSmemBytes = kOffBar + kNumBars * 8 + 16 + 32;   // barriers, TMEM slot + flags + item range, first item
 static_assert(kSmemBytes <= 227 * 1024, "shared memory budget");
 
@@ -192,10 +192,11 @@ __global__ void __launch_bounds__(kThreads, 1) attention_tc_kernel(const __grid_
   uint64_t* kv_empty = bars + kKVStages;    // [kKVStages]
   uint64_t* q_full = bars + 2 * kKVStages;  // [2]  per Q buffer
   uint64_t* q_empty = q_full + 2;           // [2]
-  uint64_t* s_full = q_full + 4;            // [2]  per softmax group
-  uint64_t* p_full = q_full + 6;            // [2]
-  uint64_t* o_full = q_full + 8;            // [2]
-  uint64_t* o_empty = q_full + 10;
+  uint64_t* s_full = q_full + 4;            // [2]  per S buffer (stage & 1); both groups wait on it
+  uint64_t* p_full = q_full + 6;            // [4]  per (softmax group, S buffer): index 2 g + (stage & 1)
+  uint64_t* pv_done = q_full + 10;          // both groups' P V products of a stage have completed
+  uint64_t* o_full = q_full + 11;
+  uint64_t* o_empty = q_full + 12;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + kNumBars);
   float2* ml_smem = reinterpret_cast<float2*>(smem + kOffML);
 
@@ -238,9 +239,10 @@ __global__ void __launch_bounds__(kThreads, 1) attention_tc_kernel(const __grid_
       mbar_init(&q_full[s], 1);
       mbar_init(&q_empty[s], 8);
       mbar_init(&s_full[s], 1);
-      mbar_init(&p_full[s], 4);
-      mbar_init(&o_full[s], 1);
     }
+    for (int s = 0; s < 4; ++s) mbar_init(&p_full[s], 4);
+    mbar_init(pv_done, 1);
+    mbar_init(o_full, 1);
     mbar_init(o_empty, 8);
     fence_barrier_init();
     asm volatile("prefetch.tensormap [%0];" ::"l"(&qmap) : "memory");
@@ -363,24 +365,24 @@ __global__ void __launch_bounds__(kThreads, 1) attention_tc_kernel(const __grid_
     } else if (warp == 1) {
       // ------------------------------------ MMA issuer ------------------------------------
       if (elect_one()) {
-        uint32_t blk = 0, item_cnt = 0;
-        uint32_t cp[2] = {0, 0};   // P V products issued for each softmax group so far
-        // S of group g = Q K^T for running block b.  The tensor pipe executes in issue order, so this runs after the
-        // group's previous P V, which read P out of the same TMEM columns.
-        auto issue_qk = [&](uint32_t b, int g, uint32_t q_addr) {
+        uint32_t blk = 0, item_cnt = 0;      // running stage (128-token KV block) and item counters
+        // Group g works on tokens [64 g, 64 g + 64) of EVERY stage.  S of stage b = Q K^T goes to S buffer b & 1 (one
+        // N = 128 product for both groups), so the S of stage b + 1 is ready while the groups still work on stage b;
+        // the tensor pipe executes in issue order, which puts it after the P V products that read the buffer's
+        // previous P.  Shared-memory descriptors are linear in the address (no carry out of the 14-bit field
+        // within the operand areas), so the per-instruction descriptors are a base plus constants.
+        auto issue_qk = [&](uint32_t b, uint64_t dq0) {
           const int s = b % kKStages;
           bwait(&kv_full[s], (b / kKStages) & 1, DEV_TIMEOUT_FULL);
           tc_fence_after();
-          const uint32_t k_addr = smem_base + kOffKV + s * kKVStageBytes;
+          // K block: 16 token groups (2 per page) 2 KB apart; the dim half selects the atom next door
+          const uint64_t dk0 = desc_kmajor(smem_base + kOffKV + s * kKVStageBytes, 2048);
 #pragma unroll
-          for (int kk = 0; kk < D / 16; ++kk) {
-            const uint64_t da = desc_kmajor(q_addr + (kk >> 2) * (128 * 128) + (kk & 3) * 32);
-            // K block: 16 token groups (2 per page) 2 KB apart; the dim half selects the atom next door
-            const uint64_t db = desc_kmajor(k_addr + (kk >> 2) * 1024 + (kk & 3) * 32, 2048);
-            umma_bf16(tmem_base + g * kBT, da, db, kIdescQK, kk ? 1u : 0u);
-          }
+          for (int kk = 0; kk < D / 16; ++kk)
+            umma_bf16(tmem_base + (b & 1) * kBT, dq0 + (uint64_t)((((kk >> 2) * (128 * 128)) + (kk & 3) * 32) >> 4),
+                      dk0 + (uint64_t)((((kk >> 2) * 1024) + (kk & 3) * 32) >> 4), kIdescQK, kk ? 1u : 0u);
+          umma_commit(&s_full[b & 1]);
           umma_commit(&kv_empty[s]);   // the K buffer is free once these MMAs have read it
-          umma_commit(&s_full[g]);
         };
         for (int item = item_begin; item < item_end; ++item, ++item_cnt) {
           const AttnItem w = w_next;
@@ -389,31 +391,34 @@ __global__ void __launch_bounds__(kThreads, 1) attention_tc_kernel(const __grid_
           const int tok_end = min(w.blk_end * 64, w.kv_len);
           const int nblk = (tok_end - tok_begin + kBT - 1) / kBT;
           const int buf = item_cnt & 1;
-          const uint32_t q_addr = smem_base + kOffQ + buf * kQBytes;
+          const uint64_t dq0 = desc_kmajor(smem_base + kOffQ + buf * kQBytes);
           bwait(&q_full[buf], (item_cnt >> 1) & 1, DEV_TIMEOUT_FULL);
           tc_fence_after();
-          issue_qk(blk, 0, q_addr);
-          if (nblk > 1) issue_qk(blk + 1, 1, q_addr);
+          issue_qk(blk, dq0);
+          if (nblk > 1) issue_qk(blk + 1, dq0);
           for (int n = 0; n < nblk; ++n, ++blk) {
-            const int g = n & 1;
-            // O of group g (+)= P V for block n: P (bf16, two tokens per 32-bit column) is read from TMEM
-            bwait(&p_full[g], cp[g] & 1, DEV_TIMEOUT_MMA);
-            ++cp[g];
-            // the previous item's accumulators must have been read out before this item's first products overwrite them
-            if (n < 2) bwait(o_empty, (item_cnt & 1) ^ 1, DEV_TIMEOUT_MMA);
             const int s = kKStages + blk % kVStages;
-            bwait(&kv_full[s], (blk / kVStages) & 1, DEV_TIMEOUT_FULL);
-            tc_fence_after();
-            const uint32_t v_addr = smem_base + kOffKV + s * kKVStageBytes;
+            // V block: tokens [16 j, 16 j + 16) = page j: two token groups 2 KB apart, the dim halves 1 KB apart
+            const uint64_t dv0 = desc_mnmajor(smem_base + kOffKV + s * kKVStageBytes, 1024, 2048);
 #pragma unroll
-            for (int kk = 0; kk < kBT / 16; ++kk) {
-              // tokens [16 kk, 16 kk + 16) = page kk: two token groups 2 KB apart, the dim halves 1 KB apart
-              const uint64_t db = desc_mnmajor(v_addr + kk * kTileBytes, 1024, 2048);
-              umma_bf16_ts(tmem_base + kTmemO + g * D, tmem_base + g * kBT + kk * 8, db, kIdescPV, (n >= 2 || kk) ? 1u : 0u);
+            for (int g = 0; g < 2; ++g) {
+              // O of group g (+)= P V over its 64 tokens of stage n: P (bf16, two tokens per 32-bit column) from TMEM
+              bwait(&p_full[2 * g + (blk & 1)], (blk >> 1) & 1, DEV_TIMEOUT_MMA);
+              if (g == 0) {
+                // the previous item's accumulators must have been read out before this item's products overwrite them
+                if (n == 0) bwait(o_empty, (item_cnt & 1) ^ 1, DEV_TIMEOUT_MMA);
+                bwait(&kv_full[s], (blk / kVStages) & 1, DEV_TIMEOUT_FULL);
+              }
+              tc_fence_after();
+#pragma unroll
+              for (int kk = 0; kk < 4; ++kk)
+                umma_bf16_ts(tmem_base + kTmemO + g * D, tmem_base + (blk & 1) * kBT + g * 64 + kk * 8,
+                             dv0 + (uint64_t)(((4 * g + kk) * kTileBytes) >> 4), kIdescPV, (n | kk) ? 1u : 0u);
             }
+            umma_commit(pv_done);
             umma_commit(&kv_empty[s]);
-            if (n + 2 >= nblk) umma_commit(&o_full[g]);   // the last block of this group in the item
-            if (n + 2 < nblk) issue_qk(blk + 2, g, q_addr);
+            if (n == nblk - 1) umma_commit(o_full);
+            if (n + 2 < nblk) issue_qk(blk + 2, dq0);
           }
         }
       }
@@ -421,12 +426,12 @@ __global__ void __launch_bounds__(kThreads, 1) attention_tc_kernel(const __grid_
   } else {
     reg_inc<216>();
     // ------------------------------------ softmax ------------------------------------
-    const int g = (warp - 4) >> 2;             // softmax group: takes blocks n = g, g + 2, ... of every item
+    const int g = (warp - 4) >> 2;             // softmax group: takes tokens [64 g, 64 g + 64) of every stage
     const int quad = warp & 3;
     const int row = quad * 32 + lane;          // query row of the tile = TMEM lane
     const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
-    const uint32_t s_addr = lane_addr + g * kBT, o_addr = lane_addr + kTmemO + g * D;
-    uint32_t cs = 0, item_cnt = 0, o1_cnt = 0;   // blocks this group has taken; items; items with two or more blocks
+    const uint32_t s_addr = lane_addr + g * 64, o_addr = lane_addr + kTmemO + g * D;
+    uint32_t cs = 0, item_cnt = 0;   // stages and items so far
     // visibility triple of this thread's row, fetched one item ahead
     auto row_vis = [&](const AttnItem& it, int& cl, int& lo, int& hi) {
       cl = -1; lo = 0; hi = 0;
@@ -452,54 +457,56 @@ __global__ void __launch_bounds__(kThreads, 1) attention_tc_kernel(const __grid_
       float m_ref = -1e30f, l_run = 0.f;
       bool first = true;
 
-      for (int n = g; n < nblk; n += 2, ++cs) {
-        bwait(&s_full[g], cs & 1, DEV_TIMEOUT_MMA);
+      for (int n = 0; n < nblk; ++n, ++cs) {
+        // this group's 64 tokens of stage n: S buffer cs & 1 (cs = running stage count, the same in every role)
+        const uint32_t s_buf = s_addr + (cs & 1) * kBT;
+        bwait(&s_full[cs & 1], (cs >> 1) & 1, DEV_TIMEOUT_MMA);
         tc_fence_after();
-        const int pos0 = tok_begin + n * kBT;
-        uint32_t sr[4][32];   // the S row of this thread: 128 scores
+        const int pos0 = tok_begin + n * kBT + g * 64;
+        uint32_t sr[2][32];   // the S row of this thread: 64 scores
         float mx = -INFINITY;
         if (warp_valid) {
 #pragma unroll
-          for (int c = 0; c < 4; ++c) tmem_ld32_nowait(s_addr + c * 32, sr[c]);
+          for (int c = 0; c < 2; ++c) tmem_ld32_nowait(s_buf + c * 32, sr[c]);
           tmem_ld_wait();
           const int lim = min(climit, tok_end - 1);
-          const bool need_mask = __any_sync(0xffffffffu, rvalid && (pos0 + kBT - 1 > lim));
+          const bool need_mask = __any_sync(0xffffffffu, rvalid && (pos0 + 63 > lim));
           if (need_mask) {
-            // visible tokens of this row within the block: [0, a] and [b, c), as a 128-bit mask over tokens
+            // visible tokens of this row within the 64: [0, a] and [b, c), as a 64-bit mask over tokens
             const int a = lim - pos0, b = vlo - pos0, cc = min(vhi, tok_end) - pos0;
             auto ones = [](int n) -> unsigned long long {      // n lowest bits set, n clamped to [0, 64]
               return n <= 0 ? 0ull : (n >= 64 ? ~0ull : ((1ull << n) - 1ull));
             };
             const unsigned long long m0 = ones(a + 1) | (ones(cc) & ~ones(b));
-            const unsigned long long m1 = ones(a + 1 - 64) | (ones(cc - 64) & ~ones(b - 64));
 #pragma unroll
-            for (int c = 0; c < 4; ++c)
+            for (int c = 0; c < 2; ++c)
 #pragma unroll
               for (int i = 0; i < 32; ++i) {
                 const int t = col_token(c * 32 + i);        // compile-time constant after unrolling
-                const bool vis = ((t < 64 ? (m0 >> t) : (m1 >> (t - 64))) & 1ull) != 0ull;
-                if (!vis) sr[c][i] = 0xff800000u;   // -inf
+                if (((m0 >> t) & 1ull) == 0ull) sr[c][i] = 0xff800000u;   // -inf
               }
           }
-          {  // four independent chains instead of one 128-long dependent one
+          {  // four independent chains instead of one long dependent one
             float mxa[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-            for (int c = 0; c < 4; ++c)
+            for (int c = 0; c < 2; ++c)
 #pragma unroll
-              for (int i = 0; i < 32; i += 2)
-                mxa[c] = fmaxf(mxa[c], fmaxf(__uint_as_float(sr[c][i]), __uint_as_float(sr[c][i + 1])));
+              for (int i = 0; i < 32; i += 4) {
+                mxa[2 * c] = fmaxf(mxa[2 * c], fmaxf(__uint_as_float(sr[c][i]), __uint_as_float(sr[c][i + 1])));
+                mxa[2 * c + 1] = fmaxf(mxa[2 * c + 1], fmaxf(__uint_as_float(sr[c][i + 2]), __uint_as_float(sr[c][i + 3])));
+              }
             mx = fmaxf(fmaxf(mxa[0], mxa[1]), fmaxf(mxa[2], mxa[3]));
           }
-          // This S was produced after the group's previous P V in tensor-pipe order, so that product is complete:
-          // O may be rescaled and the P columns rewritten.
           const float m_blk = mx * P.scale_log2;
           // move the reference maximum only when the row maximum outgrows it by more than 2^8 (or at the first
-          // block): probabilities stay below 256 relative to the reference, well inside bf16 and fp32 range
+          // stage): probabilities stay below 256 relative to the reference, well inside bf16 and fp32 range
           const bool grow = rvalid && (m_blk > m_ref + 8.f);
-          if (n == g) {
+          if (n == 0) {
             if (rvalid && m_blk > m_ref) m_ref = m_blk;
           } else if (__any_sync(0xffffffffu, grow)) {
-            // rare: O is rescaled in TMEM
+            // rare: O is rescaled in TMEM, once the group's P V of the previous stage has completed
+            bwait(pv_done, (cs - 1) & 1, DEV_TIMEOUT_MMA);
+            tc_fence_after();
             const float m_new = grow ? m_blk : m_ref;
             const float f = exp2f(m_ref - m_new);
             m_ref = m_new;
@@ -516,43 +523,34 @@ __global__ void __launch_bounds__(kThreads, 1) attention_tc_kernel(const __grid_
             tmem_st_wait();
           }
           float lsa[4] = {0.f, 0.f, 0.f, 0.f};
+          uint32_t pk[32];     // 64 tokens -> 32 packed columns over the start of this S buffer
 #pragma unroll
-          for (int h = 0; h < 2; ++h) {      // 64 tokens -> 32 packed columns [32 h, 32 h + 32) of this group's S buffer
-            uint32_t pk[32];
+          for (int c = 0; c < 2; ++c) {
 #pragma unroll
-            for (int cc = 0; cc < 2; ++cc) {
-              const int c = 2 * h + cc;
-#pragma unroll
-              for (int i = 0; i < 32; i += 2) {
-                const float p0 = exp2f(__uint_as_float(sr[c][i]) * P.scale_log2 - m_ref);   // exp2(-inf) = 0 for masked
-                const float p1 = exp2f(__uint_as_float(sr[c][i + 1]) * P.scale_log2 - m_ref);
-                lsa[(i >> 1) & 3] += p0 + p1;
-                pk[cc * 16 + (i >> 1)] = pack_bf16(p0, p1);
-              }
+            for (int i = 0; i < 32; i += 2) {
+              const float p0 = exp2f(__uint_as_float(sr[c][i]) * P.scale_log2 - m_ref);   // exp2(-inf) = 0 for masked
+              const float p1 = exp2f(__uint_as_float(sr[c][i + 1]) * P.scale_log2 - m_ref);
+              lsa[(i >> 1) & 3] += p0 + p1;
+              pk[c * 16 + (i >> 1)] = pack_bf16(p0, p1);
             }
-            tmem_st32(s_addr + h * 32, pk);
           }
+          tmem_st32(s_buf, pk);
           l_run += (lsa[0] + lsa[1]) + (lsa[2] + lsa[3]);
           tmem_st_wait();
         }
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(&p_full[g]);
+        if (lane == 0) mbar_arrive(&p_full[2 * g + (cs & 1)]);
         if (first) {      // the next item's descriptor has arrived by now: fetch its rows' visibility for later
           first = false;
           if (item + 1 < item_end) row_vis(w_next, nx_cl, nx_lo, nx_hi);
         }
       }
-      if (first && item + 1 < item_end) row_vis(w_next, nx_cl, nx_lo, nx_hi);   // this group had no block in the item
 
       // ---- merge the two groups' partial attentions and write out: this group finishes dims [64 g, 64 g + 64) ----
-      const bool two = nblk >= 2;                 // group 1 took part in this item
+      const bool two = true;                      // both groups take part in every stage
       const int buf = item_cnt & 1;
-      bwait(&o_full[0], item_cnt & 1, DEV_TIMEOUT_MMA);
-      if (two) {
-        bwait(&o_full[1], o1_cnt & 1, DEV_TIMEOUT_MMA);
-        ++o1_cnt;
-      }
+      bwait(o_full, item_cnt & 1, DEV_TIMEOUT_MMA);
       tc_fence_after();
       ml_smem[g * 128 + row] = make_float2(m_ref, l_run);
       softmax_bar();
