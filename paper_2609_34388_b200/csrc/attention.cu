@@ -73,14 +73,18 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attention_kernel(AttnParams P
   __syncthreads();
   griddep_wait();
 
-  const int item_begin = P.cta_off[blockIdx.x], item_end = P.cta_off[blockIdx.x + 1];
+  // the CTA walks two ranges of the item list one after the other (see the layout kernel)
+  const int4 r4 = *reinterpret_cast<const int4*>(P.cta_off + 4 * blockIdx.x);
+  const int range_n0 = r4.y - r4.x;
+  const int item_begin = 0, item_end = range_n0 + (r4.w - r4.z);
+  auto item_at = [&](int i) { return i < range_n0 ? r4.x + i : r4.z + (i - range_n0); };
   uint32_t it = 0;  // running block counter, identical in producer and consumers
   bool aborted = false;
 
   if (warp == kConsumerWarps) {
     // ------------------------------ producer ------------------------------
     for (int item = item_begin; item < item_end && !aborted; ++item) {
-      const AttnItem w = P.items[item];
+      const AttnItem w = P.items[item_at(item)];
       const int n_req_pages = (w.kv_len + kPageSize - 1) / kPageSize;
       const int* pt = P.page_table + (size_t)w.req * P.pt_stride;
       // lanes 0..3 each own one page of the block; ids are fetched one block ahead of their use
@@ -136,7 +140,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attention_kernel(AttnParams P
   const uint32_t ring = smem_u32(smem);
 
   for (int item = item_begin; item < item_end; ++item) {
-    const AttnItem w = P.items[item];
+    const AttnItem w = P.items[item_at(item)];
     const int R = w.ntok * P.group;
     const int RW = (R + 15) >> 4;
     const int KW = RW == 1 ? 8 : (RW == 2 ? 4 : (RW <= 4 ? 2 : 1));

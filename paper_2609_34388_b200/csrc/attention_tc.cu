@@ -13,23 +13,25 @@
 //             query heads x 128 / group tokens, 128-byte swizzle) into one of two Q buffers, so the Q of the
 //             next item is in place before the current item ends.
 //   warp 1    one elected lane issues tcgen05.mma: S = Q K^T (M 128 rows, N 128 tokens, K = d, both operands
-//             in shared memory) and O += P V (P read from TMEM, V from shared memory; N = d, K = 128 tokens).
-//             It runs ahead into the next item (its first S tiles) while the softmax groups still write
-//             the previous item's output.
-//   warps 4-7 and 8-11: two softmax groups.  The KV blocks of an item alternate between them (block n goes
-//             to group n & 1); each group has its own S buffer and O accumulator in TMEM and its own running
-//             (reference maximum, sum), i.e. the two groups are two independent partial attentions over
-//             the even and the odd blocks, merged once at the end of the item.  While one group is in its
-//             exp2 phase the other one reads S or waits for the tensor core.  Within a group ONE THREAD OWNS
-//             ONE QUERY ROW (= TMEM lane): the S row is read from TMEM once, probabilities are taken relative
-//             to a reference maximum that is only moved (and O rescaled in TMEM) when the row maximum
-//             outgrows it by more than 2^8, and bf16 P is written back over the first 64 columns of the same
-//             S buffer (two tokens per 32-bit column), from where the P V product reads it.  The tensor pipe
-//             executes in issue order, so the next S of a group is produced after its P has been consumed.
-//             No cross-thread reductions are needed.  At the end of an item group 0 finishes output dims
-//             [0,64) and group 1 dims [64,128) of every row from both accumulators; partial results (items
-//             that cover part of the KV range) go through a per-warp transposition in the item's Q buffer
-//             so that every global store is a full 128-byte line.
+//             in shared memory) into one of two S buffers in TMEM (stage & 1), and per softmax group
+//             O_g += P_g V_g (P read from TMEM, V from shared memory; N = d, K = the group's 64 tokens).  It runs
+//             two stages ahead with S and into the next item while the softmax groups still write the previous
+//             item's output.  Its per-instruction cost matters (it was the bottleneck once): descriptors are a
+//             base plus constants, one product and one barrier per stage serve both groups.
+//   warps 4-7 and 8-11: two softmax groups.  Group g takes tokens [64 g, 64 g + 64) of EVERY 128-token stage; it
+//             has its own O accumulator in TMEM and its own running (reference maximum, sum), i.e. the two
+//             groups are two independent partial attentions over interleaved 64-token chunks, merged once at
+//             the end of the item.  Within a group ONE THREAD OWNS ONE QUERY ROW (= TMEM lane): its 64 scores
+//             are read from TMEM once, probabilities are taken relative to a reference maximum that is only
+//             moved (and O rescaled in TMEM) when the row maximum outgrows it by more than 2^8, and bf16 P is
+//             written back over the first 32 of the group's 64 columns of the same S buffer (two tokens per
+//             32-bit column), from where the P V product reads it.  Because S is double buffered, the S of
+//             the next stage is already there when a group finishes a stage; the tensor pipe executes in issue
+//             order, so a buffer's next S is produced after its P has been consumed.  No cross-thread
+//             reductions are needed.  At the end of an item group 0 finishes output dims [0,64) and group 1
+//             dims [64,128) of every row from both accumulators; partial results (items that cover part of
+//             the KV range) go through a per-warp transposition in the item's Q buffer so that every global
+//             store is a full 128-byte line.
 //   Warpgroup 0 gives registers back (setmaxnreg) so that a softmax thread can hold a whole S row.
 // Only blocks that reach past a row's visibility limit evaluate the mask.  Every wait is bounded; a wait that
 // runs out raises a CTA-wide flag after which no wait blocks, so the kernel always ends.
@@ -67,7 +69,7 @@ constexpr int kOffKV = kOffQ + 2 * kQBytes;
 constexpr int kOffML = kOffKV + kKVStages * kKVStageBytes;   // float2 [2 groups][128 rows]: (reference max, sum)
 constexpr int kOffBar = kOffML + 2 * 128 * 8;
 constexpr int kNumBars = 2 * kKVStages + 2 + 2 + 2 + 4 + 1 + 1 + 1;
-constexpr int kSmemBytes = kOffBar + kNumBars * 8 + 16 + 32;   // barriers, TMEM slot + flags + item range, first item
+constexpr int kSmemBytes = kOffBar + kNumBars * 8 + 64;   // barriers, TMEM slot + flag, item ranges, first item
 static_assert(kSmemBytes <= 227 * 1024, "shared memory budget");
 
 struct TcAttnParams {
@@ -215,17 +217,27 @@ __global__ void __launch_bounds__(kThreads, 1) attention_tc_kernel(const __grid_
   // Warp 0 waits for the kernels before this one and fetches the CTA's item range and first item while the other
   // warps set up barriers, the zeroed ring and TMEM: two dependent round trips off everybody's critical path.
   int* s_range = reinterpret_cast<int*>(tmem_slot + 2);
-  AttnItem* s_first = reinterpret_cast<AttnItem*>(tmem_slot + 4);
-  int item_begin = 0, item_end = 0;
+  AttnItem* s_first = reinterpret_cast<AttnItem*>(tmem_slot + 6);
+  // the CTA walks two ranges of the item list one after the other (see the layout kernel): logical item i is
+  // entry b0 + i for i < n0 and entry b1 + (i - n0) after that
+  int range_b0 = 0, range_n0 = 0, range_b1 = 0;
+  const int item_begin = 0;
+  int item_end = 0;
+  auto item_at = [&](int i) { return i < range_n0 ? range_b0 + i : range_b1 + (i - range_n0); };
   AttnItem w_next = {};
   if (warp == 0) {
     griddep_wait();
-    item_begin = P.cta_off[blockIdx.x];
-    item_end = P.cta_off[blockIdx.x + 1];
-    if (item_begin < item_end) w_next = P.items[item_begin];
+    const int4 r4 = *reinterpret_cast<const int4*>(P.cta_off + 4 * blockIdx.x);
+    range_b0 = r4.x;
+    range_n0 = r4.y - r4.x;
+    range_b1 = r4.z;
+    item_end = range_n0 + (r4.w - r4.z);
+    if (item_begin < item_end) w_next = P.items[item_at(0)];
     if (lane == 0) {
-      s_range[0] = item_begin;
-      s_range[1] = item_end;
+      s_range[0] = range_b0;
+      s_range[1] = range_n0;
+      s_range[2] = range_b1;
+      s_range[3] = item_end;
       *s_first = w_next;
     }
   }
@@ -263,8 +275,10 @@ __global__ void __launch_bounds__(kThreads, 1) attention_tc_kernel(const __grid_
   const uint32_t tmem_base = *tmem_slot;
   if (warp != 0) {
     griddep_wait();   // these warps touched only shared memory and TMEM so far
-    item_begin = s_range[0];
-    item_end = s_range[1];
+    range_b0 = s_range[0];
+    range_n0 = s_range[1];
+    range_b1 = s_range[2];
+    item_end = s_range[3];
     w_next = *s_first;
   }
   const uint32_t smem_base = smem_u32(smem);
@@ -277,7 +291,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_tc_kernel(const __grid_
       uint32_t blk = 0, item_cnt = 0;  // running KV-block and item counters
       for (int item = item_begin; item < item_end; ++item, ++item_cnt) {
         const AttnItem w = w_next;
-        if (item + 1 < item_end) w_next = P.items[item + 1];
+        if (item + 1 < item_end) w_next = P.items[item_at(item + 1)];
         const int tok_begin = w.blk_begin * 64;
         const int tok_end = min(w.blk_end * 64, w.kv_len);
         const int nblk = (tok_end - tok_begin + kBT - 1) / kBT;
@@ -386,7 +400,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_tc_kernel(const __grid_
         };
         for (int item = item_begin; item < item_end; ++item, ++item_cnt) {
           const AttnItem w = w_next;
-          if (item + 1 < item_end) w_next = P.items[item + 1];
+          if (item + 1 < item_end) w_next = P.items[item_at(item + 1)];
           const int tok_begin = w.blk_begin * 64;
           const int tok_end = min(w.blk_end * 64, w.kv_len);
           const int nblk = (tok_end - tok_begin + kBT - 1) / kBT;
@@ -446,7 +460,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_tc_kernel(const __grid_
     if (item_begin < item_end) row_vis(w_next, nx_cl, nx_lo, nx_hi);
     for (int item = item_begin; item < item_end; ++item) {
       const AttnItem w = w_next;
-      if (item + 1 < item_end) w_next = P.items[item + 1];
+      if (item + 1 < item_end) w_next = P.items[item_at(item + 1)];
       const int R = w.ntok * P.group;
       const int tok_begin = w.blk_begin * 64;
       const int tok_end = min(w.blk_end * 64, w.kv_len);

@@ -46,9 +46,9 @@ struct BatchLayout {
   AttnItem* items;
   AttnTile* tiles;
   int* tile_off;    // [C+1] first tile entry of each request
-  int* cta_off;     // [n_ctas+1] first item of each CTA of the persistent attention grid
+  int* cta_off;     // [4 n_ctas] per CTA of the persistent attention grid: the two item index ranges [b0, e0), [b1, e1) it walks
   int* item_cta;    // [max_items] owning CTA of each item (scratch of the layout kernel)
-  int* counts;      // [0] number of items, [1] number of tiles, [2] blocks per CTA
+  int* counts;      // [0] number of items, [1] number of tiles, [2], [3] cost units per CTA / per CTA pair
   int max_items, max_parts;
 };
 

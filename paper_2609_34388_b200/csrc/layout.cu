@@ -16,25 +16,38 @@ __device__ __forceinline__ int upper_request(const int* cu, int n_req, int t) {
   return lo;
 }
 
-// One CTA.  Shared: 5 arrays of n_req+1 ints.
+// One CTA.  Shared: 8 arrays of n_req+1 ints, then n_ctas/2 + 1 and n_ctas + 1 ints.
 //
-// Attention work list: the 64-token KV blocks of all (request, kv head, row tile) tiles form one line; every
-// tile is preceded by kItemCost virtual blocks that stand for the fixed cost of starting an item (staging Q,
-// refilling and draining the pipeline).  The line of W cost units is cut into n_ctas equal contiguous ranges,
-// one per CTA of the persistent attention grid, and additionally at every tile boundary.  Each piece that holds
-// real blocks is an item; a tile whose blocks are cut by CTA boundaries gets one partial slot per piece.
+// Attention work list.  A request with n new tokens has ceil(n / tok_per_tile) row tiles per kv head.  Row tiles
+// 2 j and 2 j + 1 of a kv head are "siblings": they read the same K/V.  Two lines of 64-token KV blocks are built,
+// every tile preceded by kItemCost virtual blocks that stand for the fixed cost of starting an item (fetching Q,
+// refilling and draining the pipeline):
+//   line A holds one segment per sibling PAIR and is cut into n_ctas / 2 equal contiguous ranges, one per pair of
+//          CTAs (2 p, 2 p + 1): the even CTA works on the first sibling and the odd CTA on the second sibling of the
+//          SAME block ranges, at the same time, so that the second reader of a K/V block finds it in L2;
+//   line B holds the tiles without a sibling and is cut into n_ctas equal ranges, one per CTA.
+// Every CTA first walks its range of line A, then its range of line B; all CTAs carry the same load.  Each piece
+// that holds real blocks is an item; a tile whose blocks are cut by range boundaries gets one partial slot per piece.
+// Items: [line A, first siblings | line A, second siblings (same order) | line B]; cta_off holds, per CTA, the
+// two index ranges it walks.
 constexpr int kItemCost = 3;
 
 __global__ void __launch_bounds__(1024) layout_kernel(BatchLayout bl, int n_kv, int mask_id, int tok_per_tile,
                                                       int n_ctas, int64_t n_pages, int* status) {
   extern __shared__ int sm[];
   const int C = bl.n_req;
-  int* req_blk_off = sm;                 // first global block of request r
-  int* tile_off = sm + (C + 1);          // first tile entry of request r
-  int* item_off = sm + 2 * (C + 1);      // first item of request r
-  int* part_off = sm + 3 * (C + 1);      // first partial slot of request r
-  int* req_nb = sm + 4 * (C + 1);        // blocks per tile of request r
-  __shared__ int s_per, s_total_blocks;
+  const int n_pairs = n_ctas / 2;
+  int* off_a = sm;                       // first cost unit of request r in line A
+  int* off_b = sm + (C + 1);             // ... in line B
+  int* tile_off = sm + 2 * (C + 1);      // first tile entry of request r
+  int* item_a = sm + 3 * (C + 1);        // first line-A piece of request r
+  int* item_b = sm + 4 * (C + 1);        // first line-B piece of request r
+  int* part_off = sm + 5 * (C + 1);      // first partial slot of request r
+  int* req_nb = sm + 6 * (C + 1);        // blocks per tile of request r
+  int* req_rt = sm + 7 * (C + 1);        // row tiles per kv head of request r
+  int* a_off = sm + 8 * (C + 1);         // [n_pairs + 1] first line-A piece of every CTA pair
+  int* b_off = a_off + (n_pairs + 1);    // [n_ctas + 1]  first line-B piece of every CTA
+  __shared__ int s_per_a, s_per_b;
   const int tid = threadIdx.x, nth = blockDim.x;
   griddep_launch();
   griddep_wait();   // the previous step's kernels may still be reading the arrays this kernel rewrites
@@ -65,102 +78,149 @@ __global__ void __launch_bounds__(1024) layout_kernel(BatchLayout bl, int n_kv, 
   for (int r = tid; r < C; r += nth) {
     const int n = bl.verify_len[r] + bl.block_size[r];
     req_nb[r] = (bl.ctx_len[r] + n + 63) / 64;
-    tile_off[r + 1] = n_kv * ((n + tok_per_tile - 1) / tok_per_tile);
+    req_rt[r] = (n + tok_per_tile - 1) / tok_per_tile;
   }
   __syncthreads();
   if (tid == 0) {
-    req_blk_off[0] = 0;
-    tile_off[0] = 0;
-    long long w = 0;
+    off_a[0] = off_b[0] = tile_off[0] = 0;
+    long long wa = 0, wb = 0;
     for (int r = 0; r < C; ++r) {
-      w += (long long)tile_off[r + 1] * (req_nb[r] + kItemCost);
-      if (w > 0x3fffffff) w = 0x3fffffff;   // far beyond any pool; keeps the arithmetic in int
-      req_blk_off[r + 1] = (int)w;
-      tile_off[r + 1] += tile_off[r];
+      const int rt = req_rt[r], seg = req_nb[r] + kItemCost;
+      wa += (long long)n_kv * (rt / 2) * seg;
+      wb += (long long)n_kv * (rt & 1) * seg;
+      if (wa > 0x3fffffff) wa = 0x3fffffff;   // far beyond any pool; keeps the arithmetic in int
+      if (wb > 0x3fffffff) wb = 0x3fffffff;
+      off_a[r + 1] = (int)wa;
+      off_b[r + 1] = (int)wb;
+      tile_off[r + 1] = tile_off[r] + n_kv * rt;
     }
-    s_total_blocks = (int)w;
-    const int per = (int)((w + n_ctas - 1) / n_ctas);
-    s_per = per < 1 ? 1 : per;
+    const int pa = n_pairs > 0 ? (int)((wa + n_pairs - 1) / n_pairs) : 0x3fffffff;
+    const int pb = (int)((wb + n_ctas - 1) / n_ctas);
+    s_per_a = pa < 1 ? 1 : pa;
+    s_per_b = pb < 1 ? 1 : pb;
   }
   __syncthreads();
-  const int per = s_per, W = s_total_blocks;
+  const int per_a = s_per_a, per_b = s_per_b;
+  // pieces of a segment whose real blocks occupy the cost range [g0, g0 + nb)
+  auto n_pieces = [](int g0, int nb, int per) { return (g0 + nb - 1) / per - g0 / per + 1; };
   for (int r = tid; r < C; r += nth) {
-    const int nb = req_nb[r], nt = tile_off[r + 1] - tile_off[r];
-    int items = 0, parts_split = 0;
-    for (int k = 0; k < nt; ++k) {
-      const int g0 = req_blk_off[r] + k * (nb + kItemCost) + kItemCost, g1 = g0 + nb;   // cost range of the real blocks
-      const int parts = (g1 - 1) / per - g0 / per + 1;
-      items += parts;
-      if (parts > 1) parts_split += parts;
+    const int nb = req_nb[r], rt = req_rt[r], seg = nb + kItemCost;
+    int ia = 0, ib = 0, parts = 0;
+    for (int kvh = 0; kvh < n_kv; ++kvh) {
+      for (int j = 0; j < rt / 2; ++j) {
+        const int np = n_pieces(off_a[r] + (kvh * (rt / 2) + j) * seg + kItemCost, nb, per_a);
+        ia += np;
+        if (np > 1) parts += 2 * np;
+      }
+      if (rt & 1) {
+        const int np = n_pieces(off_b[r] + kvh * seg + kItemCost, nb, per_b);
+        ib += np;
+        if (np > 1) parts += np;
+      }
     }
-    item_off[r + 1] = items;
-    part_off[r + 1] = parts_split;
+    item_a[r + 1] = ia;
+    item_b[r + 1] = ib;
+    part_off[r + 1] = parts;
   }
   __syncthreads();
   if (tid == 0) {
-    item_off[0] = part_off[0] = 0;
+    item_a[0] = item_b[0] = part_off[0] = 0;
     for (int r = 0; r < C; ++r) {
-      item_off[r + 1] += item_off[r];
+      item_a[r + 1] += item_a[r];
+      item_b[r + 1] += item_b[r];
       part_off[r + 1] += part_off[r];
     }
-    int n_items = item_off[C];
+    int n_items = 2 * item_a[C] + item_b[C];
     if (n_items > bl.max_items || part_off[C] > bl.max_parts) {
       set_status(status, DEV_BAD_INDEX);
       n_items = 0;
     }
     bl.counts[0] = n_items;
     bl.counts[1] = tile_off[C];
-    bl.counts[2] = per;
+    bl.counts[2] = per_b;
+    bl.counts[3] = per_a;
   }
   __syncthreads();
   const int n_items = bl.counts[0];
+  const int na = n_items ? item_a[C] : 0, n_b = n_items ? item_b[C] : 0;
   for (int r = tid; r <= C; r += nth) bl.tile_off[r] = tile_off[r];
-  for (int c = tid; c <= n_ctas; c += nth)
-    bl.cta_off[c] = -1;                                                      // filled below
-  if (n_items == 0) return;
-  for (int r = tid; r < C; r += nth) {
-    const int n = bl.verify_len[r] + bl.block_size[r];
-    const int kv_len = bl.ctx_len[r] + n;
-    const int nb = req_nb[r], nt = tile_off[r + 1] - tile_off[r];
-    const int tiles = nt / n_kv;
-    int item = item_off[r], part = part_off[r];
-    for (int k = 0; k < nt; ++k) {
-      const int kvh = k / tiles, tile = k % tiles;
-      const int g0 = req_blk_off[r] + k * (nb + kItemCost) + kItemCost, g1 = g0 + nb;
-      const int c_first = g0 / per, c_last = (g1 - 1) / per;
-      const int parts = c_last - c_first + 1;
-      AttnTile tl;
-      tl.part_begin = parts > 1 ? part : -1;
-      tl.n_parts = parts;
-      tl.tok0 = bl.cu_tok[r] + tile * tok_per_tile;
-      tl.ntok = min(tok_per_tile, n - tile * tok_per_tile);
-      tl.kv_head = kvh;
-      bl.tiles[tile_off[r] + k] = tl;
-      for (int c = c_first; c <= c_last; ++c, ++item) {
-        const int gs = max(g0, c * per), ge = min(g1, (c + 1) * per);
-        AttnItem a;
-        a.req = r;
-        a.kv_head = kvh;
-        a.tok0 = tl.tok0;
-        a.ntok = tl.ntok;
-        a.blk_begin = gs - g0;
-        a.blk_end = ge - g0;
-        a.part = parts > 1 ? part++ : -1;
-        a.kv_len = kv_len;
-        bl.items[item] = a;
-        bl.item_cta[item] = c;
+  for (int p = tid; p <= n_pairs; p += nth) a_off[p] = na;     // pairs after the last owner; the rest is filled below
+  for (int c = tid; c <= n_ctas; c += nth) b_off[c] = n_b;
+  __syncthreads();
+  if (n_items) {
+    for (int r = tid; r < C; r += nth) {
+      const int n = bl.verify_len[r] + bl.block_size[r];
+      const int kv_len = bl.ctx_len[r] + n;
+      const int nb = req_nb[r], rt = req_rt[r], seg = nb + kItemCost;
+      int ia = item_a[r], ib = item_b[r], part = part_off[r];
+      // one tile's entry, and its items on one line: pieces [c_first, c_last] of the cost range [g0, g0 + nb)
+      auto emit = [&](int kvh, int tile, int g0, int per, int item0, int* owner, int owner_base) {
+        const int c_first = g0 / per, c_last = (g0 + nb - 1) / per;
+        const int parts = c_last - c_first + 1;
+        AttnTile tl;
+        tl.part_begin = parts > 1 ? part : -1;
+        tl.n_parts = parts;
+        tl.tok0 = bl.cu_tok[r] + tile * tok_per_tile;
+        tl.ntok = min(tok_per_tile, n - tile * tok_per_tile);
+        tl.kv_head = kvh;
+        bl.tiles[tile_off[r] + kvh * rt + tile] = tl;
+        for (int c = c_first; c <= c_last; ++c) {
+          const int gs = max(g0, c * per), ge = min(g0 + nb, (c + 1) * per);
+          AttnItem a;
+          a.req = r;
+          a.kv_head = kvh;
+          a.tok0 = tl.tok0;
+          a.ntok = tl.ntok;
+          a.blk_begin = gs - g0;
+          a.blk_end = ge - g0;
+          a.part = parts > 1 ? part++ : -1;
+          a.kv_len = kv_len;
+          bl.items[item0 + (c - c_first)] = a;
+          if (owner) owner[owner_base + (c - c_first)] = c;
+        }
+        return parts;
+      };
+      for (int kvh = 0; kvh < n_kv; ++kvh) {
+        for (int j = 0; j < rt / 2; ++j) {
+          const int g0 = off_a[r] + (kvh * (rt / 2) + j) * seg + kItemCost;
+          const int np = emit(kvh, 2 * j, g0, per_a, ia, bl.item_cta, ia);       // first sibling: even CTA of the pair
+          emit(kvh, 2 * j + 1, g0, per_a, na + ia, nullptr, 0);                  // second sibling: odd CTA, same ranges
+          ia += np;
+        }
+        if (rt & 1) {
+          const int g0 = off_b[r] + kvh * seg + kItemCost;
+          ib += emit(kvh, rt - 1, g0, per_b, 2 * na + ib, bl.item_cta, 2 * na + ib);
+        }
       }
     }
+    // first piece of every owner: pieces are in line order, so an owner's range starts where the owner changes
+    __syncthreads();
+    for (int it = tid; it < na; it += nth) {
+      const int p = bl.item_cta[it];
+      const int prev = it ? bl.item_cta[it - 1] : -1;
+      for (int pp = prev + 1; pp <= p && pp <= n_pairs; ++pp) a_off[pp] = it;   // pairs between two owners have no items
+    }
+    for (int it = tid; it < n_b; it += nth) {
+      const int c = bl.item_cta[2 * na + it];
+      const int prev = it ? bl.item_cta[2 * na + it - 1] : -1;
+      for (int cc = prev + 1; cc <= c && cc <= n_ctas; ++cc) b_off[cc] = it;
+    }
   }
-  // first item of every CTA: items are ordered by CTA, so a CTA's range starts where the owner changes
   __syncthreads();
-  for (int it = tid; it < n_items; it += nth) {
-    const int c = bl.item_cta[it];
-    const int prev = it ? bl.item_cta[it - 1] : -1;
-    for (int cc = prev + 1; cc <= c; ++cc) bl.cta_off[cc] = it;   // CTAs between two owners have no items
+  // the two ranges of item indices every CTA walks: its pair's pieces of line A (first or second siblings), then its own
+  // pieces of line B
+  for (int c = tid; c < n_ctas; c += nth) {
+    const int p = c >> 1;
+    int a0 = 0, a1 = 0;
+    if (p < n_pairs) {
+      a0 = ((c & 1) ? na : 0) + a_off[p];
+      a1 = ((c & 1) ? na : 0) + a_off[p + 1];
+    }
+    bl.cta_off[4 * c + 0] = a0;
+    bl.cta_off[4 * c + 1] = a1;
+    bl.cta_off[4 * c + 2] = 2 * na + b_off[c];
+    bl.cta_off[4 * c + 3] = 2 * na + b_off[c + 1];
   }
-  const int last_owner = bl.item_cta[n_items - 1];
-  for (int c = last_owner + 1 + tid; c <= n_ctas; c += nth) bl.cta_off[c] = n_items;
 }
 
 __global__ void embed_kernel(const int* __restrict__ tok_id, const __nv_bfloat16* __restrict__ embed,
@@ -262,7 +322,7 @@ __global__ void kv_io_kernel(bool write, __nv_bfloat16* pool, int64_t n_pages, i
 
 void launch_layout(const BatchLayout& bl, const Dims& dm, int tok_per_tile, int n_ctas, int64_t n_pages,
                    int* status, cudaStream_t st) {
-  const size_t smem = 5 * (size_t)(bl.n_req + 1) * sizeof(int);
+  const size_t smem = (8 * (size_t)(bl.n_req + 1) + (size_t)(n_ctas / 2 + 1) + (size_t)(n_ctas + 1)) * sizeof(int);
   launch_pdl(layout_kernel, dim3(1), dim3(1024), smem, st, bl, dm.n_kv, dm.mask_id, tok_per_tile, n_ctas, n_pages, status);
 }
 

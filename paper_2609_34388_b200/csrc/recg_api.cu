@@ -110,13 +110,13 @@ size_t carve(recg_ctx* c, DeviceArena& A) {
   bl.tok_lo = A.take<int>(Tm);
   bl.tok_hi = A.take<int>(Tm);
   const size_t max_tiles = (size_t)d.n_kv * (Cm + Tm / c->tok_per_tile + 1);
-  bl.max_parts = 2 * c->target_items;
-  bl.max_items = (int)(2 * c->target_items + max_tiles);
+  bl.max_parts = 4 * c->target_items;      // two lines of work, each cut at fewer than target_items places (see layout.cu)
+  bl.max_items = (int)(4 * c->target_items + max_tiles);
   bl.items = A.take<AttnItem>(bl.max_items);
   bl.item_cta = A.take<int>(bl.max_items);
   bl.tiles = A.take<AttnTile>(max_tiles);
   bl.tile_off = A.take<int>(Cm + 1);
-  bl.cta_off = A.take<int>(c->target_items + 1);
+  bl.cta_off = A.take<int>(4 * (c->target_items + 1));
   bl.counts = A.take<int>(4);
   c->d_status = A.take<int>(1);
   c->d_page_row = A.take<int>(Pm);
