@@ -53,8 +53,8 @@ constexpr int kSubBytes = kPageSize * 128;     // 2 KB: [16 tokens][64 dims]
 constexpr int kQBytes = 128 * D * 2;           // 32 KB
 constexpr int kTileBytes = 2 * kSubBytes;        // 4 KB: the K (or V) tile of one page and head, as stored in the pool
 constexpr int kKVStageBytes = kPagesPerBT * kTileBytes;  // one operand (K or V) of a 128-token block: 32 KB
-constexpr int kKStages = 3;                      // K ring: a buffer is free after its Q K^T
-constexpr int kVStages = 2;                      // V ring: a buffer is free after its P V.  The rings are separate so that a V
+constexpr int kKStages = 2;                      // K ring: a buffer is free after its Q K^T
+constexpr int kVStages = 3;                      // V ring: a buffer is free after its P V.  The rings are separate so that a V
                                                  // buffer never holds the unsanitised rows of a partly filled K page
 constexpr int kKVStages = kKStages + kVStages;
 constexpr int kThreads = 384;                    // warpgroup 0: producer K, MMA, producer V, idle; warpgroups 1, 2: softmax
