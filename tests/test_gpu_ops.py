@@ -237,6 +237,29 @@ def test_linear(M, N, K, flags):
     ctx.recg_free()
 
 
+@pytest.mark.parametrize("force", ["512,0", "512,1", "256,1", "128,1", "64,1", "256,0"])
+def test_linear_forced_decompositions(force, monkeypatch):
+    """Every tile width and decomposition of the projection kernel on shapes that make it cut tiles: CTA pairs
+    (512 = 256-row tiles over clusters of two), stream-K with the reduction through the idle operand ring (last
+    pieces) and through global memory (pieces followed by whole tiles), ragged M, M beyond one pair tile."""
+    monkeypatch.setenv("RECG_GEMM_FORCE", force)       # read when the context is created
+    shape = synth.tiny_shape()
+    ctx = ops_ctx(shape, 1, 8, 1)
+    for (M, N, K) in [(300, 512, 1024), (130, 4096, 4096), (470, 1024, 14336), (600, 6144, 1024), (257, 28672, 512)]:
+        g = torch.Generator().manual_seed(M * 7 + N)
+        x = torch.randn((M, K), generator=g).to(torch.bfloat16)
+        w = (torch.randn((N, K), generator=g) * 0.05).to(torch.bfloat16)
+        ref = x.double().numpy() @ w.double().numpy().T
+        y = ctx.recg_linear(x.cuda(), w.cuda(), torch.float32)
+        ctx.recg_sync()
+        err = np.max(np.abs(f64(y) - ref)) / np.max(np.abs(ref))
+        assert err < 1e-4, (force, M, N, K, err)
+        y2 = ctx.recg_linear(x.cuda(), w.cuda(), torch.float32)
+        ctx.recg_sync()
+        assert torch.equal(y, y2), (force, M, N, K)        # parts are added in a fixed order
+    ctx.recg_free()
+
+
 def test_host_side_rejections():
     shape = synth.tiny_shape()
     ctx = ops_ctx(shape, 2, 16, 4)
