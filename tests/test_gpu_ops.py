@@ -78,6 +78,15 @@ def test_attention_long_context_split_and_multi_tile():
     assert run_attention_case(synth.tiny_shape(), [(2500, 40, 30), (100, 70, 0)], seed=24) < ATTN_TOL
 
 
+def test_attention_many_row_tiles_per_request():
+    """Prefill-like chunks: many row tiles per request head (sibling pairs plus a tile without a sibling), next to
+    ordinary requests, so that both lines of the work list and several items per CTA occur."""
+    shape = synth.llama8b_shape(1)
+    assert run_attention_case(shape, [(300, 200, 0), (700, 8, 8), (0, 95, 1)], seed=41) < ATTN_TOL
+    assert run_attention_case(shape, [(64, 33, 0)] * 3 + [(2000, 16, 16)], seed=42) < ATTN_TOL
+    assert run_attention_case(synth.tiny_shape(), [(100, 130, 0), (10, 3, 4)], seed=43) < ATTN_TOL
+
+
 def test_attention_high_concurrency_mix():
     """128 requests with the high-concurrency block mix {2,4,8,16} @ (.4,.3,.2,.1): about a thousand small tiles."""
     shape = synth.llama8b_shape(1)

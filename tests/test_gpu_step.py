@@ -192,6 +192,37 @@ def test_tiny_self_speculative_loop_is_lossless():
     ctx.recg_free()
 
 
+def test_tiny_prefill_through_the_step():
+    """Chunked prefill is the same step with verify_len = chunk and block_size = 0: the K/V it leaves in the pool must be
+    the oracle's prefill K/V, and the round that follows must emit the oracle's greedy tokens."""
+    shape, W, ocfg, W64 = tiny_model(perturb=False)
+    prompt = synth.token_ids(64, shape.vocab, seed=5).tolist()
+    kv, L, y = orc.prefill(ocfg, W64, prompt)            # commits all but the last prompt token: L = 63
+    ar = orc.greedy_ar(ocfg, W64, prompt, 4)
+    pt, n_pages = synth.page_tables([L], [32], 16, seed=7)
+    ctx = binding.Context(binding.make_config(shape, 1, 64, pt.shape[1]), to_dev(W))
+    pool = binding.alloc_kv_pool(ctx, n_pages, fill=None)
+    pool.fill_(float("nan"))
+    done = 0
+    for chunk in (40, 23):                               # two chunks, the second one ragged
+        batch = binding.Batch([done], [chunk], [0], prompt[done:done + chunk], pt, pool, n_pages)
+        ctx.recg_step(batch)
+        done += chunk
+    ctx.recg_sync()
+    assert done == L
+    for l, (K, V) in enumerate(kv):
+        k_back, v_back = ctx.recg_kv_read(pool, n_pages, l, pt[0], 0, L)
+        for got, ref in ((k_back, K), (v_back, V)):
+            err = np.max(np.abs(f64(got) - ref)) / np.max(np.abs(ref))
+            assert err < HID_TOL, (l, err)
+    # one ordinary round on top of the library's own prefill
+    batch = binding.Batch([L], [1], [8], y, pt, pool, n_pages)
+    ctx.recg_step(batch)
+    g = ctx.recg_verify(batch)
+    assert int(g["accept_len"][0]) == 0 and int(g["emitted"][0]) == ar[0]
+    ctx.recg_free()
+
+
 def test_llama8b_shape_one_layer_round():
     """One 8B-shaped layer + LM head on a ragged batch (spans several GEMM tiles and a ragged tail)."""
     shape = synth.llama8b_shape(1)
