@@ -22,21 +22,22 @@ __device__ __forceinline__ int upper_request(const int* cu, int n_req, int t) {
 // 2 j and 2 j + 1 of a kv head are "siblings": they read the same K/V.  Two lines of 64-token KV blocks are built,
 // every tile preceded by kItemCost virtual blocks that stand for the fixed cost of starting an item (fetching Q,
 // refilling and draining the pipeline):
-//   line A holds one segment per sibling PAIR and is cut into n_ctas / 2 equal contiguous ranges, one per pair of
-//          CTAs (2 p, 2 p + 1): the even CTA works on the first sibling and the odd CTA on the second sibling of the
-//          SAME block ranges, at the same time, so that the second reader of a K/V block finds it in L2;
-//   line B holds the tiles without a sibling and is cut into n_ctas equal ranges, one per CTA.
-// Every CTA first walks its range of line A, then its range of line B; all CTAs carry the same load.  Each piece
-// that holds real blocks is an item; a tile whose blocks are cut by range boundaries gets one partial slot per piece.
-// Items: [line A, first siblings | line A, second siblings (same order) | line B]; cta_off holds, per CTA, the
-// two index ranges it walks.
+//   line A holds one segment per sibling PAIR and is cut into equal contiguous ranges, one per pair of CTAs
+//          (2 p, 2 p + 1): the even CTA works on the first sibling and the odd CTA on the second sibling of the SAME
+//          block ranges, at the same time, so that the second reader of a K/V block finds it in L2;
+//   line B holds the tiles without a sibling and is cut into equal ranges, one per CTA.
+// The CTAs are divided between the two lines in proportion to their work (line A: the first 2 n_pairs_a CTAs), so
+// that every CTA walks ONE range and all carry about the same load.  Each piece that holds real blocks is an item;
+// a tile whose blocks are cut by range boundaries gets one partial slot per piece.
+// Items: [line A, first siblings | line A, second siblings (same order) | line B]; cta_off holds, per CTA, two
+// index ranges it walks one after the other (the second one is empty in this division).
 constexpr int kItemCost = 3;
 
 __global__ void __launch_bounds__(1024) layout_kernel(BatchLayout bl, int n_kv, int mask_id, int tok_per_tile,
                                                       int n_ctas, int64_t n_pages, int* status) {
   extern __shared__ int sm[];
   const int C = bl.n_req;
-  const int n_pairs = n_ctas / 2;
+  const int max_pairs = n_ctas / 2;
   int* off_a = sm;                       // first cost unit of request r in line A
   int* off_b = sm + (C + 1);             // ... in line B
   int* tile_off = sm + 2 * (C + 1);      // first tile entry of request r
@@ -45,9 +46,9 @@ __global__ void __launch_bounds__(1024) layout_kernel(BatchLayout bl, int n_kv, 
   int* part_off = sm + 5 * (C + 1);      // first partial slot of request r
   int* req_nb = sm + 6 * (C + 1);        // blocks per tile of request r
   int* req_rt = sm + 7 * (C + 1);        // row tiles per kv head of request r
-  int* a_off = sm + 8 * (C + 1);         // [n_pairs + 1] first line-A piece of every CTA pair
-  int* b_off = a_off + (n_pairs + 1);    // [n_ctas + 1]  first line-B piece of every CTA
-  __shared__ int s_per_a, s_per_b;
+  int* a_off = sm + 8 * (C + 1);         // [max_pairs + 1] first line-A piece of every CTA pair
+  int* b_off = a_off + (max_pairs + 1);  // [n_ctas + 1]  first line-B piece of every line-B CTA
+  __shared__ int s_per_a, s_per_b, s_pairs_a;
   const int tid = threadIdx.x, nth = blockDim.x;
   griddep_launch();
   griddep_wait();   // the previous step's kernels may still be reading the arrays this kernel rewrites
@@ -94,13 +95,22 @@ __global__ void __launch_bounds__(1024) layout_kernel(BatchLayout bl, int n_kv, 
       off_b[r + 1] = (int)wb;
       tile_off[r + 1] = tile_off[r] + n_kv * rt;
     }
-    const int pa = n_pairs > 0 ? (int)((wa + n_pairs - 1) / n_pairs) : 0x3fffffff;
-    const int pb = (int)((wb + n_ctas - 1) / n_ctas);
+    // CTAs for line A in proportion to its CTA time (two CTAs work on every unit of it)
+    int pairs_a = (2 * wa + wb) > 0 ? (int)(0.5 * n_ctas * (2.0 * wa) / (2.0 * wa + wb) + 0.5) : 0;
+    if (wa > 0 && pairs_a < 1) pairs_a = 1;
+    if (pairs_a > max_pairs) pairs_a = max_pairs;
+    if (wb > 0 && n_ctas - 2 * pairs_a < 1) pairs_a = (n_ctas - 1) / 2;
+    if (wa == 0) pairs_a = 0;
+    const int ctas_b = n_ctas - 2 * pairs_a;
+    const int pa = pairs_a > 0 ? (int)((wa + pairs_a - 1) / pairs_a) : 0x3fffffff;
+    const int pb = ctas_b > 0 ? (int)((wb + ctas_b - 1) / ctas_b) : 0x3fffffff;
     s_per_a = pa < 1 ? 1 : pa;
     s_per_b = pb < 1 ? 1 : pb;
+    s_pairs_a = pairs_a;
   }
   __syncthreads();
   const int per_a = s_per_a, per_b = s_per_b;
+  const int n_pairs = s_pairs_a, n_ctas_b = n_ctas - 2 * s_pairs_a;
   // pieces of a segment whose real blocks occupy the cost range [g0, g0 + nb)
   auto n_pieces = [](int g0, int nb, int per) { return (g0 + nb - 1) / per - g0 / per + 1; };
   for (int r = tid; r < C; r += nth) {
@@ -144,7 +154,7 @@ __global__ void __launch_bounds__(1024) layout_kernel(BatchLayout bl, int n_kv, 
   const int n_items = bl.counts[0];
   const int na = n_items ? item_a[C] : 0, n_b = n_items ? item_b[C] : 0;
   for (int r = tid; r <= C; r += nth) bl.tile_off[r] = tile_off[r];
-  for (int p = tid; p <= n_pairs; p += nth) a_off[p] = na;     // pairs after the last owner; the rest is filled below
+  for (int p = tid; p <= max_pairs; p += nth) a_off[p] = na;   // pairs after the last owner; the rest is filled below
   for (int c = tid; c <= n_ctas; c += nth) b_off[c] = n_b;
   __syncthreads();
   if (n_items) {
@@ -198,7 +208,7 @@ __global__ void __launch_bounds__(1024) layout_kernel(BatchLayout bl, int n_kv, 
     for (int it = tid; it < na; it += nth) {
       const int p = bl.item_cta[it];
       const int prev = it ? bl.item_cta[it - 1] : -1;
-      for (int pp = prev + 1; pp <= p && pp <= n_pairs; ++pp) a_off[pp] = it;   // pairs between two owners have no items
+      for (int pp = prev + 1; pp <= p && pp <= max_pairs; ++pp) a_off[pp] = it;   // pairs between two owners have no items
     }
     for (int it = tid; it < n_b; it += nth) {
       const int c = bl.item_cta[2 * na + it];
@@ -207,19 +217,22 @@ __global__ void __launch_bounds__(1024) layout_kernel(BatchLayout bl, int n_kv, 
     }
   }
   __syncthreads();
-  // the two ranges of item indices every CTA walks: its pair's pieces of line A (first or second siblings), then its own
-  // pieces of line B
+  // the ranges of item indices every CTA walks: a CTA of line A its pair's pieces (first or second siblings), a CTA of
+  // line B its own pieces
   for (int c = tid; c < n_ctas; c += nth) {
-    const int p = c >> 1;
-    int a0 = 0, a1 = 0;
-    if (p < n_pairs) {
+    int a0 = 0, a1 = 0, b0 = 0, b1 = 0;
+    if (c < 2 * n_pairs) {
+      const int p = c >> 1;
       a0 = ((c & 1) ? na : 0) + a_off[p];
       a1 = ((c & 1) ? na : 0) + a_off[p + 1];
+    } else if (c - 2 * n_pairs < n_ctas_b) {
+      b0 = 2 * na + b_off[c - 2 * n_pairs];
+      b1 = 2 * na + b_off[c - 2 * n_pairs + 1];
     }
     bl.cta_off[4 * c + 0] = a0;
     bl.cta_off[4 * c + 1] = a1;
-    bl.cta_off[4 * c + 2] = 2 * na + b_off[c];
-    bl.cta_off[4 * c + 3] = 2 * na + b_off[c + 1];
+    bl.cta_off[4 * c + 2] = b0;
+    bl.cta_off[4 * c + 3] = b1;
   }
 }
 
