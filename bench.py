@@ -415,6 +415,35 @@ def bench_c128(binding, W, shape, peaks, args):
     pool = binding.alloc_kv_pool(ctx, n_pages, fill="normal")
     ys = synth.token_ids(int(desc.verify_len.sum()), shape.vocab, seed=9)
     batch = binding.Batch(desc.ctx_len, desc.verify_len, desc.block_size, ys, desc.page_table, pool, n_pages)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    # ---- tokens/s against concurrency: configs[2]'s recipe (blocks U{4,8,16,32}, verify_len = block, context
+    # U[512,8192]) at 1 .. 128 requests, one batch draw each, whole step (recg_step + recg_verify), device resident
+    sweep = []
+    for C, d in sweep_descs.items():
+        ysw = synth.token_ids(int(d.verify_len.sum()), shape.vocab, seed=50 + C)
+        bt = binding.Batch(d.ctx_len, d.verify_len, d.block_size, ysw, d.page_table, pool, n_pages)
+        vo = binding.VerifyOut(bt.n_req, bt.n_tok, bt.n_ver, host=False)
+        for _ in range(3):
+            ctx.recg_step(bt)
+            ctx.recg_verify(bt, out=vo)
+        torch.cuda.synchronize()
+        n_it = 5
+        e0.record()
+        for _ in range(n_it):
+            ctx.recg_step(bt)
+            ctx.recg_verify(bt, out=vo)
+        e1.record()
+        torch.cuda.synchronize()
+        msw = e0.elapsed_time(e1) / n_it
+        cw = algorithmic_counts(shape, d)
+        sweep.append({"concurrency": C, "tokens_per_step": bt.n_tok, "kv_tokens": int(np.sum(d.ctx_len + d.verify_len + d.block_size)),
+                      "ms_per_step": round(msw, 3), "tokens_per_s": round(bt.n_tok / (msw / 1e3), 1),
+                      "ideal_ms": round(max(sum(cw["wbytes"].values()) / peaks["hbm_gbs"] / 1e6,
+                                            sum(cw["flops"].values()) / peaks["bf16_tflops_sustained"] / 1e9) +
+                                        cw["attn_bytes"] / peaks["hbm_gbs"] / 1e6, 3)})
+    sweep_result = {"workload": "configs[2] recipe at other batch sizes, one draw each, processed tokens/s of the whole step; "
+                                            "ideal_ms = max(weight stream, GEMM flops at sustained peak) + KV stream, of measured peaks",
+                                "points": sweep}
     vout = binding.VerifyOut(batch.n_req, batch.n_tok, batch.n_ver, host=False)
     for _ in range(3):
         ctx.recg_step(batch)
@@ -450,34 +479,7 @@ def bench_c128(binding, W, shape, peaks, args):
                     "frac_of_bf16_sustained": round(gemm_tf / peaks["bf16_tflops_sustained"], 4)},
            "attention": {"ms_per_step": round(attn_ms, 3), "gbs": round(attn_gbs, 1),
                          "frac_of_hbm_measured": round(attn_gbs / peaks["hbm_gbs"], 4)}}
-    # ---- tokens/s against concurrency: configs[2]'s recipe (blocks U{4,8,16,32}, verify_len = block, context
-    # U[512,8192]) at 1 .. 128 requests, one batch draw each, whole step (recg_step + recg_verify), device resident
-    sweep = []
-    for C, d in sweep_descs.items():
-        ysw = synth.token_ids(int(d.verify_len.sum()), shape.vocab, seed=50 + C)
-        bt = binding.Batch(d.ctx_len, d.verify_len, d.block_size, ysw, d.page_table, pool, n_pages)
-        vo = binding.VerifyOut(bt.n_req, bt.n_tok, bt.n_ver, host=False)
-        for _ in range(3):
-            ctx.recg_step(bt)
-            ctx.recg_verify(bt, out=vo)
-        torch.cuda.synchronize()
-        n_it = 5
-        e0.record()
-        for _ in range(n_it):
-            ctx.recg_step(bt)
-            ctx.recg_verify(bt, out=vo)
-        e1.record()
-        torch.cuda.synchronize()
-        msw = e0.elapsed_time(e1) / n_it
-        cw = algorithmic_counts(shape, d)
-        sweep.append({"concurrency": C, "tokens_per_step": bt.n_tok, "kv_tokens": int(np.sum(d.ctx_len + d.verify_len + d.block_size)),
-                      "ms_per_step": round(msw, 3), "tokens_per_s": round(bt.n_tok / (msw / 1e3), 1),
-                      "ideal_ms": round(max(sum(cw["wbytes"].values()) / peaks["hbm_gbs"] / 1e6,
-                                            sum(cw["flops"].values()) / peaks["bf16_tflops_sustained"] / 1e9) +
-                                        cw["attn_bytes"] / peaks["hbm_gbs"] / 1e6, 3)})
-    out["concurrency_sweep"] = {"workload": "configs[2] recipe at other batch sizes, one draw each, processed tokens/s of the whole step; "
-                                            "ideal_ms = max(weight stream, GEMM flops at sustained peak) + KV stream, of measured peaks",
-                                "points": sweep}
+    out["concurrency_sweep"] = sweep_result
     ctx.recg_free()
     del pool
     torch.cuda.empty_cache()
