@@ -610,15 +610,23 @@ __global__ void __launch_bounds__(kThreads, 1) attention_tc_kernel(const __grid_
               }
             }
           } else {
-            // fp32 partial rows: element (lane, i) goes to word lane * 32 + (i ^ lane) (conflict free both ways), then
-            // every store instruction writes one full row segment of 128 bytes
+            // fp32 partial rows: the thread's 32 values go to shared memory as eight 16-byte chunks (chunk q of row
+            // `lane` at position q ^ (lane & 7): conflict free within every quarter warp, both ways); then each store
+            // instruction writes four whole 128-byte row segments
+            float4* s4 = reinterpret_cast<float4*>(stg);
 #pragma unroll
-            for (int i = 0; i < 32; ++i) stg[lane * 32 + (i ^ lane)] = __uint_as_float(r[i]);
+            for (int q = 0; q < 8; ++q)
+              s4[lane * 8 + (q ^ (lane & 7))] = make_float4(__uint_as_float(r[4 * q]), __uint_as_float(r[4 * q + 1]),
+                                                            __uint_as_float(r[4 * q + 2]), __uint_as_float(r[4 * q + 3]));
             __syncwarp();
-            float* dst = P.part_o + ((size_t)w.part * 128 + quad * 32) * D + c * 32 + lane;
-#pragma unroll 8
-            for (int rr = 0; rr < 32; ++rr)
-              if (rr < nrow) dst[(size_t)rr * D] = stg[rr * 32 + (lane ^ rr)];
+            const int rq = lane >> 3, q = lane & 7;
+            float4* dst = reinterpret_cast<float4*>(P.part_o + ((size_t)w.part * 128 + quad * 32) * D + c * 32) + q;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              const int rr = 4 * j + rq;
+              const float4 t = s4[rr * 8 + (q ^ (rr & 7))];
+              if (rr < nrow) __stcg(dst + (size_t)rr * (D / 4), t);
+            }
             __syncwarp();
           }
         }
