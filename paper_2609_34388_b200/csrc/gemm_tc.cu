@@ -650,6 +650,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     // ------------------------------ MMA issuer ------------------------------
     if (rank == 0 && elect_one()) {         // of a pair only the leader issues (it touches shared memory and TMEM only)
       constexpr uint32_t idesc = make_idesc(BN, kRows);
+      const uint64_t desc0 = make_smem_desc(smem_u32(smem));
       int st_idx = 0;
       uint32_t st_phase = 0, tcount = 0;
       bool ok = true;
@@ -675,14 +676,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
             break;
           }
           tc_fence_after();
-          const uint32_t a_addr = smem_u32(smem + s * stage_bytes);
-          const uint32_t b_addr = a_addr + a_bytes;
+          // descriptors are linear in the address (the ring lies inside the 14-bit address field without carry), so
+          // the descriptor of a 16-column slice is the stage's descriptor plus 32 bytes >> 4
+          const uint64_t da0 = desc0 + (uint64_t)((s * stage_bytes) >> 4);
+          const uint64_t db0 = da0 + (uint64_t)(a_bytes >> 4);
 #pragma unroll
           for (int k = 0; k < BK / 16; ++k) {
-            const uint64_t da = make_smem_desc(a_addr + k * 32);
-            const uint64_t db = make_smem_desc(b_addr + k * 32);
-            if constexpr (PAIR) umma_bf16_pair(d_tmem, da, db, idesc, ((kb - kb0) | k) ? 1u : 0u);
-            else umma_bf16(d_tmem, da, db, idesc, ((kb - kb0) | k) ? 1u : 0u);
+            if constexpr (PAIR) umma_bf16_pair(d_tmem, da0 + 2 * k, db0 + 2 * k, idesc, ((kb - kb0) | k) ? 1u : 0u);
+            else umma_bf16(d_tmem, da0 + 2 * k, db0 + 2 * k, idesc, ((kb - kb0) | k) ? 1u : 0u);
           }
           // frees the stage (in both CTAs of a pair) when these MMAs have read it
           if constexpr (PAIR) umma_commit_pair(&empty_bar[s]);
