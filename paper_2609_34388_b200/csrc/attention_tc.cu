@@ -58,7 +58,6 @@ constexpr int kVStages = 3;                      // V ring: a buffer is free aft
                                                  // buffer never holds the unsanitised rows of a partly filled K page
 constexpr int kKVStages = kKStages + kVStages;
 constexpr int kThreads = 384;                    // warpgroup 0: producer K, MMA, producer V, idle; warpgroups 1, 2: softmax
-constexpr int kSoftThreads = 256;
 constexpr uint32_t kSpin = 1u << 22;
 constexpr int kTmemCols = 512;                 // two S buffers of 128 columns (stage & 1); group g owns columns [64 g, 64 g + 64) of each
                                                // and overwrites the first 32 of them with its bf16 P; O of group g at 256 + 128 g
@@ -169,9 +168,6 @@ constexpr uint32_t kIdescQK = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(k
 constexpr uint32_t kIdescPV =
     (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(D >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
 
-__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
-  asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
-}
 __device__ __forceinline__ void tma_load_3d(uint32_t smem_dst, const CUtensorMap* map, int x, int y, int z, uint64_t* bar) {
   asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
                :

@@ -204,26 +204,12 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint64_t* bar, uint32_t parity
 
 
 // ---- register epilogue: one thread owns one output row -------------------------------------------
-// add = true accumulates into the fp32 residual stream with vector reductions at L2: every element receives
-// exactly one addend from exactly one thread per launch, so the result is the same single rounding as a
-// load-add-store, without the load's round trip in front of every chunk.
-__device__ __forceinline__ void store_chunk_f32(float* dst, const float (&v)[32], bool add) {
-#pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    float4* p = reinterpret_cast<float4*>(dst) + i;
-    if (add) {
-      asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(p), "f"(v[4 * i]), "f"(v[4 * i + 1]), "f"(v[4 * i + 2]),
-                   "f"(v[4 * i + 3])
-                   : "memory");
-    } else {
-      *p = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
-    }
-  }
-}
 // Warp-wide stores of a 32-row x 32-column chunk (lane = row holds the row's 32 values): the chunk is transposed
 // through 4 KB of shared memory so that every store instruction writes whole 128-byte (fp32) or 64-byte (bf16)
 // row segments instead of 16 bytes in each of 32 different rows.  dst0 points at (row 0 of the warp, first column
-// of the chunk); rows >= valid_rows are not written.  Every lane must call.
+// of the chunk); rows >= valid_rows are not written.  Every lane must call.  add = true accumulates into the fp32
+// residual stream with vector reductions at L2: every element receives exactly one addend from exactly one thread per
+// launch, so the result is the same single rounding as a load-add-store, without the load's round trip.
 __device__ __forceinline__ void store_rows_f32(float* dst0, size_t row_stride, int valid_rows, const float (&v)[32], bool add,
                                                float* stg, int lane) {
   float4* s4 = reinterpret_cast<float4*>(stg);
@@ -265,17 +251,6 @@ __device__ __forceinline__ void store_rows_bf16(__nv_bfloat16* dst0, size_t row_
     if (r < valid_rows) *(reinterpret_cast<uint4*>(dst0 + (size_t)r * row_stride) + q) = t;
   }
   __syncwarp();
-}
-__device__ __forceinline__ void store_chunk_bf16(__nv_bfloat16* dst, const float (&v)[32]) {
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    uint4 o;
-    o.x = pack_bf16(v[8 * i], v[8 * i + 1]);
-    o.y = pack_bf16(v[8 * i + 2], v[8 * i + 3]);
-    o.z = pack_bf16(v[8 * i + 4], v[8 * i + 5]);
-    o.w = pack_bf16(v[8 * i + 6], v[8 * i + 7]);
-    reinterpret_cast<uint4*>(dst)[i] = o;
-  }
 }
 
 // Where the epilogue takes the thread's accumulator row from: TMEM, or the sum over the K splits' partial tiles.
