@@ -17,6 +17,9 @@ What follows the paper, and where:
   first drafted token equals the verifier's bonus token)        -- Sec. 5.1
 * co-batching the next draft block with the current verify
   rows in one forward over a shared prefix                      -- Sec. 5.1, 5.3
+* risky positions (M_i < delta, earliest two), correction
+  branches with the second candidate, their reuse rule, and
+  the recursive loop over verifier + up to three branches       -- Sec. 5.1
 
 The backbone itself (RMSNorm, rotary embedding with rotate-half pairing,
 grouped-query attention, SwiGLU, untied LM head) is the generic Llama-style
@@ -27,7 +30,10 @@ Parity pins (see tests/test_oracle_*.py): brute-force loops over Eq. 1 on tiny
 shapes, a library attention routine with the same boolean mask, an independent
 library implementation of the causal decoder, losslessness of greedy
 speculation against token-by-token greedy decoding, cached == dense, closed
-forms for the statistics, and planted accept lengths.  No value printed in the
+forms for the statistics, and planted accept lengths; for the branches, each
+branch row against the standalone round it hypothesises, visibility by brute
+force, planted selection / reuse cases and losslessness of the recursive loop
+(tests/test_oracle_overlap.py).  No value printed in the
 paper exists for this path, so numeric parity with the paper itself is
 unpinned; parity is with these definitions.
 """
@@ -421,3 +427,180 @@ def spec_decode(cfg: ModelConfig, W: Weights, prompt: Sequence[int], b: int, rou
         else:
             y = [bonus]
     return out, trace, (kv, L)
+
+
+# --------------------------------------------------------------------------
+# predictive draft-verify overlap: correction and continuation branches (Sec. 5.1)
+# --------------------------------------------------------------------------
+# One request's round then holds up to four logical rows that share the
+# canonical prefix (Sec. 5.1, 5.3):
+#   verifier      y_0 .. y_{v-1}                       causal
+#   continuation  b mask tokens after the whole y      sees prefix + y + its block
+#   correction k  for a risky draft index i_k (1 <= i_k <= v-1): the replacement
+#                 token r_k standing where y_{i_k} stands, then bc mask tokens;
+#                 sees prefix + y_0 .. y_{i_k - 1} + its own tokens
+# New rows are ordered [verifier | continuation | correction 0 | correction 1];
+# their K/V occupy cache indices L, L+1, ... in that order, while the rotary
+# position of a branch token is the position it would have in the sequence the
+# branch hypothesises (r_k at L + i_k, its masks at L + i_k + 1 ...).
+DELTA_RISKY = 0.5   # margin threshold of the risky-position rule (Sec. 5.1 / experimental setup)
+
+
+def select_branches(margin: Sequence[float], second: Sequence[int], delta: float = DELTA_RISKY, keep: int = 2):
+    """Risky-position rule of Sec. 5.1 for the pending drafts y_1 .. y_{v-1}.
+
+    margin[i], second[i] are M_i and the second-ranked token id of the draft
+    row that produced y_i (entry 0 is ignored: y_0 is known to be correct).
+    A position is risky when M_i < delta; the earliest `keep` risky positions
+    get a correction branch (the draft replaced by its second candidate), and
+    the continuation branch is prepared only when no more than `keep`
+    positions are risky.  Returns ([(i, replacement)], continuation?).
+    """
+    risky = [i for i in range(1, len(margin)) if float(margin[i]) < delta]
+    corr = [(i, int(second[i])) for i in risky[:keep]]
+    return corr, len(risky) <= keep
+
+
+def overlap_round_rows(L: int, v: int, b: int, corr: Sequence[Tuple[int, int]], bc: int):
+    """Positions and visibility of the rows of a round with branches.
+
+    Returns (pos [n], vis [n, L + n], kind [n]) with n = v + b + len(corr) * (1 + bc);
+    kind is 'v' (verifier), 'c' (continuation mask), 'r' (replacement token)
+    or 'm' (mask of a correction branch).  Column j < L is committed context,
+    column L + j is new row j.
+    """
+    n = v + b + len(corr) * (1 + bc)
+    pos = np.zeros(n, dtype=np.int64)
+    vis = np.zeros((n, L + n), dtype=bool)
+    kind = []
+    for j in range(v):                      # verifier: M^AR
+        pos[j] = L + j
+        vis[j, : L + j + 1] = True
+        kind.append("v")
+    for j in range(b):                      # continuation: Eq. 1 with prefix = context + y
+        pos[v + j] = L + v + j
+        vis[v + j, : L + v] = True
+        vis[v + j, L + v: L + v + b] = True
+        kind.append("c")
+    for k, (i, _tok) in enumerate(corr):
+        assert 1 <= i <= v - 1, "a correction replaces one of the drafts y_1 .. y_{v-1}"
+        r0 = v + b + k * (1 + bc)           # row of the replacement token
+        pos[r0] = L + i
+        vis[r0, : L + i] = True             # context + y_0 .. y_{i-1}
+        vis[r0, L + r0] = True              # itself (causal token)
+        kind.append("r")
+        for j in range(bc):                 # the branch's own block: Eq. 1 with prefix = ... + replacement
+            pos[r0 + 1 + j] = L + i + 1 + j
+            vis[r0 + 1 + j, : L + i] = True
+            vis[r0 + 1 + j, L + r0: L + r0 + 1 + bc] = True
+            kind.append("m")
+    return pos, vis, kind
+
+
+def overlap_round_cached(cfg: ModelConfig, W: Weights, kv_prefix, L: int, verify_ids: Sequence[int], b: int,
+                         corr: Sequence[Tuple[int, int]], bc: int, act_round=None):
+    """One forward over the verifier and all prospective branches of a request."""
+    ids = list(verify_ids) + [cfg.mask_id()] * b
+    for (_i, tok) in corr:
+        ids += [int(tok)] + [cfg.mask_id()] * bc
+    pos, vis, _ = overlap_round_rows(L, len(verify_ids), b, corr, bc)
+    pre = [(K[:L], V[:L]) for (K, V) in kv_prefix]
+    return decoder_rows(cfg, W, ids, pos, vis, pre, act_round)
+
+
+def verify_overlap_round(logits: np.ndarray, y: Sequence[int], b: int, corr: Sequence[Tuple[int, int]], bc: int,
+                         delta: float = DELTA_RISKY) -> Dict[str, object]:
+    """verify_round() plus the branch reuse rules and the next round's risky positions.
+
+    corr_hit[k]: the verifier rejected exactly the draft the branch replaced
+    (accept length a = i_k - 1) and its own token there equals the replacement
+    (Sec. 5.1).  corr_draft[k]: argmax of the branch's mask rows, the drafts
+    that follow the replacement if the branch is reused.
+    risky[j] describes draft block j (0 = continuation, 1 + k = correction k)
+    in the indexing of the verify row it would become: the continuation gives
+    y' = [bonus, d_1, ..], so mask row m is y'_m (m >= 1); a correction gives
+    y' = [replacement, d_0, ..], so mask row m is y'_{m+1}.  Each entry is
+    (number of risky positions, [(index into y', second candidate)] for the
+    earliest two).
+    """
+    v = len(y)
+    n_corr = len(corr)
+    assert logits.shape[0] == v + b + n_corr * (1 + bc)
+    out = verify_round(logits[: v + b], y, b)
+    a = out["accept_len"]
+    st_all = list(out["stats"])
+    hits, drafts, risky = [], [], []
+
+    def block_risky(stats, first_index):
+        idx = [first_index + m for m, s in enumerate(stats) if s["margin"] < delta]
+        sec = {first_index + m: s["top2"] for m, s in enumerate(stats)}
+        return (len(idx), [(i, sec[i]) for i in idx[:2]])
+
+    risky.append(block_risky(st_all[v + 1: v + b], 1))
+    for k, (i, tok) in enumerate(corr):
+        r0 = v + b + k * (1 + bc)
+        st = [row_stats(logits[r]) for r in range(r0, r0 + 1 + bc)]
+        st_all += st
+        hits.append(bool(a == i - 1 and out["emitted"][-1] == int(tok)))
+        drafts.append([s["top1"] for s in st[1:]])
+        risky.append(block_risky(st[1:], 1))
+    out.update({"stats": st_all, "corr_hit": hits, "corr_draft": drafts, "risky": risky})
+    return out
+
+
+def spec_decode_overlap(cfg: ModelConfig, W: Weights, prompt: Sequence[int], b: int, rounds: int,
+                        delta: float = DELTA_RISKY, poison_rollback: bool = True):
+    """Self-speculative decoding with predictive draft-verify overlap (Sec. 5.1).
+
+    Every round runs one forward over the verifier row and the branches the
+    risky-position rule selects, then keeps the branch the verification outcome
+    confirms (a correction that predicted both the rejected position and the
+    verifier's token, or the continuation after full acceptance); its drafts
+    are the next round's verify tokens, and the rule is applied to them again.
+    Returns (emitted tokens, per-round trace).
+    """
+    kv, L, y = prefill(cfg, W, prompt)
+    margin: List[float] = [1.0]
+    second: List[int] = [-1]
+    out: List[int] = []
+    trace = []
+    for _t in range(rounds):
+        corr, cont = select_branches(margin, second, delta)
+        bb = b if cont else 0
+        logits, kv_new, _ = overlap_round_cached(cfg, W, kv, L, y, bb, corr, b)
+        r = verify_overlap_round(logits, y, bb, corr, b, delta)
+        a = r["accept_len"]
+        new_L = L + a + 1
+        kv = []
+        for (K, V) in kv_new:
+            K = K[: L + len(y)].copy()
+            V = V[: L + len(y)].copy()
+            if poison_rollback:
+                K[new_L:] = np.nan
+                V[new_L:] = np.nan
+            kv.append((K, V))
+        out += r["emitted"]
+        v = len(y)
+        st = r["stats"]
+        used = "none"
+        bonus = r["emitted"][-1]
+        if r["cont_hit"]:
+            used = "continuation"
+            rows = st[v + 1: v + bb]
+            y_next = [bonus] + [s["top1"] for s in rows]
+        elif any(r["corr_hit"]):
+            k = r["corr_hit"].index(True)
+            used = "correction%d" % k
+            r0 = v + bb + k * (1 + b)
+            rows = st[r0 + 1: r0 + 1 + b]
+            y_next = [bonus] + [s["top1"] for s in rows]
+        else:
+            rows = []
+            y_next = [bonus]
+        trace.append({"L": L, "y": list(y), "corr": list(corr), "cont": cont, "accept_len": a,
+                      "emitted": list(r["emitted"]), "used": used, "new_L": new_L})
+        margin = [1.0] + [s["margin"] for s in rows]
+        second = [-1] + [s["top2"] for s in rows]
+        y = y_next
+        L = new_L
+    return out, trace
