@@ -98,6 +98,20 @@ typedef struct {
  *                  (per layer, per page, per KV head: a K tile then a V tile of 16 tokens, stored in
  *                  the swizzled order the attention kernel loads; use recg_kv_write / recg_kv_read
  *                  to move logical K/V in and out).  May be NULL for a verify-only call.
+ *
+ * Prospective correction branches of the predictive draft-verify overlap (Sec. 5.1); n_corr == NULL
+ * means no request has any, and block_size[r] is then the only draft block (the continuation branch):
+ *   n_corr[r]        0..2 correction branches of request r
+ *   corr_index[2r+k] i, 1 <= i <= v_r - 1, strictly increasing in k: the draft y_i the branch replaces
+ *   corr_token[2r+k] the replacement token (the draft's second candidate)
+ *   corr_block[r]    bc_r >= 0, mask tokens that follow the replacement token in each branch of r
+ * Request r then has n_r = v_r + b_r + n_corr[r] * (1 + bc_r) rows in the ragged batch, in the order
+ * [verify | continuation masks | branch 0: replacement, masks | branch 1: replacement, masks], and their
+ * K/V occupy cache positions L_r .. L_r + n_r - 1 in that order (the page-table row must cover them).
+ * A branch token is rotated as the position it hypothesises (replacement: L_r + i, masks: L_r + i + 1 ..).
+ * It sees the committed context and y_0 .. y_{i-1}; besides those the replacement token sees itself and a
+ * mask token sees its whole branch.  Branch rows are always rolled back by recg_verify.
+ *   risk_delta       margin threshold of the risky-position outputs of recg_verify; <= 0 means 0.5
  */
 typedef struct {
   int32_t n_req;
@@ -109,6 +123,11 @@ typedef struct {
   int32_t page_table_stride;
   void *kv_pool;
   int64_t kv_pool_pages;
+  const int32_t *n_corr;
+  const int32_t *corr_index;
+  const int32_t *corr_token;
+  const int32_t *corr_block;
+  float risk_delta;
 } recg_batch;
 
 /* Logits of the last recg_step(): DEVICE, library-owned, valid until the next recg_step(). */
@@ -123,7 +142,7 @@ typedef struct {
  * Outputs of greedy verification.  All buffers are caller-provided and live where `mem` says
  * (every pointer in one struct in the same place); any pointer may be NULL to skip that output.
  * With RECG_MEM_HOST the call copies the results out and synchronises the stream before returning.
- * T = sum(v_r + b_r), Tv = sum(v_r), Tb = sum(b_r).
+ * T = sum(n_r) rows of the batch, Tv = sum(v_r), Tb = T - Tv (all rows that are not verify rows).
  *   accept_len[n_req]    a_r: drafts y_1..y_a accepted (longest prefix equal to the verifier argmax)
  *   n_emitted[n_req]     a_r + 1 (0 if v_r = 0)
  *   emitted[Tv]          per request, at its verify offset: y_1..y_a then the verifier's token at row a
@@ -133,18 +152,29 @@ typedef struct {
  *                        -(slot+1) if it is rolled back (rejected draft or mask row)
  *   freed_pages[n_req]   number of pages of request r that hold no committed token any more
  *                        (its page-table entries from ceil(new_ctx_len/page_size) on)
- *   next_draft[Tb]       argmax of every mask row: the next round's drafts
+ *   next_draft[Tb]       argmax of every row that is not a verify row, in batch order: per request its
+ *                        continuation masks, then per branch the replacement row and the branch's masks
  *   cont_hit[n_req]      1 if the block was fully accepted and the first drafted token equals the
  *                        bonus token (the continuation branch can be reused), else 0
  *   top1, top2 [T]       ids of the largest and second-largest logit per row (lowest index wins ties)
  *   p1, p2, entropy [T]  float32: softmax probability of top1 and top2, entropy in nats
  *   entropy_mean[n_req]  float32: mean verifier entropy over rows 0..a_r
+ * Branch reuse and the next round's risky positions (Sec. 5.1):
+ *   corr_hit[2 n_req]    entry 2r+k: 1 if the verifier rejected exactly the draft branch k replaced
+ *                        (a_r == i - 1) and its own token there equals the replacement token, else 0
+ *   risky_n[3 n_req]     entry 3r+j: how many drafts of block j of request r (j = 0 the continuation block,
+ *                        j = 1 + k correction branch k) have margin p1 - p2 < risk_delta; 0 for absent blocks
+ *   risky_index, risky_token [6 n_req]  entries 6r+2j+{0,1}: the earliest two of them, as the index the
+ *                        draft would have in the next round's verify tokens (continuation: mask row m is
+ *                        y'_m, m >= 1, since y'_0 is the bonus token; correction: mask row m is y'_{m+1})
+ *                        and the row's second candidate; -1 where there is none
  */
 typedef struct {
   int32_t mem; /* recg_mem */
   int32_t *accept_len, *n_emitted, *emitted, *new_ctx_len, *slot_state, *freed_pages;
   int32_t *next_draft, *cont_hit, *top1, *top2;
   float *p1, *p2, *entropy, *entropy_mean;
+  int32_t *corr_hit, *risky_n, *risky_index, *risky_token;
 } recg_verify_out;
 
 /* Bytes of KV pool needed for n_pages physical pages (all layers). */

@@ -45,7 +45,9 @@ class recg_weights(C.Structure):
 class recg_batch(C.Structure):
     _fields_ = [("n_req", C.c_int32), ("ctx_len", C.c_void_p), ("verify_len", C.c_void_p), ("block_size", C.c_void_p),
                 ("verify_tokens", C.c_void_p), ("page_table", C.c_void_p), ("page_table_stride", C.c_int32),
-                ("kv_pool", C.c_void_p), ("kv_pool_pages", C.c_int64)]
+                ("kv_pool", C.c_void_p), ("kv_pool_pages", C.c_int64), ("n_corr", C.c_void_p),
+                ("corr_index", C.c_void_p), ("corr_token", C.c_void_p), ("corr_block", C.c_void_p),
+                ("risk_delta", C.c_float)]
 
 
 class recg_logits(C.Structure):
@@ -55,10 +57,11 @@ class recg_logits(C.Structure):
 _INT_OUT = ("accept_len", "n_emitted", "emitted", "new_ctx_len", "slot_state", "freed_pages", "next_draft", "cont_hit",
             "top1", "top2")
 _FLT_OUT = ("p1", "p2", "entropy", "entropy_mean")
+_INT_OUT_BRANCH = ("corr_hit", "risky_n", "risky_index", "risky_token")
 
 
 class recg_verify_out(C.Structure):
-    _fields_ = [("mem", C.c_int32)] + [(n, C.c_void_p) for n in _INT_OUT + _FLT_OUT]
+    _fields_ = [("mem", C.c_int32)] + [(n, C.c_void_p) for n in _INT_OUT + _FLT_OUT + _INT_OUT_BRANCH]
 
 
 _lib = None
@@ -130,17 +133,27 @@ class Batch:
     """Holds the host arrays of one recg_batch alive and exposes the C struct."""
 
     def __init__(self, ctx_len, verify_len, block_size, verify_tokens=None, page_table=None, kv_pool=None,
-                 kv_pool_pages: int = 0):
+                 kv_pool_pages: int = 0, n_corr=None, corr_index=None, corr_token=None, corr_block=None,
+                 risk_delta: float = 0.0):
+        """n_corr [C], corr_index / corr_token [C, 2], corr_block [C]: the correction branches (all None = none)."""
         self.ctx_len, self.verify_len, self.block_size = _i32(ctx_len), _i32(verify_len), _i32(block_size)
         self.verify_tokens = _i32(verify_tokens) if verify_tokens is not None else np.zeros(0, np.int32)
         self.page_table = None if page_table is None else _i32(page_table)
         self.kv_pool = kv_pool
         stride = 0 if self.page_table is None else int(self.page_table.shape[1])
+        self.n_req = len(self.ctx_len)
+        self.n_corr = None if n_corr is None else _i32(n_corr)
+        self.corr_index = None if n_corr is None else _i32(corr_index).reshape(self.n_req, 2)
+        self.corr_token = None if n_corr is None else _i32(corr_token).reshape(self.n_req, 2)
+        self.corr_block = None if n_corr is None else _i32(corr_block)
         self.c = recg_batch(len(self.ctx_len), _ptr(self.ctx_len), _ptr(self.verify_len), _ptr(self.block_size),
                             _ptr(self.verify_tokens) if self.verify_tokens.size else None, _ptr(self.page_table),
-                            stride, _ptr(kv_pool), int(kv_pool_pages))
-        self.n_req = len(self.ctx_len)
-        self.n_tok = int(self.verify_len.sum() + self.block_size.sum())
+                            stride, _ptr(kv_pool), int(kv_pool_pages), _ptr(self.n_corr), _ptr(self.corr_index),
+                            _ptr(self.corr_token), _ptr(self.corr_block), float(risk_delta))
+        self.rows = self.verify_len + self.block_size          # rows of each request in the ragged batch
+        if self.n_corr is not None:
+            self.rows = self.rows + self.n_corr * (1 + self.corr_block)
+        self.n_tok = int(self.rows.sum())
         self.n_ver = int(self.verify_len.sum())
 
 
@@ -150,7 +163,8 @@ class VerifyOut:
     def __init__(self, n_req: int, n_tok: int, n_ver: int, host: bool = True):
         self.sizes = {"accept_len": n_req, "n_emitted": n_req, "emitted": n_ver, "new_ctx_len": n_req,
                       "slot_state": n_tok, "freed_pages": n_req, "next_draft": n_tok - n_ver, "cont_hit": n_req,
-                      "top1": n_tok, "top2": n_tok, "p1": n_tok, "p2": n_tok, "entropy": n_tok, "entropy_mean": n_req}
+                      "top1": n_tok, "top2": n_tok, "p1": n_tok, "p2": n_tok, "entropy": n_tok, "entropy_mean": n_req,
+                      "corr_hit": 2 * n_req, "risky_n": 3 * n_req, "risky_index": 6 * n_req, "risky_token": 6 * n_req}
         self.bufs = {}
         self.c = recg_verify_out()
         self.c.mem = MEM_HOST if host else MEM_DEVICE

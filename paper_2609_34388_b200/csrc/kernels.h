@@ -27,20 +27,22 @@ struct AttnTile {        // per (request, kv head, row tile): where its partials
 // Device-resident ragged layout of one batch (all pointers DEVICE, int32 unless noted).
 struct BatchLayout {
   int n_req, n_tok, n_ver, pt_stride;
+  float risk_delta;       // margin threshold of the risky-position outputs
   const int* ctx_len;     // [C]
   const int* verify_len;  // [C]
   const int* block_size;  // [C]
-  const int* cu_tok;      // [C+1] exclusive prefix sum of v+b
+  const int* corr;        // [C][6] correction branches: count (0..2), mask tokens per branch, index 0, index 1, token 0, token 1
+  const int* cu_tok;      // [C+1] exclusive prefix sum of the rows per request, v + b + count * (1 + mask tokens per branch)
   const int* cu_ver;      // [C+1] exclusive prefix sum of v
   const int* verify_tokens;  // [Tv]
   const int* page_table;  // [C, pt_stride] (may be null for verify-only batches)
   // per token, written by the layout kernel
   int* tok_id;
   int* tok_req;
-  int* tok_pos;
-  int* tok_slot;    // page*16 + offset, -1 without a page table
-  int* tok_climit;  // sees every position <= climit ...
-  int* tok_lo;      // ... and every position in [lo, hi)
+  int* tok_pos;     // rotary position (a branch token: the position its branch hypothesises)
+  int* tok_slot;    // page*16 + offset of cache position L + (row within the request), -1 without a page table
+  int* tok_climit;  // sees every cache position <= climit ...
+  int* tok_lo;      // ... and every cache position in [lo, hi)
   int* tok_hi;
   // attention work list
   AttnItem* items;
@@ -108,6 +110,7 @@ struct VerifyBuffers {   // DEVICE outputs (library workspace or caller buffers)
   int *accept_len, *n_emitted, *emitted, *new_ctx_len, *slot_state, *freed_pages, *next_draft, *cont_hit, *top1,
       *top2;
   float *p1, *p2, *entropy, *entropy_mean;
+  int *corr_hit, *risky_n, *risky_index, *risky_token;
 };
 struct RowPartial {      // per (row, vocab chunk)
   float m1, m2;          // largest and second-largest logit of the chunk

@@ -58,26 +58,40 @@ __global__ void __launch_bounds__(1024) layout_kernel(BatchLayout bl, int n_kv, 
     const int r = upper_request(bl.cu_tok, C, t);
     const int j = t - bl.cu_tok[r];
     const int L = bl.ctx_len[r], v = bl.verify_len[r], b = bl.block_size[r];
-    const int pos = L + j;
-    const bool is_ver = j < v;
+    const int idx = L + j;   // cache position of the token's K/V
+    int pos, id, climit, lo, hi;
+    if (j < v) {             // verifier: causal
+      pos = idx; id = bl.verify_tokens[bl.cu_ver[r] + j]; climit = idx; lo = 0; hi = 0;
+    } else if (j < v + b) {  // continuation block: the whole prefix and the block
+      pos = idx; id = mask_id; climit = L + v - 1; lo = L + v; hi = L + v + b;
+    } else {                 // correction branch k: replacement token, then its mask tokens
+      const int* cr = bl.corr + 6 * r;
+      const int span = 1 + cr[1], jj = j - v - b, k = jj / span, q = jj - k * span;
+      const int i = cr[2 + k], first = L + v + b + k * span;
+      pos = L + i + q;
+      id = q == 0 ? cr[4 + k] : mask_id;
+      climit = L + i - 1;
+      lo = first;
+      hi = q == 0 ? first + 1 : first + span;
+    }
     bl.tok_req[t] = r;
     bl.tok_pos[t] = pos;
-    bl.tok_id[t] = is_ver ? bl.verify_tokens[bl.cu_ver[r] + j] : mask_id;
-    bl.tok_climit[t] = is_ver ? pos : L + v - 1;
-    bl.tok_lo[t] = is_ver ? 0 : L + v;
-    bl.tok_hi[t] = is_ver ? 0 : L + v + b;
+    bl.tok_id[t] = id;
+    bl.tok_climit[t] = climit;
+    bl.tok_lo[t] = lo;
+    bl.tok_hi[t] = hi;
     int slot = -1;
     if (bl.page_table) {
-      const int page = bl.page_table[(size_t)r * bl.pt_stride + pos / kPageSize];
+      const int page = bl.page_table[(size_t)r * bl.pt_stride + idx / kPageSize];
       if (page < 0 || page >= n_pages) set_status(status, DEV_BAD_INDEX);
-      else slot = page * kPageSize + pos % kPageSize;
+      else slot = page * kPageSize + idx % kPageSize;
     }
     bl.tok_slot[t] = slot;
   }
 
   // ---- attention work list ----
   for (int r = tid; r < C; r += nth) {
-    const int n = bl.verify_len[r] + bl.block_size[r];
+    const int n = bl.cu_tok[r + 1] - bl.cu_tok[r];
     req_nb[r] = (bl.ctx_len[r] + n + 63) / 64;
     req_rt[r] = (n + tok_per_tile - 1) / tok_per_tile;
   }
@@ -159,7 +173,7 @@ __global__ void __launch_bounds__(1024) layout_kernel(BatchLayout bl, int n_kv, 
   __syncthreads();
   if (n_items) {
     for (int r = tid; r < C; r += nth) {
-      const int n = bl.verify_len[r] + bl.block_size[r];
+      const int n = bl.cu_tok[r + 1] - bl.cu_tok[r];
       const int kv_len = bl.ctx_len[r] + n;
       const int nb = req_nb[r], rt = req_rt[r], seg = nb + kItemCost;
       int ia = item_a[r], ib = item_b[r], part = part_off[r];

@@ -99,7 +99,7 @@ size_t carve(recg_ctx* c, DeviceArena& A) {
   const recg_config& g = c->cfg;
   const size_t Cm = g.max_requests, Tm = g.max_tokens, Pm = g.max_pages_per_request;
   const Dims& d = c->dm;
-  c->desc_ints = 3 * Cm + 2 * (Cm + 1) + Tm + Cm * Pm;
+  c->desc_ints = 9 * Cm + 2 * (Cm + 1) + Tm + Cm * Pm;
   c->d_desc = A.take<int>(c->desc_ints);
   BatchLayout& bl = c->bl;
   bl.tok_id = A.take<int>(Tm);
@@ -140,6 +140,10 @@ size_t carve(recg_ctx* c, DeviceArena& A) {
   v.p2 = A.take<float>(Tm);
   v.entropy = A.take<float>(Tm);
   v.entropy_mean = A.take<float>(Cm);
+  v.corr_hit = A.take<int>(2 * Cm);
+  v.risky_n = A.take<int>(3 * Cm);
+  v.risky_index = A.take<int>(6 * Cm);
+  v.risky_token = A.take<int>(6 * Cm);
   c->q = A.take<__nv_bfloat16>(Tm * d.n_q * d.head_dim);
   c->o = A.take<__nv_bfloat16>(Tm * d.n_q * d.head_dim);
   if (c->has_weights) {
@@ -152,7 +156,13 @@ size_t carve(recg_ctx* c, DeviceArena& A) {
   return A.used + 256;
 }
 
-// Validate a batch and pack [ctx_len | verify_len | block_size | cu_tok | cu_ver | verify_tokens | page_table].
+// Rows of request r: verify tokens, continuation masks and the correction branches (replacement + masks each).
+static inline int request_rows(const recg_batch* b, int r) {
+  const int nc = b->n_corr ? b->n_corr[r] : 0;
+  return b->verify_len[r] + b->block_size[r] + nc * (1 + (nc ? b->corr_block[r] : 0));
+}
+
+// Validate a batch and pack [ctx_len | verify_len | block_size | corr | cu_tok | cu_ver | verify_tokens | page_table].
 recg_status pack_batch(recg_ctx* ctx, const recg_batch* b, bool need_pages, bool need_tokens, int* T_out, int* Tv_out) {
   if (!b || b->n_req <= 0 || !b->ctx_len || !b->verify_len || !b->block_size)
     return fail(ctx, RECG_ERR_INVALID_ARG, "batch: null descriptor array or n_req <= 0");
@@ -163,33 +173,56 @@ recg_status pack_batch(recg_ctx* ctx, const recg_batch* b, bool need_pages, bool
     return fail(ctx, RECG_ERR_INVALID_ARG, "batch: page_table and kv_pool are required");
   if (pages && (b->page_table_stride <= 0 || b->page_table_stride > ctx->cfg.max_pages_per_request))
     return fail(ctx, RECG_ERR_CAPACITY, "batch: page_table_stride exceeds max_pages_per_request");
+  if (b->n_corr && (!b->corr_index || !b->corr_token || !b->corr_block))
+    return fail(ctx, RECG_ERR_INVALID_ARG, "batch: n_corr given without corr_index, corr_token and corr_block");
   long long T = 0, Tv = 0;
   for (int r = 0; r < C; ++r) {
     const int L = b->ctx_len[r], v = b->verify_len[r], k = b->block_size[r];
     if (L < 0 || v < 0 || k < 0 || v + k < 1)
       return fail(ctx, RECG_ERR_INVALID_ARG, "batch: negative length or a request without rows");
-    if (pages) {
-      const long long need = ((long long)L + v + k + kPageSize - 1) / kPageSize;
-      if (need > b->page_table_stride)
-        return fail(ctx, RECG_ERR_CAPACITY, "batch: page table row does not cover ctx_len + verify_len + block_size");
+    if (b->n_corr && b->n_corr[r] != 0) {
+      const int nc = b->n_corr[r];
+      if (nc < 0 || nc > 2 || b->corr_block[r] < 0)
+        return fail(ctx, RECG_ERR_INVALID_ARG, "batch: n_corr must be 0, 1 or 2 and corr_block >= 0");
+      for (int q = 0; q < nc; ++q) {
+        const int i = b->corr_index[2 * r + q], tok = b->corr_token[2 * r + q];
+        if (i < 1 || i > v - 1 || (q > 0 && i <= b->corr_index[2 * r + q - 1]))
+          return fail(ctx, RECG_ERR_INVALID_ARG, "batch: corr_index must name drafts y_1 .. y_{v-1} in increasing order");
+        if (tok < 0 || tok >= ctx->cfg.vocab) return fail(ctx, RECG_ERR_INVALID_ARG, "batch: corr_token outside the vocabulary");
+      }
     }
-    T += v + k;
+    const int n = request_rows(b, r);
+    if (pages) {
+      const long long need = ((long long)L + n + kPageSize - 1) / kPageSize;
+      if (need > b->page_table_stride)
+        return fail(ctx, RECG_ERR_CAPACITY, "batch: page table row does not cover ctx_len plus the rows of the request");
+    }
+    T += n;
     Tv += v;
   }
   if (T > ctx->cfg.max_tokens) return fail(ctx, RECG_ERR_CAPACITY, "batch: token count exceeds max_tokens");
   if (Tv > 0 && !b->verify_tokens && need_tokens) return fail(ctx, RECG_ERR_INVALID_ARG, "batch: verify_tokens is null");
   const int stride = pages ? b->page_table_stride : 0;
   std::vector<int>& hd = ctx->h_desc;
-  hd.resize(3 * (size_t)C + 2 * ((size_t)C + 1) + (size_t)Tv + (size_t)C * stride);
+  hd.resize(9 * (size_t)C + 2 * ((size_t)C + 1) + (size_t)Tv + (size_t)C * stride);
   int* p = hd.data();
   memcpy(p, b->ctx_len, C * sizeof(int));
   memcpy(p + C, b->verify_len, C * sizeof(int));
   memcpy(p + 2 * C, b->block_size, C * sizeof(int));
-  int* cu_tok = p + 3 * C;
+  int* corr = p + 3 * C;   // per request: count, mask tokens per branch, index 0, index 1, token 0, token 1
+  int* cu_tok = p + 9 * C;
   int* cu_ver = cu_tok + (C + 1);
   cu_tok[0] = cu_ver[0] = 0;
   for (int r = 0; r < C; ++r) {
-    cu_tok[r + 1] = cu_tok[r] + b->verify_len[r] + b->block_size[r];
+    const int nc = b->n_corr ? b->n_corr[r] : 0;
+    int* cr = corr + 6 * r;
+    cr[0] = nc;
+    cr[1] = nc ? b->corr_block[r] : 0;
+    for (int q = 0; q < 2; ++q) {
+      cr[2 + q] = q < nc ? b->corr_index[2 * r + q] : 0;
+      cr[4 + q] = q < nc ? b->corr_token[2 * r + q] : 0;
+    }
+    cu_tok[r + 1] = cu_tok[r] + request_rows(b, r);
     cu_ver[r + 1] = cu_ver[r] + b->verify_len[r];
   }
   int* vt = cu_ver + (C + 1);
@@ -198,7 +231,7 @@ recg_status pack_batch(recg_ctx* ctx, const recg_batch* b, bool need_pages, bool
   int* pt = vt + Tv;
   if (pages) {
     for (int r = 0; r < C; ++r) {
-      const long long need = ((long long)b->ctx_len[r] + b->verify_len[r] + b->block_size[r] + kPageSize - 1) / kPageSize;
+      const long long need = ((long long)b->ctx_len[r] + request_rows(b, r) + kPageSize - 1) / kPageSize;
       for (int i = 0; i < stride; ++i) {
         const int pg = b->page_table[(size_t)r * stride + i];
         if (i < need && (pg < 0 || pg >= b->kv_pool_pages) && b->kv_pool)
@@ -216,7 +249,9 @@ recg_status pack_batch(recg_ctx* ctx, const recg_batch* b, bool need_pages, bool
   bl.ctx_len = d;
   bl.verify_len = d + C;
   bl.block_size = d + 2 * C;
-  bl.cu_tok = d + 3 * C;
+  bl.corr = d + 3 * C;
+  bl.cu_tok = d + 9 * C;
+  bl.risk_delta = b->risk_delta > 0.f ? b->risk_delta : 0.5f;
   bl.cu_ver = bl.cu_tok + (C + 1);
   bl.verify_tokens = bl.cu_ver + (C + 1);
   bl.page_table = pages ? bl.verify_tokens + Tv : nullptr;
@@ -470,6 +505,7 @@ recg_status recg_verify(recg_ctx* ctx, const recg_batch* batch, const void* logi
 #define PICK(f) if (out->f) vb.f = out->f
     PICK(accept_len); PICK(n_emitted); PICK(emitted); PICK(new_ctx_len); PICK(slot_state); PICK(freed_pages);
     PICK(next_draft); PICK(cont_hit); PICK(top1); PICK(top2); PICK(p1); PICK(p2); PICK(entropy); PICK(entropy_mean);
+    PICK(corr_hit); PICK(risky_n); PICK(risky_index); PICK(risky_token);
 #undef PICK
   }
   ctx->mark(-1);
@@ -482,6 +518,7 @@ recg_status recg_verify(recg_ctx* ctx, const recg_batch* batch, const void* logi
     OUT(accept_len, C); OUT(n_emitted, C); OUT(emitted, Tv); OUT(new_ctx_len, C); OUT(slot_state, T);
     OUT(freed_pages, C); OUT(next_draft, Tb); OUT(cont_hit, C); OUT(top1, T); OUT(top2, T); OUT(p1, T); OUT(p2, T);
     OUT(entropy, T); OUT(entropy_mean, C);
+    OUT(corr_hit, 2 * C); OUT(risky_n, 3 * C); OUT(risky_index, 6 * C); OUT(risky_token, 6 * C);
 #undef OUT
     CU(cudaStreamSynchronize(ctx->stream));
   }

@@ -215,7 +215,9 @@ __global__ void __launch_bounds__(128) verify_finalize_kernel(BatchLayout bl, co
   const int r = blockIdx.x;
   const int t0 = bl.cu_tok[r];
   const int v = bl.verify_len[r], b = bl.block_size[r], L = bl.ctx_len[r];
-  const int n = v + b;
+  const int* cr = bl.corr + 6 * r;              // correction branches: count, mask tokens per branch, indices, tokens
+  const int n_corr = cr[0], span = 1 + cr[1];
+  const int n = bl.cu_tok[r + 1] - t0;          // v + b + n_corr * span
   for (int j = threadIdx.x; j < n; j += blockDim.x) {
     const RowPartial* p = partials + (size_t)(t0 + j) * chunks_per_row;
     Top2 tp = {-INFINITY, -INFINITY, 0x7fffffff, 0x7fffffff};
@@ -257,6 +259,28 @@ __global__ void __launch_bounds__(128) verify_finalize_kernel(BatchLayout bl, co
     const int first_free = (new_L + kPageSize - 1) / kPageSize;
     const int last = (L + n + kPageSize - 1) / kPageSize;
     vb.freed_pages[r] = bl.page_table ? last - first_free : 0;
+    // a correction branch is confirmed when the verifier rejected exactly the draft it replaced and emitted the
+    // replacement token there (Sec. 5.1)
+    for (int k = 0; k < 2; ++k)
+      vb.corr_hit[2 * r + k] = (k < n_corr && v > 0 && a == cr[2 + k] - 1 && vb.top1[t0 + a] == cr[4 + k]) ? 1 : 0;
+    // risky drafts of every draft block, indexed as the verify tokens the block would become: the continuation's
+    // mask row m is y'_m (row 0 only confirms the bonus token), a correction's mask row m is y'_{m+1}
+    for (int j = 0; j < 3; ++j) {
+      int row0 = 0, rows = 0, first_index = 1;
+      if (j == 0) { row0 = t0 + v + 1; rows = b > 0 ? b - 1 : 0; }
+      else if (j - 1 < n_corr) { row0 = t0 + v + b + (j - 1) * span + 1; rows = span - 1; }
+      int cnt = 0;
+      int* ri = vb.risky_index + 6 * r + 2 * j;
+      int* rtk = vb.risky_token + 6 * r + 2 * j;
+      ri[0] = ri[1] = rtk[0] = rtk[1] = -1;
+      for (int m = 0; m < rows; ++m) {
+        if (vb.p1[row0 + m] - vb.p2[row0 + m] < bl.risk_delta) {
+          if (cnt < 2) { ri[cnt] = first_index + m; rtk[cnt] = vb.top2[row0 + m]; }
+          ++cnt;
+        }
+      }
+      vb.risky_n[3 * r + j] = cnt;
+    }
     s_a = a;
   }
   __syncthreads();

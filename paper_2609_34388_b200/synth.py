@@ -129,14 +129,34 @@ class BatchDescriptor:
     page_table: np.ndarray     # [C, stride] physical page ids (int32), -1 where unused
     n_pages: int               # physical pages the pool must hold
     page_size: int
+    # correction branches of the draft-verify overlap (None = none anywhere)
+    n_corr: Optional[np.ndarray] = None      # [C] 0..2
+    corr_index: Optional[np.ndarray] = None  # [C, 2] replaced draft index, increasing
+    corr_token: Optional[np.ndarray] = None  # [C, 2] replacement token ids
+    corr_block: Optional[np.ndarray] = None  # [C] mask tokens per branch
 
     @property
     def n_req(self) -> int:
         return int(self.ctx_len.shape[0])
 
     @property
+    def rows(self) -> np.ndarray:
+        """Rows of each request in the ragged batch."""
+        n = self.verify_len + self.block_size
+        if self.n_corr is not None:
+            n = n + self.n_corr * (1 + self.corr_block)
+        return n
+
+    @property
     def n_tokens(self) -> int:
-        return int((self.verify_len + self.block_size).sum())
+        return int(self.rows.sum())
+
+    def branch_kwargs(self) -> dict:
+        """The branch arguments of binding.Batch."""
+        if self.n_corr is None:
+            return {}
+        return {"n_corr": self.n_corr, "corr_index": self.corr_index, "corr_token": self.corr_token,
+                "corr_block": self.corr_block}
 
 
 def page_tables(ctx_len, n_new, page_size: int, seed: int, spare_pages: int = 0, stride: Optional[int] = None):
@@ -169,12 +189,38 @@ def batch_descriptor(n_req: int, block_choices, block_probs, ctx_lo: int, ctx_hi
     return BatchDescriptor(L, v, b, pt, total, page_size)
 
 
-def fixed_descriptor(ctx_len, verify_len, block_size, seed: int = 3, page_size: int = 16) -> BatchDescriptor:
+def fixed_descriptor(ctx_len, verify_len, block_size, seed: int = 3, page_size: int = 16, corr=None,
+                     corr_block=None) -> BatchDescriptor:
+    """corr: per request a list of up to two (draft index, replacement token); corr_block: mask tokens per branch."""
     L = np.asarray(ctx_len, dtype=np.int32)
     v = np.asarray(verify_len, dtype=np.int32)
     b = np.asarray(block_size, dtype=np.int32)
-    pt, total = page_tables(L, v + b, page_size, seed + 1000)
-    return BatchDescriptor(L, v, b, pt, total, page_size)
+    if corr is None:
+        pt, total = page_tables(L, v + b, page_size, seed + 1000)
+        return BatchDescriptor(L, v, b, pt, total, page_size)
+    nc = np.asarray([len(c) for c in corr], dtype=np.int32)
+    ci = np.zeros((len(corr), 2), dtype=np.int32)
+    ct = np.zeros((len(corr), 2), dtype=np.int32)
+    for r, c in enumerate(corr):
+        for k, (i, tok) in enumerate(c):
+            ci[r, k], ct[r, k] = i, tok
+    cb = np.asarray(corr_block, dtype=np.int32)
+    pt, total = page_tables(L, v + b + nc * (1 + cb), page_size, seed + 1000)
+    return BatchDescriptor(L, v, b, pt, total, page_size, nc, ci, ct, cb)
+
+
+def with_correction_branches(desc: BatchDescriptor, vocab: int, n_branches: int = 2, seed: int = 11) -> BatchDescriptor:
+    """The same requests with n_branches correction branches each (where the verify row has that many drafts):
+    replaced draft indices drawn without replacement from 1..v-1, replacement tokens uniform, one block of the
+    request's own size per branch, and page tables that cover the extra rows."""
+    rng = np.random.default_rng(seed)
+    corr = []
+    for v in desc.verify_len:
+        k = min(n_branches, max(int(v) - 1, 0))
+        idx = np.sort(rng.choice(np.arange(1, int(v)), size=k, replace=False)) if k else []
+        corr.append([(int(i), int(rng.integers(0, vocab - 1))) for i in idx])
+    return fixed_descriptor(desc.ctx_len, desc.verify_len, desc.block_size, seed=seed, page_size=desc.page_size,
+                            corr=corr, corr_block=desc.block_size)
 
 
 def logits_normal(rows: int, vocab: int, seed: int = 6, device="cpu", dtype=torch.bfloat16):

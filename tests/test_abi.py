@@ -28,11 +28,26 @@ def test_header_symbols_are_exported():
     assert set(names) == set(binding.EXPORTS)
 
 
-def test_struct_sizes_match_header_layout():
+def test_struct_sizes_match_header_layout(tmp_path):
     # 7 ints, 2 floats, 6 ints
     assert C.sizeof(binding.recg_config) == 15 * 4
-    assert C.sizeof(binding.recg_batch) == 8 * 8 + 8  # int + 5 ptr + int + ptr + int64 with padding
-    assert C.sizeof(binding.recg_verify_out) == 8 + 14 * 8
+    # int + 5 ptr + int + ptr + int64, then 4 ptr + float, with padding
+    assert C.sizeof(binding.recg_batch) == 8 * 8 + 8 + 4 * 8 + 8
+    assert C.sizeof(binding.recg_verify_out) == 8 + 18 * 8
+    # and against the header itself, as the C compiler lays the structs out
+    import subprocess
+    src = tmp_path / "sizes.c"
+    src.write_text('#include <stdio.h>\n#include <stddef.h>\n#include "recg.h"\n'
+                   'int main(void) { printf("%zu %zu %zu %zu %zu %zu %zu\\n", sizeof(recg_config), sizeof(recg_batch), '
+                   'sizeof(recg_verify_out), offsetof(recg_batch, n_corr), offsetof(recg_batch, risk_delta), '
+                   'offsetof(recg_verify_out, corr_hit), offsetof(recg_verify_out, risky_token)); return 0; }\n')
+    exe = tmp_path / "sizes"
+    subprocess.run(["gcc", "-I", os.path.join(ROOT, "include"), str(src), "-o", str(exe)], check=True)
+    got = [int(t) for t in subprocess.run([str(exe)], check=True, capture_output=True, text=True).stdout.split()]
+    want = [C.sizeof(binding.recg_config), C.sizeof(binding.recg_batch), C.sizeof(binding.recg_verify_out),
+            binding.recg_batch.n_corr.offset, binding.recg_batch.risk_delta.offset,
+            binding.recg_verify_out.corr_hit.offset, binding.recg_verify_out.risky_token.offset]
+    assert got == want
 
 
 def test_pool_bytes_formula():

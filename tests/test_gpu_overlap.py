@@ -1,0 +1,355 @@
+"""GPU parity of rounds with prospective correction branches (Sec. 5.1): the attention operation, the
+verification outputs and the whole round against the oracle, and a loop the GPU drives itself."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import recg_oracle as orc
+from paper_2609_34388_b200 import binding, synth
+from tests._util import bf16_round, f64, oracle_cfg, oracle_weights
+
+pytestmark = pytest.mark.gpu
+
+ATTN_TOL = 1e-2     # attention outputs, relative to max |ref|
+HID_TOL = 2e-2      # hidden states and logits, relative to max |ref|
+MARGIN_FLAG = 1e-2  # integer results may differ only where the oracle's top-2 logit gap is below this
+DELTA_FLAG = 1e-3   # a risky-position decision is compared only where |M - delta| exceeds this
+
+
+def to_dev(W):
+    return {k: ([t.cuda() for t in v] if isinstance(v, list) else v.cuda()) for k, v in W.items()}
+
+
+def run_attention_case(shape, reqs, seed, flags=0):
+    """reqs: (L, v, b, [(i, tok) ..], bc).  Returns the worst error relative to max |ref|."""
+    desc = synth.fixed_descriptor([r[0] for r in reqs], [r[1] for r in reqs], [r[2] for r in reqs], seed=seed,
+                                  corr=[r[3] for r in reqs], corr_block=[r[4] for r in reqs])
+    T = desc.n_tokens
+    one_layer = synth.ModelShape(**{**shape.as_dict(), "n_layers": 1})
+    ctx = binding.Context(binding.make_config(one_layer, len(reqs), T, desc.page_table.shape[1], flags))
+    pool = binding.alloc_kv_pool(ctx, desc.n_pages, fill=None)
+    pool.fill_(float("nan"))
+    q = synth.queries(T, shape.n_q_heads, shape.head_dim, seed=seed + 5)
+    ks, vs = [], []
+    for r, (L, v, b, corr, bc) in enumerate(reqs):
+        n = int(desc.rows[r])
+        k_, v_ = synth.kv_values(L + n, shape.n_kv_heads, shape.head_dim, seed=seed * 100 + r)
+        ks.append(k_)
+        vs.append(v_)
+        ctx.recg_kv_write(pool, desc.n_pages, 0, desc.page_table[r], 0, k_.cuda(), v_.cuda())
+    batch = binding.Batch(desc.ctx_len, desc.verify_len, desc.block_size, None, desc.page_table, pool, desc.n_pages,
+                          **desc.branch_kwargs())
+    assert batch.n_tok == T
+    o = torch.full((T, shape.n_q_heads, shape.head_dim), float("nan"), dtype=torch.bfloat16, device="cuda")
+    ctx.recg_attention(batch, 0, q.cuda(), o)
+    ctx.recg_sync()
+    got = f64(o)
+    worst, t0 = 0.0, 0
+    for r, (L, v, b, corr, bc) in enumerate(reqs):
+        n = int(desc.rows[r])
+        _, vis, _ = orc.overlap_round_rows(L, v, b, corr, bc)
+        ref = orc.attention(f64(q[t0:t0 + n]), f64(ks[r]), f64(vs[r]), vis)
+        assert not np.isnan(got[t0:t0 + n]).any(), f"NaN in request {r}"
+        worst = max(worst, np.max(np.abs(got[t0:t0 + n] - ref)) / np.max(np.abs(ref)))
+        t0 += n
+    ctx.recg_free()
+    return worst
+
+
+@pytest.mark.parametrize("flags", [0, binding.FLAG_SIMT_ATTENTION])
+def test_attention_with_correction_branches(flags):
+    shape = synth.llama8b_shape(1)
+    reqs = [(100, 8, 8, [(2, 0), (5, 0)], 8),          # the ordinary case: four logical rows
+            (61, 4, 0, [(1, 0), (3, 0)], 4),           # more than two risky positions: no continuation block
+            (0, 3, 2, [(2, 0)], 2),                    # no committed context at all
+            (17, 16, 16, [(15, 0)], 0),                # a branch that is only its replacement token
+            (1000, 32, 32, [(1, 0), (31, 0)], 32),     # rows in several tiles, branch rows far from what they see
+            (3000, 8, 8, [(4, 0)], 8),                 # long context (split over CTAs)
+            (40, 2, 8, [], 0), (7, 1, 4, [], 0)]       # requests without branches in the same batch
+    assert run_attention_case(shape, reqs, seed=21, flags=flags) < ATTN_TOL
+
+
+def test_attention_branches_head_dim_64():
+    shape = synth.tiny_shape()
+    reqs = [(50, 6, 4, [(2, 0), (3, 0)], 4), (130, 9, 8, [(8, 0)], 8), (5, 2, 0, [(1, 0)], 3)]
+    assert run_attention_case(shape, reqs, seed=22) < ATTN_TOL
+
+
+def planted_logits(top1, top2, low_margin_rows, vocab, seed):
+    """Rows of N(0,1) noise with a planted winner (+12) and runner-up (+8, or +11.5 on low-margin rows)."""
+    x = synth.logits_normal(len(top1), vocab, seed=seed, dtype=torch.float32).clone()
+    for r in range(len(top1)):
+        x[r, top1[r]] = 12.0
+        x[r, top2[r]] = 11.5 if r in low_margin_rows else 8.0
+    return x
+
+
+def test_verify_branch_reuse_and_risky_positions():
+    """Standalone verification of planted logits: every reuse outcome, the risky positions of every block."""
+    vocab = 4096
+    rng = np.random.default_rng(5)
+    cases = []   # (y, b, corr, bc, verifier top1)
+    y = [3, 4, 5, 6, 7]
+    cases.append((y, 4, [(2, 20), (4, 21)], 4, [4, 20, 9, 9, 9]))      # correction 0 confirmed
+    cases.append((y, 4, [(2, 20), (4, 21)], 4, [4, 5, 6, 21, 9]))      # correction 1 confirmed
+    cases.append((y, 4, [(2, 20), (4, 21)], 4, [4, 22, 6, 21, 9]))     # predicted position, other token
+    cases.append((y, 4, [(2, 20), (4, 21)], 4, [20, 5, 6, 7, 9]))      # replacement token at an unpredicted position
+    cases.append((y, 4, [(3, 30)], 2, [4, 5, 6, 7, 11]))               # full acceptance (continuation decides)
+    cases.append((y, 0, [(1, 30), (2, 31)], 6, [30, 5, 6, 7, 11]))     # no continuation block at all
+    cases.append(([8], 8, [], 0, [9]))                                 # request without branches
+    ys, rows_top1, rows_top2, low = [], [], [], set()
+    for (y, b, corr, bc, vt) in cases:
+        n = len(y) + b + len(corr) * (1 + bc)
+        t1 = list(vt) + rng.integers(40, vocab, size=n - len(y)).tolist()
+        if b and len(y) > 1 and vt[-1] == 11:
+            t1[len(y)] = 11                                            # first draft equals the bonus token
+        t2 = rng.integers(40, vocab, size=n).tolist()
+        t2 = [b_ if b_ != a_ else b_ + 1 for a_, b_ in zip(t1, t2)]
+        base = len(rows_top1)
+        low |= {base + j for j in range(len(y), n) if rng.random() < 0.4}
+        rows_top1 += t1
+        rows_top2 += t2
+        ys += y
+    x = planted_logits(rows_top1, rows_top2, low, vocab, seed=3)
+    desc = synth.fixed_descriptor([10] * len(cases), [len(c[0]) for c in cases], [c[1] for c in cases], seed=2,
+                                  corr=[c[2] for c in cases], corr_block=[c[3] for c in cases])
+    shape = synth.ModelShape(n_layers=0, hidden=64, n_q_heads=4, n_kv_heads=2, head_dim=64, ffn=64, vocab=vocab)
+    ctx = binding.Context(binding.make_config(shape, len(cases), desc.n_tokens, desc.page_table.shape[1]))
+    batch = binding.Batch(desc.ctx_len, desc.verify_len, desc.block_size, ys, desc.page_table, None, 0,
+                          **desc.branch_kwargs())
+    got = ctx.recg_verify(batch, x.cuda())
+    t0 = tb0 = 0
+    hits = []
+    for i, (y, b, corr, bc, vt) in enumerate(cases):
+        n = int(desc.rows[i])
+        ref = orc.verify_overlap_round(f64(x[t0:t0 + n]), y, b, corr, bc)
+        assert int(got["accept_len"][i]) == ref["accept_len"] and int(got["cont_hit"][i]) == int(ref["cont_hit"])
+        assert got["corr_hit"][2 * i: 2 * i + 2].tolist() == [int(h) for h in ref["corr_hit"]] + [0] * (2 - len(corr))
+        hits.append(got["corr_hit"][2 * i: 2 * i + 2].tolist())
+        assert got["next_draft"][tb0:tb0 + n - len(y)].tolist() == [s["top1"] for s in ref["stats"][len(y):]]
+        for j in range(3):
+            want = ref["risky"][j] if j < len(ref["risky"]) else (0, [])
+            assert int(got["risky_n"][3 * i + j]) == want[0], (i, j)
+            idx = [k for k, _ in want[1]] + [-1] * (2 - len(want[1]))
+            tok = [t for _, t in want[1]] + [-1] * (2 - len(want[1]))
+            assert got["risky_index"][6 * i + 2 * j: 6 * i + 2 * j + 2].tolist() == idx, (i, j)
+            assert got["risky_token"][6 * i + 2 * j: 6 * i + 2 * j + 2].tolist() == tok, (i, j)
+        # commit / rollback: branch rows never stay
+        kc = orc.kv_commit(10, len(y), n - len(y), ref["accept_len"], desc.page_table[i], 16)
+        ss = got["slot_state"][t0:t0 + n].tolist()
+        assert [s for s in ss if s >= 0] == kc["commit_slots"]
+        assert [-(s + 1) for s in ss if s < 0] == kc["rollback_slots"]
+        assert int(got["freed_pages"][i]) == len(kc["freed_pages"])
+        t0 += n
+        tb0 += n - len(y)
+    assert hits[:6] == [[1, 0], [0, 1], [0, 0], [0, 0], [0, 0], [1, 0]]
+    assert int(got["cont_hit"][4]) == 1
+    # another threshold through the batch descriptor
+    batch = binding.Batch(desc.ctx_len, desc.verify_len, desc.block_size, ys, desc.page_table, None, 0,
+                          risk_delta=0.999, **desc.branch_kwargs())
+    got = ctx.recg_verify(batch, x.cuda())
+    for i, (y, b, corr, bc, vt) in enumerate(cases):
+        assert int(got["risky_n"][3 * i]) == max(b - 1, 0)
+        for k in range(len(corr)):
+            assert int(got["risky_n"][3 * i + 1 + k]) == bc
+    ctx.recg_free()
+
+
+def test_host_side_rejections_of_branches():
+    shape = synth.ModelShape(n_layers=0, hidden=64, n_q_heads=4, n_kv_heads=2, head_dim=64, ffn=64, vocab=512)
+    ctx = binding.Context(binding.make_config(shape, 2, 64, 4))
+    x = synth.logits_normal(64, 512, seed=1, dtype=torch.float32).cuda()
+
+    def bad(**kw):
+        args = dict(n_corr=[1], corr_index=[[2, 0]], corr_token=[[5, 0]], corr_block=[4])
+        args.update(kw)
+        b = binding.Batch([10], [4], [4], [1, 2, 3, 4], None, None, 0, **args)
+        with pytest.raises(binding.RecgError):
+            ctx.recg_verify(b, x)
+
+    bad(n_corr=[3])
+    bad(corr_index=[[0, 0]])                       # y_0 is not a draft
+    bad(corr_index=[[4, 0]])                       # beyond the verify tokens
+    bad(n_corr=[2], corr_index=[[2, 2]])           # not increasing
+    bad(corr_token=[[512, 0]])
+    bad(corr_block=[-1])
+    bad(corr_block=[60])                           # more rows than max_tokens
+    ok = binding.Batch([10], [4], [4], [1, 2, 3, 4], None, None, 0, n_corr=[1], corr_index=[[2, 0]],
+                       corr_token=[[5, 0]], corr_block=[4])
+    ctx.recg_verify(ok, x)
+    ctx.recg_free()
+
+
+def tiny_model():
+    shape = synth.tiny_shape()
+    W = synth.model_weights(shape, seed=0, dtype=torch.bfloat16)
+    synth.perturb_norm_gains(W)
+    return shape, W, oracle_cfg(shape), oracle_weights(W)
+
+
+@pytest.mark.parametrize("flags", [0, binding.FLAG_SIMT_GEMM | binding.FLAG_SIMT_ATTENTION])
+def test_tiny_round_with_correction_branches(flags):
+    """Whole round, ragged batch, all four logical rows: hidden states, logits and tentative K/V of every row
+    against the oracle's forward over the same rows; integers against the oracle's rules applied to the
+    kernel's own logits (exact) and to the oracle's logits (where its logit gap is clear)."""
+    shape, W, ocfg, W64 = tiny_model()
+    # (L, v, b, planted first mismatch m or None, [(i, token or 'truth')], bc)
+    specs = [(40, 8, 8, 3, [(2, 77), (4, "truth")], 8),    # correction 1 predicts position and token
+             (63, 6, 0, 1, [(1, 5), (2, "truth"), ], 4),   # no continuation; correction 1 confirmed
+             (17, 5, 4, 4, [(3, 9)], 4),                   # fully accepted: the branch is discarded
+             (100, 4, 4, 0, [(1, 3)], 2),                  # rejected where predicted, with another token
+             (5, 1, 8, None, [], 0),                       # no drafts, hence no branches
+             (33, 8, 8, None, [(1, 100), (7, 200)], 8)]    # random drafts
+    reqs, corr_all = [], []
+    for i, (L, v, b, m, corr, bc) in enumerate(specs):
+        prompt = synth.token_ids(L + 1, shape.vocab, seed=500 + i).tolist()
+        kv, L0, y0 = orc.prefill(ocfg, W64, prompt)
+        kv = [(bf16_round(K), bf16_round(V)) for (K, V) in kv]
+        truth = orc.greedy_ar(ocfg, W64, prompt, v) if (m is not None and v > 1) else []
+        if m is None:
+            y = y0 + synth.token_ids(v - 1, shape.vocab, seed=550 + i).tolist()
+        else:
+            y = y0 + truth[: v - 1]
+            if m + 1 <= v - 1:
+                y[m + 1] = (y[m + 1] + 1) % (shape.vocab - 1)
+        corr = [(j, truth[j - 1] if tok == "truth" else tok) for (j, tok) in corr]
+        reqs.append({"kv": kv, "y": y, "L": L, "v": v, "b": b, "m": m, "corr": corr, "bc": bc})
+        corr_all.append(corr)
+    desc = synth.fixed_descriptor([s[0] for s in specs], [s[1] for s in specs], [s[2] for s in specs], seed=9,
+                                  corr=corr_all, corr_block=[s[5] for s in specs])
+    ctx = binding.Context(binding.make_config(shape, 8, 160, desc.page_table.shape[1], flags), to_dev(W))
+    pool = binding.alloc_kv_pool(ctx, desc.n_pages, fill=None)
+    pool.fill_(float("nan"))
+    for i, r in enumerate(reqs):
+        for l, (K, V) in enumerate(r["kv"]):
+            ctx.recg_kv_write(pool, desc.n_pages, l, desc.page_table[i], 0,
+                              torch.from_numpy(K).to(torch.bfloat16).cuda(), torch.from_numpy(V).to(torch.bfloat16).cuda())
+    ys = [t for r in reqs for t in r["y"]]
+    batch = binding.Batch(desc.ctx_len, desc.verify_len, desc.block_size, ys, desc.page_table, pool, desc.n_pages,
+                          **desc.branch_kwargs())
+    lg = ctx.recg_step(batch)
+    got = ctx.recg_verify(batch)
+    ctx.recg_sync()
+    logits = f64(ctx.logits_tensor(lg))
+    hidden = f64(ctx.recg_debug_buffer(0))
+    assert logits.shape[0] == desc.n_tokens
+    t0 = tb0 = 0
+    hits = []
+    for i, r in enumerate(reqs):
+        L, v, b, corr, bc = r["L"], r["v"], r["b"], r["corr"], r["bc"]
+        n = int(desc.rows[i])
+        ref_logits, ref_kv, ref_h = orc.overlap_round_cached(ocfg, W64, r["kv"], L, r["y"], b, corr, bc)
+        assert np.max(np.abs(hidden[t0:t0 + n] - ref_h)) <= HID_TOL * np.max(np.abs(ref_h)), f"hidden, request {i}"
+        for lo, hi, what in [(0, v + b, "canonical rows")] + \
+                [(v + b + k * (1 + bc), v + b + (k + 1) * (1 + bc), f"branch {k}") for k in range(len(corr))]:
+            err = np.max(np.abs(logits[t0 + lo:t0 + hi] - ref_logits[lo:hi]))
+            assert err <= HID_TOL * np.max(np.abs(ref_logits)), f"logits of {what}, request {i}"
+        for l, (K, V) in enumerate(ref_kv):
+            kg, vg = ctx.recg_kv_read(pool, desc.n_pages, l, desc.page_table[i], L, n)
+            assert np.max(np.abs(f64(kg) - K[L:])) <= HID_TOL * np.max(np.abs(K[L:])), f"K layer {l} request {i}"
+            assert np.max(np.abs(f64(vg) - V[L:])) <= HID_TOL * np.max(np.abs(V[L:])), f"V layer {l} request {i}"
+        # integers from the kernel's own logits: exact
+        own = orc.verify_overlap_round(logits[t0:t0 + n], r["y"], b, corr, bc)
+        assert got["top1"][t0:t0 + n].tolist() == [s["top1"] for s in own["stats"]]
+        assert got["top2"][t0:t0 + n].tolist() == [s["top2"] for s in own["stats"]]
+        assert int(got["accept_len"][i]) == own["accept_len"] and int(got["cont_hit"][i]) == int(own["cont_hit"])
+        assert got["corr_hit"][2 * i: 2 * i + 2].tolist() == [int(h) for h in own["corr_hit"]] + [0] * (2 - len(corr))
+        hits.append(got["corr_hit"][2 * i: 2 * i + 2].tolist())
+        assert got["next_draft"][tb0:tb0 + n - v].tolist() == [s["top1"] for s in own["stats"][v:]]
+        margins = np.array([s["margin"] for s in own["stats"]])
+        blocks = [(v + 1, v + b)] + [(v + b + k * (1 + bc) + 1, v + b + (k + 1) * (1 + bc)) for k in range(len(corr))]
+        for j, (lo, hi) in enumerate(blocks):
+            if hi > lo and (np.abs(margins[lo:hi] - orc.DELTA_RISKY) > DELTA_FLAG).all():
+                want = own["risky"][j]
+                assert int(got["risky_n"][3 * i + j]) == want[0]
+                assert got["risky_index"][6 * i + 2 * j: 6 * i + 2 * j + 2].tolist() == \
+                    [k for k, _ in want[1]] + [-1] * (2 - len(want[1]))
+                assert got["risky_token"][6 * i + 2 * j: 6 * i + 2 * j + 2].tolist() == \
+                    [t for _, t in want[1]] + [-1] * (2 - len(want[1]))
+        kc = orc.kv_commit(L, v, n - v, own["accept_len"], desc.page_table[i], 16)
+        ss = got["slot_state"][t0:t0 + n].tolist()
+        assert int(got["new_ctx_len"][i]) == kc["new_ctx_len"] and int(got["freed_pages"][i]) == len(kc["freed_pages"])
+        assert [s for s in ss if s >= 0] == kc["commit_slots"] and [-(s + 1) for s in ss if s < 0] == kc["rollback_slots"]
+        # against the oracle's own forward, where its logit gaps are clear
+        ref = orc.verify_overlap_round(ref_logits, r["y"], b, corr, bc)
+        gaps = np.array([s["logit_gap"] for s in ref["stats"]])
+        clear = gaps >= MARGIN_FLAG
+        for j in range(n):
+            if clear[j]:
+                assert int(got["top1"][t0 + j]) == ref["stats"][j]["top1"], f"top1 row {j} request {i}"
+        if v and clear[: min(ref["accept_len"] + 1, v)].all():
+            assert own["accept_len"] == ref["accept_len"] and own["corr_hit"] == ref["corr_hit"]
+            if r["m"] is not None:
+                assert ref["accept_len"] == r["m"]
+        t0 += n
+        tb0 += n - v
+    assert hits[0] == [0, 1] and hits[1] == [0, 1] and hits[2] == [0, 0] and hits[3] == [0, 0]
+    # the canonical rows do not notice the branches: the same batch without them gives the same verifier outcome
+    plain = binding.Batch(desc.ctx_len, desc.verify_len, desc.block_size, ys, desc.page_table, pool, desc.n_pages)
+    ctx.recg_step(plain)
+    g0 = ctx.recg_verify(plain)
+    assert g0["accept_len"].tolist() == got["accept_len"].tolist()
+    assert g0["cont_hit"].tolist() == got["cont_hit"].tolist()
+    ctx.recg_sync()
+    ctx.recg_free()
+
+
+def test_tiny_overlap_loop_is_lossless():
+    """The GPU drives the recursive overlap itself: every round's branches come from the risky positions its own
+    previous verification reported, confirmed branches supply the next verify tokens.  The emitted text must be
+    the oracle's greedy continuation, and at least one correction branch must have been reused on the way."""
+    shape, W, ocfg, W64 = tiny_model()
+    prompt = synth.token_ids(48, shape.vocab, seed=2).tolist()
+    b, rounds = 8, 8
+    ar = orc.greedy_ar(ocfg, W64, prompt, rounds * (b + 1) + b)
+    kv, L, y = orc.prefill(ocfg, W64, prompt)
+    pt, n_pages = synth.page_tables([L], [rounds * (b + 1) + 4 * (b + 1)], 16, seed=3)
+    ctx = binding.Context(binding.make_config(shape, 1, 64, pt.shape[1]), to_dev(W))
+    pool = binding.alloc_kv_pool(ctx, n_pages, fill=None)
+    pool.fill_(float("nan"))
+    for l, (K, V) in enumerate(kv):
+        ctx.recg_kv_write(pool, n_pages, l, pt[0], 0, torch.from_numpy(K).to(torch.bfloat16).cuda(),
+                          torch.from_numpy(V).to(torch.bfloat16).cuda())
+    out, used = [], []
+    corr, cont = [], True
+    for t in range(rounds):
+        if t % 3 == 1:
+            # teacher-forced drafts with one wrong token whose replacement candidate is the right one: the
+            # situation the correction branch exists for
+            y = [y[0]] + ar[len(out): len(out) + 5]
+            truth = y[3]
+            y[3] = (truth + 1) % (shape.vocab - 1)
+            corr, cont = [(3, truth)], True
+        bb = b if cont else 0
+        batch = binding.Batch([L], [len(y)], [bb], y, pt, pool, n_pages, n_corr=[len(corr)],
+                              corr_index=[[c[0] for c in corr] + [0] * (2 - len(corr))],
+                              corr_token=[[c[1] for c in corr] + [0] * (2 - len(corr))], corr_block=[b])
+        ctx.recg_step(batch)
+        g = ctx.recg_verify(batch)
+        a = int(g["accept_len"][0])
+        out += g["emitted"][: a + 1].tolist()
+        L = int(g["new_ctx_len"][0])
+        bonus = int(g["emitted"][a])
+        v = len(y)
+        nd = g["next_draft"].tolist()
+        if int(g["cont_hit"][0]):
+            j, y = 0, [bonus] + nd[1:bb]
+        elif g["corr_hit"][:2].any():
+            k = int(np.argmax(g["corr_hit"][:2]))
+            j, r0 = 1 + k, bb + k * (1 + b)
+            y = [bonus] + nd[r0 + 1: r0 + 1 + b]
+        else:
+            j, y = -1, [bonus]
+        used.append(j)
+        if j >= 0:
+            nr = int(g["risky_n"][j])
+            corr = [(int(g["risky_index"][2 * j + q]), int(g["risky_token"][2 * j + q])) for q in range(min(nr, 2))]
+            cont = nr <= 2
+        else:
+            corr, cont = [], True
+        if t % 3 == 1:
+            assert a == 2 and j == 1
+    ctx.recg_sync()
+    assert out == ar[: len(out)], (out, ar[: len(out)])
+    assert 1 in used
+    ctx.recg_free()
