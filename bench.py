@@ -115,10 +115,9 @@ def algorithmic_counts(shape, desc):
     flops["lm_head"] = 2.0 * T * V * H
     wbytes = {k: 2.0 * p * nl for k, p in w_params.items()}
     wbytes["lm_head"] = 2.0 * V * H
-    kv_tokens = float((desc.ctx_len + desc.verify_len + desc.block_size).sum())
+    kv_tokens = float((desc.ctx_len + desc.rows).sum())
     attn_bytes = nl * (kv_tokens * nkv * d * 2 * 2 + 2.0 * T * nq * d * 2)   # K+V once per layer, q in, o out
-    attn_flops = nl * 4.0 * d * nq * float(((desc.ctx_len + desc.verify_len + desc.block_size) *
-                                             (desc.verify_len + desc.block_size)).sum())
+    attn_flops = nl * 4.0 * d * nq * float(((desc.ctx_len + desc.rows) * desc.rows).sum())
     logits_bytes = 4.0 * T * V
     return {"T": T, "flops": flops, "wbytes": wbytes, "attn_bytes": attn_bytes, "attn_flops": attn_flops,
             "verify_bytes": logits_bytes}
@@ -210,7 +209,7 @@ def run_ours(args, env):
     env.barrier()
     e2e_ms = env.max_float(max(e0.elapsed_time(e1), wall_ms))
     b0 = batches[0]
-    h2d = 4 * (3 * b0.n_req + 2 * (b0.n_req + 1) + b0.n_ver + b0.page_table.size)
+    h2d = 4 * (9 * b0.n_req + 2 * (b0.n_req + 1) + b0.n_ver + b0.page_table.size)
     d2h = outs_host[0].nbytes()
     e2e_value = tokens_all / (e2e_ms / 1e3)
 
@@ -306,7 +305,8 @@ def bench_attention_op(binding, peaks, args, desc=None, n_layers=32, label=None)
     with torch.cuda.stream(stream):
         ctx = binding.Context(binding.make_config(shape, desc.n_req, T, desc.page_table.shape[1]), stream=stream.cuda_stream)
         pool = binding.alloc_kv_pool(ctx, desc.n_pages, fill="normal")
-        batch = binding.Batch(desc.ctx_len, desc.verify_len, desc.block_size, None, desc.page_table, pool, desc.n_pages)
+        batch = binding.Batch(desc.ctx_len, desc.verify_len, desc.block_size, None, desc.page_table, pool, desc.n_pages,
+                              **desc.branch_kwargs())
         q = synth.queries(T, 32, 128, seed=5, device="cuda")
         o = torch.empty_like(q)
         ctx.recg_attention(batch, 0, q, o)
@@ -317,7 +317,7 @@ def bench_attention_op(binding, peaks, args, desc=None, n_layers=32, label=None)
             ctx.recg_attention(None, l, q, o)
 
     us = _time_graph(stream, rotation, 10) / n_layers
-    kv_tok = float((desc.ctx_len + desc.verify_len + desc.block_size).sum())
+    kv_tok = float((desc.ctx_len + desc.rows).sum())
     kv_bytes = kv_tok * 8 * 128 * 2 * 2 + 2 * T * 32 * 128 * 2
     ctx.recg_sync()
     ctx.recg_free()
@@ -404,7 +404,11 @@ def bench_c128(binding, W, shape, peaks, args):
     desc = c128_descriptor(5)
     # the same context and pool also serve the concurrency sweep below (configs[2]'s recipe at other batch sizes)
     sweep_descs = {C: synth.batch_descriptor(C, [4, 8, 16, 32], None, 512, 8192, seed=40 + C) for C in (1, 2, 4, 8, 16, 32, 64, 128)}
-    all_descs = [desc] + list(sweep_descs.values())
+    # rounds with prospective correction branches (two per request, one block of the request's size each), and
+    # the same requests without them
+    ov_plain = {"c16": c16_descriptor(3), "c1": c1_descriptor(11)}
+    ov_descs = {k: synth.with_correction_branches(d, shape.vocab, 2, seed=60) for k, d in ov_plain.items()}
+    all_descs = [desc] + list(sweep_descs.values()) + list(ov_descs.values())
     n_pages = max(d.n_pages for d in all_descs)
     free_b, _ = torch.cuda.mem_get_info()
     cfg = binding.make_config(shape, 128, max(2048, max(d.n_tokens for d in all_descs)), max(d.page_table.shape[1] for d in all_descs))
@@ -436,7 +440,7 @@ def bench_c128(binding, W, shape, peaks, args):
         torch.cuda.synchronize()
         msw = e0.elapsed_time(e1) / n_it
         cw = algorithmic_counts(shape, d)
-        sweep.append({"concurrency": C, "tokens_per_step": bt.n_tok, "kv_tokens": int(np.sum(d.ctx_len + d.verify_len + d.block_size)),
+        sweep.append({"concurrency": C, "tokens_per_step": bt.n_tok, "kv_tokens": int(np.sum(d.ctx_len + d.rows)),
                       "ms_per_step": round(msw, 3), "tokens_per_s": round(bt.n_tok / (msw / 1e3), 1),
                       "ideal_ms": round(max(sum(cw["wbytes"].values()) / peaks["hbm_gbs"] / 1e6,
                                             sum(cw["flops"].values()) / peaks["bf16_tflops_sustained"] / 1e9) +
@@ -444,6 +448,43 @@ def bench_c128(binding, W, shape, peaks, args):
     sweep_result = {"workload": "configs[2] recipe at other batch sizes, one draw each, processed tokens/s of the whole step; "
                                             "ideal_ms = max(weight stream, GEMM flops at sustained peak) + KV stream, of measured peaks",
                                 "points": sweep}
+    overlap = {}
+    for key in ov_descs:
+        res = {}
+        for kind, d in (("plain", ov_plain[key]), ("branches", ov_descs[key])):
+            ysw = synth.token_ids(int(d.verify_len.sum()), shape.vocab, seed=70)
+            bt = binding.Batch(d.ctx_len, d.verify_len, d.block_size, ysw, d.page_table, pool, n_pages, **d.branch_kwargs())
+            vo = binding.VerifyOut(bt.n_req, bt.n_tok, bt.n_ver, host=False)
+            for _ in range(3):
+                ctx.recg_step(bt)
+                ctx.recg_verify(bt, out=vo)
+            torch.cuda.synchronize()
+            n_it = 5
+            e0.record()
+            for _ in range(n_it):
+                ctx.recg_step(bt)
+                ctx.recg_verify(bt, out=vo)
+            e1.record()
+            torch.cuda.synchronize()
+            msw = e0.elapsed_time(e1) / n_it
+            ctx.recg_timing_enable(True)
+            ctx.recg_timing_read()
+            for _ in range(n_it):
+                ctx.recg_step(bt)
+                ctx.recg_verify(bt, out=vo)
+            cms, _ = ctx.recg_timing_read()
+            ctx.recg_timing_enable(False)
+            cw = algorithmic_counts(shape, d)
+            att = cms["attention"] / n_it
+            res[kind] = {"rows_per_step": bt.n_tok, "ms_per_step": round(msw, 3), "rows_per_s": round(bt.n_tok / (msw / 1e3), 1),
+                         "attention_ms": round(att, 3), "attention_gbs": round(cw["attn_bytes"] / (att / 1e3) / 1e9, 1),
+                         "attention_frac_of_hbm_measured": round(cw["attn_bytes"] / (att / 1e3) / 1e9 / peaks["hbm_gbs"], 4)}
+        res["step_time_ratio"] = round(res["branches"]["ms_per_step"] / res["plain"]["ms_per_step"], 3)
+        overlap[key] = res
+    overlap_result = {"workload": "configs[2] draw 0 (c16) and the concurrency-1 case (c1) with two correction branches per request "
+                                  "(replaced draft indices drawn at random, one block of the request's size per branch) beside the "
+                                  "same requests without branches; attention bytes count a request's K/V once per layer for all "
+                                  "of its rows", "points": overlap}
     vout = binding.VerifyOut(batch.n_req, batch.n_tok, batch.n_ver, host=False)
     for _ in range(3):
         ctx.recg_step(batch)
@@ -480,6 +521,7 @@ def bench_c128(binding, W, shape, peaks, args):
            "attention": {"ms_per_step": round(attn_ms, 3), "gbs": round(attn_gbs, 1),
                          "frac_of_hbm_measured": round(attn_gbs / peaks["hbm_gbs"], 4)}}
     out["concurrency_sweep"] = sweep_result
+    out["overlap_branches"] = overlap_result
     ctx.recg_free()
     del pool
     torch.cuda.empty_cache()
@@ -600,7 +642,7 @@ def main():
     ap.add_argument("--steps", type=int, default=8)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--only", default="", help="comma list of op-level sections to run alone (attention_op, attention_c16, verify_sweep, gemm_shapes): "
+    ap.add_argument("--only", default="", help="comma list of op-level sections to run alone (attention_op, attention_c16, attention_c16_branches, verify_sweep, gemm_shapes): "
                                                "small cases for profiling; prints their JSON and exits")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
@@ -622,6 +664,11 @@ def main():
                 res[sec] = bench_attention_op(binding, peaks, args, desc=c16_descriptor(3), n_layers=4,
                                               label="attention of configs[2]: 16 requests, blocks U{4,8,16,32}, context "
                                                     "U[512,8192], 4 layer caches rotated, CUDA-graph replay")
+            elif sec == "attention_c16_branches":
+                res[sec] = bench_attention_op(binding, peaks, args, n_layers=4,
+                                              desc=synth.with_correction_branches(c16_descriptor(3), 128256, 2, seed=60),
+                                              label="attention of configs[2] draw 0 with two correction branches per request "
+                                                    "(784 rows instead of 376), 4 layer caches rotated, CUDA-graph replay")
             elif sec == "verify_sweep":
                 res[sec] = bench_verify(binding, peaks)
             elif sec == "gemm_shapes":
