@@ -20,6 +20,7 @@ What follows the paper, and where:
 * risky positions (M_i < delta, earliest two), correction
   branches with the second candidate, their reuse rule, and
   the recursive loop over verifier + up to three branches       -- Sec. 5.1
+* the certainty state and the table-lookup block-size rule      -- Sec. 5.2, Eq. 2-3
 
 The backbone itself (RMSNorm, rotary embedding with rotate-half pairing,
 grouped-query attention, SwiGLU, untied LM head) is the generic Llama-style
@@ -33,7 +34,9 @@ speculation against token-by-token greedy decoding, cached == dense, closed
 forms for the statistics, and planted accept lengths; for the branches, each
 branch row against the standalone round it hypothesises, visibility by brute
 force, planted selection / reuse cases and losslessness of the recursive loop
-(tests/test_oracle_overlap.py).  No value printed in the
+(tests/test_oracle_overlap.py); for the block-size rule, pairwise comparisons
+on a closed-form acceptance model, the limits of the cost weight, ties and
+bin edges (tests/test_oracle_policy.py).  No value printed in the
 paper exists for this path, so numeric parity with the paper itself is
 unpinned; parity is with these definitions.
 """
@@ -604,3 +607,58 @@ def spec_decode_overlap(cfg: ModelConfig, W: Weights, prompt: Sequence[int], b: 
         y = y_next
         L = new_L
     return out, trace
+
+
+# --------------------------------------------------------------------------
+# verification-guided adaptive drafting: the block-size rule (Sec. 5.2, Eq. 2-3)
+# --------------------------------------------------------------------------
+# The calibrated estimate V_B(s, z) is a table: the certainty s is binned by
+# ascending edges (bin = number of edges <= s), z = (index of the previous
+# block size among the candidates, full-acceptance flag).  cost[B] is
+# rho_C * T_C(B), the profiled execution cost at the current load, already
+# weighted.  value has shape [n_blocks (candidate B), n_bins, n_blocks (previous
+# B), 2 (F)].
+def policy_certainty(e1, e2, dtype=F64):
+    """s_t = -(e_{t-1} + e_{t-2}) / 2 (Eq. 2), evaluated in `dtype`."""
+    e1 = np.asarray(e1, dtype=dtype)
+    e2 = np.asarray(e2, dtype=dtype)
+    return (e1 + e2) * dtype(-0.5)
+
+
+def policy_select(s, prev_index: int, full: int, blocks: Sequence[int], s_edges, value, cost, dtype=F64):
+    """B* = argmax_B [V_B(s, z) - rho_C T_C(B)] (Eq. 3); the first maximum wins,
+    i.e. the smaller block on a tie.  Returns (index into blocks, B*)."""
+    edges = np.asarray(s_edges, dtype=dtype)
+    k = int(np.sum(edges <= dtype(s)))
+    value = np.asarray(value, dtype=dtype)
+    cost = np.asarray(cost, dtype=dtype)
+    score = [value[j, k, prev_index, int(full)] - cost[j] for j in range(len(blocks))]
+    best = 0
+    for j in range(1, len(blocks)):
+        if score[j] > score[best]:
+            best = j
+    return best, int(blocks[best])
+
+
+def policy_step(state: Dict[str, list], entropy_mean, accept_len, verify_len, blocks, s_edges, value, cost,
+                dtype=F64):
+    """One request-wise update after a finished round, then the choice for the next one.
+
+    state holds per request e1 = e_{t-1}, e2 = e_{t-2}, block_index (the block
+    size chosen last time, the B_{t-1} of Eq. 2) and full (F_{t-1}).  A round
+    that verified at least one token shifts its mean verifier entropy into the
+    history; F is set when the round verified drafts and accepted all of them.
+    Returns the chosen block sizes; state is updated in place.
+    """
+    out = []
+    for r in range(len(state["e1"])):
+        v, a = int(verify_len[r]), int(accept_len[r])
+        if v > 0:
+            state["e2"][r] = state["e1"][r]
+            state["e1"][r] = dtype(entropy_mean[r])
+            state["full"][r] = 1 if (v > 1 and a == v - 1) else 0
+        s = policy_certainty(state["e1"][r], state["e2"][r], dtype)
+        j, B = policy_select(s, state["block_index"][r], state["full"][r], blocks, s_edges, value, cost, dtype)
+        state["block_index"][r] = j
+        out.append(B)
+    return out

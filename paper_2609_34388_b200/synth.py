@@ -256,3 +256,25 @@ def plant_drafts(row_argmax: np.ndarray, n_req: int, k: int, accept: np.ndarray,
                 wrong = (wrong + 1) % (vocab - 1)
             y[r, a + 1] = wrong
     return y.astype(np.int32)
+
+
+def policy_table(blocks=(8, 16, 32), n_bins: int = 12, rho_cost=(0.9, 1.5, 2.6), seed: int = 13):
+    """A synthetic stand-in for the calibrated estimate V_B(s, z) of the block-size rule and for the weighted
+    execution cost rho_C * T_C(B): certainty bin edges evenly spaced over s in [-3, 0], and a value that grows with
+    certainty and with the candidate block, a little more after a fully accepted block, plus seeded noise so that
+    no two entries tie.  Shapes: value [n_blocks, n_bins, n_blocks, 2], cost [n_blocks].  Calibration data of the
+    paper's models is not available; only the shape of the lookup matters here."""
+    rng = np.random.default_rng(seed)
+    nb = len(blocks)
+    edges = np.linspace(-3.0, 0.0, n_bins + 1)[1:-1].astype(np.float32)
+    centre = np.linspace(-3.0, 0.0, n_bins + 1)[:-1] + 1.5 / n_bins
+    p = 1.0 / (1.0 + np.exp(-(2.0 * centre + 4.0)))                    # per-token acceptance grows with certainty
+    value = np.zeros((nb, n_bins, nb, 2), dtype=np.float32)
+    for j, B in enumerate(blocks):
+        for k in range(n_bins):
+            for jp in range(nb):
+                for f in (0, 1):
+                    pk = min(0.995, p[k] * (1.0 + 0.05 * f) * (1.0 + 0.01 * jp))
+                    value[j, k, jp, f] = (1.0 - pk ** B) / (1.0 - pk) + 0.01 * rng.standard_normal()
+    return {"blocks": np.asarray(blocks, dtype=np.int32), "s_edges": edges, "value": value,
+            "cost": np.asarray(rho_cost, dtype=np.float32)}
