@@ -521,6 +521,23 @@ def bench_c128(binding, W, shape, peaks, args):
            "attention": {"ms_per_step": round(attn_ms, 3), "gbs": round(attn_gbs, 1),
                          "frac_of_hbm_measured": round(attn_gbs / peaks["hbm_gbs"], 4)}}
     out["concurrency_sweep"] = sweep_result
+    # block-size rule on the device after the verification of the 128-request batch (one small kernel; launch bound)
+    tb = synth.policy_table()
+    ctx.recg_policy_load(tb["blocks"], tb["s_edges"], tb["value"], tb["cost"])
+    pst = {"e1": torch.zeros(128, dtype=torch.float32, device="cuda"), "e2": torch.zeros(128, dtype=torch.float32, device="cuda"),
+           "block_index": torch.zeros(128, dtype=torch.int32, device="cuda"), "full": torch.zeros(128, dtype=torch.int32, device="cuda")}
+    nxt = torch.zeros(128, dtype=torch.int32, device="cuda")
+    for _ in range(10):
+        ctx.recg_policy_step(pst, nxt, vout.bufs["entropy_mean"], vout.bufs["accept_len"])
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(200):
+        ctx.recg_policy_step(pst, nxt, vout.bufs["entropy_mean"], vout.bufs["accept_len"])
+    e1.record()
+    torch.cuda.synchronize()
+    out["policy_step"] = {"workload": "block-size rule for 128 requests, 3 candidates x 12 certainty bins, back-to-back launches",
+                          "us_per_call": round(e0.elapsed_time(e1) / 200 * 1e3, 2),
+                          "share_of_step": round(e0.elapsed_time(e1) / 200 / ms, 6)}
     out["overlap_branches"] = overlap_result
     ctx.recg_free()
     del pool

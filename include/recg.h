@@ -257,6 +257,46 @@ recg_status recg_timing_enable(recg_ctx *ctx, int32_t enable);
 recg_status recg_timing_read(recg_ctx *ctx, float *ms, int32_t *launches);
 
 /*
+ * Verification-guided choice of the next block size (Sec. 5.2, Eq. 2-3), on the device.
+ *
+ * recg_policy_load() copies a lookup table into the context (HOST arrays, copied by the call):
+ *   blocks[n_blocks]   candidate block sizes, ascending (the paper uses 8, 16, 32); n_blocks <= 8
+ *   s_edges[n_bins-1]  ascending edges of the certainty bins; s falls into bin (number of edges <= s); n_bins <= 64
+ *   value              float32 [n_blocks][n_bins][n_blocks][2]: the calibrated estimate V_B(s, z) of the
+ *                      expected accepted progress, indexed [candidate B][bin of s][previous block][F]
+ *   cost[n_blocks]     rho_C * T_C(B): the profiled execution cost of each candidate at the current load,
+ *                      already weighted
+ * recg_policy_step() runs after recg_verify() on the batch laid out last.  Per request r (state arrays are
+ * DEVICE, caller-owned, [n_req], carried from round to round; the caller initialises them):
+ *   if v_r > 0:  e2 <- e1;  e1 <- entropy_mean[r];  full <- (v_r > 1 and accept_len[r] == v_r - 1)
+ *   s = -(e1 + e2) / 2                                                     (Eq. 2, float32)
+ *   j* = argmax_j  value[j][bin(s)][block_index][full] - cost[j]           (Eq. 3; the first maximum wins)
+ *   next_block[r] = blocks[j*];  block_index <- j*
+ * entropy_mean / accept_len: DEVICE [n_req], or NULL for the library's own buffers, which hold the results
+ * of the last recg_verify() unless that call was given DEVICE output pointers for these two fields.
+ * next_block: DEVICE int32 [n_req].  Does not synchronise and copies nothing to the host.
+ * Errors: RECG_ERR_INVALID_ARG (no table loaded, no batch laid out, null pointers, table out of limits or
+ * not ascending).
+ */
+#define RECG_POLICY_MAX_BLOCKS 8
+#define RECG_POLICY_MAX_BINS 64
+typedef struct {
+  int32_t n_blocks, n_bins;
+  const int32_t *blocks;
+  const float *s_edges;
+  const float *value;
+  const float *cost;
+} recg_policy_table;
+typedef struct {
+  float *e1, *e2;       /* e_{t-1}, e_{t-2} */
+  int32_t *block_index; /* index of B_{t-1} among the candidates */
+  int32_t *full;        /* F_{t-1} */
+} recg_policy_state;
+recg_status recg_policy_load(recg_ctx *ctx, const recg_policy_table *table);
+recg_status recg_policy_step(recg_ctx *ctx, const recg_policy_state *state, const float *entropy_mean,
+                             const int32_t *accept_len, int32_t *next_block);
+
+/*
  * Per-row logit statistics with no allocation anywhere (the paper has no counterpart: this entry point
  * exists for callers that are not allowed to allocate device memory).
  *

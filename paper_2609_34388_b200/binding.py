@@ -64,6 +64,15 @@ class recg_verify_out(C.Structure):
     _fields_ = [("mem", C.c_int32)] + [(n, C.c_void_p) for n in _INT_OUT + _FLT_OUT + _INT_OUT_BRANCH]
 
 
+class recg_policy_table(C.Structure):
+    _fields_ = [("n_blocks", C.c_int32), ("n_bins", C.c_int32), ("blocks", C.c_void_p), ("s_edges", C.c_void_p),
+                ("value", C.c_void_p), ("cost", C.c_void_p)]
+
+
+class recg_policy_state(C.Structure):
+    _fields_ = [("e1", C.c_void_p), ("e2", C.c_void_p), ("block_index", C.c_void_p), ("full", C.c_void_p)]
+
+
 _lib = None
 
 
@@ -95,9 +104,12 @@ def lib() -> C.CDLL:
         L.recg_row_stats_static_error.restype = C.c_char_p
         L.recg_timing_enable.argtypes = [C.c_void_p, C.c_int32]
         L.recg_timing_read.argtypes = [C.c_void_p, C.POINTER(C.c_float), C.POINTER(C.c_int32)]
+        L.recg_policy_load.argtypes = [C.c_void_p, C.POINTER(recg_policy_table)]
+        L.recg_policy_step.argtypes = [C.c_void_p, C.POINTER(recg_policy_state), C.c_void_p, C.c_void_p, C.c_void_p]
         L.recg_free.argtypes = [C.c_void_p]
         for f in ("recg_init", "recg_step", "recg_verify", "recg_attention", "recg_kv_write", "recg_kv_read",
-                  "recg_linear", "recg_debug_buffer", "recg_sync", "recg_free", "recg_timing_enable", "recg_timing_read"):
+                  "recg_linear", "recg_debug_buffer", "recg_sync", "recg_free", "recg_timing_enable", "recg_timing_read",
+                  "recg_policy_load", "recg_policy_step"):
             getattr(L, f).restype = C.c_int32
         _lib = L
     return _lib
@@ -105,7 +117,8 @@ def lib() -> C.CDLL:
 
 EXPORTS = ("recg_kv_pool_bytes", "recg_init", "recg_step", "recg_verify", "recg_attention", "recg_kv_write",
            "recg_kv_read", "recg_linear", "recg_debug_buffer", "recg_sync", "recg_free", "recg_last_error",
-           "recg_timing_enable", "recg_timing_read", "recg_row_stats_static", "recg_row_stats_static_error")
+           "recg_timing_enable", "recg_timing_read", "recg_row_stats_static", "recg_row_stats_static_error",
+           "recg_policy_load", "recg_policy_step")
 TIMING_CLASSES = ("layout", "rmsnorm", "gemm_qkv", "attention", "gemm_o", "gemm_gate_up", "gemm_down", "lm_head", "verify")
 
 
@@ -270,6 +283,26 @@ class Context:
         self._check(lib().recg_linear(self.h, x.data_ptr(), w.data_ptr(), y.data_ptr(), M, N, K,
                                       DTYPE_BF16 if out_dtype == torch.bfloat16 else DTYPE_F32))
         return y
+
+    def recg_policy_load(self, blocks, s_edges, value, cost):
+        """Host arrays of the block-size rule: blocks [nb], s_edges [n_bins-1], value [nb, n_bins, nb, 2], cost [nb]."""
+        b = _i32(blocks)
+        e = np.ascontiguousarray(np.asarray(s_edges, dtype=np.float32))
+        v = np.ascontiguousarray(np.asarray(value, dtype=np.float32))
+        c = np.ascontiguousarray(np.asarray(cost, dtype=np.float32))
+        n_bins = e.size + 1
+        if v.shape != (b.size, n_bins, b.size, 2) or c.size != b.size:
+            raise ValueError("value must be [n_blocks, n_bins, n_blocks, 2] and cost [n_blocks]")
+        t = recg_policy_table(b.size, n_bins, _ptr(b), _ptr(e) if e.size else None, _ptr(v), _ptr(c))
+        self._check(lib().recg_policy_load(self.h, C.byref(t)))
+
+    def recg_policy_step(self, state: Dict[str, torch.Tensor], next_block: torch.Tensor,
+                         entropy_mean: Optional[torch.Tensor] = None, accept_len: Optional[torch.Tensor] = None):
+        """state: CUDA tensors e1, e2 (float32), block_index, full (int32), updated in place; next_block: CUDA int32."""
+        st = recg_policy_state(state["e1"].data_ptr(), state["e2"].data_ptr(), state["block_index"].data_ptr(),
+                               state["full"].data_ptr())
+        self._check(lib().recg_policy_step(self.h, C.byref(st), _ptr(entropy_mean), _ptr(accept_len),
+                                           next_block.data_ptr()))
 
     def recg_debug_buffer(self, which: int) -> torch.Tensor:
         p, dt, r, c = C.c_void_p(), C.c_int32(), C.c_int32(), C.c_int32()

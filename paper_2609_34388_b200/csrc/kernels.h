@@ -121,6 +121,15 @@ void launch_verify(const BatchLayout& bl, const void* logits, int logits_dtype, 
                    int max_chunks_total, const VerifyBuffers& vb, int n_sm, cudaStream_t st);
 int verify_chunks_per_row(int rows, int vocab, int n_sm);
 
+// Block-size rule (Eq. 2-3): table = [blocks (int) x8 | cost x8 | edges x64 | value n_blocks*n_bins*n_blocks*2]
+struct PolicyTable {
+  int n_blocks, n_bins;
+  const int* blocks;
+  const float *cost, *edges, *value;
+};
+void launch_policy(const BatchLayout& bl, const PolicyTable& tb, float* e1, float* e2, int* block_index, int* full,
+                   const float* entropy_mean, const int* accept_len, int* next_block, cudaStream_t st);
+
 // KV import / export
 void launch_kv_io(bool write, void* pool, int64_t n_pages, int layer, const Dims& dm, const int* page_row_dev, int pos0,
                   int n_pos, void* k, void* v, int* status, cudaStream_t st);

@@ -58,6 +58,10 @@ struct recg_ctx {
   VerifyBuffers vws{};
   int* d_status = nullptr;
   int* d_page_row = nullptr;
+  int* d_policy = nullptr;       // block-size rule: [blocks x8 | cost x8 | edges x64 | value]
+  PolicyTable policy{};
+  bool policy_loaded = false;
+  std::vector<int> h_policy;
   void* tc_state = nullptr;
   std::vector<int> h_desc;
   // optional per-class timing
@@ -120,6 +124,7 @@ size_t carve(recg_ctx* c, DeviceArena& A) {
   bl.counts = A.take<int>(4);
   c->d_status = A.take<int>(1);
   c->d_page_row = A.take<int>(Pm);
+  c->d_policy = A.take<int>(8 + 8 + 64 + RECG_POLICY_MAX_BLOCKS * RECG_POLICY_MAX_BINS * RECG_POLICY_MAX_BLOCKS * 2);
   c->rope_cs = A.take<float2>(Tm * (d.head_dim / 2));
   c->part_o = A.take<float>((size_t)bl.max_parts * 128 * d.head_dim);
   c->part_ml = A.take<float>((size_t)bl.max_parts * 128 * 2);
@@ -522,6 +527,51 @@ recg_status recg_verify(recg_ctx* ctx, const recg_batch* batch, const void* logi
 #undef OUT
     CU(cudaStreamSynchronize(ctx->stream));
   }
+  return RECG_OK;
+}
+
+recg_status recg_policy_load(recg_ctx* ctx, const recg_policy_table* t) {
+  if (!ctx) return RECG_ERR_INVALID_ARG;
+  if (!t || !t->blocks || !t->value || !t->cost || (t->n_bins > 1 && !t->s_edges))
+    return fail(ctx, RECG_ERR_INVALID_ARG, "recg_policy_load: null table array");
+  if (t->n_blocks < 1 || t->n_blocks > RECG_POLICY_MAX_BLOCKS || t->n_bins < 1 || t->n_bins > RECG_POLICY_MAX_BINS)
+    return fail(ctx, RECG_ERR_INVALID_ARG, "recg_policy_load: n_blocks must be 1..8 and n_bins 1..64");
+  for (int j = 0; j < t->n_blocks; ++j)
+    if (t->blocks[j] < 1 || (j > 0 && t->blocks[j] <= t->blocks[j - 1]))
+      return fail(ctx, RECG_ERR_INVALID_ARG, "recg_policy_load: blocks must be positive and ascending");
+  for (int i = 1; i < t->n_bins - 1; ++i)
+    if (!(t->s_edges[i] >= t->s_edges[i - 1]))
+      return fail(ctx, RECG_ERR_INVALID_ARG, "recg_policy_load: s_edges must be ascending");
+  const size_t nv = (size_t)t->n_blocks * t->n_bins * t->n_blocks * 2;
+  std::vector<int>& h = ctx->h_policy;
+  h.assign(80 + nv, 0);
+  memcpy(h.data(), t->blocks, t->n_blocks * sizeof(int));
+  memcpy(h.data() + 8, t->cost, t->n_blocks * sizeof(float));
+  if (t->n_bins > 1) memcpy(h.data() + 16, t->s_edges, (t->n_bins - 1) * sizeof(float));
+  memcpy(h.data() + 80, t->value, nv * sizeof(float));
+  CU(cudaMemcpyAsync(ctx->d_policy, h.data(), h.size() * sizeof(int), cudaMemcpyHostToDevice, ctx->stream));
+  CU(cudaStreamSynchronize(ctx->stream));
+  ctx->policy.n_blocks = t->n_blocks;
+  ctx->policy.n_bins = t->n_bins;
+  ctx->policy.blocks = ctx->d_policy;
+  ctx->policy.cost = reinterpret_cast<const float*>(ctx->d_policy + 8);
+  ctx->policy.edges = reinterpret_cast<const float*>(ctx->d_policy + 16);
+  ctx->policy.value = reinterpret_cast<const float*>(ctx->d_policy + 80);
+  ctx->policy_loaded = true;
+  return RECG_OK;
+}
+
+recg_status recg_policy_step(recg_ctx* ctx, const recg_policy_state* state, const float* entropy_mean,
+                             const int32_t* accept_len, int32_t* next_block) {
+  if (!ctx) return RECG_ERR_INVALID_ARG;
+  if (!ctx->policy_loaded) return fail(ctx, RECG_ERR_INVALID_ARG, "recg_policy_step: no table loaded");
+  if (!ctx->layout_valid) return fail(ctx, RECG_ERR_INVALID_ARG, "recg_policy_step: no batch laid out before");
+  if (!state || !state->e1 || !state->e2 || !state->block_index || !state->full || !next_block)
+    return fail(ctx, RECG_ERR_INVALID_ARG, "recg_policy_step: null state array or next_block");
+  launch_policy(ctx->bl, ctx->policy, state->e1, state->e2, state->block_index, state->full,
+                entropy_mean ? entropy_mean : ctx->vws.entropy_mean, accept_len ? accept_len : ctx->vws.accept_len,
+                next_block, ctx->stream);
+  CU(cudaGetLastError());
   return RECG_OK;
 }
 

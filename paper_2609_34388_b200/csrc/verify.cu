@@ -327,6 +327,57 @@ void launch_verify(const BatchLayout& bl, const void* logits, int logits_dtype, 
 }  // namespace recg
 
 // ---------------------------------------------------------------------------------------------------
+// Block-size rule of verification-guided drafting (Sec. 5.2): one thread per request.
+// ---------------------------------------------------------------------------------------------------
+namespace recg {
+namespace {
+
+__global__ void policy_kernel(BatchLayout bl, PolicyTable tb, float* __restrict__ e1, float* __restrict__ e2,
+                              int* __restrict__ block_index, int* __restrict__ full,
+                              const float* __restrict__ entropy_mean, const int* __restrict__ accept_len,
+                              int* __restrict__ next_block) {
+  griddep_launch();
+  griddep_wait();
+  const int r = blockIdx.x * blockDim.x + threadIdx.x;
+  if (r >= bl.n_req) return;
+  const int v = bl.verify_len[r];
+  float a1 = e1[r], a2 = e2[r];
+  int f = full[r];
+  if (v > 0) {   // the finished round verified something: shift its mean verifier entropy into the history
+    a2 = a1;
+    a1 = entropy_mean[r];
+    f = (v > 1 && accept_len[r] == v - 1) ? 1 : 0;
+    e1[r] = a1;
+    e2[r] = a2;
+    full[r] = f;
+  }
+  const float s = __fmul_rn(__fadd_rn(a1, a2), -0.5f);   // Eq. 2
+  int k = 0;
+  for (int i = 0; i < tb.n_bins - 1; ++i) k += tb.edges[i] <= s ? 1 : 0;
+  int jp = block_index[r];
+  jp = jp < 0 ? 0 : (jp >= tb.n_blocks ? tb.n_blocks - 1 : jp);
+  int best = 0;
+  float best_score = 0.f;
+  for (int j = 0; j < tb.n_blocks; ++j) {   // Eq. 3; the first maximum wins
+    const float score = __fsub_rn(tb.value[((j * tb.n_bins + k) * tb.n_blocks + jp) * 2 + f], tb.cost[j]);
+    if (j == 0 || score > best_score) { best = j; best_score = score; }
+  }
+  block_index[r] = best;
+  next_block[r] = tb.blocks[best];
+}
+
+}  // namespace
+
+void launch_policy(const BatchLayout& bl, const PolicyTable& tb, float* e1, float* e2, int* block_index, int* full,
+                   const float* entropy_mean, const int* accept_len, int* next_block, cudaStream_t st) {
+  if (bl.n_req <= 0) return;
+  launch_pdl(policy_kernel, dim3((bl.n_req + 127) / 128), dim3(128), 0, st, bl, tb, e1, e2, block_index, full,
+             entropy_mean, accept_len, next_block);
+}
+
+}  // namespace recg
+
+// ---------------------------------------------------------------------------------------------------
 // Row statistics without any allocation: the chunk partials live in a file-scope device array.
 // ---------------------------------------------------------------------------------------------------
 namespace recg {
