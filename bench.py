@@ -448,6 +448,42 @@ def bench_c128(binding, W, shape, peaks, args):
     sweep_result = {"workload": "configs[2] recipe at other batch sizes, one draw each, processed tokens/s of the whole step; "
                                             "ideal_ms = max(weight stream, GEMM flops at sustained peak) + KV stream, of measured peaks",
                                 "points": sweep}
+    # ---- one ragged mixed batch against one batch per block size (the remedy of padded kernels) ----
+    from paper_2609_34388_b200 import schedule
+    bucketing = []
+    for C in (16, 128):
+        d = sweep_descs[C]
+        ysw = synth.token_ids(int(d.verify_len.sum()), shape.vocab, seed=50 + C)
+        plans = {"ragged": [(d, ysw)]}
+        groups = schedule.bucket_by_block(d.block_size)
+        plans["bucketed"] = []
+        for idx in groups.values():
+            toks = np.concatenate([ysw[sl] for sl in schedule.verify_token_slices(d, idx)])
+            plans["bucketed"].append((schedule.sub_descriptor(d, idx), toks))
+        res = {"concurrency": C, "rows": d.n_tokens, "rows_if_padded_to_longest": schedule.padded_rows(d),
+               "buckets": {int(b): len(idx) for b, idx in groups.items()}}
+        for name, plan in plans.items():
+            bts = [binding.Batch(x.ctx_len, x.verify_len, x.block_size, t, x.page_table, pool, n_pages) for x, t in plan]
+            vos = [binding.VerifyOut(bt.n_req, bt.n_tok, bt.n_ver, host=False) for bt in bts]
+            def run_plan():
+                for bt, vo in zip(bts, vos):
+                    ctx.recg_step(bt)
+                    ctx.recg_verify(bt, out=vo)
+            for _ in range(3):
+                run_plan()
+            torch.cuda.synchronize()
+            e0.record()
+            for _ in range(5):
+                run_plan()
+            e1.record()
+            torch.cuda.synchronize()
+            msw = e0.elapsed_time(e1) / 5
+            res[name] = {"steps": len(bts), "ms": round(msw, 3), "rows_per_s": round(d.n_tokens / (msw / 1e3), 1)}
+        res["bucketed_over_ragged"] = round(res["bucketed"]["ms"] / res["ragged"]["ms"], 3)
+        bucketing.append(res)
+    bucketing_result = {"workload": "configs[2] recipe at 16 and 128 requests: the whole mixed batch in one ragged step against one "
+                                    "step per block size (4 steps), same requests, same pool; time for all requests of the round",
+                        "points": bucketing}
     overlap = {}
     for key in ov_descs:
         res = {}
@@ -521,6 +557,7 @@ def bench_c128(binding, W, shape, peaks, args):
            "attention": {"ms_per_step": round(attn_ms, 3), "gbs": round(attn_gbs, 1),
                          "frac_of_hbm_measured": round(attn_gbs / peaks["hbm_gbs"], 4)}}
     out["concurrency_sweep"] = sweep_result
+    out["bucketing"] = bucketing_result
     # block-size rule on the device after the verification of the 128-request batch (one small kernel; launch bound)
     tb = synth.policy_table()
     ctx.recg_policy_load(tb["blocks"], tb["s_edges"], tb["value"], tb["cost"])

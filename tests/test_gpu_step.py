@@ -244,3 +244,51 @@ def test_llama8b_shape_one_layer_round():
     flagged, _ = check_round(ctx, shape, ocfg, W64, reqs, desc, pool, adaptive_flag=True)
     assert flagged < 0.5 * desc.n_tokens      # how many rows the flag excused; not a correctness criterion
     ctx.recg_free()
+
+
+def test_bucketed_schedule_gives_the_same_results_as_the_mixed_batch():
+    """One ragged step over requests with mixed block sizes against one step per block size: every request must get
+    the same integers and the same logits (within the batch-invariance tolerance)."""
+    from paper_2609_34388_b200 import schedule
+
+    shape, W, ocfg, W64 = tiny_model()
+    specs = [(63, 4, 4, 1), (40, 8, 8, 3), (17, 4, 4, 3), (90, 16, 16, 5), (21, 8, 8, 7), (33, 16, 16, 15), (8, 2, 2, 0)]
+    reqs = build_requests(ocfg, W64, shape, specs, seed=700)
+    desc = synth.fixed_descriptor([s[0] for s in specs], [s[1] for s in specs], [s[2] for s in specs], seed=19)
+    ctx = binding.Context(binding.make_config(shape, 8, 128, desc.page_table.shape[1]), to_dev(W))
+    pool = binding.alloc_kv_pool(ctx, desc.n_pages, fill=None)
+    pool.fill_(float("nan"))
+    for i, r in enumerate(reqs):
+        for l, (K, V) in enumerate(r["kv"]):
+            ctx.recg_kv_write(pool, desc.n_pages, l, desc.page_table[i], 0,
+                              torch.from_numpy(K).to(torch.bfloat16).cuda(), torch.from_numpy(V).to(torch.bfloat16).cuda())
+    ys = np.asarray([t for r in reqs for t in r["y"]], dtype=np.int32)
+    mixed = binding.Batch(desc.ctx_len, desc.verify_len, desc.block_size, ys, desc.page_table, pool, desc.n_pages)
+    full = ctx.logits_tensor(ctx.recg_step(mixed))
+    g = {k: v.copy() for k, v in ctx.recg_verify(mixed).items()}
+    row0 = np.concatenate([[0], np.cumsum(desc.rows)])
+    groups = schedule.bucket_by_block(desc.block_size)
+    assert list(groups) == [2, 4, 8, 16]
+    seen = 0
+    for b, idx in groups.items():
+        sub = schedule.sub_descriptor(desc, idx)
+        toks = np.concatenate([ys[sl] for sl in schedule.verify_token_slices(desc, idx)])
+        bt = binding.Batch(sub.ctx_len, sub.verify_len, sub.block_size, toks, sub.page_table, pool, desc.n_pages)
+        lg = ctx.logits_tensor(ctx.recg_step(bt))
+        gb = ctx.recg_verify(bt)
+        t0 = 0
+        for j, r in enumerate(idx):
+            n = int(desc.rows[r])
+            ref = full[row0[r]: row0[r] + n]
+            assert float((lg[t0:t0 + n] - ref).abs().max()) <= 0.5 * HID_TOL * float(ref.abs().max())
+            top2 = torch.topk(ref, 2, dim=1).values
+            clear = ((top2[:, 0] - top2[:, 1]) >= MARGIN_FLAG).cpu().numpy()
+            assert (gb["top1"][t0:t0 + n][clear] == g["top1"][row0[r]: row0[r] + n][clear]).all()
+            if clear[: specs[r][1]].all():
+                assert int(gb["accept_len"][j]) == int(g["accept_len"][r]) == specs[r][3]
+                assert int(gb["new_ctx_len"][j]) == int(g["new_ctx_len"][r])
+            t0 += n
+            seen += 1
+    assert seen == len(specs)
+    ctx.recg_sync()
+    ctx.recg_free()
