@@ -269,6 +269,63 @@ def run_ours(args, env):
     torch.cuda.empty_cache()
     if env.rank == 0 and env.world == 1:
         out["c128"] = bench_c128(binding, W, shape, peaks, args)
+        del W
+        torch.cuda.empty_cache()
+        out["second_model"] = bench_second_model(binding, peaks, args)
+    return out
+
+
+def bench_second_model(binding, peaks, args):
+    """The same step on an assumed 14B-class backbone (synth.dense14b_shape: 40 layers, hidden 5120, 40 / 8 heads, FFN
+    17408, vocab 152064) at concurrency 16, configs[2]'s request recipe."""
+    shape = synth.dense14b_shape()
+    W = synth.model_weights(shape, seed=0, device="cuda", dtype=torch.bfloat16)
+    desc = c16_descriptor(3)
+    ctx = binding.Context(binding.make_config(shape, 16, 1024, desc.page_table.shape[1]), W)
+    pool = binding.alloc_kv_pool(ctx, desc.n_pages, fill="normal")
+    ys = synth.token_ids(int(desc.verify_len.sum()), shape.vocab, seed=1)
+    batch = binding.Batch(desc.ctx_len, desc.verify_len, desc.block_size, ys, desc.page_table, pool, desc.n_pages)
+    vout = binding.VerifyOut(batch.n_req, batch.n_tok, batch.n_ver, host=False)
+    for _ in range(3):
+        ctx.recg_step(batch)
+        ctx.recg_verify(batch, out=vout)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    iters = 5
+    e0.record()
+    for _ in range(iters):
+        ctx.recg_step(batch)
+        ctx.recg_verify(batch, out=vout)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / iters
+    ctx.recg_timing_enable(True)
+    ctx.recg_timing_read()
+    for _ in range(iters):
+        ctx.recg_step(batch)
+        ctx.recg_verify(batch, out=vout)
+    cms, _ = ctx.recg_timing_read()
+    ctx.recg_timing_enable(False)
+    cnt = algorithmic_counts(shape, desc)
+    gemm_classes = ("gemm_qkv", "gemm_o", "gemm_gate_up", "gemm_down", "lm_head")
+    gemm_ms = sum(cms[k] for k in gemm_classes) / iters
+    gemm_tf = sum(cnt["flops"][k] for k in gemm_classes) / (gemm_ms / 1e3) / 1e12
+    attn_ms = cms["attention"] / iters
+    attn_gbs = cnt["attn_bytes"] / (attn_ms / 1e3) / 1e9
+    wbytes = sum(cnt["wbytes"].values())
+    out = {"workload": "assumed 14B-class backbone (40 layers, hidden 5120, 40/8 heads, d 128, FFN 17408, vocab 152064), "
+                       "concurrency 16, configs[2] request recipe, draw 0",
+           "tokens_per_step": batch.n_tok, "ms_per_step": round(ms, 3), "tokens_per_s": round(batch.n_tok / (ms / 1e3), 1),
+           "weight_gb": round(wbytes / 1e9, 1),
+           "ideal_ms": round(max(wbytes / peaks["hbm_gbs"] / 1e6, sum(cnt["flops"].values()) / peaks["bf16_tflops_sustained"] / 1e9)
+                             + cnt["attn_bytes"] / peaks["hbm_gbs"] / 1e6, 3),
+           "gemm": {"ms_per_step": round(gemm_ms, 3), "tflops": round(gemm_tf, 1),
+                    "frac_of_bf16_sustained": round(gemm_tf / peaks["bf16_tflops_sustained"], 4)},
+           "attention": {"ms_per_step": round(attn_ms, 3), "gbs": round(attn_gbs, 1),
+                         "frac_of_hbm_measured": round(attn_gbs / peaks["hbm_gbs"], 4)}}
+    ctx.recg_free()
+    del pool, W
+    torch.cuda.empty_cache()
     return out
 
 

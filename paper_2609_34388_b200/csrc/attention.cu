@@ -439,11 +439,10 @@ template <int D>
 void launch_attention_t(const BatchLayout& bl, const Dims& dm, int layer, const void* q, void* o, const void* kv_pool,
                         int64_t n_pages, float* part_o, float* part_ml, int tok_per_tile, int n_sm, int* status,
                         cudaStream_t st) {
-  static bool configured = false;
-  if (!configured) {
+  static bool configured[kMaxDevices] = {false};
+  if (first_use_on_device(configured))
     cudaFuncSetAttribute(attention_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnSmem<D>::kTotal);
-    configured = true;
-  }
+
   AttnParams P;
   P.items = bl.items;
   P.cta_off = bl.cta_off;

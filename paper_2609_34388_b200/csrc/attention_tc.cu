@@ -309,7 +309,8 @@ __global__ void __launch_bounds__(kThreads, 1) attention_tc_kernel(const __grid_
           const int buf = item_cnt & 1;
           bwait(&q_empty[buf], ((item_cnt >> 1) & 1) ^ 1, DEV_TIMEOUT_EMPTY);
           if (lane == 0) {
-            mbar_arrive_expect_tx(&q_full[buf], kQBytes);
+            // two boxes of 64 dims x group heads x 128 / group tokens (125 rows when the group is 5; the MMA reads 128)
+            mbar_arrive_expect_tx(&q_full[buf], 2u * 128u * (uint32_t)(P.group * (128 / P.group)));
             const uint32_t dst = smem_base + kOffQ + buf * kQBytes;
             tma_load_3d(dst, &qmap, 0, w.kv_head * P.group, w.tok0, &q_full[buf]);
             tma_load_3d(dst + kQBytes / 2, &qmap, 64, w.kv_head * P.group, w.tok0, &q_full[buf]);
@@ -661,7 +662,7 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 struct QMapEntry {
   const void* q;
-  int n_tok, n_q, group;
+  int n_tok, n_q, group, device;
   CUtensorMap map;
 };
 
@@ -670,8 +671,12 @@ const CUtensorMap* q_tensor_map(const void* q, int n_tok, int n_q, int group) {
   static EncodeTiledFn encode = nullptr;
   static QMapEntry cache[16];
   static int n_cached = 0, next_slot = 0;
+  int device = 0;
+  cudaGetDevice(&device);   // an address means something else on another device
   for (int i = 0; i < n_cached; ++i)
-    if (cache[i].q == q && cache[i].n_tok == n_tok && cache[i].n_q == n_q && cache[i].group == group) return &cache[i].map;
+    if (cache[i].q == q && cache[i].n_tok == n_tok && cache[i].n_q == n_q && cache[i].group == group &&
+        cache[i].device == device)
+      return &cache[i].map;
   if (!encode) {
     void* fn = nullptr;
     cudaDriverEntryPointQueryResult qres;
@@ -689,7 +694,7 @@ const CUtensorMap* q_tensor_map(const void* q, int n_tok, int n_q, int group) {
              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
     return nullptr;
-  e.q = q; e.n_tok = n_tok; e.n_q = n_q; e.group = group;
+  e.q = q; e.n_tok = n_tok; e.n_q = n_q; e.group = group; e.device = device;
   next_slot = (next_slot + 1) % 16;
   if (n_cached < 16) ++n_cached;
   return &e.map;
@@ -700,11 +705,10 @@ const CUtensorMap* q_tensor_map(const void* q, int n_tok, int n_q, int group) {
 void launch_attention_tc_main(const BatchLayout& bl, const Dims& dm, int layer, const void* q, void* o,
                               const void* kv_pool, int64_t n_pages, float* part_o, float* part_ml, int n_sm, int* status,
                               cudaStream_t st) {
-  static bool configured = false;
-  if (!configured) {
+  static bool configured[kMaxDevices] = {false};
+  if (first_use_on_device(configured))
     cudaFuncSetAttribute(attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
-    configured = true;
-  }
+
   TcAttnParams P;
   P.items = bl.items;
   P.cta_off = bl.cta_off;

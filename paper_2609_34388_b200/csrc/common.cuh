@@ -124,6 +124,17 @@ __host__ __device__ __forceinline__ size_t kv_tile_base(int64_t n_pages, int n_k
   return ((((size_t)layer * n_pages + page) * n_kv + kv_head) * 2) * kv_tile_elems(head_dim);
 }
 
+// Host side.  Opt-in attributes of a kernel (its dynamic shared memory size) are per device: a call site keeps one
+// flag per device and sets the attribute on first use there.  Setting it twice from two threads is harmless.
+constexpr int kMaxDevices = 64;
+inline bool first_use_on_device(bool (&seen)[kMaxDevices]) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return true;
+  if (seen[dev]) return false;
+  seen[dev] = true;
+  return true;
+}
+
 // Host side: launch with the programmatic-serialisation attribute.
 template <typename... KArgs, typename... Args>
 inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,

@@ -124,11 +124,10 @@ __global__ void __launch_bounds__(THREADS) gemm_simt_kernel(const __nv_bfloat16*
 }  // namespace
 
 void launch_gemm_simt(const GemmArgs& a, int* status, cudaStream_t st) {
-  static bool configured = false;
-  if (!configured) {
+  static bool configured[kMaxDevices] = {false};
+  if (first_use_on_device(configured))
     cudaFuncSetAttribute(gemm_simt_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
-    configured = true;
-  }
+
   EpiParams ep;
   ep.epi = a.epi;
   ep.out = a.out;

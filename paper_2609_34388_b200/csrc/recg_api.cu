@@ -313,7 +313,7 @@ recg_status recg_init(recg_ctx** out, const recg_config* cfg, const recg_weights
   if (g.head_dim != 64 && g.head_dim != 128) return fail(ctx, RECG_ERR_SHAPE, "recg_init: head_dim must be 64 or 128");
   if (g.n_q_heads % g.n_kv_heads) return fail(ctx, RECG_ERR_SHAPE, "recg_init: n_q_heads must be a multiple of n_kv_heads");
   const int group = g.n_q_heads / g.n_kv_heads;
-  if (group > 16 || (group & (group - 1))) return fail(ctx, RECG_ERR_SHAPE, "recg_init: GQA group must be 1, 2, 4, 8 or 16");
+  if (group > 16) return fail(ctx, RECG_ERR_SHAPE, "recg_init: at most 16 query heads per kv head");
   if (g.hidden % 64 || g.ffn % 64 || g.vocab % 16 || ((g.n_q_heads + 2 * g.n_kv_heads) * g.head_dim) % 128)
     return fail(ctx, RECG_ERR_SHAPE, "recg_init: hidden and ffn must be multiples of 64, vocab of 16, qkv width of 128");
   if (g.mask_token_id >= g.vocab) return fail(ctx, RECG_ERR_INVALID_ARG, "recg_init: mask_token_id outside the vocabulary");

@@ -386,7 +386,6 @@ namespace {
 constexpr int kStaticMaxPartials = 1 << 16;   // 65536 x 24 bytes = 1.5 MiB held by every GPU that loads the library
 static __device__ __align__(256) RowPartial g_static_partials[kStaticMaxPartials];
 
-constexpr int kMaxDevices = 64;
 RowPartial* g_static_ptr[kMaxDevices] = {nullptr};   // device address of the array, per device, set on first use
 int g_static_sm[kMaxDevices] = {0};
 

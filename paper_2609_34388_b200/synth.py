@@ -48,6 +48,14 @@ def llama8b_shape(n_layers: int = 32) -> ModelShape:
                       vocab=128256, rope_base=500000.0)
 
 
+def dense14b_shape(n_layers: int = 40) -> ModelShape:
+    """A 14B-class backbone.  The second model of the paper's evaluation is named but its dimensions are not given;
+    these are an ASSUMPTION in the style of current dense 14B decoders: 40 layers, hidden 5120, 40 query / 8 kv heads
+    (five query heads per kv head), head_dim 128, FFN 17408, vocab 152064 (about 14.8 B parameters)."""
+    return ModelShape(n_layers=n_layers, hidden=5120, n_q_heads=40, n_kv_heads=8, head_dim=128, ffn=17408,
+                      vocab=152064, rope_base=1000000.0)
+
+
 def _gen(seed: int, device) -> torch.Generator:
     g = torch.Generator(device=device)
     g.manual_seed(int(seed))

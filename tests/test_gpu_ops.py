@@ -95,6 +95,40 @@ def test_attention_high_concurrency_mix():
     assert run_attention_case(shape, reqs, seed=32) < ATTN_TOL
 
 
+@pytest.mark.parametrize("flags", [0, binding.FLAG_SIMT_ATTENTION])
+def test_attention_five_query_heads_per_kv_head(flags):
+    """40 query / 8 kv heads: a row tile is 25 tokens x 5 heads = 125 of the 128 rows."""
+    shape = synth.dense14b_shape(1)
+    L = [300, 77, 1500, 0, 40]
+    v = [25, 26, 50, 3, 1]
+    b = [25, 24, 14, 2, 8]
+    desc = synth.fixed_descriptor(L, v, b, seed=31)
+    T = desc.n_tokens
+    ctx = ops_ctx(shape, len(L), T, desc.page_table.shape[1], flags)
+    pool = binding.alloc_kv_pool(ctx, desc.n_pages, fill=None)
+    pool.fill_(float("nan"))
+    q = synth.queries(T, shape.n_q_heads, shape.head_dim, seed=36)
+    ks, vs = [], []
+    for r in range(len(L)):
+        k_, v_ = synth.kv_values(L[r] + v[r] + b[r], shape.n_kv_heads, shape.head_dim, seed=3100 + r)
+        ks.append(k_)
+        vs.append(v_)
+        ctx.recg_kv_write(pool, desc.n_pages, 0, desc.page_table[r], 0, k_.cuda(), v_.cuda())
+    batch = binding.Batch(desc.ctx_len, desc.verify_len, desc.block_size, None, desc.page_table, pool, desc.n_pages)
+    o = torch.full((T, shape.n_q_heads, shape.head_dim), float("nan"), dtype=torch.bfloat16, device="cuda")
+    ctx.recg_attention(batch, 0, q.cuda(), o)
+    ctx.recg_sync()
+    got = f64(o)
+    t0 = 0
+    for r in range(len(L)):
+        n = v[r] + b[r]
+        ref = orc.hybrid_attention(f64(q[t0:t0 + n]), f64(ks[r]), f64(vs[r]), L[r], v[r], b[r])
+        assert not np.isnan(got[t0:t0 + n]).any(), f"NaN in request {r}"
+        assert np.max(np.abs(got[t0:t0 + n] - ref)) / np.max(np.abs(ref)) < ATTN_TOL, r
+        t0 += n
+    ctx.recg_free()
+
+
 def test_attention_is_deterministic():
     shape = synth.llama8b_shape(1)
     desc = synth.fixed_descriptor([1500, 40], [8, 4], [8, 4], seed=3)

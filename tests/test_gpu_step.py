@@ -246,6 +246,29 @@ def test_llama8b_shape_one_layer_round():
     ctx.recg_free()
 
 
+def test_dense14b_shape_one_layer_round():
+    """One layer of the assumed 14B-class shape (hidden 5120, 40 / 8 heads, FFN 17408) + LM head on a ragged batch."""
+    shape = synth.dense14b_shape(1)
+    shape.vocab = 16384            # keeps the oracle's LM head quick; every other dimension is the 14B-class one
+    W = synth.model_weights(shape, seed=0, dtype=torch.bfloat16)
+    ocfg, W64 = oracle_cfg(shape), oracle_weights(W)
+    specs = [(200, 16, 16), (70, 4, 4), (500, 30, 32), (16, 8, 8), (129, 3, 22)]
+    L, v, b = [s[0] for s in specs], [s[1] for s in specs], [s[2] for s in specs]
+    desc = synth.fixed_descriptor(L, v, b, seed=4)
+    ctx = binding.Context(binding.make_config(shape, 8, 256, desc.page_table.shape[1]), to_dev(W))
+    pool = binding.alloc_kv_pool(ctx, desc.n_pages, fill=None)
+    pool.fill_(float("nan"))
+    reqs = []
+    for i in range(len(specs)):
+        K, V = synth.kv_values(L[i], shape.n_kv_heads, shape.head_dim, seed=300 + i)
+        ctx.recg_kv_write(pool, desc.n_pages, 0, desc.page_table[i], 0, K.cuda(), V.cuda())
+        y = synth.token_ids(v[i], shape.vocab, seed=400 + i).tolist()
+        reqs.append({"kv": [(f64(K), f64(V))], "y": y, "L": L[i], "v": v[i], "b": b[i], "m": None})
+    flagged, _ = check_round(ctx, shape, ocfg, W64, reqs, desc, pool, adaptive_flag=True)
+    assert flagged < 0.5 * desc.n_tokens
+    ctx.recg_free()
+
+
 def test_bucketed_schedule_gives_the_same_results_as_the_mixed_batch():
     """One ragged step over requests with mixed block sizes against one step per block size: every request must get
     the same integers and the same logits (within the batch-invariance tolerance)."""
