@@ -13,6 +13,7 @@ using namespace recg;
 namespace {
 
 thread_local std::string g_init_error;
+constexpr size_t kVoutMirrorMax = 1 << 20;   // verify outputs up to this size come back to the host in one copy
 
 struct DeviceArena {  // one cudaMalloc, carved with 256-byte alignment
   uint8_t* base = nullptr;
@@ -56,6 +57,8 @@ struct recg_ctx {
   RowPartial* vpart = nullptr;
   int max_chunks_total = 0;
   VerifyBuffers vws{};
+  size_t vout_off = 0, vout_bytes = 0;   // the verify outputs are one contiguous region of the arena ...
+  uint8_t* h_vout = nullptr;             // ... mirrored by one pinned host buffer: a single copy brings all results back
   int* d_status = nullptr;
   int* d_page_row = nullptr;
   int* d_policy = nullptr;       // block-size rule: [blocks x8 | cost x8 | edges x64 | value]
@@ -131,6 +134,7 @@ size_t carve(recg_ctx* c, DeviceArena& A) {
   c->max_chunks_total = (int)(Tm + 4 * c->n_sm + 64);
   c->vpart = A.take<RowPartial>(c->max_chunks_total);
   VerifyBuffers& v = c->vws;
+  c->vout_off = (A.used + 255) & ~size_t(255);
   v.accept_len = A.take<int>(Cm);
   v.n_emitted = A.take<int>(Cm);
   v.emitted = A.take<int>(Tm);
@@ -149,6 +153,7 @@ size_t carve(recg_ctx* c, DeviceArena& A) {
   v.risky_n = A.take<int>(3 * Cm);
   v.risky_index = A.take<int>(6 * Cm);
   v.risky_token = A.take<int>(6 * Cm);
+  c->vout_bytes = A.used - c->vout_off;
   c->q = A.take<__nv_bfloat16>(Tm * d.n_q * d.head_dim);
   c->o = A.take<__nv_bfloat16>(Tm * d.n_q * d.head_dim);
   if (c->has_weights) {
@@ -365,6 +370,10 @@ recg_status recg_init(recg_ctx** out, const recg_config* cfg, const recg_weights
   }
   ctx->arena.size = bytes;
   carve(ctx, ctx->arena);
+  if (ctx->vout_bytes <= kVoutMirrorMax && cudaMallocHost(reinterpret_cast<void**>(&ctx->h_vout), ctx->vout_bytes) != cudaSuccess) {
+    cudaGetLastError();
+    ctx->h_vout = nullptr;   // fall back to one copy per output array
+  }
   cudaMemsetAsync(ctx->d_status, 0, sizeof(int), ctx->stream);
   ctx->tc_state = tc_state_create(n_sm);
   *out = ctx;
@@ -401,6 +410,7 @@ recg_status recg_free(recg_ctx* ctx) {
   for (cudaEvent_t e : ctx->ev_pool) cudaEventDestroy(e);
   if (ctx->tc_state) tc_state_destroy(ctx->tc_state);
   if (ctx->arena.base) cudaFree(ctx->arena.base);
+  if (ctx->h_vout) cudaFreeHost(ctx->h_vout);
   delete ctx;
   return RECG_OK;
 }
@@ -519,6 +529,19 @@ recg_status recg_verify(recg_ctx* ctx, const recg_batch* batch, const void* logi
   ctx->mark(8, 2);
   if (!dev) {
     const size_t C = bl.n_req, T = bl.n_tok, Tv = bl.n_ver, Tb = T - Tv;
+    if (ctx->h_vout) {
+      // one copy of the whole output region into pinned memory, then plain host copies into the caller's arrays
+      const uint8_t* region = ctx->arena.base + ctx->vout_off;
+      CU(cudaMemcpyAsync(ctx->h_vout, region, ctx->vout_bytes, cudaMemcpyDeviceToHost, ctx->stream));
+      CU(cudaStreamSynchronize(ctx->stream));
+#define OUT(f, n) if (out->f && (n)) memcpy(out->f, ctx->h_vout + (reinterpret_cast<const uint8_t*>(vb.f) - region), (n) * 4)
+      OUT(accept_len, C); OUT(n_emitted, C); OUT(emitted, Tv); OUT(new_ctx_len, C); OUT(slot_state, T);
+      OUT(freed_pages, C); OUT(next_draft, Tb); OUT(cont_hit, C); OUT(top1, T); OUT(top2, T); OUT(p1, T); OUT(p2, T);
+      OUT(entropy, T); OUT(entropy_mean, C);
+      OUT(corr_hit, 2 * C); OUT(risky_n, 3 * C); OUT(risky_index, 6 * C); OUT(risky_token, 6 * C);
+#undef OUT
+      return RECG_OK;
+    }
 #define OUT(f, n) if (out->f && (n)) CU(cudaMemcpyAsync(out->f, vb.f, (n) * 4, cudaMemcpyDeviceToHost, ctx->stream))
     OUT(accept_len, C); OUT(n_emitted, C); OUT(emitted, Tv); OUT(new_ctx_len, C); OUT(slot_state, T);
     OUT(freed_pages, C); OUT(next_draft, Tb); OUT(cont_hit, C); OUT(top1, T); OUT(top2, T); OUT(p1, T); OUT(p2, T);
