@@ -62,7 +62,7 @@ typedef struct {
   int32_t mask_token_id;  /* id fed to the mask rows; < 0 means vocab - 1                        */
   int32_t page_size;      /* tokens per KV page; must be 16                                      */
   int32_t max_requests;   /* capacity: requests per step                                         */
-  int32_t max_tokens;     /* capacity: sum of v_r + b_r per step                                 */
+  int32_t max_tokens;     /* capacity: rows of a step, the sum of n_r (see recg_batch)            */
   int32_t max_pages_per_request;
   int32_t flags;          /* RECG_FLAG_*                                                         */
 } recg_config;
@@ -93,7 +93,7 @@ typedef struct {
  *   block_size[r]  b_r >= 0, mask tokens;  v_r + b_r >= 1
  *   verify_tokens  the y of all requests, concatenated in request order (sum of v_r ids)
  *   page_table     [n_req, page_table_stride] physical page ids; row r must cover
- *                  ceil((L_r + v_r + b_r) / page_size) pages, else RECG_ERR_CAPACITY
+ *                  ceil((L_r + n_r) / page_size) pages (n_r = v_r + b_r without branches), else RECG_ERR_CAPACITY
  *   kv_pool        DEVICE, recg_kv_pool_bytes(cfg, kv_pool_pages) bytes, library-defined layout
  *                  (per layer, per page, per KV head: a K tile then a V tile of 16 tokens, stored in
  *                  the swizzled order the attention kernel loads; use recg_kv_write / recg_kv_read
@@ -193,7 +193,7 @@ recg_status recg_init(recg_ctx **out, const recg_config *cfg, const recg_weights
  * One fused draft+verify forward (ragged layout, embedding, n_layers x {RMSNorm, QKV projection with
  * rotary embedding and KV append, hybrid-mask paged attention (Eq. 1), output projection + residual,
  * RMSNorm, gate|up projection + SwiGLU, down projection + residual}, final norm, LM head).
- * K/V of all v_r + b_r new positions are written into the pool slots the page table names
+ * K/V of all n_r new rows are written into the pool slots the page table names
  * (tentatively: recg_verify decides which stay).  `logits` (may be NULL) receives the view of the
  * logits.  Does not synchronise.
  */
@@ -210,7 +210,7 @@ recg_status recg_verify(recg_ctx *ctx, const recg_batch *batch, const void *logi
 
 /*
  * The hybrid-mask paged attention of one layer as a standalone operation (Eq. 1 over a shared prefix).
- * q, o: DEVICE bf16 [T, n_q_heads, head_dim] (q already rotated).  K/V of ALL L_r + v_r + b_r
+ * q, o: DEVICE bf16 [T, n_q_heads, head_dim] (q already rotated).  K/V of ALL L_r + n_r
  * positions of every request must already be in layer `layer` of the pool.
  */
 recg_status recg_attention(recg_ctx *ctx, const recg_batch *batch, int32_t layer, const void *q, void *o);
