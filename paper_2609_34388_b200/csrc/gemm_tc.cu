@@ -7,7 +7,8 @@
 //            into one of two TMEM accumulators and commits to the ring's empty barriers;
 //   warps 2-5  epilogue: tcgen05.ld of the finished accumulator (each warp its 32-lane quadrant), then the
 //            fused epilogue straight from registers (residual add, SwiGLU, rotary + paged KV append, or
-//            plain store) while the MMA warp already fills the other accumulator.
+//            plain store) while the MMA warp already fills the other accumulator; output rows leave through
+//            TMA box stores (add-reductions for the residual stream) from a small swizzled staging area.
 // Tiles are walked m-fastest so that CTAs running together share the same weight tile through L2.
 // Every wait is bounded; on a timeout the kernel records a status code, drains and frees TMEM.
 #include <cuda.h>
@@ -29,7 +30,7 @@ namespace {
 constexpr int BM = 128, BK = 64;
 constexpr int kTcThreads = 192;
 constexpr int kSmemBudget = 192 * 1024;     // operand ring (every configuration's stage size divides it)
-constexpr int kStageOutBytes = 4 * 4096;      // per epilogue warp: 32 rows x 32 fp32 for transposing output chunks
+constexpr int kStageOutBytes = 4 * 4096;      // per epilogue warp: two 2 KB boxes of output on their way to the TMA unit
 constexpr uint32_t kSpin = 1u << 22;
 
 template <int BN, bool PAIR = false> struct TcCfg {
@@ -204,52 +205,78 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint64_t* bar, uint32_t parity
 
 
 // ---- register epilogue: one thread owns one output row -------------------------------------------
-// Warp-wide stores of a 32-row x 32-column chunk (lane = row holds the row's 32 values): the chunk is transposed
-// through 4 KB of shared memory so that every store instruction writes whole 128-byte (fp32) or 64-byte (bf16)
-// row segments instead of 16 bytes in each of 32 different rows.  dst0 points at (row 0 of the warp, first column
-// of the chunk); rows >= valid_rows are not written.  Every lane must call.  add = true accumulates into the fp32
-// residual stream with vector reductions at L2: every element receives exactly one addend from exactly one thread per
-// launch, so the result is the same single rounding as a load-add-store, without the load's round trip.
-__device__ __forceinline__ void store_rows_f32(float* dst0, size_t row_stride, int valid_rows, const float (&v)[32], bool add,
-                                               float* stg, int lane) {
-  float4* s4 = reinterpret_cast<float4*>(stg);
-#pragma unroll
-  for (int q = 0; q < 8; ++q)
-    s4[lane * 8 + (q ^ (lane & 7))] = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
-  __syncwarp();
-  const int rq = lane >> 3, q = lane & 7;
-#pragma unroll
-  for (int j = 0; j < 8; ++j) {
-    const int r = 4 * j + rq;
-    const float4 t = s4[r * 8 + (q ^ (r & 7))];
-    if (r < valid_rows) {
-      float4* p = reinterpret_cast<float4*>(dst0 + (size_t)r * row_stride) + q;
-      if (add) asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(p), "f"(t.x), "f"(t.y), "f"(t.z), "f"(t.w) : "memory");
-      else *p = t;
-    }
+
+// ---- epilogue through the TMA unit --------------------------------------------------------------------------------
+// A warp's chunk (lane = row, 64 bytes per row: 32 bf16 or 16 fp32 columns) goes to one of the warp's two 2 KB staging
+// buffers in the 64-byte-swizzle order of the output tensor map (16-byte piece c of row r at piece c ^ ((r >> 1) & 3):
+// conflict free), and one lane hands it to the TMA unit as a 32-row box: the unit clips rows beyond M and columns
+// beyond N, writes whole row segments, and with add = true adds into the fp32 destination (one addend per element and
+// launch, hence the same single rounding as a load-add-store).  OutStage counts the boxes of the warp so that a
+// buffer is only rewritten after the unit has read it.
+struct OutStage {
+  uint8_t* buf;     // this warp's 4 KB (two buffers)
+  uint32_t k;       // boxes issued so far
+};
+__device__ __forceinline__ void tma_store_box(const CUtensorMap* map, OutStage& os, const uint4 (&piece)[4], int col, int row,
+                                              bool add, bool active, int lane) {
+  if (os.k >= 2) {
+    if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");   // the box before the last one has been read
+    __syncwarp();
   }
+  uint4* dst = reinterpret_cast<uint4*>(os.buf + (os.k & 1) * 2048) + lane * 4;
+  const int x = (lane >> 1) & 3;
+#pragma unroll
+  for (int c = 0; c < 4; ++c) dst[c ^ x] = piece[c];
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   __syncwarp();
+  if (lane == 0) {
+    const uint32_t src = smem_u32(os.buf + (os.k & 1) * 2048);
+    if (active) {
+      if (add)
+        asm volatile("cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.tile.bulk_group [%0, {%2, %3}], [%1];" ::"l"(map),
+                     "r"(src), "r"(col), "r"(row)
+                     : "memory");
+      else
+        asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%2, %3}], [%1];" ::"l"(map), "r"(src),
+                     "r"(col), "r"(row)
+                     : "memory");
+    }
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+  }
+  ++os.k;
 }
-__device__ __forceinline__ void store_rows_bf16(__nv_bfloat16* dst0, size_t row_stride, int valid_rows, const float (&v)[32],
-                                                float* stg, int lane) {
-  uint4* s4 = reinterpret_cast<uint4*>(stg);
+// 32 columns of the thread's row as bf16 (one box) or fp32 (two boxes of 16 columns)
+__device__ __forceinline__ void tma_store_rows_bf16(const CUtensorMap* map, OutStage& os, const float (&v)[32], int col, int row,
+                                                    bool active, int lane) {
+  uint4 piece[4];
 #pragma unroll
   for (int q = 0; q < 4; ++q) {
-    uint4 o;
-    o.x = pack_bf16(v[8 * q], v[8 * q + 1]);
-    o.y = pack_bf16(v[8 * q + 2], v[8 * q + 3]);
-    o.z = pack_bf16(v[8 * q + 4], v[8 * q + 5]);
-    o.w = pack_bf16(v[8 * q + 6], v[8 * q + 7]);
-    s4[lane * 4 + (q ^ (lane & 3))] = o;
+    piece[q].x = pack_bf16(v[8 * q], v[8 * q + 1]);
+    piece[q].y = pack_bf16(v[8 * q + 2], v[8 * q + 3]);
+    piece[q].z = pack_bf16(v[8 * q + 4], v[8 * q + 5]);
+    piece[q].w = pack_bf16(v[8 * q + 6], v[8 * q + 7]);
   }
-  __syncwarp();
-  const int rq = lane >> 2, q = lane & 3;
+  tma_store_box(map, os, piece, col, row, false, active, lane);
+}
+__device__ __forceinline__ void tma_store_rows_f32(const CUtensorMap* map, OutStage& os, const float (&v)[32], int col, int row,
+                                                   bool add, bool active, int lane) {
 #pragma unroll
-  for (int j = 0; j < 4; ++j) {
-    const int r = 8 * j + rq;
-    const uint4 t = s4[r * 4 + (q ^ (r & 3))];
-    if (r < valid_rows) *(reinterpret_cast<uint4*>(dst0 + (size_t)r * row_stride) + q) = t;
+  for (int h = 0; h < 2; ++h) {
+    uint4 piece[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q)
+      piece[q] = make_uint4(__float_as_uint(v[16 * h + 4 * q]), __float_as_uint(v[16 * h + 4 * q + 1]),
+                            __float_as_uint(v[16 * h + 4 * q + 2]), __float_as_uint(v[16 * h + 4 * q + 3]));
+    tma_store_box(map, os, piece, col + 16 * h, row, add, active, lane);
   }
+}
+// the unit has read every box of the warp (its staging may be rewritten) / has written them all
+__device__ __forceinline__ void tma_store_drain_reads(int lane) {
+  if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+  __syncwarp();
+}
+__device__ __forceinline__ void tma_store_drain_all(int lane) {
+  if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
   __syncwarp();
 }
 
@@ -374,16 +401,18 @@ __device__ __forceinline__ Piece make_piece(int& jd, int dp_tiles, long long& po
 }
 
 // Epilogue of one accumulator tile for the calling thread's row.
-// stg: this warp's 4 KB transposition buffer.  All 32 lanes of the warp call together.
+// stg: this warp's 4 KB of output staging (two boxes).  All 32 lanes of the warp call together.
 template <int BN, typename Loader>
-__device__ __forceinline__ void row_epilogue(const EpiParams& ep, const Loader& load, int m, int n0, float* stg) {
+__device__ __forceinline__ void row_epilogue(const EpiParams& ep, const Loader& load, int m, int n0, float* stg,
+                                             const CUtensorMap* omap) {
   const bool row_ok = m < ep.M;
   const int lane = threadIdx.x & 31;
   const int m_base = m - lane;                                  // first row of this warp
   const int valid_rows = ep.M - m_base < 0 ? 0 : (ep.M - m_base > 32 ? 32 : ep.M - m_base);
+  OutStage os{reinterpret_cast<uint8_t*>(stg), 0u};
+  const bool active = valid_rows > 0;      // a box that starts beyond the last row is not issued at all
   if (ep.epi == EPI_SWIGLU) {
     // accumulator columns [0, BN/2) are gate, [BN/2, BN) up; n0 is the first output column
-    __nv_bfloat16* out = static_cast<__nv_bfloat16*>(ep.out);
 #pragma unroll 1
     for (int c = 0; c < BN / 64; ++c) {
       float g[32], u[32];
@@ -392,14 +421,14 @@ __device__ __forceinline__ void row_epilogue(const EpiParams& ep, const Loader& 
       if (n0 + c * 32 < ep.N) {
 #pragma unroll
         for (int i = 0; i < 32; ++i) g[i] = silu_f(g[i]) * u[i];
-        store_rows_bf16(out + (size_t)m_base * ep.N + n0 + c * 32, ep.N, valid_rows, g, stg, lane);
+        tma_store_rows_bf16(omap, os, g, n0 + c * 32, m_base, active, lane);
       }
     }
+    tma_store_drain_reads(lane);
     return;
   }
   if (ep.epi == EPI_QKV_ROPE) {
     const int D = ep.head_dim, half = D / 2;
-    __nv_bfloat16* q = static_cast<__nv_bfloat16*>(ep.out);
     const int slot = row_ok ? ep.tok_slot[m] : -1;
 #pragma unroll 1
     for (int hl = 0; hl < BN / D; ++hl) {        // heads in this tile
@@ -431,10 +460,9 @@ __device__ __forceinline__ void row_epilogue(const EpiParams& ep, const Loader& 
             hi[i] = b;
           }
         }
-        if (is_q) {      // (the same for the whole warp)
-          __nv_bfloat16* dst0 = q + ((size_t)m_base * ep.n_q + head) * D + c * 32;
-          store_rows_bf16(dst0, (size_t)ep.n_q * D, valid_rows, lo, stg, lane);
-          store_rows_bf16(dst0 + half, (size_t)ep.n_q * D, valid_rows, hi, stg, lane);
+        if (is_q) {      // (the same for the whole warp): rows of the rotated queries [M, n_q * D] through the TMA unit
+          tma_store_rows_bf16(omap, os, lo, head * D + c * 32, m_base, active, lane);
+          tma_store_rows_bf16(omap, os, hi, head * D + half + c * 32, m_base, active, lane);
         } else if (kv_base) {
           // the pool tile is swizzled in 16-byte chunks: store chunk by chunk
 #pragma unroll
@@ -450,6 +478,7 @@ __device__ __forceinline__ void row_epilogue(const EpiParams& ep, const Loader& 
         }
       }
     }
+    tma_store_drain_reads(lane);
     return;
   }
 #pragma unroll 1
@@ -458,24 +487,17 @@ __device__ __forceinline__ void row_epilogue(const EpiParams& ep, const Loader& 
     load(c * 32, v);
     const int n = n0 + c * 32;
     if (n >= ep.N) continue;
-    if (n + 32 <= ep.N) {
-      if (ep.epi == EPI_PLAIN_BF16)
-        store_rows_bf16(static_cast<__nv_bfloat16*>(ep.out) + (size_t)m_base * ep.N + n, ep.N, valid_rows, v, stg, lane);
-      else
-        store_rows_f32(static_cast<float*>(ep.out) + (size_t)m_base * ep.N + n, ep.N, valid_rows, v, ep.epi == EPI_RESIDUAL, stg, lane);
-    } else if (row_ok) {  // ragged right edge (N is a multiple of 16 but not of 32)
-      for (int i = 0; i < ep.N - n; ++i) {
-        if (ep.epi == EPI_PLAIN_BF16) static_cast<__nv_bfloat16*>(ep.out)[(size_t)m * ep.N + n + i] = __float2bfloat16_rn(v[i]);
-        else if (ep.epi == EPI_RESIDUAL) static_cast<float*>(ep.out)[(size_t)m * ep.N + n + i] += v[i];
-        else static_cast<float*>(ep.out)[(size_t)m * ep.N + n + i] = v[i];
-      }
-    }
+    // the box is clipped at the right edge (N is a multiple of 16 but not always of 32) and at the last row
+    if (ep.epi == EPI_PLAIN_BF16) tma_store_rows_bf16(omap, os, v, n, m_base, active, lane);
+    else tma_store_rows_f32(omap, os, v, n, m_base, ep.epi == EPI_RESIDUAL, active, lane);
   }
+  tma_store_drain_reads(lane);
 }
 
 template <int BN, bool PAIR>
 __global__ void __launch_bounds__(kTcThreads, 1)
-gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w, int M, int n_tiles_n,
+gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
+               const __grid_constant__ CUtensorMap map_out, int M, int n_tiles_n,
                int K, int up_row_offset, int dp_tiles, long long per, int thin, float* split_ws, int* split_counters,
                EpiParams ep) {
   using Cfg = TcCfg<BN, PAIR>;
@@ -702,7 +724,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
       };
       const int n0 = swiglu ? tn * (BN / 2) : tn * BN;
       if (n_splits == 1) {
-        row_epilogue<BN>(ep, TmemLoader{tacc}, m, n0, stg);
+        row_epilogue<BN>(ep, TmemLoader{tacc}, m, n0, stg, &map_out);
         release_acc();
       } else {
         // park this split's partial tile and let the LAST split to arrive reduce all partials in split order
@@ -758,10 +780,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
             }
             if (!mbar_wait(red_bar, 0, kSpin)) set_status(ep.status, DEV_TIMEOUT_FULL);
             RingLoader ld{tacc, reinterpret_cast<const float4*>(smem) + row_in_tile, BN, pc.part, n_splits};
-            row_epilogue<BN>(ep, ld, m, n0, stg);
+            row_epilogue<BN>(ep, ld, m, n0, stg, &map_out);
           } else {
             SplitLoader ld{split_ws, BN, row_in_tile, slot0, slot_next, slot_stride, n_splits, m < ep.M};
-            row_epilogue<BN>(ep, ld, m, n0, stg);
+            row_epilogue<BN>(ep, ld, m, n0, stg, &map_out);
           }
         }
         asm volatile("bar.sync 1, 128;" ::: "memory");       // s_last is reused by the next unit
@@ -769,6 +791,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     }
   }
 
+  if (warp >= 2) tma_store_drain_all(threadIdx.x & 31);   // the output boxes handed to the TMA unit have been written
   griddep_launch();   // this CTA's work is done: the next kernel's CTAs may be scheduled onto freed SMs
   tc_fence_before();
   __syncthreads();
@@ -829,6 +852,24 @@ const CUtensorMap* get_map(TcState* st, const void* ptr, uint64_t rows, uint64_t
   return &st->maps.emplace(key, m).first->second;
 }
 
+// Output [rows, cols] of 2- or 4-byte elements, row-major: box = 32 rows x 64 bytes, 64-byte swizzle
+const CUtensorMap* get_out_map(TcState* st, const void* ptr, uint64_t rows, uint64_t cols, int elem_bytes) {
+  MapKey key{ptr, rows, cols, (uint32_t)(0x10000 + elem_bytes)};
+  auto it = st->maps.find(key);
+  if (it != st->maps.end()) return &it->second;
+  if (st->maps.size() > 4096) st->maps.clear();
+  CUtensorMap m;
+  cuuint64_t dims[2] = {cols, rows};
+  cuuint64_t strides[1] = {cols * (uint64_t)elem_bytes};
+  cuuint32_t box[2] = {(cuuint32_t)(64 / elem_bytes), 32};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = st->encode(&m, elem_bytes == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2,
+                          const_cast<void*>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                          CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return nullptr;
+  return &st->maps.emplace(key, m).first->second;
+}
+
 template <int BN, bool PAIR>
 bool launch_bn(TcState* st, int idx, const GemmArgs& a, const EpiParams& ep, bool stream_k, cudaStream_t stream) {
   using Cfg = TcCfg<BN, PAIR>;
@@ -845,6 +886,12 @@ bool launch_bn(TcState* st, int idx, const GemmArgs& a, const EpiParams& ep, boo
   const CUtensorMap* mx = get_map(st, a.x, a.M, a.K, thin ? 32 : BM);
   const CUtensorMap* mw = get_map(st, a.w, w_rows, a.K, (swiglu || PAIR) ? BN / 2 : BN);
   if (!mx || !mw) return false;
+  // the epilogue stores through the TMA unit (of the rotary / KV-append epilogue: the rotated queries [M, n_q * d];
+  // K and V are scattered into the paged pool by hand)
+  const bool f32 = a.epi == EPI_PLAIN_F32 || a.epi == EPI_RESIDUAL;
+  const CUtensorMap* mo = get_out_map(st, a.out, a.M, a.epi == EPI_QKV_ROPE ? (uint64_t)a.n_q * a.head_dim : (uint64_t)a.N,
+                                      f32 ? 4 : 2);
+  if (!mo) return false;
   const int out_per_tile = swiglu ? BN / 2 : BN;
   const int n_tiles_n = (a.N + out_per_tile - 1) / out_per_tile;
   const int mt = (a.M + kRows - 1) / kRows;
@@ -890,7 +937,7 @@ bool launch_bn(TcState* st, int idx, const GemmArgs& a, const EpiParams& ep, boo
   }
   cfg.attrs = attr;
   cfg.numAttrs = n_attr;
-  return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<BN, PAIR>, *mx, *mw, a.M, n_tiles_n, a.K, a.N, dp_tiles, per, thin,
+  return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<BN, PAIR>, *mx, *mw, *mo, a.M, n_tiles_n, a.K, a.N, dp_tiles, per, thin,
                             st->split_ws, st->split_counters, ep) == cudaSuccess;
 }
 
