@@ -256,9 +256,9 @@ def run_ours(args, env):
         n_gemm_launch = sum(launches[k] for k in gemm_classes)
         ach = gemm_flops / (gemm_ms / 1e3) / 1e12
         # DRAM traffic of one launch of the largest projection (gate|up, M = 480), from the ncu capture summarised in
-        # profiles/gemm_tc_kernel_shapes.md: 265.8 MB read + 54.0 MB written, against 2 x 28672 x 4096 x 2 B of weights
+        # profiles/gemm_tc_kernel_shapes.md: 264.1 MB read + 53.7 MB written, against 2 x 28672 x 4096 x 2 B of weights
         # + x + y = 266.4 MB algorithmic.  The mix of shapes in a step has no single per-launch figure.
-        out["roofline"] = roofline_entry("tensor", ach, peaks["bf16_tflops_sustained"], 319.8e6,
+        out["roofline"] = roofline_entry("tensor", ach, peaks["bf16_tflops_sustained"], 317.8e6,
                                          f"projection GEMM kernel (tcgen05), {n_gemm_launch} launches, avg "
                                          f"{gemm_ms / max(n_gemm_launch, 1) * 1e3:.1f} us; peak = sustained bf16 of {peaks['source']}; "
                                          "traffic = DRAM bytes of one gate|up launch at M = 480 under ncu (algorithmic 266.4e6)")
