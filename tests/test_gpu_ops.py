@@ -280,6 +280,35 @@ def test_linear(M, N, K, flags):
     ctx.recg_free()
 
 
+def test_linear_random_shapes():
+    """Seeded sweep over row counts, widths that are not multiples of the tile widths (N % 16 == 0 only) and depths:
+    every tile decomposition the scheduler can pick, the clipped right edge and the clipped last rows, both output
+    types.  The output buffer is poisoned and padded so that a store beyond the matrix would show."""
+    rng = np.random.default_rng(77)
+    shape = synth.tiny_shape()
+    ctx = ops_ctx(shape, 1, 8, 1)
+    for case in range(48):
+        M = int(rng.choice([1, 2, 15, 17, 31, 32, 33, 63, 64, 65, 100, 127, 128, 129, 200, 255, 257, 376, 400, 480, 513, 700]))
+        N = 16 * int(rng.integers(1, 80)) if case % 3 else 16 * int(rng.integers(80, 700))
+        K = 64 * int(rng.integers(1, 24))
+        out_dtype = torch.bfloat16 if case % 2 else torch.float32
+        g = torch.Generator().manual_seed(1000 + case)
+        x = torch.randn((M, K), generator=g).to(torch.bfloat16)
+        w = (torch.randn((N, K), generator=g) * 0.05).to(torch.bfloat16)
+        ref = x.double().numpy() @ w.double().numpy().T
+        buf = torch.full((M + 2, N), float("nan"), dtype=out_dtype, device="cuda")   # two guard rows behind the matrix
+        xd, wd = x.cuda(), w.cuda()
+        ctx._check(binding.lib().recg_linear(ctx.h, xd.data_ptr(), wd.data_ptr(), buf.data_ptr(), M, N, K,
+                                             binding.DTYPE_BF16 if out_dtype == torch.bfloat16 else binding.DTYPE_F32))
+        ctx.recg_sync()
+        got = f64(buf[:M])
+        assert not np.isnan(got).any(), (M, N, K)
+        assert torch.isnan(buf[M:].float()).all(), f"stored beyond the last row: {(M, N, K)}"
+        tol = 1e-4 if out_dtype == torch.float32 else 5e-3       # bf16 output: half an ulp is 2^-9
+        assert np.max(np.abs(got - ref)) / np.max(np.abs(ref)) < tol, (M, N, K, str(out_dtype))
+    ctx.recg_free()
+
+
 @pytest.mark.parametrize("force", ["512,0", "512,1", "256,1", "128,1", "64,1", "256,0"])
 def test_linear_forced_decompositions(force, monkeypatch):
     """Every tile width and decomposition of the projection kernel on shapes that make it cut tiles: CTA pairs
