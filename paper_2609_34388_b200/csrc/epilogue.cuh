@@ -13,7 +13,7 @@ struct EpiParams {
   int M, N;       // logical output extent (EPI_SWIGLU: N = F)
   // EPI_QKV_ROPE
   const int* tok_slot;
-  const float2* rope_cs;  // [M][head_dim/2] (cos, sin) of each token's position
+  const float2* rope_cs;  // [head_dim/2][M] (cos, sin) of each token's position, frequency-major
   __nv_bfloat16* kv_pool;
   int64_t n_pages;
   int layer, n_q, n_kv, head_dim;
@@ -58,7 +58,7 @@ __device__ __forceinline__ void tile_epilogue(const EpiParams& ep, const float* 
       const float* x = tile + (size_t)r * ld + hl * D;
       float lo0 = x[i], lo1 = x[i + 1], hi0 = x[i + half], hi1 = x[i + half + 1];
       if (head < ep.n_q + ep.n_kv) {
-        const float2 cs0 = ep.rope_cs[(size_t)m * half + i], cs1 = ep.rope_cs[(size_t)m * half + i + 1];
+        const float2 cs0 = ep.rope_cs[(size_t)i * ep.M + m], cs1 = ep.rope_cs[(size_t)(i + 1) * ep.M + m];
         const float a0 = lo0 * cs0.x - hi0 * cs0.y, b0 = hi0 * cs0.x + lo0 * cs0.y;
         const float a1 = lo1 * cs1.x - hi1 * cs1.y, b1 = hi1 * cs1.x + lo1 * cs1.y;
         lo0 = a0; hi0 = b0; lo1 = a1; hi1 = b1;

@@ -451,10 +451,10 @@ __device__ __forceinline__ void row_epilogue(const EpiParams& ep, const Loader& 
         load(hl * D + c * 32, lo);
         load(hl * D + half + c * 32, hi);
         if (row_ok && !is_v) {
-          const float2* cs = ep.rope_cs + (size_t)m * half + c * 32;
+          const float2* cs = ep.rope_cs + (size_t)(c * 32) * ep.M + m;   // [frequency][token]
 #pragma unroll
           for (int i = 0; i < 32; ++i) {
-            const float2 t = cs[i];
+            const float2 t = cs[(size_t)i * ep.M];
             const float a = lo[i] * t.x - hi[i] * t.y, b = hi[i] * t.x + lo[i] * t.y;
             lo[i] = a;
             hi[i] = b;

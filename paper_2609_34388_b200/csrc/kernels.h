@@ -62,7 +62,7 @@ void launch_embed(const BatchLayout& bl, const Dims& dm, const void* embed, floa
 // x = rmsnorm(h) * g, bf16 out.
 void launch_rmsnorm(const float* h, const void* gain, void* x, int rows, int hidden, float eps, cudaStream_t st);
 
-// (cos, sin) of pos * base^(-2i/d), angles evaluated in double: cs float2 [T][head_dim/2].
+// (cos, sin) of pos * base^(-2i/d), angles evaluated in double: cs float2 [head_dim/2][T] (frequency-major).
 void launch_rope_table(const int* tok_pos, int n_tok, int head_dim, float rope_base, void* cs, cudaStream_t st);
 
 // Projection epilogues.
@@ -85,7 +85,7 @@ struct GemmArgs {
   void* kv_pool;
   int64_t n_pages;
   int layer, n_q, n_kv, head_dim;
-  const void* rope_cs;  // float2 [M][head_dim/2]: (cos, sin) of each token's rotary angles
+  const void* rope_cs;  // float2 [head_dim/2][M]: (cos, sin) of each token's rotary angles, frequency-major
 };
 // legacy tensor path (mma.sync), any M; N multiple of 64 (EPI_SWIGLU: F multiple of 32), K multiple of 32
 void launch_gemm_simt(const GemmArgs& a, int* status, cudaStream_t st);

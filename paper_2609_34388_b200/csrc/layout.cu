@@ -380,9 +380,11 @@ __global__ void rope_table_kernel(const int* __restrict__ tok_pos, int n_tok, in
                                   float2* __restrict__ cs) {
   griddep_launch();
   griddep_wait();
+  // frequency-major [half][n_tok]: the projection epilogue has one token per thread, so a warp reads 32 consecutive
+  // tokens of one frequency in one 256-byte request
   const int idx = blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= n_tok * half) return;
-  const int t = idx / half, i = idx % half;
+  const int i = idx / n_tok, t = idx % n_tok;
   const double theta = exp(-log_base * (double)i / (double)half);  // base^(-2i/d)
   const double ang = (double)tok_pos[t] * theta;
   cs[idx] = make_float2((float)cos(ang), (float)sin(ang));
