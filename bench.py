@@ -469,7 +469,10 @@ def bench_c128(binding, W, shape, peaks, args):
     # the same requests without them
     ov_plain = {"c16": c16_descriptor(3), "c1": c1_descriptor(11)}
     ov_descs = {k: synth.with_correction_branches(d, shape.vocab, 2, seed=60) for k, d in ov_plain.items()}
-    all_descs = [desc] + list(sweep_descs.values()) + list(ov_descs.values())
+    # forward time against concurrency for one block size at a time (the paper's Fig. 2b on random weights): T_C(B), the
+    # profile the block-size rule weighs against the expected progress
+    tcb_descs = {(C, B): synth.batch_descriptor(C, [B], None, 512, 8192, seed=80 + C) for C in (1, 4, 16, 64, 128) for B in (8, 16, 32)}
+    all_descs = [desc] + list(sweep_descs.values()) + list(ov_descs.values()) + list(tcb_descs.values())
     n_pages = max(d.n_pages for d in all_descs)
     free_b, _ = torch.cuda.mem_get_info()
     cfg = binding.make_config(shape, 128, max(2048, max(d.n_tokens for d in all_descs)), max(d.page_table.shape[1] for d in all_descs))
@@ -509,6 +512,25 @@ def bench_c128(binding, W, shape, peaks, args):
     sweep_result = {"workload": "configs[2] recipe at other batch sizes, one draw each, processed tokens/s of the whole step; "
                                             "ideal_ms = max(weight stream, GEMM flops at sustained peak) + KV stream, of measured peaks",
                                 "points": sweep}
+    tcb = []
+    for (C, B), d in tcb_descs.items():
+        ysw = synth.token_ids(int(d.verify_len.sum()), shape.vocab, seed=90)
+        bt = binding.Batch(d.ctx_len, d.verify_len, d.block_size, ysw, d.page_table, pool, n_pages)
+        vo = binding.VerifyOut(bt.n_req, bt.n_tok, bt.n_ver, host=False)
+        n_it = 4 if C >= 64 else 20          # short steps: enough of them for the clocks to settle
+        for _ in range(n_it):
+            ctx.recg_step(bt)
+            ctx.recg_verify(bt, out=vo)
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(n_it):
+            ctx.recg_step(bt)
+            ctx.recg_verify(bt, out=vo)
+        e1.record()
+        torch.cuda.synchronize()
+        tcb.append({"concurrency": C, "block": B, "rows": bt.n_tok, "ms_per_step": round(e0.elapsed_time(e1) / n_it, 3)})
+    tcb_result = {"workload": "whole step, every request with verify_len = block = B, context U[512,8192], one draw per point",
+                  "points": tcb}
     # ---- one ragged mixed batch against one batch per block size (the remedy of padded kernels) ----
     from paper_2609_34388_b200 import schedule
     bucketing = []
@@ -619,6 +641,7 @@ def bench_c128(binding, W, shape, peaks, args):
                          "frac_of_hbm_measured": round(attn_gbs / peaks["hbm_gbs"], 4)}}
     out["concurrency_sweep"] = sweep_result
     out["bucketing"] = bucketing_result
+    out["forward_time_by_block"] = tcb_result
     # block-size rule on the device after the verification of the 128-request batch (one small kernel; launch bound)
     tb = synth.policy_table()
     ctx.recg_policy_load(tb["blocks"], tb["s_edges"], tb["value"], tb["cost"])
