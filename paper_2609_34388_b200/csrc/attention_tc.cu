@@ -38,6 +38,7 @@
 #include <cuda.h>
 #include <cstdio>
 #include <cstdlib>
+#include <mutex>
 
 #include "common.cuh"
 #include "kernels.h"
@@ -666,23 +667,28 @@ struct QMapEntry {
   CUtensorMap map;
 };
 
-// q is bf16 [n_tok][n_q][128]; box = 64 dims x group heads x (128 / group) tokens, 128-byte swizzle, zero fill
-const CUtensorMap* q_tensor_map(const void* q, int n_tok, int n_q, int group) {
+// q is bf16 [n_tok][n_q][128]; box = 64 dims x group heads x (128 / group) tokens, 128-byte swizzle, zero fill.
+// The map is copied out under a lock: contexts on several host threads share the small cache.
+bool q_tensor_map(const void* q, int n_tok, int n_q, int group, CUtensorMap* out) {
+  static std::mutex mu;
   static EncodeTiledFn encode = nullptr;
   static QMapEntry cache[16];
   static int n_cached = 0, next_slot = 0;
   int device = 0;
   cudaGetDevice(&device);   // an address means something else on another device
+  std::lock_guard<std::mutex> lock(mu);
   for (int i = 0; i < n_cached; ++i)
     if (cache[i].q == q && cache[i].n_tok == n_tok && cache[i].n_q == n_q && cache[i].group == group &&
-        cache[i].device == device)
-      return &cache[i].map;
+        cache[i].device == device) {
+      *out = cache[i].map;
+      return true;
+    }
   if (!encode) {
     void* fn = nullptr;
     cudaDriverEntryPointQueryResult qres;
     if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
         qres != cudaDriverEntryPointSuccess || !fn)
-      return nullptr;
+      return false;
     encode = reinterpret_cast<EncodeTiledFn>(fn);
   }
   QMapEntry& e = cache[next_slot];
@@ -690,14 +696,16 @@ const CUtensorMap* q_tensor_map(const void* q, int n_tok, int n_q, int group) {
   cuuint64_t strides[2] = {(cuuint64_t)D * 2, (cuuint64_t)n_q * D * 2};
   cuuint32_t box[3] = {64, (cuuint32_t)group, (cuuint32_t)(128 / group)};
   cuuint32_t estr[3] = {1, 1, 1};
+  e.q = nullptr;   // the slot is invalid until the new map is in place
   if (encode(&e.map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(q), dims, strides, box, estr,
              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-    return nullptr;
+    return false;
   e.q = q; e.n_tok = n_tok; e.n_q = n_q; e.group = group; e.device = device;
   next_slot = (next_slot + 1) % 16;
   if (n_cached < 16) ++n_cached;
-  return &e.map;
+  *out = e.map;
+  return true;
 }
 
 }  // namespace
@@ -728,12 +736,15 @@ void launch_attention_tc_main(const BatchLayout& bl, const Dims& dm, int layer, 
   P.part_o = part_o;
   P.part_ml = part_ml;
   P.status = status;
-  const CUtensorMap* qmap = q_tensor_map(q, bl.n_tok, dm.n_q, P.group);
-  if (!qmap) {
+  CUtensorMap qmap;
+  if (!q_tensor_map(q, bl.n_tok, dm.n_q, P.group, &qmap)) {
+    // nothing is launched; the status word makes the next recg_sync() fail instead of returning stale outputs
     fprintf(stderr, "recg: cannot encode the tensor map over q\n");
+    static const int code = DEV_BAD_INDEX;
+    if (status) cudaMemcpyAsync(status, &code, sizeof(int), cudaMemcpyHostToDevice, st);
     return;
   }
-  launch_pdl(attention_tc_kernel, dim3(n_sm), dim3(kThreads), kSmemBytes, st, *qmap, P);
+  launch_pdl(attention_tc_kernel, dim3(n_sm), dim3(kThreads), kSmemBytes, st, qmap, P);
 }
 
 }  // namespace recg
