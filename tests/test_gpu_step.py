@@ -315,3 +315,43 @@ def test_bucketed_schedule_gives_the_same_results_as_the_mixed_batch():
     assert seen == len(specs)
     ctx.recg_sync()
     ctx.recg_free()
+
+
+def test_step_is_deterministic_and_survives_many_rounds():
+    """The same batch gives bit-identical logits and results every time (partial tiles are reduced in a fixed order, the
+    residual stream receives one addend per element and launch), also with other batches in between; and a longer run
+    over changing batches (with and without correction branches) leaves the device status clean."""
+    shape = synth.llama8b_shape(2)
+    shape.vocab = 8192
+    W = synth.model_weights(shape, seed=0, dtype=torch.bfloat16)
+    descs = [synth.batch_descriptor(12, [4, 8, 16, 32], None, 100, 2000, seed=900 + i) for i in range(4)]
+    descs += [synth.with_correction_branches(d, shape.vocab, 2, seed=910 + i) for i, d in enumerate(descs[:2])]
+    n_pages = sum(d.n_pages for d in descs)          # every batch gets pages of its own: nobody's context is overwritten
+    stride = max(d.page_table.shape[1] for d in descs)
+    ctx = binding.Context(binding.make_config(shape, 12, max(d.n_tokens for d in descs), stride), to_dev(W))
+    pool = binding.alloc_kv_pool(ctx, n_pages, fill="normal")
+    batches = []
+    first_page = 0
+    for i, d in enumerate(descs):
+        ys = synth.token_ids(int(d.verify_len.sum()), shape.vocab, seed=920 + i)
+        pt = np.where(d.page_table >= 0, d.page_table + first_page, -1).astype(np.int32)
+        first_page += d.n_pages
+        batches.append(binding.Batch(d.ctx_len, d.verify_len, d.block_size, ys, pt, pool, n_pages, **d.branch_kwargs()))
+    first = {}
+    for rnd in range(30):
+        j = (rnd * 5 + rnd // 7) % len(batches)
+        # every batch rewrites the K/V of its new rows only, from its own inputs: its logits do not depend on what ran before
+        lg = ctx.logits_tensor(ctx.recg_step(batches[j]))
+        g = ctx.recg_verify(batches[j])
+        key = (lg, {k: v.copy() for k, v in g.items()})
+        if j not in first:
+            first[j] = key
+        else:
+            assert torch.equal(lg, first[j][0]), f"logits of batch {j} changed in round {rnd}"
+            for k, v in key[1].items():
+                assert np.array_equal(v, first[j][1][k], equal_nan=True), (k, j, rnd)
+        if rnd % 10 == 9:
+            ctx.recg_sync()
+    assert len(first) == len(batches)
+    ctx.recg_sync()
+    ctx.recg_free()
