@@ -831,7 +831,7 @@ struct TcState {
   int* split_counters = nullptr;
   EncodeTiledFn encode = nullptr;
   std::unordered_map<MapKey, CUtensorMap, MapKeyHash> maps;
-  bool configured[4] = {false, false, false, false};
+  bool configured[5] = {false, false, false, false, false};
 };
 
 // [rows, cols] bf16 row-major, box = [box_rows, 64 columns], 128-byte swizzle, zero fill out of bounds
@@ -1003,16 +1003,19 @@ bool launch_gemm_tc(const GemmArgs& a, void* tc_state, int* status, cudaStream_t
   int best_bn = 0;
   bool best_sk = false, best_pair = false;
   double best_t = 1e30;
-  // configurations: single CTAs with 128-row tiles of width 256 / 128 / 64, and CTA pairs with 256 x 256 tiles (a
-  // k-block of a pair takes about 0.87 of the single CTA's, for twice the rows: the pair halves the weight bytes
-  // each SM's tensor core pulls out of its own shared memory)
-  const int bns[4] = {256, 128, 64, 256};
-  const double kb_tensor[4] = {0.44, 0.27, 0.22, 0.385};
+  // configurations: single CTAs with 128-row tiles of width 256 / 128 / 64, and CTA pairs with 256 x 256 or 256 x 128
+  // tiles (a k-block of a pair takes about 0.87 / 0.76 of the single CTA's, for twice the rows: the pair halves the
+  // weight bytes each SM's tensor core pulls out of its own shared memory)
+  constexpr int kConfigs = 5;
+  const int bns[kConfigs] = {256, 128, 64, 256, 128};
+  const double kb_tensor[kConfigs] = {0.44, 0.27, 0.22, 0.385, 0.205};
   const bool pair_ok = a.M > BM && (swiglu ? a.N % 128 == 0 : a.N % 256 == 0) && !(a.epi == EPI_QKV_ROPE && 256 % a.head_dim);
-  for (int bi = 0; bi < 4; ++bi) {
+  const bool pair128_ok = a.M > BM && !swiglu && a.N % 128 == 0 && !(a.epi == EPI_QKV_ROPE && 128 % a.head_dim);
+  for (int bi = 0; bi < kConfigs; ++bi) {
     const int bn = bns[bi];
-    const bool pair = bi == 3;
-    if (pair && !pair_ok) continue;
+    const bool pair = bi >= 3;
+    if (bi == 3 && !pair_ok) continue;
+    if (bi == 4 && !pair128_ok) continue;
     const int rows_tile = pair ? 2 * BM : BM;
     const int units = pair ? st->n_sm / 2 : st->n_sm;            // CTAs or clusters
     const int mtc = (a.M + rows_tile - 1) / rows_tile;
@@ -1046,7 +1049,10 @@ bool launch_gemm_tc(const GemmArgs& a, void* tc_state, int* status, cudaStream_t
       best_t = t_sk; best_bn = bn; best_sk = true; best_pair = pair;
     }
   }
-  if (st->force_bn == 512) {    // tuning aid: the CTA-pair kernel, "512,<0 whole tiles | 1 stream-K>"
+  if (st->force_bn == 384) {    // tuning aid: CTA pairs with 256 x 128 tiles, "384,<0 whole tiles | 1 stream-K>"
+    if (pair128_ok && (a.M + 255) / 256 <= st->n_sm / 2) return launch_bn<128, true>(st, 4, a, ep, st->force_s != 0, stream);
+  } else
+  if (st->force_bn == 512) {    // tuning aid: the 256 x 256 CTA-pair kernel, "512,<0 whole tiles | 1 stream-K>"
     if (pair_ok && (a.M + 255) / 256 <= st->n_sm / 2) return launch_bn<256, true>(st, 3, a, ep, st->force_s != 0, stream);
   } else
   if (st->force_bn) {   // tuning aid: RECG_GEMM_FORCE="<bn>,<0 whole tiles | 1 stream-K>"; ignored where it does not fit
@@ -1063,6 +1069,7 @@ bool launch_gemm_tc(const GemmArgs& a, void* tc_state, int* status, cudaStream_t
   }
   if (!best_bn) return false;
   if (swiglu && (a.N % 32)) return false;
+  if (best_pair && best_bn == 128) return launch_bn<128, true>(st, 4, a, ep, best_sk, stream);
   if (best_pair) return launch_bn<256, true>(st, 3, a, ep, best_sk, stream);
   switch (best_bn) {
     case 256: return launch_bn<256, false>(st, 0, a, ep, best_sk, stream);

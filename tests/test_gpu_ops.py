@@ -309,7 +309,7 @@ def test_linear_random_shapes():
     ctx.recg_free()
 
 
-@pytest.mark.parametrize("force", ["512,0", "512,1", "256,1", "128,1", "64,1", "256,0"])
+@pytest.mark.parametrize("force", ["512,0", "512,1", "384,0", "384,1", "256,1", "128,1", "64,1", "256,0"])
 def test_linear_forced_decompositions(force, monkeypatch):
     """Every tile width and decomposition of the projection kernel on shapes that make it cut tiles: CTA pairs
     (512 = 256-row tiles over clusters of two), stream-K with the reduction through the idle operand ring (last
