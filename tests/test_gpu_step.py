@@ -347,7 +347,7 @@ def test_step_is_deterministic_and_survives_many_rounds():
         if j not in first:
             first[j] = key
         else:
-            assert torch.equal(lg, first[j][0]), f"logits of batch {j} changed in round {rnd}"
+            assert torch.equal(lg, first[j][0]), f"logits of batch {j} changed in iteration {rnd}"
             for k, v in key[1].items():
                 assert np.array_equal(v, first[j][1][k], equal_nan=True), (k, j, rnd)
         if rnd % 10 == 9:
