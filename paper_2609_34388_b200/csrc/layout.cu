@@ -31,7 +31,7 @@ __device__ __forceinline__ int upper_request(const int* cu, int n_req, int t) {
 // a tile whose blocks are cut by range boundaries gets one partial slot per piece.
 // Items: [line A, first siblings | line A, second siblings (same order) | line B]; cta_off holds, per CTA, two
 // index ranges it walks one after the other (the second one is empty in this division).
-constexpr int kItemCost = 3;
+constexpr int kItemCost = 4;
 
 __global__ void __launch_bounds__(1024) layout_kernel(BatchLayout bl, int n_kv, int mask_id, int tok_per_tile,
                                                       int n_ctas, int64_t n_pages, int* status) {
