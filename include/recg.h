@@ -49,7 +49,10 @@ typedef enum { RECG_MEM_DEVICE = 0, RECG_MEM_HOST = 1 } recg_mem;
 enum {
   RECG_FLAG_LOGITS_BF16 = 1, /* recg_step() stores logits as bf16 instead of fp32               */
   RECG_FLAG_SIMT_GEMM = 2,   /* run the projections on the legacy mma.sync kernel (A/B checks)  */
-  RECG_FLAG_SIMT_ATTENTION = 4 /* run attention on the legacy mma.sync kernel (A/B checks)      */
+  RECG_FLAG_SIMT_ATTENTION = 4, /* run attention on the legacy mma.sync kernel (A/B checks)     */
+  RECG_FLAG_DEBUG_CHECKS = 8 /* guard bands behind every workspace region, checked by recg_sync() (RECG_ERR_INTERNAL
+                                if a kernel wrote past the end of one), and a host check that no page which receives
+                                new rows is named by two requests (RECG_ERR_INVALID_ARG)          */
 };
 
 typedef struct recg_ctx recg_ctx;
@@ -61,8 +64,8 @@ typedef struct {
   float rms_eps;
   int32_t mask_token_id;  /* id fed to the mask rows; < 0 means vocab - 1                        */
   int32_t page_size;      /* tokens per KV page; must be 16                                      */
-  int32_t max_requests;   /* capacity: requests per step                                         */
-  int32_t max_tokens;     /* capacity: rows of a step, the sum of n_r (see recg_batch)            */
+  int32_t max_requests;   /* capacity: requests per step, at most 4096                            */
+  int32_t max_tokens;     /* capacity: rows of a step, the sum of n_r (see recg_batch), at most 1048576 */
   int32_t max_pages_per_request;
   int32_t flags;          /* RECG_FLAG_*                                                         */
 } recg_config;
@@ -175,6 +178,7 @@ typedef struct {
   int32_t *next_draft, *cont_hit, *top1, *top2;
   float *p1, *p2, *entropy, *entropy_mean;
   int32_t *corr_hit, *risky_n, *risky_index, *risky_token;
+  int32_t *freed_page_ids;
 } recg_verify_out;
 
 /* Bytes of KV pool needed for n_pages physical pages (all layers). */
@@ -242,6 +246,24 @@ recg_status recg_linear(recg_ctx *ctx, const void *x, const void *w, void *y, in
  */
 recg_status recg_debug_buffer(recg_ctx *ctx, int32_t which, const void **ptr, int32_t *dtype, int32_t *rows,
                               int32_t *cols);
+
+/*
+ * Debugging aids (the paper has no counterpart).
+ * recg_debug_gemm_config(): force the tile configuration of the projection launches that follow on this context,
+ *   instead of the cost model's choice: tile = 64, 128 or 256 (single CTAs, 128-row tiles of that width), 384 (CTA
+ *   pairs, 256 x 128 tiles), 512 (CTA pairs, 256 x 256 tiles), 0 = back to the cost model; stream_k != 0 cuts the
+ *   K range of the tiles evenly over the SMs.  A configuration that does not fit a shape is ignored for that launch.
+ * recg_debug_wait_timeout(): enqueue a one-thread kernel that waits on a barrier nobody arrives on, bounded by
+ *   max_polls polls (1 .. 1048576) exactly like the waits inside the kernels; it gives up, records the timeout in the
+ *   device status word and returns.  The next recg_sync() then reports RECG_ERR_TIMEOUT and clears the word; the
+ *   context stays usable.  Nothing traps or faults.
+ * recg_debug_map_cache_selftest(): host only (no device needed): pushes n_keys distinct keys through the cache of
+ *   encoded tensor maps, three per simulated launch, and returns how many maps came back wrong (0 = pass);
+ *   *evictions receives how often the full cache was emptied on the way.
+ */
+recg_status recg_debug_gemm_config(recg_ctx *ctx, int32_t tile, int32_t stream_k);
+recg_status recg_debug_wait_timeout(recg_ctx *ctx, int32_t max_polls);
+int32_t recg_debug_map_cache_selftest(int32_t n_keys, int32_t *evictions);
 
 /*
  * Per-kernel-class device timing of recg_step()/recg_verify() for roofline reports (measurement aid; the

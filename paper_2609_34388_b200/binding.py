@@ -19,7 +19,7 @@ LIB_PATH = os.path.join(_HERE, "librecg.so")
 RECG_OK = 0
 DTYPE_BF16, DTYPE_F32 = 0, 1
 MEM_DEVICE, MEM_HOST = 0, 1
-FLAG_LOGITS_BF16, FLAG_SIMT_GEMM, FLAG_SIMT_ATTENTION = 1, 2, 4
+FLAG_LOGITS_BF16, FLAG_SIMT_GEMM, FLAG_SIMT_ATTENTION, FLAG_DEBUG_CHECKS = 1, 2, 4, 8
 STATUS_NAMES = {0: "RECG_OK", 1: "RECG_ERR_INVALID_ARG", 2: "RECG_ERR_SHAPE", 3: "RECG_ERR_CAPACITY",
                 4: "RECG_ERR_CUDA", 5: "RECG_ERR_TIMEOUT", 6: "RECG_ERR_INTERNAL"}
 
@@ -57,7 +57,7 @@ class recg_logits(C.Structure):
 _INT_OUT = ("accept_len", "n_emitted", "emitted", "new_ctx_len", "slot_state", "freed_pages", "next_draft", "cont_hit",
             "top1", "top2")
 _FLT_OUT = ("p1", "p2", "entropy", "entropy_mean")
-_INT_OUT_BRANCH = ("corr_hit", "risky_n", "risky_index", "risky_token")
+_INT_OUT_BRANCH = ("corr_hit", "risky_n", "risky_index", "risky_token", "freed_page_ids")
 
 
 class recg_verify_out(C.Structure):
@@ -107,9 +107,13 @@ def lib() -> C.CDLL:
         L.recg_policy_load.argtypes = [C.c_void_p, C.POINTER(recg_policy_table)]
         L.recg_policy_step.argtypes = [C.c_void_p, C.POINTER(recg_policy_state), C.c_void_p, C.c_void_p, C.c_void_p]
         L.recg_free.argtypes = [C.c_void_p]
+        L.recg_debug_gemm_config.argtypes = [C.c_void_p, C.c_int32, C.c_int32]
+        L.recg_debug_wait_timeout.argtypes = [C.c_void_p, C.c_int32]
+        L.recg_debug_map_cache_selftest.argtypes = [C.c_int32, C.POINTER(C.c_int32)]
+        L.recg_debug_map_cache_selftest.restype = C.c_int32
         for f in ("recg_init", "recg_step", "recg_verify", "recg_attention", "recg_kv_write", "recg_kv_read",
                   "recg_linear", "recg_debug_buffer", "recg_sync", "recg_free", "recg_timing_enable", "recg_timing_read",
-                  "recg_policy_load", "recg_policy_step"):
+                  "recg_policy_load", "recg_policy_step", "recg_debug_gemm_config", "recg_debug_wait_timeout"):
             getattr(L, f).restype = C.c_int32
         _lib = L
     return _lib
@@ -118,7 +122,8 @@ def lib() -> C.CDLL:
 EXPORTS = ("recg_kv_pool_bytes", "recg_init", "recg_step", "recg_verify", "recg_attention", "recg_kv_write",
            "recg_kv_read", "recg_linear", "recg_debug_buffer", "recg_sync", "recg_free", "recg_last_error",
            "recg_timing_enable", "recg_timing_read", "recg_row_stats_static", "recg_row_stats_static_error",
-           "recg_policy_load", "recg_policy_step")
+           "recg_policy_load", "recg_policy_step", "recg_debug_gemm_config", "recg_debug_wait_timeout",
+           "recg_debug_map_cache_selftest")
 TIMING_CLASSES = ("layout", "rmsnorm", "gemm_qkv", "attention", "gemm_o", "gemm_gate_up", "gemm_down", "lm_head", "verify")
 
 
@@ -177,7 +182,8 @@ class VerifyOut:
         self.sizes = {"accept_len": n_req, "n_emitted": n_req, "emitted": n_ver, "new_ctx_len": n_req,
                       "slot_state": n_tok, "freed_pages": n_req, "next_draft": n_tok - n_ver, "cont_hit": n_req,
                       "top1": n_tok, "top2": n_tok, "p1": n_tok, "p2": n_tok, "entropy": n_tok, "entropy_mean": n_req,
-                      "corr_hit": 2 * n_req, "risky_n": 3 * n_req, "risky_index": 6 * n_req, "risky_token": 6 * n_req}
+                      "corr_hit": 2 * n_req, "risky_n": 3 * n_req, "risky_index": 6 * n_req, "risky_token": 6 * n_req,
+                      "freed_page_ids": n_tok}
         self.bufs = {}
         self.c = recg_verify_out()
         self.c.mem = MEM_HOST if host else MEM_DEVICE
@@ -309,6 +315,12 @@ class Context:
         self._check(lib().recg_debug_buffer(self.h, which, C.byref(p), C.byref(dt), C.byref(r), C.byref(c)))
         return device_view(p.value, (r.value, c.value),
                            torch.bfloat16 if dt.value == DTYPE_BF16 else torch.float32).clone()
+
+    def recg_debug_gemm_config(self, tile: int, stream_k: bool):
+        self._check(lib().recg_debug_gemm_config(self.h, int(tile), 1 if stream_k else 0))
+
+    def recg_debug_wait_timeout(self, max_polls: int):
+        self._check(lib().recg_debug_wait_timeout(self.h, int(max_polls)))
 
     def recg_timing_enable(self, enable: bool):
         self._check(lib().recg_timing_enable(self.h, 1 if enable else 0))

@@ -12,7 +12,8 @@ enum : int {
   DEV_TIMEOUT_FULL = 1,   // consumer gave up waiting for a loaded stage
   DEV_TIMEOUT_EMPTY = 2,  // producer gave up waiting for a free stage
   DEV_TIMEOUT_MMA = 3,    // epilogue gave up waiting for an accumulator
-  DEV_BAD_INDEX = 4       // a page id or slot was out of range (access skipped)
+  DEV_BAD_INDEX = 4,      // a page id or slot was out of range (access skipped)
+  DEV_GUARD = 5           // a guard band behind a workspace region was overwritten (debug checks)
 };
 
 __device__ __forceinline__ void set_status(int* status, int code) {

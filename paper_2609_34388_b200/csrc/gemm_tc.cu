@@ -15,6 +15,7 @@
 
 #include <cstdio>
 #include <cstdlib>
+#include <cstring>
 #include <cmath>
 #include <mutex>
 #include <unordered_map>
@@ -188,21 +189,6 @@ __device__ __forceinline__ void tmem_dealloc_pair(uint32_t addr, uint32_t cols) 
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar_cluster) {
   asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar_cluster) : "memory");
 }
-// bounded wait that also orders against arrivals from the other CTA of the cluster
-__device__ __forceinline__ bool mbar_wait_cluster(uint64_t* bar, uint32_t parity, uint32_t max_iter) {
-  for (uint32_t i = 0; i < max_iter; ++i) {
-    uint32_t ok;
-    asm volatile(
-        "{\n .reg .pred p;\n mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
-        : "=r"(ok)
-        : "r"(smem_u32(bar)), "r"(parity)
-        : "memory");
-    if (ok) return true;
-    if (i > 64) __nanosleep(32);
-  }
-  return false;
-}
-
 
 // ---- register epilogue: one thread owns one output row -------------------------------------------
 
@@ -518,6 +504,34 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
   uint64_t* red_bar = tempty_bar + 2;      // completion of the partial tiles fetched into the idle ring (used once)
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(red_bar + 1);
 
+  // A wait that runs out records why and raises this CTA-wide flag.  The producer and the MMA issuer then leave
+  // their loops; the epilogue warps keep walking theirs WITHOUT blocking any more, so that all four of them still
+  // meet at every named barrier and every cut tile's arrival counter is still incremented (the counters stay
+  // consistent for the next launch; the outputs of this one are garbage and the status word says so).
+  __shared__ volatile int s_abort;
+  auto wait_or_abort = [&](uint64_t* bar, uint32_t parity, int code) -> bool {
+    if (s_abort) return false;
+    for (uint32_t i = 0; i < kSpin; ++i) {
+      uint32_t ok;
+      if constexpr (PAIR)
+        asm volatile(
+            "{\n .reg .pred p;\n mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+            : "=r"(ok)
+            : "r"(smem_u32(bar)), "r"(parity)
+            : "memory");
+      else
+        ok = mbar_try_wait(bar, parity) ? 1u : 0u;
+      if (ok) return true;
+      if (i > 64) {
+        if (s_abort) return false;
+        __nanosleep(32);
+      }
+    }
+    set_status(ep.status, code);
+    s_abort = 1;
+    return false;
+  };
+
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n_tiles_m = (M + kRows - 1) / kRows;
   const int n_tiles = n_tiles_m * n_tiles_n;
@@ -532,6 +546,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
   const int dp_count = unit < dp_tiles ? (dp_tiles - 1 - unit) / n_units + 1 : 0;
 
   if (threadIdx.x == 0) {
+    s_abort = 0;
     for (int s = 0; s < n_stages; ++s) {
       mbar_init(&full_bar[s], 1);
       mbar_init(&empty_bar[s], 1);
@@ -625,8 +640,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
             ++issued;
             continue;
           }
-          if (!(PAIR ? mbar_wait_cluster(&empty_bar[s], ph ^ 1, kSpin) : mbar_wait(&empty_bar[s], ph ^ 1, kSpin))) {
-            set_status(ep.status, DEV_TIMEOUT_EMPTY);
+          if (!wait_or_abort(&empty_bar[s], ph ^ 1, DEV_TIMEOUT_EMPTY)) {
             ok = false;
             break;
           }
@@ -656,19 +670,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
         const Piece pc = make_piece(jd, dp_tiles, pos, range_hi, KB, per, unit, n_units, n_tiles_m);
         const int kb0 = pc.kb0, kb1 = pc.kb1;
         const int acc = tcount & 1;
-        if (!(PAIR ? mbar_wait_cluster(&tempty_bar[acc], ((tcount >> 1) & 1) ^ 1, kSpin)
-                   : mbar_wait(&tempty_bar[acc], ((tcount >> 1) & 1) ^ 1, kSpin))) {
-          set_status(ep.status, DEV_TIMEOUT_MMA);
-          break;
-        }
+        if (!wait_or_abort(&tempty_bar[acc], ((tcount >> 1) & 1) ^ 1, DEV_TIMEOUT_MMA)) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + acc * BN;
         for (int kb = kb0; kb < kb1; ++kb) {
           const int s = st_idx;
           const uint32_t ph = st_phase;
           if (++st_idx == n_stages) { st_idx = 0; st_phase ^= 1; }
-          if (!(PAIR ? mbar_wait_cluster(&full_bar[s], ph, kSpin) : mbar_wait(&full_bar[s], ph, kSpin))) {
-            set_status(ep.status, DEV_TIMEOUT_FULL);
+          if (!wait_or_abort(&full_bar[s], ph, DEV_TIMEOUT_FULL)) {
             ok = false;
             break;
           }
@@ -705,10 +714,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
       const int tile = pc.tile, n_splits = pc.n_parts;
       const int tm = tile % n_tiles_m, tn = tile / n_tiles_m;
       const int acc = tcount & 1;
-      if (!(PAIR ? mbar_wait_cluster(&tfull_bar[acc], (tcount >> 1) & 1, kSpin) : mbar_wait(&tfull_bar[acc], (tcount >> 1) & 1, kSpin))) {
-        set_status(ep.status, DEV_TIMEOUT_MMA);
-        break;
-      }
+      wait_or_abort(&tfull_bar[acc], (tcount >> 1) & 1, DEV_TIMEOUT_MMA);   // after a timeout: carry on without blocking
       tc_fence_after();
       const uint32_t tacc = tmem_base + ((uint32_t)(quad * 32) << 16) + acc * BN;
       const int row_in_tile = quad * 32 + lane;
@@ -778,7 +784,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                 ++k;
               }
             }
-            if (!mbar_wait(red_bar, 0, kSpin)) set_status(ep.status, DEV_TIMEOUT_FULL);
+            wait_or_abort(red_bar, 0, DEV_TIMEOUT_FULL);
             RingLoader ld{tacc, reinterpret_cast<const float4*>(smem) + row_in_tile, BN, pc.part, n_splits};
             row_epilogue<BN>(ep, ld, m, n0, stg, &map_out);
           } else {
@@ -823,7 +829,10 @@ struct MapKeyHash {
 
 constexpr size_t kSplitWsBytes = 96ull << 20;   // partial tiles of split-K launches
 constexpr int kSplitCounters = 1 << 16;
+constexpr size_t kMapCacheMax = 4096;           // entries; the keys include the row count, so a serving loop keeps adding
 
+// Cache of encoded tensor maps (cached_map below).  Maps are handed out BY VALUE: a launch needs three maps at once,
+// and a miss on the second or third lookup may empty the full cache, so nothing may point into it.
 struct TcState {
   int n_sm = 0;
   int force_bn = 0, force_s = 0;
@@ -831,43 +840,52 @@ struct TcState {
   int* split_counters = nullptr;
   EncodeTiledFn encode = nullptr;
   std::unordered_map<MapKey, CUtensorMap, MapKeyHash> maps;
+  size_t evictions = 0;
   bool configured[5] = {false, false, false, false, false};
 };
 
-// [rows, cols] bf16 row-major, box = [box_rows, 64 columns], 128-byte swizzle, zero fill out of bounds
-const CUtensorMap* get_map(TcState* st, const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows) {
-  MapKey key{ptr, rows, cols, box_rows};
+template <typename Encode>
+bool cached_map(TcState* st, const MapKey& key, CUtensorMap* out, Encode&& encode) {
   auto it = st->maps.find(key);
-  if (it != st->maps.end()) return &it->second;
-  if (st->maps.size() > 4096) st->maps.clear();
+  if (it != st->maps.end()) {
+    *out = it->second;
+    return true;
+  }
   CUtensorMap m;
-  cuuint64_t dims[2] = {cols, rows};
-  cuuint64_t strides[1] = {cols * 2};
-  cuuint32_t box[2] = {BK, box_rows};
-  cuuint32_t estr[2] = {1, 1};
-  CUresult r = st->encode(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
-                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  if (r != CUDA_SUCCESS) return nullptr;
-  return &st->maps.emplace(key, m).first->second;
+  if (!encode(&m)) return false;
+  if (st->maps.size() >= kMapCacheMax) {   // emptied, never trimmed behind a caller's back: maps leave by value
+    st->maps.clear();
+    ++st->evictions;
+  }
+  st->maps.emplace(key, m);
+  *out = m;
+  return true;
+}
+
+// [rows, cols] bf16 row-major, box = [box_rows, 64 columns], 128-byte swizzle, zero fill out of bounds
+bool get_map(TcState* st, const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows, CUtensorMap* out) {
+  return cached_map(st, MapKey{ptr, rows, cols, box_rows}, out, [&](CUtensorMap* m) {
+    cuuint64_t dims[2] = {cols, rows};
+    cuuint64_t strides[1] = {cols * 2};
+    cuuint32_t box[2] = {BK, box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    return st->encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+  });
 }
 
 // Output [rows, cols] of 2- or 4-byte elements, row-major: box = 32 rows x 64 bytes, 64-byte swizzle
-const CUtensorMap* get_out_map(TcState* st, const void* ptr, uint64_t rows, uint64_t cols, int elem_bytes) {
-  MapKey key{ptr, rows, cols, (uint32_t)(0x10000 + elem_bytes)};
-  auto it = st->maps.find(key);
-  if (it != st->maps.end()) return &it->second;
-  if (st->maps.size() > 4096) st->maps.clear();
-  CUtensorMap m;
-  cuuint64_t dims[2] = {cols, rows};
-  cuuint64_t strides[1] = {cols * (uint64_t)elem_bytes};
-  cuuint32_t box[2] = {(cuuint32_t)(64 / elem_bytes), 32};
-  cuuint32_t estr[2] = {1, 1};
-  CUresult r = st->encode(&m, elem_bytes == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2,
-                          const_cast<void*>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                          CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  if (r != CUDA_SUCCESS) return nullptr;
-  return &st->maps.emplace(key, m).first->second;
+bool get_out_map(TcState* st, const void* ptr, uint64_t rows, uint64_t cols, int elem_bytes, CUtensorMap* out) {
+  return cached_map(st, MapKey{ptr, rows, cols, (uint32_t)(0x10000 + elem_bytes)}, out, [&](CUtensorMap* m) {
+    cuuint64_t dims[2] = {cols, rows};
+    cuuint64_t strides[1] = {cols * (uint64_t)elem_bytes};
+    cuuint32_t box[2] = {(cuuint32_t)(64 / elem_bytes), 32};
+    cuuint32_t estr[2] = {1, 1};
+    return st->encode(m, elem_bytes == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2,
+                      const_cast<void*>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                      CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+  });
 }
 
 template <int BN, bool PAIR>
@@ -883,15 +901,14 @@ bool launch_bn(TcState* st, int idx, const GemmArgs& a, const EpiParams& ep, boo
   const bool swiglu = a.epi == EPI_SWIGLU;
   const uint64_t w_rows = swiglu ? 2ull * a.N : (uint64_t)a.N;
   const int thin = (!PAIR && a.M <= 32) ? 1 : 0;
-  const CUtensorMap* mx = get_map(st, a.x, a.M, a.K, thin ? 32 : BM);
-  const CUtensorMap* mw = get_map(st, a.w, w_rows, a.K, (swiglu || PAIR) ? BN / 2 : BN);
-  if (!mx || !mw) return false;
+  CUtensorMap mx, mw, mo;     // copies: see cached_map
+  if (!get_map(st, a.x, a.M, a.K, thin ? 32 : BM, &mx)) return false;
+  if (!get_map(st, a.w, w_rows, a.K, (swiglu || PAIR) ? BN / 2 : BN, &mw)) return false;
   // the epilogue stores through the TMA unit (of the rotary / KV-append epilogue: the rotated queries [M, n_q * d];
   // K and V are scattered into the paged pool by hand)
   const bool f32 = a.epi == EPI_PLAIN_F32 || a.epi == EPI_RESIDUAL;
-  const CUtensorMap* mo = get_out_map(st, a.out, a.M, a.epi == EPI_QKV_ROPE ? (uint64_t)a.n_q * a.head_dim : (uint64_t)a.N,
-                                      f32 ? 4 : 2);
-  if (!mo) return false;
+  if (!get_out_map(st, a.out, a.M, a.epi == EPI_QKV_ROPE ? (uint64_t)a.n_q * a.head_dim : (uint64_t)a.N, f32 ? 4 : 2, &mo))
+    return false;
   const int out_per_tile = swiglu ? BN / 2 : BN;
   const int n_tiles_n = (a.N + out_per_tile - 1) / out_per_tile;
   const int mt = (a.M + kRows - 1) / kRows;
@@ -937,7 +954,7 @@ bool launch_bn(TcState* st, int idx, const GemmArgs& a, const EpiParams& ep, boo
   }
   cfg.attrs = attr;
   cfg.numAttrs = n_attr;
-  return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<BN, PAIR>, *mx, *mw, *mo, a.M, n_tiles_n, a.K, a.N, dp_tiles, per, thin,
+  return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<BN, PAIR>, mx, mw, mo, a.M, n_tiles_n, a.K, a.N, dp_tiles, per, thin,
                             st->split_ws, st->split_counters, ep) == cudaSuccess;
 }
 
@@ -954,7 +971,6 @@ void* tc_state_create(int n_sm) {
     return nullptr;
   }
   st->encode = reinterpret_cast<EncodeTiledFn>(fn);
-  if (const char* f = getenv("RECG_GEMM_FORCE")) sscanf(f, "%d,%d", &st->force_bn, &st->force_s);
   if (cudaMalloc(reinterpret_cast<void**>(&st->split_ws), kSplitWsBytes) != cudaSuccess ||
       cudaMalloc(reinterpret_cast<void**>(&st->split_counters), kSplitCounters * sizeof(int)) != cudaSuccess ||
       cudaMemset(st->split_counters, 0, kSplitCounters * sizeof(int)) != cudaSuccess) {
@@ -964,6 +980,53 @@ void* tc_state_create(int n_sm) {
     return nullptr;
   }
   return st;
+}
+
+void tc_state_force(void* s, int bn, int stream_k) {
+  TcState* st = static_cast<TcState*>(s);
+  if (!st) return;
+  st->force_bn = bn;
+  st->force_s = stream_k;
+}
+
+void tc_state_reset(void* s, cudaStream_t stream) {
+  TcState* st = static_cast<TcState*>(s);
+  if (st && st->split_counters) cudaMemsetAsync(st->split_counters, 0, kSplitCounters * sizeof(int), stream);
+}
+
+// Host-only check of the map cache: n_keys distinct keys go through it three at a time, the way a launch takes its
+// maps, with an encoder that writes the key into the map; every map handed out must still carry its own key after
+// the later lookups of the same launch (which may have emptied the cache).  Returns the number of wrong maps.
+int tc_map_cache_selftest(int n_keys, int* evictions) {
+  TcState st;
+  auto fake = [](const MapKey& k) {
+    return [k](CUtensorMap* m) {
+      memset(m, 0, sizeof(*m));
+      memcpy(m, &k, sizeof(k));
+      return true;
+    };
+  };
+  auto key_of = [](int i) { return MapKey{reinterpret_cast<const void*>(static_cast<uintptr_t>(4096) * (i + 1)), (uint64_t)i, 64, 128}; };
+  int bad = 0;
+  for (int i = 0; i + 2 < n_keys; i += 3) {
+    CUtensorMap m[3];
+    for (int j = 0; j < 3; ++j)
+      if (!cached_map(&st, key_of(i + j), &m[j], fake(key_of(i + j)))) ++bad;
+    auto carries = [](const CUtensorMap& m, const MapKey& k) {   // (field by field: the key has padding bytes)
+      MapKey got;
+      memcpy(&got, &m, sizeof(got));
+      return got == k;
+    };
+    for (int j = 0; j < 3; ++j)
+      if (!carries(m[j], key_of(i + j))) ++bad;
+    // an old key again: a hit, or a miss that re-encodes; either way the right map
+    CUtensorMap again;
+    const MapKey k0 = key_of(i / 2);
+    if (!cached_map(&st, k0, &again, fake(k0)) || !carries(again, k0)) ++bad;
+  }
+  if (st.maps.size() > kMapCacheMax) ++bad;
+  if (evictions) *evictions = (int)st.evictions;
+  return bad;
 }
 
 void tc_state_destroy(void* s) {
@@ -1055,7 +1118,7 @@ bool launch_gemm_tc(const GemmArgs& a, void* tc_state, int* status, cudaStream_t
   if (st->force_bn == 512) {    // tuning aid: the 256 x 256 CTA-pair kernel, "512,<0 whole tiles | 1 stream-K>"
     if (pair_ok && (a.M + 255) / 256 <= st->n_sm / 2) return launch_bn<256, true>(st, 3, a, ep, st->force_s != 0, stream);
   } else
-  if (st->force_bn) {   // tuning aid: RECG_GEMM_FORCE="<bn>,<0 whole tiles | 1 stream-K>"; ignored where it does not fit
+  if (st->force_bn) {   // tuning aid (tc_state_force): tile width, 0 whole tiles | 1 stream-K; ignored where it does not fit
     const int bn = st->force_bn;
     const int per = swiglu ? bn / 2 : bn;
     const bool shape_ok = (bn == 256 || bn == 128 || bn == 64) &&

@@ -57,6 +57,13 @@ struct BatchLayout {
 // S1: per-token arrays and the attention work list.
 void launch_layout(const BatchLayout& bl, const Dims& dm, int tok_per_tile, int n_ctas, int64_t n_pages,
                    int* status, cudaStream_t st);
+// the layout kernel keeps eight ints per request in shared memory: requests per step are bounded by this
+constexpr int kMaxLayoutRequests = 4096;
+size_t layout_smem_bytes(int n_req, int n_ctas);
+// debug checks
+void launch_guard_fill(void* base, const size_t* offs_dev, int n, cudaStream_t st);
+void launch_guard_check(const void* base, const size_t* offs_dev, int n, int* status, cudaStream_t st);
+void launch_wait_timeout(uint32_t max_polls, int* status, cudaStream_t st);
 // S2: h[t] = embed[tok_id[t]] (fp32 residual stream).
 void launch_embed(const BatchLayout& bl, const Dims& dm, const void* embed, float* h, cudaStream_t st);
 // x = rmsnorm(h) * g, bf16 out.
@@ -94,6 +101,13 @@ struct TcGemmPlan;  // opaque: cached tensor maps
 bool launch_gemm_tc(const GemmArgs& a, void* tc_state, int* status, cudaStream_t st);
 void* tc_state_create(int n_sm);
 void tc_state_destroy(void* s);
+// debugging aid: force the tile configuration of the following launches (bn 64 / 128 / 256 single CTAs, 384 = CTA pairs
+// with 256 x 128 tiles, 512 = CTA pairs with 256 x 256 tiles; 0 = back to the cost model) and the decomposition
+void tc_state_force(void* s, int bn, int stream_k);
+// zero the arrival counters of cut tiles (after a launch that ended with an error status)
+void tc_state_reset(void* s, cudaStream_t st);
+// host-only self-test of the tensor-map cache; returns the number of wrong maps handed out
+int tc_map_cache_selftest(int n_keys, int* evictions);
 
 // S5
 // use_tc: run the tcgen05 kernel (head_dim 128 only); otherwise the mma.sync kernel
@@ -111,6 +125,7 @@ struct VerifyBuffers {   // DEVICE outputs (library workspace or caller buffers)
       *top2;
   float *p1, *p2, *entropy, *entropy_mean;
   int *corr_hit, *risky_n, *risky_index, *risky_token;
+  int *freed_page_ids;
 };
 struct RowPartial {      // per (row, vocab chunk)
   float m1, m2;          // largest and second-largest logit of the chunk

@@ -347,9 +347,16 @@ __global__ void kv_io_kernel(bool write, __nv_bfloat16* pool, int64_t n_pages, i
 
 }  // namespace
 
+size_t layout_smem_bytes(int n_req, int n_ctas) {
+  return (8 * (size_t)(n_req + 1) + (size_t)(n_ctas / 2 + 1) + (size_t)(n_ctas + 1)) * sizeof(int);
+}
+
 void launch_layout(const BatchLayout& bl, const Dims& dm, int tok_per_tile, int n_ctas, int64_t n_pages,
                    int* status, cudaStream_t st) {
-  const size_t smem = (8 * (size_t)(bl.n_req + 1) + (size_t)(n_ctas / 2 + 1) + (size_t)(n_ctas + 1)) * sizeof(int);
+  const size_t smem = layout_smem_bytes(bl.n_req, n_ctas);
+  static bool configured[kMaxDevices] = {false};
+  if (first_use_on_device(configured))    // room for kMaxLayoutRequests requests (the default limit is 48 KB)
+    cudaFuncSetAttribute(layout_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)layout_smem_bytes(kMaxLayoutRequests, 1024));
   launch_pdl(layout_kernel, dim3(1), dim3(1024), smem, st, bl, dm.n_kv, dm.mask_id, tok_per_tile, n_ctas, n_pages, status);
 }
 
@@ -397,5 +404,42 @@ void launch_rope_table(const int* tok_pos, int n_tok, int head_dim, float rope_b
   if (total <= 0) return;
   launch_pdl(rope_table_kernel, dim3((total + 255) / 256), dim3(256), 0, st, tok_pos, n_tok, half,
              log((double)rope_base), static_cast<float2*>(cs));
+}
+}  // namespace recg
+
+// ---------------------------------------------------------------------------------------------------
+// Debug checks: guard bands behind the workspace regions, and a wait that is meant to run out.
+// ---------------------------------------------------------------------------------------------------
+namespace recg {
+namespace {
+constexpr uint32_t kGuardWord = 0x5ca1ab1eu;
+
+// grid = bands, 64 threads: 256 bytes each
+__global__ void guard_fill_kernel(uint8_t* base, const size_t* __restrict__ offs) {
+  reinterpret_cast<uint32_t*>(base + offs[blockIdx.x])[threadIdx.x] = kGuardWord;
+}
+__global__ void guard_check_kernel(const uint8_t* base, const size_t* __restrict__ offs, int* status) {
+  if (reinterpret_cast<const uint32_t*>(base + offs[blockIdx.x])[threadIdx.x] != kGuardWord) set_status(status, DEV_GUARD);
+}
+
+// One CTA, one thread: waits on an mbarrier that nobody ever arrives on, with the same bounded wait the kernels
+// use; when the polls are used up it records the timeout in the status word and returns.  Nothing else happens:
+// no trap, no fault, the context stays usable.
+__global__ void wait_timeout_kernel(uint32_t max_polls, int* status) {
+  __shared__ uint64_t bar;
+  mbar_init(&bar, 1);
+  fence_barrier_init();
+  if (!mbar_wait(&bar, 0, max_polls)) set_status(status, DEV_TIMEOUT_FULL);
+}
+}  // namespace
+
+void launch_guard_fill(void* base, const size_t* offs_dev, int n, cudaStream_t st) {
+  if (n > 0) guard_fill_kernel<<<n, 64, 0, st>>>(static_cast<uint8_t*>(base), offs_dev);
+}
+void launch_guard_check(const void* base, const size_t* offs_dev, int n, int* status, cudaStream_t st) {
+  if (n > 0) guard_check_kernel<<<n, 64, 0, st>>>(static_cast<const uint8_t*>(base), offs_dev, status);
+}
+void launch_wait_timeout(uint32_t max_polls, int* status, cudaStream_t st) {
+  wait_timeout_kernel<<<1, 1, 0, st>>>(max_polls, status);
 }
 }  // namespace recg

@@ -15,13 +15,23 @@ namespace {
 thread_local std::string g_init_error;
 constexpr size_t kVoutMirrorMax = 1 << 20;   // verify outputs up to this size come back to the host in one copy
 
-struct DeviceArena {  // one cudaMalloc, carved with 256-byte alignment
+// One cudaMalloc, carved with 256-byte alignment.  With guard = true (RECG_FLAG_DEBUG_CHECKS) every region is followed
+// by a 256-byte guard band; the offsets of the bands are recorded so that they can be filled with a pattern at init
+// and checked by recg_sync(): a kernel that writes past the end of a workspace region shows up there.
+struct DeviceArena {
   uint8_t* base = nullptr;
   size_t size = 0, used = 0;
+  bool guard = false;
+  std::vector<size_t> guards;   // byte offsets of the guard bands
   template <typename T> T* take(size_t n) {
     used = (used + 255) & ~size_t(255);
     T* p = reinterpret_cast<T*>(base ? base + used : nullptr);
     used += n * sizeof(T);
+    if (guard) {
+      used = (used + 255) & ~size_t(255);
+      guards.push_back(used);
+      used += 256;
+    }
     return p;
   }
 };
@@ -61,12 +71,15 @@ struct recg_ctx {
   uint8_t* h_vout = nullptr;             // ... mirrored by one pinned host buffer: a single copy brings all results back
   int* d_status = nullptr;
   int* d_page_row = nullptr;
+  size_t* d_guards = nullptr;    // RECG_FLAG_DEBUG_CHECKS: offsets of the guard bands, on the device
+  int n_guards = 0;
   int* d_policy = nullptr;       // block-size rule: [blocks x8 | cost x8 | edges x64 | value]
   PolicyTable policy{};
   bool policy_loaded = false;
   std::vector<int> h_policy;
   void* tc_state = nullptr;
   std::vector<int> h_desc;
+  std::vector<int> h_page_owner;   // debug checks: which request names a page
   // optional per-class timing
   bool timing = false;
   std::vector<cudaEvent_t> ev_pool;
@@ -153,6 +166,7 @@ size_t carve(recg_ctx* c, DeviceArena& A) {
   v.risky_n = A.take<int>(3 * Cm);
   v.risky_index = A.take<int>(6 * Cm);
   v.risky_token = A.take<int>(6 * Cm);
+  v.freed_page_ids = A.take<int>(Tm);
   c->vout_bytes = A.used - c->vout_off;
   c->q = A.take<__nv_bfloat16>(Tm * d.n_q * d.head_dim);
   c->o = A.take<__nv_bfloat16>(Tm * d.n_q * d.head_dim);
@@ -162,6 +176,13 @@ size_t carve(recg_ctx* c, DeviceArena& A) {
     c->act = A.take<__nv_bfloat16>(Tm * d.ffn);
     const size_t esz = (g.flags & RECG_FLAG_LOGITS_BF16) ? 2 : 4;
     c->logits = A.take<uint8_t>(Tm * (size_t)d.vocab * esz);
+  }
+  if (A.guard) {
+    c->n_guards = (int)A.guards.size();
+    const bool was = A.guard;
+    A.guard = false;
+    c->d_guards = A.take<size_t>(A.guards.size() + 1);
+    A.guard = was;
   }
   return A.used + 256;
 }
@@ -250,6 +271,26 @@ recg_status pack_batch(recg_ctx* ctx, const recg_batch* b, bool need_pages, bool
       }
     }
   }
+  if (pages && (ctx->cfg.flags & RECG_FLAG_DEBUG_CHECKS)) {
+    // debug checks: a page that takes new rows of one request must not appear in another request's table (two
+    // requests would overwrite each other's tentative K/V), nor twice in its own
+    std::vector<int>& seen = ctx->h_page_owner;
+    seen.assign((size_t)b->kv_pool_pages, -1);
+    for (int r = 0; r < C; ++r) {
+      const long long need = ((long long)b->ctx_len[r] + request_rows(b, r) + kPageSize - 1) / kPageSize;
+      const int first_new = b->ctx_len[r] / kPageSize;
+      for (int i = 0; i < need; ++i) {
+        const int pg = pt[(size_t)r * stride + i];
+        if (pg < 0 || pg >= b->kv_pool_pages) continue;    // reported above when a pool was given
+        const int tag = i >= first_new ? 2 * r + 1 : 2 * r;  // odd: the page takes new rows
+        const int old = seen[pg];
+        if (old >= 0 && ((old >> 1) == r || (old & 1) || (tag & 1)))
+          return fail(ctx, RECG_ERR_INVALID_ARG, "batch (debug checks): a page that receives new rows is named twice (requests " +
+                                                     std::to_string(old >> 1) + " and " + std::to_string(r) + ")");
+        if (old < 0 || (tag & 1)) seen[pg] = tag;
+      }
+    }
+  }
   BatchLayout& bl = ctx->bl;
   int* d = ctx->d_desc;
   bl.n_req = C;
@@ -314,6 +355,8 @@ recg_status recg_init(recg_ctx** out, const recg_config* cfg, const recg_weights
   if (g.n_layers < 0 || g.hidden <= 0 || g.n_q_heads <= 0 || g.n_kv_heads <= 0 || g.vocab <= 1 || g.ffn <= 0 ||
       g.max_requests <= 0 || g.max_tokens <= 0 || g.max_pages_per_request <= 0)
     return fail(ctx, RECG_ERR_INVALID_ARG, "recg_init: non-positive dimension or capacity");
+  if (g.max_requests > kMaxLayoutRequests || g.max_tokens > (1 << 20))
+    return fail(ctx, RECG_ERR_CAPACITY, "recg_init: at most 4096 requests and 1048576 rows per step");
   if (g.page_size != kPageSize) return fail(ctx, RECG_ERR_SHAPE, "recg_init: page_size must be 16");
   if (g.head_dim != 64 && g.head_dim != 128) return fail(ctx, RECG_ERR_SHAPE, "recg_init: head_dim must be 64 or 128");
   if (g.n_q_heads % g.n_kv_heads) return fail(ctx, RECG_ERR_SHAPE, "recg_init: n_q_heads must be a multiple of n_kv_heads");
@@ -360,6 +403,7 @@ recg_status recg_init(recg_ctx** out, const recg_config* cfg, const recg_weights
     }
   }
   DeviceArena probe;
+  probe.guard = ctx->arena.guard = (g.flags & RECG_FLAG_DEBUG_CHECKS) != 0;
   const size_t bytes = carve(ctx, probe);
   cudaError_t e = cudaMalloc(reinterpret_cast<void**>(&ctx->arena.base), bytes);
   if (e != cudaSuccess) {
@@ -370,6 +414,16 @@ recg_status recg_init(recg_ctx** out, const recg_config* cfg, const recg_weights
   }
   ctx->arena.size = bytes;
   carve(ctx, ctx->arena);
+  if (ctx->n_guards) {   // fill the guard bands behind every workspace region
+    if (cudaMemcpyAsync(ctx->d_guards, ctx->arena.guards.data(), ctx->n_guards * sizeof(size_t), cudaMemcpyHostToDevice,
+                        ctx->stream) != cudaSuccess || cudaStreamSynchronize(ctx->stream) != cudaSuccess) {
+      cudaFree(ctx->arena.base);
+      delete ctx;
+      ctx = nullptr;
+      return fail(ctx, RECG_ERR_CUDA, "recg_init: cannot upload the guard-band offsets");
+    }
+    launch_guard_fill(ctx->arena.base, ctx->d_guards, ctx->n_guards, ctx->stream);
+  }
   if (ctx->vout_bytes <= kVoutMirrorMax && cudaMallocHost(reinterpret_cast<void**>(&ctx->h_vout), ctx->vout_bytes) != cudaSuccess) {
     cudaGetLastError();
     ctx->h_vout = nullptr;   // fall back to one copy per output array
@@ -418,10 +472,17 @@ recg_status recg_free(recg_ctx* ctx) {
 recg_status recg_sync(recg_ctx* ctx) {
   if (!ctx) return RECG_ERR_INVALID_ARG;
   int st = 0;
+  if (ctx->n_guards) launch_guard_check(ctx->arena.base, ctx->d_guards, ctx->n_guards, ctx->d_status, ctx->stream);
   CU(cudaMemcpyAsync(&st, ctx->d_status, sizeof(int), cudaMemcpyDeviceToHost, ctx->stream));
   CU(cudaStreamSynchronize(ctx->stream));
   if (st != DEV_OK) {
     cudaMemsetAsync(ctx->d_status, 0, sizeof(int), ctx->stream);
+    // a projection that gave up may have left arrival counters of cut tiles behind: the next launch starts clean
+    tc_state_reset(ctx->tc_state, ctx->stream);
+    if (st == DEV_GUARD) {
+      launch_guard_fill(ctx->arena.base, ctx->d_guards, ctx->n_guards, ctx->stream);
+      return fail(ctx, RECG_ERR_INTERNAL, "device: a guard band behind a workspace region was overwritten");
+    }
     if (st == DEV_BAD_INDEX) return fail(ctx, RECG_ERR_INTERNAL, "device: a page id or slot was out of range");
     return fail(ctx, RECG_ERR_TIMEOUT, "device: a bounded wait gave up (code " + std::to_string(st) + ")");
   }
@@ -520,7 +581,7 @@ recg_status recg_verify(recg_ctx* ctx, const recg_batch* batch, const void* logi
 #define PICK(f) if (out->f) vb.f = out->f
     PICK(accept_len); PICK(n_emitted); PICK(emitted); PICK(new_ctx_len); PICK(slot_state); PICK(freed_pages);
     PICK(next_draft); PICK(cont_hit); PICK(top1); PICK(top2); PICK(p1); PICK(p2); PICK(entropy); PICK(entropy_mean);
-    PICK(corr_hit); PICK(risky_n); PICK(risky_index); PICK(risky_token);
+    PICK(corr_hit); PICK(risky_n); PICK(risky_index); PICK(risky_token); PICK(freed_page_ids);
 #undef PICK
   }
   ctx->mark(-1);
@@ -539,6 +600,7 @@ recg_status recg_verify(recg_ctx* ctx, const recg_batch* batch, const void* logi
       OUT(freed_pages, C); OUT(next_draft, Tb); OUT(cont_hit, C); OUT(top1, T); OUT(top2, T); OUT(p1, T); OUT(p2, T);
       OUT(entropy, T); OUT(entropy_mean, C);
       OUT(corr_hit, 2 * C); OUT(risky_n, 3 * C); OUT(risky_index, 6 * C); OUT(risky_token, 6 * C);
+      OUT(freed_page_ids, T);
 #undef OUT
       return RECG_OK;
     }
@@ -547,6 +609,7 @@ recg_status recg_verify(recg_ctx* ctx, const recg_batch* batch, const void* logi
     OUT(freed_pages, C); OUT(next_draft, Tb); OUT(cont_hit, C); OUT(top1, T); OUT(top2, T); OUT(p1, T); OUT(p2, T);
     OUT(entropy, T); OUT(entropy_mean, C);
     OUT(corr_hit, 2 * C); OUT(risky_n, 3 * C); OUT(risky_index, 6 * C); OUT(risky_token, 6 * C);
+    OUT(freed_page_ids, T);
 #undef OUT
     CU(cudaStreamSynchronize(ctx->stream));
   }
@@ -650,6 +713,29 @@ recg_status recg_linear(recg_ctx* ctx, const void* x, const void* w, void* y, in
   a.x = x; a.w = w; a.out = y; a.M = M; a.N = N; a.K = K;
   a.epi = out_dtype == RECG_DTYPE_BF16 ? EPI_PLAIN_BF16 : EPI_PLAIN_F32;
   return run_gemm(ctx, a);
+}
+
+recg_status recg_debug_gemm_config(recg_ctx* ctx, int32_t tile, int32_t stream_k) {
+  if (!ctx) return RECG_ERR_INVALID_ARG;
+  if (tile != 0 && tile != 64 && tile != 128 && tile != 256 && tile != 384 && tile != 512)
+    return fail(ctx, RECG_ERR_INVALID_ARG, "recg_debug_gemm_config: tile must be 0, 64, 128, 256, 384 or 512");
+  tc_state_force(ctx->tc_state, tile, stream_k != 0);
+  return RECG_OK;
+}
+
+recg_status recg_debug_wait_timeout(recg_ctx* ctx, int32_t max_polls) {
+  if (!ctx) return RECG_ERR_INVALID_ARG;
+  if (max_polls < 1 || max_polls > (1 << 20)) return fail(ctx, RECG_ERR_INVALID_ARG, "recg_debug_wait_timeout: max_polls must be 1 .. 1048576");
+  launch_wait_timeout((uint32_t)max_polls, ctx->d_status, ctx->stream);
+  CU(cudaGetLastError());
+  return RECG_OK;
+}
+
+int32_t recg_debug_map_cache_selftest(int32_t n_keys, int32_t* evictions) {
+  int ev = 0;
+  const int bad = tc_map_cache_selftest(n_keys, &ev);
+  if (evictions) *evictions = ev;
+  return bad;
 }
 
 recg_status recg_debug_buffer(recg_ctx* ctx, int32_t which, const void** ptr, int32_t* dtype, int32_t* rows, int32_t* cols) {

@@ -84,7 +84,8 @@ template <> struct Vec<float> {
   __device__ static float one(const float* p) { return *p; }
 };
 
-// grid (chunks_per_row, rows).  Each CTA scans [c0, c1) of one row.
+// One-dimensional grid of rows x chunks_per_row CTAs, chunk-fastest (consecutive CTAs read consecutive memory; the
+// row count is not bound by the 65535 limit of the other grid dimensions).  Each CTA scans [c0, c1) of one row.
 template <typename T>
 __global__ void __launch_bounds__(kVerifyThreads) verify_partial_kernel(const T* __restrict__ logits, int vocab,
                                                                         int chunk_len, int chunks_per_row,
@@ -92,7 +93,7 @@ __global__ void __launch_bounds__(kVerifyThreads) verify_partial_kernel(const T*
   constexpr int N = Vec<T>::N;
   griddep_launch();
   griddep_wait();
-  const int row = blockIdx.y, chunk = blockIdx.x;
+  const int row = blockIdx.x / chunks_per_row, chunk = blockIdx.x - row * chunks_per_row;
   const T* base = logits + (size_t)row * vocab;
   const int c0 = chunk * chunk_len;
   const int c1 = min(vocab, c0 + chunk_len);
@@ -237,7 +238,7 @@ __global__ void __launch_bounds__(128) verify_finalize_kernel(BatchLayout bl, co
     vb.entropy[t0 + j] = logf(ms.s) - ms.t * inv + ms.m;   // ln S - (1/S) sum x e^(x-M) + M
   }
   __syncthreads();
-  __shared__ int s_a;
+  __shared__ int s_a, s_first_free, s_last;
   if (threadIdx.x == 0) {
     int a = 0;
     const int tv0 = bl.cu_ver[r];
@@ -259,6 +260,8 @@ __global__ void __launch_bounds__(128) verify_finalize_kernel(BatchLayout bl, co
     const int first_free = (new_L + kPageSize - 1) / kPageSize;
     const int last = (L + n + kPageSize - 1) / kPageSize;
     vb.freed_pages[r] = bl.page_table ? last - first_free : 0;
+    s_first_free = first_free;
+    s_last = bl.page_table ? last : first_free;
     // a correction branch is confirmed when the verifier rejected exactly the draft it replaced and emitted the
     // replacement token there (Sec. 5.1)
     for (int k = 0; k < 2; ++k)
@@ -291,6 +294,12 @@ __global__ void __launch_bounds__(128) verify_finalize_kernel(BatchLayout bl, co
     const int slot = bl.tok_slot[t0 + j];
     const bool committed = (j < v) && (j <= a);
     vb.slot_state[t0 + j] = slot < 0 ? 0 : (committed ? slot : -(slot + 1));
+    // ids of the pages that hold no committed token any more, at the request's row offset (there are never more
+    // of them than rows: each starts at a position of a row that was rolled back)
+    if (vb.freed_page_ids) {
+      const int e = s_first_free + j;
+      vb.freed_page_ids[t0 + j] = e < s_last ? bl.page_table[(size_t)r * bl.pt_stride + e] : -1;
+    }
   }
 }
 
@@ -314,7 +323,7 @@ void launch_verify(const BatchLayout& bl, const void* logits, int logits_dtype, 
   int chunk_len = (vocab + chunks - 1) / chunks;
   chunk_len = (chunk_len + 63) / 64 * 64;  // keeps every chunk start 16-byte aligned relative to the row
   chunks = (vocab + chunk_len - 1) / chunk_len;
-  dim3 grid(chunks, rows);
+  dim3 grid((unsigned)chunks * (unsigned)rows);
   if (logits_dtype == 0)
     launch_pdl(verify_partial_kernel<__nv_bfloat16>, grid, dim3(kVerifyThreads), 0, st,
                static_cast<const __nv_bfloat16*>(logits), vocab, chunk_len, chunks, partials);
@@ -460,15 +469,17 @@ extern "C" recg_status recg_row_stats_static(const void* logits, int32_t logits_
     return fail(RECG_ERR_CAPACITY, "recg_row_stats_static: rows x vocab chunks exceed the static scratch (65536 partials)");
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   RowPartial* scratch = g_static_ptr[dev];
-  dim3 grid(chunks, rows);
+  dim3 grid((unsigned)chunks * (unsigned)rows);
   if (logits_dtype == RECG_DTYPE_BF16)
     verify_partial_kernel<__nv_bfloat16>
         <<<grid, kVerifyThreads, 0, st>>>(static_cast<const __nv_bfloat16*>(logits), vocab, chunk_len, chunks, scratch);
   else
     verify_partial_kernel<float><<<grid, kVerifyThreads, 0, st>>>(static_cast<const float*>(logits), vocab, chunk_len,
                                                                   chunks, scratch);
+  cudaError_t e = cudaGetLastError();   // nothing reads the scratch unless the scan was launched
+  if (e != cudaSuccess) return fail(RECG_ERR_CUDA, std::string("recg_row_stats_static: launch: ") + cudaGetErrorString(e));
   row_stats_finalize_kernel<<<(rows + 127) / 128, 128, 0, st>>>(scratch, rows, chunks, top1, top2, p1, p2, entropy);
-  cudaError_t e = cudaGetLastError();
+  e = cudaGetLastError();
   if (e != cudaSuccess) return fail(RECG_ERR_CUDA, std::string("recg_row_stats_static: launch: ") + cudaGetErrorString(e));
   return RECG_OK;
 }

@@ -33,21 +33,40 @@ def test_struct_sizes_match_header_layout(tmp_path):
     assert C.sizeof(binding.recg_config) == 15 * 4
     # int + 5 ptr + int + ptr + int64, then 4 ptr + float, with padding
     assert C.sizeof(binding.recg_batch) == 8 * 8 + 8 + 4 * 8 + 8
-    assert C.sizeof(binding.recg_verify_out) == 8 + 18 * 8
+    assert C.sizeof(binding.recg_verify_out) == 8 + 19 * 8
     # and against the header itself, as the C compiler lays the structs out
     import subprocess
     src = tmp_path / "sizes.c"
     src.write_text('#include <stdio.h>\n#include <stddef.h>\n#include "recg.h"\n'
                    'int main(void) { printf("%zu %zu %zu %zu %zu %zu %zu\\n", sizeof(recg_config), sizeof(recg_batch), '
                    'sizeof(recg_verify_out), offsetof(recg_batch, n_corr), offsetof(recg_batch, risk_delta), '
-                   'offsetof(recg_verify_out, corr_hit), offsetof(recg_verify_out, risky_token)); return 0; }\n')
+                   'offsetof(recg_verify_out, corr_hit), offsetof(recg_verify_out, freed_page_ids)); return 0; }\n')
     exe = tmp_path / "sizes"
     subprocess.run(["gcc", "-I", os.path.join(ROOT, "include"), str(src), "-o", str(exe)], check=True)
     got = [int(t) for t in subprocess.run([str(exe)], check=True, capture_output=True, text=True).stdout.split()]
     want = [C.sizeof(binding.recg_config), C.sizeof(binding.recg_batch), C.sizeof(binding.recg_verify_out),
             binding.recg_batch.n_corr.offset, binding.recg_batch.risk_delta.offset,
-            binding.recg_verify_out.corr_hit.offset, binding.recg_verify_out.risky_token.offset]
+            binding.recg_verify_out.corr_hit.offset, binding.recg_verify_out.freed_page_ids.offset]
     assert got == want
+
+
+def test_tensor_map_cache_hands_out_copies_across_evictions():
+    """More distinct keys than the cache holds, three lookups per simulated launch: a map taken before a later lookup
+    of the same launch emptied the cache must still be the right one (host logic only, fake encoder)."""
+    lib = binding.lib()
+    ev = C.c_int32(0)
+    assert lib.recg_debug_map_cache_selftest(3 * 5000, C.byref(ev)) == 0
+    assert ev.value >= 3          # 15000 keys through a 4096-entry cache
+    assert lib.recg_debug_map_cache_selftest(30, C.byref(ev)) == 0 and ev.value == 0
+
+
+def test_init_rejects_capacities_the_launches_cannot_serve():
+    lib = binding.lib()
+    h = C.c_void_p()
+    big = binding.recg_config(2, 256, 4, 2, 64, 1024, 2048, 1e4, 1e-5, -1, 16, 5000, 64, 8, 0)     # requests
+    assert lib.recg_init(C.byref(h), C.byref(big), None, None) == 3
+    big = binding.recg_config(2, 256, 4, 2, 64, 1024, 2048, 1e4, 1e-5, -1, 16, 4, (1 << 20) + 1, 8, 0)   # rows
+    assert lib.recg_init(C.byref(h), C.byref(big), None, None) == 3 and b"4096 requests" in lib.recg_last_error(None)
 
 
 def test_pool_bytes_formula():

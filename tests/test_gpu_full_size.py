@@ -1,7 +1,8 @@
 """Full-size parity: the 32-layer 8B-class backbone at concurrency 16, exactly the batch shape bench.py times.
 
-The oracle cannot run the whole batch in reasonable time, so one sampled request is followed through all 32 layers
-(its K/V context is generated on the CPU and written into the pool; weights are widened layer by layer on access),
+The oracle cannot run the whole batch in reasonable time, so three sampled requests are followed through all 32
+layers (their K/V contexts are generated on the CPU and written into the pool; weights are widened layer by layer on
+access),
 and properties that hold at any size cover the rest: integer outputs are the oracle's verification of the kernel's
 own logits for every request, and the attention operation is checked at full size on sampled requests.
 """
@@ -11,7 +12,7 @@ import torch
 
 from oracle import recg_oracle as orc
 from paper_2609_34388_b200 import binding, synth
-from tests._util import f64, oracle_cfg
+from tests._util import bf16_round, f64, flip_histogram, oracle_cfg, oracle_rounds_together
 
 pytestmark = pytest.mark.gpu
 
@@ -39,13 +40,22 @@ def test_full_model_c16_round():
     ctx = binding.Context(binding.make_config(shape, 16, 1024, desc.page_table.shape[1]), W)
     pool = binding.alloc_kv_pool(ctx, desc.n_pages, fill="normal")
     n = desc.verify_len + desc.block_size
-    r = int(np.argmin(n * desc.ctx_len))                   # the cheapest request for the oracle
-    L, v, b = int(desc.ctx_len[r]), int(desc.verify_len[r]), int(desc.block_size[r])
-    kv = []
-    for l in range(shape.n_layers):
-        K, V = synth.kv_values(L, shape.n_kv_heads, shape.head_dim, seed=5000 + l)
-        ctx.recg_kv_write(pool, desc.n_pages, l, desc.page_table[r], 0, K.cuda(), V.cuda())
-        kv.append((f64(K), f64(V)))
+    # three requests for the oracle: the cheapest ones that differ in block size (shortest context per block size)
+    cost = n * desc.ctx_len
+    sample = []
+    for i in np.argsort(cost):
+        if int(desc.block_size[i]) not in [int(desc.block_size[j]) for j in sample]:
+            sample.append(int(i))
+        if len(sample) == 3:
+            break
+    kvs = {}
+    for r in sample:
+        kv = []
+        for l in range(shape.n_layers):
+            K, V = synth.kv_values(int(desc.ctx_len[r]), shape.n_kv_heads, shape.head_dim, seed=5000 + 100 * r + l)
+            ctx.recg_kv_write(pool, desc.n_pages, l, desc.page_table[r], 0, K.cuda(), V.cuda())
+            kv.append((f64(K), f64(V)))
+        kvs[r] = kv
     ys = synth.token_ids(int(desc.verify_len.sum()), shape.vocab, seed=1)
     batch = binding.Batch(desc.ctx_len, desc.verify_len, desc.block_size, ys, desc.page_table, pool, desc.n_pages)
     lg = ctx.recg_step(batch)
@@ -74,26 +84,54 @@ def test_full_model_c16_round():
         assert [s for s in ss if s >= 0] == kc["commit_slots"]
         np.testing.assert_allclose(got["entropy"][rows], [s["entropy"] for s in own["stats"]], rtol=2e-4, atol=1e-5)
 
-    # ---- the sampled request through all 32 layers of the oracle ----
+    # ---- three sampled requests through all 32 layers of the oracle, twice: in pure float64, and with the activations
+    # rounded to bf16 where the kernels store them in bf16 (the oracle's act_round hook).  The second run has the
+    # kernels' rounding points, so what remains against it is accumulation order and the rare values that round the
+    # other way: hidden states and logits must agree with IT within 2e-2 of max|ref|, and a row's top-1 may differ from
+    # ITS top-1 only where its top-2 logit gap is below 1e-2.  The gap to the pure float64 run is what bf16 storage of
+    # six activations per layer costs at depth 32; it is printed, not asserted against the shallow bound.
     W64 = {"embed": W["embed"].float().cpu().numpy(), "final_norm": f64(W["final_norm"]), "lm_head": f64(W["lm_head"])}
     for k in ("attn_norm", "wqkv", "wo", "ffn_norm", "w_gate_up", "w_down"):
         W64[k] = LazyLayers(W[k])
-    y_r = ys[int(cuv[r]): int(cuv[r + 1])].tolist()
-    ref_logits, _, ref_h = orc.fused_round_cached(oracle_cfg(shape), W64, kv, L, y_r, b)
-    rows = slice(int(cu[r]), int(cu[r + 1]))
-    gh, gl = f64(hidden[rows]), f64(logits[rows])
-    eh = np.max(np.abs(gh - ref_h)) / np.max(np.abs(ref_h))
-    el = np.max(np.abs(gl - ref_logits)) / np.max(np.abs(ref_logits))
-    rh = np.sqrt(np.mean((gh - ref_h) ** 2) / np.mean(ref_h ** 2))
-    rl = np.sqrt(np.mean((gl - ref_logits) ** 2) / np.mean(ref_logits ** 2))
-    print(f"\nfull-size request {r} (L={L}, v={v}, b={b}): max-abs error / max|ref| hidden {eh:.3e} logits {el:.3e}; "
-          f"rms error / rms hidden {rh:.3e} logits {rl:.3e}")
-    # bf16 storage of the normalised input, q/k/v, attention output and SwiGLU output adds an independent relative
-    # error of about 8e-3 (max-norm, measured on one layer) per layer, which accumulates like a random walk in the
-    # fp32 residual stream: 8e-3 * sqrt(n_layers) = 4.5e-2 at depth 32; the 2e-2 bound is a shallow-model bound
-    tol = max(2e-2, 8e-3 * np.sqrt(shape.n_layers))
-    assert eh <= tol and el <= tol
-    assert rh <= tol and rl <= tol
+    reqs = []
+    for r in sample:
+        reqs.append({"kv": kvs[r], "L": int(desc.ctx_len[r]), "y": ys[int(cuv[r]): int(cuv[r + 1])].tolist(),
+                     "b": int(desc.block_size[r])})
+    ocfg = oracle_cfg(shape)
+    pure = oracle_rounds_together(ocfg, W64, reqs)
+    points = oracle_rounds_together(ocfg, W64, reqs, bf16_round)
+    flips, n_rows, n_flagged = [], 0, 0
+    for r, rq, (p_lg, p_h), (b_lg, b_h) in zip(sample, reqs, pure, points):
+        rows = slice(int(cu[r]), int(cu[r + 1]))
+        gh, gl = f64(hidden[rows]), f64(logits[rows])
+        e64h = np.max(np.abs(gh - p_h)) / np.max(np.abs(p_h))
+        e64l = np.max(np.abs(gl - p_lg)) / np.max(np.abs(p_lg))
+        ebh = np.max(np.abs(gh - b_h)) / np.max(np.abs(b_h))
+        ebl = np.max(np.abs(gl - b_lg)) / np.max(np.abs(b_lg))
+        print(f"\nfull-size request {r} (L={rq['L']}, v={len(rq['y'])}, b={rq['b']}): max-abs error / max|ref| against the "
+              f"oracle with bf16 storage points: hidden {ebh:.3e} logits {ebl:.3e}; against pure float64: hidden {e64h:.3e} "
+              f"logits {e64l:.3e}")
+        assert ebh <= 2e-2 and ebl <= 2e-2, (r, ebh, ebl)
+        assert e64h <= 6e-2 and e64l <= 6e-2, (r, e64h, e64l)       # sanity only: see the comment above
+        ref = orc.verify_round(b_lg, rq["y"], rq["b"])
+        gaps = np.array([s["logit_gap"] for s in ref["stats"]])
+        top1 = got["top1"][rows]
+        n_rows += len(gaps)
+        n_flagged += int((gaps < 1e-2).sum())
+        for j, s in enumerate(ref["stats"]):
+            if int(top1[j]) != s["top1"]:
+                flips.append(float(gaps[j]))
+                assert gaps[j] < 1e-2, f"request {r} row {j}: top-1 differs at oracle gap {gaps[j]:.3e}"
+        a = ref["accept_len"]
+        v = len(rq["y"])
+        if v and (gaps[: min(a + 1, v)] >= 1e-2).all():
+            assert int(got["accept_len"][r]) == a
+            assert got["emitted"][int(cuv[r]): int(cuv[r]) + a + 1].tolist() == ref["emitted"]
+            kc = orc.kv_commit(rq["L"], v, rq["b"], a, desc.page_table[r], 16)
+            assert int(got["new_ctx_len"][r]) == kc["new_ctx_len"]
+            assert [s for s in got["slot_state"][rows].tolist() if s >= 0] == kc["commit_slots"]
+    print(f"depth 32, {n_rows} rows of 3 requests: {n_flagged} rows with oracle gap < 1e-2; top-1 differs on {len(flips)} rows, "
+          f"by oracle gap: {flip_histogram(flips)}")
     ctx.recg_free()
 
 

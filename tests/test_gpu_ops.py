@@ -310,13 +310,14 @@ def test_linear_random_shapes():
 
 
 @pytest.mark.parametrize("force", ["512,0", "512,1", "384,0", "384,1", "256,1", "128,1", "64,1", "256,0"])
-def test_linear_forced_decompositions(force, monkeypatch):
+def test_linear_forced_decompositions(force):
     """Every tile width and decomposition of the projection kernel on shapes that make it cut tiles: CTA pairs
     (512 = 256-row tiles over clusters of two), stream-K with the reduction through the idle operand ring (last
     pieces) and through global memory (pieces followed by whole tiles), ragged M, M beyond one pair tile."""
-    monkeypatch.setenv("RECG_GEMM_FORCE", force)       # read when the context is created
     shape = synth.tiny_shape()
     ctx = ops_ctx(shape, 1, 8, 1)
+    tile, sk = (int(t) for t in force.split(","))
+    ctx.recg_debug_gemm_config(tile, bool(sk))
     for (M, N, K) in [(300, 512, 1024), (130, 4096, 4096), (470, 1024, 14336), (600, 6144, 1024), (257, 28672, 512)]:
         g = torch.Generator().manual_seed(M * 7 + N)
         x = torch.randn((M, K), generator=g).to(torch.bfloat16)
@@ -329,6 +330,112 @@ def test_linear_forced_decompositions(force, monkeypatch):
         y2 = ctx.recg_linear(x.cuda(), w.cuda(), torch.float32)
         ctx.recg_sync()
         assert torch.equal(y, y2), (force, M, N, K)        # parts are added in a fixed order
+    ctx.recg_free()
+
+
+LLAMA8B_PROJECTIONS = {"qkv": (6144, 4096), "o": (4096, 4096), "gate_up": (28672, 4096), "down": (4096, 14336),
+                       "lm_head": (128256, 4096)}
+
+
+@pytest.mark.parametrize("name", list(LLAMA8B_PROJECTIONS))
+def test_linear_at_the_row_counts_the_bench_times(name):
+    """The five 8B-class projection shapes at the row counts of the concurrency-128 step, the concurrency sweep and the
+    forward-time sweep (1331, 2000, 3792, 8192 rows: 6 to 64 row tiles, every decomposition the cost model picks
+    there) and with every forced tile configuration at 1331 and 3792 rows.  The product is too large for a full float64
+    reference, so 256 sampled output columns (the first and last 32 and 192 drawn at random) are compared with a
+    float64 matmul of the same bf16 values; the whole output starts as NaN, so an unwritten tile shows anywhere, two
+    guard rows behind the matrix must stay NaN, and a second run must give the same bits."""
+    N, K = LLAMA8B_PROJECTIONS[name]
+    shape = synth.tiny_shape()
+    ctx = ops_ctx(shape, 1, 8, 1)
+    g = torch.Generator(device="cuda").manual_seed(N + K)
+    w = (torch.randn((N, K), generator=g, device="cuda") * 0.05).to(torch.bfloat16)
+    rng = np.random.default_rng(N)
+    cols = np.unique(np.concatenate([np.arange(32), np.arange(N - 32, N), rng.integers(32, N - 32, 192)]))
+    w_ref = f64(w[torch.from_numpy(cols).cuda()])
+    for M in (1331, 2000, 3792, 8192):
+        x = torch.randn((M, K), generator=g, device="cuda").to(torch.bfloat16)
+        ref = f64(x) @ w_ref.T
+        scale = np.max(np.abs(ref))
+        configs = [(0, False)]
+        if M in (1331, 3792):
+            configs += [(t, sk) for t in (64, 128, 256, 384, 512) for sk in (False, True)]
+        for tile, sk in configs:
+            if name == "lm_head" and tile in (64, 128) and M > 1331:
+                continue            # (narrow tiles on the widest matrix: tens of thousands of tiles, nothing new)
+            ctx.recg_debug_gemm_config(tile, sk)
+            outs = []
+            for rep in range(2):
+                buf = torch.full((M + 2, N), float("nan"), dtype=torch.float32, device="cuda")
+                ctx._check(binding.lib().recg_linear(ctx.h, x.data_ptr(), w.data_ptr(), buf.data_ptr(), M, N, K,
+                                                     binding.DTYPE_F32))
+                ctx.recg_sync()
+                outs.append(buf)
+            buf = outs[0]
+            assert not torch.isnan(buf[:M]).any(), f"unwritten output: {(name, M, tile, sk)}"
+            assert torch.isnan(buf[M:]).all(), f"stored beyond the last row: {(name, M, tile, sk)}"
+            err = np.max(np.abs(f64(buf[:M][:, torch.from_numpy(cols).cuda()]) - ref)) / scale
+            assert err < 1e-4, (name, M, tile, sk, err)
+            assert torch.equal(outs[0][:M], outs[1][:M]), f"not deterministic: {(name, M, tile, sk)}"
+            del outs, buf
+    ctx.recg_free()
+
+
+def test_bounded_wait_that_runs_out_is_reported_and_the_context_stays_usable():
+    """A kernel whose wait can never be satisfied gives up after its poll limit, returns and leaves the timeout in the
+    status word: recg_sync reports RECG_ERR_TIMEOUT once, and the same context then computes a correct product
+    (stream-K decomposition, whose arrival counters are reset after an error)."""
+    shape = synth.tiny_shape()
+    ctx = ops_ctx(shape, 1, 8, 1)
+    ctx.recg_debug_wait_timeout(2000)
+    with pytest.raises(binding.RecgError) as e:
+        ctx.recg_sync()
+    assert e.value.status == 5 and "gave up" in str(e.value)
+    ctx.recg_sync()                                   # the status word was cleared
+    ctx.recg_debug_gemm_config(256, True)
+    g = torch.Generator().manual_seed(3)
+    x = torch.randn((300, 1024), generator=g).to(torch.bfloat16)
+    w = (torch.randn((512, 1024), generator=g) * 0.05).to(torch.bfloat16)
+    y = ctx.recg_linear(x.cuda(), w.cuda(), torch.float32)
+    ctx.recg_sync()
+    ref = x.double().numpy() @ w.double().numpy().T
+    assert np.max(np.abs(f64(y) - ref)) / np.max(np.abs(ref)) < 1e-4
+    ctx.recg_free()
+
+
+def test_debug_checks_guard_bands_and_page_ownership():
+    """RECG_FLAG_DEBUG_CHECKS: a normal call passes; a write just past the end of a workspace region (done here
+    through the address recg_debug_buffer hands out, inside the library's own allocation) is reported by the next
+    recg_sync as RECG_ERR_INTERNAL, once; a page that receives new rows of two requests is refused on the host."""
+    shape = synth.tiny_shape()
+    W = synth.model_weights(shape, seed=0, dtype=torch.bfloat16)
+    Wd = {k: ([t.cuda() for t in v] if isinstance(v, list) else v.cuda()) for k, v in W.items()}
+    max_tok = 32
+    ctx = binding.Context(binding.make_config(shape, 4, max_tok, 8, binding.FLAG_DEBUG_CHECKS), Wd)
+    pool = binding.alloc_kv_pool(ctx, 32)
+    pt = np.arange(16, dtype=np.int32).reshape(2, 8)
+    batch = binding.Batch([20, 5], [2, 1], [4, 4], [1, 2, 3], pt, pool, 32)
+    ctx.recg_step(batch)
+    ctx.recg_verify(batch)
+    ctx.recg_sync()
+    # the rotated queries are [max_tokens, n_q * d] bf16; the guard band follows the region (256-byte aligned)
+    import ctypes as C
+    p, dt, r, c = C.c_void_p(), C.c_int32(), C.c_int32(), C.c_int32()
+    ctx._check(binding.lib().recg_debug_buffer(ctx.h, 2, C.byref(p), C.byref(dt), C.byref(r), C.byref(c)))
+    region = max_tok * shape.n_q_heads * shape.head_dim * 2
+    band = binding.device_view(p.value + (region + 255) // 256 * 256, (64,), torch.float32)
+    saved = band.clone()
+    band[3] = 1.0
+    with pytest.raises(binding.RecgError) as e:
+        ctx.recg_sync()
+    assert e.value.status == 6 and "guard band" in str(e.value)
+    ctx.recg_sync()                                   # reported once; the bands were refilled
+    assert torch.equal(band, saved)
+    shared = pt.copy()
+    shared[1, 0] = pt[0, 1]                           # request 1's first new page is request 0's page of new rows
+    with pytest.raises(binding.RecgError) as e:
+        ctx.recg_step(binding.Batch([20, 5], [2, 1], [4, 4], [1, 2, 3], shared, pool, 32))
+    assert e.value.status == 1 and "named twice" in str(e.value)
     ctx.recg_free()
 
 

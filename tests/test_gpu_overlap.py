@@ -6,7 +6,7 @@ import torch
 
 from oracle import recg_oracle as orc
 from paper_2609_34388_b200 import binding, synth
-from tests._util import bf16_round, f64, oracle_cfg, oracle_weights
+from tests._util import bf16_round, f64, flip_histogram, oracle_cfg, oracle_weights
 
 pytestmark = pytest.mark.gpu
 
@@ -187,7 +187,7 @@ def tiny_model():
     return shape, W, oracle_cfg(shape), oracle_weights(W)
 
 
-def check_branch_round(shape, W, ocfg, W64, reqs, flags=0, max_tokens=160, adaptive_flag=False):
+def check_branch_round(shape, W, ocfg, W64, reqs, flags=0, max_tokens=160, bf16_points=False):
     """reqs: dicts with kv (per-layer bf16-rounded prefix K/V as float64), y, L, v, b, m (planted accept length or None),
     corr [(index, token)], bc.  Runs the round on the GPU and checks every row against the oracle; returns the
     per-request correction hits, the results and what is needed to run the batch again."""
@@ -210,7 +210,7 @@ def check_branch_round(shape, W, ocfg, W64, reqs, flags=0, max_tokens=160, adapt
     hidden = f64(ctx.recg_debug_buffer(0))
     assert logits.shape[0] == desc.n_tokens
     t0 = tb0 = 0
-    hits = []
+    hits, flips = [], []
     for i, r in enumerate(reqs):
         L, v, b, corr, bc = r["L"], r["v"], r["b"], r["corr"], r["bc"]
         n = int(desc.rows[i])
@@ -247,19 +247,27 @@ def check_branch_round(shape, W, ocfg, W64, reqs, flags=0, max_tokens=160, adapt
         assert int(got["new_ctx_len"][i]) == kc["new_ctx_len"] and int(got["freed_pages"][i]) == len(kc["freed_pages"])
         assert [s for s in ss if s >= 0] == kc["commit_slots"] and [-(s + 1) for s in ss if s < 0] == kc["rollback_slots"]
         # against the oracle's own forward, where its logit gaps are clear
-        ref = orc.verify_overlap_round(ref_logits, r["y"], b, corr, bc)
+        # (with bf16_points: the oracle with its activations rounded to bf16 where the kernels store them in bf16);
+        # a top-1 may differ only where that run's top-2 logit gap is below the flat flag
+        int_logits = ref_logits
+        if bf16_points:
+            int_logits, _, _ = orc.overlap_round_cached(ocfg, W64, r["kv"], L, r["y"], b, corr, bc, bf16_round)
+            assert np.max(np.abs(logits[t0:t0 + n] - int_logits)) <= HID_TOL * np.max(np.abs(int_logits))
+        ref = orc.verify_overlap_round(int_logits, r["y"], b, corr, bc)
         gaps = np.array([s["logit_gap"] for s in ref["stats"]])
-        row_err = np.max(np.abs(logits[t0:t0 + n] - ref_logits), axis=1)
-        clear = gaps >= (np.maximum(MARGIN_FLAG, 2.0 * row_err) if adaptive_flag else MARGIN_FLAG)
+        clear = gaps >= MARGIN_FLAG
         for j in range(n):
-            if clear[j]:
-                assert int(got["top1"][t0 + j]) == ref["stats"][j]["top1"], f"top1 row {j} request {i}"
+            if int(got["top1"][t0 + j]) != ref["stats"][j]["top1"]:
+                flips.append(float(gaps[j]))
+                assert not clear[j], f"top1 row {j} request {i}: oracle gap {gaps[j]:.3e}"
         if v and clear[: min(ref["accept_len"] + 1, v)].all():
             assert own["accept_len"] == ref["accept_len"] and own["corr_hit"] == ref["corr_hit"]
             if r["m"] is not None:
                 assert ref["accept_len"] == r["m"]
         t0 += n
         tb0 += n - v
+    print(f"\nround with branches, {desc.n_tokens} rows: top-1 differs from the oracle's on {len(flips)} rows, by oracle gap: "
+          + flip_histogram(flips))
     return hits, got, ctx, desc, pool, ys
 
 
@@ -317,7 +325,7 @@ def test_llama8b_shape_one_layer_round_with_branches():
         K, V = synth.kv_values(L, shape.n_kv_heads, shape.head_dim, seed=300 + i)
         y = synth.token_ids(v, shape.vocab, seed=400 + i).tolist()
         reqs.append({"kv": [(f64(K), f64(V))], "y": y, "L": L, "v": v, "b": b, "m": None, "corr": corr, "bc": bc})
-    hits, got, ctx, desc, pool, ys = check_branch_round(shape, W, ocfg, W64, reqs, max_tokens=256, adaptive_flag=True)
+    hits, got, ctx, desc, pool, ys = check_branch_round(shape, W, ocfg, W64, reqs, max_tokens=256, bf16_points=True)
     assert desc.n_tokens == 233
     ctx.recg_sync()
     ctx.recg_free()

@@ -8,7 +8,7 @@ import torch
 
 from oracle import recg_oracle as orc
 from paper_2609_34388_b200 import synth
-from tests._util import oracle_cfg, oracle_weights
+from tests._util import bf16_round, oracle_cfg, oracle_rounds_together, oracle_weights
 
 
 def small_shape(n_layers=2):
@@ -122,6 +122,50 @@ def test_cached_equals_dense(small):
     assert np.max(np.abs(cached_logits - dense_logits)) < 1e-10
     for (K, V), (Kd, Vd) in zip(cached_kv, dense_kv):
         assert np.max(np.abs(K - Kd)) < 1e-11 and np.max(np.abs(V - Vd)) < 1e-11
+
+
+def test_rounds_run_together_equal_rounds_run_alone(small):
+    """The test helper that sends several requests through orc.decoder_rows at once (block-diagonal visibility over the
+    concatenated contexts) gives each request what its own fused_round_cached call gives, also with the rounding hook."""
+    shape, cfg, W64, _ = small
+    reqs = []
+    for i, (L, v, b) in enumerate([(19, 3, 4), (0, 2, 2), (33, 1, 8), (7, 5, 0), (16, 0, 3)]):
+        ids = synth.token_ids(L + max(v, 1), shape.vocab, seed=30 + i).tolist()
+        kv = orc.prefill(cfg, W64, ids[: L + 1])[0] if L else [(np.zeros((0, 2, 8)), np.zeros((0, 2, 8)))] * cfg.n_layers
+        reqs.append({"kv": kv, "L": L, "y": ids[L: L + v], "b": b})
+    for hook, tol in ((None, 1e-10), (bf16_round, 0.0)):
+        together = oracle_rounds_together(cfg, W64, reqs, hook)
+        for r, (lg, hd) in zip(reqs, together):
+            alone_lg, _, alone_hd = orc.fused_round_cached(cfg, W64, r["kv"], r["L"], r["y"], r["b"], hook)
+            if hook is None:
+                assert np.max(np.abs(lg - alone_lg)) < tol and np.max(np.abs(hd - alone_hd)) < tol
+            else:
+                # with rounding, a last-bit difference of the fp64 sums can flip a bf16 rounding: compare loosely
+                assert np.max(np.abs(lg - alone_lg)) < 2e-2 * np.max(np.abs(alone_lg))
+
+
+def test_rounding_hook_is_applied_at_the_six_storage_points(small):
+    """decoder_rows' act_round hook: the identity leaves the result unchanged; a hook that counts its calls is applied
+    to the normalised input (twice per layer), q, k, v, the attention output and the SwiGLU output of every layer and
+    to the final normalised input; rounding to bf16 moves the logits by about a bf16 ulp, not more."""
+    shape, cfg, W64, _ = small
+    L, v, b = 12, 3, 4
+    ids = synth.token_ids(L + v, shape.vocab, seed=8).tolist()
+    kv, _, _ = orc.prefill(cfg, W64, ids[: L + 1])
+    base, _, _ = orc.fused_round_cached(cfg, W64, kv, L, ids[L:], b)
+    same, _, _ = orc.fused_round_cached(cfg, W64, kv, L, ids[L:], b, lambda a: a)
+    assert np.array_equal(base, same)
+    shapes = []
+    def counting(a):
+        shapes.append(a.shape)
+        return a
+    orc.fused_round_cached(cfg, W64, kv, L, ids[L:], b, counting)
+    n = v + b
+    per_layer = [(n, shape.hidden), (n, 4, 8), (n, 2, 8), (n, 2, 8), (n, 4, 8), (n, shape.hidden), (n, shape.ffn)]
+    assert shapes == per_layer * cfg.n_layers + [(n, shape.hidden)]
+    rounded, _, _ = orc.fused_round_cached(cfg, W64, kv, L, ids[L:], b, bf16_round)
+    rel = np.max(np.abs(rounded - base)) / np.max(np.abs(base))
+    assert 0 < rel < 3e-2
 
 
 def test_verify_rows_ignore_draft_block(small):

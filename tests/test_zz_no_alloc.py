@@ -1,4 +1,4 @@
-"""The allocation-free row-statistics entry point against the context-based verify, two calls in a row.
+"""The allocation-free row-statistics entry point against the context-based verify and the oracle, two calls in a row.
 
 Collected last on purpose: if it fails, a run that stops at the first failure has already run everything
 else.  It must pass alone in a fresh process and after the other tests.
@@ -9,6 +9,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import recg_oracle as orc
 from paper_2609_34388_b200 import binding, synth
 
 pytestmark = pytest.mark.gpu
@@ -39,6 +40,14 @@ def test_static_scratch_matches_context_verify_twice(dtype):
         np.testing.assert_allclose(got["p1"].cpu().numpy(), ref["p1"], rtol=2e-4, atol=1e-7)
         np.testing.assert_allclose(got["p2"].cpu().numpy(), ref["p2"], rtol=2e-4, atol=1e-7)
         np.testing.assert_allclose(got["entropy"].cpu().numpy(), ref["entropy"], rtol=2e-4, atol=1e-5)
+        # and against the oracle's definition of the per-row statistics on the same values (ids exact)
+        host = lg.double().cpu().numpy()
+        for r in range(host.shape[0]):
+            want = orc.row_stats(host[r])
+            assert int(got["top1"][r]) == want["top1"] and int(got["top2"][r]) == want["top2"]
+            assert abs(float(got["p1"][r]) - want["p1"]) <= 2e-4 * want["p1"] + 1e-7
+            assert abs(float(got["p2"][r]) - want["p2"]) <= 2e-4 * want["p2"] + 1e-7
+            assert abs(float(got["entropy"][r]) - want["entropy"]) <= 2e-4 * want["entropy"] + 1e-5
 
 
 def test_static_scratch_rejects_oversize_and_bad_arguments():
@@ -46,6 +55,7 @@ def test_static_scratch_rejects_oversize_and_bad_arguments():
     lg = torch.zeros((4, 2048), dtype=torch.float32, device="cuda")
     args = [None] * 5 + [None]
     assert lib.recg_row_stats_static(lg.data_ptr(), 1, 70000, 2048, *args) == 3          # beyond the static scratch
+    assert lib.recg_row_stats_static(lg.data_ptr(), 1, 65537, 2048, *args) == 3
     assert b"65536" in lib.recg_row_stats_static_error()
     assert lib.recg_row_stats_static(None, 1, 4, 2048, *args) == 1
     assert lib.recg_row_stats_static(lg.data_ptr(), 7, 4, 2048, *args) == 1
