@@ -21,6 +21,9 @@ What follows the paper, and where:
   branches with the second candidate, their reuse rule, and
   the recursive loop over verifier + up to three branches       -- Sec. 5.1
 * the certainty state and the table-lookup block-size rule      -- Sec. 5.2, Eq. 2-3
+* the transition probabilities of acceptance intervals between
+  adjacent rounds, as a Markov chain that supplies synthetic
+  acceptance lengths                                            -- Sec. 4.2, Table 1
 
 The backbone itself (RMSNorm, rotary embedding with rotate-half pairing,
 grouped-query attention, SwiGLU, untied LM head) is the generic Llama-style
@@ -36,7 +39,11 @@ branch row against the standalone round it hypothesises, visibility by brute
 force, planted selection / reuse cases and losslessness of the recursive loop
 (tests/test_oracle_overlap.py); for the block-size rule, pairwise comparisons
 on a closed-form acceptance model, the limits of the cost weight, ties and
-bin edges (tests/test_oracle_policy.py).  No value printed in the
+bin edges (tests/test_oracle_policy.py); for the acceptance chain, the printed
+table itself (tests/golden/table1_transitions.txt), its stationary distribution
+solved two ways and the transition counts of a long run
+(tests/test_oracle_chain.py); for the bookkeeping between rounds, the trace of
+the pinned round loop.  No value printed in the
 paper exists for this path, so numeric parity with the paper itself is
 unpinned; parity is with these definitions.
 """
@@ -661,4 +668,85 @@ def policy_step(state: Dict[str, list], entropy_mean, accept_len, verify_len, bl
         j, B = policy_select(s, state["block_index"][r], state["full"][r], blocks, s_edges, value, cost, dtype)
         state["block_index"][r] = j
         out.append(B)
+    return out
+
+
+# --------------------------------------------------------------------------
+# synthetic acceptance lengths: the interval chain of Table 1 (Sec. 4.2)
+# --------------------------------------------------------------------------
+# With block size 32 the paper sorts a round's acceptance length A (emitted
+# tokens of the round, a + 1 here) into three intervals and prints the
+# probability of the next round's interval given this round's.  Random-init
+# weights accept almost nothing, so multi-round runs take their acceptance
+# lengths from this chain instead.  The paper prints nothing about the
+# distribution INSIDE an interval; it is taken uniform over the interval's
+# integers.  All random numbers are inputs (uniforms in [0, 1)).
+TABLE1_INTERVALS = ((1, 8), (9, 16), (17, 32))
+TABLE1_PERCENT = ((70.30, 18.11, 11.60),
+                  (58.39, 22.42, 19.19),
+                  (20.83, 12.51, 66.66))
+
+
+def chain_matrix(percent=TABLE1_PERCENT) -> np.ndarray:
+    """Row-stochastic transition matrix from the printed percentages (the rows
+    add up to 100 only to the printed precision; each row is divided by its sum)."""
+    P = np.asarray(percent, dtype=F64)
+    return P / P.sum(axis=1, keepdims=True)
+
+
+def chain_stationary(P: np.ndarray) -> np.ndarray:
+    """The distribution pi with pi P = pi and sum(pi) = 1, by solving the linear system."""
+    n = P.shape[0]
+    A = np.vstack([P.T - np.eye(n), np.ones((1, n))])
+    rhs = np.concatenate([np.zeros(n), [1.0]])
+    pi, *_ = np.linalg.lstsq(A, rhs, rcond=None)
+    return pi
+
+
+def acceptance_chain(P: np.ndarray, intervals, state0: int, u_state: Sequence[float], u_len: Sequence[float]):
+    """Walk the chain: round t is in state s_t (s_0 = state0); its acceptance
+    length is lo + floor(u_len[t] * (hi - lo + 1)) within the state's interval;
+    the next state is the first j whose cumulative probability in row s_t
+    exceeds u_state[t].  Returns (states, lengths)."""
+    states, lengths = [], []
+    s = int(state0)
+    for t in range(len(u_len)):
+        lo, hi = intervals[s]
+        states.append(s)
+        lengths.append(min(hi, lo + int(np.floor(F64(u_len[t]) * (hi - lo + 1)))))
+        c = np.cumsum(P[s])
+        j = int(np.sum(c <= F64(u_state[t])))
+        s = min(j, len(intervals) - 1)
+    return states, lengths
+
+
+def advance_round(L: int, y: Sequence[int], b: int, accept_len: int, verifier_token: int, cont_hit: bool,
+                  next_draft: Sequence[int]):
+    """Bookkeeping between two rounds of the fused loop (Sec. 3.1, 5.1): K/V of
+    y_0..y_a are committed, the verifier's token at row a is emitted last and
+    becomes the next y_0; a reused continuation block supplies the next drafts
+    (its first token only confirmed the bonus token), otherwise the next round
+    verifies the single emitted token.  Returns (new L, next y)."""
+    new_L = L + accept_len + 1
+    if cont_hit:
+        return new_L, [int(verifier_token)] + [int(t) for t in next_draft[1:]]
+    return new_L, [int(verifier_token)]
+
+
+def planted_rounds(L0: int, v0: int, blocks: Sequence[int], lengths: Sequence[int]):
+    """Lengths-only trace of the loop under synthetic acceptance (token values
+    play no role): round t has context L_t, v_t verify tokens and block
+    blocks[t]; it accepts a_t = min(lengths[t], v_t) - 1 drafts, i.e. emits
+    min(lengths[t], v_t) tokens; the continuation block is taken as reused
+    exactly when the round accepted all its drafts and drafted a block.
+    Returns per round (L, v, b, a, emitted, reused)."""
+    L, v = int(L0), int(v0)
+    out = []
+    for t, b in enumerate(blocks):
+        emitted = max(1, min(int(lengths[t]), v)) if v > 0 else 0
+        a = emitted - 1 if v > 0 else 0
+        reused = v > 0 and b > 0 and a == v - 1
+        out.append((L, v, int(b), a, emitted, reused))
+        L = L + (a + 1 if v > 0 else 0)
+        v = int(b) if reused else 1
     return out
