@@ -147,7 +147,7 @@ def run_ours(args, env):
     descs = [c16_descriptor(3 + i + 100 * env.rank) for i in range(4)]           # rotate over 4 batch draws
     max_pages = max(d.page_table.shape[1] for d in descs)
     n_pages = max(d.n_pages for d in descs)
-    cfg = binding.make_config(shape, 16, 1024, max_pages)
+    cfg = binding.make_config(shape, 16, 1024, max_pages, args.flags)
     ctx = binding.Context(cfg, W)
     pool = binding.alloc_kv_pool(ctx, n_pages, fill="normal")
     batches = []
@@ -263,6 +263,12 @@ def run_ours(args, env):
                                          f"{gemm_ms / max(n_gemm_launch, 1) * 1e3:.1f} us; peak = sustained bf16 of {peaks['source']}; "
                                          "traffic = DRAM bytes of one gate|up launch at M = 480 under ncu (algorithmic 266.4e6)")
         out["step_time_share"] = {k: round(v / sum(ms.values()), 4) for k, v in ms.items()}
+    if args.quick:
+        if env.rank == 0:
+            out["c1"] = bench_c1(binding, ctx, shape, pool, n_pages, peaks, args)
+        ctx.recg_free()
+        return out
+    if env.rank == 0:
         # the short-step and single-operation points are compared with peaks that were measured on an idle device, so the
         # device is left idle for a moment after the long step loops
         torch.cuda.synchronize()
@@ -396,6 +402,35 @@ def bench_attention_op(binding, peaks, args, desc=None, n_layers=32, label=None)
             "us_per_call": round(us, 2), "calls_include": "attention kernel + combine kernel", "algorithmic_bytes": int(kv_bytes),
             "gbs": round(gbs, 1), "frac_of_hbm_measured": round(gbs / peaks["hbm_gbs"], 4),
             "frac_of_8000": round(gbs / 8000.0, 4)}
+
+
+def bench_small_step(binding, peaks, args, n_layers=2, n_req=16):
+    """A small case of the whole step for profiler captures: n_layers 8B-shaped layers + LM head, n_req requests with
+    configs[2]'s block sizes and contexts U[64, 1024] (about 1.5 GB of weights and a pool of a few hundred MB, so a
+    capture that saves and restores device memory stays short).  Timed too, but it is not a benchmark figure."""
+    shape = synth.llama8b_shape(n_layers)
+    W = synth.model_weights(shape, seed=0, device="cuda", dtype=torch.bfloat16)
+    desc = synth.batch_descriptor(n_req, [4, 8, 16, 32], None, 64, 1024, seed=3)
+    ctx = binding.Context(binding.make_config(shape, n_req, desc.n_tokens, desc.page_table.shape[1], args.flags), W)
+    pool = binding.alloc_kv_pool(ctx, desc.n_pages, fill="normal")
+    ys = synth.token_ids(int(desc.verify_len.sum()), shape.vocab, seed=1)
+    batch = binding.Batch(desc.ctx_len, desc.verify_len, desc.block_size, ys, desc.page_table, pool, desc.n_pages)
+    vout = binding.VerifyOut(batch.n_req, batch.n_tok, batch.n_ver, host=False)
+    for _ in range(3):
+        ctx.recg_step(batch)
+        ctx.recg_verify(batch, out=vout)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(5):
+        ctx.recg_step(batch)
+        ctx.recg_verify(batch, out=vout)
+    e1.record()
+    torch.cuda.synchronize()
+    ctx.recg_sync()
+    ctx.recg_free()
+    return {"workload": f"{n_layers} 8B-shaped layers + LM head, {n_req} requests, {batch.n_tok} rows, contexts U[64,1024]",
+            "ms_per_step": round(e0.elapsed_time(e1) / 5, 3)}
 
 
 def bench_gemm_shapes(binding, peaks):
@@ -788,7 +823,9 @@ def main():
     ap.add_argument("--steps", type=int, default=8)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--only", default="", help="comma list of op-level sections to run alone (attention_op, attention_c16, attention_c16_branches, verify_sweep, gemm_shapes): "
+    ap.add_argument("--flags", type=int, default=0, help="recg_config.flags of the timed context (A/B checks)")
+    ap.add_argument("--quick", action="store_true", help="the timed step, its per-class times and the concurrency-1 point only")
+    ap.add_argument("--only", default="", help="comma list of op-level sections to run alone (attention_op, attention_c16, attention_c16_branches, small_step, verify_sweep, gemm_shapes): "
                                                "small cases for profiling; prints their JSON and exits")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
@@ -815,6 +852,8 @@ def main():
                                               desc=synth.with_correction_branches(c16_descriptor(3), 128256, 2, seed=60),
                                               label="attention of configs[2] draw 0 with two correction branches per request "
                                                     "(784 rows instead of 376), 4 layer caches rotated, CUDA-graph replay")
+            elif sec == "small_step":
+                res[sec] = bench_small_step(binding, peaks, args)
             elif sec == "verify_sweep":
                 res[sec] = bench_verify(binding, peaks)
             elif sec == "gemm_shapes":

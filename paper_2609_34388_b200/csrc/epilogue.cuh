@@ -18,6 +18,15 @@ struct EpiParams {
   int64_t n_pages;
   int layer, n_q, n_kv, head_dim;
   int* status;
+  // RMSNorm folded into the projections.  A projection whose input is a normalised residual stream reads
+  // x = bf16(h * g) (not yet divided by the row's root mean square) and multiplies its accumulator rows by
+  // rstd = rsqrt(sum_k ss_in[k][row] / norm_n + eps); EPI_RESIDUAL_NORM writes that x and the partial sums of squares
+  // of the rows it updates, one slot per column tile, for the projection that follows.
+  const float* ss_in;      // [ss_slots][ss_stride] partial sums of h^2 per row, or null: no scaling
+  int ss_slots, ss_stride;
+  float norm_inv_n, norm_eps;
+  const __nv_bfloat16* gain;   // EPI_RESIDUAL_NORM: gain of the NEXT norm, [N]
+  float* ss_out;               // EPI_RESIDUAL_NORM: [n column tiles][ss_stride]
 };
 
 __device__ __forceinline__ float silu_f(float z) { return z / (1.f + __expf(-z)); }

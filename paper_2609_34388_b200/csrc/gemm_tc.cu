@@ -32,13 +32,19 @@ constexpr int BM = 128, BK = 64;
 constexpr int kTcThreads = 192;
 constexpr int kSmemBudget = 192 * 1024;     // operand ring (every configuration's stage size divides it)
 constexpr int kStageOutBytes = 4 * 4096;      // per epilogue warp: two 2 KB boxes of output on their way to the TMA unit
+// EPI_RESIDUAL_NORM kernels also stage the OLD residual rows (two 4 KB chunks per epilogue warp, fetched by the TMA unit
+// ahead of their use) and the gains of the tile's columns (512 bytes per warp); their operand ring is that much shorter
+constexpr int kNormHBytes = 4 * 2 * 4096;
+constexpr int kNormGBytes = 4 * 512;
+constexpr int kNormBytes = kNormHBytes + kNormGBytes + 6 * 1024;   // (rounded so that the ring budget stays a multiple of 8 KB)
 constexpr uint32_t kSpin = 1u << 22;
 
-template <int BN, bool PAIR = false> struct TcCfg {
+template <int BN, bool PAIR = false, bool NORM = false> struct TcCfg {
+  static constexpr int kBudget = NORM ? kSmemBudget - kNormBytes : kSmemBudget;
   static constexpr int kABytes = BM * BK * 2;
   static constexpr int kBBytes = (PAIR ? BN / 2 : BN) * BK * 2;     // per CTA: a pair splits the weight tile
   static constexpr int kStageBytes = kABytes + kBBytes;
-  static constexpr int kStages = (kSmemBudget / kStageBytes) > 8 ? 8 : (kSmemBudget / kStageBytes);
+  static constexpr int kStages = (kBudget / kStageBytes) > 8 ? 8 : (kBudget / kStageBytes);
   static constexpr int kMaxStages = 16;
   // thin problems (M <= 32) load only 32 rows of x per stage: the stage shrinks and more stages fit.  The MMA
   // still reads 128 rows; rows 32.. alias the bytes that follow (harmless: those accumulator rows are never
@@ -46,10 +52,12 @@ template <int BN, bool PAIR = false> struct TcCfg {
   static constexpr int kThinABytes = 32 * BK * 2;
   static constexpr int kThinStageBytes = kThinABytes + kBBytes;
   static constexpr int kThinStages =
-      (kSmemBudget / kThinStageBytes) > kMaxStages ? kMaxStages : (kSmemBudget / kThinStageBytes);
-  static constexpr int kRingBytes = kSmemBudget + kABytes;     // either ring plus the pad
-  static constexpr int kBarBytes = (2 * kMaxStages + 5) * 8 + 16;
-  static constexpr int kSmemBytes = kRingBytes + kStageOutBytes + kBarBytes + 1024;  // + slack for 1024-byte alignment
+      (kBudget / kThinStageBytes) > kMaxStages ? kMaxStages : (kBudget / kThinStageBytes);
+  static constexpr int kRingBytes = kBudget + kABytes;     // either ring plus the pad
+  static constexpr int kBarBytes = (2 * kMaxStages + 5 + 8) * 8 + 16;
+  static constexpr int kNormOff = kRingBytes + kStageOutBytes;             // old residual rows, then gains (NORM only)
+  static constexpr int kBarOff = kNormOff + (NORM ? kNormHBytes + kNormGBytes : 0);
+  static constexpr int kSmemBytes = kBarOff + kBarBytes + 1024;  // + slack for 1024-byte alignment
   static constexpr int kTmemCols = 2 * BN < 32 ? 32 : 2 * BN;                  // power of two: 128, 256, 512
 };
 
@@ -386,17 +394,100 @@ __device__ __forceinline__ Piece make_piece(int& jd, int dp_tiles, long long& po
   return p;
 }
 
+// EPI_RESIDUAL_NORM: besides the accumulator a thread needs its row of the OLD residual stream and the gains of the
+// next norm.  Both come through shared memory: the TMA unit fetches the old rows of a 32-column chunk as two boxes (the
+// boxes of the output map: 32 rows x 16 columns, 64-byte swizzle) two chunks ahead of their use, completing on one
+// mbarrier per slot, and the tile's gains are staged once per tile.  (Plain global loads in flight would be waited for
+// by the proxy fence of every output box.)
+struct NormStage {
+  uint8_t* h;        // this warp's two 4 KB slots
+  uint4* g;          // this warp's 32 x 16 bytes of gains
+  uint64_t* bar;     // this warp's two barriers
+  uint32_t count;    // chunks fetched so far by this warp (slot = count & 1, phase = (count >> 1) & 1)
+};
+__device__ __forceinline__ void norm_issue(NormStage& ns, const CUtensorMap* omap, uint32_t idx, int n, int m_base, int lane) {
+  if (lane == 0) {
+    uint64_t* bar = &ns.bar[idx & 1];
+    uint8_t* dst = ns.h + (idx & 1) * 4096;
+    mbar_arrive_expect_tx(bar, 4096);
+    tma_load_2d(dst, omap, n, m_base, bar);
+    tma_load_2d(dst + 2048, omap, n + 16, m_base, bar);
+  }
+}
+// gains of the tile's columns and the first two chunks of old rows; returns the chunks the tile has
+__device__ __forceinline__ int norm_prepare(const EpiParams& ep, NormStage& ns, const CUtensorMap* omap, int n0, int bn, int m_base,
+                                            int lane) {
+  const int left = ep.N - n0;
+  const int nch = left <= 0 ? 0 : ((left < bn ? left : bn) + 31) / 32;
+  if (lane * 8 < bn && n0 + lane * 8 < ep.N) ns.g[lane] = __ldg(reinterpret_cast<const uint4*>(ep.gain + n0) + lane);
+  __syncwarp();
+  for (int c = 0; c < 2 && c < nch; ++c) norm_issue(ns, omap, ns.count + c, n0 + c * 32, m_base, lane);
+  return nch;
+}
+
 // Epilogue of one accumulator tile for the calling thread's row.
 // stg: this warp's 4 KB of output staging (two boxes).  All 32 lanes of the warp call together.
-template <int BN, typename Loader>
+// rstd: factor of this thread's row when the input of the projection was a residual stream that is normalised on the
+// fly (1 otherwise); xmap: the tensor map over x_out of EPI_RESIDUAL_NORM; tile_col: index of the tile's column.
+template <int BN, bool NORM, typename Loader>
 __device__ __forceinline__ void row_epilogue(const EpiParams& ep, const Loader& load, int m, int n0, float* stg,
-                                             const CUtensorMap* omap) {
+                                             const CUtensorMap* omap, const CUtensorMap* xmap, float rstd, int tile_col,
+                                             NormStage& ns, bool prepared) {
   const bool row_ok = m < ep.M;
   const int lane = threadIdx.x & 31;
   const int m_base = m - lane;                                  // first row of this warp
   const int valid_rows = ep.M - m_base < 0 ? 0 : (ep.M - m_base > 32 ? 32 : ep.M - m_base);
   OutStage os{reinterpret_cast<uint8_t*>(stg), 0u};
   const bool active = valid_rows > 0;      // a box that starts beyond the last row is not issued at all
+  if constexpr (NORM) {
+    // The residual stream itself is updated by the TMA unit's add-reduction (one addend per element and launch: the
+    // rounding of a load-add-store).  The new value is formed here as well, from the old rows staged in shared memory,
+    // for the next norm's input x = bf16(h * gain) and the row's sum of squares over this tile's columns.
+    const int nch = prepared ? (ep.N - n0 <= 0 ? 0 : ((ep.N - n0 < BN ? ep.N - n0 : BN) + 31) / 32)
+                             : norm_prepare(ep, ns, omap, n0, BN, m_base, lane);
+    const int sw = (lane >> 1) & 3;
+    float ss = 0.f;
+#pragma unroll 1
+    for (int c = 0; c < nch; ++c) {
+      const uint32_t idx = ns.count + c;
+      if (!mbar_wait(&ns.bar[idx & 1], (idx >> 1) & 1, kSpin)) set_status(ep.status, DEV_TIMEOUT_FULL);
+      float hv[32];
+      const uint8_t* slot = ns.h + (idx & 1) * 4096 + lane * 64;
+#pragma unroll
+      for (int b = 0; b < 2; ++b)
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const float4 t = *reinterpret_cast<const float4*>(slot + b * 2048 + ((q ^ sw) << 4));
+          hv[16 * b + 4 * q] = t.x; hv[16 * b + 4 * q + 1] = t.y; hv[16 * b + 4 * q + 2] = t.z; hv[16 * b + 4 * q + 3] = t.w;
+        }
+      __syncwarp();                 // every lane has read the slot: it may be refilled
+      if (c + 2 < nch) norm_issue(ns, omap, idx + 2, n0 + (c + 2) * 32, m_base, lane);
+      float v[32];
+      load(c * 32, v);
+      const int n = n0 + c * 32;
+      tma_store_rows_f32(omap, os, v, n, m_base, true, active, lane);
+#pragma unroll
+      for (int i = 0; i < 32; ++i) {
+        v[i] += hv[i];
+        ss = fmaf(v[i], v[i], ss);
+      }
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const uint4 gq = ns.g[c * 4 + q];
+        const uint32_t w[4] = {gq.x, gq.y, gq.z, gq.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          v[8 * q + 2 * j] *= __uint_as_float(w[j] << 16);
+          v[8 * q + 2 * j + 1] *= __uint_as_float(w[j] & 0xffff0000u);
+        }
+      }
+      tma_store_rows_bf16(xmap, os, v, n, m_base, active, lane);
+    }
+    ns.count += nch;
+    if (row_ok) ep.ss_out[(size_t)tile_col * ep.ss_stride + m] = ss;
+    tma_store_drain_reads(lane);
+    return;
+  }
   if (ep.epi == EPI_SWIGLU) {
     // accumulator columns [0, BN/2) are gate, [BN/2, BN) up; n0 is the first output column
 #pragma unroll 1
@@ -406,7 +497,7 @@ __device__ __forceinline__ void row_epilogue(const EpiParams& ep, const Loader& 
       load(BN / 2 + c * 32, u);
       if (n0 + c * 32 < ep.N) {
 #pragma unroll
-        for (int i = 0; i < 32; ++i) g[i] = silu_f(g[i]) * u[i];
+        for (int i = 0; i < 32; ++i) g[i] = silu_f(g[i] * rstd) * (u[i] * rstd);
         tma_store_rows_bf16(omap, os, g, n0 + c * 32, m_base, active, lane);
       }
     }
@@ -436,6 +527,11 @@ __device__ __forceinline__ void row_epilogue(const EpiParams& ep, const Loader& 
         float lo[32], hi[32];
         load(hl * D + c * 32, lo);
         load(hl * D + half + c * 32, hi);
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          lo[i] *= rstd;
+          hi[i] *= rstd;
+        }
         if (row_ok && !is_v) {
           const float2* cs = ep.rope_cs + (size_t)(c * 32) * ep.M + m;   // [frequency][token]
 #pragma unroll
@@ -473,6 +569,10 @@ __device__ __forceinline__ void row_epilogue(const EpiParams& ep, const Loader& 
     load(c * 32, v);
     const int n = n0 + c * 32;
     if (n >= ep.N) continue;
+    if (ep.ss_in) {
+#pragma unroll
+      for (int i = 0; i < 32; ++i) v[i] *= rstd;
+    }
     // the box is clipped at the right edge (N is a multiple of 16 but not always of 32) and at the last row
     if (ep.epi == EPI_PLAIN_BF16) tma_store_rows_bf16(omap, os, v, n, m_base, active, lane);
     else tma_store_rows_f32(omap, os, v, n, m_base, ep.epi == EPI_RESIDUAL, active, lane);
@@ -480,13 +580,13 @@ __device__ __forceinline__ void row_epilogue(const EpiParams& ep, const Loader& 
   tma_store_drain_reads(lane);
 }
 
-template <int BN, bool PAIR>
+template <int BN, bool PAIR, bool NORM>
 __global__ void __launch_bounds__(kTcThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
-               const __grid_constant__ CUtensorMap map_out, int M, int n_tiles_n,
+               const __grid_constant__ CUtensorMap map_out, const __grid_constant__ CUtensorMap map_xout, int M, int n_tiles_n,
                int K, int up_row_offset, int dp_tiles, long long per, int thin, float* split_ws, int* split_counters,
                EpiParams ep) {
-  using Cfg = TcCfg<BN, PAIR>;
+  using Cfg = TcCfg<BN, PAIR, NORM>;
   constexpr int kRows = PAIR ? 2 * BM : BM;              // rows of a scheduling unit's tile
   constexpr int kSlotMul = PAIR ? 2 : 1;                 // the CTAs of a pair use separate slots and counters
   const uint32_t rank = PAIR ? cluster_ctarank() : 0u;
@@ -497,20 +597,22 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
   const int n_stages = thin ? Cfg::kThinStages : Cfg::kStages;
   const int a_bytes = thin ? Cfg::kThinABytes : Cfg::kABytes;
   const int stage_bytes = a_bytes + Cfg::kBBytes;
-  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + Cfg::kRingBytes + kStageOutBytes);
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + Cfg::kBarOff);
   uint64_t* empty_bar = full_bar + Cfg::kMaxStages;
   uint64_t* tfull_bar = empty_bar + Cfg::kMaxStages;
   uint64_t* tempty_bar = tfull_bar + 2;
   uint64_t* red_bar = tempty_bar + 2;      // completion of the partial tiles fetched into the idle ring (used once)
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(red_bar + 1);
+  uint64_t* h_bar = red_bar + 1;           // [4 epilogue warps][2 slots]: old residual rows have landed (NORM only)
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(h_bar + 8);
 
-  // A wait that runs out records why and raises this CTA-wide flag.  The producer and the MMA issuer then leave
-  // their loops; the epilogue warps keep walking theirs WITHOUT blocking any more, so that all four of them still
-  // meet at every named barrier and every cut tile's arrival counter is still incremented (the counters stay
-  // consistent for the next launch; the outputs of this one are garbage and the status word says so).
+  // Bounded waits.  The producer and the MMA issuer leave their loops when a wait runs out.  The four epilogue warps
+  // must all keep meeting at the named barriers and must keep counting the arrivals of cut tiles (so that the counters
+  // stay consistent for the next launch), so they never leave their loop: a wait of theirs that runs out records why
+  // and raises a CTA-wide flag, after which their waits return at once; the outputs of such a launch are garbage and
+  // the status word says so.  (The flag is only looked at between waits: polling it inside the producer's and the
+  // issuer's per-k-block waits cost up to 40 % on narrow tiles.)
   __shared__ volatile int s_abort;
-  auto wait_or_abort = [&](uint64_t* bar, uint32_t parity, int code) -> bool {
-    if (s_abort) return false;
+  auto wait_bar = [&](uint64_t* bar, uint32_t parity) -> bool {
     for (uint32_t i = 0; i < kSpin; ++i) {
       uint32_t ok;
       if constexpr (PAIR)
@@ -522,14 +624,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
       else
         ok = mbar_try_wait(bar, parity) ? 1u : 0u;
       if (ok) return true;
-      if (i > 64) {
-        if (s_abort) return false;
-        __nanosleep(32);
-      }
+      if (i > 64) __nanosleep(32);
     }
-    set_status(ep.status, code);
-    s_abort = 1;
     return false;
+  };
+  auto wait_or_abort = [&](uint64_t* bar, uint32_t parity, int code) {   // epilogue warps only
+    if (s_abort) return;
+    if (!wait_bar(bar, parity)) {
+      set_status(ep.status, code);
+      s_abort = 1;
+    }
   };
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -556,6 +660,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
       mbar_init(&tempty_bar[a], PAIR ? 8 : 4);
     }
     mbar_init(red_bar, 1);
+    for (int i = 0; i < 8; ++i) mbar_init(&h_bar[i], 1);
     fence_barrier_init();
     prefetch_tmap(&map_x);
     prefetch_tmap(&map_w);
@@ -640,7 +745,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
             ++issued;
             continue;
           }
-          if (!wait_or_abort(&empty_bar[s], ph ^ 1, DEV_TIMEOUT_EMPTY)) {
+          if (!wait_bar(&empty_bar[s], ph ^ 1)) {
+            set_status(ep.status, DEV_TIMEOUT_EMPTY);
             ok = false;
             break;
           }
@@ -670,14 +776,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
         const Piece pc = make_piece(jd, dp_tiles, pos, range_hi, KB, per, unit, n_units, n_tiles_m);
         const int kb0 = pc.kb0, kb1 = pc.kb1;
         const int acc = tcount & 1;
-        if (!wait_or_abort(&tempty_bar[acc], ((tcount >> 1) & 1) ^ 1, DEV_TIMEOUT_MMA)) break;
+        if (!wait_bar(&tempty_bar[acc], ((tcount >> 1) & 1) ^ 1)) {
+          set_status(ep.status, DEV_TIMEOUT_MMA);
+          break;
+        }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + acc * BN;
         for (int kb = kb0; kb < kb1; ++kb) {
           const int s = st_idx;
           const uint32_t ph = st_phase;
           if (++st_idx == n_stages) { st_idx = 0; st_phase ^= 1; }
-          if (!wait_or_abort(&full_bar[s], ph, DEV_TIMEOUT_FULL)) {
+          if (!wait_bar(&full_bar[s], ph)) {
+            set_status(ep.status, DEV_TIMEOUT_FULL);
             ok = false;
             break;
           }
@@ -707,6 +817,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     float* stg = reinterpret_cast<float*>(smem + Cfg::kRingBytes) + (warp - 2) * 1024;
     uint32_t tcount = 0;
     __shared__ int s_last;
+    NormStage ns{smem + Cfg::kNormOff + (warp - 2) * 8192, reinterpret_cast<uint4*>(smem + Cfg::kNormOff + kNormHBytes) + (warp - 2) * 32,
+                 h_bar + (warp - 2) * 2, 0u};
     griddep_wait();                        // the epilogue reads and writes what earlier kernels produced
     long long pos = range_lo;
     for (int jd = 0; jd < dp_count || pos < range_hi; ++tcount) {
@@ -714,11 +826,25 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
       const int tile = pc.tile, n_splits = pc.n_parts;
       const int tm = tile % n_tiles_m, tn = tile / n_tiles_m;
       const int acc = tcount & 1;
+      const int row_in_tile = quad * 32 + lane;
+      const int m = tm * kRows + (int)rank * BM + row_in_tile;
+      // the row's normalisation factor, fetched while the accumulator is still being computed: the partial sums of
+      // squares in slot order (the same bits in every tile of the row)
+      float rstd = 1.f;
+      if (ep.ss_in) {
+        float sq = 0.f;
+        if (m < ep.M)
+          for (int k = 0; k < ep.ss_slots; ++k) sq += __ldcg(ep.ss_in + (size_t)k * ep.ss_stride + m);
+        rstd = rsqrtf(sq * ep.norm_inv_n + ep.norm_eps);
+      }
+      // (likewise, for a whole tile, the gains and the first old residual rows)
+      const bool prepared = NORM && n_splits == 1;
+      if constexpr (NORM) {
+        if (prepared) norm_prepare(ep, ns, &map_out, tn * BN, BN, m - lane, lane);
+      }
       wait_or_abort(&tfull_bar[acc], (tcount >> 1) & 1, DEV_TIMEOUT_MMA);   // after a timeout: carry on without blocking
       tc_fence_after();
       const uint32_t tacc = tmem_base + ((uint32_t)(quad * 32) << 16) + acc * BN;
-      const int row_in_tile = quad * 32 + lane;
-      const int m = tm * kRows + (int)rank * BM + row_in_tile;
       // hands the accumulator back to the MMA issuer (of a pair: the leader's barrier collects both CTAs' warps)
       auto release_acc = [&]() {
         tc_fence_before();
@@ -730,7 +856,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
       };
       const int n0 = swiglu ? tn * (BN / 2) : tn * BN;
       if (n_splits == 1) {
-        row_epilogue<BN>(ep, TmemLoader{tacc}, m, n0, stg, &map_out);
+        row_epilogue<BN, NORM>(ep, TmemLoader{tacc}, m, n0, stg, &map_out, &map_xout, rstd, tn, ns, prepared);
         release_acc();
       } else {
         // park this split's partial tile and let the LAST split to arrive reduce all partials in split order
@@ -769,7 +895,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
           // taken from TMEM.  Otherwise the parts are read from global memory while the next piece's main loop runs.
           constexpr int kPartBytes = BM * BN * 4;
           const bool final_piece = !(jd < dp_count || pos < range_hi);
-          if (final_piece && (n_splits - 1) * kPartBytes <= kSmemBudget) {
+          if (final_piece && (n_splits - 1) * kPartBytes <= Cfg::kBudget) {
             if (warp == 2 && lane == 0) {
               asm volatile("fence.proxy.async;" ::: "memory");   // the parts were written with ordinary stores
               mbar_arrive_expect_tx(red_bar, (uint32_t)((n_splits - 1) * kPartBytes));
@@ -786,10 +912,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
             }
             wait_or_abort(red_bar, 0, DEV_TIMEOUT_FULL);
             RingLoader ld{tacc, reinterpret_cast<const float4*>(smem) + row_in_tile, BN, pc.part, n_splits};
-            row_epilogue<BN>(ep, ld, m, n0, stg, &map_out);
+            row_epilogue<BN, NORM>(ep, ld, m, n0, stg, &map_out, &map_xout, rstd, tn, ns, false);
           } else {
             SplitLoader ld{split_ws, BN, row_in_tile, slot0, slot_next, slot_stride, n_splits, m < ep.M};
-            row_epilogue<BN>(ep, ld, m, n0, stg, &map_out);
+            row_epilogue<BN, NORM>(ep, ld, m, n0, stg, &map_out, &map_xout, rstd, tn, ns, false);
           }
         }
         asm volatile("bar.sync 1, 128;" ::: "memory");       // s_last is reused by the next unit
@@ -841,7 +967,8 @@ struct TcState {
   EncodeTiledFn encode = nullptr;
   std::unordered_map<MapKey, CUtensorMap, MapKeyHash> maps;
   size_t evictions = 0;
-  bool configured[5] = {false, false, false, false, false};
+  int last_tiles_n = 0;       // column tiles of the last launch
+  bool configured[10] = {false, false, false, false, false, false, false, false, false, false};
 };
 
 template <typename Encode>
@@ -888,11 +1015,21 @@ bool get_out_map(TcState* st, const void* ptr, uint64_t rows, uint64_t cols, int
   });
 }
 
+template <int BN, bool PAIR, bool NORM>
+bool launch_bn_t(TcState* st, int idx, const GemmArgs& a, const EpiParams& ep, bool stream_k, cudaStream_t stream);
+
 template <int BN, bool PAIR>
 bool launch_bn(TcState* st, int idx, const GemmArgs& a, const EpiParams& ep, bool stream_k, cudaStream_t stream) {
-  using Cfg = TcCfg<BN, PAIR>;
+  return a.epi == EPI_RESIDUAL_NORM ? launch_bn_t<BN, PAIR, true>(st, idx + 5, a, ep, stream_k, stream)
+                                    : launch_bn_t<BN, PAIR, false>(st, idx, a, ep, stream_k, stream);
+}
+
+template <int BN, bool PAIR, bool NORM>
+bool launch_bn_t(TcState* st, int idx, const GemmArgs& a, const EpiParams& ep, bool stream_k, cudaStream_t stream) {
+  st->last_tiles_n = (a.N + (a.epi == EPI_SWIGLU ? BN / 2 : BN) - 1) / (a.epi == EPI_SWIGLU ? BN / 2 : BN);
+  using Cfg = TcCfg<BN, PAIR, NORM>;
   if (!st->configured[idx]) {
-    if (cudaFuncSetAttribute(gemm_tc_kernel<BN, PAIR>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes) !=
+    if (cudaFuncSetAttribute(gemm_tc_kernel<BN, PAIR, NORM>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes) !=
         cudaSuccess)
       return false;
     st->configured[idx] = true;
@@ -906,7 +1043,9 @@ bool launch_bn(TcState* st, int idx, const GemmArgs& a, const EpiParams& ep, boo
   if (!get_map(st, a.w, w_rows, a.K, (swiglu || PAIR) ? BN / 2 : BN, &mw)) return false;
   // the epilogue stores through the TMA unit (of the rotary / KV-append epilogue: the rotated queries [M, n_q * d];
   // K and V are scattered into the paged pool by hand)
-  const bool f32 = a.epi == EPI_PLAIN_F32 || a.epi == EPI_RESIDUAL;
+  const bool f32 = a.epi == EPI_PLAIN_F32 || a.epi == EPI_RESIDUAL || a.epi == EPI_RESIDUAL_NORM;
+  CUtensorMap mxo = mx;       // only read by EPI_RESIDUAL_NORM
+  if (a.epi == EPI_RESIDUAL_NORM && !get_out_map(st, a.x_out, a.M, (uint64_t)a.N, 2, &mxo)) return false;
   if (!get_out_map(st, a.out, a.M, a.epi == EPI_QKV_ROPE ? (uint64_t)a.n_q * a.head_dim : (uint64_t)a.N, f32 ? 4 : 2, &mo))
     return false;
   const int out_per_tile = swiglu ? BN / 2 : BN;
@@ -954,7 +1093,7 @@ bool launch_bn(TcState* st, int idx, const GemmArgs& a, const EpiParams& ep, boo
   }
   cfg.attrs = attr;
   cfg.numAttrs = n_attr;
-  return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<BN, PAIR>, mx, mw, mo, a.M, n_tiles_n, a.K, a.N, dp_tiles, per, thin,
+  return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<BN, PAIR, NORM>, mx, mw, mo, mxo, a.M, n_tiles_n, a.K, a.N, dp_tiles, per, thin,
                             st->split_ws, st->split_counters, ep) == cudaSuccess;
 }
 
@@ -1037,9 +1176,18 @@ void tc_state_destroy(void* s) {
   delete st;
 }
 
-bool launch_gemm_tc(const GemmArgs& a, void* tc_state, int* status, cudaStream_t stream) {
+static bool launch_gemm_tc_impl(const GemmArgs& a, TcState* st, int* status, cudaStream_t stream);
+
+bool launch_gemm_tc(const GemmArgs& a, void* tc_state, int* status, cudaStream_t stream, int* ss_slots_out) {
   TcState* st = static_cast<TcState*>(tc_state);
   if (!st || a.M <= 0) return false;
+  if (a.epi == EPI_RESIDUAL_NORM && (!a.x_out || !a.gain || !a.ss_out || a.N % 32)) return false;
+  const bool ok = launch_gemm_tc_impl(a, st, status, stream);
+  if (ok && ss_slots_out) *ss_slots_out = st->last_tiles_n;
+  return ok;
+}
+
+static bool launch_gemm_tc_impl(const GemmArgs& a, TcState* st, int* status, cudaStream_t stream) {
   if (a.K % BK) return false;
   if ((reinterpret_cast<uintptr_t>(a.x) | reinterpret_cast<uintptr_t>(a.w)) & 15) return false;
   EpiParams ep;
@@ -1056,6 +1204,13 @@ bool launch_gemm_tc(const GemmArgs& a, void* tc_state, int* status, cudaStream_t
   ep.n_kv = a.n_kv;
   ep.head_dim = a.head_dim;
   ep.status = status;
+  ep.ss_in = a.ss_in;
+  ep.ss_slots = a.ss_slots;
+  ep.ss_stride = a.ss_stride;
+  ep.norm_inv_n = 1.f / (float)a.K;
+  ep.norm_eps = a.norm_eps;
+  ep.gain = static_cast<const __nv_bfloat16*>(a.gain);
+  ep.ss_out = a.ss_out;
   const bool swiglu = a.epi == EPI_SWIGLU;
   // Choose the tile width and the decomposition with a small cost model in microseconds, calibrated on B200:
   // whole tiles cost waves x k-blocks x (tensor time of one k-block at that width); the stream-K decomposition

@@ -64,8 +64,10 @@ size_t layout_smem_bytes(int n_req, int n_ctas);
 void launch_guard_fill(void* base, const size_t* offs_dev, int n, cudaStream_t st);
 void launch_guard_check(const void* base, const size_t* offs_dev, int n, int* status, cudaStream_t st);
 void launch_wait_timeout(uint32_t max_polls, int* status, cudaStream_t st);
-// S2: h[t] = embed[tok_id[t]] (fp32 residual stream).
-void launch_embed(const BatchLayout& bl, const Dims& dm, const void* embed, float* h, cudaStream_t st);
+// S2: h[t] = embed[tok_id[t]] (fp32 residual stream).  With gain != null also the input of the first normalised
+// projection: x[t] = bf16(h[t] * gain) and ss[t] = sum h[t]^2 (one slot).
+void launch_embed(const BatchLayout& bl, const Dims& dm, const void* embed, float* h, const void* gain, void* x, float* ss,
+                  cudaStream_t st);
 // x = rmsnorm(h) * g, bf16 out.
 void launch_rmsnorm(const float* h, const void* gain, void* x, int rows, int hidden, float eps, cudaStream_t st);
 
@@ -78,7 +80,9 @@ enum Epilogue : int {
   EPI_PLAIN_F32 = 1,   // C fp32 [M,N]
   EPI_RESIDUAL = 2,    // h fp32 [M,N] += acc
   EPI_SWIGLU = 3,      // w is [2F,K]; out bf16 [M,F] = silu(x.wg) * (x.wu)
-  EPI_QKV_ROPE = 4     // rotate q and k heads, q -> bf16 [M, n_q*d], k/v -> paged pool at tok_slot
+  EPI_QKV_ROPE = 4,    // rotate q and k heads, q -> bf16 [M, n_q*d], k/v -> paged pool at tok_slot
+  EPI_RESIDUAL_NORM = 5  // h fp32 [M,N] += acc, and the input of the next RMSNorm-ed projection: x_out bf16 [M,N] =
+                         // h * gain, ss_out[column tile][row] = sum over the tile's columns of h^2 (tcgen05 path only)
 };
 struct GemmArgs {
   const void* x;   // bf16 [M,K]
@@ -93,12 +97,20 @@ struct GemmArgs {
   int64_t n_pages;
   int layer, n_q, n_kv, head_dim;
   const void* rope_cs;  // float2 [head_dim/2][M]: (cos, sin) of each token's rotary angles, frequency-major
+  // folded RMSNorm (see EpiParams in epilogue.cuh); all null / 0 when unused
+  const float* ss_in;   // consumer: partial sums of squares of the rows of x's source, [ss_slots][ss_stride]
+  int ss_slots, ss_stride;
+  float norm_eps;       // the mean is over K (the width of x)
+  void* x_out;          // EPI_RESIDUAL_NORM: bf16 [M,N]
+  const void* gain;     // EPI_RESIDUAL_NORM: bf16 [N]
+  float* ss_out;        // EPI_RESIDUAL_NORM: [column tiles][ss_stride]; *ss_slots_out receives the tile count
 };
 // legacy tensor path (mma.sync), any M; N multiple of 64 (EPI_SWIGLU: F multiple of 32), K multiple of 32
 void launch_gemm_simt(const GemmArgs& a, int* status, cudaStream_t st);
 // tcgen05 + TMA path; returns false if the shape is not supported by it
 struct TcGemmPlan;  // opaque: cached tensor maps
-bool launch_gemm_tc(const GemmArgs& a, void* tc_state, int* status, cudaStream_t st);
+// ss_slots_out (may be null): how many slots of ss_out an EPI_RESIDUAL_NORM launch fills
+bool launch_gemm_tc(const GemmArgs& a, void* tc_state, int* status, cudaStream_t st, int* ss_slots_out = nullptr);
 void* tc_state_create(int n_sm);
 void tc_state_destroy(void* s);
 // debugging aid: force the tile configuration of the following launches (bn 64 / 128 / 256 single CTAs, 384 = CTA pairs

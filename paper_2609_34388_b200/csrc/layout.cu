@@ -250,8 +250,10 @@ __global__ void __launch_bounds__(1024) layout_kernel(BatchLayout bl, int n_kv, 
   }
 }
 
-__global__ void embed_kernel(const int* __restrict__ tok_id, const __nv_bfloat16* __restrict__ embed,
-                             float* __restrict__ h, int hidden, int vocab) {
+__global__ void __launch_bounds__(256) embed_kernel(const int* __restrict__ tok_id, const __nv_bfloat16* __restrict__ embed,
+                                                    float* __restrict__ h, int hidden, int vocab,
+                                                    const __nv_bfloat16* __restrict__ gain, __nv_bfloat16* __restrict__ x,
+                                                    float* __restrict__ ss) {
   griddep_launch();
   griddep_wait();
   const int t = blockIdx.x;
@@ -259,7 +261,27 @@ __global__ void embed_kernel(const int* __restrict__ tok_id, const __nv_bfloat16
   id = id < 0 ? 0 : (id >= vocab ? vocab - 1 : id);
   const __nv_bfloat162* src = reinterpret_cast<const __nv_bfloat162*>(embed + (size_t)id * hidden);
   float2* dst = reinterpret_cast<float2*>(h + (size_t)t * hidden);
-  for (int i = threadIdx.x; i < hidden / 2; i += blockDim.x) dst[i] = __bfloat1622float2(src[i]);
+  float sq = 0.f;
+  for (int i = threadIdx.x; i < hidden / 2; i += blockDim.x) {
+    const float2 v = __bfloat1622float2(src[i]);
+    dst[i] = v;
+    if (gain) {
+      const float2 g = __bfloat1622float2(reinterpret_cast<const __nv_bfloat162*>(gain)[i]);
+      reinterpret_cast<uint32_t*>(x + (size_t)t * hidden)[i] = pack_bf16(v.x * g.x, v.y * g.y);
+      sq += v.x * v.x + v.y * v.y;
+    }
+  }
+  if (gain) {
+    __shared__ float red[8];
+    for (int o = 16; o; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = sq;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      float tot = 0.f;
+      for (int i = 0; i < 8; ++i) tot += red[i];
+      ss[t] = tot;
+    }
+  }
 }
 
 // One CTA per row; fp32 in, bf16 out.  hidden a multiple of 4.  The row is read once and kept in registers
@@ -360,9 +382,10 @@ void launch_layout(const BatchLayout& bl, const Dims& dm, int tok_per_tile, int 
   launch_pdl(layout_kernel, dim3(1), dim3(1024), smem, st, bl, dm.n_kv, dm.mask_id, tok_per_tile, n_ctas, n_pages, status);
 }
 
-void launch_embed(const BatchLayout& bl, const Dims& dm, const void* embed, float* h, cudaStream_t st) {
+void launch_embed(const BatchLayout& bl, const Dims& dm, const void* embed, float* h, const void* gain, void* x, float* ss,
+                  cudaStream_t st) {
   launch_pdl(embed_kernel, dim3(bl.n_tok), dim3(256), 0, st, (const int*)bl.tok_id, static_cast<const __nv_bfloat16*>(embed), h,
-             dm.hidden, dm.vocab);
+             dm.hidden, dm.vocab, static_cast<const __nv_bfloat16*>(gain), static_cast<__nv_bfloat16*>(x), ss);
 }
 
 void launch_rmsnorm(const float* h, const void* gain, void* x, int rows, int hidden, float eps, cudaStream_t st) {

@@ -63,6 +63,8 @@ struct recg_ctx {
   void* logits = nullptr;
   bool logits_valid = false;
   float2* rope_cs = nullptr;
+  float* ss = nullptr;           // folded RMSNorm: partial sums of squares of the residual rows, [slot][max_tokens]
+  int ss_slots = 0;              // slots the last producer filled
   float *part_o = nullptr, *part_ml = nullptr;
   RowPartial* vpart = nullptr;
   int max_chunks_total = 0;
@@ -173,6 +175,7 @@ size_t carve(recg_ctx* c, DeviceArena& A) {
   if (c->has_weights) {
     c->h = A.take<float>(Tm * d.hidden);
     c->x = A.take<__nv_bfloat16>(Tm * d.hidden);
+    c->ss = A.take<float>(Tm * (size_t)(d.hidden / 64 + 1));   // a column tile is at least 64 wide
     c->act = A.take<__nv_bfloat16>(Tm * d.ffn);
     const size_t esz = (g.flags & RECG_FLAG_LOGITS_BF16) ? 2 : 4;
     c->logits = A.take<uint8_t>(Tm * (size_t)d.vocab * esz);
@@ -328,10 +331,17 @@ recg_status upload_and_layout(recg_ctx* ctx, const recg_batch* b, bool need_page
   return RECG_OK;
 }
 
-recg_status run_gemm(recg_ctx* ctx, const GemmArgs& a) {
+recg_status run_gemm(recg_ctx* ctx, const GemmArgs& a, int* ss_slots_out = nullptr) {
   bool done = false;
-  if (!(ctx->cfg.flags & RECG_FLAG_SIMT_GEMM)) done = launch_gemm_tc(a, ctx->tc_state, ctx->d_status, ctx->stream);
-  if (!done) launch_gemm_simt(a, ctx->d_status, ctx->stream);
+  if (!(ctx->cfg.flags & RECG_FLAG_SIMT_GEMM)) done = launch_gemm_tc(a, ctx->tc_state, ctx->d_status, ctx->stream, ss_slots_out);
+  if (!done) {
+    // the folded RMSNorm exists on the tcgen05 path only: a projection that takes part in it must not fall back
+    if (a.ss_in || a.epi == EPI_RESIDUAL_NORM) {
+      cudaGetLastError();
+      return fail(ctx, RECG_ERR_INTERNAL, "projection: the tcgen05 kernel refused a shape of the step");
+    }
+    launch_gemm_simt(a, ctx->d_status, ctx->stream);
+  }
   CU(cudaGetLastError());
   return RECG_OK;
 }
@@ -501,16 +511,37 @@ recg_status recg_step(recg_ctx* ctx, const recg_batch* batch, recg_logits* logit
   const int T = bl.n_tok;
   cudaStream_t st = ctx->stream;
   launch_rope_table(bl.tok_pos, T, d.head_dim, d.rope_base, ctx->rope_cs, st);
-  launch_embed(bl, d, ctx->embed, ctx->h, st);
+  // RMSNorm runs as a kernel of its own, or (RECG_FLAG_FOLD_NORM, tcgen05 path only) folded into the projections:
+  // whoever writes the residual stream also writes x = bf16(h * gain of the next norm) and partial sums of squares per
+  // row, and the projection that reads x scales its accumulator rows by the row's rstd.
+  const bool fold = (ctx->cfg.flags & RECG_FLAG_FOLD_NORM) && !(ctx->cfg.flags & RECG_FLAG_SIMT_GEMM);
+  const int Tm = ctx->cfg.max_tokens;
+  const void* first_gain = d.n_layers > 0 ? ctx->attn_norm[0] : ctx->final_norm;
+  launch_embed(bl, d, ctx->embed, ctx->h, fold ? first_gain : nullptr, ctx->x, ctx->ss, st);
+  int slots = 1;
   CU(cudaGetLastError());
   ctx->mark(0, 3);
   const int qdim = d.n_q * d.head_dim;
+  auto normed = [&](GemmArgs& g) {       // g reads the normalised residual stream
+    g.x = ctx->x;
+    g.K = d.hidden;
+    if (fold) { g.ss_in = ctx->ss; g.ss_slots = slots; g.ss_stride = Tm; g.norm_eps = d.rms_eps; }
+  };
+  auto residual = [&](GemmArgs& g, const void* next_gain) {   // g adds into the residual stream
+    g.out = ctx->h;
+    g.N = d.hidden;
+    g.epi = fold ? EPI_RESIDUAL_NORM : EPI_RESIDUAL;
+    if (fold) { g.x_out = ctx->x; g.gain = next_gain; g.ss_out = ctx->ss; g.ss_stride = Tm; }
+  };
   for (int l = 0; l < d.n_layers; ++l) {
-    launch_rmsnorm(ctx->h, ctx->attn_norm[l], ctx->x, T, d.hidden, d.rms_eps, st);
-    ctx->mark(1, 1);
+    if (!fold) {
+      launch_rmsnorm(ctx->h, ctx->attn_norm[l], ctx->x, T, d.hidden, d.rms_eps, st);
+      ctx->mark(1, 1);
+    }
     GemmArgs a{};
-    a.x = ctx->x; a.w = ctx->wqkv[l]; a.out = ctx->q;
-    a.M = T; a.N = (d.n_q + 2 * d.n_kv) * d.head_dim; a.K = d.hidden; a.epi = EPI_QKV_ROPE;
+    normed(a);
+    a.w = ctx->wqkv[l]; a.out = ctx->q;
+    a.M = T; a.N = (d.n_q + 2 * d.n_kv) * d.head_dim; a.epi = EPI_QKV_ROPE;
     a.tok_pos = bl.tok_pos; a.tok_slot = bl.tok_slot; a.kv_pool = batch->kv_pool; a.n_pages = batch->kv_pool_pages;
     a.layer = l; a.n_q = d.n_q; a.n_kv = d.n_kv; a.head_dim = d.head_dim; a.rope_cs = ctx->rope_cs;
     if ((s = run_gemm(ctx, a)) != RECG_OK) return s;
@@ -520,25 +551,33 @@ recg_status recg_step(recg_ctx* ctx, const recg_batch* batch, recg_logits* logit
     CU(cudaGetLastError());
     ctx->mark(3, 2);
     GemmArgs b{};
-    b.x = ctx->o; b.w = ctx->wo[l]; b.out = ctx->h; b.M = T; b.N = d.hidden; b.K = qdim; b.epi = EPI_RESIDUAL;
-    if ((s = run_gemm(ctx, b)) != RECG_OK) return s;
+    residual(b, ctx->ffn_norm[l]);
+    b.x = ctx->o; b.w = ctx->wo[l]; b.M = T; b.K = qdim;
+    if ((s = run_gemm(ctx, b, &slots)) != RECG_OK) return s;
     ctx->mark(4, 1);
-    launch_rmsnorm(ctx->h, ctx->ffn_norm[l], ctx->x, T, d.hidden, d.rms_eps, st);
-    ctx->mark(1, 1);
+    if (!fold) {
+      launch_rmsnorm(ctx->h, ctx->ffn_norm[l], ctx->x, T, d.hidden, d.rms_eps, st);
+      ctx->mark(1, 1);
+    }
     GemmArgs c{};
-    c.x = ctx->x; c.w = ctx->w_gate_up[l]; c.out = ctx->act; c.M = T; c.N = d.ffn; c.K = d.hidden; c.epi = EPI_SWIGLU;
+    normed(c);
+    c.w = ctx->w_gate_up[l]; c.out = ctx->act; c.M = T; c.N = d.ffn; c.epi = EPI_SWIGLU;
     if ((s = run_gemm(ctx, c)) != RECG_OK) return s;
     ctx->mark(5, 1);
     GemmArgs e{};
-    e.x = ctx->act; e.w = ctx->w_down[l]; e.out = ctx->h; e.M = T; e.N = d.hidden; e.K = d.ffn; e.epi = EPI_RESIDUAL;
-    if ((s = run_gemm(ctx, e)) != RECG_OK) return s;
+    residual(e, l + 1 < d.n_layers ? ctx->attn_norm[l + 1] : ctx->final_norm);
+    e.x = ctx->act; e.w = ctx->w_down[l]; e.M = T; e.K = d.ffn;
+    if ((s = run_gemm(ctx, e, &slots)) != RECG_OK) return s;
     ctx->mark(6, 1);
   }
-  launch_rmsnorm(ctx->h, ctx->final_norm, ctx->x, T, d.hidden, d.rms_eps, st);
-  ctx->mark(1, 1);
+  if (!fold) {
+    launch_rmsnorm(ctx->h, ctx->final_norm, ctx->x, T, d.hidden, d.rms_eps, st);
+    ctx->mark(1, 1);
+  }
   const bool lbf = ctx->cfg.flags & RECG_FLAG_LOGITS_BF16;
   GemmArgs f{};
-  f.x = ctx->x; f.w = ctx->lm_head; f.out = ctx->logits; f.M = T; f.N = d.vocab; f.K = d.hidden;
+  normed(f);
+  f.w = ctx->lm_head; f.out = ctx->logits; f.M = T; f.N = d.vocab;
   f.epi = lbf ? EPI_PLAIN_BF16 : EPI_PLAIN_F32;
   if ((s = run_gemm(ctx, f)) != RECG_OK) return s;
   ctx->mark(7, 1);
