@@ -92,10 +92,10 @@ def c16_descriptor(seed):
     return synth.batch_descriptor(16, [4, 8, 16, 32], None, 512, 8192, seed=seed)
 
 
-def c128_descriptor(seed, ctx_scale=0.5):
-    """configs[3]: concurrency 128, blocks {2,4,8,16} @ (.4,.3,.2,.1).  Context lengths are U[1024,16384] x ctx_scale:
-    at full length the KV pool alone is ~146 GB, which does not fit beside weights and workspace; 0.5 keeps it at
-    ~73 GB (still far beyond L2) and is stated in the result."""
+def c128_descriptor(seed, ctx_scale=1.0):
+    """configs[3]: concurrency 128, blocks {2,4,8,16} @ (.4,.3,.2,.1), context lengths U[1024,16384] x ctx_scale.  At
+    full length the KV pool alone is about 146 GB; bench_c128 takes ctx_scale = 1 when the device has room for it
+    beside weights and workspace and 0.5 otherwise, and says which in its result."""
     return synth.batch_descriptor(128, [2, 4, 8, 16], [0.4, 0.3, 0.2, 0.1], int(1024 * ctx_scale), int(16384 * ctx_scale),
                                   seed=seed)
 
@@ -123,6 +123,20 @@ def algorithmic_counts(shape, desc):
             "verify_bytes": logits_bytes}
 
 
+NOMINAL_HBM_GBS = 8000.0        # the workload statement's "about 8 TB/s"
+
+
+def hbm_fracs(gbs, peaks):
+    """Every bandwidth fraction is stated against both denominators: the measured copy bandwidth and 8 TB/s."""
+    return {"frac_of_hbm_measured": round(gbs / peaks["hbm_gbs"], 4), "frac_of_8000": round(gbs / NOMINAL_HBM_GBS, 4)}
+
+
+def tensor_fracs(tflops, peaks):
+    """... and every tensor fraction against the measured burst and sustained bf16 rates."""
+    return {"frac_of_bf16_burst": round(tflops / peaks["bf16_tflops"], 4),
+            "frac_of_bf16_sustained": round(tflops / peaks["bf16_tflops_sustained"], 4)}
+
+
 def roofline_entry(kind, achieved, peak, traffic=None, note=None):
     unit = "GB/s" if kind == "hbm" else "TFLOP/s"
     e = {"bound": kind, "achieved": round(achieved, 2), "peak": peak, "unit": unit, "frac": round(achieved / peak, 4),
@@ -144,7 +158,7 @@ def run_ours(args, env):
     shape = synth.llama8b_shape(32)
     t_setup = time.time()
     W = synth.model_weights(shape, seed=0, device=dev, dtype=torch.bfloat16)
-    descs = [c16_descriptor(3 + i + 100 * env.rank) for i in range(4)]           # rotate over 4 batch draws
+    descs = [c16_descriptor(3 + i + 100 * env.rank) for i in range(10)]          # ten batch draws (seeds 3..12), rotated
     max_pages = max(d.page_table.shape[1] for d in descs)
     n_pages = max(d.n_pages for d in descs)
     cfg = binding.make_config(shape, 16, 1024, max_pages, args.flags)
@@ -217,7 +231,7 @@ def run_ours(args, env):
            "warmup": args.warmup, "ms_per_step": round(ms_total_max / args.steps, 4), "higher_is_better": True,
            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
            "config": {"workload": "configs[2]: 32-layer 8B-class backbone, concurrency 16 per GPU, block sizes U{4,8,16,32}, "
-                                  "verify_len = block, context U[512,8192], 4 batch draws rotated",
+                                  "verify_len = block, context U[512,8192], 10 batch draws (seeds 3..12) rotated",
                       "tokens_per_step": [b.n_tok for b in batches], "l2": "inputs (15 GB weights, 10-20 GB KV) larger than L2",
                       "logits": "fp32", "parallelism": f"replicas x{env.world}" if env.world > 1 else "single GPU"},
            "clocks": clocks,
@@ -242,27 +256,48 @@ def run_ours(args, env):
         for k in gemm_classes:
             fl = sum(c["flops"][k] for c in counts)
             kern[k] = {"ms_per_step": round(ms[k] / args.steps, 4), "tflops": round(fl / (ms[k] / 1e3) / 1e12, 1),
-                       "frac_of_bf16_burst": round(fl / (ms[k] / 1e3) / 1e12 / peaks["bf16_tflops"], 4)}
+                       **tensor_fracs(fl / (ms[k] / 1e3) / 1e12, peaks)}
         ab = sum(c["attn_bytes"] for c in counts)
         kern["attention"] = {"ms_per_step": round(ms["attention"] / args.steps, 4),
                              "gbs": round(ab / (ms["attention"] / 1e3) / 1e9, 1),
-                             "frac_of_hbm": round(ab / (ms["attention"] / 1e3) / 1e9 / peaks["hbm_gbs"], 4)}
+                             **hbm_fracs(ab / (ms["attention"] / 1e3) / 1e9, peaks)}
         vb = sum(c["verify_bytes"] for c in counts)
         kern["verify"] = {"ms_per_step": round(ms["verify"] / args.steps, 4), "gbs": round(vb / (ms["verify"] / 1e3) / 1e9, 1),
-                          "frac_of_hbm": round(vb / (ms["verify"] / 1e3) / 1e9 / peaks["hbm_gbs"], 4)}
+                          **hbm_fracs(vb / (ms["verify"] / 1e3) / 1e9, peaks)}
         kern["rmsnorm"] = {"ms_per_step": round(ms["rmsnorm"] / args.steps, 4)}
         kern["layout"] = {"ms_per_step": round(ms["layout"] / args.steps, 4)}
         out["kernels"] = kern
         n_gemm_launch = sum(launches[k] for k in gemm_classes)
         ach = gemm_flops / (gemm_ms / 1e3) / 1e12
-        # DRAM traffic of one launch of the largest projection (gate|up, M = 480), from the ncu capture summarised in
-        # profiles/gemm_tc_kernel_shapes.md: 264.1 MB read + 53.7 MB written, against 2 x 28672 x 4096 x 2 B of weights
-        # + x + y = 266.4 MB algorithmic.  The mix of shapes in a step has no single per-launch figure.
-        out["roofline"] = roofline_entry("tensor", ach, peaks["bf16_tflops_sustained"], 317.8e6,
+        # `traffic` (DRAM bytes of one launch under the profiler) cannot be measured inside this run; it is null here and the
+        # profiler summary of the largest projection is kept with the other summaries under profiles/
+        out["roofline"] = roofline_entry("tensor", ach, peaks["bf16_tflops_sustained"], None,
                                          f"projection GEMM kernel (tcgen05), {n_gemm_launch} launches, avg "
-                                         f"{gemm_ms / max(n_gemm_launch, 1) * 1e3:.1f} us; peak = sustained bf16 of {peaks['source']}; "
-                                         "traffic = DRAM bytes of one gate|up launch at M = 480 under ncu (algorithmic 266.4e6)")
+                                         f"{gemm_ms / max(n_gemm_launch, 1) * 1e3:.1f} us; peak = sustained bf16 of {peaks['source']} "
+                                         f"(the kernel is timed inside a long step); of the burst rate: {ach / peaks['bf16_tflops']:.4f}; "
+                                         "traffic: not measurable in this run (the ncu summary of the gate|up launch is under profiles/)")
         out["step_time_share"] = {k: round(v / sum(ms.values()), 4) for k, v in ms.items()}
+    if env.rank == 0:
+        # ---- every batch draw by itself: mean and range over the ten draws ----
+        per = []
+        for j, bt in enumerate(batches):
+            for _ in range(2):
+                ctx.recg_step(bt)
+                ctx.recg_verify(bt, out=outs_dev[j])
+            torch.cuda.synchronize()
+            e0.record()
+            for _ in range(3):
+                ctx.recg_step(bt)
+                ctx.recg_verify(bt, out=outs_dev[j])
+            e1.record()
+            torch.cuda.synchronize()
+            per.append(e0.elapsed_time(e1) / 3)
+        tps = [b.n_tok / (m / 1e3) for b, m in zip(batches, per)]
+        out["draws"] = {"seeds": list(range(3, 13)), "tokens_per_step": [b.n_tok for b in batches],
+                        "ms_per_step": [round(m, 3) for m in per],
+                        "ms_mean": round(float(np.mean(per)), 3), "ms_min": round(min(per), 3), "ms_max": round(max(per), 3),
+                        "tokens_per_s_mean": round(float(np.mean(tps)), 1), "tokens_per_s_min": round(min(tps), 1),
+                        "tokens_per_s_max": round(max(tps), 1)}
     if args.quick:
         if env.rank == 0:
             out["c1"] = bench_c1(binding, ctx, shape, pool, n_pages, peaks, args)
@@ -337,10 +372,8 @@ def bench_second_model(binding, peaks, args):
            "weight_gb": round(wbytes / 1e9, 1),
            "ideal_ms": round(max(wbytes / peaks["hbm_gbs"] / 1e6, sum(cnt["flops"].values()) / peaks["bf16_tflops_sustained"] / 1e9)
                              + cnt["attn_bytes"] / peaks["hbm_gbs"] / 1e6, 3),
-           "gemm": {"ms_per_step": round(gemm_ms, 3), "tflops": round(gemm_tf, 1),
-                    "frac_of_bf16_sustained": round(gemm_tf / peaks["bf16_tflops_sustained"], 4)},
-           "attention": {"ms_per_step": round(attn_ms, 3), "gbs": round(attn_gbs, 1),
-                         "frac_of_hbm_measured": round(attn_gbs / peaks["hbm_gbs"], 4)}}
+           "gemm": {"ms_per_step": round(gemm_ms, 3), "tflops": round(gemm_tf, 1), **tensor_fracs(gemm_tf, peaks)},
+           "attention": {"ms_per_step": round(attn_ms, 3), "gbs": round(attn_gbs, 1), **hbm_fracs(attn_gbs, peaks)}}
     ctx.recg_free()
     del pool, W
     torch.cuda.empty_cache()
@@ -400,8 +433,7 @@ def bench_attention_op(binding, peaks, args, desc=None, n_layers=32, label=None)
     return {"workload": label or "configs[1]: 32/8 heads, d 128, context 4096, 16 causal + 16 bidirectional rows, "
                                  f"{n_layers} caches rotated, CUDA-graph replay",
             "us_per_call": round(us, 2), "calls_include": "attention kernel + combine kernel", "algorithmic_bytes": int(kv_bytes),
-            "gbs": round(gbs, 1), "frac_of_hbm_measured": round(gbs / peaks["hbm_gbs"], 4),
-            "frac_of_8000": round(gbs / 8000.0, 4)}
+            "gbs": round(gbs, 1), **hbm_fracs(gbs, peaks)}
 
 
 def bench_small_step(binding, peaks, args, n_layers=2, n_req=16):
@@ -461,51 +493,70 @@ def bench_gemm_shapes(binding, peaks):
             tf = 2.0 * M * N * K / (us * 1e-6) / 1e12
             gbs = N * K * 2 / (us * 1e-6) / 1e9
             out.append({"M": M, "name": name, "N": N, "K": K, "us": round(us, 1), "tflops": round(tf, 1),
-                        "frac_of_bf16_burst": round(tf / peaks["bf16_tflops"], 4), "weight_gbs": round(gbs, 1),
-                        "frac_of_hbm_measured": round(gbs / peaks["hbm_gbs"], 4)})
+                        **tensor_fracs(tf, peaks), "weight_gbs": round(gbs, 1), **hbm_fracs(gbs, peaks)})
             del x, w, y
     ctx.recg_free()
     return out
 
 
 def bench_verify(binding, peaks):
-    """configs[4]: verify kernel sweep over bf16 logits [B (k+1), 128256]; copies of the logits are rotated so
-    that the scan does not sit in L2, and one rotation is replayed from a CUDA graph (kernel time, not launch latency)."""
+    """configs[4]: the verify kernel over bf16 logits [B (k+1), 128256] ~ N(0,1) for every B in {1,8,32,128,256} and k in
+    {4,8,16,32}.  Drafts are planted: a prefix of Geometric(0.25) length (cut at k) equals the rows' argmax, the next
+    draft differs, the rest is random; the accept lengths that come back must be the planted ones.  Copies of the
+    logits are rotated so that the scan does not sit in L2, and one rotation is replayed from a CUDA graph (kernel
+    time, not launch latency)."""
     V = 128256
     res = []
     shape = synth.ModelShape(n_layers=0, hidden=64, n_q_heads=4, n_kv_heads=2, head_dim=64, ffn=64, vocab=V)
-    for B, k in [(1, 4), (8, 8), (32, 16), (128, 16), (256, 32)]:
-        R = B * (k + 1)
-        stream = torch.cuda.Stream()
-        with torch.cuda.stream(stream):
-            ctx = binding.Context(binding.make_config(shape, B, R, 1), stream=stream.cuda_stream)
-            lg = synth.logits_normal(R, V, seed=6, device="cuda")
-            y = synth.token_ids(R, V, seed=1)
-            batch = binding.Batch([0] * B, [k + 1] * B, [0] * B, y)
-            vout = binding.VerifyOut(B, R, R, host=False)
-            ctx.recg_verify(batch, lg, out=vout)
-            n_rot = max(2, min(64, int(np.ceil(300e6 / (R * V * 2)))))
-            copies = [lg] + [lg.clone() for _ in range(n_rot - 1)]
-            stream.synchronize()
+    for B in (1, 8, 32, 128, 256):
+        for k in (4, 8, 16, 32):
+            R = B * (k + 1)
+            stream = torch.cuda.Stream()
+            with torch.cuda.stream(stream):
+                ctx = binding.Context(binding.make_config(shape, B, R, 1), stream=stream.cuda_stream)
+                lg = synth.logits_normal(R, V, seed=6, device="cuda")
+                # the ids the rows select (lowest index among equal maxima), for the planting only
+                ids = torch.arange(V, device="cuda", dtype=torch.int32)
+                sel = []
+                for r0 in range(0, R, 512):
+                    part = lg[r0:r0 + 512].float()
+                    mx = part.max(dim=1, keepdim=True).values
+                    sel.append(torch.where(part == mx, ids, V).min(dim=1).values)
+                sel = torch.cat(sel)
+                accept = synth.planted_accept_lengths(B, k, 0.25, seed=4)
+                y = synth.plant_drafts(sel.cpu().numpy(), B, k, accept, V, seed=4).reshape(-1)
+                del mx, sel, part, ids
+                batch = binding.Batch([0] * B, [k + 1] * B, [0] * B, y)
+                vout = binding.VerifyOut(B, R, R, host=False)
+                ctx.recg_verify(batch, lg, out=vout)
+                stream.synchronize()
+                planted_ok = bool((vout.bufs["accept_len"][:B].cpu().numpy() == accept).all())
+                n_rot = max(2, min(64, int(np.ceil(300e6 / (R * V * 2)))))
+                copies = [lg] + [lg.clone() for _ in range(n_rot - 1)]
+                stream.synchronize()
 
-        def rotation():
-            for c in copies:
-                ctx.recg_verify(None, c, out=vout)
+            def rotation():
+                for c in copies:
+                    ctx.recg_verify(None, c, out=vout)
 
-        us = _time_graph(stream, rotation, 5) / len(copies)
-        gbs = R * V * 2 / (us * 1e-6) / 1e9
-        res.append({"B": B, "k": k, "rows": R, "us": round(us, 2), "gbs": round(gbs, 1),
-                    "frac_of_hbm_measured": round(gbs / peaks["hbm_gbs"], 4)})
-        ctx.recg_sync()
-        ctx.recg_free()
-        del copies, lg
-        torch.cuda.empty_cache()
+            us = _time_graph(stream, rotation, 5) / len(copies)
+            gbs = R * V * 2 / (us * 1e-6) / 1e9
+            res.append({"B": B, "k": k, "rows": R, "us": round(us, 2), "gbs": round(gbs, 1), **hbm_fracs(gbs, peaks),
+                        "emitted_tokens": int(accept.sum() + B), "accept_lengths_as_planted": planted_ok})
+            ctx.recg_sync()
+            ctx.recg_free()
+            del copies, lg
+            torch.cuda.empty_cache()
     return res
 
 
 def bench_c128(binding, W, shape, peaks, args):
     """High-concurrency point: full model, 128 requests (see c128_descriptor), per-class times."""
-    desc = c128_descriptor(5)
+    free_b, _ = torch.cuda.mem_get_info()
+    desc, ctx_scale = c128_descriptor(5, 1.0), 1.0
+    # pool + workspace (logits for 8192 rows and the rest: about 6 GB) + a margin must fit, else halve the contexts
+    if desc.n_pages * 16 * 131072 + (14 << 30) > free_b:
+        desc, ctx_scale = c128_descriptor(5, 0.5), 0.5
     # the same context and pool also serve the concurrency sweep below (configs[2]'s recipe at other batch sizes)
     sweep_descs = {C: synth.batch_descriptor(C, [4, 8, 16, 32], None, 512, 8192, seed=40 + C) for C in (1, 2, 4, 8, 16, 32, 64, 128)}
     # rounds with prospective correction branches (two per request, one block of the request's size each), and
@@ -515,12 +566,16 @@ def bench_c128(binding, W, shape, peaks, args):
     # forward time against concurrency for one block size at a time (the paper's Fig. 2b on random weights): T_C(B), the
     # profile the block-size rule weighs against the expected progress
     tcb_descs = {(C, B): synth.batch_descriptor(C, [B], None, 512, 8192, seed=80 + C) for C in (1, 4, 16, 64, 128) for B in (8, 16, 32)}
-    all_descs = [desc] + list(sweep_descs.values()) + list(ov_descs.values()) + list(tcb_descs.values())
+    # the block mixtures the paper's adaptive policy ends up with on its 8B model (its block-distribution table: shares
+    # of blocks 8 / 16 / 32 at each concurrency), contexts as in configs[2]: the paper-shaped points of the sweep
+    mix_descs = {C: synth.batch_descriptor(C, [8, 16, 32], [p / sum(mix) for p in mix], 512, 8192, seed=120 + C)
+                 for C, mix in ((2, (9.33, 2.54, 88.13)), (8, (3.70, 36.96, 59.34)), (32, (41.17, 43.33, 15.50)),
+                                (128, (78.21, 12.04, 9.75)))}
+    all_descs = [desc] + list(sweep_descs.values()) + list(ov_descs.values()) + list(tcb_descs.values()) + list(mix_descs.values())
     n_pages = max(d.n_pages for d in all_descs)
-    free_b, _ = torch.cuda.mem_get_info()
     cfg = binding.make_config(shape, 128, max(2048, max(d.n_tokens for d in all_descs)), max(d.page_table.shape[1] for d in all_descs))
     need = binding.lib().recg_kv_pool_bytes(__import__("ctypes").byref(cfg), n_pages)
-    if need + (10 << 30) > free_b:
+    if need + (8 << 30) > free_b:
         return {"skipped": f"pool of {need / 1e9:.0f} GB does not fit in the {free_b / 1e9:.0f} GB that are free"}
     ctx = binding.Context(cfg, W)
     pool = binding.alloc_kv_pool(ctx, n_pages, fill="normal")
@@ -555,6 +610,32 @@ def bench_c128(binding, W, shape, peaks, args):
     sweep_result = {"workload": "configs[2] recipe at other batch sizes, one draw each, processed tokens/s of the whole step; "
                                             "ideal_ms = max(weight stream, GEMM flops at sustained peak) + KV stream, of measured peaks",
                                 "points": sweep}
+    mix = []
+    for C, d in mix_descs.items():
+        ysw = synth.token_ids(int(d.verify_len.sum()), shape.vocab, seed=130 + C)
+        bt = binding.Batch(d.ctx_len, d.verify_len, d.block_size, ysw, d.page_table, pool, n_pages)
+        vo = binding.VerifyOut(bt.n_req, bt.n_tok, bt.n_ver, host=False)
+        n_it = 5 if C >= 32 else 20
+        for _ in range(3):
+            ctx.recg_step(bt)
+            ctx.recg_verify(bt, out=vo)
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(n_it):
+            ctx.recg_step(bt)
+            ctx.recg_verify(bt, out=vo)
+        e1.record()
+        torch.cuda.synchronize()
+        msw = e0.elapsed_time(e1) / n_it
+        cw = algorithmic_counts(shape, d)
+        mix.append({"concurrency": C, "blocks": {int(b): int((d.block_size == b).sum()) for b in (8, 16, 32)},
+                    "tokens_per_step": bt.n_tok, "ms_per_step": round(msw, 3), "tokens_per_s": round(bt.n_tok / (msw / 1e3), 1),
+                    "ideal_ms": round(max(sum(cw["wbytes"].values()) / peaks["hbm_gbs"] / 1e6,
+                                          sum(cw["flops"].values()) / peaks["bf16_tflops_sustained"] / 1e9) +
+                                      cw["attn_bytes"] / peaks["hbm_gbs"] / 1e6, 3)})
+    mix_result = {"workload": "block sizes drawn from the paper's reported 8B block distribution at each concurrency (shares of 8 / "
+                              "16 / 32), verify_len = block, context U[512,8192], one draw per point; whole step",
+                  "points": mix}
     tcb = []
     for (C, B), d in tcb_descs.items():
         ysw = synth.token_ids(int(d.verify_len.sum()), shape.vocab, seed=90)
@@ -640,7 +721,7 @@ def bench_c128(binding, W, shape, peaks, args):
             att = cms["attention"] / n_it
             res[kind] = {"rows_per_step": bt.n_tok, "ms_per_step": round(msw, 3), "rows_per_s": round(bt.n_tok / (msw / 1e3), 1),
                          "attention_ms": round(att, 3), "attention_gbs": round(cw["attn_bytes"] / (att / 1e3) / 1e9, 1),
-                         "attention_frac_of_hbm_measured": round(cw["attn_bytes"] / (att / 1e3) / 1e9 / peaks["hbm_gbs"], 4)}
+                         "attention": hbm_fracs(cw["attn_bytes"] / (att / 1e3) / 1e9, peaks)}
         res["step_time_ratio"] = round(res["branches"]["ms_per_step"] / res["plain"]["ms_per_step"], 3)
         overlap[key] = res
     overlap_result = {"workload": "configs[2] draw 0 (c16) and the concurrency-1 case (c1) with two correction branches per request "
@@ -674,15 +755,20 @@ def bench_c128(binding, W, shape, peaks, args):
     gemm_tf = sum(cnt["flops"][k] for k in gemm_classes) / (gemm_ms / 1e3) / 1e12
     attn_ms = cms["attention"] / iters
     attn_gbs = cnt["attn_bytes"] / (attn_ms / 1e3) / 1e9
-    out = {"workload": "configs[3] with context lengths halved (U[512,8192]) so that the 73 GB pool fits: concurrency 128, "
-                       "blocks {2,4,8,16} @ (.4,.3,.2,.1), verify_len = block",
-           "tokens_per_step": batch.n_tok, "kv_pool_gb": round(need / 1e9, 1), "ms_per_step": round(ms, 3),
-           "tokens_per_s": round(batch.n_tok / (ms / 1e3), 1),
-           "gemm": {"ms_per_step": round(gemm_ms, 3), "tflops": round(gemm_tf, 1),
-                    "frac_of_bf16_sustained": round(gemm_tf / peaks["bf16_tflops_sustained"], 4)},
-           "attention": {"ms_per_step": round(attn_ms, 3), "gbs": round(attn_gbs, 1),
-                         "frac_of_hbm_measured": round(attn_gbs / peaks["hbm_gbs"], 4)}}
+    label = ("configs[3] as stated: concurrency 128, blocks {2,4,8,16} @ (.4,.3,.2,.1), verify_len = block, context lengths "
+             "U[1024,16384]") if ctx_scale == 1.0 else \
+            ("configs[3] at HALF context (U[512,8192]: the full-length pool did not fit beside weights and workspace): "
+             "concurrency 128, blocks {2,4,8,16} @ (.4,.3,.2,.1), verify_len = block")
+    wb = sum(cnt["wbytes"].values())
+    out = {"workload": label, "context_scale": ctx_scale,
+           "tokens_per_step": batch.n_tok, "kv_tokens": int(np.sum(desc.ctx_len + desc.rows)), "kv_pool_gb": round(need / 1e9, 1),
+           "ms_per_step": round(ms, 3), "tokens_per_s": round(batch.n_tok / (ms / 1e3), 1),
+           "ideal_ms": round(max(wb / peaks["hbm_gbs"] / 1e6, sum(cnt["flops"].values()) / peaks["bf16_tflops_sustained"] / 1e9) +
+                             cnt["attn_bytes"] / peaks["hbm_gbs"] / 1e6, 3),
+           "gemm": {"ms_per_step": round(gemm_ms, 3), "tflops": round(gemm_tf, 1), **tensor_fracs(gemm_tf, peaks)},
+           "attention": {"ms_per_step": round(attn_ms, 3), "gbs": round(attn_gbs, 1), **hbm_fracs(attn_gbs, peaks)}}
     out["concurrency_sweep"] = sweep_result
+    out["block_mixture_sweep"] = mix_result
     out["bucketing"] = bucketing_result
     out["forward_time_by_block"] = tcb_result
     # block-size rule on the device after the verification of the 128-request batch (one small kernel; launch bound)
@@ -741,18 +827,17 @@ def bench_c1(binding, ctx, shape, pool, n_pages, peaks, args):
                     shape.vocab * shape.hidden)
     return {"workload": "concurrency 1, context 4096, verify 16 + block 16", "ms_per_step": round(ms, 4),
             "tokens_per_s": round(32 / (ms / 1e3), 1), "weight_stream_gbs": round(wbytes / (ms / 1e3) / 1e9, 1),
-            "frac_of_hbm_measured": round(wbytes / (ms / 1e3) / 1e9 / peaks["hbm_gbs"], 4),
-            "class_ms_per_step": classes}
+            **hbm_fracs(wbytes / (ms / 1e3) / 1e9, peaks), "class_ms_per_step": classes}
 
 
 # ------------------------------------------------------------------------------------------------
 # the oracle, timed as it stands on the host cores (reported baseline, and the --impl reference arm)
 # ------------------------------------------------------------------------------------------------
 class OracleSample:
-    """The CPU oracle, as it stands, on a bounded sample of the workload: request 0 of the batch through ONE of
-    the n_layers layers plus the LM head and verification; the layer time is scaled by n_layers."""
+    """The CPU oracle, as it stands, on a bounded sample of the workload: the first n_req requests of the batch through
+    ONE of the n_layers layers plus the LM head and verification; the layer time is scaled by n_layers."""
 
-    def __init__(self, shape, desc):
+    def __init__(self, shape, desc, n_req=1):
         from oracle import recg_oracle as orc
 
         self.orc = orc
@@ -763,39 +848,48 @@ class OracleSample:
                     for k, v in W.items() if k != "embed"}
         self.W64["embed"] = W["embed"].float().numpy()       # exact widening; rows are widened to fp64 on lookup
         self.ocfg = orc.ModelConfig(**one.as_dict())
-        self.L, self.v, self.b = int(desc.ctx_len[0]), int(desc.verify_len[0]), int(desc.block_size[0])
-        K, V = synth.kv_values(self.L, shape.n_kv_heads, shape.head_dim, seed=2, device="cpu")
-        self.kv = [(K.double().numpy(), V.double().numpy())]
-        self.y = synth.token_ids(self.v, shape.vocab, seed=1).tolist()
+        self.reqs = []
+        for r in range(min(n_req, desc.n_req)):
+            L, v, b = int(desc.ctx_len[r]), int(desc.verify_len[r]), int(desc.block_size[r])
+            K, V = synth.kv_values(L, shape.n_kv_heads, shape.head_dim, seed=2 + r, device="cpu")
+            self.reqs.append((L, b, [(K.double().numpy(), V.double().numpy())], synth.token_ids(v, shape.vocab, seed=1 + r).tolist()))
 
     def step(self):
         """Returns (tokens/s, seconds for the whole model by the scaling rule, tokens)."""
         orc = self.orc
-        t0 = time.perf_counter()
-        logits, _, h = orc.fused_round_cached(self.ocfg, self.W64, self.kv, self.L, self.y, self.b)
-        t1 = time.perf_counter()
-        x = orc.rmsnorm(h, self.W64["final_norm"], self.ocfg.rms_eps)     # the head alone, to split layer / head time
-        _ = x @ self.W64["lm_head"].T
-        t2 = time.perf_counter()
-        orc.verify_round(logits, self.y, self.b)
-        t3 = time.perf_counter()
-        head = t2 - t1
-        total = ((t1 - t0) - head) * self.shape.n_layers + head + (t3 - t2)
-        toks = self.v + self.b
+        layer = head = ver = 0.0
+        toks = 0
+        for (L, b, kv, y) in self.reqs:
+            t0 = time.perf_counter()
+            logits, _, h = orc.fused_round_cached(self.ocfg, self.W64, kv, L, y, b)
+            t1 = time.perf_counter()
+            x = orc.rmsnorm(h, self.W64["final_norm"], self.ocfg.rms_eps)     # the head alone, to split layer / head time
+            _ = x @ self.W64["lm_head"].T
+            t2 = time.perf_counter()
+            orc.verify_round(logits, y, b)
+            t3 = time.perf_counter()
+            head += t2 - t1
+            layer += (t1 - t0) - (t2 - t1)
+            ver += t3 - t2
+            toks += len(y) + b
+        total = layer * self.shape.n_layers + head + ver
         return toks / total, total, toks
 
     def describe(self):
-        return (f"request 0 of the concurrency-16 batch ({self.v + self.b} rows over {self.L} context tokens) through 1 of "
+        rows = sum(len(y) + b for (_, b, _, y) in self.reqs)
+        ctxs = sum(L for (L, _, _, _) in self.reqs)
+        return (f"{len(self.reqs)} request(s) of the concurrency-16 batch ({rows} rows over {ctxs} context tokens) through 1 of "
                 f"{self.shape.n_layers} layers (time x{self.shape.n_layers}) plus the full LM head and verification; fp64 numpy")
 
 
 def cpu_baseline(shape, desc):
     import multiprocessing
 
-    s = OracleSample(shape, desc)
+    s = OracleSample(shape, desc, n_req=desc.n_req)       # the whole batch: some tens of seconds of CPU work
+    t0 = time.perf_counter()
     tps, secs, toks = s.step()
     return {"value": round(tps, 2), "unit": UNIT, "cores": multiprocessing.cpu_count(), "kind": "oracle",
-            "sample": s.describe(), "seconds_scaled": round(secs, 2)}
+            "sample": s.describe(), "seconds_scaled": round(secs, 2), "seconds_spent": round(time.perf_counter() - t0, 1)}
 
 
 def run_reference(args, env):

@@ -27,6 +27,10 @@ struct AttnTile {        // per (request, kv head, row tile): where its partials
 // Device-resident ragged layout of one batch (all pointers DEVICE, int32 unless noted).
 struct BatchLayout {
   int n_req, n_tok, n_ver, pt_stride;
+  // Device-resident rounds: the row counts are only known on the device.  dyn (null otherwise) points to
+  // {n_tok, n_ver}; n_tok / n_ver above are then the capacities the launches are sized for, and every kernel takes the
+  // true counts from dyn.
+  const int* dyn;
   float risk_delta;       // margin threshold of the risky-position outputs
   const int* ctx_len;     // [C]
   const int* verify_len;  // [C]
@@ -68,11 +72,36 @@ void launch_wait_timeout(uint32_t max_polls, int* status, cudaStream_t st);
 // projection: x[t] = bf16(h[t] * gain) and ss[t] = sum h[t]^2 (one slot).
 void launch_embed(const BatchLayout& bl, const Dims& dm, const void* embed, float* h, const void* gain, void* x, float* ss,
                   cudaStream_t st);
-// x = rmsnorm(h) * g, bf16 out.
-void launch_rmsnorm(const float* h, const void* gain, void* x, int rows, int hidden, float eps, cudaStream_t st);
+// x = rmsnorm(h) * g, bf16 out.  rows_dev (may be null): the true row count on the device (rows is then the capacity).
+void launch_rmsnorm(const float* h, const void* gain, void* x, int rows, int hidden, float eps, cudaStream_t st,
+                    const int* rows_dev = nullptr);
+
+struct VerifyBuffers;
+// Device-resident rounds (Sec. 5.2).  pack: builds the packed descriptor (the layout recg_api.cu uploads in the host
+// mode: ctx_len | verify_len | block_size | corr | cu_tok | cu_ver | verify_tokens) in `desc` from the caller's device
+// arrays and writes {n_tok, n_ver} to dyn; violations of the capacities set the status word and give an empty round.
+struct DeviceRound {
+  int n_req, max_verify, pt_stride, max_tokens;
+  int *ctx_len, *verify_len, *block_size, *verify_tokens;    // caller's device arrays; verify tokens of request r at r * max_verify
+};
+void launch_pack_device(const DeviceRound& dr, int* desc, int* dyn, int* status, cudaStream_t st);
+// next: turns the results of the finished round into the next round's arrays (in place) and appends to the logs.
+struct RoundLog {
+  int* tokens;       // [n_req][max_out] emitted tokens
+  int max_out;
+  int* n_tokens;     // [n_req]
+  int* accept_len;   // [max_rounds][n_req] accepted drafts, block size used and verify length of every round
+  int* block_size;
+  int* verify_len;
+  int max_rounds;
+  int* n_rounds;     // [1]
+};
+void launch_next_round(const DeviceRound& dr, const BatchLayout& bl, const VerifyBuffers& vb, const int* next_block,
+                       const int* planted_emitted, const RoundLog& log, int* status, cudaStream_t st);
 
 // (cos, sin) of pos * base^(-2i/d), angles evaluated in double: cs float2 [head_dim/2][T] (frequency-major).
-void launch_rope_table(const int* tok_pos, int n_tok, int head_dim, float rope_base, void* cs, cudaStream_t st);
+void launch_rope_table(const int* tok_pos, int n_tok, int head_dim, float rope_base, void* cs, cudaStream_t st,
+                       const int* n_tok_dev = nullptr);
 
 // Projection epilogues.
 enum Epilogue : int {
@@ -97,6 +126,10 @@ struct GemmArgs {
   int64_t n_pages;
   int layer, n_q, n_kv, head_dim;
   const void* rope_cs;  // float2 [head_dim/2][M]: (cos, sin) of each token's rotary angles, frequency-major
+  // device-resident rounds: the true row count (M is then the capacity the tensor maps cover), and the row count the
+  // tile configuration is chosen for (0: M)
+  const int* m_dev;
+  int m_hint;
   // folded RMSNorm (see EpiParams in epilogue.cuh); all null / 0 when unused
   const float* ss_in;   // consumer: partial sums of squares of the rows of x's source, [ss_slots][ss_stride]
   int ss_slots, ss_stride;
@@ -145,7 +178,7 @@ struct RowPartial {      // per (row, vocab chunk)
   float s, t;            // sum exp(x - m1), sum x exp(x - m1)
 };
 void launch_verify(const BatchLayout& bl, const void* logits, int logits_dtype, int vocab, RowPartial* partials,
-                   int max_chunks_total, const VerifyBuffers& vb, int n_sm, cudaStream_t st);
+                   int max_chunks_total, const VerifyBuffers& vb, int n_sm, cudaStream_t st);   // (bl.dyn: rows from the device)
 int verify_chunks_per_row(int rows, int vocab, int n_sm);
 
 // Block-size rule (Eq. 2-3): table = [blocks (int) x8 | cost x8 | edges x64 | value n_blocks*n_bins*n_blocks*2]
