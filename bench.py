@@ -321,6 +321,9 @@ def run_ours(args, env):
     del pool, ctx
     torch.cuda.empty_cache()
     if env.rank == 0 and env.world == 1:
+        out["device_loop"] = {"workload": "8 rounds with planted acceptance and the block-size rule, device-resident against "
+                                          "host-driven, 32-layer 8B-class backbone",
+                              "points": [bench_device_loop(binding, W, shape, peaks, n) for n in (1, 16)]}
         out["c128"] = bench_c128(binding, W, shape, peaks, args)
         del W
         torch.cuda.empty_cache()
@@ -830,6 +833,102 @@ def bench_c1(binding, ctx, shape, pool, n_pages, peaks, args):
             **hbm_fracs(wbytes / (ms / 1e3) / 1e9, peaks), "class_ms_per_step": classes}
 
 
+def bench_device_loop(binding, W, shape, peaks, n_req, rounds=8):
+    """Rounds per second with and without host round trips: the same requests run `rounds` rounds (a) device-resident --
+    step, verification, block-size rule and next-round bookkeeping enqueued back to back, one sync at the end -- and
+    (b) host-driven -- results copied to the host after every round and the next descriptor built there.  Acceptance
+    lengths are planted from the interval chain of the paper's transition table (random weights accept nothing); block
+    sizes come from the rule with a synthetic value table over {8, 16, 32}; contexts U[512, 8192]."""
+    rng = np.random.default_rng(200 + n_req)
+    Ls = rng.integers(512, 8193, size=n_req).astype(np.int32)
+    grow = rounds * 33 + 64
+    pt, n_pages = synth.page_tables(Ls, [grow] * n_req, 16, seed=201)
+    max_tok = n_req * 64
+    ctx = binding.Context(binding.make_config(shape, n_req, max_tok, pt.shape[1]), W)
+    pool = binding.alloc_kv_pool(ctx, n_pages, fill="normal")
+    tb = synth.policy_table()
+    ctx.recg_policy_load(tb["blocks"], tb["s_edges"], tb["value"], tb["cost"])
+    planted = synth.acceptance_chain_lengths(rounds, n_req, seed=202)            # [rounds, n_req] emitted tokens per round
+    pl_dev = torch.from_numpy(planted).cuda()
+    y0 = [[int(t)] for t in synth.token_ids(n_req, shape.vocab, seed=203)]
+
+    def fresh_state():
+        return {"e1": torch.zeros(n_req, dtype=torch.float32, device="cuda"), "e2": torch.zeros(n_req, dtype=torch.float32, device="cuda"),
+                "block_index": torch.zeros(n_req, dtype=torch.int32, device="cuda"), "full": torch.zeros(n_req, dtype=torch.int32, device="cuda")}
+
+    nxt = torch.zeros(n_req, dtype=torch.int32, device="cuda")
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+    def run_device():
+        db = binding.DeviceBatch(Ls, [1] * n_req, [16] * n_req, y0, 32, pt, pool, n_pages, rows_hint=n_req * 24)
+        st = fresh_state()
+        log = binding.RoundLog(n_req, rounds, rounds * 33)
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        e0.record()
+        for r in range(rounds):
+            ctx.recg_step_device(db)
+            ctx.recg_verify_device()
+            ctx.recg_policy_step(st, nxt)
+            ctx.recg_next_round(db, r, next_block=nxt, planted_emitted=pl_dev[r], log=log)
+        e1.record()
+        torch.cuda.synchronize()
+        wall = (time.perf_counter() - t0) * 1e3
+        return max(e0.elapsed_time(e1), wall), int(log.n_tokens.sum()), log.block_size.cpu().numpy()
+
+    def run_host():
+        L, v, b = Ls.copy(), np.ones(n_req, np.int32), np.full(n_req, 16, np.int32)
+        ys = [list(y) for y in y0]
+        st = fresh_state()
+        emitted = 0
+        blocks = []
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        e0.record()
+        for r in range(rounds):
+            bt = binding.Batch(L, v, b, [t for y in ys for t in y], pt, pool, n_pages)
+            ctx.recg_step(bt)
+            g = ctx.recg_verify(bt)                       # host results: copies and a sync every round
+            ctx.recg_policy_step(st, nxt)
+            nb = nxt.cpu().numpy()                        # the host needs the next block sizes to size the next batch
+            blocks.append(b.copy())
+            cuv = np.concatenate([[0], np.cumsum(v)])
+            cub = np.concatenate([[0], np.cumsum(b)])
+            for i in range(n_req):                        # the bookkeeping between rounds, on the host
+                e = max(1, min(int(planted[r, i]), int(v[i])))
+                a = e - 1
+                last = int(g["top1"][int(cuv[i] + cub[i]) + a])
+                reuse = b[i] > 0 and a == v[i] - 1
+                emitted += e
+                L[i] += e
+                if reuse:
+                    ys[i] = [last] + g["next_draft"][int(cub[i]) + 1: int(cub[i]) + int(b[i])].tolist()
+                else:
+                    ys[i] = [last]
+                v[i] = len(ys[i])
+                b[i] = nb[i]
+        e1.record()
+        torch.cuda.synchronize()
+        wall = (time.perf_counter() - t0) * 1e3
+        return max(e0.elapsed_time(e1), wall), emitted, np.asarray(blocks)
+
+    run_device()
+    run_host()
+    ms_d, em_d, blk_d = run_device()
+    ms_h, em_h, blk_h = run_host()
+    ctx.recg_sync()
+    ctx.recg_free()
+    del pool
+    torch.cuda.empty_cache()
+    return {"concurrency": n_req, "rounds": rounds,
+            "device_resident": {"ms_per_round": round(ms_d / rounds, 3), "rounds_per_s": round(rounds / (ms_d / 1e3), 1),
+                                "emitted_tokens": em_d, "emitted_tokens_per_s": round(em_d / (ms_d / 1e3), 1)},
+            "host_driven": {"ms_per_round": round(ms_h / rounds, 3), "rounds_per_s": round(rounds / (ms_h / 1e3), 1),
+                            "emitted_tokens": em_h, "emitted_tokens_per_s": round(em_h / (ms_h / 1e3), 1)},
+            "same_emitted_tokens": em_d == em_h, "same_block_sizes": bool((blk_d == blk_h).all()),
+            "host_over_device": round(ms_h / ms_d, 3)}
+
+
 # ------------------------------------------------------------------------------------------------
 # the oracle, timed as it stands on the host cores (reported baseline, and the --impl reference arm)
 # ------------------------------------------------------------------------------------------------
@@ -919,7 +1018,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--flags", type=int, default=0, help="recg_config.flags of the timed context (A/B checks)")
     ap.add_argument("--quick", action="store_true", help="the timed step, its per-class times and the concurrency-1 point only")
-    ap.add_argument("--only", default="", help="comma list of op-level sections to run alone (attention_op, attention_c16, attention_c16_branches, small_step, verify_sweep, gemm_shapes): "
+    ap.add_argument("--only", default="", help="comma list of op-level sections to run alone (attention_op, attention_c16, attention_c16_branches, small_step, device_loop, verify_sweep, gemm_shapes): "
                                                "small cases for profiling; prints their JSON and exits")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
@@ -946,6 +1045,10 @@ def main():
                                               desc=synth.with_correction_branches(c16_descriptor(3), 128256, 2, seed=60),
                                               label="attention of configs[2] draw 0 with two correction branches per request "
                                                     "(784 rows instead of 376), 4 layer caches rotated, CUDA-graph replay")
+            elif sec == "device_loop":
+                shape2 = synth.llama8b_shape(2)
+                W2 = synth.model_weights(shape2, seed=0, device="cuda", dtype=torch.bfloat16)
+                res[sec] = [bench_device_loop(binding, W2, shape2, peaks, n) for n in (1, 16)]
             elif sec == "small_step":
                 res[sec] = bench_small_step(binding, peaks, args)
             elif sec == "verify_sweep":

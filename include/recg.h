@@ -325,6 +325,61 @@ recg_status recg_policy_step(recg_ctx *ctx, const recg_policy_state *state, cons
                              const int32_t *accept_len, int32_t *next_block);
 
 /*
+ * Device-resident rounds (Sec. 5.2: the verification history of one round guides the next one; nothing has to come back
+ * to the host in between).  The descriptor arrays live on the DEVICE and belong to the caller; the library reads them
+ * when the step executes and recg_next_round() rewrites them in place, so N rounds are N x { recg_step_device,
+ * recg_verify(ctx, NULL, NULL, 0, out with mem = RECG_MEM_DEVICE), optionally recg_policy_step, recg_next_round }
+ * enqueued back to back with one synchronisation at the end.
+ *
+ * recg_device_batch (all pointers DEVICE):
+ *   ctx_len, verify_len, block_size [n_req]   as in recg_batch; rewritten by recg_next_round()
+ *   verify_tokens [n_req, max_verify]         request r's y_0.. at r * max_verify (a fixed stride, not ragged)
+ *   page_table [n_req, page_table_stride]     fixed over the loop: row r must cover every position the request can
+ *                                             reach (a request whose next round would not fit stops drafting: its
+ *                                             block size becomes 0; if even one more token does not fit the status
+ *                                             word is set)
+ *   rows_hint                                 the expected number of rows per round, used to choose the projections'
+ *                                             tile configurations (0: the context's max_tokens)
+ * Correction branches are not available in this mode.  Because the row count of a round is only known on the device,
+ * every launch is sized for the context's max_tokens and max_requests, projections use whole tiles only, and
+ * recg_logits.n_rows reports max_tokens; the true counts are in the device arrays.  Lengths that break a capacity
+ * (negative, a request without rows, verify_len > max_verify, rows beyond the page-table row, more than max_tokens rows
+ * in total) set the device status word and turn the round into an empty one: recg_sync() then returns
+ * RECG_ERR_INTERNAL.  Not available with RECG_FLAG_SIMT_GEMM or RECG_FLAG_FOLD_NORM.
+ *
+ * recg_next_round() turns the finished round (the library's own verification buffers: call recg_verify with NULL
+ * output pointers or leave them out) into the next one, per request:
+ *   a = accept_len; the tokens y_1..y_a and the verifier's token t at row a are appended to the log;
+ *   ctx_len += a + 1;  if the continuation block is reusable (cont_hit): verify tokens = [t, d_1 .. d_{b-1}] (the drafted
+ *   block, whose first token only confirmed t), else [t];  block_size = next_block[r] (DEVICE, e.g. the output of
+ *   recg_policy_step; NULL keeps the block size).
+ *   planted_emitted (DEVICE [n_req] or NULL): synthetic acceptance for random-weight runs -- the round is taken to have
+ *   emitted min(planted_emitted[r], verify_len) tokens (at least 1), and its continuation block to be reusable exactly
+ *   when every draft was accepted.
+ * recg_round_log (DEVICE, caller-owned, any part may be NULL): tokens [n_req, max_tokens_per_request] with n_tokens
+ * [n_req] (initialise to 0); accept_len / block_size / verify_len (int32) and entropy_mean (float32) [max_rounds, n_req]
+ * receive row `round` (the caller's round counter): what the round accepted, the block size and verify length it ran
+ * with and its mean verifier entropy; n_rounds [1] receives round + 1.
+ */
+typedef struct {
+  int32_t n_req, max_verify, page_table_stride, rows_hint;
+  int32_t *ctx_len, *verify_len, *block_size, *verify_tokens;
+  const int32_t *page_table;
+  void *kv_pool;
+  int64_t kv_pool_pages;
+} recg_device_batch;
+typedef struct {
+  int32_t *tokens, *n_tokens;
+  int32_t max_tokens_per_request;
+  int32_t max_rounds;
+  int32_t *accept_len, *block_size, *verify_len, *n_rounds;
+  float *entropy_mean;
+} recg_round_log;
+recg_status recg_step_device(recg_ctx *ctx, const recg_device_batch *batch, recg_logits *logits);
+recg_status recg_next_round(recg_ctx *ctx, const recg_device_batch *batch, const int32_t *next_block,
+                            const int32_t *planted_emitted, const recg_round_log *log, int32_t round);
+
+/*
  * Per-row logit statistics with no allocation anywhere (the paper has no counterpart: this entry point
  * exists for callers that are not allowed to allocate device memory).
  *

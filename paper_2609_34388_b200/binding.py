@@ -73,6 +73,18 @@ class recg_policy_state(C.Structure):
     _fields_ = [("e1", C.c_void_p), ("e2", C.c_void_p), ("block_index", C.c_void_p), ("full", C.c_void_p)]
 
 
+class recg_device_batch(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("n_req", "max_verify", "page_table_stride", "rows_hint")] + \
+               [(n, C.c_void_p) for n in ("ctx_len", "verify_len", "block_size", "verify_tokens", "page_table", "kv_pool")] + \
+               [("kv_pool_pages", C.c_int64)]
+
+
+class recg_round_log(C.Structure):
+    _fields_ = [("tokens", C.c_void_p), ("n_tokens", C.c_void_p), ("max_tokens_per_request", C.c_int32), ("max_rounds", C.c_int32),
+                ("accept_len", C.c_void_p), ("block_size", C.c_void_p), ("verify_len", C.c_void_p), ("n_rounds", C.c_void_p),
+                ("entropy_mean", C.c_void_p)]
+
+
 _lib = None
 
 
@@ -107,13 +119,17 @@ def lib() -> C.CDLL:
         L.recg_policy_load.argtypes = [C.c_void_p, C.POINTER(recg_policy_table)]
         L.recg_policy_step.argtypes = [C.c_void_p, C.POINTER(recg_policy_state), C.c_void_p, C.c_void_p, C.c_void_p]
         L.recg_free.argtypes = [C.c_void_p]
+        L.recg_step_device.argtypes = [C.c_void_p, C.POINTER(recg_device_batch), C.POINTER(recg_logits)]
+        L.recg_next_round.argtypes = [C.c_void_p, C.POINTER(recg_device_batch), C.c_void_p, C.c_void_p, C.POINTER(recg_round_log),
+                                      C.c_int32]
         L.recg_debug_gemm_config.argtypes = [C.c_void_p, C.c_int32, C.c_int32]
         L.recg_debug_wait_timeout.argtypes = [C.c_void_p, C.c_int32]
         L.recg_debug_map_cache_selftest.argtypes = [C.c_int32, C.POINTER(C.c_int32)]
         L.recg_debug_map_cache_selftest.restype = C.c_int32
         for f in ("recg_init", "recg_step", "recg_verify", "recg_attention", "recg_kv_write", "recg_kv_read",
                   "recg_linear", "recg_debug_buffer", "recg_sync", "recg_free", "recg_timing_enable", "recg_timing_read",
-                  "recg_policy_load", "recg_policy_step", "recg_debug_gemm_config", "recg_debug_wait_timeout"):
+                  "recg_policy_load", "recg_policy_step", "recg_debug_gemm_config", "recg_debug_wait_timeout",
+                  "recg_step_device", "recg_next_round"):
             getattr(L, f).restype = C.c_int32
         _lib = L
     return _lib
@@ -123,7 +139,7 @@ EXPORTS = ("recg_kv_pool_bytes", "recg_init", "recg_step", "recg_verify", "recg_
            "recg_kv_read", "recg_linear", "recg_debug_buffer", "recg_sync", "recg_free", "recg_last_error",
            "recg_timing_enable", "recg_timing_read", "recg_row_stats_static", "recg_row_stats_static_error",
            "recg_policy_load", "recg_policy_step", "recg_debug_gemm_config", "recg_debug_wait_timeout",
-           "recg_debug_map_cache_selftest")
+           "recg_debug_map_cache_selftest", "recg_step_device", "recg_next_round")
 TIMING_CLASSES = ("layout", "rmsnorm", "gemm_qkv", "attention", "gemm_o", "gemm_gate_up", "gemm_down", "lm_head", "verify")
 
 
@@ -173,6 +189,41 @@ class Batch:
             self.rows = self.rows + self.n_corr * (1 + self.corr_block)
         self.n_tok = int(self.rows.sum())
         self.n_ver = int(self.verify_len.sum())
+
+
+class DeviceBatch:
+    """A recg_device_batch: the descriptor arrays as CUDA int32 tensors that recg_next_round rewrites in place."""
+
+    def __init__(self, ctx_len, verify_len, block_size, verify_tokens, max_verify: int, page_table, kv_pool, kv_pool_pages: int,
+                 rows_hint: int = 0):
+        """verify_tokens: per request a list of its y (padded here to max_verify)."""
+        self.n_req = len(ctx_len)
+        dev = kv_pool.device
+        i32 = lambda a: torch.as_tensor(np.asarray(a, dtype=np.int32), device=dev).contiguous()
+        self.ctx_len, self.verify_len, self.block_size = i32(ctx_len), i32(verify_len), i32(block_size)
+        vt = np.zeros((self.n_req, max_verify), dtype=np.int32)
+        for r, y in enumerate(verify_tokens):
+            vt[r, :len(y)] = y
+        self.verify_tokens = i32(vt)
+        self.page_table = i32(page_table)
+        self.kv_pool = kv_pool
+        self.c = recg_device_batch(self.n_req, max_verify, int(self.page_table.shape[1]), rows_hint, self.ctx_len.data_ptr(),
+                                   self.verify_len.data_ptr(), self.block_size.data_ptr(), self.verify_tokens.data_ptr(),
+                                   self.page_table.data_ptr(), kv_pool.data_ptr(), int(kv_pool_pages))
+
+
+class RoundLog:
+    """Device logs of a run of device-resident rounds."""
+
+    def __init__(self, n_req: int, max_rounds: int, max_tokens_per_request: int, device="cuda"):
+        z = lambda *shape: torch.zeros(shape, dtype=torch.int32, device=device)
+        self.tokens, self.n_tokens = z(n_req, max_tokens_per_request), z(n_req)
+        self.accept_len, self.block_size, self.verify_len = z(max_rounds, n_req), z(max_rounds, n_req), z(max_rounds, n_req)
+        self.n_rounds = z(1)
+        self.entropy_mean = torch.zeros((max_rounds, n_req), dtype=torch.float32, device=device)
+        self.c = recg_round_log(self.tokens.data_ptr(), self.n_tokens.data_ptr(), max_tokens_per_request, max_rounds,
+                                self.accept_len.data_ptr(), self.block_size.data_ptr(), self.verify_len.data_ptr(),
+                                self.n_rounds.data_ptr(), self.entropy_mean.data_ptr())
 
 
 class VerifyOut:
@@ -315,6 +366,22 @@ class Context:
         self._check(lib().recg_debug_buffer(self.h, which, C.byref(p), C.byref(dt), C.byref(r), C.byref(c)))
         return device_view(p.value, (r.value, c.value),
                            torch.bfloat16 if dt.value == DTYPE_BF16 else torch.float32).clone()
+
+    def recg_step_device(self, batch: "DeviceBatch"):
+        lg = recg_logits()
+        self._check(lib().recg_step_device(self.h, C.byref(batch.c), C.byref(lg)))
+        return lg
+
+    def recg_verify_device(self):
+        """Verification of the last recg_step_device into the library's own device buffers (nothing is copied)."""
+        out = recg_verify_out()
+        out.mem = MEM_DEVICE
+        self._check(lib().recg_verify(self.h, None, None, 0, C.byref(out)))
+
+    def recg_next_round(self, batch: "DeviceBatch", round_index: int, next_block: Optional[torch.Tensor] = None,
+                        planted_emitted: Optional[torch.Tensor] = None, log: Optional["RoundLog"] = None):
+        self._check(lib().recg_next_round(self.h, C.byref(batch.c), _ptr(next_block), _ptr(planted_emitted),
+                                          C.byref(log.c) if log is not None else None, int(round_index)))
 
     def recg_debug_gemm_config(self, tile: int, stream_k: bool):
         self._check(lib().recg_debug_gemm_config(self.h, int(tile), 1 if stream_k else 0))

@@ -583,9 +583,15 @@ __device__ __forceinline__ void row_epilogue(const EpiParams& ep, const Loader& 
 template <int BN, bool PAIR, bool NORM>
 __global__ void __launch_bounds__(kTcThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
-               const __grid_constant__ CUtensorMap map_out, const __grid_constant__ CUtensorMap map_xout, int M, int n_tiles_n,
-               int K, int up_row_offset, int dp_tiles, long long per, int thin, float* split_ws, int* split_counters,
-               EpiParams ep) {
+               const __grid_constant__ CUtensorMap map_out, const __grid_constant__ CUtensorMap map_xout, int M_cap, int n_tiles_n,
+               int K, int up_row_offset, int dp_tiles_in, long long per, int thin, float* split_ws, int* split_counters,
+               const int* __restrict__ m_dev, EpiParams ep_in) {
+  // Device-resident rounds: the row count comes from device memory (written by a kernel at least two launches back, so
+  // it may be read before this kernel waits for its predecessor); the tensor maps cover the capacity M_cap, rows
+  // between the count and the capacity hold stale data and are computed but never used, and all tiles are whole.
+  const int M = m_dev ? __ldg(m_dev) : M_cap;
+  EpiParams ep = ep_in;
+  ep.M = M;
   using Cfg = TcCfg<BN, PAIR, NORM>;
   constexpr int kRows = PAIR ? 2 * BM : BM;              // rows of a scheduling unit's tile
   constexpr int kSlotMul = PAIR ? 2 : 1;                 // the CTAs of a pair use separate slots and counters
@@ -639,6 +645,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n_tiles_m = (M + kRows - 1) / kRows;
   const int n_tiles = n_tiles_m * n_tiles_n;
+  const int dp_tiles = dp_tiles_in < 0 ? n_tiles : dp_tiles_in;
   const int KB = K / BK;
   const bool swiglu = ep.epi == EPI_SWIGLU;
   // schedule: the k-blocks of tiles [dp_tiles, n_tiles) as one line cut into equal ranges per CTA; then tiles
@@ -1057,6 +1064,10 @@ bool launch_bn_t(TcState* st, int idx, const GemmArgs& a, const EpiParams& ep, b
   int units = n_tiles < n_units ? n_tiles : n_units;
   int dp_tiles = n_tiles;       // whole tiles, strided
   long long per = 1;
+  if (a.m_dev) {                // the row count is on the device: whole tiles only, counted by the kernel
+    dp_tiles = -1;
+    stream_k = false;
+  }
   if (stream_k) {
     // all but the last one-to-two waves as whole tiles; the k-blocks of the remaining tile columns evenly over
     // teams of mt units (one per row tile)
@@ -1094,7 +1105,7 @@ bool launch_bn_t(TcState* st, int idx, const GemmArgs& a, const EpiParams& ep, b
   cfg.attrs = attr;
   cfg.numAttrs = n_attr;
   return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<BN, PAIR, NORM>, mx, mw, mo, mxo, a.M, n_tiles_n, a.K, a.N, dp_tiles, per, thin,
-                            st->split_ws, st->split_counters, ep) == cudaSuccess;
+                            st->split_ws, st->split_counters, a.m_dev, ep) == cudaSuccess;
 }
 
 }  // namespace
@@ -1216,7 +1227,9 @@ static bool launch_gemm_tc_impl(const GemmArgs& a, TcState* st, int* status, cud
   // whole tiles cost waves x k-blocks x (tensor time of one k-block at that width); the stream-K decomposition
   // spreads all k-blocks evenly over the SMs and pays a fixed hand-over for the cut tiles (park the partial,
   // fence, counter, reduction read).  Rotary tiles must hold whole heads.
-  const int mt = (a.M + BM - 1) / BM;
+  // (device-resident rounds: the configuration is chosen for the caller's hint of the row count, the launch covers the capacity)
+  const int Mc = (a.m_dev && a.m_hint > 0 && a.m_hint < a.M) ? a.m_hint : a.M;
+  const int mt = (Mc + BM - 1) / BM;
   const int KB = a.K / BK;
   int best_bn = 0;
   bool best_sk = false, best_pair = false;
@@ -1227,8 +1240,8 @@ static bool launch_gemm_tc_impl(const GemmArgs& a, TcState* st, int* status, cud
   constexpr int kConfigs = 5;
   const int bns[kConfigs] = {256, 128, 64, 256, 128};
   const double kb_tensor[kConfigs] = {0.44, 0.27, 0.22, 0.385, 0.205};
-  const bool pair_ok = a.M > BM && (swiglu ? a.N % 128 == 0 : a.N % 256 == 0) && !(a.epi == EPI_QKV_ROPE && 256 % a.head_dim);
-  const bool pair128_ok = a.M > BM && !swiglu && a.N % 128 == 0 && !(a.epi == EPI_QKV_ROPE && 128 % a.head_dim);
+  const bool pair_ok = Mc > BM && (swiglu ? a.N % 128 == 0 : a.N % 256 == 0) && !(a.epi == EPI_QKV_ROPE && 256 % a.head_dim);
+  const bool pair128_ok = Mc > BM && !swiglu && a.N % 128 == 0 && !(a.epi == EPI_QKV_ROPE && 128 % a.head_dim);
   for (int bi = 0; bi < kConfigs; ++bi) {
     const int bn = bns[bi];
     const bool pair = bi >= 3;
@@ -1236,7 +1249,7 @@ static bool launch_gemm_tc_impl(const GemmArgs& a, TcState* st, int* status, cud
     if (bi == 4 && !pair128_ok) continue;
     const int rows_tile = pair ? 2 * BM : BM;
     const int units = pair ? st->n_sm / 2 : st->n_sm;            // CTAs or clusters
-    const int mtc = (a.M + rows_tile - 1) / rows_tile;
+    const int mtc = (Mc + rows_tile - 1) / rows_tile;
     const int per = swiglu ? bn / 2 : bn;
     if (a.epi == EPI_QKV_ROPE && (bn < a.head_dim || a.N % bn)) continue;
     if (swiglu && (a.N % per)) continue;
@@ -1246,7 +1259,7 @@ static bool launch_gemm_tc_impl(const GemmArgs& a, TcState* st, int* status, cud
     // a k-block costs its tensor time, or the time one SM needs to stream its share of the weight bytes (the
     // CTAs that work on one weight tile at the same time share them through L2)
     const double kbt = fmax(kb_tensor[bi], (bn * 128.0 / mt) / 35e3);
-    const double rows = a.M < BM ? a.M : BM;
+    const double rows = Mc < BM ? Mc : BM;
     const double t_plain = (double)waves * KB * kbt;
     const int sk_units = mtc <= units ? (units / mtc) * mtc : 1;     // teams of mtc units
     const double t_sk = ((double)tiles * KB / sk_units + 1.0) * kbt + 3.0 + rows * bn * 4.0 * 2.5 / 16e3;

@@ -95,9 +95,10 @@ struct RoundLog {
   int* verify_len;
   int max_rounds;
   int* n_rounds;     // [1]
+  float* entropy_mean;   // [max_rounds][n_req]
 };
 void launch_next_round(const DeviceRound& dr, const BatchLayout& bl, const VerifyBuffers& vb, const int* next_block,
-                       const int* planted_emitted, const RoundLog& log, int* status, cudaStream_t st);
+                       const int* planted_emitted, const RoundLog& log, int round, int* status, cudaStream_t st);
 
 // (cos, sin) of pos * base^(-2i/d), angles evaluated in double: cs float2 [head_dim/2][T] (frequency-major).
 void launch_rope_table(const int* tok_pos, int n_tok, int head_dim, float rope_base, void* cs, cudaStream_t st,

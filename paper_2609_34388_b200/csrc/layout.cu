@@ -52,9 +52,10 @@ __global__ void __launch_bounds__(1024) layout_kernel(BatchLayout bl, int n_kv, 
   const int tid = threadIdx.x, nth = blockDim.x;
   griddep_launch();
   griddep_wait();   // the previous step's kernels may still be reading the arrays this kernel rewrites
+  const int n_tok = bl.dyn ? bl.dyn[0] : bl.n_tok;
 
   // ---- per-token arrays ----
-  for (int t = tid; t < bl.n_tok; t += nth) {
+  for (int t = tid; t < n_tok; t += nth) {
     const int r = upper_request(bl.cu_tok, C, t);
     const int j = t - bl.cu_tok[r];
     const int L = bl.ctx_len[r], v = bl.verify_len[r], b = bl.block_size[r];
@@ -253,10 +254,11 @@ __global__ void __launch_bounds__(1024) layout_kernel(BatchLayout bl, int n_kv, 
 __global__ void __launch_bounds__(256) embed_kernel(const int* __restrict__ tok_id, const __nv_bfloat16* __restrict__ embed,
                                                     float* __restrict__ h, int hidden, int vocab,
                                                     const __nv_bfloat16* __restrict__ gain, __nv_bfloat16* __restrict__ x,
-                                                    float* __restrict__ ss) {
+                                                    float* __restrict__ ss, const int* __restrict__ rows_dev) {
   griddep_launch();
   griddep_wait();
   const int t = blockIdx.x;
+  if (rows_dev && t >= rows_dev[0]) return;
   int id = tok_id[t];
   id = id < 0 ? 0 : (id >= vocab ? vocab - 1 : id);
   const __nv_bfloat162* src = reinterpret_cast<const __nv_bfloat162*>(embed + (size_t)id * hidden);
@@ -288,10 +290,12 @@ __global__ void __launch_bounds__(256) embed_kernel(const int* __restrict__ tok_
 // when it fits (hidden <= 256 threads x kRegVecs float4), otherwise it is read a second time.
 constexpr int kRegVecs = 8;
 __global__ void __launch_bounds__(256) rmsnorm_kernel(const float* __restrict__ h, const __nv_bfloat16* __restrict__ g,
-                                                      __nv_bfloat16* __restrict__ x, int hidden, float eps) {
+                                                      __nv_bfloat16* __restrict__ x, int hidden, float eps,
+                                                      const int* __restrict__ rows_dev) {
   griddep_launch();
   griddep_wait();
   const int row = blockIdx.x;
+  if (rows_dev && row >= rows_dev[0]) return;
   const int nvec = hidden / 4;
   const float4* src = reinterpret_cast<const float4*>(h + (size_t)row * hidden);
   const bool in_regs = nvec <= 256 * kRegVecs;
@@ -385,12 +389,13 @@ void launch_layout(const BatchLayout& bl, const Dims& dm, int tok_per_tile, int 
 void launch_embed(const BatchLayout& bl, const Dims& dm, const void* embed, float* h, const void* gain, void* x, float* ss,
                   cudaStream_t st) {
   launch_pdl(embed_kernel, dim3(bl.n_tok), dim3(256), 0, st, (const int*)bl.tok_id, static_cast<const __nv_bfloat16*>(embed), h,
-             dm.hidden, dm.vocab, static_cast<const __nv_bfloat16*>(gain), static_cast<__nv_bfloat16*>(x), ss);
+             dm.hidden, dm.vocab, static_cast<const __nv_bfloat16*>(gain), static_cast<__nv_bfloat16*>(x), ss, bl.dyn);
 }
 
-void launch_rmsnorm(const float* h, const void* gain, void* x, int rows, int hidden, float eps, cudaStream_t st) {
+void launch_rmsnorm(const float* h, const void* gain, void* x, int rows, int hidden, float eps, cudaStream_t st,
+                    const int* rows_dev) {
   launch_pdl(rmsnorm_kernel, dim3(rows), dim3(256), 0, st, h, static_cast<const __nv_bfloat16*>(gain),
-             static_cast<__nv_bfloat16*>(x), hidden, eps);
+             static_cast<__nv_bfloat16*>(x), hidden, eps, rows_dev);
 }
 
 void launch_kv_io(bool write, void* pool, int64_t n_pages, int layer, const Dims& dm, const int* page_row_dev, int pos0,
@@ -407,9 +412,10 @@ void launch_kv_io(bool write, void* pool, int64_t n_pages, int layer, const Dims
 namespace recg {
 namespace {
 __global__ void rope_table_kernel(const int* __restrict__ tok_pos, int n_tok, int half, double log_base,
-                                  float2* __restrict__ cs) {
+                                  float2* __restrict__ cs, const int* __restrict__ n_tok_dev) {
   griddep_launch();
   griddep_wait();
+  if (n_tok_dev) n_tok = n_tok_dev[0];     // (the grid was sized for the capacity)
   // frequency-major [half][n_tok]: the projection epilogue has one token per thread, so a warp reads 32 consecutive
   // tokens of one frequency in one 256-byte request
   const int idx = blockIdx.x * blockDim.x + threadIdx.x;
@@ -421,12 +427,13 @@ __global__ void rope_table_kernel(const int* __restrict__ tok_pos, int n_tok, in
 }
 }  // namespace
 
-void launch_rope_table(const int* tok_pos, int n_tok, int head_dim, float rope_base, void* cs, cudaStream_t st) {
+void launch_rope_table(const int* tok_pos, int n_tok, int head_dim, float rope_base, void* cs, cudaStream_t st,
+                       const int* n_tok_dev) {
   const int half = head_dim / 2;
   const int total = n_tok * half;
   if (total <= 0) return;
   launch_pdl(rope_table_kernel, dim3((total + 255) / 256), dim3(256), 0, st, tok_pos, n_tok, half,
-             log((double)rope_base), static_cast<float2*>(cs));
+             log((double)rope_base), static_cast<float2*>(cs), n_tok_dev);
 }
 }  // namespace recg
 
@@ -464,5 +471,147 @@ void launch_guard_check(const void* base, const size_t* offs_dev, int n, int* st
 }
 void launch_wait_timeout(uint32_t max_polls, int* status, cudaStream_t st) {
   wait_timeout_kernel<<<1, 1, 0, st>>>(max_polls, status);
+}
+}  // namespace recg
+
+// ---------------------------------------------------------------------------------------------------
+// Device-resident rounds (Sec. 5.2): descriptor of a round from device arrays, and the step from one round to the next.
+// ---------------------------------------------------------------------------------------------------
+namespace recg {
+namespace {
+
+// One CTA.  Writes the packed descriptor [ctx_len | verify_len | block_size | corr (all zero: no correction branches in
+// this mode) | cu_tok | cu_ver | verify_tokens (ragged)] and {n_tok, n_ver}.  A request whose lengths break a capacity
+// (negative, no rows, more verify tokens than max_verify, rows beyond its page-table row, or a total beyond max_tokens)
+// flags the status word and the round becomes empty (n_tok = 0): later kernels then do nothing.
+__global__ void __launch_bounds__(256) pack_device_kernel(DeviceRound dr, int* __restrict__ desc, int* __restrict__ dyn,
+                                                          int* status) {
+  griddep_launch();
+  griddep_wait();
+  const int C = dr.n_req;
+  int* ctx = desc;
+  int* ver = desc + C;
+  int* blk = desc + 2 * C;
+  int* corr = desc + 3 * C;
+  int* cu_tok = desc + 9 * C;
+  int* cu_ver = cu_tok + (C + 1);
+  int* vt = cu_ver + (C + 1);
+  __shared__ int s_bad, s_tok, s_ver;
+  if (threadIdx.x == 0) s_bad = 0;
+  __syncthreads();
+  for (int r = threadIdx.x; r < C; r += blockDim.x) {
+    const int L = dr.ctx_len[r], v = dr.verify_len[r], b = dr.block_size[r];
+    if (L < 0 || v < 0 || b < 0 || v + b < 1 || v > dr.max_verify ||
+        ((long long)L + v + b + kPageSize - 1) / kPageSize > dr.pt_stride)
+      s_bad = 1;
+    ctx[r] = L;
+    ver[r] = v;
+    blk[r] = b;
+    for (int k = 0; k < 6; ++k) corr[6 * r + k] = 0;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int t = 0, tv = 0;
+    cu_tok[0] = cu_ver[0] = 0;
+    for (int r = 0; r < C; ++r) {
+      t += ver[r] + blk[r];
+      tv += ver[r];
+      if (t > dr.max_tokens || t < 0) {
+        s_bad = 1;
+        t = tv = 0;
+      }
+      cu_tok[r + 1] = t;
+      cu_ver[r + 1] = tv;
+    }
+    if (s_bad) {
+      set_status(status, DEV_BAD_INDEX);
+      t = tv = 0;
+      for (int r = 0; r <= C; ++r) cu_tok[r] = cu_ver[r] = 0;
+    }
+    s_tok = t;
+    s_ver = tv;
+    dyn[0] = t;
+    dyn[1] = tv;
+  }
+  __syncthreads();
+  if (s_tok == 0) return;
+  for (int r = threadIdx.x; r < C; r += blockDim.x)
+    for (int j = 0; j < ver[r]; ++j) vt[cu_ver[r] + j] = dr.verify_tokens[(size_t)r * dr.max_verify + j];
+}
+
+// One thread per request: the bookkeeping between two rounds (Sec. 3.1, 5.1) from the verification results that are
+// still on the device.  planted_emitted (may be null): synthetic acceptance -- the round is taken to have emitted
+// min(planted_emitted[r], v) tokens, and its continuation block to be reusable exactly when all drafts were accepted.
+__global__ void next_round_kernel(DeviceRound dr, BatchLayout bl, VerifyBuffers vb, const int* __restrict__ next_block,
+                                  const int* __restrict__ planted_emitted, RoundLog log, int round, int* status) {
+  griddep_launch();
+  griddep_wait();
+  const int r = blockIdx.x * blockDim.x + threadIdx.x;
+  if (r < dr.n_req) {
+    const int L = bl.ctx_len[r], v = bl.verify_len[r], b = bl.block_size[r];
+    const int t0 = bl.cu_tok[r], tv0 = bl.cu_ver[r];
+    const bool ran = bl.cu_tok[dr.n_req] > 0;       // an empty round (a capacity was broken) changes nothing
+    int a = 0, emitted = 0, cont = 0;
+    if (ran && v > 0) {
+      a = vb.accept_len[r];
+      cont = vb.cont_hit[r];
+      if (planted_emitted) {
+        const int e = planted_emitted[r] < 1 ? 1 : (planted_emitted[r] > v ? v : planted_emitted[r]);
+        a = e - 1;
+        cont = (b > 0 && a == v - 1) ? 1 : 0;
+      }
+      emitted = a + 1;
+    }
+    if (log.accept_len && round < log.max_rounds) {
+      log.accept_len[(size_t)round * dr.n_req + r] = a;
+      log.block_size[(size_t)round * dr.n_req + r] = b;
+      log.verify_len[(size_t)round * dr.n_req + r] = v;
+      if (log.entropy_mean) log.entropy_mean[(size_t)round * dr.n_req + r] = (ran && v > 0) ? vb.entropy_mean[r] : 0.f;
+    }
+    if (ran && v > 0) {
+      // emitted tokens: the accepted drafts y_1 .. y_a, then the verifier's token at row a
+      const int last = vb.top1[t0 + a];
+      if (log.tokens) {
+        int n = log.n_tokens[r];
+        for (int i = 1; i <= a && n < log.max_out; ++i) log.tokens[(size_t)r * log.max_out + n++] = bl.verify_tokens[tv0 + i];
+        if (n < log.max_out) log.tokens[(size_t)r * log.max_out + n++] = last;
+        log.n_tokens[r] = n;
+      }
+      int nb = next_block ? next_block[r] : b;
+      int nv = 1;
+      int* y = dr.verify_tokens + (size_t)r * dr.max_verify;
+      y[0] = last;
+      if (cont) {                      // the drafted block becomes the next verify tokens (its first token only
+        nv = b < dr.max_verify ? b : dr.max_verify;   // confirmed the one just emitted)
+        const int tb0 = t0 - tv0;      // offset of the request's draft rows in next_draft
+        for (int j = 1; j < nv; ++j) y[j] = vb.next_draft[tb0 + j];
+      }
+      const int nL = L + emitted;
+      // the next round must fit the page-table row; a request that has run out of room stops growing
+      if (((long long)nL + nv + nb + kPageSize - 1) / kPageSize > dr.pt_stride) {
+        nb = 0;
+        nv = 1;
+        if (((long long)nL + 1 + kPageSize - 1) / kPageSize > dr.pt_stride) set_status(status, DEV_BAD_INDEX);
+      }
+      dr.ctx_len[r] = nL;
+      dr.verify_len[r] = nv;
+      dr.block_size[r] = nb;
+    } else if (ran && next_block) {
+      dr.block_size[r] = next_block[r];
+    }
+  }
+  if (r == 0 && log.n_rounds) log.n_rounds[0] = round + 1;     // rounds logged so far
+}
+
+}  // namespace
+
+void launch_pack_device(const DeviceRound& dr, int* desc, int* dyn, int* status, cudaStream_t st) {
+  launch_pdl(pack_device_kernel, dim3(1), dim3(256), 0, st, dr, desc, dyn, status);
+}
+
+void launch_next_round(const DeviceRound& dr, const BatchLayout& bl, const VerifyBuffers& vb, const int* next_block,
+                       const int* planted_emitted, const RoundLog& log, int round, int* status, cudaStream_t st) {
+  launch_pdl(next_round_kernel, dim3((dr.n_req + 127) / 128), dim3(128), 0, st, dr, bl, vb, next_block, planted_emitted, log,
+             round, status);
 }
 }  // namespace recg

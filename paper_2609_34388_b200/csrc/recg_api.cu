@@ -72,6 +72,7 @@ struct recg_ctx {
   size_t vout_off = 0, vout_bytes = 0;   // the verify outputs are one contiguous region of the arena ...
   uint8_t* h_vout = nullptr;             // ... mirrored by one pinned host buffer: a single copy brings all results back
   int* d_status = nullptr;
+  int* d_dyn = nullptr;          // device-resident rounds: {n_tok, n_ver} of the round laid out last
   int* d_page_row = nullptr;
   size_t* d_guards = nullptr;    // RECG_FLAG_DEBUG_CHECKS: offsets of the guard bands, on the device
   int n_guards = 0;
@@ -141,6 +142,7 @@ size_t carve(recg_ctx* c, DeviceArena& A) {
   bl.cta_off = A.take<int>(4 * (c->target_items + 1));
   bl.counts = A.take<int>(4);
   c->d_status = A.take<int>(1);
+  c->d_dyn = A.take<int>(4);
   c->d_page_row = A.take<int>(Pm);
   c->d_policy = A.take<int>(8 + 8 + 64 + RECG_POLICY_MAX_BLOCKS * RECG_POLICY_MAX_BINS * RECG_POLICY_MAX_BLOCKS * 2);
   c->rope_cs = A.take<float2>(Tm * (d.head_dim / 2));
@@ -296,6 +298,7 @@ recg_status pack_batch(recg_ctx* ctx, const recg_batch* b, bool need_pages, bool
   }
   BatchLayout& bl = ctx->bl;
   int* d = ctx->d_desc;
+  bl.dyn = nullptr;
   bl.n_req = C;
   bl.n_tok = (int)T;
   bl.n_ver = (int)Tv;
@@ -335,8 +338,8 @@ recg_status run_gemm(recg_ctx* ctx, const GemmArgs& a, int* ss_slots_out = nullp
   bool done = false;
   if (!(ctx->cfg.flags & RECG_FLAG_SIMT_GEMM)) done = launch_gemm_tc(a, ctx->tc_state, ctx->d_status, ctx->stream, ss_slots_out);
   if (!done) {
-    // the folded RMSNorm exists on the tcgen05 path only: a projection that takes part in it must not fall back
-    if (a.ss_in || a.epi == EPI_RESIDUAL_NORM) {
+    // the folded RMSNorm and device-side row counts exist on the tcgen05 path only: such a projection must not fall back
+    if (a.ss_in || a.epi == EPI_RESIDUAL_NORM || a.m_dev) {
       cudaGetLastError();
       return fail(ctx, RECG_ERR_INTERNAL, "projection: the tcgen05 kernel refused a shape of the step");
     }
@@ -499,18 +502,15 @@ recg_status recg_sync(recg_ctx* ctx) {
   return RECG_OK;
 }
 
-recg_status recg_step(recg_ctx* ctx, const recg_batch* batch, recg_logits* logits) {
-  if (!ctx) return RECG_ERR_INVALID_ARG;
-  if (!ctx->has_weights) return fail(ctx, RECG_ERR_INVALID_ARG, "recg_step: the context was created without weights");
-  ctx->logits_valid = false;
-  ctx->mark(-1);
-  recg_status s = upload_and_layout(ctx, batch, true);
-  if (s != RECG_OK) return s;
+// The forward over the batch laid out last (ctx->bl): embedding, the layers, final norm and LM head.  m_hint: device-
+// resident rounds only, the row count the projections' tile configurations are chosen for.
+static recg_status run_forward(recg_ctx* ctx, void* kv_pool, int64_t kv_pool_pages, int m_hint, recg_logits* logits) {
+  recg_status s = RECG_OK;
   const Dims& d = ctx->dm;
   const BatchLayout& bl = ctx->bl;
   const int T = bl.n_tok;
   cudaStream_t st = ctx->stream;
-  launch_rope_table(bl.tok_pos, T, d.head_dim, d.rope_base, ctx->rope_cs, st);
+  launch_rope_table(bl.tok_pos, T, d.head_dim, d.rope_base, ctx->rope_cs, st, bl.dyn);
   // RMSNorm runs as a kernel of its own, or (RECG_FLAG_FOLD_NORM, tcgen05 path only) folded into the projections:
   // whoever writes the residual stream also writes x = bf16(h * gain of the next norm) and partial sums of squares per
   // row, and the projection that reads x scales its accumulator rows by the row's rstd.
@@ -525,28 +525,32 @@ recg_status recg_step(recg_ctx* ctx, const recg_batch* batch, recg_logits* logit
   auto normed = [&](GemmArgs& g) {       // g reads the normalised residual stream
     g.x = ctx->x;
     g.K = d.hidden;
+    g.m_dev = bl.dyn;
+    g.m_hint = m_hint;
     if (fold) { g.ss_in = ctx->ss; g.ss_slots = slots; g.ss_stride = Tm; g.norm_eps = d.rms_eps; }
   };
   auto residual = [&](GemmArgs& g, const void* next_gain) {   // g adds into the residual stream
     g.out = ctx->h;
     g.N = d.hidden;
+    g.m_dev = bl.dyn;
+    g.m_hint = m_hint;
     g.epi = fold ? EPI_RESIDUAL_NORM : EPI_RESIDUAL;
     if (fold) { g.x_out = ctx->x; g.gain = next_gain; g.ss_out = ctx->ss; g.ss_stride = Tm; }
   };
   for (int l = 0; l < d.n_layers; ++l) {
     if (!fold) {
-      launch_rmsnorm(ctx->h, ctx->attn_norm[l], ctx->x, T, d.hidden, d.rms_eps, st);
+      launch_rmsnorm(ctx->h, ctx->attn_norm[l], ctx->x, T, d.hidden, d.rms_eps, st, bl.dyn);
       ctx->mark(1, 1);
     }
     GemmArgs a{};
     normed(a);
     a.w = ctx->wqkv[l]; a.out = ctx->q;
     a.M = T; a.N = (d.n_q + 2 * d.n_kv) * d.head_dim; a.epi = EPI_QKV_ROPE;
-    a.tok_pos = bl.tok_pos; a.tok_slot = bl.tok_slot; a.kv_pool = batch->kv_pool; a.n_pages = batch->kv_pool_pages;
+    a.tok_pos = bl.tok_pos; a.tok_slot = bl.tok_slot; a.kv_pool = kv_pool; a.n_pages = kv_pool_pages;
     a.layer = l; a.n_q = d.n_q; a.n_kv = d.n_kv; a.head_dim = d.head_dim; a.rope_cs = ctx->rope_cs;
     if ((s = run_gemm(ctx, a)) != RECG_OK) return s;
     ctx->mark(2, 1);
-    launch_attention(bl, d, l, ctx->q, ctx->o, batch->kv_pool, batch->kv_pool_pages, ctx->part_o, ctx->part_ml,
+    launch_attention(bl, d, l, ctx->q, ctx->o, kv_pool, kv_pool_pages, ctx->part_o, ctx->part_ml,
                      ctx->tok_per_tile, ctx->n_sm, ctx->d_status, st, !(ctx->cfg.flags & RECG_FLAG_SIMT_ATTENTION));
     CU(cudaGetLastError());
     ctx->mark(3, 2);
@@ -556,7 +560,7 @@ recg_status recg_step(recg_ctx* ctx, const recg_batch* batch, recg_logits* logit
     if ((s = run_gemm(ctx, b, &slots)) != RECG_OK) return s;
     ctx->mark(4, 1);
     if (!fold) {
-      launch_rmsnorm(ctx->h, ctx->ffn_norm[l], ctx->x, T, d.hidden, d.rms_eps, st);
+      launch_rmsnorm(ctx->h, ctx->ffn_norm[l], ctx->x, T, d.hidden, d.rms_eps, st, bl.dyn);
       ctx->mark(1, 1);
     }
     GemmArgs c{};
@@ -571,7 +575,7 @@ recg_status recg_step(recg_ctx* ctx, const recg_batch* batch, recg_logits* logit
     ctx->mark(6, 1);
   }
   if (!fold) {
-    launch_rmsnorm(ctx->h, ctx->final_norm, ctx->x, T, d.hidden, d.rms_eps, st);
+    launch_rmsnorm(ctx->h, ctx->final_norm, ctx->x, T, d.hidden, d.rms_eps, st, bl.dyn);
     ctx->mark(1, 1);
   }
   const bool lbf = ctx->cfg.flags & RECG_FLAG_LOGITS_BF16;
@@ -588,6 +592,106 @@ recg_status recg_step(recg_ctx* ctx, const recg_batch* batch, recg_logits* logit
     logits->n_rows = T;
     logits->vocab = d.vocab;
   }
+  return RECG_OK;
+}
+
+recg_status recg_step(recg_ctx* ctx, const recg_batch* batch, recg_logits* logits) {
+  if (!ctx) return RECG_ERR_INVALID_ARG;
+  if (!ctx->has_weights) return fail(ctx, RECG_ERR_INVALID_ARG, "recg_step: the context was created without weights");
+  ctx->logits_valid = false;
+  ctx->mark(-1);
+  recg_status s = upload_and_layout(ctx, batch, true);
+  if (s != RECG_OK) return s;
+  return run_forward(ctx, batch->kv_pool, batch->kv_pool_pages, 0, logits);
+}
+
+// ---- device-resident rounds ----
+static recg_status check_device_batch(recg_ctx* ctx, const recg_device_batch* b, const char* who) {
+  if (!b || b->n_req <= 0 || !b->ctx_len || !b->verify_len || !b->block_size || !b->verify_tokens || !b->page_table ||
+      !b->kv_pool || b->kv_pool_pages <= 0)
+    return fail(ctx, RECG_ERR_INVALID_ARG, std::string(who) + ": null array, n_req <= 0 or no KV pool");
+  if (b->n_req > ctx->cfg.max_requests) return fail(ctx, RECG_ERR_CAPACITY, std::string(who) + ": n_req exceeds max_requests");
+  if (b->max_verify < 1 || b->max_verify > ctx->cfg.max_tokens)
+    return fail(ctx, RECG_ERR_INVALID_ARG, std::string(who) + ": max_verify must be 1 .. max_tokens");
+  if (b->page_table_stride <= 0 || b->page_table_stride > ctx->cfg.max_pages_per_request)
+    return fail(ctx, RECG_ERR_CAPACITY, std::string(who) + ": page_table_stride exceeds max_pages_per_request");
+  return RECG_OK;
+}
+
+static DeviceRound device_round(const recg_ctx* ctx, const recg_device_batch* b) {
+  DeviceRound dr;
+  dr.n_req = b->n_req;
+  dr.max_verify = b->max_verify;
+  dr.pt_stride = b->page_table_stride;
+  dr.max_tokens = ctx->cfg.max_tokens;
+  dr.ctx_len = b->ctx_len;
+  dr.verify_len = b->verify_len;
+  dr.block_size = b->block_size;
+  dr.verify_tokens = b->verify_tokens;
+  return dr;
+}
+
+recg_status recg_step_device(recg_ctx* ctx, const recg_device_batch* b, recg_logits* logits) {
+  if (!ctx) return RECG_ERR_INVALID_ARG;
+  if (!ctx->has_weights) return fail(ctx, RECG_ERR_INVALID_ARG, "recg_step_device: the context was created without weights");
+  if (ctx->cfg.flags & (RECG_FLAG_SIMT_GEMM | RECG_FLAG_FOLD_NORM))
+    return fail(ctx, RECG_ERR_INVALID_ARG, "recg_step_device: not available with RECG_FLAG_SIMT_GEMM or RECG_FLAG_FOLD_NORM");
+  recg_status s = check_device_batch(ctx, b, "recg_step_device");
+  if (s != RECG_OK) return s;
+  ctx->logits_valid = false;
+  ctx->layout_valid = false;
+  ctx->mark(-1);
+  const int C = b->n_req;
+  BatchLayout& bl = ctx->bl;
+  int* d = ctx->d_desc;
+  bl.dyn = ctx->d_dyn;
+  bl.n_req = C;
+  bl.n_tok = ctx->cfg.max_tokens;      // capacities: the true counts are in dyn
+  bl.n_ver = ctx->cfg.max_tokens;
+  bl.pt_stride = b->page_table_stride;
+  bl.ctx_len = d;
+  bl.verify_len = d + C;
+  bl.block_size = d + 2 * C;
+  bl.corr = d + 3 * C;
+  bl.cu_tok = d + 9 * C;
+  bl.cu_ver = bl.cu_tok + (C + 1);
+  bl.verify_tokens = bl.cu_ver + (C + 1);
+  bl.page_table = b->page_table;
+  bl.risk_delta = 0.5f;
+  launch_pack_device(device_round(ctx, b), ctx->d_desc, ctx->d_dyn, ctx->d_status, ctx->stream);
+  launch_layout(bl, ctx->dm, ctx->tok_per_tile, ctx->target_items, b->kv_pool_pages, ctx->d_status, ctx->stream);
+  CU(cudaGetLastError());
+  ctx->layout_valid = true;
+  ctx->layout_has_pages = true;
+  ctx->last_pool = b->kv_pool;
+  ctx->last_pool_pages = b->kv_pool_pages;
+  return run_forward(ctx, b->kv_pool, b->kv_pool_pages, b->rows_hint, logits);
+}
+
+recg_status recg_next_round(recg_ctx* ctx, const recg_device_batch* b, const int32_t* next_block, const int32_t* planted_emitted,
+                            const recg_round_log* log, int32_t round) {
+  if (!ctx) return RECG_ERR_INVALID_ARG;
+  recg_status s = check_device_batch(ctx, b, "recg_next_round");
+  if (s != RECG_OK) return s;
+  if (!ctx->layout_valid || !ctx->bl.dyn || ctx->bl.n_req != b->n_req)
+    return fail(ctx, RECG_ERR_INVALID_ARG, "recg_next_round: no recg_step_device + recg_verify of this batch before");
+  RoundLog lg{};
+  if (log) {
+    if (round < 0 || (log->accept_len && (!log->block_size || !log->verify_len || log->max_rounds <= 0)) ||
+        (log->tokens && (!log->n_tokens || log->max_tokens_per_request <= 0)))
+      return fail(ctx, RECG_ERR_INVALID_ARG, "recg_next_round: inconsistent log arrays");
+    lg.tokens = log->tokens;
+    lg.max_out = log->max_tokens_per_request;
+    lg.n_tokens = log->n_tokens;
+    lg.accept_len = log->accept_len;
+    lg.block_size = log->block_size;
+    lg.verify_len = log->verify_len;
+    lg.max_rounds = log->max_rounds;
+    lg.n_rounds = log->n_rounds;
+    lg.entropy_mean = log->entropy_mean;
+  }
+  launch_next_round(device_round(ctx, b), ctx->bl, ctx->vws, next_block, planted_emitted, lg, round, ctx->d_status, ctx->stream);
+  CU(cudaGetLastError());
   return RECG_OK;
 }
 
@@ -616,6 +720,8 @@ recg_status recg_verify(recg_ctx* ctx, const recg_batch* batch, const void* logi
   const BatchLayout& bl = ctx->bl;
   VerifyBuffers vb = ctx->vws;
   const bool dev = out->mem == RECG_MEM_DEVICE;
+  if (bl.dyn && !dev)
+    return fail(ctx, RECG_ERR_INVALID_ARG, "recg_verify: after recg_step_device the outputs stay on the device (RECG_MEM_DEVICE)");
   if (dev) {
 #define PICK(f) if (out->f) vb.f = out->f
     PICK(accept_len); PICK(n_emitted); PICK(emitted); PICK(new_ctx_len); PICK(slot_state); PICK(freed_pages);

@@ -89,11 +89,13 @@ template <> struct Vec<float> {
 template <typename T>
 __global__ void __launch_bounds__(kVerifyThreads) verify_partial_kernel(const T* __restrict__ logits, int vocab,
                                                                         int chunk_len, int chunks_per_row,
-                                                                        RowPartial* __restrict__ partials) {
+                                                                        RowPartial* __restrict__ partials,
+                                                                        const int* __restrict__ rows_dev) {
   constexpr int N = Vec<T>::N;
   griddep_launch();
   griddep_wait();
   const int row = blockIdx.x / chunks_per_row, chunk = blockIdx.x - row * chunks_per_row;
+  if (rows_dev && row >= rows_dev[0]) return;      // (the grid was sized for the capacity)
   const T* base = logits + (size_t)row * vocab;
   const int c0 = chunk * chunk_len;
   const int c1 = min(vocab, c0 + chunk_len);
@@ -326,10 +328,10 @@ void launch_verify(const BatchLayout& bl, const void* logits, int logits_dtype, 
   dim3 grid((unsigned)chunks * (unsigned)rows);
   if (logits_dtype == 0)
     launch_pdl(verify_partial_kernel<__nv_bfloat16>, grid, dim3(kVerifyThreads), 0, st,
-               static_cast<const __nv_bfloat16*>(logits), vocab, chunk_len, chunks, partials);
+               static_cast<const __nv_bfloat16*>(logits), vocab, chunk_len, chunks, partials, bl.dyn);
   else
     launch_pdl(verify_partial_kernel<float>, grid, dim3(kVerifyThreads), 0, st, static_cast<const float*>(logits), vocab,
-               chunk_len, chunks, partials);
+               chunk_len, chunks, partials, bl.dyn);
   launch_pdl(verify_finalize_kernel, dim3(bl.n_req), dim3(128), 0, st, bl, (const RowPartial*)partials, chunks, vb);
 }
 
@@ -472,10 +474,10 @@ extern "C" recg_status recg_row_stats_static(const void* logits, int32_t logits_
   dim3 grid((unsigned)chunks * (unsigned)rows);
   if (logits_dtype == RECG_DTYPE_BF16)
     verify_partial_kernel<__nv_bfloat16>
-        <<<grid, kVerifyThreads, 0, st>>>(static_cast<const __nv_bfloat16*>(logits), vocab, chunk_len, chunks, scratch);
+        <<<grid, kVerifyThreads, 0, st>>>(static_cast<const __nv_bfloat16*>(logits), vocab, chunk_len, chunks, scratch, nullptr);
   else
     verify_partial_kernel<float><<<grid, kVerifyThreads, 0, st>>>(static_cast<const float*>(logits), vocab, chunk_len,
-                                                                  chunks, scratch);
+                                                                  chunks, scratch, nullptr);
   cudaError_t e = cudaGetLastError();   // nothing reads the scratch unless the scan was launched
   if (e != cudaSuccess) return fail(RECG_ERR_CUDA, std::string("recg_row_stats_static: launch: ") + cudaGetErrorString(e));
   row_stats_finalize_kernel<<<(rows + 127) / 128, 128, 0, st>>>(scratch, rows, chunks, top1, top2, p1, p2, entropy);

@@ -286,3 +286,27 @@ def policy_table(blocks=(8, 16, 32), n_bins: int = 12, rho_cost=(0.9, 1.5, 2.6),
                     value[j, k, jp, f] = (1.0 - pk ** B) / (1.0 - pk) + 0.01 * rng.standard_normal()
     return {"blocks": np.asarray(blocks, dtype=np.int32), "s_edges": edges, "value": value,
             "cost": np.asarray(rho_cost, dtype=np.float32)}
+
+
+# Transition percentages between acceptance intervals [1,8], (8,16], (16,32] of adjacent rounds at block size 32, as
+# printed in the paper's transition table (Sec. 4.2).  Random-init weights accept almost nothing, so multi-round
+# workloads draw their acceptance lengths from this chain: the interval follows the table, the length is uniform over
+# the interval's integers (the paper prints nothing about the distribution inside an interval).
+ACCEPT_INTERVALS = ((1, 8), (9, 16), (17, 32))
+ACCEPT_TRANSITIONS = ((70.30, 18.11, 11.60), (58.39, 22.42, 19.19), (20.83, 12.51, 66.66))
+
+
+def acceptance_chain_lengths(n_rounds: int, n_req: int, seed: int = 4) -> np.ndarray:
+    """Emitted tokens per round and request, int32 [n_rounds, n_req]: one independent chain per request, started from
+    a state drawn uniformly."""
+    rng = np.random.default_rng(seed)
+    P = np.asarray(ACCEPT_TRANSITIONS, dtype=np.float64)
+    P = P / P.sum(axis=1, keepdims=True)
+    out = np.zeros((n_rounds, n_req), dtype=np.int32)
+    for r in range(n_req):
+        s = int(rng.integers(0, 3))
+        for t in range(n_rounds):
+            lo, hi = ACCEPT_INTERVALS[s]
+            out[t, r] = rng.integers(lo, hi + 1)
+            s = int(rng.choice(3, p=P[s]))
+    return out

@@ -38,15 +38,19 @@ def test_struct_sizes_match_header_layout(tmp_path):
     import subprocess
     src = tmp_path / "sizes.c"
     src.write_text('#include <stdio.h>\n#include <stddef.h>\n#include "recg.h"\n'
-                   'int main(void) { printf("%zu %zu %zu %zu %zu %zu %zu\\n", sizeof(recg_config), sizeof(recg_batch), '
+                   'int main(void) { printf("%zu %zu %zu %zu %zu %zu %zu %zu %zu %zu %zu\\n", sizeof(recg_config), sizeof(recg_batch), '
                    'sizeof(recg_verify_out), offsetof(recg_batch, n_corr), offsetof(recg_batch, risk_delta), '
-                   'offsetof(recg_verify_out, corr_hit), offsetof(recg_verify_out, freed_page_ids)); return 0; }\n')
+                   'offsetof(recg_verify_out, corr_hit), offsetof(recg_verify_out, freed_page_ids), sizeof(recg_device_batch), '
+                   'offsetof(recg_device_batch, kv_pool_pages), sizeof(recg_round_log), offsetof(recg_round_log, entropy_mean)); '
+                   'return 0; }\n')
     exe = tmp_path / "sizes"
     subprocess.run(["gcc", "-I", os.path.join(ROOT, "include"), str(src), "-o", str(exe)], check=True)
     got = [int(t) for t in subprocess.run([str(exe)], check=True, capture_output=True, text=True).stdout.split()]
     want = [C.sizeof(binding.recg_config), C.sizeof(binding.recg_batch), C.sizeof(binding.recg_verify_out),
             binding.recg_batch.n_corr.offset, binding.recg_batch.risk_delta.offset,
-            binding.recg_verify_out.corr_hit.offset, binding.recg_verify_out.freed_page_ids.offset]
+            binding.recg_verify_out.corr_hit.offset, binding.recg_verify_out.freed_page_ids.offset,
+            C.sizeof(binding.recg_device_batch), binding.recg_device_batch.kv_pool_pages.offset,
+            C.sizeof(binding.recg_round_log), binding.recg_round_log.entropy_mean.offset]
     assert got == want
 
 

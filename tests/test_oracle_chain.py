@@ -119,3 +119,19 @@ def test_planted_rounds_lengths():
     assert all(tr[i + 1][0] == tr[i][0] + tr[i][4] for i in range(4))
     # no block: nothing to reuse
     assert orc.planted_rounds(10, 4, [0, 0], [4, 4]) == [(10, 4, 0, 3, 4, False), (14, 1, 0, 0, 1, False)]
+
+
+def test_workload_generator_draws_from_the_same_chain():
+    """The benchmark's input generator (synth.acceptance_chain_lengths) has its own copy of the table: its transition
+    counts over a long run must match the oracle's matrix, and its lengths must stay inside the intervals."""
+    assert synth.ACCEPT_TRANSITIONS == orc.TABLE1_PERCENT and synth.ACCEPT_INTERVALS == orc.TABLE1_INTERVALS
+    L = synth.acceptance_chain_lengths(60000, 2, seed=8)
+    assert L.min() == 1 and L.max() == 32
+    P = orc.chain_matrix()
+    for r in range(2):
+        states = np.digitize(L[:, r], [9, 17])
+        counts = np.zeros((3, 3))
+        np.add.at(counts, (states[:-1], states[1:]), 1)
+        emp = counts / counts.sum(axis=1, keepdims=True)
+        sigma = np.sqrt(P * (1 - P) / counts.sum(axis=1, keepdims=True))
+        assert np.all(np.abs(emp - P) < 4.5 * sigma)
