@@ -56,6 +56,11 @@ enum {
                                 row's rstd.  Same results within bf16 rounding (x is rounded before the division instead
                                 of after it); measured 3 % slower than the separate kernel, which hides behind the next
                                 projection's weight prefetch, hence off by default                            */
+  RECG_FLAG_CHAIN = 32,      /* steps of at most 128 rows (low concurrency): run the projections between two attention
+                                calls (output projection, gate|up, down, the next layer's QKV projection or the LM head)
+                                as ONE persistent kernel with grid-wide barriers, so that the weight stream does not stop
+                                at kernel boundaries; implies the folded RMSNorm.  head_dim 128 only; larger steps and
+                                captured streams take the ordinary path                                       */
   RECG_FLAG_DEBUG_CHECKS = 8 /* guard bands behind every workspace region, checked by recg_sync() (RECG_ERR_INTERNAL
                                 if a kernel wrote past the end of one), and a host check that no page which receives
                                 new rows is named by two requests (RECG_ERR_INVALID_ARG)          */

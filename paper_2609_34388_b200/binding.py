@@ -19,7 +19,7 @@ LIB_PATH = os.path.join(_HERE, "librecg.so")
 RECG_OK = 0
 DTYPE_BF16, DTYPE_F32 = 0, 1
 MEM_DEVICE, MEM_HOST = 0, 1
-FLAG_LOGITS_BF16, FLAG_SIMT_GEMM, FLAG_SIMT_ATTENTION, FLAG_DEBUG_CHECKS, FLAG_FOLD_NORM = 1, 2, 4, 8, 16
+FLAG_LOGITS_BF16, FLAG_SIMT_GEMM, FLAG_SIMT_ATTENTION, FLAG_DEBUG_CHECKS, FLAG_FOLD_NORM, FLAG_CHAIN = 1, 2, 4, 8, 16, 32
 STATUS_NAMES = {0: "RECG_OK", 1: "RECG_ERR_INVALID_ARG", 2: "RECG_ERR_SHAPE", 3: "RECG_ERR_CAPACITY",
                 4: "RECG_ERR_CUDA", 5: "RECG_ERR_TIMEOUT", 6: "RECG_ERR_INTERNAL"}
 

@@ -155,6 +155,37 @@ void tc_state_reset(void* s, cudaStream_t st);
 // host-only self-test of the tensor-map cache; returns the number of wrong maps handed out
 int tc_map_cache_selftest(int n_keys, int* evictions);
 
+// A chain of projections in one persistent kernel (steps with at most 128 rows; see gemm_chain.cu).  Every op reads
+// x [M, K] bf16 and w (layout as in GemmArgs); RMSNorm is folded as in EpiParams: EPI_RESIDUAL_NORM ops write x_out and
+// the sum-of-squares slots (one per 128-column tile), ops with scale_in multiply their rows by the rstd of ss_slots_in slots.
+constexpr int kChainMaxOps = 5;
+struct ChainOp {
+  const void* x;
+  const void* w;
+  void* out;
+  int N, K, epi;
+  int scale_in, ss_slots_in;
+  void* x_out;          // EPI_RESIDUAL_NORM
+  const void* gain;     // EPI_RESIDUAL_NORM
+};
+struct ChainCommon {
+  float* ss;
+  int ss_stride;
+  float eps;
+  // EPI_QKV_ROPE
+  const int* tok_slot;
+  const void* rope_cs;
+  void* kv_pool;
+  int64_t n_pages;
+  int layer, n_q, n_kv, head_dim;
+};
+void* chain_state_create(int n_sm);
+void chain_state_destroy(void* s);
+void chain_state_reset(void* s, cudaStream_t st);    // after an error status: the grid barrier's counter starts from zero again
+bool chain_state_reserve(void* s, int max_rows, long long max_total_kblocks, int min_kb);
+// false: not launched (shape not supported, no workspace, or the stream is being captured)
+bool launch_gemm_chain(void* s, const ChainOp* ops, int n_ops, int M, const ChainCommon& cm, int* status, cudaStream_t st);
+
 // S5
 // use_tc: run the tcgen05 kernel (head_dim 128 only); otherwise the mma.sync kernel
 void launch_attention(const BatchLayout& bl, const Dims& dm, int layer, const void* q, void* o, const void* kv_pool,

@@ -81,6 +81,7 @@ struct recg_ctx {
   bool policy_loaded = false;
   std::vector<int> h_policy;
   void* tc_state = nullptr;
+  void* chain_state = nullptr;   // RECG_FLAG_CHAIN
   std::vector<int> h_desc;
   std::vector<int> h_page_owner;   // debug checks: which request names a page
   // optional per-class timing
@@ -443,6 +444,18 @@ recg_status recg_init(recg_ctx** out, const recg_config* cfg, const recg_weights
   }
   cudaMemsetAsync(ctx->d_status, 0, sizeof(int), ctx->stream);
   ctx->tc_state = tc_state_create(n_sm);
+  if ((g.flags & RECG_FLAG_CHAIN) && w && g.head_dim == 128 && !(g.flags & RECG_FLAG_SIMT_GEMM)) {
+    ctx->chain_state = chain_state_create(n_sm);
+    // the widest line of k-blocks in the model: the LM head (128-column tiles) or gate|up (64 output columns per tile)
+    const long long kb_h = g.hidden / 64;
+    long long most = (long long)((g.vocab + 127) / 128) * kb_h;
+    const long long gu = (long long)((g.ffn + 63) / 64) * kb_h;
+    if (gu > most) most = gu;
+    if (ctx->chain_state && !chain_state_reserve(ctx->chain_state, g.max_tokens < 128 ? g.max_tokens : 128, most, (int)kb_h)) {
+      chain_state_destroy(ctx->chain_state);
+      ctx->chain_state = nullptr;
+    }
+  }
   *out = ctx;
   return RECG_OK;
 }
@@ -476,6 +489,7 @@ recg_status recg_free(recg_ctx* ctx) {
   cudaStreamSynchronize(ctx->stream);
   for (cudaEvent_t e : ctx->ev_pool) cudaEventDestroy(e);
   if (ctx->tc_state) tc_state_destroy(ctx->tc_state);
+  if (ctx->chain_state) chain_state_destroy(ctx->chain_state);
   if (ctx->arena.base) cudaFree(ctx->arena.base);
   if (ctx->h_vout) cudaFreeHost(ctx->h_vout);
   delete ctx;
@@ -492,6 +506,7 @@ recg_status recg_sync(recg_ctx* ctx) {
     cudaMemsetAsync(ctx->d_status, 0, sizeof(int), ctx->stream);
     // a projection that gave up may have left arrival counters of cut tiles behind: the next launch starts clean
     tc_state_reset(ctx->tc_state, ctx->stream);
+    chain_state_reset(ctx->chain_state, ctx->stream);
     if (st == DEV_GUARD) {
       launch_guard_fill(ctx->arena.base, ctx->d_guards, ctx->n_guards, ctx->stream);
       return fail(ctx, RECG_ERR_INTERNAL, "device: a guard band behind a workspace region was overwritten");
@@ -514,7 +529,12 @@ static recg_status run_forward(recg_ctx* ctx, void* kv_pool, int64_t kv_pool_pag
   // RMSNorm runs as a kernel of its own, or (RECG_FLAG_FOLD_NORM, tcgen05 path only) folded into the projections:
   // whoever writes the residual stream also writes x = bf16(h * gain of the next norm) and partial sums of squares per
   // row, and the projection that reads x scales its accumulator rows by the row's rstd.
-  const bool fold = (ctx->cfg.flags & RECG_FLAG_FOLD_NORM) && !(ctx->cfg.flags & RECG_FLAG_SIMT_GEMM);
+  // (RECG_FLAG_CHAIN: steps of at most 128 rows run the projections between two attention calls as one persistent kernel)
+  cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+  const bool chain = ctx->chain_state && !bl.dyn && T <= 128 && d.n_layers > 0 && (d.n_q * d.head_dim) % 64 == 0 &&
+                     d.hidden % 128 == 0 && d.ffn % 64 == 0 &&
+                     cudaStreamIsCapturing(st, &cap) == cudaSuccess && cap == cudaStreamCaptureStatusNone;
+  const bool fold = ((ctx->cfg.flags & RECG_FLAG_FOLD_NORM) || chain) && !(ctx->cfg.flags & RECG_FLAG_SIMT_GEMM);
   const int Tm = ctx->cfg.max_tokens;
   const void* first_gain = d.n_layers > 0 ? ctx->attn_norm[0] : ctx->final_norm;
   launch_embed(bl, d, ctx->embed, ctx->h, fold ? first_gain : nullptr, ctx->x, ctx->ss, st);
@@ -537,7 +557,11 @@ static recg_status run_forward(recg_ctx* ctx, void* kv_pool, int64_t kv_pool_pag
     g.epi = fold ? EPI_RESIDUAL_NORM : EPI_RESIDUAL;
     if (fold) { g.x_out = ctx->x; g.gain = next_gain; g.ss_out = ctx->ss; g.ss_stride = Tm; }
   };
+  const bool lbf = ctx->cfg.flags & RECG_FLAG_LOGITS_BF16;
   for (int l = 0; l < d.n_layers; ++l) {
+    if (chain && l > 0) {
+      // the QKV projection of this layer was the last op of the previous layer's chain
+    } else {
     if (!fold) {
       launch_rmsnorm(ctx->h, ctx->attn_norm[l], ctx->x, T, d.hidden, d.rms_eps, st, bl.dyn);
       ctx->mark(1, 1);
@@ -550,10 +574,38 @@ static recg_status run_forward(recg_ctx* ctx, void* kv_pool, int64_t kv_pool_pag
     a.layer = l; a.n_q = d.n_q; a.n_kv = d.n_kv; a.head_dim = d.head_dim; a.rope_cs = ctx->rope_cs;
     if ((s = run_gemm(ctx, a)) != RECG_OK) return s;
     ctx->mark(2, 1);
+    }
     launch_attention(bl, d, l, ctx->q, ctx->o, kv_pool, kv_pool_pages, ctx->part_o, ctx->part_ml,
                      ctx->tok_per_tile, ctx->n_sm, ctx->d_status, st, !(ctx->cfg.flags & RECG_FLAG_SIMT_ATTENTION));
     CU(cudaGetLastError());
     ctx->mark(3, 2);
+    if (chain) {
+      const bool last = l + 1 == d.n_layers;
+      const int slots_h = d.hidden / 128;      // sum-of-squares slots a residual op of the chain fills
+      ChainOp ops[4] = {};
+      ops[0].x = ctx->o; ops[0].w = ctx->wo[l]; ops[0].out = ctx->h; ops[0].N = d.hidden; ops[0].K = qdim;
+      ops[0].epi = EPI_RESIDUAL_NORM; ops[0].x_out = ctx->x; ops[0].gain = ctx->ffn_norm[l];
+      ops[1].x = ctx->x; ops[1].w = ctx->w_gate_up[l]; ops[1].out = ctx->act; ops[1].N = d.ffn; ops[1].K = d.hidden;
+      ops[1].epi = EPI_SWIGLU; ops[1].scale_in = 1; ops[1].ss_slots_in = slots_h;
+      ops[2].x = ctx->act; ops[2].w = ctx->w_down[l]; ops[2].out = ctx->h; ops[2].N = d.hidden; ops[2].K = d.ffn;
+      ops[2].epi = EPI_RESIDUAL_NORM; ops[2].x_out = ctx->x; ops[2].gain = last ? ctx->final_norm : ctx->attn_norm[l + 1];
+      ops[3].x = ctx->x; ops[3].K = d.hidden; ops[3].scale_in = 1; ops[3].ss_slots_in = slots_h;
+      if (last) {
+        ops[3].w = ctx->lm_head; ops[3].out = ctx->logits; ops[3].N = d.vocab; ops[3].epi = lbf ? EPI_PLAIN_BF16 : EPI_PLAIN_F32;
+      } else {
+        ops[3].w = ctx->wqkv[l + 1]; ops[3].out = ctx->q; ops[3].N = (d.n_q + 2 * d.n_kv) * d.head_dim; ops[3].epi = EPI_QKV_ROPE;
+      }
+      ChainCommon cm{};
+      cm.ss = ctx->ss; cm.ss_stride = Tm; cm.eps = d.rms_eps; cm.tok_slot = bl.tok_slot; cm.rope_cs = ctx->rope_cs;
+      cm.kv_pool = kv_pool; cm.n_pages = kv_pool_pages; cm.layer = l + 1; cm.n_q = d.n_q; cm.n_kv = d.n_kv; cm.head_dim = d.head_dim;
+      if (!launch_gemm_chain(ctx->chain_state, ops, 4, T, cm, ctx->d_status, st)) {
+        cudaGetLastError();
+        return fail(ctx, RECG_ERR_INTERNAL, "projection chain: launch refused");
+      }
+      CU(cudaGetLastError());
+      ctx->mark(5, 1);
+      continue;
+    }
     GemmArgs b{};
     residual(b, ctx->ffn_norm[l]);
     b.x = ctx->o; b.w = ctx->wo[l]; b.M = T; b.K = qdim;
@@ -574,17 +626,18 @@ static recg_status run_forward(recg_ctx* ctx, void* kv_pool, int64_t kv_pool_pag
     if ((s = run_gemm(ctx, e, &slots)) != RECG_OK) return s;
     ctx->mark(6, 1);
   }
-  if (!fold) {
-    launch_rmsnorm(ctx->h, ctx->final_norm, ctx->x, T, d.hidden, d.rms_eps, st, bl.dyn);
-    ctx->mark(1, 1);
+  if (!chain) {      // (the chain of the last layer ends with the LM head)
+    if (!fold) {
+      launch_rmsnorm(ctx->h, ctx->final_norm, ctx->x, T, d.hidden, d.rms_eps, st, bl.dyn);
+      ctx->mark(1, 1);
+    }
+    GemmArgs f{};
+    normed(f);
+    f.w = ctx->lm_head; f.out = ctx->logits; f.M = T; f.N = d.vocab;
+    f.epi = lbf ? EPI_PLAIN_BF16 : EPI_PLAIN_F32;
+    if ((s = run_gemm(ctx, f)) != RECG_OK) return s;
+    ctx->mark(7, 1);
   }
-  const bool lbf = ctx->cfg.flags & RECG_FLAG_LOGITS_BF16;
-  GemmArgs f{};
-  normed(f);
-  f.w = ctx->lm_head; f.out = ctx->logits; f.M = T; f.N = d.vocab;
-  f.epi = lbf ? EPI_PLAIN_BF16 : EPI_PLAIN_F32;
-  if ((s = run_gemm(ctx, f)) != RECG_OK) return s;
-  ctx->mark(7, 1);
   ctx->logits_valid = true;
   if (logits) {
     logits->data = ctx->logits;

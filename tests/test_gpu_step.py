@@ -447,3 +447,47 @@ def test_step_is_deterministic_and_survives_many_rounds():
     assert len(first) == len(batches)
     ctx.recg_sync()
     ctx.recg_free()
+
+
+@pytest.mark.parametrize("specs", [
+    [(200, 16, 16)],                                      # one request, 32 rows: the low-concurrency shape
+    [(70, 4, 4), (33, 2, 2), (500, 8, 8), (16, 3, 5)],    # four requests, 40 rows: padded to 64
+    [(129, 16, 16), (300, 30, 32), (64, 8, 8)],           # 110 rows: padded to 128
+    [(40, 1, 0)],                                         # a single row
+])
+def test_projection_chain_on_8b_shaped_layers(specs):
+    """RECG_FLAG_CHAIN: the projections between two attention calls as one persistent kernel (two 8B-shaped layers, so
+    that the chain's last op is once the next layer's QKV projection with rotary embedding and K/V append, and once the
+    LM head).  Compared with the oracle like the ordinary step, and with the ordinary step of the same context-free
+    inputs (same integers wherever the top-2 gap is not a near tie)."""
+    shape = synth.llama8b_shape(2)
+    shape.vocab = 16384
+    W = synth.model_weights(shape, seed=0, dtype=torch.bfloat16)
+    synth.perturb_norm_gains(W)
+    ocfg, W64 = oracle_cfg(shape), oracle_weights(W)
+    L, v, b = [s[0] for s in specs], [s[1] for s in specs], [s[2] for s in specs]
+    desc = synth.fixed_descriptor(L, v, b, seed=4)
+    stats = {}
+    for flags in (binding.FLAG_CHAIN, 0):
+        ctx = binding.Context(binding.make_config(shape, 8, 128, desc.page_table.shape[1], flags), to_dev(W))
+        pool = binding.alloc_kv_pool(ctx, desc.n_pages, fill=None)
+        pool.fill_(float("nan"))
+        reqs = []
+        for i in range(len(specs)):
+            kv = []
+            for l in range(shape.n_layers):
+                K, V = synth.kv_values(L[i], shape.n_kv_heads, shape.head_dim, seed=300 + 10 * i + l)
+                ctx.recg_kv_write(pool, desc.n_pages, l, desc.page_table[i], 0, K.cuda(), V.cuda())
+                kv.append((f64(K), f64(V)))
+            y = synth.token_ids(v[i], shape.vocab, seed=400 + i).tolist()
+            reqs.append({"kv": kv, "y": y, "L": L[i], "v": v[i], "b": b[i], "m": None})
+        stats[flags], got = check_round(ctx, shape, ocfg, W64, reqs, desc, pool, margin_flag=MARGIN_LARGE_SHAPES)
+        # a second run gives the same bits (parts are added in part order)
+        ys = [t for r in reqs for t in r["y"]]
+        batch = binding.Batch(desc.ctx_len, desc.verify_len, desc.block_size, ys, desc.page_table, pool, desc.n_pages)
+        a1 = ctx.logits_tensor(ctx.recg_step(batch))
+        a2 = ctx.logits_tensor(ctx.recg_step(batch))
+        ctx.recg_sync()
+        assert torch.equal(a1, a2)
+        ctx.recg_free()
+    report_flat_flag(stats[binding.FLAG_CHAIN])
