@@ -25,9 +25,6 @@
 // sets the status word, after which nothing in this CTA blocks any more.
 #include <cuda.h>
 
-#include <cstdio>
-#include <unordered_map>
-
 #include "common.cuh"
 #include "epilogue.cuh"
 #include "kernels.h"
