@@ -284,6 +284,25 @@ struct RingLoader {
 // of its row tile ("part").  Part p >= 1 of a tile is always the FIRST piece of its CTA, part 0 the last piece (or
 // the first, when the range starts exactly at the column): that decides the workspace slot,
 // 2 * cta + (first piece ? 0 : 1).
+// The stream-K division of a problem of mt x (n_tiles / mt) tiles with KB k-blocks each over n_units scheduling units:
+// all but the last one-to-two waves stay whole tiles (dp_tiles of them, done after the cut ones), the k-blocks of the
+// remaining tile columns are spread evenly over teams of mt units.  Computed on the host, or in the kernel when the row
+// count (hence mt) is only known on the device.  Needs mt <= n_units.
+__host__ __device__ inline void stream_k_schedule(int n_tiles, int mt, int KB, int n_units, int* dp_tiles, long long* per,
+                                                  int* used_units) {
+  const int n_teams = n_units / mt;
+  const int full = n_tiles / n_units;
+  *dp_tiles = full >= 2 ? ((full - 1) * n_units / mt) * mt : 0;
+  const long long total = (long long)((n_tiles - *dp_tiles) / mt) * KB;
+  const long long teams = total < n_teams ? total : n_teams;
+  long long p = teams > 0 ? (total + teams - 1) / teams : 1;
+  if (p < 4 && total >= 4) p = 4;                     // keep pieces long enough to amortise their hand-over
+  if (p < 1) p = 1;
+  *per = p;
+  const int used = (int)((total + p - 1) / p);        // teams that get a range
+  *used_units = *dp_tiles ? n_units : used * mt;      // (with whole tiles behind, the grid stays at full size)
+}
+
 struct Piece {
   int tile, kb0, kb1;     // k-block range [kb0, kb1) of the tile
   int part, n_parts;      // which part of the tile this is
@@ -514,12 +533,13 @@ template <int BN, bool PAIR, bool NORM>
 __global__ void __launch_bounds__(kTcThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
                const __grid_constant__ CUtensorMap map_out, const __grid_constant__ CUtensorMap map_xout, int M_cap, int n_tiles_n,
-               int K, int up_row_offset, int dp_tiles_in, long long per, int thin, float* split_ws, int* split_counters,
+               int K, int up_row_offset, int dp_tiles_in, long long per_in, int thin, float* split_ws, int* split_counters,
                const int* __restrict__ m_dev, EpiParams ep_in) {
   // Device-resident rounds: the row count comes from device memory (written by a kernel at least two launches back, so
   // it may be read before this kernel waits for its predecessor); the tensor maps cover the capacity M_cap, rows
   // between the count and the capacity hold stale data and are computed but never used, and all tiles are whole.
   const int M = m_dev ? __ldg(m_dev) : M_cap;
+  if (M <= 0) return;          // an empty round (the same for every thread of the grid): nothing to do, nothing was set up yet
   EpiParams ep = ep_in;
   ep.M = M;
   using Cfg = TcCfg<BN, PAIR, NORM>;
@@ -575,8 +595,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n_tiles_m = (M + kRows - 1) / kRows;
   const int n_tiles = n_tiles_m * n_tiles_n;
-  const int dp_tiles = dp_tiles_in < 0 ? n_tiles : dp_tiles_in;
   const int KB = K / BK;
+  // dp_tiles_in >= 0: the host's schedule; -1: whole tiles only; -2: stream-K, divided here from the device's row count
+  int dp_tiles = dp_tiles_in < 0 ? n_tiles : dp_tiles_in;
+  long long per = per_in;
+  if (dp_tiles_in == -2) {
+    if (n_tiles_m >= 1 && n_tiles_m <= n_units) {
+      int used;
+      stream_k_schedule(n_tiles, n_tiles_m, KB, n_units, &dp_tiles, &per, &used);
+    } else {
+      dp_tiles = n_tiles;
+    }
+  }
   const bool swiglu = ep.epi == EPI_SWIGLU;
   // schedule: the k-blocks of tiles [dp_tiles, n_tiles) as one line cut into equal ranges per CTA; then tiles
   // [0, dp_tiles) whole, strided over the grid (CTAs that run together share a weight tile through L2)
@@ -994,22 +1024,13 @@ bool launch_bn_t(TcState* st, int idx, const GemmArgs& a, const EpiParams& ep, b
   int units = n_tiles < n_units ? n_tiles : n_units;
   int dp_tiles = n_tiles;       // whole tiles, strided
   long long per = 1;
-  if (a.m_dev) {                // the row count is on the device: whole tiles only, counted by the kernel
-    dp_tiles = -1;
-    stream_k = false;
-  }
-  if (stream_k) {
-    // all but the last one-to-two waves as whole tiles; the k-blocks of the remaining tile columns evenly over
-    // teams of mt units (one per row tile)
-    const int n_teams = n_units / mt;                   // the caller made sure that mt <= n_units
-    const int full = n_tiles / n_units;
-    dp_tiles = full >= 2 ? ((full - 1) * n_units / mt) * mt : 0;
-    const long long total = (long long)((n_tiles - dp_tiles) / mt) * KB;
-    const long long teams = total < n_teams ? total : n_teams;
-    per = (total + teams - 1) / teams;
-    if (per < 4 && total >= 4) per = 4;                 // keep pieces long enough to amortise their hand-over
-    const int used = (int)((total + per - 1) / per);    // teams that get a range
-    units = dp_tiles ? n_units : used * mt;             // (with whole tiles behind, the grid stays at full size)
+  if (a.m_dev) {
+    // the row count is on the device: the kernel counts the tiles and, for stream-K, divides the k-blocks itself; the
+    // grid has every unit (units without work leave at once)
+    dp_tiles = stream_k ? -2 : -1;
+    units = n_units;
+  } else if (stream_k) {
+    stream_k_schedule(n_tiles, mt, (int)KB, n_units, &dp_tiles, &per, &units);     // the caller made sure that mt <= n_units
   }
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(PAIR ? 2 * units : units);
