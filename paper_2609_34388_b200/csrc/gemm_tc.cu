@@ -535,10 +535,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                const __grid_constant__ CUtensorMap map_out, const __grid_constant__ CUtensorMap map_xout, int M_cap, int n_tiles_n,
                int K, int up_row_offset, int dp_tiles_in, long long per_in, int thin, float* split_ws, int* split_counters,
                const int* __restrict__ m_dev, EpiParams ep_in) {
-  // Device-resident rounds: the row count comes from device memory (written by a kernel at least two launches back, so
-  // it may be read before this kernel waits for its predecessor); the tensor maps cover the capacity M_cap, rows
-  // between the count and the capacity hold stale data and are computed but never used, and all tiles are whole.
-  const int M = m_dev ? __ldg(m_dev) : M_cap;
+  // Device-resident rounds: the row count comes from device memory; the tensor maps cover the capacity M_cap, and rows
+  // between the count and the capacity hold stale data and are computed but never used.  The count is written by the
+  // first kernel of the step, and the small kernels between it and the first projection signal their dependents before
+  // they wait themselves, so this kernel can be running before that one has finished: it has to wait for its
+  // predecessors before it reads the count (and gives up the early weight requests in this mode).
+  if (m_dev) griddep_wait();
+  const int M = m_dev ? *reinterpret_cast<const volatile int*>(m_dev) : M_cap;
   if (M <= 0) return;          // an empty round (the same for every thread of the grid): nothing to do, nothing was set up yet
   EpiParams ep = ep_in;
   ep.M = M;
