@@ -476,9 +476,9 @@ size_t attention_smem_bytes(int head_dim) {
 
 void launch_attention(const BatchLayout& bl, const Dims& dm, int layer, const void* q, void* o, const void* kv_pool,
                       int64_t n_pages, float* part_o, float* part_ml, int tok_per_tile, int n_sm, int* status,
-                      cudaStream_t st, bool use_tc) {
+                      cudaStream_t st, bool use_tc, bool layout_settled) {
   if (use_tc && dm.head_dim == 128) {
-    launch_attention_tc_main(bl, dm, layer, q, o, kv_pool, n_pages, part_o, part_ml, n_sm, status, st);
+    launch_attention_tc_main(bl, dm, layer, q, o, kv_pool, n_pages, part_o, part_ml, n_sm, status, st, layout_settled);
     launch_pdl(attention_combine_kernel<128>, dim3(4 * n_sm), dim3(512), 0, st, (const AttnTile*)bl.tiles,
                (const int*)bl.counts, dm.n_q, dm.n_q / dm.n_kv, (const float*)part_o, (const float*)part_ml,
                static_cast<__nv_bfloat16*>(o));

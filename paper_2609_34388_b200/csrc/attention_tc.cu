@@ -89,6 +89,7 @@ struct TcAttnParams {
   float* part_o;
   float* part_ml;
   int* status;
+  int early_desc;     // the work list is settled: it may be read before the wait for the kernel in front of this one
 };
 
 // ---- PTX wrappers (tcgen05) ------------------------------------------------------------------------
@@ -222,7 +223,10 @@ __global__ void __launch_bounds__(kThreads, 1) attention_tc_kernel(const __grid_
   auto item_at = [&](int i) { return i < range_n0 ? range_b0 + i : range_b1 + (i - range_n0); };
   AttnItem w_next = {};
   if (warp == 0) {
-    griddep_wait();
+    // (inside a step the work list was written many launches ago and the kernel in front of this one, the QKV
+    // projection, only signals its dependents when its own work is done: the two dependent reads below then overlap
+    // that kernel's tail instead of following it)
+    if (!P.early_desc) griddep_wait();
     const int4 r4 = *reinterpret_cast<const int4*>(P.cta_off + 4 * blockIdx.x);
     range_b0 = r4.x;
     range_n0 = r4.y - r4.x;
@@ -236,6 +240,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_tc_kernel(const __grid_
       s_range[3] = item_end;
       *s_first = w_next;
     }
+    if (P.early_desc) griddep_wait();
   }
   if (threadIdx.x == 32) {
     *abort_flag = 0;
@@ -709,7 +714,7 @@ bool q_tensor_map(const void* q, int n_tok, int n_q, int group, CUtensorMap* out
 
 void launch_attention_tc_main(const BatchLayout& bl, const Dims& dm, int layer, const void* q, void* o,
                               const void* kv_pool, int64_t n_pages, float* part_o, float* part_ml, int n_sm, int* status,
-                              cudaStream_t st) {
+                              cudaStream_t st, bool layout_settled) {
   static bool configured[kMaxDevices] = {false};
   if (first_use_on_device(configured))
     cudaFuncSetAttribute(attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
@@ -733,6 +738,7 @@ void launch_attention_tc_main(const BatchLayout& bl, const Dims& dm, int layer, 
   P.part_o = part_o;
   P.part_ml = part_ml;
   P.status = status;
+  P.early_desc = layout_settled ? 1 : 0;
   CUtensorMap qmap;
   if (!q_tensor_map(q, bl.n_tok, dm.n_q, P.group, &qmap)) {
     // nothing is launched; the status word makes the next recg_sync() fail instead of returning stale outputs

@@ -188,12 +188,14 @@ bool launch_gemm_chain(void* s, const ChainOp* ops, int n_ops, int M, const Chai
 
 // S5
 // use_tc: run the tcgen05 kernel (head_dim 128 only); otherwise the mma.sync kernel
+// layout_settled: the work list was written by a kernel that is known to have finished when this one starts (anything but
+// the launch right before it): the tcgen05 kernel then reads its work range before it waits for its predecessor
 void launch_attention(const BatchLayout& bl, const Dims& dm, int layer, const void* q, void* o, const void* kv_pool,
                       int64_t n_pages, float* part_o, float* part_ml, int tok_per_tile, int n_sm, int* status,
-                      cudaStream_t st, bool use_tc);
+                      cudaStream_t st, bool use_tc, bool layout_settled = false);
 void launch_attention_tc_main(const BatchLayout& bl, const Dims& dm, int layer, const void* q, void* o,
                               const void* kv_pool, int64_t n_pages, float* part_o, float* part_ml, int n_sm, int* status,
-                              cudaStream_t st);
+                              cudaStream_t st, bool layout_settled);
 size_t attention_smem_bytes(int head_dim);
 
 // S9b + S10

@@ -576,7 +576,7 @@ static recg_status run_forward(recg_ctx* ctx, void* kv_pool, int64_t kv_pool_pag
     ctx->mark(2, 1);
     }
     launch_attention(bl, d, l, ctx->q, ctx->o, kv_pool, kv_pool_pages, ctx->part_o, ctx->part_ml,
-                     ctx->tok_per_tile, ctx->n_sm, ctx->d_status, st, !(ctx->cfg.flags & RECG_FLAG_SIMT_ATTENTION));
+                     ctx->tok_per_tile, ctx->n_sm, ctx->d_status, st, !(ctx->cfg.flags & RECG_FLAG_SIMT_ATTENTION), true);
     CU(cudaGetLastError());
     ctx->mark(3, 2);
     if (chain) {
@@ -870,7 +870,8 @@ recg_status recg_attention(recg_ctx* ctx, const recg_batch* batch, int32_t layer
     return fail(ctx, RECG_ERR_INVALID_ARG, "recg_attention: no batch given and none with a KV pool laid out before");
   }
   launch_attention(ctx->bl, ctx->dm, layer, q, o, ctx->last_pool, ctx->last_pool_pages, ctx->part_o, ctx->part_ml,
-                   ctx->tok_per_tile, ctx->n_sm, ctx->d_status, ctx->stream, !(ctx->cfg.flags & RECG_FLAG_SIMT_ATTENTION));
+                   ctx->tok_per_tile, ctx->n_sm, ctx->d_status, ctx->stream, !(ctx->cfg.flags & RECG_FLAG_SIMT_ATTENTION),
+                   batch == nullptr);      // (a batch given with the call was laid out by the launch right before this one)
   CU(cudaGetLastError());
   return RECG_OK;
 }
