@@ -262,8 +262,11 @@ recg_status recg_debug_buffer(recg_ctx *ctx, int32_t which, const void **ptr, in
  * Debugging aids (the paper has no counterpart).
  * recg_debug_gemm_config(): force the tile configuration of the projection launches that follow on this context,
  *   instead of the cost model's choice: tile = 64, 128 or 256 (single CTAs, 128-row tiles of that width), 384 (CTA
- *   pairs, 256 x 128 tiles), 512 (CTA pairs, 256 x 256 tiles), 0 = back to the cost model; stream_k != 0 cuts the
- *   K range of the tiles evenly over the SMs.  A configuration that does not fit a shape is ignored for that launch.
+ *   pairs, 256 x 128 tiles), 512 (CTA pairs, 256 x 256 tiles), 0 = back to the cost model; stream_k = 1 cuts the
+ *   K range of the tiles evenly over the SMs, stream_k = 2 does the same and also (with any tile value, 0 included)
+ *   keeps problems of at most 32 rows from handing their partial tiles over inside thread-block clusters: they go
+ *   through the partial-tile workspace like everything else; stream_k = 0: whole tiles.  A configuration that does not
+ *   fit a shape is ignored for that launch.
  * recg_debug_wait_timeout(): enqueue a one-thread kernel that waits on a barrier nobody arrives on, bounded by
  *   max_polls polls (1 .. 1048576) exactly like the waits inside the kernels; it gives up, records the timeout in the
  *   device status word and returns.  The next recg_sync() then reports RECG_ERR_TIMEOUT and clears the word; the

@@ -383,8 +383,8 @@ class Context:
         self._check(lib().recg_next_round(self.h, C.byref(batch.c), _ptr(next_block), _ptr(planted_emitted),
                                           C.byref(log.c) if log is not None else None, int(round_index)))
 
-    def recg_debug_gemm_config(self, tile: int, stream_k: bool):
-        self._check(lib().recg_debug_gemm_config(self.h, int(tile), 1 if stream_k else 0))
+    def recg_debug_gemm_config(self, tile: int, stream_k: int):
+        self._check(lib().recg_debug_gemm_config(self.h, int(tile), int(stream_k)))
 
     def recg_debug_wait_timeout(self, max_polls: int):
         self._check(lib().recg_debug_wait_timeout(self.h, int(max_polls)))

@@ -10,6 +10,9 @@
 //            plain store) while the MMA warp already fills the other accumulator; output rows leave through
 //            TMA box stores (add-reductions for the residual stream) from a small swizzled staging area.
 // Tiles are walked m-fastest so that CTAs running together share the same weight tile through L2.
+// Tiles can be cut over K (stream-K): partial tiles are parked in a workspace and reduced by the last part to arrive; for
+// problems of at most 32 rows the parts of a tile form a thread-block cluster instead and hand their partial tiles to the
+// cluster's leader through distributed shared memory.
 // Every wait is bounded; on a timeout the kernel records a status code, drains and frees TMEM.
 #include <cuda.h>
 
@@ -126,6 +129,10 @@ __device__ __forceinline__ void tmem_dealloc_pair(uint32_t addr, uint32_t cols) 
 }
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar_cluster) {
   asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar_cluster) : "memory");
+}
+__device__ __forceinline__ void st_cluster_f4(uint32_t addr_cluster, const float4& v) {
+  asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(addr_cluster), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w)
+               : "memory");
 }
 
 // ---- register epilogue: one thread owns one output row -------------------------------------------
@@ -245,12 +252,13 @@ struct SplitLoader {
 };
 
 // The reducing CTA's own part comes from its TMEM accumulator, the other parts from copies in shared memory (the
-// idle operand ring, one [BN/4][BM] float4 tile after the other in part order without the own part).  Parts are
-// added in part order starting from zero, exactly like SplitLoader, so both give the same bits.
+// idle operand ring, one [BN/4][rows] float4 tile after the other in part order without the own part; rows = BM, or
+// 32 for the parts that the CTAs of a cluster hand to their leader).  Parts are added in part order starting from
+// zero, exactly like SplitLoader, so both give the same bits.
 struct RingLoader {
   uint32_t tacc;
   const float4* ring;     // + row
-  int bn, own, n_parts;
+  int bn, own, n_parts, rows;
   // Every lane takes part, also those whose row lies beyond M (the TMEM load is a warp-wide instruction; their
   // sums are never stored).
   __device__ __forceinline__ void operator()(int col, float (&v)[32]) const {
@@ -264,11 +272,11 @@ struct RingLoader {
 #pragma unroll
         for (int i = 0; i < 32; ++i) v[i] += t[i];
       } else {
-        const float4* src = ring + ((size_t)k * (bn / 4) + col / 4) * BM;
+        const float4* src = ring + ((size_t)k * (bn / 4) + col / 4) * rows;
         ++k;
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
-          const float4 a = src[(size_t)i * BM];
+          const float4 a = src[(size_t)i * rows];
           v[4 * i] += a.x; v[4 * i + 1] += a.y; v[4 * i + 2] += a.z; v[4 * i + 3] += a.w;
         }
       }
@@ -533,8 +541,8 @@ template <int BN, bool PAIR, bool NORM>
 __global__ void __launch_bounds__(kTcThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
                const __grid_constant__ CUtensorMap map_out, const __grid_constant__ CUtensorMap map_xout, int M_cap, int n_tiles_n,
-               int K, int up_row_offset, int dp_tiles_in, long long per_in, int thin, float* split_ws, int* split_counters,
-               const int* __restrict__ m_dev, EpiParams ep_in) {
+               int K, int up_row_offset, int dp_tiles_in, long long per_in, int thin, int cl_parts, float* split_ws,
+               int* split_counters, const int* __restrict__ m_dev, EpiParams ep_in) {
   // Device-resident rounds: the row count comes from device memory; the tensor maps cover the capacity M_cap, and rows
   // between the count and the capacity hold stale data and are computed but never used.  The count is written by the
   // first kernel of the step, and the small kernels between it and the first projection signal their dependents before
@@ -553,9 +561,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
   const int n_units = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  const int n_stages = thin ? Cfg::kThinStages : Cfg::kStages;
+  // Thin problems whose tiles are cut over K can run as CLUSTERS of cl CTAs per tile (cl_parts > 1; at most 32 rows, one
+  // row tile, single CTAs only): rank r computes k-blocks [r KB / cl, (r + 1) KB / cl) and hands its 32 x BN partial to
+  // the cluster's leader (rank 0) through distributed shared memory, into a reserve at the top of the leader's ring
+  // budget; the leader adds the parts in rank order and runs the epilogue.  No trip through global memory, no counter.
+  const int cl = (!PAIR && thin && cl_parts > 1) ? cl_parts : 0;
+  const uint32_t crank = cl ? cluster_ctarank() : 0u;
+  constexpr int kClPartBytes = 32 * BN * 4;
+  const int cl_reserve = cl ? (cl - 1) * kClPartBytes : 0;
   const int a_bytes = thin ? Cfg::kThinABytes : Cfg::kABytes;
   const int stage_bytes = a_bytes + Cfg::kBBytes;
+  const int cl_stages = (Cfg::kBudget - cl_reserve) / stage_bytes;
+  const int n_stages = cl ? (cl_stages > Cfg::kMaxStages ? Cfg::kMaxStages : cl_stages) : (thin ? Cfg::kThinStages : Cfg::kStages);
   uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + Cfg::kBarOff);
   uint64_t* empty_bar = full_bar + Cfg::kMaxStages;
   uint64_t* tfull_bar = empty_bar + Cfg::kMaxStages;
@@ -615,9 +632,24 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
   // [0, dp_tiles) whole, strided over the grid (CTAs that run together share a weight tile through L2)
   const long long total = (long long)((n_tiles - dp_tiles) / n_tiles_m) * KB;
   const long long lo_raw = (long long)(unit / n_tiles_m) * per;
-  const long long range_lo = lo_raw < total ? lo_raw : total;
-  const long long range_hi = range_lo + per < total ? range_lo + per : total;
-  const int dp_count = unit < dp_tiles ? (dp_tiles - 1 - unit) / n_units + 1 : 0;
+  const long long range_lo = cl ? 0 : (lo_raw < total ? lo_raw : total);
+  const long long range_hi = cl ? 1 : (range_lo + per < total ? range_lo + per : total);
+  const int dp_count = cl ? 0 : (unit < dp_tiles ? (dp_tiles - 1 - unit) / n_units + 1 : 0);
+  // the next piece of this CTA (a cluster member has exactly one)
+  auto next_piece = [&](int& jd, long long& pos) -> Piece {
+    if (cl) {
+      Piece p;
+      p.tile = (int)blockIdx.x / cl;
+      p.kb0 = (int)((long long)crank * KB / cl);
+      p.kb1 = (int)((long long)(crank + 1) * KB / cl);
+      p.part = (int)crank;
+      p.n_parts = cl;
+      p.slot = p.slot0 = p.slot_next = 0;
+      pos = range_hi;
+      return p;
+    }
+    return make_piece(jd, dp_tiles, pos, range_hi, KB, per, unit, n_units, n_tiles_m);
+  };
 
   if (threadIdx.x == 0) {
     s_abort = 0;
@@ -629,7 +661,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
       mbar_init(&tfull_bar[a], 1);
       mbar_init(&tempty_bar[a], PAIR ? 8 : 4);
     }
-    mbar_init(red_bar, 1);
+    mbar_init(red_bar, cl ? cl - 1 : 1);      // (cluster leader: one arrival per peer)
     for (int i = 0; i < 8; ++i) mbar_init(&h_bar[i], 1);
     fence_barrier_init();
     prefetch_tmap(&map_x);
@@ -647,6 +679,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
   tc_fence_before();
   __syncthreads();
   if constexpr (PAIR) cluster_sync_all();   // both CTAs' barriers are initialised before anyone signals across
+  else if (cl) cluster_sync_all();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
   // (each role waits for the kernels before this one where it first needs their results)
@@ -688,7 +721,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
       if (dp_count > 0 || range_lo < range_hi) {
         long long p0 = range_lo;
         int j0 = 0;
-        const Piece pc = make_piece(j0, dp_tiles, p0, range_hi, KB, per, unit, n_units, n_tiles_m);
+        const Piece pc = next_piece(j0, p0);
         n_pre = pc.kb1 - pc.kb0 < n_stages ? pc.kb1 - pc.kb0 : n_stages;
         pre_kb0 = pc.kb0;
         pre_tm = pc.tile % n_tiles_m;
@@ -704,7 +737,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
       bool ok = true;
       long long pos = range_lo;
       for (int jd = 0; (jd < dp_count || pos < range_hi) && ok;) {
-        const Piece pc = make_piece(jd, dp_tiles, pos, range_hi, KB, per, unit, n_units, n_tiles_m);
+        const Piece pc = next_piece(jd, pos);
         const int tm = pc.tile % n_tiles_m, tn = pc.tile / n_tiles_m;
         const int kb0 = pc.kb0, kb1 = pc.kb1;
         for (int kb = kb0; kb < kb1; ++kb) {
@@ -743,7 +776,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
       bool ok = true;
       long long pos = range_lo;
       for (int jd = 0; (jd < dp_count || pos < range_hi) && ok; ++tcount) {
-        const Piece pc = make_piece(jd, dp_tiles, pos, range_hi, KB, per, unit, n_units, n_tiles_m);
+        const Piece pc = next_piece(jd, pos);
         const int kb0 = pc.kb0, kb1 = pc.kb1;
         const int acc = tcount & 1;
         if (!wait_bar(&tempty_bar[acc], ((tcount >> 1) & 1) ^ 1)) {
@@ -792,7 +825,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     griddep_wait();                        // the epilogue reads and writes what earlier kernels produced
     long long pos = range_lo;
     for (int jd = 0; jd < dp_count || pos < range_hi; ++tcount) {
-      const Piece pc = make_piece(jd, dp_tiles, pos, range_hi, KB, per, unit, n_units, n_tiles_m);
+      const Piece pc = next_piece(jd, pos);
       const int tile = pc.tile, n_splits = pc.n_parts;
       const int tm = tile % n_tiles_m, tn = tile / n_tiles_m;
       const int acc = tcount & 1;
@@ -828,6 +861,45 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
       if (n_splits == 1) {
         row_epilogue<BN, NORM>(ep, TmemLoader{tacc}, m, n0, stg, &map_out, &map_xout, rstd, tn, ns, prepared);
         release_acc();
+      } else if (cl) {
+        uint8_t* reserve = smem + Cfg::kBudget - cl_reserve;       // the leader's: cl - 1 parts of [BN/4][32] float4
+        if (crank != 0) {
+          if (quad == 0) {           // the warp that holds rows 0..31 of the accumulator
+            const uint32_t dst = mapa_rank(smem_u32(reserve + (crank - 1) * kClPartBytes), 0) + lane * 16;
+#pragma unroll 1
+            for (int c = 0; c < BN / 32; ++c) {
+              float v[32];
+              tmem_ld32(tacc + c * 32, v);
+#pragma unroll
+              for (int i = 0; i < 8; ++i)
+                st_cluster_f4(dst + (uint32_t)(c * 8 + i) * 512u, make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]));
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(mapa_rank(smem_u32(red_bar), 0));   // release: the warp's stores are visible
+          }
+          release_acc();
+        } else {
+          if (!s_abort) {            // the peers' parts have landed (acquire at cluster scope)
+            bool ok = false;
+            for (uint32_t i = 0; i < kSpin && !ok; ++i) {
+              uint32_t got;
+              asm volatile(
+                  "{\n .reg .pred p;\n mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+                  : "=r"(got)
+                  : "r"(smem_u32(red_bar)), "r"(0u)
+                  : "memory");
+              ok = got != 0;
+              if (!ok && i > 64) __nanosleep(32);
+            }
+            if (!ok) {
+              set_status(ep.status, DEV_TIMEOUT_FULL);
+              s_abort = 1;
+            }
+          }
+          RingLoader ld{tacc, reinterpret_cast<const float4*>(reserve) + lane, BN, 0, n_splits, 32};
+          row_epilogue<BN, NORM>(ep, ld, m, n0, stg, &map_out, &map_xout, rstd, tn, ns, false);
+          release_acc();
+        }
       } else {
         // park this split's partial tile and let the LAST split to arrive reduce all partials in split order
         // (deterministic) and run the fused epilogue
@@ -881,7 +953,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
               }
             }
             wait_or_abort(red_bar, 0, DEV_TIMEOUT_FULL);
-            RingLoader ld{tacc, reinterpret_cast<const float4*>(smem) + row_in_tile, BN, pc.part, n_splits};
+            RingLoader ld{tacc, reinterpret_cast<const float4*>(smem) + row_in_tile, BN, pc.part, n_splits, BM};
             row_epilogue<BN, NORM>(ep, ld, m, n0, stg, &map_out, &map_xout, rstd, tn, ns, false);
           } else {
             SplitLoader ld{split_ws, BN, row_in_tile, slot0, slot_next, slot_stride, n_splits, m < ep.M};
@@ -898,6 +970,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
   tc_fence_before();
   __syncthreads();
   if constexpr (PAIR) cluster_sync_all();   // the peer may read this CTA's operands and signal its barriers until here
+  // (a cluster of a thin problem needs no meeting here: only the leader's shared memory is written by others, and the
+  // leader has waited for those stores; the peers are free to leave)
   if (warp == 1) {
     tc_fence_after();
     if constexpr (PAIR) tmem_dealloc_pair(tmem_base, Cfg::kTmemCols);
@@ -939,6 +1013,12 @@ struct TcState {
   size_t evictions = 0;
   int last_tiles_n = 0;       // column tiles of the last launch
   bool configured[10] = {false, false, false, false, false, false, false, false, false, false};
+  bool thin_clusters = true;  // thin problems with cut tiles run as clusters that reduce through distributed shared memory
+  int max_clusters[10][5];    // cached occupancy answers per kernel and cluster size (-1: not asked yet)
+  TcState() {
+    for (auto& row : max_clusters)
+      for (int& v : row) v = -1;
+  }
 };
 
 template <typename Encode>
@@ -995,6 +1075,48 @@ bool launch_bn(TcState* st, int idx, const GemmArgs& a, const EpiParams& ep, boo
 }
 
 template <int BN, bool PAIR, bool NORM>
+int max_active_clusters(TcState* st, int idx, int n_tiles, int parts);
+
+// Thin problems (at most 32 rows) whose tiles would be cut over K: how many CTAs form the cluster that shares a tile
+// (0: no clusters).  The whole grid has to be resident at once, which the occupancy query decides (cached).
+template <int BN, bool PAIR, bool NORM>
+int cluster_parts(TcState* st, int idx, int n_tiles, int KB) {
+  if (PAIR || !st->thin_clusters || n_tiles <= 0) return 0;
+  int parts = st->n_sm / n_tiles;
+  if (parts > 4) parts = 4;
+  if (parts > KB) parts = KB;
+  for (; parts >= 2; --parts) {
+    if (max_active_clusters<BN, PAIR, NORM>(st, idx, n_tiles, parts) >= n_tiles) return parts;
+  }
+  return 0;
+}
+
+template <int BN, bool PAIR, bool NORM>
+int max_active_clusters(TcState* st, int idx, int n_tiles, int parts) {
+  int& cached = st->max_clusters[idx][parts];
+  if (cached < 0) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(n_tiles * parts);
+    cfg.blockDim = dim3(kTcThreads);
+    cfg.dynamicSmemBytes = TcCfg<BN, PAIR, NORM>::kSmemBytes;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = parts;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, gemm_tc_kernel<BN, PAIR, NORM>, &cfg) != cudaSuccess) {
+      cudaGetLastError();
+      n = 0;
+    }
+    cached = n;
+  }
+  return cached;
+}
+
+template <int BN, bool PAIR, bool NORM>
 bool launch_bn_t(TcState* st, int idx, const GemmArgs& a, const EpiParams& ep, bool stream_k, cudaStream_t stream) {
   st->last_tiles_n = (a.N + (a.epi == EPI_SWIGLU ? BN / 2 : BN) - 1) / (a.epi == EPI_SWIGLU ? BN / 2 : BN);
   using Cfg = TcCfg<BN, PAIR, NORM>;
@@ -1027,7 +1149,10 @@ bool launch_bn_t(TcState* st, int idx, const GemmArgs& a, const EpiParams& ep, b
   int units = n_tiles < n_units ? n_tiles : n_units;
   int dp_tiles = n_tiles;       // whole tiles, strided
   long long per = 1;
-  if (a.m_dev) {
+  const int cl = (thin && stream_k && mt == 1) ? cluster_parts<BN, PAIR, NORM>(st, idx, n_tiles, (int)KB) : 0;
+  if (cl) {
+    units = n_tiles * cl;       // one cluster per tile; the kernel derives each member's k-blocks from its rank
+  } else if (a.m_dev) {
     // the row count is on the device: the kernel counts the tiles and, for stream-K, divides the k-blocks itself; the
     // grid has every unit (units without work leave at once)
     dp_tiles = stream_k ? -2 : -1;
@@ -1042,9 +1167,9 @@ bool launch_bn_t(TcState* st, int idx, const GemmArgs& a, const EpiParams& ep, b
   cfg.stream = stream;
   cudaLaunchAttribute attr[2];
   int n_attr = 0;
-  if (PAIR) {
+  if (PAIR || cl) {
     attr[n_attr].id = cudaLaunchAttributeClusterDimension;
-    attr[n_attr].val.clusterDim.x = 2;
+    attr[n_attr].val.clusterDim.x = PAIR ? 2 : cl;
     attr[n_attr].val.clusterDim.y = 1;
     attr[n_attr].val.clusterDim.z = 1;
     ++n_attr;
@@ -1058,7 +1183,7 @@ bool launch_bn_t(TcState* st, int idx, const GemmArgs& a, const EpiParams& ep, b
   }
   cfg.attrs = attr;
   cfg.numAttrs = n_attr;
-  return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<BN, PAIR, NORM>, mx, mw, mo, mxo, a.M, n_tiles_n, a.K, a.N, dp_tiles, per, thin,
+  return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<BN, PAIR, NORM>, mx, mw, mo, mxo, a.M, n_tiles_n, a.K, a.N, dp_tiles, per, thin, cl,
                             st->split_ws, st->split_counters, a.m_dev, ep) == cudaSuccess;
 }
 
@@ -1090,7 +1215,8 @@ void tc_state_force(void* s, int bn, int stream_k) {
   TcState* st = static_cast<TcState*>(s);
   if (!st) return;
   st->force_bn = bn;
-  st->force_s = stream_k;
+  st->force_s = stream_k != 0;
+  st->thin_clusters = stream_k != 2;     // 2: cut tiles always go through the partial-tile workspace
 }
 
 void tc_state_reset(void* s, cudaStream_t stream) {

@@ -149,6 +149,7 @@ void* tc_state_create(int n_sm);
 void tc_state_destroy(void* s);
 // debugging aid: force the tile configuration of the following launches (bn 64 / 128 / 256 single CTAs, 384 = CTA pairs
 // with 256 x 128 tiles, 512 = CTA pairs with 256 x 256 tiles; 0 = back to the cost model) and the decomposition
+// (0 whole tiles, 1 tiles cut over K, 2 the same without the cluster hand-over of thin problems)
 void tc_state_force(void* s, int bn, int stream_k);
 // zero the arrival counters of cut tiles (after a launch that ended with an error status)
 void tc_state_reset(void* s, cudaStream_t st);

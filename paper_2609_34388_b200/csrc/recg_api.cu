@@ -918,7 +918,8 @@ recg_status recg_debug_gemm_config(recg_ctx* ctx, int32_t tile, int32_t stream_k
   if (!ctx) return RECG_ERR_INVALID_ARG;
   if (tile != 0 && tile != 64 && tile != 128 && tile != 256 && tile != 384 && tile != 512)
     return fail(ctx, RECG_ERR_INVALID_ARG, "recg_debug_gemm_config: tile must be 0, 64, 128, 256, 384 or 512");
-  tc_state_force(ctx->tc_state, tile, stream_k != 0);
+  if (stream_k < 0 || stream_k > 2) return fail(ctx, RECG_ERR_INVALID_ARG, "recg_debug_gemm_config: stream_k must be 0, 1 or 2");
+  tc_state_force(ctx->tc_state, tile, stream_k);
   return RECG_OK;
 }
 

@@ -317,7 +317,7 @@ def test_linear_forced_decompositions(force):
     shape = synth.tiny_shape()
     ctx = ops_ctx(shape, 1, 8, 1)
     tile, sk = (int(t) for t in force.split(","))
-    ctx.recg_debug_gemm_config(tile, bool(sk))
+    ctx.recg_debug_gemm_config(tile, sk)
     for (M, N, K) in [(300, 512, 1024), (130, 4096, 4096), (470, 1024, 14336), (600, 6144, 1024), (257, 28672, 512)]:
         g = torch.Generator().manual_seed(M * 7 + N)
         x = torch.randn((M, K), generator=g).to(torch.bfloat16)
@@ -378,6 +378,46 @@ def test_linear_at_the_row_counts_the_bench_times(name):
             assert err < 1e-4, (name, M, tile, sk, err)
             assert torch.equal(outs[0][:M], outs[1][:M]), f"not deterministic: {(name, M, tile, sk)}"
             del outs, buf
+    ctx.recg_free()
+
+
+@pytest.mark.parametrize("name", ["qkv", "o", "down"])
+def test_linear_thin_rows_hand_over_inside_clusters(name):
+    """Problems of at most 32 rows whose tiles are cut over K: the CTAs that share a tile form a cluster and hand their
+    partial tiles to the cluster's leader through distributed shared memory.  The 8B-class shapes at 1, 7 and 32 rows,
+    with the cost model's choice and with forced tile widths (which give clusters of 2 to 4), against a float64 product
+    of the same bf16 values; the same launches with the hand-over through the partial-tile workspace (stream_k = 2) must
+    agree with it as closely; reruns give the same bits; rows behind the last one stay untouched."""
+    N, K = LLAMA8B_PROJECTIONS[name]
+    shape = synth.tiny_shape()
+    ctx = ops_ctx(shape, 1, 8, 1)
+    g = torch.Generator(device="cuda").manual_seed(N + K + 1)
+    w = (torch.randn((N, K), generator=g, device="cuda") * 0.05).to(torch.bfloat16)
+    w64 = f64(w)
+    for M in (1, 7, 32):
+        x = torch.randn((M, K), generator=g, device="cuda").to(torch.bfloat16)
+        ref = f64(x) @ w64.T
+        scale = np.max(np.abs(ref))
+        got = {}
+        for tile, sk in [(0, 1), (0, 2), (64, 1), (64, 2), (128, 1), (128, 2), (256, 1)]:
+            ctx.recg_debug_gemm_config(tile, sk)
+            outs = []
+            for rep in range(2):
+                buf = torch.full((M + 2, N), float("nan"), dtype=torch.float32, device="cuda")
+                ctx._check(binding.lib().recg_linear(ctx.h, x.data_ptr(), w.data_ptr(), buf.data_ptr(), M, N, K,
+                                                     binding.DTYPE_F32))
+                ctx.recg_sync()
+                outs.append(buf)
+            assert not torch.isnan(outs[0][:M]).any(), f"unwritten output: {(name, M, tile, sk)}"
+            assert torch.isnan(outs[0][M:]).all(), f"stored beyond the last row: {(name, M, tile, sk)}"
+            err = np.max(np.abs(f64(outs[0][:M]) - ref)) / scale
+            assert err < 1e-4, (name, M, tile, sk, err)
+            assert torch.equal(outs[0][:M], outs[1][:M]), f"not deterministic: {(name, M, tile, sk)}"
+            got[(tile, sk)] = outs[0][:M].clone()
+        # same tiles, other hand-over: the K ranges of the parts differ, so the sums differ in rounding only
+        for tile in (0, 64, 128):
+            d = float((got[(tile, 1)] - got[(tile, 2)]).abs().max()) / scale
+            assert d < 1e-5, (name, M, tile, d)
     ctx.recg_free()
 
 
