@@ -469,7 +469,9 @@ def bench_small_step(binding, peaks, args, n_layers=2, n_req=16):
 
 
 def bench_gemm_shapes(binding, peaks):
-    """The five projection shapes of one 8B-class layer (+ LM head) as standalone y = x w^T calls (plain epilogue)."""
+    """The five projection shapes of one 8B-class layer (+ LM head) as standalone y = x w^T calls (plain epilogue).
+    Copies of the weight matrix are rotated (at least 300 MB in total, more than L2 holds) so that every call streams
+    its weights from HBM like the calls inside a step do."""
     shape = synth.tiny_shape()
     shape.n_layers = 1
     ctx = binding.Context(binding.make_config(shape, 1, 8, 1))
@@ -480,24 +482,29 @@ def bench_gemm_shapes(binding, peaks):
             g = torch.Generator(device="cuda")
             g.manual_seed(M + N)
             x = torch.randn((M, K), generator=g, device="cuda").to(torch.bfloat16)
-            w = (torch.randn((N, K), generator=g, device="cuda") * 0.02).to(torch.bfloat16)
+            n_copies = max(1, int(np.ceil(300e6 / (N * K * 2))))
+            ws = [(torch.randn((N, K), generator=g, device="cuda") * 0.02).to(torch.bfloat16)]
+            ws += [ws[0].clone() for _ in range(n_copies - 1)]
             y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
-            call = lambda: binding.lib().recg_linear(ctx.h, x.data_ptr(), w.data_ptr(), y.data_ptr(), M, N, K, 0)
-            for _ in range(3):
-                call()
+            calls = 12 if n_copies == 1 else n_copies * max(1, 12 // n_copies)
+
+            def run(n):
+                for i in range(n):
+                    binding.lib().recg_linear(ctx.h, x.data_ptr(), ws[i % n_copies].data_ptr(), y.data_ptr(), M, N, K, 0)
+
+            run(max(3, n_copies))
             torch.cuda.synchronize()
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record()
-            for _ in range(10):
-                call()
+            run(calls)
             e1.record()
             torch.cuda.synchronize()
-            us = e0.elapsed_time(e1) / 10 * 1e3
+            us = e0.elapsed_time(e1) / calls * 1e3
             tf = 2.0 * M * N * K / (us * 1e-6) / 1e12
             gbs = N * K * 2 / (us * 1e-6) / 1e9
-            out.append({"M": M, "name": name, "N": N, "K": K, "us": round(us, 1), "tflops": round(tf, 1),
-                        **tensor_fracs(tf, peaks), "weight_gbs": round(gbs, 1), **hbm_fracs(gbs, peaks)})
-            del x, w, y
+            out.append({"M": M, "name": name, "N": N, "K": K, "us": round(us, 1), "weight_copies_rotated": n_copies,
+                        "tflops": round(tf, 1), **tensor_fracs(tf, peaks), "weight_gbs": round(gbs, 1), **hbm_fracs(gbs, peaks)})
+            del x, ws, y
     ctx.recg_free()
     return out
 

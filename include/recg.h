@@ -264,7 +264,7 @@ recg_status recg_debug_buffer(recg_ctx *ctx, int32_t which, const void **ptr, in
  *   instead of the cost model's choice: tile = 64, 128 or 256 (single CTAs, 128-row tiles of that width), 384 (CTA
  *   pairs, 256 x 128 tiles), 512 (CTA pairs, 256 x 256 tiles), 0 = back to the cost model; stream_k = 1 cuts the
  *   K range of the tiles evenly over the SMs, stream_k = 2 does the same and also (with any tile value, 0 included)
- *   keeps problems of at most 32 rows from handing their partial tiles over inside thread-block clusters: they go
+ *   keeps problems of at most 128 rows from handing their partial tiles over inside thread-block clusters: they go
  *   through the partial-tile workspace like everything else; stream_k = 0: whole tiles.  A configuration that does not
  *   fit a shape is ignored for that launch.
  * recg_debug_wait_timeout(): enqueue a one-thread kernel that waits on a barrier nobody arrives on, bounded by

@@ -11,8 +11,8 @@
 //            TMA box stores (add-reductions for the residual stream) from a small swizzled staging area.
 // Tiles are walked m-fastest so that CTAs running together share the same weight tile through L2.
 // Tiles can be cut over K (stream-K): partial tiles are parked in a workspace and reduced by the last part to arrive; for
-// problems of at most 32 rows the parts of a tile form a thread-block cluster instead and hand their partial tiles to the
-// cluster's leader through distributed shared memory.
+// problems of one row tile (at most 128 rows) the parts of a tile form a thread-block cluster instead and hand their
+// partial tiles to the cluster's leader through distributed shared memory.
 // Every wait is bounded; on a timeout the kernel records a status code, drains and frees TMEM.
 #include <cuda.h>
 
@@ -542,15 +542,19 @@ __global__ void __launch_bounds__(kTcThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
                const __grid_constant__ CUtensorMap map_out, const __grid_constant__ CUtensorMap map_xout, int M_cap, int n_tiles_n,
                int K, int up_row_offset, int dp_tiles_in, long long per_in, int thin, int cl_parts, float* split_ws,
-               int* split_counters, const int* __restrict__ m_dev, EpiParams ep_in) {
+               int* split_counters, const int* __restrict__ m_dev, int m_dev_wait, EpiParams ep_in) {
   // Device-resident rounds: the row count comes from device memory; the tensor maps cover the capacity M_cap, and rows
   // between the count and the capacity hold stale data and are computed but never used.  The count is written by the
   // first kernel of the step, and the small kernels between it and the first projection signal their dependents before
-  // they wait themselves, so this kernel can be running before that one has finished: it has to wait for its
-  // predecessors before it reads the count (and gives up the early weight requests in this mode).
-  if (m_dev) griddep_wait();
+  // they wait themselves, so the FIRST projection of a step can be running before that one has finished: it has to wait
+  // for its predecessors before it reads the count (m_dev_wait; it gives up the early weight requests).  The first
+  // projection signals its own dependents only after that wait, so for every kernel behind it the count is settled.
+  if (m_dev && m_dev_wait) griddep_wait();
   const int M = m_dev ? *reinterpret_cast<const volatile int*>(m_dev) : M_cap;
-  if (M <= 0) return;          // an empty round (the same for every thread of the grid): nothing to do, nothing was set up yet
+  if (M <= 0) {                // an empty round (the same for every thread of the grid): nothing to do, nothing was set up yet
+    griddep_wait();            // (this grid must not count as complete before the ones it follows are)
+    return;
+  }
   EpiParams ep = ep_in;
   ep.M = M;
   using Cfg = TcCfg<BN, PAIR, NORM>;
@@ -561,14 +565,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
   const int n_units = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  // Thin problems whose tiles are cut over K can run as CLUSTERS of cl CTAs per tile (cl_parts > 1; at most 32 rows, one
-  // row tile, single CTAs only): rank r computes k-blocks [r KB / cl, (r + 1) KB / cl) and hands its 32 x BN partial to
-  // the cluster's leader (rank 0) through distributed shared memory, into a reserve at the top of the leader's ring
-  // budget; the leader adds the parts in rank order and runs the epilogue.  No trip through global memory, no counter.
-  const int cl = (!PAIR && thin && cl_parts > 1) ? cl_parts : 0;
+  // Problems of one row tile (at most 128 rows) whose tiles are cut over K can run as CLUSTERS of cl CTAs per tile
+  // (cl_parts > 1; single CTAs only): rank r computes k-blocks [r KB / cl, (r + 1) KB / cl) and hands its partial tile
+  // (the rows in use, rounded up to 32) to the cluster's leader (rank 0) through distributed shared memory, into a
+  // reserve at the top of the leader's ring budget; the leader adds the parts in rank order and runs the epilogue.  No
+  // trip through global memory, no counter.
+  const int cl = (!PAIR && cl_parts > 1) ? cl_parts : 0;
   const uint32_t crank = cl ? cluster_ctarank() : 0u;
-  constexpr int kClPartBytes = 32 * BN * 4;
-  const int cl_reserve = cl ? (cl - 1) * kClPartBytes : 0;
+  const int cl_rows = ((M < BM ? M : BM) + 31) & ~31;            // rows of a handed-over part
+  const int cl_part_bytes = cl_rows * BN * 4;
+  const int cl_reserve = cl ? (cl - 1) * cl_part_bytes : 0;
   const int a_bytes = thin ? Cfg::kThinABytes : Cfg::kABytes;
   const int stage_bytes = a_bytes + Cfg::kBBytes;
   const int cl_stages = (Cfg::kBudget - cl_reserve) / stage_bytes;
@@ -661,7 +667,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
       mbar_init(&tfull_bar[a], 1);
       mbar_init(&tempty_bar[a], PAIR ? 8 : 4);
     }
-    mbar_init(red_bar, cl ? cl - 1 : 1);      // (cluster leader: one arrival per peer)
+    mbar_init(red_bar, cl ? (cl - 1) * (cl_rows / 32) : 1);      // (cluster leader: one arrival per peer and 32 rows)
     for (int i = 0; i < 8; ++i) mbar_init(&h_bar[i], 1);
     fence_barrier_init();
     prefetch_tmap(&map_x);
@@ -862,17 +868,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
         row_epilogue<BN, NORM>(ep, TmemLoader{tacc}, m, n0, stg, &map_out, &map_xout, rstd, tn, ns, prepared);
         release_acc();
       } else if (cl) {
-        uint8_t* reserve = smem + Cfg::kBudget - cl_reserve;       // the leader's: cl - 1 parts of [BN/4][32] float4
+        uint8_t* reserve = smem + Cfg::kBudget - cl_reserve;       // the leader's: cl - 1 parts of [BN/4][cl_rows] float4
         if (crank != 0) {
-          if (quad == 0) {           // the warp that holds rows 0..31 of the accumulator
-            const uint32_t dst = mapa_rank(smem_u32(reserve + (crank - 1) * kClPartBytes), 0) + lane * 16;
+          if (quad * 32 < cl_rows) {           // the warps that hold rows in use
+            const uint32_t dst = mapa_rank(smem_u32(reserve + (crank - 1) * cl_part_bytes), 0) + row_in_tile * 16;
+            const uint32_t col_stride = (uint32_t)cl_rows * 16u;
 #pragma unroll 1
             for (int c = 0; c < BN / 32; ++c) {
               float v[32];
               tmem_ld32(tacc + c * 32, v);
 #pragma unroll
               for (int i = 0; i < 8; ++i)
-                st_cluster_f4(dst + (uint32_t)(c * 8 + i) * 512u, make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]));
+                st_cluster_f4(dst + (uint32_t)(c * 8 + i) * col_stride, make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]));
             }
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(mapa_rank(smem_u32(red_bar), 0));   // release: the warp's stores are visible
@@ -896,7 +903,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
               s_abort = 1;
             }
           }
-          RingLoader ld{tacc, reinterpret_cast<const float4*>(reserve) + lane, BN, 0, n_splits, 32};
+          RingLoader ld{tacc, reinterpret_cast<const float4*>(reserve) + row_in_tile, BN, 0, n_splits, cl_rows};
           row_epilogue<BN, NORM>(ep, ld, m, n0, stg, &map_out, &map_xout, rstd, tn, ns, false);
           release_acc();
         }
@@ -1013,7 +1020,7 @@ struct TcState {
   size_t evictions = 0;
   int last_tiles_n = 0;       // column tiles of the last launch
   bool configured[10] = {false, false, false, false, false, false, false, false, false, false};
-  bool thin_clusters = true;  // thin problems with cut tiles run as clusters that reduce through distributed shared memory
+  bool thin_clusters = true;  // problems of one row tile with cut tiles run as clusters that reduce through distributed shared memory
   int max_clusters[10][5];    // cached occupancy answers per kernel and cluster size (-1: not asked yet)
   TcState() {
     for (auto& row : max_clusters)
@@ -1077,14 +1084,19 @@ bool launch_bn(TcState* st, int idx, const GemmArgs& a, const EpiParams& ep, boo
 template <int BN, bool PAIR, bool NORM>
 int max_active_clusters(TcState* st, int idx, int n_tiles, int parts);
 
-// Thin problems (at most 32 rows) whose tiles would be cut over K: how many CTAs form the cluster that shares a tile
-// (0: no clusters).  The whole grid has to be resident at once, which the occupancy query decides (cached).
+// Problems of one row tile (at most 128 rows) whose tiles would be cut over K: how many CTAs form the cluster that shares
+// a tile (0: no clusters).  The whole grid has to be resident at once, which the occupancy query decides (cached).
 template <int BN, bool PAIR, bool NORM>
-int cluster_parts(TcState* st, int idx, int n_tiles, int KB) {
+int cluster_parts(TcState* st, int idx, int n_tiles, int KB, int rows) {
   if (PAIR || !st->thin_clusters || n_tiles <= 0) return 0;
+  using Cfg = TcCfg<BN, PAIR, NORM>;
   int parts = st->n_sm / n_tiles;
   if (parts > 4) parts = 4;
   if (parts > KB) parts = KB;
+  // the leader keeps the peers' parts at the top of its ring budget: at least four stages must remain
+  const int part_bytes = ((rows + 31) & ~31) * BN * 4;
+  const int stage_bytes = (rows <= 32 ? Cfg::kThinABytes : Cfg::kABytes) + Cfg::kBBytes;
+  while (parts >= 2 && (Cfg::kBudget - (parts - 1) * part_bytes) / stage_bytes < 4) --parts;
   for (; parts >= 2; --parts) {
     if (max_active_clusters<BN, PAIR, NORM>(st, idx, n_tiles, parts) >= n_tiles) return parts;
   }
@@ -1149,7 +1161,7 @@ bool launch_bn_t(TcState* st, int idx, const GemmArgs& a, const EpiParams& ep, b
   int units = n_tiles < n_units ? n_tiles : n_units;
   int dp_tiles = n_tiles;       // whole tiles, strided
   long long per = 1;
-  const int cl = (thin && stream_k && mt == 1) ? cluster_parts<BN, PAIR, NORM>(st, idx, n_tiles, (int)KB) : 0;
+  const int cl = (stream_k && mt == 1 && a.M <= BM) ? cluster_parts<BN, PAIR, NORM>(st, idx, n_tiles, (int)KB, a.M) : 0;
   if (cl) {
     units = n_tiles * cl;       // one cluster per tile; the kernel derives each member's k-blocks from its rank
   } else if (a.m_dev) {
@@ -1184,7 +1196,7 @@ bool launch_bn_t(TcState* st, int idx, const GemmArgs& a, const EpiParams& ep, b
   cfg.attrs = attr;
   cfg.numAttrs = n_attr;
   return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<BN, PAIR, NORM>, mx, mw, mo, mxo, a.M, n_tiles_n, a.K, a.N, dp_tiles, per, thin, cl,
-                            st->split_ws, st->split_counters, a.m_dev, ep) == cudaSuccess;
+                            st->split_ws, st->split_counters, a.m_dev, a.m_dev_settled ? 0 : 1, ep) == cudaSuccess;
 }
 
 }  // namespace

@@ -131,6 +131,7 @@ struct GemmArgs {
   // tile configuration is chosen for (0: M)
   const int* m_dev;
   int m_hint;
+  bool m_dev_settled;   // a projection of this stream has already run since the count was written (no need to wait before reading it)
   // folded RMSNorm (see EpiParams in epilogue.cuh); all null / 0 when unused
   const float* ss_in;   // consumer: partial sums of squares of the rows of x's source, [ss_slots][ss_stride]
   int ss_slots, ss_stride;

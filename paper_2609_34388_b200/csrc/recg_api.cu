@@ -542,10 +542,12 @@ static recg_status run_forward(recg_ctx* ctx, void* kv_pool, int64_t kv_pool_pag
   CU(cudaGetLastError());
   ctx->mark(0, 3);
   const int qdim = d.n_q * d.head_dim;
+  int n_proj = 0;                        // projections enqueued so far in this step
   auto normed = [&](GemmArgs& g) {       // g reads the normalised residual stream
     g.x = ctx->x;
     g.K = d.hidden;
     g.m_dev = bl.dyn;
+    g.m_dev_settled = n_proj++ > 0;
     g.m_hint = m_hint;
     if (fold) { g.ss_in = ctx->ss; g.ss_slots = slots; g.ss_stride = Tm; g.norm_eps = d.rms_eps; }
   };
@@ -553,6 +555,7 @@ static recg_status run_forward(recg_ctx* ctx, void* kv_pool, int64_t kv_pool_pag
     g.out = ctx->h;
     g.N = d.hidden;
     g.m_dev = bl.dyn;
+    g.m_dev_settled = n_proj++ > 0;
     g.m_hint = m_hint;
     g.epi = fold ? EPI_RESIDUAL_NORM : EPI_RESIDUAL;
     if (fold) { g.x_out = ctx->x; g.gain = next_gain; g.ss_out = ctx->ss; g.ss_stride = Tm; }

@@ -383,8 +383,9 @@ def test_linear_at_the_row_counts_the_bench_times(name):
 
 @pytest.mark.parametrize("name", ["qkv", "o", "down"])
 def test_linear_thin_rows_hand_over_inside_clusters(name):
-    """Problems of at most 32 rows whose tiles are cut over K: the CTAs that share a tile form a cluster and hand their
-    partial tiles to the cluster's leader through distributed shared memory.  The 8B-class shapes at 1, 7 and 32 rows,
+    """Problems of one row tile (at most 128 rows) whose tiles are cut over K: the CTAs that share a tile form a cluster and
+    hand their partial tiles to the cluster's leader through distributed shared memory.  The 8B-class shapes at 1, 7, 32,
+    33, 66, 100 and 128 rows,
     with the cost model's choice and with forced tile widths (which give clusters of 2 to 4), against a float64 product
     of the same bf16 values; the same launches with the hand-over through the partial-tile workspace (stream_k = 2) must
     agree with it as closely; reruns give the same bits; rows behind the last one stay untouched."""
@@ -394,7 +395,7 @@ def test_linear_thin_rows_hand_over_inside_clusters(name):
     g = torch.Generator(device="cuda").manual_seed(N + K + 1)
     w = (torch.randn((N, K), generator=g, device="cuda") * 0.05).to(torch.bfloat16)
     w64 = f64(w)
-    for M in (1, 7, 32):
+    for M in (1, 7, 32, 33, 66, 100, 128):
         x = torch.randn((M, K), generator=g, device="cuda").to(torch.bfloat16)
         ref = f64(x) @ w64.T
         scale = np.max(np.abs(ref))
