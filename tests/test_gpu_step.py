@@ -269,25 +269,31 @@ def test_llama8b_shape_one_layer_round(flags):
     report_flat_flag(stats)
 
 
-@pytest.mark.parametrize("clusters", [True, False])
-def test_llama8b_shape_one_layer_round_at_concurrency_1(clusters):
-    """One 8B-shaped layer + LM head for a single request of 16 + 16 rows: the thin projections (rotary + K/V append,
-    residual update) hand their cut tiles over inside clusters, or through the partial-tile workspace."""
+@pytest.mark.parametrize("clusters,specs", [(True, [(700, 16, 16)]), (False, [(700, 16, 16)]), (True, [(300, 1, 16)]),
+                                            (True, [(513, 16, 32)]), (True, [(90, 32, 32)]), (True, [(200, 32, 32), (64, 32, 32)]),
+                                            (True, [(40, 3, 8), (130, 1, 4), (77, 30, 32)])])
+def test_llama8b_shape_one_layer_round_at_low_concurrency(clusters, specs):
+    """One 8B-shaped layer + LM head for one to three requests with 16 to 128 rows in all (one row tile): the projections
+    whose tiles are cut over K (rotary + K/V append, residual update) hand their partial tiles over inside clusters, or
+    (clusters = False) through the partial-tile workspace."""
     shape = synth.llama8b_shape(1)
     shape.vocab = 16384
     W = synth.model_weights(shape, seed=0, dtype=torch.bfloat16)
     ocfg, W64 = oracle_cfg(shape), oracle_weights(W)
-    L, v, b = [700], [16], [16]
+    L, v, b = [s[0] for s in specs], [s[1] for s in specs], [s[2] for s in specs]
     desc = synth.fixed_descriptor(L, v, b, seed=4)
-    ctx = binding.Context(binding.make_config(shape, 1, 32, desc.page_table.shape[1]), to_dev(W))
+    assert desc.n_tokens <= 128
+    ctx = binding.Context(binding.make_config(shape, len(specs), desc.n_tokens, desc.page_table.shape[1]), to_dev(W))
     if not clusters:
         ctx.recg_debug_gemm_config(0, 2)
     pool = binding.alloc_kv_pool(ctx, desc.n_pages, fill=None)
     pool.fill_(float("nan"))
-    K, V = synth.kv_values(L[0], shape.n_kv_heads, shape.head_dim, seed=300)
-    ctx.recg_kv_write(pool, desc.n_pages, 0, desc.page_table[0], 0, K.cuda(), V.cuda())
-    y = synth.token_ids(v[0], shape.vocab, seed=400).tolist()
-    reqs = [{"kv": [(f64(K), f64(V))], "y": y, "L": L[0], "v": v[0], "b": b[0], "m": None}]
+    reqs = []
+    for i in range(len(specs)):
+        K, V = synth.kv_values(L[i], shape.n_kv_heads, shape.head_dim, seed=300 + i)
+        ctx.recg_kv_write(pool, desc.n_pages, 0, desc.page_table[i], 0, K.cuda(), V.cuda())
+        y = synth.token_ids(v[i], shape.vocab, seed=400 + i).tolist()
+        reqs.append({"kv": [(f64(K), f64(V))], "y": y, "L": L[i], "v": v[i], "b": b[i], "m": None})
     stats, _ = check_round(ctx, shape, ocfg, W64, reqs, desc, pool, margin_flag=MARGIN_LARGE_SHAPES)
     ctx.recg_free()
     report_flat_flag(stats)
