@@ -154,17 +154,20 @@ def test_device_round_that_breaks_a_capacity_is_refused_on_the_device():
     ctx.recg_free()
 
 
-def test_device_round_on_8b_shaped_layers_equals_the_host_round():
+@pytest.mark.parametrize("n_req,capacity,blocks", [(12, 512, [4, 8, 16, 32]), (3, 128, [4, 8, 16]), (1, 64, [16]), (1, 32, [8])])
+def test_device_round_on_8b_shaped_layers_equals_the_host_round(n_req, capacity, blocks):
     """The same ragged batch through two 8B-shaped layers (tcgen05 projections and attention) once with host descriptor
-    arrays and once with device arrays (row count unknown to the host, launches sized for the capacity, whole tiles
-    only): logits agree within the batch-invariance tolerance, integers wherever the top-2 gap is not a near tie."""
+    arrays and once with device arrays (row count unknown to the host, launches sized for the capacity): logits agree
+    within the batch-invariance tolerance, integers wherever the top-2 gap is not a near tie.  Capacities of at most 128
+    rows take the projections whose cut tiles are handed over inside clusters, with the row count read on the device."""
     shape = synth.llama8b_shape(2)
     shape.vocab = 8192
     W = synth.model_weights(shape, seed=0, dtype=torch.bfloat16)
     Wd = {k: ([t.cuda() for t in v] if isinstance(v, list) else v.cuda()) for k, v in W.items()}
-    desc = synth.batch_descriptor(12, [4, 8, 16, 32], None, 100, 2000, seed=31)
+    desc = synth.batch_descriptor(n_req, blocks, None, 100, 2000, seed=31)
     T = desc.n_tokens
-    ctx = binding.Context(binding.make_config(shape, 12, 512, desc.page_table.shape[1]), Wd)     # capacity above the row count
+    assert T <= capacity
+    ctx = binding.Context(binding.make_config(shape, n_req, capacity, desc.page_table.shape[1]), Wd)     # capacity above the row count
     pool = binding.alloc_kv_pool(ctx, desc.n_pages, fill="normal")
     ys = synth.token_ids(int(desc.verify_len.sum()), shape.vocab, seed=1)
     host = binding.Batch(desc.ctx_len, desc.verify_len, desc.block_size, ys, desc.page_table, pool, desc.n_pages)
@@ -175,7 +178,7 @@ def test_device_round_on_8b_shaped_layers_equals_the_host_round():
     pt = np.where(desc.page_table >= 0, desc.page_table, 0)
     db = binding.DeviceBatch(desc.ctx_len, desc.verify_len, desc.block_size, per_req, 32, pt, pool, desc.n_pages, rows_hint=T)
     lg = ctx.recg_step_device(db)
-    assert lg.n_rows == 512
+    assert lg.n_rows == capacity
     got = binding.device_view(lg.data, (lg.n_rows, lg.vocab), torch.float32)[:T].clone()
     out = binding.VerifyOut(desc.n_req, T, int(desc.verify_len.sum()), host=False)
     ctx.recg_verify(None, None, host=False, out=out)
