@@ -439,6 +439,40 @@ def test_bucketed_schedule_gives_the_same_results_as_the_mixed_batch():
     ctx.recg_free()
 
 
+def test_low_concurrency_step_is_deterministic():
+    """One to three requests (17 to 128 rows: the projections hand their cut tiles over inside clusters, the parts are
+    added in rank order): the same batch gives bit-identical logits and results every time, with other batches in between."""
+    shape = synth.llama8b_shape(2)
+    shape.vocab = 8192
+    W = synth.model_weights(shape, seed=0, dtype=torch.bfloat16)
+    specs = [([900], [16], [16]), ([300], [1], [16]), ([64, 700], [32, 32], [32, 32]), ([40, 130, 77], [3, 1, 30], [8, 4, 32])]
+    descs = [synth.fixed_descriptor(L, v, b, seed=40 + i) for i, (L, v, b) in enumerate(specs)]
+    n_pages = sum(d.n_pages for d in descs)
+    stride = max(d.page_table.shape[1] for d in descs)
+    ctx = binding.Context(binding.make_config(shape, 3, 128, stride), to_dev(W))
+    pool = binding.alloc_kv_pool(ctx, n_pages, fill="normal")
+    batches, first_page = [], 0
+    for i, d in enumerate(descs):
+        ys = synth.token_ids(int(d.verify_len.sum()), shape.vocab, seed=60 + i)
+        pt = np.where(d.page_table >= 0, d.page_table + first_page, -1).astype(np.int32)
+        first_page += d.n_pages
+        batches.append(binding.Batch(d.ctx_len, d.verify_len, d.block_size, ys, pt, pool, n_pages))
+    first = {}
+    for rnd in range(24):
+        j = (rnd * 3 + rnd // 5) % len(batches)
+        lg = ctx.logits_tensor(ctx.recg_step(batches[j]))
+        g = ctx.recg_verify(batches[j])
+        if j not in first:
+            first[j] = (lg, {k: v.copy() for k, v in g.items()})
+        else:
+            assert torch.equal(lg, first[j][0]), f"logits of batch {j} changed in iteration {rnd}"
+            for k, v in g.items():
+                assert np.array_equal(v, first[j][1][k], equal_nan=True), (k, j, rnd)
+    assert len(first) == len(batches)
+    ctx.recg_sync()
+    ctx.recg_free()
+
+
 def test_step_is_deterministic_and_survives_many_rounds():
     """The same batch gives bit-identical logits and results every time (partial tiles are reduced in a fixed order, the
     residual stream receives one addend per element and launch), also with other batches in between; and a longer run
